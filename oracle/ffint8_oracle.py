@@ -1,0 +1,453 @@
+"""CPU oracle for the FF-INT8 per-layer train step.  TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plain restatement of what the CUDA library computes.  Only the
+tests, the smoke check and the benchmark's CPU-baseline leg may import it; the product
+path never does, and this module imports nothing from the CUDA package.
+
+Every function follows one passage of the FF-INT8 paper (cited per function).  Where the
+paper leaves arithmetic unspecified, the function implements the written numerics contract
+of this project (one correctly rounded IEEE operation at a time, in a stated order, no
+fused multiply-add), so that the INT8 tensors it produces have exactly one correct bit
+pattern.  numpy float32/float64 ufuncs are individually correctly rounded and never
+contracted, which is what makes numpy a suitable language for that contract.
+
+Notation (paper, Sec. IV-B and Algorithm 1): A / X = layer input, W = weights, Y = neuron
+activity, G = goodness = ||y||^2, theta = threshold, g^Y = dH = dL/dY, g^W = dW.
+Rows 0..B-1 of every batch tensor are the positive set, rows B..2B-1 the negative set.
+
+Pins (tests/test_oracle_*.py): hand-computed tiny layers, closed forms of Eq. 1-2,
+brute-force loops, finite differences of the unquantised loss, quantiser error bounds,
+library cross-checks (float64 conv2d).  Parity unpinned: the look-ahead *gradient* (Eq. 4)
+is a reading of the paper (scalar-coefficient look-ahead); only its closed form, its
+lambda=0 and single-layer reductions are pinned.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+F32 = np.float32
+F64 = np.float64
+
+ROUND_NEAREST = 0
+ROUND_STOCHASTIC = 1
+
+ROLE_X = 0   # hash stream of the layer-input quantiser
+ROLE_W = 1   # hash stream of the weight quantiser
+ROLE_DH = 2  # hash stream of the output-gradient quantiser
+
+KIND_LINEAR = 0
+KIND_CONV3X3 = 1
+
+_M64 = (1 << 64) - 1
+
+
+# --------------------------------------------------------------------------------------
+# Layer description
+# --------------------------------------------------------------------------------------
+@dataclass
+class LayerSpec:
+    """One FF layer.  linear: X [2B,K] -> Y [2B,N].  conv3x3 (stride 1, zero pad 1, NHWC):
+    X [2B,H,W,Cin] -> Y [2B,H,W,N] with K = 9*Cin and weights [N,3,3,Cin] flattened to [N,K]."""
+    kind: int
+    K: int
+    N: int
+    theta: float
+    lr: float
+    tau: float            # length-normalisation target norm of the NEXT layer's input
+    eps: float = 1e-8
+    H: int = 1
+    Wd: int = 1
+    Cin: int = 0
+    round_x: int = ROUND_STOCHASTIC
+    round_w: int = ROUND_NEAREST
+    round_dh: int = ROUND_STOCHASTIC
+    seed: int = 0
+    index: int = 0        # position of the layer in the network (feeds the rounding hash)
+
+    @property
+    def rows_per_sample(self) -> int:
+        return self.H * self.Wd if self.kind == KIND_CONV3X3 else 1
+
+
+# --------------------------------------------------------------------------------------
+# Symmetric uniform quantiser with nearest / stochastic rounding  (Sec. IV; Sec. IV-B)
+# --------------------------------------------------------------------------------------
+def absmax(x: np.ndarray) -> np.float32:
+    """Per-tensor max |x| (the SUQ range, Sec. IV).  Exact: max involves no rounding."""
+    x = np.asarray(x, dtype=F32)
+    if x.size == 0:
+        return F32(0.0)
+    if not np.all(np.isfinite(x)):
+        raise FloatingPointError("non-finite value in a tensor to be quantised")
+    return F32(np.max(np.abs(x)))
+
+
+def scale_pair(a: np.float32):
+    """SUQ scale s = a/127 and its reciprocal factor inv = 127/a, each ONE float32 division.
+    A zero tensor (a == 0) quantises to all zeros: s = 1, inv = 0."""
+    a = F32(a)
+    if a == F32(0.0):
+        return F32(1.0), F32(0.0)
+    return F32(a / F32(127.0)), F32(F32(127.0) / a)
+
+
+def _splitmix64(x: int) -> int:
+    """SplitMix64 output function (Steele/Lea/Flood; public-domain reference by Vigna)."""
+    x = (x + 0x9E3779B97F4A7C15) & _M64
+    z = x
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return z ^ (z >> 31)
+
+
+def rounding_key(seed: int, role: int, layer: int, step: int):
+    """Two 32-bit keys for one (seed, tensor role, layer, step) quantiser call."""
+    s0 = _splitmix64(seed & _M64)
+    s1 = _splitmix64(s0 ^ ((role & 0xFF) | ((layer & 0xFFFFFF) << 8)))
+    s2 = _splitmix64(s1 ^ (step & _M64))
+    return s2 & 0xFFFFFFFF, (s2 >> 32) & 0xFFFFFFFF
+
+
+def rounding_uniform(idx: np.ndarray, k0: int, k1: int) -> np.ndarray:
+    """u in [0,1) with 24 random bits for each linear element index (counter-based, so the
+    value does not depend on how the tensor is tiled or which thread handles the element)."""
+    h = idx.astype(np.uint32) ^ np.uint32(k0)
+    h = h * np.uint32(0x9E3779B1)
+    h = h ^ (h >> np.uint32(15))
+    h = (h + np.uint32(k1)) * np.uint32(0x85EBCA6B)
+    h = h ^ (h >> np.uint32(13))
+    h = h * np.uint32(0xC2B2AE35)
+    h = h ^ (h >> np.uint32(16))
+    return (h >> np.uint32(8)).astype(F32) * F32(2.0 ** -24)
+
+
+def quantize(x: np.ndarray, a: np.float32, mode: int, key=None, idx0: int = 0,
+             u: Optional[np.ndarray] = None) -> np.ndarray:
+    """SUQ to INT8 in [-127,127], zero point 0 (Sec. IV).  t = x*inv (one multiply), then
+    nearest-even (rint) or stochastic rounding floor(t+u) (Sec. IV-B, Gupta et al.), then clip.
+    `idx0` is the linear index of x.flat[0] inside the whole tensor (for per-pass slices);
+    `u` overrides the hash (used by the hand-computed pins)."""
+    x = np.asarray(x, dtype=F32)
+    if x.size >= 1 << 32:
+        raise ValueError("tensor too large for 32-bit rounding counters")
+    _, inv = scale_pair(a)
+    t = x * inv
+    if mode == ROUND_NEAREST:
+        q = np.rint(t)
+    else:
+        if u is None:
+            idx = (np.arange(x.size, dtype=np.uint64) + np.uint64(idx0)).reshape(x.shape)
+            u = rounding_uniform(idx, key[0], key[1])
+        q = np.floor(t + np.asarray(u, dtype=F32))
+    return np.clip(q, -127.0, 127.0).astype(np.int8)
+
+
+def quantize_two_pass(x: np.ndarray, B: int, mode: int, key):
+    """Quantise the positive rows [0,B) and the negative rows [B,2B) with separate per-tensor
+    scales ('for each dataset (positive or negative)', Sec. IV-B).  Returns q, (a_pos, a_neg)."""
+    q = np.empty(x.shape, dtype=np.int8)
+    per_row = int(np.prod(x.shape[1:])) if x.ndim > 1 else 1
+    a = []
+    for p in range(2):
+        sl = slice(p * B, (p + 1) * B)
+        ap = absmax(x[sl])
+        q[sl] = quantize(x[sl], ap, mode, key, idx0=p * B * per_row)
+        a.append(ap)
+    return q, (a[0], a[1])
+
+
+# --------------------------------------------------------------------------------------
+# INT8 MAC with INT32 accumulation  (Sec. IV-B)
+# --------------------------------------------------------------------------------------
+def _check_i32(acc64: np.ndarray) -> np.ndarray:
+    if acc64.size and np.max(np.abs(acc64)) >= 2.0 ** 31:
+        raise OverflowError("INT32 accumulator range exceeded")
+    return acc64.astype(np.int32)
+
+
+def _matmul_exact(a_i8: np.ndarray, b_i8: np.ndarray) -> np.ndarray:
+    """a @ b for INT8 operands as an exact integer result.  The float64 library matmul is the
+    step: every product and partial sum is an integer below 2^53, so no rounding occurs."""
+    return a_i8.astype(F64) @ b_i8.astype(F64)
+
+
+def int8_gemm_nt(xq: np.ndarray, wq: np.ndarray, row_chunk: int = 4096) -> np.ndarray:
+    """acc[m,n] = sum_k xq[m,k]*wq[n,k], INT8 x INT8 -> INT32 (dense layer, Sec. IV-B)."""
+    M = xq.shape[0]
+    out = np.empty((M, wq.shape[0]), dtype=np.int32)
+    wt = wq.astype(F64).T
+    for m0 in range(0, M, row_chunk):
+        out[m0:m0 + row_chunk] = _check_i32(xq[m0:m0 + row_chunk].astype(F64) @ wt)
+    return out
+
+
+def int8_gemm_tn(dhq: np.ndarray, xq: np.ndarray) -> np.ndarray:
+    """accW[n,k] = sum_m dhq[m,n]*xq[m,k]  (g^W = g^Y^T A as an INT8 MAC, Sec. IV-B)."""
+    return _check_i32(_matmul_exact(dhq.T, xq))
+
+
+def _pad_hw(xq: np.ndarray) -> np.ndarray:
+    return np.pad(xq, ((0, 0), (1, 1), (1, 1), (0, 0)))
+
+
+def int8_conv3x3(xq: np.ndarray, wq: np.ndarray) -> np.ndarray:
+    """acc[b,h,w,co] = sum_{r,s,ci} xq[b,h+r-1,w+s-1,ci]*wq[co,r,s,ci], zero padding
+    ('dense or convolution layers', Sec. IV-B).  xq NHWC int8, wq [Cout,3,3,Cin] int8."""
+    Bn, H, Wd, Cin = xq.shape
+    Cout = wq.shape[0]
+    xp = _pad_hw(xq)
+    acc = np.zeros((Bn * H * Wd, Cout), dtype=F64)
+    for r in range(3):
+        for s in range(3):
+            win = xp[:, r:r + H, s:s + Wd, :].reshape(-1, Cin)
+            acc += _matmul_exact(win, wq[:, r, s, :].T)
+    return _check_i32(acc).reshape(Bn, H, Wd, Cout)
+
+
+def int8_conv3x3_wgrad(dhq: np.ndarray, xq: np.ndarray) -> np.ndarray:
+    """accW[co,r,s,ci] = sum_{b,h,w} dhq[b,h,w,co]*xq[b,h+r-1,w+s-1,ci] (weight gradient of the
+    convolution above; there is no input gradient in FF, Sec. IV-B)."""
+    Bn, H, Wd, Cin = xq.shape
+    Cout = dhq.shape[-1]
+    xp = _pad_hw(xq)
+    d2 = dhq.reshape(-1, Cout)
+    out = np.empty((Cout, 3, 3, Cin), dtype=np.int32)
+    for r in range(3):
+        for s in range(3):
+            win = xp[:, r:r + H, s:s + Wd, :].reshape(-1, Cin)
+            out[:, r, s, :] = _check_i32(_matmul_exact(d2.T, win))
+    return out
+
+
+# --------------------------------------------------------------------------------------
+# Epilogue: dequantise, ReLU, goodness, length normalisation  (Sec. III; Alg. 1 line 6)
+# --------------------------------------------------------------------------------------
+def dequant_relu(acc: np.ndarray, c_rows: np.ndarray) -> np.ndarray:
+    """y = max(0, float(acc) * c) with c = s_x*s_w of the row's pass; int->float conversion and
+    the multiply are each one rounding."""
+    accf = acc.astype(F32)
+    c = c_rows.reshape((-1,) + (1,) * (acc.ndim - 1)).astype(F32)
+    return np.maximum(F32(0.0), accf * c)
+
+
+def goodness(acc: np.ndarray, c_rows: np.ndarray):
+    """G = ||y||^2 per sample ('sum of squared neural activities', Sec. III; Alg. 1 line 6),
+    evaluated as the exact integer S = sum relu(acc)^2 scaled once: G = float(double(S)*c*c).
+    Also returns S and the per-sample max of relu(acc) (used for the absmax short-cuts)."""
+    n = acc.shape[0]
+    relu = np.maximum(acc.reshape(n, -1), 0).astype(np.uint64)
+    approx = (relu.astype(F64) ** 2).sum(axis=1)
+    if approx.size and approx.max() >= 2.0 ** 63:
+        raise OverflowError("goodness integer sum exceeds 64 bits")
+    S = (relu * relu).sum(axis=1, dtype=np.uint64)
+    c64 = c_rows.astype(F64)
+    G = (S.astype(F64) * (c64 * c64)).astype(F32)
+    rowmax = relu.max(axis=1).astype(np.int32) if relu.shape[1] else np.zeros(n, np.int32)
+    return G, S, rowmax
+
+
+def length_normalise(y: np.ndarray, G: np.ndarray, tau: float, eps: float) -> np.ndarray:
+    """Next layer's input x = y * tau/(||y|| + eps) with ||y|| = sqrt(G) (FF length
+    normalisation; the paper is silent, the benchmark spec asks for it).  One sqrt, one add,
+    one divide per sample; one multiply per element."""
+    r = F32(tau) / (np.sqrt(G.astype(F32)) + F32(eps))
+    return y * r.reshape((-1,) + (1,) * (y.ndim - 1)).astype(F32)
+
+
+# --------------------------------------------------------------------------------------
+# FF loss, sigma and the look-ahead coefficient  (Eq. 1-4; Alg. 1 lines 8-9)
+# --------------------------------------------------------------------------------------
+_LOG2E = F64(1.4426950408889634)            # nearest double to 1/ln 2
+_LN2_HI = F64(6.93147180369123816490e-01)   # ln 2 split so that n*LN2_HI is exact
+_LN2_LO = F64(1.90821492927058770002e-10)
+_EXP_DEG = 13
+
+
+def exp_nonpos(v: np.ndarray) -> np.ndarray:
+    """e^v for v <= 0 in float64 by a fixed recipe (clamp at -700; n = rint(v/ln2);
+    r = (v - n*LN2_HI) - n*LN2_LO; degree-13 Taylor polynomial by Horner with separate
+    multiply and add; scale by 2^n).  A recipe instead of libm so that any two
+    implementations agree bit for bit."""
+    v = np.maximum(np.asarray(v, dtype=F64), F64(-700.0))
+    n = np.rint(v * _LOG2E)
+    r = (v - n * _LN2_HI) - n * _LN2_LO
+    fact = 1
+    coef = []
+    for k in range(_EXP_DEG + 1):
+        fact = fact * k if k > 0 else 1
+        coef.append(F64(1.0) / F64(fact))
+    p = np.full_like(r, coef[_EXP_DEG])
+    for k in range(_EXP_DEG - 1, -1, -1):
+        p = p * r
+        p = p + coef[k]
+    return np.ldexp(p, n.astype(np.int64))
+
+
+def sigmoid_spec(x: np.ndarray) -> np.ndarray:
+    """sigma(x) = 1/(1+e^-x) from e = e^{-|x|}: x >= 0 -> 1/(1+e), else e/(1+e)."""
+    x = np.asarray(x, dtype=F64)
+    e = exp_nonpos(-np.abs(x))
+    d = F64(1.0) + e
+    return np.where(x >= 0, F64(1.0) / d, e / d)
+
+
+def ff_loss_terms(G: np.ndarray, theta: float, B: int):
+    """Per-sample loss and dL/dG.  Positive rows (Eq. 1): L = log(1+e^{-(G-theta)}),
+    dL/dG = -sigma(-(G-theta)).  Negative rows (Eq. 2): L = log(1+e^{G-theta}),
+    dL/dG = +sigma(G-theta)."""
+    z = G.astype(F64) - F64(F32(theta))
+    sign = np.concatenate([-np.ones(B), np.ones(B)])        # -1 positive set, +1 negative set
+    arg = sign * z                                          # L = softplus(arg)
+    L = np.maximum(arg, 0.0) + np.log1p(np.exp(-np.abs(arg)))
+    gprime = sign * sigmoid_spec(arg)
+    return L, gprime
+
+
+def lookahead_loss_coef(G_layers: Sequence[np.ndarray], thetas: Sequence[float], B: int,
+                        lam: float):
+    """Loss of the current layer (first entry) with the look-ahead term over the later layers
+    (Eq. 3):  L_new = L_1 + lambda*(L_2+...+L_final), averaged over the 2B samples, and the
+    per-sample coefficient of Eq. 4 under the scalar-coefficient reading:
+        coef_m = (g'_1,m + lambda * sum_{j>1} g'_j,m) / (2B),   g'_j = dL_j/dG_j,
+    so that dH = 2*coef*Y.  All of it in float64, coef rounded once to float32."""
+    M = 2 * B
+    lam64 = F64(F32(lam))
+    L0, g0 = ff_loss_terms(G_layers[0], thetas[0], B)
+    Lsum = np.zeros(M, dtype=F64)
+    gsum = np.zeros(M, dtype=F64)
+    for Gj, tj in zip(G_layers[1:], thetas[1:]):
+        Lj, gj = ff_loss_terms(Gj, tj, B)
+        Lsum = Lsum + Lj
+        gsum = gsum + gj
+    inv_m = F64(1.0) / F64(M)
+    coef = ((g0 + lam64 * gsum) * inv_m).astype(F32)
+    loss = float(np.sum(L0 + lam64 * Lsum) * inv_m) if M else 0.0
+    return loss, coef
+
+
+# --------------------------------------------------------------------------------------
+# One layer: forward, loss/gradient, update  (Fig. 4 dataflow, Sec. IV-B)
+# --------------------------------------------------------------------------------------
+@dataclass
+class LayerState:
+    """Everything one layer produces during a step (all of it compared against the GPU)."""
+    Xq: np.ndarray = None
+    Wq: np.ndarray = None
+    a_x: tuple = None          # (absmax pos, absmax neg) of the layer input
+    a_w: np.float32 = None
+    acc: np.ndarray = None     # int32 forward accumulator
+    Y: np.ndarray = None
+    S: np.ndarray = None       # exact integer sum of relu(acc)^2 per sample
+    rowmax: np.ndarray = None
+    G: np.ndarray = None
+    Xnext: np.ndarray = None
+    loss: float = None
+    coef: np.ndarray = None
+    a_dh: tuple = None
+    dHq: np.ndarray = None
+    accW: np.ndarray = None    # [2, N, K] int32, pass-separated
+    W_new: np.ndarray = None
+    dW: np.ndarray = None      # dequantised weight gradient (float32)
+
+
+def _pass_rows(v_pos, v_neg, B):
+    return np.concatenate([np.full(B, v_pos, dtype=F32), np.full(B, v_neg, dtype=F32)])
+
+
+def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: int) -> LayerState:
+    """Quantise A and W, INT8 MAC, dequantise + ReLU, goodness, normalised output."""
+    st = LayerState()
+    X = np.asarray(X, dtype=F32)
+    W = np.asarray(W, dtype=F32)
+    st.Xq, st.a_x = quantize_two_pass(X, B, spec.round_x,
+                                      rounding_key(spec.seed, ROLE_X, spec.index, step))
+    st.a_w = absmax(W)
+    st.Wq = quantize(W, st.a_w, spec.round_w, rounding_key(spec.seed, ROLE_W, spec.index, step))
+    if spec.kind == KIND_LINEAR:
+        st.acc = int8_gemm_nt(st.Xq, st.Wq)
+    else:
+        st.acc = int8_conv3x3(st.Xq, st.Wq.reshape(spec.N, 3, 3, spec.Cin))
+    s_w, _ = scale_pair(st.a_w)
+    c_rows = _pass_rows(scale_pair(st.a_x[0])[0] * s_w, scale_pair(st.a_x[1])[0] * s_w, B)
+    st.Y = dequant_relu(st.acc, c_rows)
+    st.G, st.S, st.rowmax = goodness(st.acc, c_rows)
+    st.Xnext = length_normalise(st.Y, st.G, spec.tau, spec.eps)
+    return st
+
+
+def layer_loss_grad(spec: LayerSpec, st: LayerState, B: int, G_later: Sequence[np.ndarray],
+                    theta_later: Sequence[float], lam: float, step: int) -> LayerState:
+    """Loss (Eq. 1-3), g^Y = dH = 2*coef*Y, and its INT8 quantisation per pass (Sec. IV-B)."""
+    st.loss, st.coef = lookahead_loss_coef([st.G] + list(G_later),
+                                           [spec.theta] + list(theta_later), B, lam)
+    k2 = F32(2.0) * st.coef
+    dH = k2.reshape((-1,) + (1,) * (st.Y.ndim - 1)) * st.Y
+    st.dHq, st.a_dh = quantize_two_pass(dH, B, spec.round_dh,
+                                        rounding_key(spec.seed, ROLE_DH, spec.index, step))
+    return st
+
+
+def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int) -> LayerState:
+    """g^W per pass as an INT8 MAC, dequantised and applied as plain SGD (Sec. IV-B; Alg. 1
+    line 9):  g = float(accP)*cP + float(accN)*cN,  W <- W - lr*g."""
+    W = np.asarray(W, dtype=F32)
+    accW = []
+    for p in range(2):
+        sl = slice(p * B, (p + 1) * B)
+        if spec.kind == KIND_LINEAR:
+            accW.append(int8_gemm_tn(st.dHq[sl], st.Xq[sl]))
+        else:
+            accW.append(int8_conv3x3_wgrad(st.dHq[sl], st.Xq[sl]).reshape(spec.N, spec.K))
+    st.accW = np.stack(accW)
+    cP = scale_pair(st.a_dh[0])[0] * scale_pair(st.a_x[0])[0]
+    cN = scale_pair(st.a_dh[1])[0] * scale_pair(st.a_x[1])[0]
+    st.dW = st.accW[0].astype(F32) * cP + st.accW[1].astype(F32) * cN
+    st.W_new = W - F32(spec.lr) * st.dW
+    return st
+
+
+def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: int, lam: float,
+               step: int) -> List[LayerState]:
+    """Body of Algorithm 1's epoch loop: one INT8 forward through all k layers with the
+    pre-update weights (line 5), goodness of every layer (line 6), then for each layer its
+    loss from the G's (line 8) and its INT8 gradient and update (line 9).  lambda is the
+    caller's (lines 2 and 11).  With one layer and lambda = 0 this is the vanilla step."""
+    states = []
+    x = X
+    for spec, W in zip(specs, Ws):
+        st = layer_forward(spec, x, W, B, step)
+        states.append(st)
+        x = st.Xnext
+    for l, (spec, W) in enumerate(zip(specs, Ws)):
+        later = list(range(l + 1, len(specs)))
+        layer_loss_grad(spec, states[l], B, [states[j].G for j in later],
+                        [specs[j].theta for j in later], lam, step)
+        layer_update(spec, states[l], W, B)
+    return states
+
+
+# --------------------------------------------------------------------------------------
+# Unquantised float64 model of one layer (for the finite-difference pin only)
+# --------------------------------------------------------------------------------------
+def fp64_layer_loss(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int) -> float:
+    """Mean over the 2B samples of Eq. 1 / Eq. 2 with G = ||relu(X W^T)||^2, no quantisation."""
+    X = np.asarray(X, dtype=F64)
+    W = np.asarray(W, dtype=F64)
+    if spec.kind == KIND_LINEAR:
+        Y = np.maximum(X @ W.T, 0.0)
+    else:
+        xp = np.pad(X, ((0, 0), (1, 1), (1, 1), (0, 0)))
+        w4 = W.reshape(spec.N, 3, 3, spec.Cin)
+        Y = np.zeros(X.shape[:3] + (spec.N,))
+        for r in range(3):
+            for s in range(3):
+                Y += xp[:, r:r + spec.H, s:s + spec.Wd, :] @ w4[:, r, s, :].T
+        Y = np.maximum(Y, 0.0)
+    G = (Y.reshape(2 * B, -1) ** 2).sum(axis=1)
+    z = G - spec.theta
+    sign = np.concatenate([-np.ones(B), np.ones(B)])
+    arg = sign * z
+    return float(np.mean(np.maximum(arg, 0.0) + np.log1p(np.exp(-np.abs(arg)))))

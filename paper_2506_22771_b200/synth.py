@@ -1,0 +1,137 @@
+"""Seeded synthetic inputs shaped like the paper's workloads (Sec. V-A: MNIST-style MLP data,
+CIFAR-style CNN data).  Serves the oracle tests, the GPU parity tests and the benchmark alike,
+and holds none of the method's arithmetic: it only draws numbers, writes the one-hot label
+into the input ('Generate positive and negative sets', Alg. 1 line 3; Sec. III) and scales
+each sample to the length the first layer expects (the layer-1 input arrives length-normalised).
+
+Nothing here is real MNIST / CIFAR-10 data: only their shapes and value ranges are used.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List
+
+import numpy as np
+
+F32 = np.float32
+
+
+@dataclass
+class LayerCfg:
+    kind: int          # 0 linear, 1 conv3x3 (stride 1, pad 1, NHWC)
+    K: int
+    N: int
+    theta: float
+    lr: float
+    tau: float
+    H: int = 1
+    Wd: int = 1
+    Cin: int = 0
+    eps: float = 1e-8
+
+
+@dataclass
+class Workload:
+    name: str
+    B: int                       # positives per batch = negatives per batch
+    layers: List[LayerCfg]
+    in_shape: tuple              # per-sample input shape
+    data: str                    # "uniform01" | "normal"
+    weights: str                 # "kaiming_uniform" | "normal_1_over_k"
+    steps: int
+    lam_per_step: float = 0.0    # look-ahead lambda increment per step (0: vanilla)
+    greedy: bool = False         # train layers one after another (config 2)
+
+
+def _rng(seed: int, stream: int) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[seed & 0xFFFFFFFFFFFFFFFF, stream]))
+
+
+def _mlp(widths, theta=None, lr=0.03):
+    out = []
+    for K, N in zip(widths[:-1], widths[1:]):
+        out.append(LayerCfg(0, K, N, float(N if theta is None else theta), lr, float(np.sqrt(N))))
+    return out
+
+
+def workload(name: str) -> Workload:
+    """The five configurations of the benchmark spec (sizes only; data are drawn by make_*)."""
+    if name == "tiny_mlp":          # config 1
+        return Workload(name, 64, _mlp([784, 500, 500]), (784,), "uniform01", "kaiming_uniform", 10)
+    if name == "mlp_greedy":        # config 2
+        return Workload(name, 1024, _mlp([784, 2000, 2000, 2000, 2000]), (784,), "uniform01",
+                        "kaiming_uniform", 58, greedy=True)
+    if name == "mlp_lookahead":     # config 3
+        return Workload(name, 4096, _mlp([784, 2000, 2000, 2000, 2000]), (784,), "uniform01",
+                        "kaiming_uniform", 200, lam_per_step=0.001)
+    if name == "cnn":               # config 4
+        chans = [3, 64, 128, 256]
+        layers = [LayerCfg(1, 9 * ci, co, float(co * 1024), 0.03, float(np.sqrt(co * 1024)),
+                           H=32, Wd=32, Cin=ci) for ci, co in zip(chans[:-1], chans[1:])]
+        return Workload(name, 256, layers, (32, 32, 3), "normal", "kaiming_uniform", 50)
+    if name == "roofline":          # config 5
+        return Workload(name, 16384, [LayerCfg(0, 8192, 8192, 4096.0, 0.03, float(np.sqrt(8192)))],
+                        (8192,), "normal", "normal_1_over_k", 100)
+    raise KeyError(name)
+
+
+def scaled(w: Workload, B: int = None, width_div: int = 1) -> Workload:
+    """A smaller copy of a workload (fewer rows and/or narrower layers) for parity tests."""
+    layers = []
+    for l in w.layers:
+        first = l is w.layers[0]
+        per = l.H * l.Wd
+        ratio = l.theta / float(l.N * per)          # theta relative to the layer's output size
+        if l.kind == 0:
+            K = l.K if first else max(8, l.K // width_div)
+            N = max(8, l.N // width_div)
+            layers.append(LayerCfg(0, K, N, ratio * N, l.lr, float(np.sqrt(N))))
+        else:
+            Cin = l.Cin if first else max(4, l.Cin // width_div)
+            N = max(4, l.N // width_div)
+            layers.append(LayerCfg(1, 9 * Cin, N, ratio * N * per, l.lr, float(np.sqrt(N * per)),
+                                   H=l.H, Wd=l.Wd, Cin=Cin))
+    return Workload(w.name + "_scaled", B or w.B, layers, w.in_shape, w.data, w.weights, w.steps,
+                    w.lam_per_step, w.greedy)
+
+
+def make_weights(w: Workload, seed: int) -> List[np.ndarray]:
+    """Random-init FP32 weights [N,K] per layer (conv: [N,3,3,Cin] flattened to [N,9*Cin])."""
+    out = []
+    for i, l in enumerate(w.layers):
+        g = _rng(seed, 1000 + i)
+        if w.weights == "kaiming_uniform":
+            bound = np.sqrt(6.0 / l.K)
+            Wt = g.uniform(-bound, bound, size=(l.N, l.K))
+        else:
+            Wt = g.normal(0.0, np.sqrt(1.0 / l.K), size=(l.N, l.K))
+        out.append(np.ascontiguousarray(Wt.astype(F32)))
+    return out
+
+
+def make_batch(w: Workload, seed: int, batch_index: int = 0, B: int = None) -> np.ndarray:
+    """One batch [2B, *in_shape] FP32: rows 0..B-1 positive (true label), B..2B-1 negative (a
+    random wrong label), label written one-hot into the first 10 entries (CNN: channel 0, row 0,
+    pixels 0..9), each sample scaled to length tau0 = sqrt(number of input values)."""
+    B = B or w.B
+    g = _rng(seed, 2000 + batch_index)
+    n_in = int(np.prod(w.in_shape))
+    if w.data == "uniform01":
+        base = g.random((B, n_in), dtype=np.float64)
+    else:
+        base = g.normal(0.0, 1.0, size=(B, n_in))
+    label = g.integers(0, 10, size=B)
+    wrong = (label + g.integers(1, 10, size=B)) % 10
+    x = np.concatenate([base, base], axis=0).reshape((2 * B,) + tuple(w.in_shape))
+    for p, lab in enumerate((label, wrong)):
+        rows = np.arange(B) + p * B
+        if len(w.in_shape) == 1:
+            x[rows, :10] = 0.0
+            x[rows, lab] = 1.0
+        else:
+            x[rows, 0, :10, 0] = 0.0
+            x[rows, 0, lab, 0] = 1.0
+    flat = x.reshape(2 * B, -1)
+    norm = np.sqrt((flat ** 2).sum(axis=1, keepdims=True))
+    flat *= np.sqrt(float(n_in)) / (norm + 1e-8)
+    return np.ascontiguousarray(x.astype(F32))

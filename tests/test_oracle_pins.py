@@ -1,0 +1,476 @@
+"""Pins of the CPU oracle against things other than itself: hand-computed fixtures, closed
+forms of Eq. 1-3, brute-force loops, finite differences, library routines, error bounds.
+CPU only."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import ffint8_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+F32 = np.float32
+
+
+def _rows(name):
+    out = []
+    for line in open(os.path.join(GOLD, name)):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            out.append(line.split())
+    return out
+
+
+def _spec(K, N, theta=None, kind=0, H=1, Wd=1, Cin=0, rnd=O.ROUND_NEAREST, lr=0.03, index=0, seed=3):
+    per = H * Wd
+    return O.LayerSpec(kind, K, N, float(theta if theta is not None else N * per), lr,
+                       float(np.sqrt(N * per)), 1e-8, H, Wd, Cin, rnd, O.ROUND_NEAREST, rnd, seed, index)
+
+
+# ------------------------------------------------------------------ quantiser (Sec. IV)
+def test_quant_nearest_hand_example():
+    rows = _rows("quant_nearest_2x3.txt")
+    x = np.array([float(r[0]) for r in rows], dtype=F32)
+    q = np.array([int(r[1]) for r in rows], dtype=np.int8)
+    a = O.absmax(x)
+    assert a == F32(2.0)
+    assert np.array_equal(O.quantize(x, a, O.ROUND_NEAREST), q)
+
+
+def test_quant_stochastic_hand_example():
+    rows = _rows("quant_stochastic_1x6.txt")
+    x = np.array([float(r[0]) for r in rows], dtype=F32)
+    u = np.array([float(r[1]) for r in rows], dtype=F32)
+    q = np.array([int(r[2]) for r in rows], dtype=np.int8)
+    assert np.array_equal(O.quantize(x, F32(4.0), O.ROUND_STOCHASTIC, u=u), q)
+
+
+def test_quant_error_bounds_and_range():
+    g = np.random.default_rng(0)
+    x = g.normal(size=5000).astype(F32)
+    a = O.absmax(x)
+    s, _ = O.scale_pair(a)
+    q = O.quantize(x, a, O.ROUND_NEAREST)
+    err = np.abs(x.astype(np.float64) - float(s) * q.astype(np.float64))
+    assert err.max() <= float(s) / 2 * (1 + 1e-5)                 # |x - s q| <= s/2
+    assert abs(int(q[np.argmax(np.abs(x))])) == 127               # absmax element -> +-127
+    assert q.min() >= -127 and q.max() <= 127
+    qs = O.quantize(x, a, O.ROUND_STOCHASTIC, key=O.rounding_key(1, 0, 0, 0))
+    errs = np.abs(x.astype(np.float64) - float(s) * qs.astype(np.float64))
+    assert errs.max() < float(s) * (1 + 1e-5)                     # |x - s q| < s
+    assert np.array_equal(O.quantize(x, a, O.ROUND_STOCHASTIC, u=np.zeros_like(x)),
+                          np.clip(np.floor(x * O.scale_pair(a)[1]), -127, 127).astype(np.int8))
+
+
+def test_quant_zero_tensor_and_idempotence():
+    z = np.zeros((3, 4), dtype=F32)
+    assert O.absmax(z) == 0 and not O.quantize(z, O.absmax(z), O.ROUND_NEAREST).any()
+    assert not O.quantize(z, O.absmax(z), O.ROUND_STOCHASTIC, key=(1, 2)).any()
+    g = np.random.default_rng(1)
+    x = g.uniform(-3, 3, size=1000).astype(F32)
+    x[0] = 3.0
+    a = O.absmax(x)
+    s, _ = O.scale_pair(a)
+    q = O.quantize(x, a, O.ROUND_NEAREST)
+    xr = (s * q.astype(F32)).astype(F32)
+    assert np.array_equal(O.quantize(xr, O.absmax(xr), O.ROUND_NEAREST), q)
+
+
+def test_quant_rejects_nonfinite():
+    with pytest.raises(FloatingPointError):
+        O.absmax(np.array([1.0, np.inf], dtype=F32))
+    with pytest.raises(FloatingPointError):
+        O.absmax(np.array([np.nan], dtype=F32))
+
+
+def test_stochastic_rounding_is_unbiased():
+    # E[q] = t for every element (the property the paper takes stochastic rounding for)
+    x = np.array([0.013, -0.4, 0.77, 0.5001, -0.9999, 1.0], dtype=F32)
+    a = O.absmax(x)
+    t = x.astype(np.float64) * 127.0
+    acc = np.zeros_like(t)
+    n = 20000
+    for seed in range(n):
+        acc += O.quantize(x, a, O.ROUND_STOCHASTIC, key=O.rounding_key(seed, 0, 0, 0))
+    assert np.max(np.abs(acc / n - t)) < 4 * 0.5 / math.sqrt(n)
+
+
+def test_rounding_hash_statistics_and_splitmix_vectors():
+    # SplitMix64 reference outputs for state 1234567 (published test vector of the generator)
+    s = 1234567
+    want = [6457827717110365317, 3203168211198807973, 9817491932198370423]
+    got = [O._splitmix64((s + i * 0x9E3779B97F4A7C15) & ((1 << 64) - 1)) for i in range(3)]
+    assert got == want
+    k = O.rounding_key(5, O.ROLE_X, 2, 9)
+    u = O.rounding_uniform(np.arange(1 << 20, dtype=np.uint64), *k)
+    assert u.dtype == F32 and u.min() >= 0.0 and u.max() < 1.0
+    assert abs(float(u.mean()) - 0.5) < 2e-3
+    hist = np.bincount((u * 64).astype(int), minlength=64)
+    chi2 = float(((hist - u.size / 64) ** 2 / (u.size / 64)).sum())
+    assert chi2 < 130                                   # 63 dof; p ~ 1e-6
+    assert abs(np.corrcoef(u[:-1], u[1:])[0, 1]) < 5e-3  # neighbouring counters uncorrelated
+    # different role / layer / step give different streams
+    for other in (O.rounding_key(5, O.ROLE_DH, 2, 9), O.rounding_key(5, O.ROLE_X, 3, 9),
+                  O.rounding_key(5, O.ROLE_X, 2, 10), O.rounding_key(6, O.ROLE_X, 2, 9)):
+        v = O.rounding_uniform(np.arange(4096, dtype=np.uint64), *other)
+        assert abs(np.corrcoef(u[:4096], v)[0, 1]) < 0.06
+
+
+# ------------------------------------------------------------------ INT8 MAC (Sec. IV-B)
+def _brute_gemm_nt(a, b):
+    M, K = a.shape
+    N = b.shape[0]
+    out = [[0] * N for _ in range(M)]
+    for m in range(M):
+        for n in range(N):
+            s = 0
+            for k in range(K):
+                s += int(a[m, k]) * int(b[n, k])
+            out[m][n] = s
+    return np.array(out, dtype=np.int64)
+
+
+@pytest.mark.parametrize("M,N,K", [(3, 5, 33), (1, 1, 1), (7, 2, 27), (16, 9, 64)])
+def test_gemm_against_brute_force(M, N, K):
+    g = np.random.default_rng(M * 100 + N * 10 + K)
+    a = g.integers(-127, 128, size=(M, K)).astype(np.int8)
+    b = g.integers(-127, 128, size=(N, K)).astype(np.int8)
+    assert np.array_equal(O.int8_gemm_nt(a, b, row_chunk=2), _brute_gemm_nt(a, b))
+    # weight-gradient orientation: accW[n,k] = sum_m d[m,n] x[m,k]
+    d = g.integers(-127, 128, size=(M, N)).astype(np.int8)
+    want = _brute_gemm_nt(np.ascontiguousarray(d.T), np.ascontiguousarray(a.T))
+    assert np.array_equal(O.int8_gemm_tn(d, a), want)
+
+
+def test_gemm_extreme_values_exact_and_overflow_check():
+    K = 8192
+    a = np.full((2, K), 127, dtype=np.int8)
+    b = np.full((3, K), -127, dtype=np.int8)
+    assert np.all(O.int8_gemm_nt(a, b) == -127 * 127 * K)
+    g = np.random.default_rng(3)
+    a = g.integers(-127, 128, size=(64, 1000)).astype(np.int8)
+    b = g.integers(-127, 128, size=(48, 1000)).astype(np.int8)
+    want = np.einsum("mk,nk->mn", a.astype(np.int64), b.astype(np.int64))
+    assert np.array_equal(O.int8_gemm_nt(a, b), want)
+    big = np.full((1, 140000), 127, dtype=np.int8)      # 127*127*140000 > 2^31
+    with pytest.raises(OverflowError):
+        O.int8_gemm_nt(big, big)
+
+
+def _brute_conv(x, w):
+    Bn, H, Wd, Cin = x.shape
+    Cout = w.shape[0]
+    out = np.zeros((Bn, H, Wd, Cout), dtype=np.int64)
+    for b in range(Bn):
+        for h in range(H):
+            for ww in range(Wd):
+                for co in range(Cout):
+                    s = 0
+                    for r in range(3):
+                        for t in range(3):
+                            hh, wx = h + r - 1, ww + t - 1
+                            if 0 <= hh < H and 0 <= wx < Wd:
+                                for ci in range(Cin):
+                                    s += int(x[b, hh, wx, ci]) * int(w[co, r, t, ci])
+                    out[b, h, ww, co] = s
+    return out
+
+
+def _brute_wgrad(d, x):
+    Bn, H, Wd, Cin = x.shape
+    Cout = d.shape[-1]
+    out = np.zeros((Cout, 3, 3, Cin), dtype=np.int64)
+    for co in range(Cout):
+        for r in range(3):
+            for t in range(3):
+                for ci in range(Cin):
+                    s = 0
+                    for b in range(Bn):
+                        for h in range(H):
+                            for ww in range(Wd):
+                                hh, wx = h + r - 1, ww + t - 1
+                                if 0 <= hh < H and 0 <= wx < Wd:
+                                    s += int(d[b, h, ww, co]) * int(x[b, hh, wx, ci])
+                    out[co, r, t, ci] = s
+    return out
+
+
+def test_conv_against_brute_force_and_library():
+    g = np.random.default_rng(11)
+    x = g.integers(-127, 128, size=(2, 4, 5, 3)).astype(np.int8)
+    w = g.integers(-127, 128, size=(4, 3, 3, 3)).astype(np.int8)
+    d = g.integers(-127, 128, size=(2, 4, 5, 4)).astype(np.int8)
+    assert np.array_equal(O.int8_conv3x3(x, w), _brute_conv(x, w))
+    assert np.array_equal(O.int8_conv3x3_wgrad(d, x), _brute_wgrad(d, x))
+    torch = pytest.importorskip("torch")
+    x = g.integers(-127, 128, size=(3, 8, 8, 16)).astype(np.int8)
+    w = g.integers(-127, 128, size=(24, 3, 3, 16)).astype(np.int8)
+    tx = torch.from_numpy(x.astype(np.float64)).permute(0, 3, 1, 2)
+    tw = torch.from_numpy(w.astype(np.float64)).permute(0, 3, 1, 2)
+    want = torch.nn.functional.conv2d(tx, tw, padding=1).permute(0, 2, 3, 1).numpy()
+    assert np.array_equal(O.int8_conv3x3(x, w).astype(np.float64), want)
+
+
+# ------------------------------------------------------------------ epilogue / goodness
+def test_tiny_layer_hand_example():
+    vals = {r[0]: np.array([int(v) for v in r[1:]]) for r in _rows("tiny_layer.txt")}
+    X = np.array([[1, 0.5], [-0.25, 0.5]], dtype=F32)
+    W = np.array([[1, -1], [0.5, 0.25]], dtype=F32)
+    st = O.layer_forward(_spec(2, 2), X, W, 1, 0)
+    assert np.array_equal(st.Xq.ravel(), vals["Xq"])
+    assert np.array_equal(st.Wq.ravel(), vals["Wq"])
+    assert np.array_equal(st.acc.ravel(), vals["acc"])
+    assert np.array_equal(st.S, vals["S"].astype(np.uint64))
+    assert np.array_equal(st.rowmax, vals["rowmax"])
+    c = (1.0 / 127) ** 2
+    assert np.allclose(st.Y, [[8001 * c, 10176 * c], [0, 0]], rtol=1e-6)
+    assert np.allclose(st.G, [167566977 * c * c, 0.0], rtol=1e-6)
+    nrm = np.sqrt(167566977.0) * c
+    assert np.allclose(st.Xnext[0], np.array([8001, 10176]) * c * np.sqrt(2.0) / nrm, rtol=1e-6)
+    assert not st.Xnext[1].any()
+
+
+def test_goodness_zero_input_and_fp64_sum():
+    g = np.random.default_rng(5)
+    W = g.normal(size=(40, 30)).astype(F32)
+    st = O.layer_forward(_spec(30, 40), np.zeros((6, 30), F32), W, 3, 0)
+    assert not st.G.any() and not st.Y.any() and not st.Xnext.any()
+    X = g.normal(size=(6, 30)).astype(F32)
+    st = O.layer_forward(_spec(30, 40), X, W, 3, 0)
+    ref = (st.Y.astype(np.float64) ** 2).sum(axis=1)
+    assert np.allclose(st.G, ref, rtol=1e-6)
+    nrm = np.sqrt((st.Xnext.astype(np.float64) ** 2).sum(axis=1))
+    assert np.allclose(nrm, np.sqrt(40.0), rtol=1e-5)             # normalised to length tau
+
+
+def test_dequantised_forward_tracks_float_layer():
+    g = np.random.default_rng(6)
+    X = g.normal(size=(8, 256)).astype(F32)
+    W = (g.normal(size=(64, 256)) / 16).astype(F32)
+    st = O.layer_forward(_spec(256, 64), X, W, 4, 0)
+    ref = np.maximum(X.astype(np.float64) @ W.astype(np.float64).T, 0)
+    assert np.abs(st.Y - ref).max() < 0.05 * np.abs(ref).max()
+
+
+# ------------------------------------------------------------------ loss (Eq. 1-3)
+def test_loss_closed_forms():
+    theta = 2.0
+    G = np.array([0.0, 1.0, 2.0, 5.0, 0.0, 1.0, 2.0, 5.0], dtype=F32)
+    L, gp = O.ff_loss_terms(G, theta, 4)
+    z = G.astype(np.float64) - theta
+    assert np.allclose(L[:4], np.log(1 + np.exp(-z[:4])), rtol=1e-14)      # Eq. 1
+    assert np.allclose(L[4:], np.log(1 + np.exp(z[4:])), rtol=1e-14)       # Eq. 2
+    assert math.isclose(L[2], math.log(2), rel_tol=1e-15) and math.isclose(L[6], math.log(2), rel_tol=1e-15)
+    assert gp[2] == -0.5 and gp[6] == 0.5                                   # sigma(0) = 1/2
+    assert np.allclose(gp[:4], -1 / (1 + np.exp(z[:4])), rtol=1e-14)
+    assert np.allclose(gp[4:], 1 / (1 + np.exp(-z[4:])), rtol=1e-14)
+    # symmetry L_pos(G) = L_neg(2 theta - G)
+    Gs = np.array([0.5, 3.0, 3.5, 1.0], dtype=F32)
+    Ls, _ = O.ff_loss_terms(Gs, theta, 2)
+    assert math.isclose(Ls[0], Ls[2], rel_tol=1e-14) and math.isclose(Ls[1], Ls[3], rel_tol=1e-14)
+    # asymptotes without overflow
+    Gb = np.array([1e6, 0.0, 1e6, 0.0], dtype=F32)
+    Lb, gb = O.ff_loss_terms(Gb, 1000.0, 2)
+    assert np.all(np.isfinite(Lb)) and Lb[0] == 0.0 and math.isclose(Lb[2], 1e6 - 1000.0)
+    assert math.isclose(Lb[1], 1000.0) and gb[1] == -1.0 and gb[2] == 1.0 and abs(gb[0]) < 1e-300
+    # derivative of the loss by finite differences of the closed form
+    for G0, pos in [(1.3, True), (2.9, False), (7.0, True)]:
+        f = (lambda v: math.log1p(math.exp(-(v - theta)))) if pos else (lambda v: math.log1p(math.exp(v - theta)))
+        fd = (f(G0 + 1e-6) - f(G0 - 1e-6)) / 2e-6
+        arr = np.array([G0, G0], dtype=np.float64)
+        _, gq = O.ff_loss_terms(arr, theta, 1)
+        assert math.isclose(gq[0 if pos else 1], fd, rel_tol=1e-6)
+
+
+def test_exp_and_sigmoid_recipe_accuracy():
+    v = -np.concatenate([np.linspace(0, 50, 200001), np.linspace(50, 700, 20001)])
+    got = O.exp_nonpos(v)
+    want = np.exp(v)
+    ulp = np.abs(got - want) / np.spacing(want)
+    assert ulp.max() <= 2.0
+    assert O.exp_nonpos(np.array([0.0]))[0] == 1.0
+    assert O.exp_nonpos(np.array([-1e9]))[0] == O.exp_nonpos(np.array([-700.0]))[0] > 0
+    x = np.linspace(-40, 40, 100001)
+    s = O.sigmoid_spec(x)
+    assert np.allclose(s, 1 / (1 + np.exp(-x)), rtol=1e-15, atol=0)
+    assert np.allclose(s + O.sigmoid_spec(-x), 1.0, atol=2e-16)
+
+
+def test_lookahead_loss_and_coef_closed_form():
+    g = np.random.default_rng(8)
+    B = 5
+    Gs = [g.uniform(0, 6, size=2 * B).astype(F32) for _ in range(3)]
+    th = [2.0, 3.0, 2.5]
+    lam = 0.125
+    loss, coef = O.lookahead_loss_coef(Gs, th, B, lam)
+    per = [O.ff_loss_terms(G, t, B) for G, t in zip(Gs, th)]
+    want_loss = np.mean(per[0][0] + lam * (per[1][0] + per[2][0]))          # Eq. 3
+    assert math.isclose(loss, want_loss, rel_tol=1e-14)
+    want_coef = (per[0][1] + lam * (per[1][1] + per[2][1])) / (2 * B)       # Eq. 4, scalar reading
+    assert np.allclose(coef, want_coef, rtol=1e-6)
+    # lambda = 0 and "no later layer" both reduce to the vanilla coefficient, bit for bit
+    _, c0 = O.lookahead_loss_coef(Gs, th, B, 0.0)
+    _, c1 = O.lookahead_loss_coef(Gs[:1], th[:1], B, 0.7)
+    assert np.array_equal(c0, c1)
+    assert np.all(c0[:B] <= 0) and np.all(c0[B:] >= 0)     # raise G on positives, lower on negatives
+
+
+# ------------------------------------------------------------------ gradient (Sec. IV-B)
+def _analytic_grad(spec, X, W, B):
+    """dW of the unquantised mean loss through the oracle's own coefficient and dH = 2*coef*Y."""
+    X64, W64 = X.astype(np.float64), W.astype(np.float64)
+    Y = np.maximum(X64 @ W64.T, 0)
+    G = (Y ** 2).sum(axis=1)
+    z = G - spec.theta
+    sign = np.concatenate([-np.ones(B), np.ones(B)])
+    coef = sign * O.sigmoid_spec(sign * z) / (2 * B)
+    return (2 * coef[:, None] * Y).T @ X64
+
+
+def test_gradient_matches_finite_differences_fp64():
+    g = np.random.default_rng(9)
+    B, K, N = 3, 6, 5
+    X = g.normal(size=(2 * B, K)).astype(F32)
+    W = (g.normal(size=(N, K)) * 0.4).astype(F32)
+    spec = _spec(K, N, theta=2.0)
+    ana = _analytic_grad(spec, X, W, B)
+    fd = np.zeros_like(ana)
+    h = 1e-6
+    for n in range(N):
+        for k in range(K):
+            Wp, Wm = W.astype(np.float64).copy(), W.astype(np.float64).copy()
+            Wp[n, k] += h
+            Wm[n, k] -= h
+            fd[n, k] = (O.fp64_layer_loss(spec, X, Wp, B) - O.fp64_layer_loss(spec, X, Wm, B)) / (2 * h)
+    assert np.allclose(ana, fd, rtol=1e-5, atol=1e-8)
+    # the oracle's coefficient equals the one used above (float32-rounded)
+    st = O.layer_forward(spec, X, W, B, 0)
+    O.layer_loss_grad(spec, st, B, [], [], 0.0, 0)
+    z = st.G.astype(np.float64) - 2.0
+    sign = np.concatenate([-np.ones(B), np.ones(B)])
+    assert np.allclose(st.coef, sign * O.sigmoid_spec(sign * z) / (2 * B), rtol=1e-6)
+
+
+@pytest.mark.parametrize("kind", [0, 1])
+def test_int8_gradient_tracks_fp64_gradient(kind):
+    """The whole quantised chain (dH -> INT8 -> INT8 MAC -> dequantise) must point the way the
+    finite-difference-checked gradient points: catches sign, transposition and scale mistakes."""
+    g = np.random.default_rng(10 + kind)
+    if kind == 0:
+        B, K, N = 32, 96, 48
+        spec = _spec(K, N, theta=float(N))
+        X = g.normal(size=(2 * B, K)).astype(F32)
+        W = (g.normal(size=(N, K)) * np.sqrt(2.0 / K)).astype(F32)
+    else:
+        B, H, Cin, N = 4, 6, 8, 8
+        K = 9 * Cin
+        spec = _spec(K, N, theta=float(N * H * H), kind=1, H=H, Wd=H, Cin=Cin)
+        X = g.normal(size=(2 * B, H, H, Cin)).astype(F32)
+        W = (g.normal(size=(N, K)) * np.sqrt(2.0 / K)).astype(F32)
+    st = O.layer_forward(spec, X, W, B, 0)
+    O.layer_loss_grad(spec, st, B, [], [], 0.0, 0)
+    O.layer_update(spec, st, W, B)
+    # float64 gradient of the unquantised loss by central differences on a sample of entries
+    idx = [(int(g.integers(spec.N)), int(g.integers(spec.K))) for _ in range(40)]
+    h = 1e-5
+    fd = []
+    for n, k in idx:
+        Wp, Wm = W.astype(np.float64).copy(), W.astype(np.float64).copy()
+        Wp[n, k] += h
+        Wm[n, k] -= h
+        fd.append((O.fp64_layer_loss(spec, X, Wp, B) - O.fp64_layer_loss(spec, X, Wm, B)) / (2 * h))
+    fd = np.array(fd)
+    got = np.array([st.dW[n, k] for n, k in idx], dtype=np.float64)
+    cos = float(got @ fd / (np.linalg.norm(got) * np.linalg.norm(fd)))
+    assert cos > 0.98
+    assert 0.8 < np.linalg.norm(got) / np.linalg.norm(fd) < 1.25
+    assert np.array_equal(st.W_new, W - F32(spec.lr) * st.dW)
+
+
+def test_absmax_shortcuts_hold_bitwise():
+    """max|dH| and max|Xnext| per pass equal the values obtained from the per-sample max of
+    relu(acc) alone (rounded multiplication by a fixed factor is monotone)."""
+    g = np.random.default_rng(12)
+    B, K, N = 16, 64, 40
+    spec = _spec(K, N, rnd=O.ROUND_STOCHASTIC)
+    X = g.normal(size=(2 * B, K)).astype(F32)
+    W = (g.normal(size=(N, K)) / 8).astype(F32)
+    st = O.layer_forward(spec, X, W, B, 3)
+    O.layer_loss_grad(spec, st, B, [], [], 0.0, 3)
+    s_w = O.scale_pair(st.a_w)[0]
+    r = F32(spec.tau) / (np.sqrt(st.G) + F32(spec.eps))
+    for p in range(2):
+        sl = slice(p * B, (p + 1) * B)
+        c = O.scale_pair(st.a_x[p])[0] * s_w
+        ymax = st.rowmax[sl].astype(F32) * c
+        k2 = F32(2.0) * st.coef[sl]
+        assert np.max(np.abs(k2 * ymax)) == st.a_dh[p]
+        assert np.max(ymax * r[sl]) == O.absmax(st.Xnext[sl])
+
+
+# ------------------------------------------------------------------ update / step
+def test_update_hand_example_and_fixed_points():
+    spec = _spec(2, 2, theta=0.5, lr=0.5)
+    X = np.array([[1, 0.5], [-0.25, 0.5]], dtype=F32)
+    W = np.array([[1, -1], [0.5, 0.25]], dtype=F32)
+    st = O.layer_forward(spec, X, W, 1, 0)
+    O.layer_loss_grad(spec, st, 1, [], [], 0.0, 0)
+    O.layer_update(spec, st, W, 1)
+    # negative row has Y = 0 -> dH = 0 -> its pass contributes nothing
+    assert not st.dHq[1].any() and not st.accW[1].any() and st.a_dh[1] == 0
+    # positive row: dH = 2*coef*y, |dH| max at y = 10176*c -> dHq = [-100 (rint(-99.86)), -127]
+    assert np.array_equal(st.dHq[0], [-100, -127])
+    assert np.array_equal(st.accW[0], [[-100 * 127, -100 * 64], [-127 * 127, -127 * 64]])
+    G0 = 167566977 / 127.0 ** 4
+    coef = -1 / (1 + math.exp(G0 - 0.5)) / 2
+    dH1 = 2 * coef * 10176 / 127.0 ** 2
+    dW = np.array(st.accW[0], dtype=np.float64) * (abs(dH1) / 127) * (1 / 127)
+    assert np.allclose(st.dW, dW, rtol=1e-5)
+    assert np.allclose(st.W_new, W - 0.5 * dW, rtol=1e-6)
+    # lr = 0 leaves W untouched; so does a zero gradient
+    spec0 = _spec(2, 2, theta=0.5, lr=0.0)
+    st0 = O.layer_update(spec0, O.layer_loss_grad(spec0, O.layer_forward(spec0, X, W, 1, 0), 1, [], [], 0.0, 0), W, 1)
+    assert np.array_equal(st0.W_new, W)
+    Xz = np.zeros_like(X)
+    stz = O.layer_update(spec, O.layer_loss_grad(spec, O.layer_forward(spec, Xz, W, 1, 0), 1, [], [], 0.0, 0), W, 1)
+    assert np.array_equal(stz.W_new, W)
+
+
+def _net(g, widths, B, rnd=O.ROUND_STOCHASTIC):
+    specs = [_spec(K, N, rnd=rnd, index=i) for i, (K, N) in enumerate(zip(widths[:-1], widths[1:]))]
+    Ws = [(g.normal(size=(s.N, s.K)) * np.sqrt(2.0 / s.K)).astype(F32) for s in specs]
+    X = g.normal(size=(2 * B, widths[0])).astype(F32)
+    return specs, Ws, X
+
+
+def test_train_step_reductions_and_determinism():
+    g = np.random.default_rng(13)
+    B = 8
+    specs, Ws, X = _net(g, [20, 24, 16, 12], B)
+    a = O.train_step(specs, Ws, X, B, 0.0, 4)
+    b = O.train_step(specs, Ws, X, B, 0.0, 4)
+    for sa, sb in zip(a, b):                                  # run-to-run identity
+        assert np.array_equal(sa.W_new, sb.W_new) and np.array_equal(sa.dHq, sb.dHq)
+    # lambda = 0: every layer's step equals the stand-alone (vanilla) step on the same input
+    x = X
+    for l, spec in enumerate(specs):
+        st = O.layer_forward(spec, x, Ws[l], B, 4)
+        O.layer_loss_grad(spec, st, B, [], [], 0.0, 4)
+        O.layer_update(spec, st, Ws[l], B)
+        assert np.array_equal(st.W_new, a[l].W_new) and np.array_equal(st.dHq, a[l].dHq)
+        assert st.loss == a[l].loss
+        x = st.Xnext
+    # lambda > 0 changes every layer but the last; all G's come from the pre-update forward
+    c = O.train_step(specs, Ws, X, B, 0.5, 4)
+    assert np.array_equal(c[-1].W_new, a[-1].W_new)
+    assert not np.array_equal(c[0].coef, a[0].coef)
+    for sa, sc in zip(a, c):
+        assert np.array_equal(sa.G, sc.G) and np.array_equal(sa.Xq, sc.Xq)
+    # Eq. 3 from the per-layer vanilla losses
+    lam32 = float(F32(0.5))
+    per = [O.ff_loss_terms(s.G, sp.theta, B)[0] for s, sp in zip(a, specs)]
+    assert math.isclose(c[0].loss, float(np.mean(per[0] + lam32 * (per[1] + per[2]))), rel_tol=1e-12)
+    # different step index -> different stochastic rounding, same scales
+    d = O.train_step(specs, Ws, X, B, 0.0, 5)
+    assert d[0].a_x == a[0].a_x and not np.array_equal(d[0].Xq, a[0].Xq)
