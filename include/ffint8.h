@@ -1,0 +1,170 @@
+/*
+ * ffint8.h — C ABI of libffint8: the FF-INT8 per-layer Forward-Forward train step on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library implements the single-layer dataflow of the FF-INT8 paper (Sec. IV-B, Fig. 4):
+ * symmetric uniform quantisation (Sec. IV) of the layer input A (stochastic rounding) and of
+ * the weights W, an INT8 x INT8 -> INT32 MAC (dense or 3x3 convolution), goodness
+ * G = ||y||^2 (Sec. III; Alg. 1 line 6), the negative-log-likelihood losses of Eq. 1 / Eq. 2
+ * with the look-ahead term of Eq. 3 / Eq. 4, the output gradient g^Y quantised to INT8, the
+ * weight gradient g^W as a second INT8 MAC, and the weight update (Alg. 1 line 9).  No input
+ * gradient g^A is ever formed (Sec. IV-B).
+ *
+ * Conventions
+ *  - Every pointer inside ff_layer_bufs is a DEVICE pointer owned by the caller, 16-byte
+ *    aligned, valid on the device the context was created for.  Pointers to ff_layer_desc /
+ *    ff_layer_bufs structs and all by-value scalars are HOST data.
+ *  - Batch layout: B positive samples followed by B negative samples ("positive and negative
+ *    sets", Alg. 1 line 3).  M = 2B.  R = rows per sample: 1 for a linear layer, H*Wd for a
+ *    convolution (one row per output position, NHWC).
+ *  - Calls are asynchronous on the given CUDA stream (a cudaStream_t passed as void*; NULL =
+ *    the legacy default stream) and never synchronise.  Host-detectable errors are returned
+ *    before anything is launched.  Device-detected conditions (non-finite input, a bounded wait
+ *    that ran out) are OR-ed into a status word that ff_poll_status reads.
+ *  - The library never allocates device memory after ff_create; scratch space is the caller's
+ *    workspace (ff_set_workspace).
+ *  - Arithmetic contract: all INT8 tensors, INT32 accumulators, absmax values, S, rowmax, coef
+ *    and the updated weights have exactly one correct bit pattern (each FP32/FP64 operation is
+ *    a single IEEE round-to-nearest operation in a fixed order, no fused multiply-add); only the
+ *    scalar `loss` depends on summation order.
+ */
+#ifndef FFINT8_H
+#define FFINT8_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ff_ctx ff_ctx; /* opaque; holds device id, workspace pointer, last error text */
+
+typedef enum {
+  FF_OK = 0,
+  FF_ERR_ARG = -1,             /* NULL pointer, non-positive size, unknown enum value          */
+  FF_ERR_ALIGN = -2,           /* a device pointer is not 16-byte aligned                      */
+  FF_ERR_WORKSPACE = -3,       /* workspace missing or smaller than ff_workspace_bytes says    */
+  FF_ERR_NONFINITE = -4,       /* an input tensor held Inf/NaN (device-detected)               */
+  FF_ERR_RANGE = -5,           /* worst-case INT32 accumulator or 32-bit index range exceeded  */
+  FF_ERR_DEVICE_TIMEOUT = -6,  /* a bounded in-kernel wait ran out (device-detected)           */
+  FF_ERR_CUDA = -7,            /* a CUDA runtime / driver call failed                          */
+  FF_ERR_UNSUPPORTED_ARCH = -8 /* the device is not compute capability 10.x                    */
+} ff_status;
+
+enum { FF_LINEAR = 0, FF_CONV3X3 = 1 };                  /* ff_layer_desc.kind      */
+enum { FF_ROUND_NEAREST_EVEN = 0, FF_ROUND_STOCHASTIC = 1 }; /* rounding modes (Sec. IV-B) */
+enum { FF_GEMM_AUTO = 0, FF_GEMM_SIMT = 1, FF_GEMM_TENSOR = 2 }; /* ff_set_gemm_path       */
+
+/* indices into ff_layer_bufs.absmax (per-tensor SUQ ranges a = max|x|, Sec. IV; s = a/127) */
+enum {
+  FF_A_X_POS = 0, FF_A_X_NEG = 1, /* layer input, positive / negative set                    */
+  FF_A_W = 2,                     /* weights                                                 */
+  FF_A_DH_POS = 3, FF_A_DH_NEG = 4, /* output gradient g^Y                                   */
+  FF_A_XNEXT_POS = 5, FF_A_XNEXT_NEG = 6, /* the normalised output (next layer's input)      */
+  FF_ABSMAX_LEN = 8
+};
+
+/* One FF layer (host struct).  linear: X[M,K] -> Y[M,N], W[N,K].
+ * conv3x3 (stride 1, zero padding 1, NHWC): X[M,H,Wd,Cin] -> Y[M,H,Wd,N], W[N,3,3,Cin] stored as
+ * [N,K] with K = 9*Cin and k = (r*3+s)*Cin + ci. */
+typedef struct {
+  int32_t kind;
+  int32_t K, N;
+  int32_t H, Wd, Cin;   /* conv only; 1,1,0 for linear                                        */
+  int32_t index;        /* position of the layer in the network (keys the rounding hash)      */
+  int32_t round_x, round_w, round_dh; /* rounding of A, W, g^Y (paper: stochastic for A)      */
+  float theta;          /* threshold of Eq. 1 / Eq. 2                                         */
+  float lr;             /* SGD step size of the update (Alg. 1 line 9)                        */
+  float tau, eps;       /* length normalisation of the output: x = y*tau/(sqrt(G)+eps), eps>0 */
+  uint64_t seed;        /* keys the stochastic-rounding hash                                  */
+} ff_layer_desc;
+
+/* Device buffers of one layer (host struct of device pointers; caller-owned). */
+typedef struct {
+  float* W;          /* [N,K] FP32 master weights; ff_layer_update rewrites them in place      */
+  const float* X;    /* [M*R,Kin] FP32 input, already length-normalised (Kin = K, conv: Cin).   */
+                     /* In ff_train_step it may be NULL for layers > 0: the layer then takes   */
+                     /* the previous layer's normalised output without materialising it.      */
+  float* Y;          /* [M*R,N] FP32 out: max(0, float(acc)*s_x*s_w)                           */
+  float* G;          /* [M] FP32 out: goodness per sample                                      */
+  float* Xnext;      /* [M*R,N] FP32 out, nullable: Y*tau/(sqrt(G)+eps)                         */
+  int8_t* Xq;        /* [M*R,Kin] INT8 out                                                     */
+  int8_t* Wq;        /* [N,K] INT8 out                                                         */
+  int8_t* dHq;       /* [M*R,N] INT8 out (ff_layer_loss_grad)                                  */
+  float* absmax;     /* [FF_ABSMAX_LEN] FP32 out, see FF_A_*                                   */
+  uint64_t* S;       /* [M] out: exact integer sum over the sample of relu(acc)^2              */
+  int32_t* rowmax;   /* [M] out: max over the sample of relu(acc)                              */
+  float* coef;       /* [M] out: per-sample dL_new/dG / M  (g^Y = 2*coef*Y)                    */
+  float* loss;       /* [1] out: L_new averaged over the M samples (Eq. 3)                     */
+  int32_t* acc_dump; /* [M*R,N] INT32 out, nullable: the forward accumulators                  */
+  int32_t* accW_dump;/* [2,N,K] INT32 out, nullable: g^W accumulators of the two sets          */
+} ff_layer_bufs;
+
+/* Create / destroy a context for CUDA device `device` (must be compute capability 10.x).
+ * ff_create makes the device current and allocates nothing on it. */
+ff_status ff_create(ff_ctx** out, int device);
+ff_status ff_destroy(ff_ctx* ctx);
+
+/* Scratch bytes needed for n_layers layers at batch B (host computation only). */
+ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, size_t* out_bytes);
+/* Hand the context a caller-owned device buffer (256-byte aligned) of at least that size.  The
+ * first call on a stream after this zeroes the status word. */
+ff_status ff_set_workspace(ff_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* Choose the contraction kernels: AUTO picks the tcgen05 tensor-core kernels whenever the shape
+ * allows and the SIMT kernels otherwise; SIMT / TENSOR force one (TENSOR fails with FF_ERR_ARG on
+ * shapes it cannot take).  Both produce identical bits. */
+ff_status ff_set_gemm_path(ff_ctx* ctx, int path);
+
+/* Forward of one layer (Sec. IV-B: quantise A and W, INT8 MAC with INT32 accumulation; Sec. III /
+ * Alg. 1 line 6: goodness).  Reads X, W.  Writes Xq, Wq, absmax[X,W,XNEXT], Y, S, rowmax, G,
+ * Xnext (if non-NULL), acc_dump (if non-NULL).  `step` keys the stochastic rounding. */
+ff_status ff_layer_forward(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs,
+                           int B, uint64_t step, void* cuda_stream);
+
+/* Loss and output gradient of one layer (Eq. 1, Eq. 2; look-ahead Eq. 3, Eq. 4; Sec. IV-B "the
+ * gradient g^Y is computed and quantized into INT8").  G_later[j] (device, [M] each) and
+ * theta_later[j] (host) are the goodness and thresholds of the n_later subsequent layers; with
+ * n_later = 0 or lambda = 0 this is the vanilla FF loss.  Reads G, Y, rowmax, absmax[X,W].
+ * Writes loss, coef, absmax[DH], dHq. */
+ff_status ff_layer_loss_grad(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs,
+                             int B, const float* const* G_later, const float* theta_later,
+                             int n_later, float lambda, uint64_t step, void* cuda_stream);
+
+/* Weight gradient and update of one layer (Sec. IV-B: g^W as an INT8 MAC, "only gradients of
+ * weights are computed and updated"; Alg. 1 line 9).  Reads dHq, Xq, absmax, W.  Writes W
+ * (W - lr*(float(accP)*cP + float(accN)*cN)) and accW_dump (if non-NULL). */
+ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs,
+                          int B, void* cuda_stream);
+
+/* Body of Algorithm 1's epoch loop for n_layers layers: one INT8 forward through all layers with
+ * the pre-update weights (line 5), goodness of every layer (line 6), then per layer the loss with
+ * look-ahead weight `lambda` (line 8, Eq. 3) and the INT8 gradient + update (line 9).  Layer 0
+ * reads bufs[0].X; layer l > 0 reads bufs[l].X if non-NULL, else layer l-1's normalised output.
+ * With n_layers = 1 and lambda = 0 it equals forward -> loss_grad -> update. */
+ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs,
+                        int n_layers, int B, float lambda, uint64_t step, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, reads the device status word and clears it.  Returns FF_OK,
+ * FF_ERR_NONFINITE, FF_ERR_DEVICE_TIMEOUT or FF_ERR_CUDA. */
+ff_status ff_poll_status(ff_ctx* ctx, void* cuda_stream);
+
+/* Text of the last error returned for this context (host string, valid until the next call). */
+const char* ff_last_error(const ff_ctx* ctx);
+
+/* Number of kernels the library has launched through this context so far (host counter). */
+uint64_t ff_launch_count(const ff_ctx* ctx);
+
+/* Stand-alone INT8 contraction used by the unit tests and the kernel benchmark (Sec. IV-B,
+ * "integer matrix multiplication with INT8 inputs and INT32 accumulation"):
+ *   trans = 0: C[m,n] = sum_k A[m,k]*B[n,k]   A [M,K], B [N,K]  (forward orientation)
+ *   trans = 1: C[m,n] = sum_k A[k,m]*B[k,n]   A [K,M], B [K,N]  (weight-gradient orientation)
+ * A, B device INT8 row-major; C device INT32 [M,N] row-major. */
+ff_status ff_int8_gemm(ff_ctx* ctx, const int8_t* A, const int8_t* B, int32_t* C, int M, int N,
+                       int K, int trans, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FFINT8_H */

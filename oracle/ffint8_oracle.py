@@ -112,16 +112,20 @@ def rounding_key(seed: int, role: int, layer: int, step: int):
 
 
 def rounding_uniform(idx: np.ndarray, k0: int, k1: int) -> np.ndarray:
-    """u in [0,1) with 24 random bits for each linear element index (counter-based, so the
-    value does not depend on how the tensor is tiled or which thread handles the element)."""
-    h = idx.astype(np.uint32) ^ np.uint32(k0)
+    """u in [0,1) with 16 random bits for each linear element index (counter-based, so the
+    value does not depend on how the tensor is tiled or which thread handles the element).
+    One 32-bit hash serves the element pair (2j, 2j+1): low half for the even index, high half
+    for the odd one."""
+    idx = idx.astype(np.uint64)
+    h = (idx >> np.uint64(1)).astype(np.uint32) ^ np.uint32(k0)
     h = h * np.uint32(0x9E3779B1)
     h = h ^ (h >> np.uint32(15))
     h = (h + np.uint32(k1)) * np.uint32(0x85EBCA6B)
     h = h ^ (h >> np.uint32(13))
     h = h * np.uint32(0xC2B2AE35)
     h = h ^ (h >> np.uint32(16))
-    return (h >> np.uint32(8)).astype(F32) * F32(2.0 ** -24)
+    half = np.where((idx & np.uint64(1)) == 0, h & np.uint32(0xFFFF), h >> np.uint32(16))
+    return half.astype(F32) * F32(2.0 ** -16)
 
 
 def quantize(x: np.ndarray, a: np.float32, mode: int, key=None, idx0: int = 0,

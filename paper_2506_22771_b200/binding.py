@@ -1,0 +1,207 @@
+"""Thin ctypes binding of libffint8.so: same names as the C ABI (include/ffint8.h), argument
+marshalling only.  PyTorch supplies device memory and streams; every step of the path runs in
+the library's CUDA kernels.  There is no CPU fallback: a missing library raises."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+from . import build as _build
+
+FF_OK = 0
+FF_ERR_ARG, FF_ERR_ALIGN, FF_ERR_WORKSPACE, FF_ERR_NONFINITE = -1, -2, -3, -4
+FF_ERR_RANGE, FF_ERR_DEVICE_TIMEOUT, FF_ERR_CUDA, FF_ERR_UNSUPPORTED_ARCH = -5, -6, -7, -8
+FF_LINEAR, FF_CONV3X3 = 0, 1
+FF_ROUND_NEAREST_EVEN, FF_ROUND_STOCHASTIC = 0, 1
+FF_GEMM_AUTO, FF_GEMM_SIMT, FF_GEMM_TENSOR = 0, 1, 2
+FF_A_X_POS, FF_A_X_NEG, FF_A_W, FF_A_DH_POS, FF_A_DH_NEG, FF_A_XNEXT_POS, FF_A_XNEXT_NEG = range(7)
+FF_ABSMAX_LEN = 8
+
+EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", "ff_set_gemm_path",
+           "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step",
+           "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm"]
+
+
+class ff_layer_desc(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("K", C.c_int32), ("N", C.c_int32), ("H", C.c_int32),
+                ("Wd", C.c_int32), ("Cin", C.c_int32), ("index", C.c_int32),
+                ("round_x", C.c_int32), ("round_w", C.c_int32), ("round_dh", C.c_int32),
+                ("theta", C.c_float), ("lr", C.c_float), ("tau", C.c_float), ("eps", C.c_float),
+                ("seed", C.c_uint64)]
+
+
+class ff_layer_bufs(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in
+                ("W", "X", "Y", "G", "Xnext", "Xq", "Wq", "dHq", "absmax", "S", "rowmax", "coef",
+                 "loss", "acc_dump", "accW_dump")]
+
+
+class FFError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"libffint8 error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB_PATH
+
+
+def load(build_if_missing: bool = True):
+    """Load libffint8.so (building it first when the file is absent and nvcc is there)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_build.LIB_PATH):
+        if not build_if_missing:
+            raise FileNotFoundError(_build.LIB_PATH)
+        _build.build()
+    lib = C.CDLL(_build.LIB_PATH)
+    vp, i32, u64, f32 = C.c_void_p, C.c_int, C.c_uint64, C.c_float
+    lib.ff_create.argtypes = [C.POINTER(vp), i32]
+    lib.ff_destroy.argtypes = [vp]
+    lib.ff_workspace_bytes.argtypes = [C.POINTER(ff_layer_desc), i32, i32, C.POINTER(C.c_size_t)]
+    lib.ff_set_workspace.argtypes = [vp, vp, C.c_size_t]
+    lib.ff_set_gemm_path.argtypes = [vp, i32]
+    lib.ff_layer_forward.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, u64, vp]
+    lib.ff_layer_loss_grad.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32,
+                                       C.POINTER(vp), C.POINTER(f32), i32, f32, u64, vp]
+    lib.ff_layer_update.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, vp]
+    lib.ff_train_step.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, i32, f32, u64, vp]
+    lib.ff_poll_status.argtypes = [vp, vp]
+    lib.ff_last_error.argtypes = [vp]
+    lib.ff_last_error.restype = C.c_char_p
+    lib.ff_launch_count.argtypes = [vp]
+    lib.ff_launch_count.restype = u64
+    lib.ff_int8_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    for name in EXPORTS:
+        if name not in ("ff_last_error", "ff_launch_count"):
+            getattr(lib, name).restype = i32
+    _lib = lib
+    return lib
+
+
+def _check(ctx, code: int):
+    if code != FF_OK:
+        msg = load().ff_last_error(ctx).decode() if ctx else ""
+        raise FFError(code, msg)
+
+
+def ff_create(device: int = 0):
+    ctx = C.c_void_p()
+    code = load().ff_create(C.byref(ctx), device)
+    if code != FF_OK:
+        raise FFError(code, "ff_create failed")
+    return ctx
+
+
+def ff_destroy(ctx):
+    load().ff_destroy(ctx)
+
+
+def ff_workspace_bytes(descs: Sequence[ff_layer_desc], B: int) -> int:
+    arr = (ff_layer_desc * len(descs))(*descs)
+    out = C.c_size_t()
+    _check(None, load().ff_workspace_bytes(arr, len(descs), B, C.byref(out)))
+    return out.value
+
+
+def ff_set_workspace(ctx, dev_ptr: int, nbytes: int):
+    _check(ctx, load().ff_set_workspace(ctx, dev_ptr, nbytes))
+
+
+def ff_set_gemm_path(ctx, path: int):
+    _check(ctx, load().ff_set_gemm_path(ctx, path))
+
+
+def ff_layer_forward(ctx, desc, bufs, B: int, step: int, stream: int = 0):
+    _check(ctx, load().ff_layer_forward(ctx, C.byref(desc), C.byref(bufs), B, step, stream))
+
+
+def ff_layer_loss_grad(ctx, desc, bufs, B: int, G_later: Sequence[int], theta_later: Sequence[float],
+                       lam: float, step: int, stream: int = 0):
+    n = len(G_later)
+    gp = (C.c_void_p * max(n, 1))(*G_later)
+    th = (C.c_float * max(n, 1))(*theta_later)
+    _check(ctx, load().ff_layer_loss_grad(ctx, C.byref(desc), C.byref(bufs), B, gp, th, n, lam, step, stream))
+
+
+def ff_layer_update(ctx, desc, bufs, B: int, stream: int = 0):
+    _check(ctx, load().ff_layer_update(ctx, C.byref(desc), C.byref(bufs), B, stream))
+
+
+def ff_train_step(ctx, descs_arr, bufs_arr, n_layers: int, B: int, lam: float, step: int, stream: int = 0):
+    """descs_arr / bufs_arr: ctypes arrays (ff_layer_desc * n), (ff_layer_bufs * n)."""
+    _check(ctx, load().ff_train_step(ctx, descs_arr, bufs_arr, n_layers, B, lam, step, stream))
+
+
+def ff_poll_status(ctx, stream: int = 0):
+    _check(ctx, load().ff_poll_status(ctx, stream))
+
+
+def ff_launch_count(ctx) -> int:
+    return int(load().ff_launch_count(ctx))
+
+
+def ff_int8_gemm(ctx, A: int, B: int, Cptr: int, M: int, N: int, K: int, trans: int, stream: int = 0):
+    _check(ctx, load().ff_int8_gemm(ctx, A, B, Cptr, M, N, K, trans, stream))
+
+
+# --------------------------------------------------------------------------------------------
+# Convenience: device buffers for a stack of layers (torch is used for allocation only)
+# --------------------------------------------------------------------------------------------
+def make_desc(cfg, index: int, seed: int, round_x=FF_ROUND_STOCHASTIC, round_w=FF_ROUND_NEAREST_EVEN,
+              round_dh=FF_ROUND_STOCHASTIC) -> ff_layer_desc:
+    """cfg: an object with kind, K, N, H, Wd, Cin, theta, lr, tau, eps (e.g. synth.LayerCfg)."""
+    return ff_layer_desc(cfg.kind, cfg.K, cfg.N, cfg.H, cfg.Wd, cfg.Cin, index, round_x, round_w, round_dh,
+                         cfg.theta, cfg.lr, cfg.tau, cfg.eps, seed)
+
+
+class LayerBuffers:
+    """Torch-allocated device tensors of one layer plus the ff_layer_bufs struct pointing at them."""
+
+    def __init__(self, desc: ff_layer_desc, B: int, device, dumps: bool = False, xnext: bool = True,
+                 own_x: bool = True):
+        import torch
+        R = desc.H * desc.Wd if desc.kind == FF_CONV3X3 else 1
+        kin = desc.Cin if desc.kind == FF_CONV3X3 else desc.K
+        rows = 2 * B * R
+        z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)
+        self.W = z((desc.N, desc.K), torch.float32)
+        self.X = z((rows, kin), torch.float32) if own_x else None
+        self.Y = z((rows, desc.N), torch.float32)
+        self.G = z((2 * B,), torch.float32)
+        self.Xnext = z((rows, desc.N), torch.float32) if xnext else None
+        self.Xq = z((rows, kin), torch.int8)
+        self.Wq = z((desc.N, desc.K), torch.int8)
+        self.dHq = z((rows, desc.N), torch.int8)
+        self.absmax = z((FF_ABSMAX_LEN,), torch.float32)
+        self.S = z((2 * B,), torch.int64)
+        self.rowmax = z((2 * B,), torch.int32)
+        self.coef = z((2 * B,), torch.float32)
+        self.loss = z((4,), torch.float32)
+        self.acc_dump = z((rows, desc.N), torch.int32) if dumps else None
+        self.accW_dump = z((2, desc.N, desc.K), torch.int32) if dumps else None
+        p = lambda t: t.data_ptr() if t is not None else None
+        self.struct = ff_layer_bufs(p(self.W), p(self.X), p(self.Y), p(self.G), p(self.Xnext), p(self.Xq),
+                                    p(self.Wq), p(self.dHq), p(self.absmax), p(self.S), p(self.rowmax),
+                                    p(self.coef), p(self.loss), p(self.acc_dump), p(self.accW_dump))
+
+
+class Context:
+    """ff_ctx plus a torch-allocated workspace."""
+
+    def __init__(self, descs: Sequence[ff_layer_desc], B: int, device_index: int = 0):
+        import torch
+        self.ctx = ff_create(device_index)
+        n = ff_workspace_bytes(descs, B)
+        self.workspace = torch.zeros(max(n, 256), dtype=torch.uint8, device=f"cuda:{device_index}")
+        ff_set_workspace(self.ctx, self.workspace.data_ptr(), self.workspace.numel())
+
+    def close(self):
+        if self.ctx is not None:
+            ff_destroy(self.ctx)
+            self.ctx = None

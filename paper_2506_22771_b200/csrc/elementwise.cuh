@@ -1,0 +1,306 @@
+// Memory-bound passes of the FF-INT8 step: absmax reduction, SUQ quantisation (Sec. IV) with
+// nearest / stochastic rounding (Sec. IV-B), goodness finalisation and length normalisation
+// (Sec. III; Alg. 1 line 6), the loss / look-ahead coefficient kernel (Eq. 1-4) and the output
+// gradient quantiser ("g^Y is computed and quantized into INT8", Sec. IV-B).
+// All are coalesced 128-bit-load kernels with warp-shuffle reductions; grids are sized in
+// multiples of the SM count by the host code.
+#pragma once
+#include "common.cuh"
+
+namespace ffi8 {
+
+constexpr int EW_THREADS = 256;
+
+__device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) { return __reduce_max_sync(0xffffffffu, v); }
+
+// Block-wide max of a u32; result valid in thread 0.
+__device__ __forceinline__ uint32_t block_max_u32(uint32_t v) {
+  __shared__ uint32_t sm[32];
+  v = warp_max_u32(v);
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) sm[w] = v;
+  __syncthreads();
+  if (w == 0) {
+    v = (lane < (int)((blockDim.x + 31) >> 5)) ? sm[lane] : 0u;
+    v = warp_max_u32(v);
+  }
+  return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// absmax over `passes` consecutive slices of n_per_pass floats each; out[p] must be zero before.
+// |x| compared as bit patterns (monotone for finite floats); Inf/NaN raise ST_NONFINITE.
+// grid = (blocks, passes)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restrict__ x, size_t n_per_pass,
+                                                            float* __restrict__ out, uint32_t* __restrict__ status) {
+  const float* xp = x + (size_t)blockIdx.y * n_per_pass;
+  uint32_t m = 0;
+  const bool vec = ((n_per_pass & 3) == 0) && ((((uintptr_t)xp) & 15) == 0);
+  size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  size_t stride = (size_t)gridDim.x * blockDim.x;
+  if (vec) {
+    const uint4* x4 = reinterpret_cast<const uint4*>(xp);
+    size_t n4 = n_per_pass >> 2;
+    for (size_t i = tid; i < n4; i += stride) {
+      uint4 v = __ldg(x4 + i);
+      m = max(m, max(max(v.x & 0x7fffffffu, v.y & 0x7fffffffu), max(v.z & 0x7fffffffu, v.w & 0x7fffffffu)));
+    }
+  } else {
+    for (size_t i = tid; i < n_per_pass; i += stride) m = max(m, __float_as_uint(xp[i]) & 0x7fffffffu);
+  }
+  m = block_max_u32(m);
+  if (threadIdx.x == 0) {
+    if (m >= 0x7f800000u) atomicOr(status, ST_NONFINITE);
+    if (m) atomicMax(reinterpret_cast<uint32_t*>(out) + blockIdx.y, m);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// q = clip(round(x * 127/a_p)) for `passes` slices, a_p read from device memory (absmax[p]).
+// Linear element index (over the whole tensor) keys the stochastic rounding.
+// grid = (blocks, passes)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __restrict__ x, int8_t* __restrict__ q,
+                                                              size_t n_per_pass, const float* __restrict__ a,
+                                                              int mode, RoundKey key) {
+  const size_t base = (size_t)blockIdx.y * n_per_pass;
+  const float* xp = x + base;
+  int8_t* qp = q + base;
+  const float inv = inv_of(a[blockIdx.y]);
+  const bool vec = ((n_per_pass & 3) == 0) && ((((uintptr_t)xp) & 15) == 0) && ((((uintptr_t)qp) & 3) == 0);
+  size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  size_t stride = (size_t)gridDim.x * blockDim.x;
+  if (vec) {
+    const float4* x4 = reinterpret_cast<const float4*>(xp);
+    uint32_t* q4 = reinterpret_cast<uint32_t*>(qp);
+    size_t n4 = n_per_pass >> 2;
+    for (size_t i = tid; i < n4; i += stride) {
+      float4 v = __ldg(x4 + i);
+      uint32_t idx = (uint32_t)(base + (i << 2));
+      int q0, q1, q2, q3;
+      quant_pair(v.x, v.y, inv, mode, idx, key, q0, q1);
+      quant_pair(v.z, v.w, inv, mode, idx + 2, key, q2, q3);
+      q4[i] = pack4(q0, q1, q2, q3);
+    }
+  } else {
+    for (size_t i = tid; i < n_per_pass; i += stride)
+      qp[i] = (int8_t)quant_one(xp[i], inv, mode, (uint32_t)(base + i), key);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Goodness per sample from the exact integer sum: G = float(double(S) * c*c), c = s_x[p]*s_w.
+// Also the per-pass absmax of the normalised output via the per-sample max of relu(acc):
+// max_n y*r = (float(rowmax)*c)*r because each rounded multiply by a fixed non-negative factor is
+// monotone.  a_next (and a_next2, if non-NULL) receive it by atomicMax; both must be zero before.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) finalize_goodness_kernel(
+    const unsigned long long* __restrict__ S, const int32_t* __restrict__ rowmax, const float* __restrict__ absmax,
+    int B, float tau, float eps, float* __restrict__ G, float* __restrict__ a_next, float* __restrict__ a_next2) {
+  const int p = blockIdx.y;
+  const float c = __fmul_rn(scale_of(absmax[p]), scale_of(absmax[2]));
+  const double c2 = __dmul_rn((double)c, (double)c);
+  uint32_t mx = 0;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < B; i += gridDim.x * blockDim.x) {
+    int m = p * B + i;
+    float g = __double2float_rn(__dmul_rn(__ull2double_rn(S[m]), c2));
+    G[m] = g;
+    float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(g), eps));
+    float xm = __fmul_rn(__fmul_rn(__int2float_rn(rowmax[m]), c), r);
+    mx = max(mx, __float_as_uint(xm));
+  }
+  mx = block_max_u32(mx);
+  if (threadIdx.x == 0 && mx) {
+    atomicMax(reinterpret_cast<uint32_t*>(a_next) + p, mx);
+    if (a_next2) atomicMax(reinterpret_cast<uint32_t*>(a_next2) + p, mx);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Length normalisation x = y * tau/(sqrt(G)+eps) per sample, written as FP32 (xnext, nullable)
+// and / or quantised straight to the next layer's INT8 input (xq, nullable) with per-pass range
+// a[p].  per_sample = R*N elements per sample; per_pass = B*per_sample.   grid = (blocks, 2)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __restrict__ Y, const float* __restrict__ G,
+                                                               float tau, float eps, size_t per_sample,
+                                                               size_t per_pass, float* __restrict__ xnext,
+                                                               int8_t* __restrict__ xq, const float* __restrict__ a,
+                                                               int mode, RoundKey key) {
+  const size_t base = (size_t)blockIdx.y * per_pass;
+  const float inv = xq ? inv_of(a[blockIdx.y]) : 0.0f;
+  size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  size_t stride = (size_t)gridDim.x * blockDim.x;
+  const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) &&
+                   (!xnext || (((uintptr_t)xnext) & 15) == 0) && (!xq || (((uintptr_t)xq) & 3) == 0);
+  if (vec) {
+    size_t n4 = per_pass >> 2;
+    for (size_t i = tid; i < n4; i += stride) {
+      size_t e = base + (i << 2);
+      float g = __ldg(G + (uint32_t)e / (uint32_t)per_sample);
+      float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(g), eps));
+      float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
+      v.x = __fmul_rn(v.x, r);
+      v.y = __fmul_rn(v.y, r);
+      v.z = __fmul_rn(v.z, r);
+      v.w = __fmul_rn(v.w, r);
+      if (xnext) *reinterpret_cast<float4*>(xnext + e) = v;
+      if (xq) {
+        int q0, q1, q2, q3;
+        quant_pair(v.x, v.y, inv, mode, (uint32_t)e, key, q0, q1);
+        quant_pair(v.z, v.w, inv, mode, (uint32_t)e + 2, key, q2, q3);
+        *reinterpret_cast<uint32_t*>(xq + e) = pack4(q0, q1, q2, q3);
+      }
+    }
+  } else {
+    for (size_t i = tid; i < per_pass; i += stride) {
+      size_t e = base + i;
+      float g = G[(uint32_t)e / (uint32_t)per_sample];
+      float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(g), eps));
+      float v = __fmul_rn(Y[e], r);
+      if (xnext) xnext[e] = v;
+      if (xq) xq[e] = (int8_t)quant_one(v, inv, mode, (uint32_t)e, key);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// e^v for v <= 0 in FP64 by a fixed recipe so that every implementation agrees bit for bit:
+// clamp at -700, n = rint(v*log2e), r = (v - n*LN2_HI) - n*LN2_LO, degree-13 Taylor polynomial by
+// Horner with separately rounded multiply and add, exact scaling by 2^n.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ double exp_nonpos(double v) {
+  constexpr double LOG2E = 1.4426950408889634;
+  constexpr double LN2_HI = 6.93147180369123816490e-01;
+  constexpr double LN2_LO = 1.90821492927058770002e-10;
+  constexpr double C[14] = {1.0 / 1.0,         1.0 / 1.0,          1.0 / 2.0,          1.0 / 6.0,         1.0 / 24.0,
+                            1.0 / 120.0,       1.0 / 720.0,        1.0 / 5040.0,       1.0 / 40320.0,     1.0 / 362880.0,
+                            1.0 / 3628800.0,   1.0 / 39916800.0,   1.0 / 479001600.0,  1.0 / 6227020800.0};
+  v = fmax(v, -700.0);
+  double n = rint(__dmul_rn(v, LOG2E));
+  double r = __dsub_rn(__dsub_rn(v, __dmul_rn(n, LN2_HI)), __dmul_rn(n, LN2_LO));
+  double p = C[13];
+#pragma unroll
+  for (int k = 12; k >= 0; --k) p = __dadd_rn(__dmul_rn(p, r), C[k]);
+  return scalbn(p, (int)n);
+}
+// sigma(x) from e = e^{-|x|}: x >= 0 -> 1/(1+e), else e/(1+e).
+__device__ __forceinline__ double sigmoid_spec(double x) {
+  double e = exp_nonpos(-fabs(x));
+  double d = __dadd_rn(1.0, e);
+  return x >= 0.0 ? __ddiv_rn(1.0, d) : __ddiv_rn(e, d);
+}
+
+constexpr int FF_MAX_LATER = 31;
+struct LaterLayers {
+  const float* G[FF_MAX_LATER];
+  float theta[FF_MAX_LATER];
+  int n;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Loss (Eq. 1, Eq. 2), look-ahead loss (Eq. 3) and the per-sample coefficient of Eq. 4 under the
+// scalar-coefficient reading: coef_m = (g'_l,m + lambda * sum_{j>l} g'_j,m)/M with g' = dL/dG.
+// Also the per-pass absmax of dH = 2*coef*y via the per-sample max of relu(acc).
+// One block (M is at most a few 10^4 samples); fixed-order tree reduction for the loss.
+// ---------------------------------------------------------------------------------------------
+constexpr int LOSS_THREADS = 1024;
+__global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __restrict__ G, float theta, LaterLayers later,
+                                                                 float lambda, int B, const int32_t* __restrict__ rowmax,
+                                                                 float* __restrict__ absmax, float* __restrict__ coef,
+                                                                 float* __restrict__ loss) {
+  __shared__ double red[LOSS_THREADS / 32];
+  __shared__ uint32_t redmax[2][LOSS_THREADS / 32];
+  const int M = 2 * B;
+  const double lam = (double)lambda;
+  const double inv_m = __ddiv_rn(1.0, (double)M);
+  const float s_w = scale_of(absmax[2]);
+  const float cpass[2] = {__fmul_rn(scale_of(absmax[0]), s_w), __fmul_rn(scale_of(absmax[1]), s_w)};
+  double lsum = 0.0;
+  uint32_t amax[2] = {0u, 0u};
+  for (int m = threadIdx.x; m < M; m += LOSS_THREADS) {
+    const int p = m >= B;
+    const double sign = p ? 1.0 : -1.0;
+    double arg = __dmul_rn(sign, __dsub_rn((double)G[m], (double)theta));
+    double g0 = __dmul_rn(sign, sigmoid_spec(arg));
+    double L0 = fmax(arg, 0.0) + log1p(exp(-fabs(arg)));
+    double gsum = 0.0, Lsum = 0.0;
+    for (int j = 0; j < later.n; ++j) {
+      double aj = __dmul_rn(sign, __dsub_rn((double)later.G[j][m], (double)later.theta[j]));
+      gsum = __dadd_rn(gsum, __dmul_rn(sign, sigmoid_spec(aj)));
+      Lsum += fmax(aj, 0.0) + log1p(exp(-fabs(aj)));
+    }
+    float cf = __double2float_rn(__dmul_rn(__dadd_rn(g0, __dmul_rn(lam, gsum)), inv_m));
+    coef[m] = cf;
+    lsum += L0 + lam * Lsum;
+    float k2 = __fmul_rn(2.0f, cf);
+    float d = fabsf(__fmul_rn(k2, __fmul_rn(__int2float_rn(rowmax[m]), cpass[p])));
+    amax[p] = max(amax[p], __float_as_uint(d));
+  }
+  // block reductions (fixed order)
+  for (int o = 16; o > 0; o >>= 1) lsum += __shfl_down_sync(0xffffffffu, lsum, o);
+  amax[0] = warp_max_u32(amax[0]);
+  amax[1] = warp_max_u32(amax[1]);
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) {
+    red[w] = lsum;
+    redmax[0][w] = amax[0];
+    redmax[1][w] = amax[1];
+  }
+  __syncthreads();
+  if (w == 0) {
+    double v = red[lane];
+    uint32_t a0 = redmax[0][lane], a1 = redmax[1][lane];
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    a0 = warp_max_u32(a0);
+    a1 = warp_max_u32(a1);
+    if (lane == 0) {
+      loss[0] = (float)(v * inv_m);
+      absmax[3] = __uint_as_float(a0);
+      absmax[4] = __uint_as_float(a1);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// dHq = clip(round((2*coef_m * y) * 127/a_dh[p])).  grid = (blocks, 2)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) dh_quantize_kernel(const float* __restrict__ Y, const float* __restrict__ coef,
+                                                                 const float* __restrict__ absmax, size_t per_sample,
+                                                                 size_t per_pass, int8_t* __restrict__ dHq, int mode,
+                                                                 RoundKey key) {
+  const size_t base = (size_t)blockIdx.y * per_pass;
+  const float inv = inv_of(absmax[3 + blockIdx.y]);
+  size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  size_t stride = (size_t)gridDim.x * blockDim.x;
+  const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)dHq) & 3) == 0);
+  if (vec) {
+    size_t n4 = per_pass >> 2;
+    for (size_t i = tid; i < n4; i += stride) {
+      size_t e = base + (i << 2);
+      float k2 = __fmul_rn(2.0f, __ldg(coef + (uint32_t)e / (uint32_t)per_sample));
+      float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
+      int q0, q1, q2, q3;
+      quant_pair(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, mode, (uint32_t)e, key, q0, q1);
+      quant_pair(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, mode, (uint32_t)e + 2, key, q2, q3);
+      *reinterpret_cast<uint32_t*>(dHq + e) = pack4(q0, q1, q2, q3);
+    }
+  } else {
+    for (size_t i = tid; i < per_pass; i += stride) {
+      size_t e = base + i;
+      float k2 = __fmul_rn(2.0f, coef[(uint32_t)e / (uint32_t)per_sample]);
+      dHq[e] = (int8_t)quant_one(__fmul_rn(k2, Y[e]), inv, mode, (uint32_t)e, key);
+    }
+  }
+}
+
+// Zero the per-sample integer accumulators of the forward epilogue (S: u64 sum, rowmax: i32 max).
+__global__ void __launch_bounds__(EW_THREADS) zero_sample_stats_kernel(unsigned long long* S, int32_t* rowmax, int M) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < M) {
+    S[i] = 0ull;
+    rowmax[i] = 0;
+  }
+}
+
+}  // namespace ffi8

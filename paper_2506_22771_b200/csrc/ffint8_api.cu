@@ -1,0 +1,412 @@
+// C ABI of libffint8 (declared in include/ffint8.h): host-side validation, launch sequencing of
+// the per-layer FF-INT8 step (Sec. IV-B, Fig. 4) and of Algorithm 1's epoch body.
+#include "../../include/ffint8.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+
+using namespace ffi8;
+
+struct ff_ctx {
+  int device = 0;
+  int sm_count = 148;
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  bool status_zeroed = false;
+  int gemm_path = FF_GEMM_AUTO;
+  uint64_t launches = 0;
+  TcState tc;
+  char err[512] = {0};
+};
+
+namespace {
+
+constexpr size_t WS_STATUS_BYTES = 256;  // status word lives at the start of the workspace
+
+ff_status fail(ff_ctx* ctx, ff_status st, const char* fmt, const char* a = "", long long b = 0) {
+  if (ctx) snprintf(ctx->err, sizeof(ctx->err), fmt, a, b);
+  return st;
+}
+
+#define FF_CUDA(ctx, call)                                                                  \
+  do {                                                                                      \
+    cudaError_t e__ = (call);                                                               \
+    if (e__ != cudaSuccess) return fail(ctx, FF_ERR_CUDA, "%s (line %lld)", cudaGetErrorString(e__), __LINE__); \
+  } while (0)
+
+#define FF_LAUNCH_CHECK(ctx)                                                                \
+  do {                                                                                      \
+    (ctx)->launches++;                                                                      \
+    cudaError_t e__ = cudaGetLastError();                                                   \
+    if (e__ != cudaSuccess) return fail(ctx, FF_ERR_CUDA, "launch: %s (line %lld)", cudaGetErrorString(e__), __LINE__); \
+  } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+inline int rows_per_sample(const ff_layer_desc& L) { return L.kind == FF_CONV3X3 ? L.H * L.Wd : 1; }
+inline int in_features(const ff_layer_desc& L) { return L.kind == FF_CONV3X3 ? L.Cin : L.K; }
+
+ff_status check_layer(ff_ctx* ctx, const ff_layer_desc* L, int B) {
+  if (!L) return fail(ctx, FF_ERR_ARG, "layer descriptor is NULL");
+  if (B <= 0) return fail(ctx, FF_ERR_ARG, "B must be positive");
+  if (L->kind != FF_LINEAR && L->kind != FF_CONV3X3) return fail(ctx, FF_ERR_ARG, "unknown layer kind");
+  if (L->K <= 0 || L->N <= 0) return fail(ctx, FF_ERR_ARG, "K and N must be positive");
+  if (L->kind == FF_CONV3X3 && (L->H <= 0 || L->Wd <= 0 || L->Cin <= 0 || L->K != 9 * L->Cin))
+    return fail(ctx, FF_ERR_ARG, "conv3x3 needs H, Wd, Cin > 0 and K = 9*Cin");
+  for (int r : {L->round_x, L->round_w, L->round_dh})
+    if (r != FF_ROUND_NEAREST_EVEN && r != FF_ROUND_STOCHASTIC) return fail(ctx, FF_ERR_ARG, "unknown rounding mode");
+  if (!(L->eps > 0.0f)) return fail(ctx, FF_ERR_ARG, "eps must be > 0");
+  const long long R = rows_per_sample(*L);
+  const long long rows = 2LL * B * R;
+  // 32-bit rounding counters and element indices
+  if (rows * L->N >= (1LL << 32) || rows * in_features(*L) >= (1LL << 32) || (long long)L->N * L->K >= (1LL << 32))
+    return fail(ctx, FF_ERR_RANGE, "tensor has 2^32 or more elements");
+  if (rows >= (1LL << 31)) return fail(ctx, FF_ERR_RANGE, "too many rows");
+  // worst-case INT32 accumulator range: 127*127*contraction length < 2^31  (Sec. IV-B: INT32 accumulation)
+  const long long lim = ((1LL << 31) - 1) / (127LL * 127LL);
+  if (L->K > lim) return fail(ctx, FF_ERR_RANGE, "forward contraction %s%lld too long for INT32", "", L->K);
+  if (L->kind == FF_LINEAR && (long long)B * R > lim)
+    return fail(ctx, FF_ERR_RANGE, "weight-gradient contraction %s%lld too long for INT32", "", (long long)B * R);
+  return FF_OK;
+}
+
+ff_status check_bufs(ff_ctx* ctx, const ff_layer_bufs* b, bool need_x) {
+  if (!b) return fail(ctx, FF_ERR_ARG, "buffer struct is NULL");
+  const void* req[] = {b->W, b->Y, b->G, b->Xq, b->Wq, b->dHq, b->absmax, b->S, b->rowmax, b->coef, b->loss};
+  for (const void* p : req)
+    if (!p) return fail(ctx, FF_ERR_ARG, "a required device pointer is NULL");
+  if (need_x && !b->X) return fail(ctx, FF_ERR_ARG, "X is NULL");
+  const void* all[] = {b->W, b->X, b->Y, b->G, b->Xnext, b->Xq, b->Wq, b->dHq, b->absmax, b->S, b->rowmax, b->coef,
+                       b->loss, b->acc_dump, b->accW_dump};
+  for (const void* p : all)
+    if (p && !aligned16(p)) return fail(ctx, FF_ERR_ALIGN, "a device pointer is not 16-byte aligned");
+  return FF_OK;
+}
+
+ff_status check_ctx(ff_ctx* ctx) {
+  if (!ctx) return FF_ERR_ARG;
+  if (!ctx->workspace) return fail(ctx, FF_ERR_WORKSPACE, "no workspace set");
+  return FF_OK;
+}
+
+inline uint32_t* status_ptr(ff_ctx* ctx) { return reinterpret_cast<uint32_t*>(ctx->workspace); }
+
+ff_status ensure_status(ff_ctx* ctx, cudaStream_t st) {
+  if (!ctx->status_zeroed) {
+    FF_CUDA(ctx, cudaMemsetAsync(ctx->workspace, 0, WS_STATUS_BYTES, st));
+    ctx->status_zeroed = true;
+  }
+  return FF_OK;
+}
+
+inline int ew_blocks(ff_ctx* ctx, size_t work_items, int per_thread = 4) {
+  size_t need = (work_items + (size_t)EW_THREADS * per_thread - 1) / ((size_t)EW_THREADS * per_thread);
+  size_t cap = (size_t)ctx->sm_count * 8;
+  size_t b = need < cap ? need : cap;
+  return (int)(b ? b : 1);
+}
+
+// ---- contraction dispatch ----------------------------------------------------------------
+template <class LA, class LB, bool TRANS, int NPASS, class Epi>
+ff_status launch_simt(ff_ctx* ctx, LA la, LB lb, int out_rows, int out_cols, int clen, Epi epi, cudaStream_t st) {
+  dim3 grid((out_cols + SG_BN - 1) / SG_BN, (out_rows + SG_BM - 1) / SG_BM);
+  gemm_simt_kernel<LA, LB, TRANS, NPASS, Epi><<<grid, SG_THREADS, 0, st>>>(la, lb, clen, epi);
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
+
+inline DenseView dense(const int8_t* p, int rows, int cols) {
+  return DenseView{p, rows, cols, (cols % 8 == 0) && ((reinterpret_cast<uintptr_t>(p) & 7) == 0)};
+}
+inline Im2colView im2col(const int8_t* p, const ff_layer_desc& L, int samples) {
+  return Im2colView{p, samples * L.H * L.Wd, 9 * L.Cin, L.H, L.Wd, L.Cin,
+                    (L.Cin % 8 == 0) && ((reinterpret_cast<uintptr_t>(p) & 7) == 0)};
+}
+
+// Forward contraction + fused epilogue.
+ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  const int R = rows_per_sample(L);
+  const int rows = 2 * B * R;
+  bool tc_ok = tc_forward_supported(L, B);
+  if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core forward");
+  if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT) {
+    ff_status s = tc_forward(ctx->tc, L, b, B, status_ptr(ctx), st);
+    if (s != FF_OK) return fail(ctx, s, "tensor-core forward launch failed: %s", ctx->tc.err);
+    ctx->launches++;
+    return FF_OK;
+  }
+  ForwardEpilogue epi{b.Y, b.acc_dump, reinterpret_cast<unsigned long long*>(b.S), b.rowmax, b.absmax, rows, L.N, B * R, R};
+  if (L.kind == FF_LINEAR)
+    return launch_simt<DenseView, DenseView, false, 1>(ctx, dense(b.Xq, rows, L.K), dense(b.Wq, L.N, L.K), rows, L.N, L.K, epi, st);
+  return launch_simt<Im2colView, DenseView, false, 1>(ctx, im2col(b.Xq, L, 2 * B), dense(b.Wq, L.N, L.K), rows, L.N, L.K, epi, st);
+}
+
+// Weight-gradient contraction + fused update.
+ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  const int R = rows_per_sample(L);
+  const int rows = 2 * B * R;
+  bool tc_ok = tc_update_supported(L, B);
+  if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core weight gradient");
+  if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT) {
+    ff_status s = tc_update(ctx->tc, L, b, B, status_ptr(ctx), st);
+    if (s != FF_OK) return fail(ctx, s, "tensor-core weight-gradient launch failed: %s", ctx->tc.err);
+    ctx->launches++;
+    return FF_OK;
+  }
+  UpdateEpilogue epi{b.W, b.accW_dump, b.absmax, L.lr, L.N, L.K};
+  if (L.kind == FF_LINEAR)
+    return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, B * R, epi, st);
+  return launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, B * R, epi, st);
+}
+
+// ---- step pieces --------------------------------------------------------------------------
+// Quantise the weights and run the forward contraction; the layer input is already in Xq and
+// its ranges in absmax[X_POS..X_NEG].
+ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint64_t step,
+                          float* a_next2, cudaStream_t st) {
+  const size_t nW = (size_t)L.N * L.K;
+  absmax_kernel<<<dim3(ew_blocks(ctx, nW / 4 + 1), 1), EW_THREADS, 0, st>>>(b.W, nW, b.absmax + FF_A_W, status_ptr(ctx));
+  FF_LAUNCH_CHECK(ctx);
+  quantize_kernel<<<dim3(ew_blocks(ctx, nW / 4 + 1), 1), EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, L.round_w,
+                                                                           make_round_key(L.seed, ROLE_W, L.index, step));
+  FF_LAUNCH_CHECK(ctx);
+  const int M = 2 * B;
+  zero_sample_stats_kernel<<<(M + EW_THREADS - 1) / EW_THREADS, EW_THREADS, 0, st>>>(
+      reinterpret_cast<unsigned long long*>(b.S), b.rowmax, M);
+  FF_LAUNCH_CHECK(ctx);
+  ff_status s = run_forward_gemm(ctx, L, b, B, st);
+  if (s != FF_OK) return s;
+  finalize_goodness_kernel<<<dim3(ew_blocks(ctx, B, 1), 2), EW_THREADS, 0, st>>>(
+      reinterpret_cast<const unsigned long long*>(b.S), b.rowmax, b.absmax, B, L.tau, L.eps, b.G, b.absmax + FF_A_XNEXT_POS,
+      a_next2);
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
+
+ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint64_t step, cudaStream_t st) {
+  const size_t per_pass = (size_t)B * rows_per_sample(L) * in_features(L);
+  absmax_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(b.X, per_pass, b.absmax + FF_A_X_POS,
+                                                                               status_ptr(ctx));
+  FF_LAUNCH_CHECK(ctx);
+  quantize_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(
+      b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, L.round_x, make_round_key(L.seed, ROLE_X, L.index, step));
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
+
+// Normalised output of layer `L` as FP32 (b.Xnext, if non-NULL) and / or as the INT8 input of the
+// next layer (xq_next, nullable; rounding keyed by the next layer).
+ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, int8_t* xq_next,
+                           const ff_layer_desc* next, uint64_t step, cudaStream_t st) {
+  if (!b.Xnext && !xq_next) return FF_OK;
+  const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
+  const size_t per_pass = per_sample * B;
+  RoundKey key = next ? make_round_key(next->seed, ROLE_X, next->index, step) : RoundKey{0, 0};
+  normalize_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(
+      b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext, xq_next, b.absmax + FF_A_XNEXT_POS,
+      next ? next->round_x : 0, key);
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
+
+ff_status loss_grad_impl(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, const float* const* G_later,
+                         const float* theta_later, int n_later, float lambda, uint64_t step, cudaStream_t st) {
+  LaterLayers later;
+  later.n = n_later;
+  for (int j = 0; j < n_later; ++j) {
+    later.G[j] = G_later[j];
+    later.theta[j] = theta_later[j];
+  }
+  loss_coef_kernel<<<1, LOSS_THREADS, 0, st>>>(b.G, L.theta, later, lambda, B, b.rowmax, b.absmax, b.coef, b.loss);
+  FF_LAUNCH_CHECK(ctx);
+  const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
+  const size_t per_pass = per_sample * B;
+  dh_quantize_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(
+      b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, L.round_dh, make_round_key(L.seed, ROLE_DH, L.index, step));
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
+
+}  // namespace
+
+// ================================================================================================
+extern "C" {
+
+ff_status ff_create(ff_ctx** out, int device) {
+  if (!out) return FF_ERR_ARG;
+  *out = nullptr;
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return FF_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return FF_ERR_CUDA;
+  if (prop.major != 10) return FF_ERR_UNSUPPORTED_ARCH;
+  if (cudaSetDevice(device) != cudaSuccess) return FF_ERR_CUDA;
+  ff_ctx* c = new (std::nothrow) ff_ctx();
+  if (!c) return FF_ERR_ARG;
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  c->tc.sm_count = prop.multiProcessorCount;
+  *out = c;
+  return FF_OK;
+}
+
+ff_status ff_destroy(ff_ctx* ctx) {
+  delete ctx;
+  return FF_OK;
+}
+
+ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, size_t* out_bytes) {
+  if (!layers || n_layers <= 0 || B <= 0 || !out_bytes) return FF_ERR_ARG;
+  *out_bytes = WS_STATUS_BYTES;
+  return FF_OK;
+}
+
+ff_status ff_set_workspace(ff_ctx* ctx, void* dev_ptr, size_t bytes) {
+  if (!ctx) return FF_ERR_ARG;
+  if (!dev_ptr || bytes < WS_STATUS_BYTES) return fail(ctx, FF_ERR_WORKSPACE, "workspace too small");
+  if (reinterpret_cast<uintptr_t>(dev_ptr) & 255) return fail(ctx, FF_ERR_ALIGN, "workspace must be 256-byte aligned");
+  ctx->workspace = dev_ptr;
+  ctx->workspace_bytes = bytes;
+  ctx->status_zeroed = false;
+  return FF_OK;
+}
+
+ff_status ff_set_gemm_path(ff_ctx* ctx, int path) {
+  if (!ctx) return FF_ERR_ARG;
+  if (path != FF_GEMM_AUTO && path != FF_GEMM_SIMT && path != FF_GEMM_TENSOR) return fail(ctx, FF_ERR_ARG, "unknown gemm path");
+  ctx->gemm_path = path;
+  return FF_OK;
+}
+
+ff_status ff_layer_forward(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs, int B, uint64_t step,
+                           void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if ((s = check_layer(ctx, layer, B)) != FF_OK) return s;
+  if ((s = check_bufs(ctx, bufs, true)) != FF_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  FF_CUDA(ctx, cudaMemsetAsync(bufs->absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
+  if ((s = quantize_input(ctx, *layer, *bufs, B, step, st)) != FF_OK) return s;
+  if ((s = forward_from_xq(ctx, *layer, *bufs, B, step, nullptr, st)) != FF_OK) return s;
+  return normalize_output(ctx, *layer, *bufs, B, nullptr, nullptr, step, st);
+}
+
+ff_status ff_layer_loss_grad(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs, int B,
+                             const float* const* G_later, const float* theta_later, int n_later, float lambda,
+                             uint64_t step, void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if ((s = check_layer(ctx, layer, B)) != FF_OK) return s;
+  if ((s = check_bufs(ctx, bufs, false)) != FF_OK) return s;
+  if (n_later < 0 || n_later > FF_MAX_LATER) return fail(ctx, FF_ERR_ARG, "n_later out of range");
+  if (n_later > 0 && (!G_later || !theta_later)) return fail(ctx, FF_ERR_ARG, "G_later / theta_later is NULL");
+  for (int j = 0; j < n_later; ++j)
+    if (!G_later[j]) return fail(ctx, FF_ERR_ARG, "a G_later pointer is NULL");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  return loss_grad_impl(ctx, *layer, *bufs, B, G_later, theta_later, n_later, lambda, step, st);
+}
+
+ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs, int B, void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if ((s = check_layer(ctx, layer, B)) != FF_OK) return s;
+  if ((s = check_bufs(ctx, bufs, false)) != FF_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  return run_update_gemm(ctx, *layer, *bufs, B, st);
+}
+
+ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
+                        float lambda, uint64_t step, void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if (!layers || !bufs || n_layers <= 0 || n_layers > FF_MAX_LATER + 1) return fail(ctx, FF_ERR_ARG, "bad layer list");
+  for (int l = 0; l < n_layers; ++l) {
+    if ((s = check_layer(ctx, &layers[l], B)) != FF_OK) return s;
+    if ((s = check_bufs(ctx, &bufs[l], l == 0)) != FF_OK) return s;
+    if (l > 0 && !bufs[l].X) {
+      const ff_layer_desc &p = layers[l - 1], &c = layers[l];
+      if ((long long)rows_per_sample(p) * p.N != (long long)rows_per_sample(c) * in_features(c))
+        return fail(ctx, FF_ERR_ARG, "layer output / next layer input sizes differ");
+    }
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  for (int l = 0; l < n_layers; ++l) FF_CUDA(ctx, cudaMemsetAsync(bufs[l].absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
+  // Alg. 1 line 5-6: one forward through all layers with the pre-update weights
+  for (int l = 0; l < n_layers; ++l) {
+    const bool chained = l > 0 && !bufs[l].X;
+    if (!chained && (s = quantize_input(ctx, layers[l], bufs[l], B, step, st)) != FF_OK) return s;
+    const bool feeds_next = l + 1 < n_layers && !bufs[l + 1].X;
+    if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, step, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st)) != FF_OK)
+      return s;
+    if ((s = normalize_output(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].Xq : nullptr,
+                              feeds_next ? &layers[l + 1] : nullptr, step, st)) != FF_OK)
+      return s;
+  }
+  // Alg. 1 line 7-9: per layer, loss from the G's (Eq. 3), INT8 gradient and update
+  for (int l = 0; l < n_layers; ++l) {
+    const float* Gl[FF_MAX_LATER];
+    float th[FF_MAX_LATER];
+    int n_later = n_layers - 1 - l;
+    for (int j = 0; j < n_later; ++j) {
+      Gl[j] = bufs[l + 1 + j].G;
+      th[j] = layers[l + 1 + j].theta;
+    }
+    if ((s = loss_grad_impl(ctx, layers[l], bufs[l], B, Gl, th, n_later, lambda, step, st)) != FF_OK) return s;
+    if ((s = run_update_gemm(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
+  }
+  return FF_OK;
+}
+
+ff_status ff_poll_status(ff_ctx* ctx, void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t h = 0;
+  if (!ctx->status_zeroed) return FF_OK;
+  FF_CUDA(ctx, cudaMemcpyAsync(&h, ctx->workspace, sizeof(h), cudaMemcpyDeviceToHost, st));
+  FF_CUDA(ctx, cudaMemsetAsync(ctx->workspace, 0, sizeof(uint32_t), st));
+  FF_CUDA(ctx, cudaStreamSynchronize(st));
+  if (h & ST_TIMEOUT) return fail(ctx, FF_ERR_DEVICE_TIMEOUT, "a bounded in-kernel wait ran out");
+  if (h & ST_NONFINITE) return fail(ctx, FF_ERR_NONFINITE, "a tensor to be quantised held Inf or NaN");
+  return FF_OK;
+}
+
+const char* ff_last_error(const ff_ctx* ctx) { return ctx ? ctx->err : "context is NULL"; }
+
+uint64_t ff_launch_count(const ff_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+ff_status ff_int8_gemm(ff_ctx* ctx, const int8_t* A, const int8_t* Bm, int32_t* C, int M, int N, int K, int trans,
+                       void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if (!A || !Bm || !C || M <= 0 || N <= 0 || K <= 0) return fail(ctx, FF_ERR_ARG, "bad gemm arguments");
+  if (!aligned16(A) || !aligned16(Bm) || !aligned16(C)) return fail(ctx, FF_ERR_ALIGN, "gemm pointers must be 16-byte aligned");
+  if (K > ((1LL << 31) - 1) / (127LL * 127LL)) return fail(ctx, FF_ERR_RANGE, "contraction too long for INT32");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  bool tc_ok = tc_gemm_supported(M, N, K, trans);
+  if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core gemm");
+  if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT) {
+    s = tc_gemm(ctx->tc, A, Bm, C, M, N, K, trans, status_ptr(ctx), st);
+    if (s != FF_OK) return fail(ctx, s, "tensor-core gemm launch failed: %s", ctx->tc.err);
+    ctx->launches++;
+    return FF_OK;
+  }
+  RawEpilogue epi{C, M, N};
+  if (!trans) return launch_simt<DenseView, DenseView, false, 1>(ctx, dense(A, M, K), dense(Bm, N, K), M, N, K, epi, st);
+  return launch_simt<DenseView, DenseView, true, 1>(ctx, dense(A, K, M), dense(Bm, K, N), M, N, K, epi, st);
+}
+
+}  // extern "C"

@@ -1,0 +1,235 @@
+// Shape-generic INT8 x INT8 -> INT32 contraction on the CUDA cores (dp4a), used for every shape
+// the tensor-core kernels do not take (ragged K or N, Cin = 3 convolution, tiny layers) and as
+// the second implementation the tensor-core kernels are tested against.
+//   forward:          acc[m,n] = sum_k A(m,k) * Wq[n,k]             (Sec. IV-B, INT8 MAC)
+//   weight gradient:  accW_p[n,k] = sum_{m in set p} dHq[m,n] * A(m,k)   (Sec. IV-B, g^W)
+// A(m,k) is Xq[m,k] for a dense layer and the im2col view of the NHWC input for a 3x3
+// convolution (zero outside the image).  Epilogues are fused: dequantise + ReLU + goodness
+// statistics for the forward, the SGD update for the weight gradient.
+#pragma once
+#include "common.cuh"
+
+namespace ffi8 {
+
+constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 32, SG_THREADS = 256;
+constexpr int SG_PITCH = SG_BK + 4;  // bytes per smem row (36 = 9 words)
+
+// ---- operand views -----------------------------------------------------------------------
+// load8(row, col0, out): 8 consecutive columns col0..col0+7 of one row, zero outside the matrix.
+struct DenseView {
+  const int8_t* p;
+  int rows, cols;
+  bool vec8;  // cols % 8 == 0 and p 8-byte aligned
+  __device__ __forceinline__ void load8(int row, int col0, int8_t* out) const {
+    if (row < rows && vec8 && col0 + 8 <= cols) {
+      *reinterpret_cast<uint2*>(out) = __ldg(reinterpret_cast<const uint2*>(p + (size_t)row * cols + col0));
+      return;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int c = col0 + i;
+      out[i] = (row < rows && c < cols) ? p[(size_t)row * cols + c] : (int8_t)0;
+    }
+  }
+};
+// im2col view of an NHWC INT8 tensor for a 3x3 / stride 1 / pad 1 convolution:
+// row = (b*H + h)*W + w, col = (r*3 + s)*Cin + ci  ->  x[b, h+r-1, w+s-1, ci].
+struct Im2colView {
+  const int8_t* p;
+  int rows, cols;  // rows = Bn*H*W, cols = 9*Cin
+  int H, W, Cin;
+  bool vec8;  // Cin % 8 == 0 and p 8-byte aligned
+  __device__ __forceinline__ void load8(int row, int col0, int8_t* out) const {
+    if (row >= rows) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) out[i] = 0;
+      return;
+    }
+    int w = row % W, t = row / W;
+    int h = t % H, b = t / H;
+    if (vec8 && col0 + 8 <= cols) {
+      int tap = col0 / Cin, ci = col0 - tap * Cin;
+      int hh = h + tap / 3 - 1, ww = w + tap % 3 - 1;
+      uint2 v = make_uint2(0u, 0u);
+      if (hh >= 0 && hh < H && ww >= 0 && ww < W)
+        v = __ldg(reinterpret_cast<const uint2*>(p + ((size_t)(b * H + hh) * W + ww) * Cin + ci));
+      *reinterpret_cast<uint2*>(out) = v;
+      return;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int c = col0 + i;
+      int8_t v = 0;
+      if (c < cols) {
+        int tap = c / Cin, ci = c - tap * Cin;
+        int hh = h + tap / 3 - 1, ww = w + tap % 3 - 1;
+        if (hh >= 0 && hh < H && ww >= 0 && ww < W) v = p[((size_t)(b * H + hh) * W + ww) * Cin + ci];
+      }
+      out[i] = v;
+    }
+  }
+};
+
+// ---- epilogues ---------------------------------------------------------------------------
+// Each thread owns a 4x4 patch: rows i0..i0+3, cols j0..j0+3 of the output, acc[pass][r][c].
+struct RawEpilogue {  // plain INT32 store
+  int32_t* C;
+  int rows, cols;
+  __device__ __forceinline__ void operator()(int i0, int j0, const int (&acc)[2][4][4]) const {
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        if (i0 + r < rows && j0 + c < cols) C[(size_t)(i0 + r) * cols + j0 + c] = acc[0][r][c];
+  }
+};
+
+// Forward epilogue (dequantise, ReLU, goodness statistics; Sec. III, Alg. 1 line 6).
+struct ForwardEpilogue {
+  float* Y;
+  int32_t* acc_dump;  // nullable
+  unsigned long long* S;
+  int32_t* rowmax;
+  const float* absmax;
+  int rows, cols;             // M*R, N
+  int rows_per_pass;          // B*R
+  int rows_per_sample;        // R
+  __device__ __forceinline__ void operator()(int i0, int j0, const int (&acc)[2][4][4]) const {
+    const float s_w = scale_of(absmax[2]);
+    const float c0 = __fmul_rn(scale_of(absmax[0]), s_w), c1 = __fmul_rn(scale_of(absmax[1]), s_w);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int i = i0 + r;
+      unsigned long long s = 0ull;
+      int mx = 0;
+      if (i < rows) {
+        const float c = i < rows_per_pass ? c0 : c1;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          const int j = j0 + cc;
+          if (j < cols) {
+            const int a = acc[0][r][cc];
+            Y[(size_t)i * cols + j] = dequant_relu(a, c);
+            if (acc_dump) acc_dump[(size_t)i * cols + j] = a;
+            const int rl = max(a, 0);
+            s += (unsigned long long)rl * (unsigned long long)rl;
+            mx = max(mx, rl);
+          }
+        }
+      }
+      // the 16 threads that share this row sit in one half-warp (tx = lane & 15)
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) {
+        s += __shfl_xor_sync(0xffffffffu, s, o);
+        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
+      if ((threadIdx.x & 15) == 0 && i < rows && mx > 0) {
+        const int sample = i / rows_per_sample;
+        atomicAdd(S + sample, s);
+        atomicMax(rowmax + sample, mx);
+      }
+    }
+  }
+};
+
+// Weight-gradient epilogue (dequantise both sets, SGD update; Sec. IV-B, Alg. 1 line 9).
+struct UpdateEpilogue {
+  float* W;
+  int32_t* accW_dump;  // nullable, [2, rows, cols]
+  const float* absmax;
+  float lr;
+  int rows, cols;  // N, K
+  __device__ __forceinline__ void operator()(int i0, int j0, const int (&acc)[2][4][4]) const {
+    const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
+    const float cN = __fmul_rn(scale_of(absmax[4]), scale_of(absmax[1]));
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int i = i0 + r, j = j0 + c;
+        if (i < rows && j < cols) {
+          const size_t o = (size_t)i * cols + j;
+          const float g = __fadd_rn(__fmul_rn(__int2float_rn(acc[0][r][c]), cP), __fmul_rn(__int2float_rn(acc[1][r][c]), cN));
+          W[o] = __fsub_rn(W[o], __fmul_rn(lr, g));
+          if (accW_dump) {
+            accW_dump[o] = acc[0][r][c];
+            accW_dump[(size_t)rows * cols + o] = acc[1][r][c];
+          }
+        }
+      }
+  }
+};
+
+// ---- kernel ------------------------------------------------------------------------------
+// !TRANS: C[i,j] = sum_c LA(i,c) * LB(j,c)          (operands contraction-contiguous)
+//  TRANS: C[i,j] = sum_c LA(c,i) * LB(c,j)          (operands contraction-strided)
+// The contraction index runs over NPASS consecutive ranges of `clen` each (one accumulator set
+// per range: the positive and the negative set of the weight gradient).
+template <class LA, class LB, bool TRANS, int NPASS, class Epi>
+__global__ void __launch_bounds__(SG_THREADS) gemm_simt_kernel(LA la, LB lb, int clen, Epi epi) {
+  __shared__ __align__(16) int8_t As[SG_BM * SG_PITCH];
+  __shared__ __align__(16) int8_t Bs[SG_BN * SG_PITCH];
+  const int tid = threadIdx.x;
+  const int tx = tid & 15, ty = tid >> 4;
+  const int i_blk = blockIdx.y * SG_BM, j_blk = blockIdx.x * SG_BN;
+  int acc[2][4][4];
+#pragma unroll
+  for (int p = 0; p < 2; ++p)
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[p][r][c] = 0;
+
+#pragma unroll
+  for (int pass = 0; pass < NPASS; ++pass) {
+    const int cbeg = pass * clen, cend = cbeg + clen;
+    for (int c0 = cbeg; c0 < cend; c0 += SG_BK) {
+      int8_t va[8], vb[8];
+      if (!TRANS) {
+        const int row = tid >> 2, kk = (tid & 3) * 8;  // 64 rows x 4 groups of 8 contraction bytes
+        la.load8(i_blk + row, c0 + kk, va);
+        lb.load8(j_blk + row, c0 + kk, vb);
+        // mask the tail of the contraction range (ranges need not be multiples of SG_BK)
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (c0 + kk + i >= cend) {
+            va[i] = 0;
+            vb[i] = 0;
+          }
+        *reinterpret_cast<uint32_t*>(&As[row * SG_PITCH + kk]) = *reinterpret_cast<uint32_t*>(&va[0]);
+        *reinterpret_cast<uint32_t*>(&As[row * SG_PITCH + kk + 4]) = *reinterpret_cast<uint32_t*>(&va[4]);
+        *reinterpret_cast<uint32_t*>(&Bs[row * SG_PITCH + kk]) = *reinterpret_cast<uint32_t*>(&vb[0]);
+        *reinterpret_cast<uint32_t*>(&Bs[row * SG_PITCH + kk + 4]) = *reinterpret_cast<uint32_t*>(&vb[4]);
+      } else {
+        const int cl = tid >> 3, g = (tid & 7) * 8;  // 32 contraction rows x 8 groups of 8 outputs
+        const bool ok = c0 + cl < cend;
+        if (ok) {
+          la.load8(c0 + cl, i_blk + g, va);
+          lb.load8(c0 + cl, j_blk + g, vb);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          As[(g + i) * SG_PITCH + cl] = ok ? va[i] : (int8_t)0;
+          Bs[(g + i) * SG_PITCH + cl] = ok ? vb[i] : (int8_t)0;
+        }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int kw = 0; kw < SG_BK / 4; ++kw) {
+        int a[4], b[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) a[r] = *reinterpret_cast<const int*>(&As[(ty * 4 + r) * SG_PITCH + kw * 4]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) b[c] = *reinterpret_cast<const int*>(&Bs[(tx * 4 + c) * SG_PITCH + kw * 4]);
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) acc[pass][r][c] = __dp4a(a[r], b[c], acc[pass][r][c]);
+      }
+      __syncthreads();
+    }
+  }
+  epi(i_blk + ty * 4, j_blk + tx * 4, acc);
+}
+
+}  // namespace ffi8

@@ -1,0 +1,577 @@
+// INT8 x INT8 -> INT32 contractions of the FF-INT8 step on the 5th-generation tensor cores
+// (tcgen05.mma kind::i8, accumulators in tensor memory, operands staged by TMA):
+//   forward           acc[m,n]    = sum_k Xq[m,k] * Wq[n,k]                    (Sec. IV-B, INT8 MAC)
+//   weight gradient   accW_p[n,k] = sum_{m in set p} dHq[m,n] * Xq[m,k]        (Sec. IV-B, g^W)
+// Persistent kernel, one CTA per SM, 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer
+// (one elected lane each), warps 2..5 = epilogue (one TMEM lane quadrant each).
+// Output tile 128 x 256, contraction block 128 bytes (4 MMAs of K = 32), 4-stage smem ring.
+// The forward operands are K-major (contraction contiguous); the weight-gradient operands are
+// read in their natural row-major layout as MN-major operands, so no transposed copy of dHq or Xq
+// is ever written.  The forward double-buffers the accumulator (2 x 256 TMEM columns) so that the
+// epilogue of tile i overlaps the MMAs of tile i+1; the weight gradient holds the accumulators
+// of the positive and the negative set side by side (2 x 256 columns) and applies the update
+// W <- W - lr*(float(accP)*cP + float(accN)*cN) (Alg. 1 line 9) in its epilogue.
+// Every wait is bounded: when one runs out the CTA raises ST_TIMEOUT, drains and returns.
+#pragma once
+#include <cuda.h>
+
+#include <cstdio>
+
+#include "../../include/ffint8.h"
+#include "common.cuh"
+
+namespace ffi8 {
+
+constexpr int TC_BM = 128, TC_BN = 256, TC_BKB = 128;  // tile rows, tile cols, contraction bytes per block
+constexpr int TC_STAGES = 4;
+constexpr int TC_THREADS = 192;
+constexpr uint32_t TC_A_BYTES = TC_BM * TC_BKB;      // 16 KiB
+constexpr uint32_t TC_B_BYTES = TC_BN * TC_BKB;      // 32 KiB
+constexpr uint32_t TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
+constexpr uint32_t TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr uint32_t TC_TMEM_COLS = 512;
+constexpr unsigned long long TC_WAIT_NS = 2000000000ull;  // 2 s bound on every wait
+
+enum { TC_MODE_RAW = 0, TC_MODE_FWD = 1, TC_MODE_UPD = 2 };
+
+struct TcParams {
+  int out_rows, out_cols;   // extent of the output matrix
+  int tiles_m, tiles_n;
+  int kblocks;              // contraction blocks per pass
+  int npass;                // 1, or 2 for the weight gradient (positive / negative set)
+  uint32_t* status;
+  // raw
+  int32_t* C;
+  // forward epilogue
+  float* Y;
+  int32_t* acc_dump;
+  unsigned long long* S;
+  int32_t* rowmax;
+  const float* absmax;
+  int rows_per_pass, rows_per_sample;
+  // update epilogue
+  float* W;
+  int32_t* accW_dump;
+  float lr;
+};
+
+// ---- PTX wrappers --------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false when the time limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 0xFFu) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > TC_WAIT_NS) return false;
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+               "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+               "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Load 32 consecutive accumulator columns of this thread's TMEM lane and wait for them.
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, int (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+// (the wait for the load is part of tc_ld32, so the registers are valid when it returns)
+
+// Shared-memory matrix descriptor for a 128-byte-swizzled operand tile (rows of 128 bytes, groups
+// of 8 rows = 1024 bytes).  K-major: rows are M/N indices, SBO = 1024 between 8-row groups, LBO
+// unused.  MN-major: rows are contraction indices, SBO = 1024 between groups of 8 contraction
+// rows, LBO = distance between successive 128-element chunks along M/N.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;  // descriptor version of this architecture
+  d |= 2ull << 61;  // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: INT8 x INT8 -> INT32, dense, M = 128, N = 256.
+__host__ __device__ constexpr uint32_t make_idesc_i8(bool a_mn_major, bool b_mn_major) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+
+// ---- kernel --------------------------------------------------------------------------------
+template <int MODE, bool MN_MAJOR>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+    tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte aligned operand ring, then the barriers
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t ring = (raw + 1023u) & ~1023u;
+  uint8_t* ring_ptr = smem_raw + (ring - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring_ptr + TC_STAGES * TC_STAGE_BYTES);
+  const uint32_t bar_full = smem_u32(bars);                      // [TC_STAGES]
+  const uint32_t bar_empty = bar_full + 8 * TC_STAGES;           // [TC_STAGES]
+  const uint32_t bar_tfull = bar_empty + 8 * TC_STAGES;          // [2]
+  const uint32_t bar_tempty = bar_tfull + 16;                    // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_STAGES + 4);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int ACC_STAGES = (MODE == TC_MODE_UPD || MN_MAJOR) ? 1 : 2;
+  const int total_tiles = p.tiles_m * p.tiles_n;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < TC_STAGES; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar_tfull + 8 * s, 1);
+      mbar_init(bar_tempty + 8 * s, 4);  // one arrive per epilogue warp
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TC_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer -------------------------------------------
+    if (lane == 0) {
+      uint32_t it = 0;  // running k-block counter (ring position)
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+        for (int pass = 0; pass < p.npass && ok; ++pass) {
+          for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+            const uint32_t s = it % TC_STAGES, ph = (it / TC_STAGES) & 1u;
+            if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) {
+              ok = false;
+              break;
+            }
+            const uint32_t a_dst = ring + s * TC_STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
+            mbar_expect_tx(bar_full + 8 * s, TC_STAGE_BYTES);
+            if (!MN_MAJOR) {
+              tma_load_2d(a_dst, &tmA, bar_full + 8 * s, kb * TC_BKB, tm * TC_BM);
+              tma_load_2d(b_dst, &tmB, bar_full + 8 * s, kb * TC_BKB, tn * TC_BN);
+            } else {
+              // tile of 128 contraction rows x 128 output indices; B takes two such boxes
+              tma_load_3d(a_dst, &tmA, bar_full + 8 * s, tm * TC_BM, kb * 128, pass);
+              tma_load_3d(b_dst, &tmB, bar_full + 8 * s, tn * TC_BN, kb * 128, pass);
+              tma_load_3d(b_dst + 16384, &tmB, bar_full + 8 * s, tn * TC_BN + 128, kb * 128, pass);
+            }
+          }
+        }
+      }
+      if (!ok) {
+        atomicOr(p.status, ST_TIMEOUT);
+        *abort_flag = 1;
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer ---------------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_i8(MN_MAJOR, MN_MAJOR);
+      uint32_t it = 0, tile_it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+        const uint32_t as = tile_it % ACC_STAGES, aph = (tile_it / ACC_STAGES) & 1u;
+        if (!mbar_wait(bar_tempty + 8 * as, aph ^ 1u, abort_flag)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        for (int pass = 0; pass < p.npass && ok; ++pass) {
+          const uint32_t d_tmem = tmem_base + (MODE == TC_MODE_UPD ? pass * TC_BN : as * TC_BN);
+          for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+            const uint32_t s = it % TC_STAGES, ph = (it / TC_STAGES) & 1u;
+            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t a_src = ring + s * TC_STAGE_BYTES, b_src = a_src + TC_A_BYTES;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              uint64_t ad, bd;
+              if (!MN_MAJOR) {
+                ad = make_smem_desc(a_src + k * 32, 16, 1024);
+                bd = make_smem_desc(b_src + k * 32, 16, 1024);
+              } else {
+                ad = make_smem_desc(a_src + k * 4096, 16384, 1024);
+                bd = make_smem_desc(b_src + k * 4096, 16384, 1024);
+              }
+              tc_mma_i8(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            tc_commit(bar_empty + 8 * s);  // frees the smem stage once these MMAs have read it
+          }
+        }
+        if (ok) tc_commit(bar_tfull + 8 * as);  // accumulator complete
+      }
+      if (!ok) {
+        atomicOr(p.status, ST_TIMEOUT);
+        *abort_flag = 1;
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------- epilogue (warps 2..5) ----------------------------------
+    const int quad = warp & 3;  // TMEM lane quadrant this warp may read
+    uint32_t tile_it = 0;
+    bool ok = true;
+    float c0 = 0.f, c1 = 0.f, cP = 0.f, cN = 0.f;
+    if (MODE == TC_MODE_FWD) {
+      const float s_w = scale_of(p.absmax[2]);
+      c0 = __fmul_rn(scale_of(p.absmax[0]), s_w);
+      c1 = __fmul_rn(scale_of(p.absmax[1]), s_w);
+    }
+    if (MODE == TC_MODE_UPD) {
+      cP = __fmul_rn(scale_of(p.absmax[3]), scale_of(p.absmax[0]));
+      cN = __fmul_rn(scale_of(p.absmax[4]), scale_of(p.absmax[1]));
+    }
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+      const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+      const uint32_t as = tile_it % ACC_STAGES, aph = (tile_it / ACC_STAGES) & 1u;
+      if (!mbar_wait(bar_tfull + 8 * as, aph, abort_flag)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const int row = tm * TC_BM + quad * 32 + lane;
+      const bool row_ok = row < p.out_rows;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
+      const int col0 = tn * TC_BN;
+      if (MODE == TC_MODE_RAW) {
+        for (int cb = 0; cb < TC_BN; cb += 32) {
+          int v[32];
+          tc_ld32(t_row + as * TC_BN + cb, v);
+          if (row_ok) {
+            int32_t* dst = p.C + (size_t)row * p.out_cols + col0 + cb;
+            if (col0 + cb + 32 <= p.out_cols && (p.out_cols & 3) == 0) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) *reinterpret_cast<int4*>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + cb + j < p.out_cols) dst[j] = v[j];
+            }
+          }
+        }
+      } else if (MODE == TC_MODE_FWD) {
+        const float c = row < p.rows_per_pass ? c0 : c1;
+        unsigned long long ssum = 0ull;
+        int mx = 0;
+        for (int cb = 0; cb < TC_BN; cb += 32) {
+          if (col0 + cb >= p.out_cols) break;  // uniform across the warp
+          int v[32];
+          tc_ld32(t_row + as * TC_BN + cb, v);
+          if (row_ok) {
+            const size_t o = (size_t)row * p.out_cols + col0 + cb;
+            const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              float y[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const int a = v[j + q];
+                y[q] = dequant_relu(a, c);
+                if (full || col0 + cb + j + q < p.out_cols) {
+                  const int rl = max(a, 0);
+                  ssum += (unsigned long long)((long long)rl * (long long)rl);
+                  mx = max(mx, rl);
+                }
+              }
+              if (full) {
+                *reinterpret_cast<float4*>(p.Y + o + j) = make_float4(y[0], y[1], y[2], y[3]);
+                if (p.acc_dump) *reinterpret_cast<int4*>(p.acc_dump + o + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              } else {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  if (col0 + cb + j + q < p.out_cols) {
+                    p.Y[o + j + q] = y[q];
+                    if (p.acc_dump) p.acc_dump[o + j + q] = v[j + q];
+                  }
+              }
+            }
+          }
+        }
+        if (row_ok && mx > 0) {
+          const int sample = row / p.rows_per_sample;
+          atomicAdd(p.S + sample, ssum);
+          atomicMax(p.rowmax + sample, mx);
+        }
+      } else {  // TC_MODE_UPD
+        for (int cb = 0; cb < TC_BN; cb += 32) {
+          if (col0 + cb >= p.out_cols) break;
+          int vp[32], vn[32];
+          tc_ld32(t_row + cb, vp);
+          tc_ld32(t_row + TC_BN + cb, vn);
+          if (row_ok) {
+            const size_t o = (size_t)row * p.out_cols + col0 + cb;
+            const size_t plane = (size_t)p.out_rows * p.out_cols;
+            const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              if (full) {
+                float4 w = *reinterpret_cast<const float4*>(p.W + o + j);
+                float wv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const float g = __fadd_rn(__fmul_rn(__int2float_rn(vp[j + q]), cP), __fmul_rn(__int2float_rn(vn[j + q]), cN));
+                  wv[q] = __fsub_rn(wv[q], __fmul_rn(p.lr, g));
+                }
+                *reinterpret_cast<float4*>(p.W + o + j) = make_float4(wv[0], wv[1], wv[2], wv[3]);
+                if (p.accW_dump) {
+                  *reinterpret_cast<int4*>(p.accW_dump + o + j) = make_int4(vp[j], vp[j + 1], vp[j + 2], vp[j + 3]);
+                  *reinterpret_cast<int4*>(p.accW_dump + plane + o + j) = make_int4(vn[j], vn[j + 1], vn[j + 2], vn[j + 3]);
+                }
+              } else {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  if (col0 + cb + j + q < p.out_cols) {
+                    const float g = __fadd_rn(__fmul_rn(__int2float_rn(vp[j + q]), cP), __fmul_rn(__int2float_rn(vn[j + q]), cN));
+                    p.W[o + j + q] = __fsub_rn(p.W[o + j + q], __fmul_rn(p.lr, g));
+                    if (p.accW_dump) {
+                      p.accW_dump[o + j + q] = vp[j + q];
+                      p.accW_dump[plane + o + j + q] = vn[j + q];
+                    }
+                  }
+              }
+            }
+          }
+        }
+      }
+      // accumulator stage drained: hand it back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8 * as);
+    }
+    if (!ok && lane == 0) {
+      atomicOr(p.status, ST_TIMEOUT);
+      *abort_flag = 1;
+    }
+  }
+
+  // ---- teardown: everyone meets, outstanding copies are waited for, TMEM is released ---------
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) {
+    // give in-flight TMA copies a bounded time to land before the CTA (and its smem) goes away
+    const unsigned long long t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 2000000ull) {
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+  }
+}
+
+// ---- host side -----------------------------------------------------------------------------
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcState {
+  int sm_count = 148;
+  PFN_encodeTiled encode = nullptr;
+  bool attr_set[3][2] = {{false, false}, {false, false}, {false, false}};
+  char err[256] = {0};
+};
+
+inline ff_status tc_init(TcState& t) {
+  if (t.encode) return FF_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+  if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
+    snprintf(t.err, sizeof(t.err), "cuTensorMapEncodeTiled not available");
+    return FF_ERR_CUDA;
+  }
+  t.encode = reinterpret_cast<PFN_encodeTiled>(fn);
+  return FF_OK;
+}
+
+// INT8 row-major matrix [rows, cols] viewed as `passes` stacked matrices of rows_per_pass rows;
+// box = box_cols x box_rows (x 1), 128-byte swizzle, zero fill outside.
+inline ff_status tc_make_map(TcState& t, CUtensorMap* tm, const int8_t* base, uint64_t cols, uint64_t rows_per_pass, uint64_t passes,
+                             uint32_t box_cols, uint32_t box_rows) {
+  cuuint64_t dims[3] = {cols, rows_per_pass, passes};
+  cuuint64_t strides[2] = {cols, cols * rows_per_pass};
+  cuuint32_t box[3] = {box_cols, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const cuuint32_t rank = passes > 0 ? 3 : 2;
+  if (rank == 2) dims[2] = 1;
+  CUresult r = t.encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, rank, const_cast<int8_t*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(t.err, sizeof(t.err), "cuTensorMapEncodeTiled failed (%d) cols=%llu rows=%llu", (int)r, (unsigned long long)cols,
+             (unsigned long long)rows_per_pass);
+    return FF_ERR_CUDA;
+  }
+  return FF_OK;
+}
+
+template <int MODE, bool MN_MAJOR>
+inline ff_status tc_launch(TcState& t, const CUtensorMap& a, const CUtensorMap& b, TcParams p, cudaStream_t st) {
+  if (!t.attr_set[MODE][MN_MAJOR]) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<MODE, MN_MAJOR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES);
+    if (e != cudaSuccess) {
+      snprintf(t.err, sizeof(t.err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+      return FF_ERR_CUDA;
+    }
+    t.attr_set[MODE][MN_MAJOR] = true;
+  }
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int grid = tiles < t.sm_count ? tiles : t.sm_count;
+  tc_gemm_kernel<MODE, MN_MAJOR><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(a, b, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    snprintf(t.err, sizeof(t.err), "launch: %s", cudaGetErrorString(e));
+    return FF_ERR_CUDA;
+  }
+  return FF_OK;
+}
+
+inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+// K-major ("NT") problem: A [M,K], B [N,K]; K % 16 == 0 (TMA row pitch), everything else ragged.
+inline bool tc_nt_ok(long long M, long long N, long long K) { return K % 16 == 0 && K >= 16 && M >= 1 && N >= 1; }
+// MN-major ("TN") problem: A [Kc,M], B [Kc,N]; M % 16 == 0 and N % 16 == 0.
+inline bool tc_tn_ok(long long M, long long N, long long Kc) { return M % 16 == 0 && N % 16 == 0 && Kc >= 1; }
+
+inline bool tc_gemm_supported(int M, int N, int K, int trans) { return trans ? tc_tn_ok(M, N, K) : tc_nt_ok(M, N, K); }
+inline bool tc_forward_supported(const ff_layer_desc& L, int B) { return L.kind == FF_LINEAR && tc_nt_ok(2LL * B, L.N, L.K); }
+inline bool tc_update_supported(const ff_layer_desc& L, int B) { return L.kind == FF_LINEAR && tc_tn_ok(L.N, L.K, B); }
+
+inline ff_status tc_gemm(TcState& t, const int8_t* A, const int8_t* Bm, int32_t* C, int M, int N, int K, int trans,
+                         uint32_t* status, cudaStream_t st) {
+  ff_status s = tc_init(t);
+  if (s != FF_OK) return s;
+  CUtensorMap ta, tb;
+  TcParams p = {};
+  p.out_rows = M;
+  p.out_cols = N;
+  p.tiles_m = cdiv(M, TC_BM);
+  p.tiles_n = cdiv(N, TC_BN);
+  p.npass = 1;
+  p.status = status;
+  p.C = C;
+  if (!trans) {
+    p.kblocks = cdiv(K, TC_BKB);
+    if ((s = tc_make_map(t, &ta, A, K, M, 0, TC_BKB, TC_BM)) != FF_OK) return s;
+    if ((s = tc_make_map(t, &tb, Bm, K, N, 0, TC_BKB, TC_BN)) != FF_OK) return s;
+    return tc_launch<TC_MODE_RAW, false>(t, ta, tb, p, st);
+  }
+  p.kblocks = cdiv(K, 128);
+  if ((s = tc_make_map(t, &ta, A, M, K, 1, 128, 128)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &tb, Bm, N, K, 1, 128, 128)) != FF_OK) return s;
+  return tc_launch<TC_MODE_RAW, true>(t, ta, tb, p, st);
+}
+
+inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint32_t* status, cudaStream_t st) {
+  ff_status s = tc_init(t);
+  if (s != FF_OK) return s;
+  const int M = 2 * B;
+  CUtensorMap ta, tb;
+  TcParams p = {};
+  p.out_rows = M;
+  p.out_cols = L.N;
+  p.tiles_m = cdiv(M, TC_BM);
+  p.tiles_n = cdiv(L.N, TC_BN);
+  p.kblocks = cdiv(L.K, TC_BKB);
+  p.npass = 1;
+  p.status = status;
+  p.Y = b.Y;
+  p.acc_dump = b.acc_dump;
+  p.S = reinterpret_cast<unsigned long long*>(b.S);
+  p.rowmax = b.rowmax;
+  p.absmax = b.absmax;
+  p.rows_per_pass = B;
+  p.rows_per_sample = 1;
+  if ((s = tc_make_map(t, &ta, b.Xq, L.K, M, 0, TC_BKB, TC_BM)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, TC_BKB, TC_BN)) != FF_OK) return s;
+  return tc_launch<TC_MODE_FWD, false>(t, ta, tb, p, st);
+}
+
+inline ff_status tc_update(TcState& t, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint32_t* status, cudaStream_t st) {
+  ff_status s = tc_init(t);
+  if (s != FF_OK) return s;
+  CUtensorMap ta, tb;
+  TcParams p = {};
+  p.out_rows = L.N;
+  p.out_cols = L.K;
+  p.tiles_m = cdiv(L.N, TC_BM);
+  p.tiles_n = cdiv(L.K, TC_BN);
+  p.kblocks = cdiv(B, 128);
+  p.npass = 2;
+  p.status = status;
+  p.W = b.W;
+  p.accW_dump = b.accW_dump;
+  p.absmax = b.absmax;
+  p.lr = L.lr;
+  if ((s = tc_make_map(t, &ta, b.dHq, L.N, B, 2, 128, 128)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &tb, b.Xq, L.K, B, 2, 128, 128)) != FF_OK) return s;
+  return tc_launch<TC_MODE_UPD, true>(t, ta, tb, p, st);
+}
+
+}  // namespace ffi8

@@ -1,0 +1,190 @@
+"""GPU parity tests: the CUDA path (through the C ABI) against the CPU oracle, element by element.
+Bit-exact for INT8 / INT32 / index work and, by the arithmetic contract, for every FP32 state
+tensor too (which is tighter than the 1e-5 relative tolerance the task allows); the loss scalar
+is compared at 1e-5 relative."""
+import numpy as np
+import pytest
+
+from oracle import ffint8_oracle as O
+from paper_2506_22771_b200 import binding as ffb
+from paper_2506_22771_b200 import synth
+from tests.ffharness import GpuNet, compare_layer, specs_and_descs
+
+pytestmark = pytest.mark.gpu
+
+PATHS = [ffb.FF_GEMM_SIMT, ffb.FF_GEMM_AUTO]
+
+
+def _gemm_case(M, N, K, trans, path):
+    import torch
+    g = np.random.default_rng(M * 7 + N * 3 + K + trans)
+    ctx = ffb.Context([ffb.ff_layer_desc(0, 16, 16, 1, 1, 0, 0, 0, 0, 0, 1.0, 0.1, 1.0, 1e-8, 0)], 1, 0)
+    ffb.ff_set_gemm_path(ctx.ctx, path)
+    if not trans:
+        a = g.integers(-127, 128, size=(M, K)).astype(np.int8)
+        b = g.integers(-127, 128, size=(N, K)).astype(np.int8)
+        want = a.astype(np.int64) @ b.astype(np.int64).T
+    else:
+        a = g.integers(-127, 128, size=(K, M)).astype(np.int8)
+        b = g.integers(-127, 128, size=(K, N)).astype(np.int8)
+        want = a.astype(np.int64).T @ b.astype(np.int64)
+    ta, tb = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
+    tc = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+    ffb.ff_int8_gemm(ctx.ctx, ta.data_ptr(), tb.data_ptr(), tc.data_ptr(), M, N, K, trans, 0)
+    ffb.ff_poll_status(ctx.ctx, 0)
+    got = tc.cpu().numpy()
+    ctx.close()
+    assert np.array_equal(got, want), (np.argwhere(got != want)[:5], got[got != want][:5], want[got != want][:5])
+
+
+@pytest.mark.parametrize("M,N,K", [(3, 5, 33), (64, 64, 32), (130, 70, 100), (1, 500, 784)])
+@pytest.mark.parametrize("trans", [0, 1])
+def test_int8_gemm_simt(M, N, K, trans):
+    _gemm_case(M, N, K, trans, ffb.FF_GEMM_SIMT)
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 128), (128, 256, 512), (256, 512, 1024), (200, 300, 784),
+                                   (1000, 2000, 2000), (16, 16, 16), (4096, 2048, 4096)])
+def test_int8_gemm_tensor_forward_orientation(M, N, K):
+    _gemm_case(M, N, K, 0, ffb.FF_GEMM_TENSOR)
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 128), (128, 256, 512), (256, 512, 1000), (208, 304, 77),
+                                   (2000, 784, 1024), (16, 16, 3), (2048, 4096, 4096)])
+def test_int8_gemm_tensor_weight_gradient_orientation(M, N, K):
+    _gemm_case(M, N, K, 1, ffb.FF_GEMM_TENSOR)
+
+
+def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), chain=True, check_every=1):
+    specs, descs = specs_and_descs(w.layers, seed, *rounding)
+    Ws = synth.make_weights(w, seed)
+    X = synth.make_batch(w, seed)
+    net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path)
+    net.set_input(X)
+    for step in range(steps):
+        lam = lam_per_step * step
+        net.train_step(lam, step)
+        states = O.train_step(specs, Ws, X, w.B, lam, step)
+        if step % check_every == 0 or step == steps - 1:
+            for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
+                compare_layer(st, b, sp, w.B, tag=f"step{step}/layer{l}/")
+        Ws = [st.W_new for st in states]
+    net.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_config1_tiny_mlp_ten_steps(path):
+    _run_and_compare(synth.workload("tiny_mlp"), seed=11, steps=10, lam_per_step=0.0, path=path)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("rounding", [(0, 0, 0), (1, 1, 1)])
+def test_rounding_modes(path, rounding):
+    w = synth.scaled(synth.workload("tiny_mlp"), B=24, width_div=4)
+    _run_and_compare(w, seed=5, steps=2, lam_per_step=0.0, path=path, rounding=rounding)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_config3_lookahead_scaled(path):
+    # 4-layer MLP with the look-ahead loss, lambda growing per step; widths cut to keep the oracle fast,
+    # several 128x256 tiles plus ragged tails in M (2*200), N (496) and K (784, 496)
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=200, width_div=4)
+    w.layers[0].N = w.layers[1].K = 496
+    w.layers[0].tau = float(np.sqrt(496))
+    w.layers[0].theta = 496.0
+    _run_and_compare(w, seed=3, steps=3, lam_per_step=0.25, path=path)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_config2_greedy_scaled(path):
+    # greedy: each layer trained on the frozen forward of the earlier ones = separate single-layer steps
+    w = synth.scaled(synth.workload("mlp_greedy"), B=96, width_div=8)
+    specs, descs = specs_and_descs(w.layers, 9)
+    Ws = synth.make_weights(w, 9)
+    x = synth.make_batch(w, 9)
+    for l in range(len(specs)):
+        net = GpuNet([descs[l]], w.B, [Ws[l]], gemm_path=path)
+        net.set_input(x)
+        for step in range(2):
+            net.train_step(0.0, step)
+            st = O.train_step([specs[l]], [Ws[l]], x, w.B, 0.0, step)[0]
+            compare_layer(st, net.bufs[0], specs[l], w.B, tag=f"layer{l}/step{step}/")
+            Ws[l] = st.W_new
+        st = O.layer_forward(specs[l], x, Ws[l], w.B, 99)
+        x = st.Xnext
+        net.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_config4_cnn_scaled(path):
+    w = synth.scaled(synth.workload("cnn"), B=2, width_div=4)      # 3 -> 16 -> 32 -> 64 channels, 32x32
+    _run_and_compare(w, seed=21, steps=2, lam_per_step=0.0, path=path)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_config5_roofline_scaled(path):
+    w = synth.scaled(synth.workload("roofline"), B=256, width_div=8)   # 8192 -> 1024, theta = N/2
+    w.layers[0].K = 1024
+    w.in_shape = (1024,)
+    _run_and_compare(w, seed=2, steps=2, lam_per_step=0.0, path=path)
+
+
+def test_separate_calls_equal_train_step():
+    w = synth.scaled(synth.workload("tiny_mlp"), B=40, width_div=2)
+    w.layers = w.layers[:1]
+    specs, descs = specs_and_descs(w.layers, 4)
+    Ws = synth.make_weights(w, 4)
+    X = synth.make_batch(w, 4)
+    net = GpuNet(descs, w.B, Ws)
+    net.set_input(X)
+    ctx, d, b = net.ctx.ctx, descs[0], net.bufs[0].struct
+    ffb.ff_layer_forward(ctx, d, b, w.B, 7, 0)
+    ffb.ff_layer_loss_grad(ctx, d, b, w.B, [], [], 0.0, 7, 0)
+    ffb.ff_layer_update(ctx, d, b, w.B, 0)
+    ffb.ff_poll_status(ctx, 0)
+    st = O.train_step(specs, Ws, X, w.B, 0.0, 7)[0]
+    compare_layer(st, net.bufs[0], specs[0], w.B)
+    net.close()
+
+
+def test_edge_cases_zero_input_and_nonfinite():
+    import torch
+    w = synth.scaled(synth.workload("tiny_mlp"), B=8, width_div=4)
+    w.layers = w.layers[:1]
+    specs, descs = specs_and_descs(w.layers, 1)
+    Ws = synth.make_weights(w, 1)
+    X = np.zeros((16, 784), dtype=np.float32)
+    net = GpuNet(descs, w.B, Ws)
+    net.set_input(X)
+    net.train_step(0.0, 0)
+    st = O.train_step(specs, Ws, X, w.B, 0.0, 0)[0]
+    compare_layer(st, net.bufs[0], specs[0], w.B)
+    assert not net.bufs[0].G.any() and torch.equal(net.bufs[0].W.cpu(), torch.from_numpy(Ws[0]))
+    X[3, 5] = np.inf
+    net.set_input(X)
+    with pytest.raises(ffb.FFError) as e:
+        net.train_step(0.0, 1)
+    assert e.value.code == ffb.FF_ERR_NONFINITE
+    net.close()
+
+
+def test_host_side_argument_errors():
+    w = synth.scaled(synth.workload("tiny_mlp"), B=8, width_div=4)
+    specs, descs = specs_and_descs(w.layers[:1], 1)
+    net = GpuNet(descs, w.B, synth.make_weights(w, 1)[:1])
+    bad = ffb.ff_layer_desc.from_buffer_copy(descs[0])
+    bad.eps = 0.0
+    with pytest.raises(ffb.FFError) as e:
+        ffb.ff_layer_forward(net.ctx.ctx, bad, net.bufs[0].struct, w.B, 0, 0)
+    assert e.value.code == ffb.FF_ERR_ARG
+    bad = ffb.ff_layer_desc.from_buffer_copy(descs[0])
+    bad.K = 200000
+    with pytest.raises(ffb.FFError) as e:
+        ffb.ff_layer_forward(net.ctx.ctx, bad, net.bufs[0].struct, w.B, 0, 0)
+    assert e.value.code == ffb.FF_ERR_RANGE
+    bufs = ffb.ff_layer_bufs.from_buffer_copy(net.bufs[0].struct)
+    bufs.Y = net.bufs[0].Y.data_ptr() + 4
+    with pytest.raises(ffb.FFError) as e:
+        ffb.ff_layer_forward(net.ctx.ctx, descs[0], bufs, w.B, 0, 0)
+    assert e.value.code == ffb.FF_ERR_ALIGN
+    net.close()
