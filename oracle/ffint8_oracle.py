@@ -85,11 +85,15 @@ def absmax(x: np.ndarray) -> np.float32:
     return F32(np.max(np.abs(x)))
 
 
+TINY_RANGE = F32(2.0 ** -100)
+
+
 def scale_pair(a: np.float32):
     """SUQ scale s = a/127 and its reciprocal factor inv = 127/a, each ONE float32 division.
-    A zero tensor (a == 0) quantises to all zeros: s = 1, inv = 0."""
+    A zero tensor quantises to all zeros: s = 1, inv = 0.  So does a tensor whose range is below
+    2^-100 (127/a would leave the float32 range for subnormal a; such a gradient carries nothing)."""
     a = F32(a)
-    if a == F32(0.0):
+    if a < TINY_RANGE:
         return F32(1.0), F32(0.0)
     return F32(a / F32(127.0)), F32(F32(127.0) / a)
 

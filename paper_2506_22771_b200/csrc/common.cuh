@@ -42,21 +42,14 @@ __host__ inline RoundKey make_round_key(uint64_t seed, int role, int layer, uint
   return k;
 }
 
-// s = a/127, inv = 127/a; a zero tensor quantises to zeros (s = 1, inv = 0).
-__device__ __forceinline__ void scale_pair(float a, float& s, float& inv) {
-  if (a == 0.0f) {
-    s = 1.0f;
-    inv = 0.0f;
-  } else {
-    s = __fdiv_rn(a, 127.0f);
-    inv = __fdiv_rn(127.0f, a);
-  }
-}
+// s = a/127, inv = 127/a.  A zero tensor, or one whose range is below 2^-100 (127/a would leave
+// the FP32 range for subnormal a), quantises to zeros: s = 1, inv = 0.
+constexpr float TINY_RANGE = 7.888609052210118e-31f;  // 2^-100
 __device__ __forceinline__ float scale_of(float a) {
-  return a == 0.0f ? 1.0f : __fdiv_rn(a, 127.0f);
+  return a < TINY_RANGE ? 1.0f : __fdiv_rn(a, 127.0f);
 }
 __device__ __forceinline__ float inv_of(float a) {
-  return a == 0.0f ? 0.0f : __fdiv_rn(127.0f, a);
+  return a < TINY_RANGE ? 0.0f : __fdiv_rn(127.0f, a);
 }
 
 // One 32-bit hash per element PAIR (pair index = linear index >> 1).

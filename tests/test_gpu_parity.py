@@ -23,11 +23,11 @@ def _gemm_case(M, N, K, trans, path):
     if not trans:
         a = g.integers(-127, 128, size=(M, K)).astype(np.int8)
         b = g.integers(-127, 128, size=(N, K)).astype(np.int8)
-        want = a.astype(np.int64) @ b.astype(np.int64).T
+        want = (a.astype(np.float64) @ b.astype(np.float64).T).astype(np.int64)
     else:
         a = g.integers(-127, 128, size=(K, M)).astype(np.int8)
         b = g.integers(-127, 128, size=(K, N)).astype(np.int8)
-        want = a.astype(np.int64).T @ b.astype(np.int64)
+        want = (a.astype(np.float64).T @ b.astype(np.float64)).astype(np.int64)
     ta, tb = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
     tc = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
     ffb.ff_int8_gemm(ctx.ctx, ta.data_ptr(), tb.data_ptr(), tc.data_ptr(), M, N, K, trans, 0)

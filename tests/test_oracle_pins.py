@@ -474,3 +474,15 @@ def test_train_step_reductions_and_determinism():
     # different step index -> different stochastic rounding, same scales
     d = O.train_step(specs, Ws, X, B, 0.0, 5)
     assert d[0].a_x == a[0].a_x and not np.array_equal(d[0].Xq, a[0].Xq)
+
+
+def test_tiny_range_is_treated_as_zero_tensor():
+    # a subnormal range would make 127/a overflow; below 2^-100 the tensor quantises to zeros
+    x = np.array([1e-40, -3e-41, 0.0], dtype=F32)
+    a = O.absmax(x)
+    assert a > 0 and O.scale_pair(a) == (F32(1.0), F32(0.0))
+    assert not O.quantize(x, a, O.ROUND_NEAREST).any()
+    assert not O.quantize(x, a, O.ROUND_STOCHASTIC, key=(3, 4)).any()
+    b = F32(2.0 ** -99)
+    s, inv = O.scale_pair(b)
+    assert np.isfinite(inv) and s == b / F32(127.0)
