@@ -28,7 +28,11 @@ constexpr int TC_THREADS = 192;
 constexpr uint32_t TC_A_BYTES = TC_BM * TC_BKB;      // 16 KiB
 constexpr uint32_t TC_B_BYTES = TC_BN * TC_BKB;      // 32 KiB
 constexpr uint32_t TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
-constexpr uint32_t TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int TC_STG_PITCH = 36;                       // floats per staged row (32 + 4: 16-byte aligned, conflict-free)
+constexpr uint32_t TC_STG_BYTES = 32 * TC_STG_PITCH * 4;  // one 32 x 32 FP32 staging patch per epilogue warp
+constexpr uint32_t TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 4 * TC_STG_BYTES;
+constexpr int TC_PREFETCH_KB = 8;                      // W tile is prefetched into L2 this many k-blocks before the epilogue
+constexpr int TC_GROUP_M = 16;                          // tile rows per rasterisation group (L2 reuse)
 constexpr uint32_t TC_TMEM_COLS = 512;
 constexpr unsigned long long TC_WAIT_NS = 2000000000ull;  // 2 s bound on every wait
 
@@ -103,6 +107,9 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
                "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "r"(z)
                : "memory");
 }
+__device__ __forceinline__ void l2_prefetch(const void* gptr, uint32_t bytes) {  // 16-byte aligned, multiple of 16
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -148,6 +155,16 @@ __host__ __device__ constexpr uint32_t make_idesc_i8(bool a_mn_major, bool b_mn_
          ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
+// Tile order: groups of TC_GROUP_M tile rows, column by column inside a group, so that the CTAs
+// running at one time share a small set of operand row / column panels in L2.
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
+  const int per_group = TC_GROUP_M * tiles_n;
+  const int g = tile / per_group, r = tile - g * per_group;
+  const int rows = min(TC_GROUP_M, tiles_m - g * TC_GROUP_M);
+  tm = g * TC_GROUP_M + r % rows;
+  tn = r / rows;
+}
+
 // ---- kernel --------------------------------------------------------------------------------
 template <int MODE, bool MN_MAJOR>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -164,6 +181,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   const uint32_t bar_tempty = bar_tfull + 16;                    // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_STAGES + 4);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* stage_all = reinterpret_cast<float*>(ring_ptr + TC_STAGES * TC_STAGE_BYTES + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int ACC_STAGES = (MODE == TC_MODE_UPD || MN_MAJOR) ? 1 : 2;
@@ -198,7 +216,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       uint32_t it = 0;  // running k-block counter (ring position)
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+        int tm, tn;
+        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
         for (int pass = 0; pass < p.npass && ok; ++pass) {
           for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
             const uint32_t s = it % TC_STAGES, ph = (it / TC_STAGES) & 1u;
@@ -207,6 +226,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               break;
             }
             const uint32_t a_dst = ring + s * TC_STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
+            if (MODE == TC_MODE_UPD && pass == p.npass - 1 && kb == max(0, p.kblocks - TC_PREFETCH_KB)) {
+              // pull this tile's W rows into L2 shortly before the epilogue's read-modify-write
+              const int c0w = tn * TC_BN;
+              const int ncols = min(TC_BN, p.out_cols - c0w);
+              if ((p.out_cols & 3) == 0 && ncols > 0) {
+                const int nrows = min(TC_BM, p.out_rows - tm * TC_BM);
+                for (int r = 0; r < nrows; ++r)
+                  l2_prefetch(p.W + (size_t)(tm * TC_BM + r) * p.out_cols + c0w, (uint32_t)ncols * 4u);
+              }
+            }
             mbar_expect_tx(bar_full + 8 * s, TC_STAGE_BYTES);
             if (!MN_MAJOR) {
               tma_load_2d(a_dst, &tmA, bar_full + 8 * s, kb * TC_BKB, tm * TC_BM);
@@ -275,6 +304,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   } else {
     // ------------------------------- epilogue (warps 2..5) ----------------------------------
     const int quad = warp & 3;  // TMEM lane quadrant this warp may read
+    float* stg = stage_all + (warp - 2) * (32 * TC_STG_PITCH);
     uint32_t tile_it = 0;
     bool ok = true;
     float c0 = 0.f, c1 = 0.f, cP = 0.f, cN = 0.f;
@@ -288,7 +318,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       cN = __fmul_rn(scale_of(p.absmax[4]), scale_of(p.absmax[1]));
     }
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
-      const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+      int tm, tn;
+      tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
       const uint32_t as = tile_it % ACC_STAGES, aph = (tile_it / ACC_STAGES) & 1u;
       if (!mbar_wait(bar_tfull + 8 * as, aph, abort_flag)) {
         ok = false;
@@ -316,42 +347,56 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           }
         }
       } else if (MODE == TC_MODE_FWD) {
+        // thread = one accumulator row; y staged through smem so that global stores are row-contiguous
         const float c = row < p.rows_per_pass ? c0 : c1;
         unsigned long long ssum = 0ull;
         int mx = 0;
+        const int wrow0 = tm * TC_BM + quad * 32;  // first output row of this warp
         for (int cb = 0; cb < TC_BN; cb += 32) {
           if (col0 + cb >= p.out_cols) break;  // uniform across the warp
           int v[32];
           tc_ld32(t_row + as * TC_BN + cb, v);
-          if (row_ok) {
-            const size_t o = (size_t)row * p.out_cols + col0 + cb;
-            const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
+          const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              float y[4];
+          for (int j = 0; j < 32; j += 4) {
+            float y[4];
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const int a = v[j + q];
-                y[q] = dequant_relu(a, c);
-                if (full || col0 + cb + j + q < p.out_cols) {
-                  const int rl = max(a, 0);
-                  ssum += (unsigned long long)((long long)rl * (long long)rl);
-                  mx = max(mx, rl);
-                }
+            for (int q = 0; q < 4; ++q) {
+              const int a = v[j + q];
+              y[q] = dequant_relu(a, c);
+              if (full || col0 + cb + j + q < p.out_cols) {
+                const int rl = max(a, 0);
+                ssum += (unsigned long long)((long long)rl * (long long)rl);
+                mx = max(mx, rl);
               }
+            }
+            *reinterpret_cast<float4*>(stg + lane * TC_STG_PITCH + j) = make_float4(y[0], y[1], y[2], y[3]);
+          }
+          __syncwarp();
+          // lanes 0..7 of each quarter-warp cover one staged row: 4 rows x 128 bytes per store instruction
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 4 + (lane >> 3), cc = (lane & 7) * 4;
+            const int grow = wrow0 + r, gcol = col0 + cb + cc;
+            if (grow < p.out_rows) {
+              const float4 yv = *reinterpret_cast<const float4*>(stg + r * TC_STG_PITCH + cc);
+              float* dst = p.Y + (size_t)grow * p.out_cols + gcol;
               if (full) {
-                *reinterpret_cast<float4*>(p.Y + o + j) = make_float4(y[0], y[1], y[2], y[3]);
-                if (p.acc_dump) *reinterpret_cast<int4*>(p.acc_dump + o + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                *reinterpret_cast<float4*>(dst) = yv;
               } else {
+                const float yy[4] = {yv.x, yv.y, yv.z, yv.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                  if (col0 + cb + j + q < p.out_cols) {
-                    p.Y[o + j + q] = y[q];
-                    if (p.acc_dump) p.acc_dump[o + j + q] = v[j + q];
-                  }
+                  if (gcol + q < p.out_cols) dst[q] = yy[q];
               }
             }
           }
+          if (p.acc_dump && row_ok) {  // parity dump: plain per-row stores
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + cb + j < p.out_cols) p.acc_dump[(size_t)row * p.out_cols + col0 + cb + j] = v[j];
+          }
+          __syncwarp();
         }
         if (row_ok && mx > 0) {
           const int sample = row / p.rows_per_sample;
@@ -359,44 +404,68 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           atomicMax(p.rowmax + sample, mx);
         }
       } else {  // TC_MODE_UPD
+        // thread = one accumulator row computes d = lr*(float(accP)*cP + float(accN)*cN); d is staged
+        // through smem so that the read-modify-write of W is row-contiguous
+        const int wrow0 = tm * TC_BM + quad * 32;
+        const size_t plane = (size_t)p.out_rows * p.out_cols;
         for (int cb = 0; cb < TC_BN; cb += 32) {
           if (col0 + cb >= p.out_cols) break;
+          const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
+          // issue the (row-contiguous) W loads first so that they are in flight during the TMEM reads
+          float4 wv[8];
+          if (full) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int grow = wrow0 + i * 4 + (lane >> 3);
+              if (grow < p.out_rows)
+                wv[i] = *reinterpret_cast<const float4*>(p.W + (size_t)grow * p.out_cols + col0 + cb + (lane & 7) * 4);
+            }
+          }
           int vp[32], vn[32];
           tc_ld32(t_row + cb, vp);
           tc_ld32(t_row + TC_BN + cb, vn);
-          if (row_ok) {
-            const size_t o = (size_t)row * p.out_cols + col0 + cb;
-            const size_t plane = (size_t)p.out_rows * p.out_cols;
-            const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
+          for (int j = 0; j < 32; j += 4) {
+            float d[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float g = __fadd_rn(__fmul_rn(__int2float_rn(vp[j + q]), cP), __fmul_rn(__int2float_rn(vn[j + q]), cN));
+              d[q] = __fmul_rn(p.lr, g);
+            }
+            *reinterpret_cast<float4*>(stg + lane * TC_STG_PITCH + j) = make_float4(d[0], d[1], d[2], d[3]);
+          }
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 4 + (lane >> 3), cc = (lane & 7) * 4;
+            const int grow = wrow0 + r, gcol = col0 + cb + cc;
+            if (grow < p.out_rows) {
+              const float4 dv = *reinterpret_cast<const float4*>(stg + r * TC_STG_PITCH + cc);
+              float* dst = p.W + (size_t)grow * p.out_cols + gcol;
               if (full) {
-                float4 w = *reinterpret_cast<const float4*>(p.W + o + j);
-                float wv[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const float g = __fadd_rn(__fmul_rn(__int2float_rn(vp[j + q]), cP), __fmul_rn(__int2float_rn(vn[j + q]), cN));
-                  wv[q] = __fsub_rn(wv[q], __fmul_rn(p.lr, g));
-                }
-                *reinterpret_cast<float4*>(p.W + o + j) = make_float4(wv[0], wv[1], wv[2], wv[3]);
-                if (p.accW_dump) {
-                  *reinterpret_cast<int4*>(p.accW_dump + o + j) = make_int4(vp[j], vp[j + 1], vp[j + 2], vp[j + 3]);
-                  *reinterpret_cast<int4*>(p.accW_dump + plane + o + j) = make_int4(vn[j], vn[j + 1], vn[j + 2], vn[j + 3]);
-                }
+                float4 w = wv[i];
+                w.x = __fsub_rn(w.x, dv.x);
+                w.y = __fsub_rn(w.y, dv.y);
+                w.z = __fsub_rn(w.z, dv.z);
+                w.w = __fsub_rn(w.w, dv.w);
+                *reinterpret_cast<float4*>(dst) = w;
               } else {
+                const float dd[4] = {dv.x, dv.y, dv.z, dv.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                  if (col0 + cb + j + q < p.out_cols) {
-                    const float g = __fadd_rn(__fmul_rn(__int2float_rn(vp[j + q]), cP), __fmul_rn(__int2float_rn(vn[j + q]), cN));
-                    p.W[o + j + q] = __fsub_rn(p.W[o + j + q], __fmul_rn(p.lr, g));
-                    if (p.accW_dump) {
-                      p.accW_dump[o + j + q] = vp[j + q];
-                      p.accW_dump[plane + o + j + q] = vn[j + q];
-                    }
-                  }
+                  if (gcol + q < p.out_cols) dst[q] = __fsub_rn(dst[q], dd[q]);
               }
             }
           }
+          if (p.accW_dump && row_ok) {  // parity dump
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + cb + j < p.out_cols) {
+                p.accW_dump[(size_t)row * p.out_cols + col0 + cb + j] = vp[j];
+                p.accW_dump[plane + (size_t)row * p.out_cols + col0 + cb + j] = vn[j];
+              }
+          }
+          __syncwarp();
         }
       }
       // accumulator stage drained: hand it back to the MMA issuer
