@@ -5,10 +5,10 @@
 
 A step is one pass of the whole hot path (quantise -> INT8 GEMM -> goodness -> loss -> dH ->
 quantise -> INT8 dW GEMM -> update) over one batch of seeded synthetic input.  The default
-workload is the task's largest single-GPU configuration ("roofline": one 8192 -> 8192 FF layer,
+workload is the largest single-GPU configuration ("roofline": one 8192 -> 8192 FF layer,
 16384 positive + 16384 negative samples), the one the GEMM-roofline target is quoted on.
-Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs the same per-GPU batch on its
-own GPU (independent batches, no data-path collective: weak scaling).
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank trains its own replica on its own
+batches (no data-path collective: weak scaling); the time is the maximum over ranks.
 
 --impl reference times the CPU oracle (oracle/) on the host cores on a bounded sample of the
 same workload; it is a deliberately plain program, not a target.
@@ -33,6 +33,8 @@ from paper_2506_22771_b200 import synth  # noqa: E402
 
 METRIC = "FF-INT8 train samples/s"
 UNIT = "samples/s"
+INT8_TO_BF16 = 2.0          # nominal dense tensor ratio (4.5 : 2.25 PFLOP/s)
+BURST_SECONDS = 2.0         # timed regions shorter than this are compared with the burst GEMM peak
 
 
 def _peaks():
@@ -58,7 +60,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -67,9 +69,9 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append(line.strip())
+            self.rows.append((time.time(), line.strip()))
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -77,22 +79,61 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             pass
-        sm, smax, reasons = [], [], set()
+        sm, smax, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for t, r in self.rows:
+            if t_begin is not None and not (t_begin <= t <= t_end + 0.05):
+                continue
             f = [x.strip() for x in r.split(",")]
             if len(f) < 7:
                 continue
             try:
                 sm.append(float(f[0]))
                 smax.append(float(f[1]))
+                power.append(float(f[2]))
             except ValueError:
                 continue
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def whole_job_throughput(ms_local: float, units_local: float, device=None):
+    """(max over ranks of the local time, units of all ranks / that time).  Uses the default
+    process group when one is initialised (NCCL on GPUs, gloo in the CPU tests)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms_local, units_local / (ms_local * 1e-3)
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item()) / (float(t.item()) * 1e-3)
+
+
+def algorithmic_work(w, B: int):
+    """Algorithmic bytes (memory-bound kernels) and INT8 ops (contractions) of ONE train step, per
+    kernel kind, from the layer shapes: absmax reads 4 B/element, the quantisers read 4 B and write
+    1 B per element, a contraction does 2*rows*N*K operations."""
+    out = {k: 0.0 for k in ("absmax", "quantize", "normalize", "dh_quantize", "fwd_gemm", "upd_gemm")}
+    for i, l in enumerate(w.layers):
+        R = l.H * l.Wd
+        rows = 2 * B * R
+        kin = l.Cin if l.kind == 1 else l.K
+        n_w = l.N * l.K
+        n_x = rows * kin
+        n_y = rows * l.N
+        out["absmax"] += 4.0 * n_w + (4.0 * n_x if i == 0 else 0.0)
+        out["quantize"] += 5.0 * n_w + (5.0 * n_x if i == 0 else 0.0)
+        if i + 1 < len(w.layers):
+            out["normalize"] += 5.0 * n_y            # reads Y, writes the next layer's INT8 input
+        out["dh_quantize"] += 5.0 * n_y
+        out["fwd_gemm"] += 2.0 * rows * l.N * l.K
+        out["upd_gemm"] += 2.0 * rows * l.N * l.K
+    return out
 
 
 def _oracle_step_time(w, B_sample: int, steps: int, seed: int = 1):
@@ -123,16 +164,15 @@ def run_reference(args):
         return
     w = synth.workload(args.workload)
     B_sample = min(w.B, args.cpu_sample)
-    for _ in range(args.warmup if args.warmup < 2 else 1):
-        _oracle_step_time(w, B_sample, 1)
+    _oracle_step_time(w, B_sample, 1)
     steps = max(1, min(args.steps, 3))
     t, cores = _oracle_step_time(w, B_sample, steps)
     v = B_sample / t
     sample = f"{B_sample} positive + {B_sample} negative samples of the {args.workload} workload per step, full layer widths"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int8", "data": "synthetic", "config": {"workload": args.workload, "B": B_sample},
+        "warmup": 1, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8", "data": "synthetic", "config": {"workload": args.workload, "B_pos": B_sample, "B_neg": B_sample},
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
@@ -140,20 +180,19 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="roofline")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-sample", type=int, default=256, help="positives per step of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--B", type=int, default=0, help="override positives per batch (parity / profiling runs)")
+    ap.add_argument("--B", type=int, default=0, help="override positives per batch (profiling runs on a smaller case)")
+    ap.add_argument("--tensor-form", type=int, default=0, help="CTAs per tensor-core tile: 0 auto, 1, 2")
     args = ap.parse_args()
-    if args.warmup < 3 and args.impl == "ours":
-        args.warmup = max(args.warmup, 1)
-
     if args.impl == "reference":
         return run_reference(args)
+    args.warmup = max(args.warmup, 3)
 
     import torch
     import torch.distributed as dist
@@ -174,6 +213,7 @@ def main():
     seed = 1 + rank
     descs = [ffb.make_desc(l, i, seed) for i, l in enumerate(w.layers)]
     ctx = ffb.Context(descs, B, local)
+    ffb.ff_set_tensor_form(ctx.ctx, args.tensor_form)
     bufs = [ffb.LayerBuffers(d, B, dev, dumps=False, xnext=False, own_x=(i == 0)) for i, d in enumerate(descs)]
     Ws = synth.make_weights(w, seed)
     for b, W in zip(bufs, Ws):
@@ -185,6 +225,7 @@ def main():
     bufs_arr = (ffb.ff_layer_bufs * len(descs))(*[b.struct for b in bufs])
     stream = torch.cuda.current_stream().cuda_stream
     n_layers = len(descs)
+    last = n_layers - 1
 
     def step(i):
         ffb.ff_train_step(ctx.ctx, descs_arr, bufs_arr, n_layers, B, w.lam_per_step * i, i, stream)
@@ -198,7 +239,7 @@ def main():
         for b, W in zip(bufs, W0):
             b.W.copy_(W)
 
-    # ---------------- device-resident timing (value) ----------------
+    # ---------------- device-resident timing (value), per-kernel events inside the same region --------
     for i in range(args.warmup):
         step(i)
     ffb.ff_poll_status(ctx.ctx, stream)
@@ -209,37 +250,22 @@ def main():
         time.sleep(0.3)
     barrier()
     l0 = ffb.ff_launch_count(ctx.ctx)
+    ffb.ff_profile_start(ctx.ctx)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin = time.time()
     e0.record()
     for i in range(args.steps):
         step(i)
     e1.record()
     barrier()
+    t_end = time.time()
+    kernel_ms = ffb.ff_profile_stop(ctx.ctx, stream)
     launches = ffb.ff_launch_count(ctx.ctx) - l0
-    ms = e0.elapsed_time(e1)
-    clocks = sampler.stop() if rank == 0 else None
+    ms_local = e0.elapsed_time(e1)
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     ffb.ff_poll_status(ctx.ctx, stream)
-    loss_last = float(bufs[0].loss[0].item())
-
-    # ---------------- dominant kernel: the weight-gradient GEMM + update (one launch per call) ---------
-    reset_weights()
-    step(0)
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    evf = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    last = n_layers - 1
-    for i in range(args.steps):
-        evf[i][0].record()
-        ffb.ff_layer_forward(ctx.ctx, descs[0], bufs[0].struct, B, i, stream) if n_layers == 1 else step(i)
-        evf[i][1].record()
-        if n_layers == 1:
-            ffb.ff_layer_loss_grad(ctx.ctx, descs[0], bufs[0].struct, B, [], [], 0.0, i, stream)
-        ev[i][0].record()
-        ffb.ff_layer_update(ctx.ctx, descs[last], bufs[last].struct, B, stream)
-        ev[i][1].record()
-    torch.cuda.synchronize()
-    upd_ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
-    fwd_ms = float(np.mean([a.elapsed_time(b) for a, b in evf]))
-    ffb.ff_poll_status(ctx.ctx, stream)
+    loss_last = float(bufs[last].loss[0].item())
+    ms, value = whole_job_throughput(ms_local, B * args.steps, dev)
 
     # ---------------- end to end: host buffers, H2D of the batch + D2H of the loss every step ---------
     e2e = None
@@ -256,41 +282,50 @@ def main():
             torch.cuda.current_stream().synchronize()
         e1.record()
         barrier()
-        ms_e2e = e0.elapsed_time(e1)
-        e2e_ms = ms_e2e
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": world * B * n_e2e / (e2e_ms * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": int(X_host.numel() * 4), "d2h_bytes_per_step": 16, "steps": n_e2e}
-
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+        _, e2e_value = whole_job_throughput(e0.elapsed_time(e1), B * n_e2e, dev)
+        e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(X_host.numel() * 4),
+               "d2h_bytes_per_step": 16, "steps": n_e2e}
 
     if rank == 0:
         peaks = _peaks()
+        work = algorithmic_work(w, B)
+        burst = ms * 1e-3 < BURST_SECONDS
+        bf16 = peaks["bf16_burst"] if burst else peaks["bf16_sustained"]
+        int8_peak = INT8_TO_BF16 * bf16
+        per_kernel = {}
+        for k, (tot_ms, n) in kernel_ms.items():
+            ent = {"launches_per_step": n / args.steps, "ms_per_step": tot_ms / args.steps,
+                   "share": tot_ms / ms_local}
+            if k in work and work[k] > 0 and tot_ms > 0:
+                rate = work[k] * args.steps / (tot_ms * 1e-3)
+                if k.endswith("gemm"):
+                    ent.update(bound="tensor", achieved=rate / 1e12, unit="TOP/s", frac=rate / 1e12 / int8_peak)
+                else:
+                    ent.update(bound="hbm", achieved=rate / 1e9, unit="GB/s", frac=rate / 1e9 / peaks["hbm_gbs"])
+            per_kernel[k] = ent
+        gemms = [k for k in ("fwd_gemm", "upd_gemm") if k in per_kernel]
+        dom = max(gemms, key=lambda k: per_kernel[k]["ms_per_step"])
+        names = {"fwd_gemm": "tc_gemm_kernel<FWD> (forward INT8 GEMM + dequant/ReLU/goodness epilogue)",
+                 "upd_gemm": "tc_gemm_kernel<UPD> (INT8 dW GEMM of both sets + SGD epilogue)"}
         l = w.layers[-1]
-        R = l.H * l.Wd
-        ops = 2.0 * (2 * B * R) * l.N * l.K                      # INT8 ops of the weight-gradient GEMM (2*M*N*K)
-        int8_peak = 2.0 * peaks["bf16_sustained"]                # nominal INT8 : bf16 ratio = 2
-        ach = ops / (upd_ms * 1e-3) / 1e12
         out = {
-            "metric": METRIC, "value": world * B * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": {"workload": args.workload, "B_pos": B, "B_neg": B,
-                       "layers": [[x.K, x.N] for x in w.layers], "l2": "inputs larger than L2 (no flush needed)"
-                       if 2 * B * R * l.K * 4 > 126e6 else "inputs smaller than L2, not flushed"},
+                       "layers": [[x.K, x.N] for x in w.layers],
+                       "l2": "inputs larger than L2 (no flush needed)"
+                       if 2 * B * l.H * l.Wd * l.K * 4 > 126e6 else "inputs smaller than L2, not flushed"},
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "loss_last": loss_last,
-            "phases_ms": {"forward_all_kernels": fwd_ms, "update_gemm_kernel": upd_ms},
-            "roofline": {"bound": "tensor", "kernel": "tc_gemm_kernel<update> (INT8 dW GEMM + SGD epilogue)",
-                         "achieved": ach, "peak": int8_peak, "unit": "TOP/s", "frac": ach / int8_peak,
-                         "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_sustained']} TF/s)",
-                         "frac_of_burst": ach / (2.0 * peaks["bf16_burst"]), "frac_of_nominal_4500": ach / 4500.0,
+            "roofline": {"bound": "tensor", "kernel": names[dom], "achieved": per_kernel[dom]["achieved"],
+                         "peak": int8_peak, "unit": "TOP/s", "frac": per_kernel[dom]["frac"],
+                         "peak_source": f"{INT8_TO_BF16:g} x {peaks['source']} bf16 cuBLAS "
+                                        f"{'burst' if burst else 'sustained'} ({bf16} TF/s): the timed region lasted "
+                                        f"{ms * 1e-3:.2f} s",
+                         "frac_of_sustained_x2": per_kernel[dom]["achieved"] / (INT8_TO_BF16 * peaks["bf16_sustained"]),
+                         "frac_of_nominal_4500": per_kernel[dom]["achieved"] / 4500.0,
                          "traffic": None},
+            "kernels": per_kernel,
         }
         if not args.no_cpu_baseline and world == 1:
             Bs = min(B, args.cpu_sample)

@@ -117,6 +117,11 @@ ff_status ff_set_workspace(ff_ctx* ctx, void* dev_ptr, size_t bytes);
  * shapes it cannot take).  Both produce identical bits. */
 ff_status ff_set_gemm_path(ff_ctx* ctx, int path);
 
+/* The tensor-core kernels run either one CTA per 128 x 256 output tile or a pair of CTAs (tcgen05
+ * cta_group::2) per 256 x 256 tile.  ctas_per_tile = 0 chooses by problem size (pairs once the
+ * output has enough tiles to occupy every SM pair), 1 / 2 force one form.  Identical bits. */
+ff_status ff_set_tensor_form(ff_ctx* ctx, int ctas_per_tile);
+
 /* Forward of one layer (Sec. IV-B: quantise A and W, INT8 MAC with INT32 accumulation; Sec. III /
  * Alg. 1 line 6: goodness).  Reads X, W.  Writes Xq, Wq, absmax[X,W,XNEXT], Y, S, rowmax, G,
  * Xnext (if non-NULL), acc_dump (if non-NULL).  `step` keys the stochastic rounding. */
@@ -155,6 +160,26 @@ const char* ff_last_error(const ff_ctx* ctx);
 
 /* Number of kernels the library has launched through this context so far (host counter). */
 uint64_t ff_launch_count(const ff_ctx* ctx);
+
+/* Per-kernel device timing.  Between ff_profile_start and ff_profile_stop every kernel the library
+ * launches through this context is bracketed by a pair of CUDA events on its stream.
+ * ff_profile_stop synchronises `cuda_stream` and returns, per kernel kind (FF_K_*), the summed
+ * device time in milliseconds and the number of launches (host arrays of FF_K_COUNT entries). */
+enum {
+  FF_K_ABSMAX = 0,   /* per-tensor max|x| (Sec. IV, SUQ range)                                   */
+  FF_K_QUANTIZE,     /* SUQ of A or W to INT8                                                    */
+  FF_K_ZERO_STATS,   /* clears S and rowmax                                                      */
+  FF_K_FWD_GEMM,     /* forward INT8 MAC + dequantise/ReLU/goodness epilogue                     */
+  FF_K_FINALIZE,     /* G from S, range of the normalised output                                 */
+  FF_K_NORMALIZE,    /* length normalisation (+ next layer's SUQ)                                */
+  FF_K_LOSS,         /* Eq. 1-4: loss and per-sample coefficient                                 */
+  FF_K_DH_QUANTIZE,  /* g^Y to INT8                                                              */
+  FF_K_UPD_GEMM,     /* g^W INT8 MAC + SGD update epilogue                                       */
+  FF_K_RAW_GEMM,     /* ff_int8_gemm                                                             */
+  FF_K_COUNT
+};
+ff_status ff_profile_start(ff_ctx* ctx);
+ff_status ff_profile_stop(ff_ctx* ctx, void* cuda_stream, float* ms_per_kernel, uint32_t* launches_per_kernel);
 
 /* Stand-alone INT8 contraction used by the unit tests and the kernel benchmark (Sec. IV-B,
  * "integer matrix multiplication with INT8 inputs and INT32 accumulation"):

@@ -18,9 +18,12 @@ FF_GEMM_AUTO, FF_GEMM_SIMT, FF_GEMM_TENSOR = 0, 1, 2
 FF_A_X_POS, FF_A_X_NEG, FF_A_W, FF_A_DH_POS, FF_A_DH_NEG, FF_A_XNEXT_POS, FF_A_XNEXT_NEG = range(7)
 FF_ABSMAX_LEN = 8
 
-EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", "ff_set_gemm_path",
+EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", "ff_set_gemm_path", "ff_set_tensor_form",
            "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step",
-           "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm"]
+           "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
+           "ff_profile_start", "ff_profile_stop"]
+FF_K_NAMES = ["absmax", "quantize", "zero_stats", "fwd_gemm", "finalize", "normalize", "loss", "dh_quantize",
+              "upd_gemm", "raw_gemm"]
 
 
 class ff_layer_desc(C.Structure):
@@ -66,6 +69,7 @@ def load(build_if_missing: bool = True):
     lib.ff_workspace_bytes.argtypes = [C.POINTER(ff_layer_desc), i32, i32, C.POINTER(C.c_size_t)]
     lib.ff_set_workspace.argtypes = [vp, vp, C.c_size_t]
     lib.ff_set_gemm_path.argtypes = [vp, i32]
+    lib.ff_set_tensor_form.argtypes = [vp, i32]
     lib.ff_layer_forward.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, u64, vp]
     lib.ff_layer_loss_grad.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32,
                                        C.POINTER(vp), C.POINTER(f32), i32, f32, u64, vp]
@@ -77,6 +81,8 @@ def load(build_if_missing: bool = True):
     lib.ff_launch_count.argtypes = [vp]
     lib.ff_launch_count.restype = u64
     lib.ff_int8_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.ff_profile_start.argtypes = [vp]
+    lib.ff_profile_stop.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(C.c_uint32)]
     for name in EXPORTS:
         if name not in ("ff_last_error", "ff_launch_count"):
             getattr(lib, name).restype = i32
@@ -117,6 +123,10 @@ def ff_set_gemm_path(ctx, path: int):
     _check(ctx, load().ff_set_gemm_path(ctx, path))
 
 
+def ff_set_tensor_form(ctx, ctas_per_tile: int):
+    _check(ctx, load().ff_set_tensor_form(ctx, ctas_per_tile))
+
+
 def ff_layer_forward(ctx, desc, bufs, B: int, step: int, stream: int = 0):
     _check(ctx, load().ff_layer_forward(ctx, C.byref(desc), C.byref(bufs), B, step, stream))
 
@@ -144,6 +154,19 @@ def ff_poll_status(ctx, stream: int = 0):
 
 def ff_launch_count(ctx) -> int:
     return int(load().ff_launch_count(ctx))
+
+
+def ff_profile_start(ctx):
+    _check(ctx, load().ff_profile_start(ctx))
+
+
+def ff_profile_stop(ctx, stream: int = 0):
+    """Returns {kernel kind: (total ms, launches)} for the kinds that were launched."""
+    n = len(FF_K_NAMES)
+    ms = (C.c_float * n)()
+    cnt = (C.c_uint32 * n)()
+    _check(ctx, load().ff_profile_stop(ctx, stream, ms, cnt))
+    return {FF_K_NAMES[i]: (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i]}
 
 
 def ff_int8_gemm(ctx, A: int, B: int, Cptr: int, M: int, N: int, K: int, trans: int, stream: int = 0):

@@ -64,41 +64,49 @@ __device__ __forceinline__ uint32_t pair_hash(uint32_t pair, RoundKey key) {
   return h;
 }
 // u in [0,1) with 16 random bits: low half of the pair hash for even indices, high half for odd.
+// u = half16 * 2^-16, formed without an integer-to-float conversion: the float 1.m with the 16 bits
+// at the top of the mantissa is 1 + half16*2^-16, and subtracting 1 is exact.
 __device__ __forceinline__ float u_from_half(uint32_t half16) {
-  return __fmul_rn(__uint2float_rn(half16), 1.52587890625e-05f);  // * 2^-16, exact
+  return __fsub_rn(__uint_as_float(0x3F800000u | (half16 << 7)), 1.0f);
 }
 
-__device__ __forceinline__ int round_clip(float t, float u, int mode) {
-  float r = (mode == ROUND_NEAREST) ? rintf(t) : floorf(__fadd_rn(t, u));
-  r = fminf(fmaxf(r, -127.0f), 127.0f);
-  return __float2int_rn(r);
+// rint(t) (ties to even) or floor(t+u), then clip to [-127, 127].  The float-to-int conversion does
+// the rounding (|t| stays far inside the int range: |x| <= a gives |t| <= 127 up to one rounding).
+// MODE is a compile-time constant so that only one conversion is issued per element.
+template <int MODE>
+__device__ __forceinline__ int round_clip(float t, float u) {
+  const int r = (MODE == ROUND_NEAREST) ? __float2int_rn(t) : __float2int_rd(__fadd_rn(t, u));
+  return min(max(r, -127), 127);
 }
 
 // Quantise two neighbouring elements (even linear index idx_even and idx_even+1).
-__device__ __forceinline__ void quant_pair(float x0, float x1, float inv, int mode, uint32_t idx_even,
-                                           RoundKey key, int& q0, int& q1) {
+template <int MODE>
+__device__ __forceinline__ void quant_pair(float x0, float x1, float inv, uint32_t idx_even, RoundKey key, int& q0, int& q1) {
   float u0 = 0.0f, u1 = 0.0f;
-  if (mode != ROUND_NEAREST) {
-    uint32_t h = pair_hash(idx_even >> 1, key);
+  if (MODE != ROUND_NEAREST) {
+    const uint32_t h = pair_hash(idx_even >> 1, key);
     u0 = u_from_half(h & 0xFFFFu);
     u1 = u_from_half(h >> 16);
   }
-  q0 = round_clip(__fmul_rn(x0, inv), u0, mode);
-  q1 = round_clip(__fmul_rn(x1, inv), u1, mode);
+  q0 = round_clip<MODE>(__fmul_rn(x0, inv), u0);
+  q1 = round_clip<MODE>(__fmul_rn(x1, inv), u1);
 }
 // Quantise one element at an arbitrary linear index.
-__device__ __forceinline__ int quant_one(float x, float inv, int mode, uint32_t idx, RoundKey key) {
+template <int MODE>
+__device__ __forceinline__ int quant_one(float x, float inv, uint32_t idx, RoundKey key) {
   float u = 0.0f;
-  if (mode != ROUND_NEAREST) {
-    uint32_t h = pair_hash(idx >> 1, key);
+  if (MODE != ROUND_NEAREST) {
+    const uint32_t h = pair_hash(idx >> 1, key);
     u = u_from_half((idx & 1u) ? (h >> 16) : (h & 0xFFFFu));
   }
-  return round_clip(__fmul_rn(x, inv), u, mode);
+  return round_clip<MODE>(__fmul_rn(x, inv), u);
 }
 
+// Low bytes of four ints as one little-endian word (three byte permutes).
 __device__ __forceinline__ uint32_t pack4(int q0, int q1, int q2, int q3) {
-  return (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) |
-         ((uint32_t)(q3 & 0xFF) << 24);
+  const uint32_t lo = __byte_perm((uint32_t)q0, (uint32_t)q1, 0x0040);
+  const uint32_t hi = __byte_perm((uint32_t)q2, (uint32_t)q3, 0x0040);
+  return __byte_perm(lo, hi, 0x5410);
 }
 
 __device__ __forceinline__ float dequant_relu(int acc, float c) {

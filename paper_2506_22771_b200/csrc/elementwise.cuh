@@ -42,6 +42,7 @@ __global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restr
   if (vec) {
     const uint4* x4 = reinterpret_cast<const uint4*>(xp);
     size_t n4 = n_per_pass >> 2;
+#pragma unroll 4
     for (size_t i = tid; i < n4; i += stride) {
       uint4 v = __ldg(x4 + i);
       m = max(m, max(max(v.x & 0x7fffffffu, v.y & 0x7fffffffu), max(v.z & 0x7fffffffu, v.w & 0x7fffffffu)));
@@ -61,9 +62,10 @@ __global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restr
 // Linear element index (over the whole tensor) keys the stochastic rounding.
 // grid = (blocks, passes)
 // ---------------------------------------------------------------------------------------------
+template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __restrict__ x, int8_t* __restrict__ q,
                                                               size_t n_per_pass, const float* __restrict__ a,
-                                                              int mode, RoundKey key) {
+                                                              RoundKey key) {
   const size_t base = (size_t)blockIdx.y * n_per_pass;
   const float* xp = x + base;
   int8_t* qp = q + base;
@@ -75,17 +77,18 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __res
     const float4* x4 = reinterpret_cast<const float4*>(xp);
     uint32_t* q4 = reinterpret_cast<uint32_t*>(qp);
     size_t n4 = n_per_pass >> 2;
+#pragma unroll 4
     for (size_t i = tid; i < n4; i += stride) {
       float4 v = __ldg(x4 + i);
       uint32_t idx = (uint32_t)(base + (i << 2));
       int q0, q1, q2, q3;
-      quant_pair(v.x, v.y, inv, mode, idx, key, q0, q1);
-      quant_pair(v.z, v.w, inv, mode, idx + 2, key, q2, q3);
+      quant_pair<MODE>(v.x, v.y, inv, idx, key, q0, q1);
+      quant_pair<MODE>(v.z, v.w, inv, idx + 2, key, q2, q3);
       q4[i] = pack4(q0, q1, q2, q3);
     }
   } else {
     for (size_t i = tid; i < n_per_pass; i += stride)
-      qp[i] = (int8_t)quant_one(xp[i], inv, mode, (uint32_t)(base + i), key);
+      qp[i] = (int8_t)quant_one<MODE>(xp[i], inv, (uint32_t)(base + i), key);
   }
 }
 
@@ -117,28 +120,53 @@ __global__ void __launch_bounds__(EW_THREADS) finalize_goodness_kernel(
   }
 }
 
+// The per-sample passes below stream float4 groups with a grid-stride loop.  The sample a group
+// belongs to is tracked incrementally (one division per thread at the start, none per element):
+// advancing by `stride` groups adds stride / g4 samples and stride % g4 groups, with one carry.
+struct SampleCursor {
+  uint32_t sample, offset;      // current sample (within the pass) and float4 group inside it
+  uint32_t step_q, step_r, g4;  // stride / g4, stride % g4, groups per sample
+  __device__ __forceinline__ SampleCursor(uint32_t first_group, uint32_t stride, uint32_t groups_per_sample) {
+    g4 = groups_per_sample;
+    sample = first_group / g4;
+    offset = first_group - sample * g4;
+    step_q = stride / g4;
+    step_r = stride - step_q * g4;
+  }
+  __device__ __forceinline__ void advance() {
+    sample += step_q;
+    offset += step_r;
+    if (offset >= g4) {
+      offset -= g4;
+      ++sample;
+    }
+  }
+};
+
 // ---------------------------------------------------------------------------------------------
 // Length normalisation x = y * tau/(sqrt(G)+eps) per sample, written as FP32 (xnext, nullable)
 // and / or quantised straight to the next layer's INT8 input (xq, nullable) with per-pass range
 // a[p].  per_sample = R*N elements per sample; per_pass = B*per_sample.   grid = (blocks, 2)
 // ---------------------------------------------------------------------------------------------
+template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __restrict__ Y, const float* __restrict__ G,
                                                                float tau, float eps, size_t per_sample,
                                                                size_t per_pass, float* __restrict__ xnext,
                                                                int8_t* __restrict__ xq, const float* __restrict__ a,
-                                                               int mode, RoundKey key) {
+                                                               RoundKey key) {
   const size_t base = (size_t)blockIdx.y * per_pass;
   const float inv = xq ? inv_of(a[blockIdx.y]) : 0.0f;
-  size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  size_t stride = (size_t)gridDim.x * blockDim.x;
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) &&
                    (!xnext || (((uintptr_t)xnext) & 15) == 0) && (!xq || (((uintptr_t)xq) & 3) == 0);
+  const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
   if (vec) {
-    size_t n4 = per_pass >> 2;
-    for (size_t i = tid; i < n4; i += stride) {
-      size_t e = base + (i << 2);
-      float g = __ldg(G + (uint32_t)e / (uint32_t)per_sample);
-      float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(g), eps));
+    const uint32_t n4 = (uint32_t)(per_pass >> 2);
+    const float* Gp = G + (uint32_t)(base / per_sample);
+    SampleCursor cur(tid, stride, (uint32_t)(per_sample >> 2));
+#pragma unroll 4
+    for (uint32_t i = tid; i < n4; i += stride, cur.advance()) {
+      const size_t e = base + ((size_t)i << 2);
+      const float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(__ldg(Gp + cur.sample)), eps));
       float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
       v.x = __fmul_rn(v.x, r);
       v.y = __fmul_rn(v.y, r);
@@ -147,8 +175,8 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
       if (xnext) *reinterpret_cast<float4*>(xnext + e) = v;
       if (xq) {
         int q0, q1, q2, q3;
-        quant_pair(v.x, v.y, inv, mode, (uint32_t)e, key, q0, q1);
-        quant_pair(v.z, v.w, inv, mode, (uint32_t)e + 2, key, q2, q3);
+        quant_pair<MODE>(v.x, v.y, inv, (uint32_t)e, key, q0, q1);
+        quant_pair<MODE>(v.z, v.w, inv, (uint32_t)e + 2, key, q2, q3);
         *reinterpret_cast<uint32_t*>(xq + e) = pack4(q0, q1, q2, q3);
       }
     }
@@ -159,7 +187,7 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
       float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(g), eps));
       float v = __fmul_rn(Y[e], r);
       if (xnext) xnext[e] = v;
-      if (xq) xq[e] = (int8_t)quant_one(v, inv, mode, (uint32_t)e, key);
+      if (xq) xq[e] = (int8_t)quant_one<MODE>(v, inv, (uint32_t)e, key);
     }
   }
 }
@@ -202,15 +230,25 @@ struct LaterLayers {
 // Loss (Eq. 1, Eq. 2), look-ahead loss (Eq. 3) and the per-sample coefficient of Eq. 4 under the
 // scalar-coefficient reading: coef_m = (g'_l,m + lambda * sum_{j>l} g'_j,m)/M with g' = dL/dG.
 // Also the per-pass absmax of dH = 2*coef*y via the per-sample max of relu(acc).
-// One block (M is at most a few 10^4 samples); fixed-order tree reduction for the loss.
+// Several blocks; each leaves its partial loss sum and maxima in `scratch`, and the block that
+// finishes last (ticket counter) combines them in block order, so the loss is reproducible and
+// nothing has to be zeroed beforehand.  scratch: LossScratch, ticket zero on entry and on exit.
 // ---------------------------------------------------------------------------------------------
-constexpr int LOSS_THREADS = 1024;
+constexpr int LOSS_THREADS = 256;
+constexpr int LOSS_MAX_BLOCKS = 256;
+struct LossScratch {
+  unsigned int ticket;
+  unsigned int pad[3];
+  double lsum[LOSS_MAX_BLOCKS];
+  uint32_t amax[2][LOSS_MAX_BLOCKS];
+};
 __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __restrict__ G, float theta, LaterLayers later,
                                                                  float lambda, int B, const int32_t* __restrict__ rowmax,
                                                                  float* __restrict__ absmax, float* __restrict__ coef,
-                                                                 float* __restrict__ loss) {
+                                                                 float* __restrict__ loss, LossScratch* __restrict__ scratch) {
   __shared__ double red[LOSS_THREADS / 32];
   __shared__ uint32_t redmax[2][LOSS_THREADS / 32];
+  __shared__ bool is_last;
   const int M = 2 * B;
   const double lam = (double)lambda;
   const double inv_m = __ddiv_rn(1.0, (double)M);
@@ -218,7 +256,7 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
   const float cpass[2] = {__fmul_rn(scale_of(absmax[0]), s_w), __fmul_rn(scale_of(absmax[1]), s_w)};
   double lsum = 0.0;
   uint32_t amax[2] = {0u, 0u};
-  for (int m = threadIdx.x; m < M; m += LOSS_THREADS) {
+  for (int m = blockIdx.x * LOSS_THREADS + threadIdx.x; m < M; m += gridDim.x * LOSS_THREADS) {
     const int p = m >= B;
     const double sign = p ? 1.0 : -1.0;
     double arg = __dmul_rn(sign, __dsub_rn((double)G[m], (double)theta));
@@ -237,7 +275,7 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
     float d = fabsf(__fmul_rn(k2, __fmul_rn(__int2float_rn(rowmax[m]), cpass[p])));
     amax[p] = max(amax[p], __float_as_uint(d));
   }
-  // block reductions (fixed order)
+  // block reduction (fixed order)
   for (int o = 16; o > 0; o >>= 1) lsum += __shfl_down_sync(0xffffffffu, lsum, o);
   amax[0] = warp_max_u32(amax[0]);
   amax[1] = warp_max_u32(amax[1]);
@@ -248,9 +286,30 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
     redmax[1][w] = amax[1];
   }
   __syncthreads();
-  if (w == 0) {
-    double v = red[lane];
-    uint32_t a0 = redmax[0][lane], a1 = redmax[1][lane];
+  if (threadIdx.x == 0) {
+    double v = 0.0;
+    uint32_t a0 = 0u, a1 = 0u;
+    for (int i = 0; i < LOSS_THREADS / 32; ++i) {
+      v += red[i];
+      a0 = max(a0, redmax[0][i]);
+      a1 = max(a1, redmax[1][i]);
+    }
+    scratch->lsum[blockIdx.x] = v;
+    scratch->amax[0][blockIdx.x] = a0;
+    scratch->amax[1][blockIdx.x] = a1;
+    __threadfence();
+    is_last = atomicAdd(&scratch->ticket, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (is_last && threadIdx.x < 32) {
+    __threadfence();
+    double v = 0.0;
+    uint32_t a0 = 0u, a1 = 0u;
+    for (int i = lane; i < (int)gridDim.x; i += 32) {
+      v += __ldcg(&scratch->lsum[i]);
+      a0 = max(a0, __ldcg(&scratch->amax[0][i]));
+      a1 = max(a1, __ldcg(&scratch->amax[1][i]));
+    }
     for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
     a0 = warp_max_u32(a0);
     a1 = warp_max_u32(a1);
@@ -258,6 +317,7 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
       loss[0] = (float)(v * inv_m);
       absmax[3] = __uint_as_float(a0);
       absmax[4] = __uint_as_float(a1);
+      scratch->ticket = 0u;  // ready for the next launch on this stream
     }
   }
 }
@@ -265,31 +325,33 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
 // ---------------------------------------------------------------------------------------------
 // dHq = clip(round((2*coef_m * y) * 127/a_dh[p])).  grid = (blocks, 2)
 // ---------------------------------------------------------------------------------------------
+template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) dh_quantize_kernel(const float* __restrict__ Y, const float* __restrict__ coef,
                                                                  const float* __restrict__ absmax, size_t per_sample,
-                                                                 size_t per_pass, int8_t* __restrict__ dHq, int mode,
-                                                                 RoundKey key) {
+                                                                 size_t per_pass, int8_t* __restrict__ dHq, RoundKey key) {
   const size_t base = (size_t)blockIdx.y * per_pass;
   const float inv = inv_of(absmax[3 + blockIdx.y]);
-  size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  size_t stride = (size_t)gridDim.x * blockDim.x;
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)dHq) & 3) == 0);
+  const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
   if (vec) {
-    size_t n4 = per_pass >> 2;
-    for (size_t i = tid; i < n4; i += stride) {
-      size_t e = base + (i << 2);
-      float k2 = __fmul_rn(2.0f, __ldg(coef + (uint32_t)e / (uint32_t)per_sample));
-      float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
+    const uint32_t n4 = (uint32_t)(per_pass >> 2);
+    const float* cp = coef + (uint32_t)(base / per_sample);
+    SampleCursor cur(tid, stride, (uint32_t)(per_sample >> 2));
+#pragma unroll 4
+    for (uint32_t i = tid; i < n4; i += stride, cur.advance()) {
+      const size_t e = base + ((size_t)i << 2);
+      const float k2 = __fmul_rn(2.0f, __ldg(cp + cur.sample));
+      const float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
       int q0, q1, q2, q3;
-      quant_pair(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, mode, (uint32_t)e, key, q0, q1);
-      quant_pair(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, mode, (uint32_t)e + 2, key, q2, q3);
+      quant_pair<MODE>(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, (uint32_t)e, key, q0, q1);
+      quant_pair<MODE>(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, (uint32_t)e + 2, key, q2, q3);
       *reinterpret_cast<uint32_t*>(dHq + e) = pack4(q0, q1, q2, q3);
     }
   } else {
     for (size_t i = tid; i < per_pass; i += stride) {
       size_t e = base + i;
       float k2 = __fmul_rn(2.0f, coef[(uint32_t)e / (uint32_t)per_sample]);
-      dHq[e] = (int8_t)quant_one(__fmul_rn(k2, Y[e]), inv, mode, (uint32_t)e, key);
+      dHq[e] = (int8_t)quant_one<MODE>(__fmul_rn(k2, Y[e]), inv, (uint32_t)e, key);
     }
   }
 }

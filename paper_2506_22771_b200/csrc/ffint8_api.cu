@@ -7,6 +7,8 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <type_traits>
+#include <vector>
 
 #include "common.cuh"
 #include "elementwise.cuh"
@@ -24,12 +26,23 @@ struct ff_ctx {
   int gemm_path = FF_GEMM_AUTO;
   uint64_t launches = 0;
   TcState tc;
+  // optional per-kernel timing (ff_profile_start / ff_profile_stop)
+  bool profiling = false;
+  struct ProfRec {
+    int kid;
+    cudaEvent_t a, b;
+  };
+  std::vector<ProfRec> prof_recs;
+  std::vector<cudaEvent_t> prof_pool;
   char err[512] = {0};
 };
 
 namespace {
 
-constexpr size_t WS_STATUS_BYTES = 256;  // status word lives at the start of the workspace
+// workspace layout: [0, 256) status word (+ padding), then the loss kernel's partial-sum scratch
+constexpr size_t WS_STATUS_BYTES = 256;
+constexpr size_t WS_LOSS_OFFSET = WS_STATUS_BYTES;
+constexpr size_t WS_BYTES = (WS_LOSS_OFFSET + sizeof(LossScratch) + 255) / 256 * 256;
 
 ff_status fail(ff_ctx* ctx, ff_status st, const char* fmt, const char* a = "", long long b = 0) {
   if (ctx) snprintf(ctx->err, sizeof(ctx->err), fmt, a, b);
@@ -48,6 +61,33 @@ ff_status fail(ff_ctx* ctx, ff_status st, const char* fmt, const char* a = "", l
     cudaError_t e__ = cudaGetLastError();                                                   \
     if (e__ != cudaSuccess) return fail(ctx, FF_ERR_CUDA, "launch: %s (line %lld)", cudaGetErrorString(e__), __LINE__); \
   } while (0)
+
+// CUDA-event pair around one kernel launch while profiling is on (events come from a pool that grows
+// on the host only; nothing is allocated on the device).
+struct ProfScope {
+  ff_ctx* ctx;
+  cudaStream_t st;
+  cudaEvent_t b = nullptr;
+  ProfScope(ff_ctx* c, int kid, cudaStream_t s) : ctx(c), st(s) {
+    if (!c->profiling) return;
+    cudaEvent_t ev[2] = {nullptr, nullptr};
+    for (auto& e : ev) {
+      if (!c->prof_pool.empty()) {
+        e = c->prof_pool.back();
+        c->prof_pool.pop_back();
+      } else if (cudaEventCreate(&e) != cudaSuccess) {
+        e = nullptr;
+      }
+    }
+    if (!ev[0] || !ev[1]) return;
+    cudaEventRecord(ev[0], s);
+    b = ev[1];
+    c->prof_recs.push_back({kid, ev[0], ev[1]});
+  }
+  ~ProfScope() {
+    if (b) cudaEventRecord(b, st);
+  }
+};
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
@@ -101,7 +141,7 @@ inline uint32_t* status_ptr(ff_ctx* ctx) { return reinterpret_cast<uint32_t*>(ct
 
 ff_status ensure_status(ff_ctx* ctx, cudaStream_t st) {
   if (!ctx->status_zeroed) {
-    FF_CUDA(ctx, cudaMemsetAsync(ctx->workspace, 0, WS_STATUS_BYTES, st));
+    FF_CUDA(ctx, cudaMemsetAsync(ctx->workspace, 0, WS_BYTES, st));  // status word and the loss kernel's ticket
     ctx->status_zeroed = true;
   }
   return FF_OK;
@@ -118,6 +158,7 @@ inline int ew_blocks(ff_ctx* ctx, size_t work_items, int per_thread = 4) {
 template <class LA, class LB, bool TRANS, int NPASS, class Epi>
 ff_status launch_simt(ff_ctx* ctx, LA la, LB lb, int out_rows, int out_cols, int clen, Epi epi, cudaStream_t st) {
   dim3 grid((out_cols + SG_BN - 1) / SG_BN, (out_rows + SG_BM - 1) / SG_BM);
+  ProfScope prof(ctx, std::is_same<Epi, ForwardEpilogue>::value ? FF_K_FWD_GEMM : std::is_same<Epi, UpdateEpilogue>::value ? FF_K_UPD_GEMM : FF_K_RAW_GEMM, st);
   gemm_simt_kernel<LA, LB, TRANS, NPASS, Epi><<<grid, SG_THREADS, 0, st>>>(la, lb, clen, epi);
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -138,6 +179,7 @@ ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
   bool tc_ok = tc_forward_supported(L, B);
   if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core forward");
   if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT) {
+    ProfScope prof(ctx, FF_K_FWD_GEMM, st);
     ff_status s = tc_forward(ctx->tc, L, b, B, status_ptr(ctx), st);
     if (s != FF_OK) return fail(ctx, s, "tensor-core forward launch failed: %s", ctx->tc.err);
     ctx->launches++;
@@ -156,6 +198,7 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
   bool tc_ok = tc_update_supported(L, B);
   if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core weight gradient");
   if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT) {
+    ProfScope prof(ctx, FF_K_UPD_GEMM, st);
     ff_status s = tc_update(ctx->tc, L, b, B, status_ptr(ctx), st);
     if (s != FF_OK) return fail(ctx, s, "tensor-core weight-gradient launch failed: %s", ctx->tc.err);
     ctx->launches++;
@@ -173,31 +216,57 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
 ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint64_t step,
                           float* a_next2, cudaStream_t st) {
   const size_t nW = (size_t)L.N * L.K;
-  absmax_kernel<<<dim3(ew_blocks(ctx, nW / 4 + 1), 1), EW_THREADS, 0, st>>>(b.W, nW, b.absmax + FF_A_W, status_ptr(ctx));
+  {
+    ProfScope prof(ctx, FF_K_ABSMAX, st);
+    absmax_kernel<<<dim3(ew_blocks(ctx, nW / 4 + 1), 1), EW_THREADS, 0, st>>>(b.W, nW, b.absmax + FF_A_W, status_ptr(ctx));
+  }
   FF_LAUNCH_CHECK(ctx);
-  quantize_kernel<<<dim3(ew_blocks(ctx, nW / 4 + 1), 1), EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, L.round_w,
-                                                                           make_round_key(L.seed, ROLE_W, L.index, step));
+  {
+    ProfScope prof(ctx, FF_K_QUANTIZE, st);
+    const dim3 grid(ew_blocks(ctx, nW / 4 + 1), 1);
+    const RoundKey key = make_round_key(L.seed, ROLE_W, L.index, step);
+    if (L.round_w == FF_ROUND_NEAREST_EVEN)
+      quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, key);
+    else
+      quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, key);
+  }
   FF_LAUNCH_CHECK(ctx);
   const int M = 2 * B;
-  zero_sample_stats_kernel<<<(M + EW_THREADS - 1) / EW_THREADS, EW_THREADS, 0, st>>>(
-      reinterpret_cast<unsigned long long*>(b.S), b.rowmax, M);
+  {
+    ProfScope prof(ctx, FF_K_ZERO_STATS, st);
+    zero_sample_stats_kernel<<<(M + EW_THREADS - 1) / EW_THREADS, EW_THREADS, 0, st>>>(
+        reinterpret_cast<unsigned long long*>(b.S), b.rowmax, M);
+  }
   FF_LAUNCH_CHECK(ctx);
   ff_status s = run_forward_gemm(ctx, L, b, B, st);
   if (s != FF_OK) return s;
-  finalize_goodness_kernel<<<dim3(ew_blocks(ctx, B, 1), 2), EW_THREADS, 0, st>>>(
-      reinterpret_cast<const unsigned long long*>(b.S), b.rowmax, b.absmax, B, L.tau, L.eps, b.G, b.absmax + FF_A_XNEXT_POS,
-      a_next2);
+  {
+    ProfScope prof(ctx, FF_K_FINALIZE, st);
+    finalize_goodness_kernel<<<dim3(ew_blocks(ctx, B, 1), 2), EW_THREADS, 0, st>>>(
+        reinterpret_cast<const unsigned long long*>(b.S), b.rowmax, b.absmax, B, L.tau, L.eps, b.G,
+        b.absmax + FF_A_XNEXT_POS, a_next2);
+  }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
 
 ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint64_t step, cudaStream_t st) {
   const size_t per_pass = (size_t)B * rows_per_sample(L) * in_features(L);
-  absmax_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(b.X, per_pass, b.absmax + FF_A_X_POS,
-                                                                               status_ptr(ctx));
+  {
+    ProfScope prof(ctx, FF_K_ABSMAX, st);
+    absmax_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(b.X, per_pass, b.absmax + FF_A_X_POS,
+                                                                                 status_ptr(ctx));
+  }
   FF_LAUNCH_CHECK(ctx);
-  quantize_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(
-      b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, L.round_x, make_round_key(L.seed, ROLE_X, L.index, step));
+  {
+    ProfScope prof(ctx, FF_K_QUANTIZE, st);
+    const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
+    const RoundKey key = make_round_key(L.seed, ROLE_X, L.index, step);
+    if (L.round_x == FF_ROUND_NEAREST_EVEN)
+      quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, key);
+    else
+      quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, key);
+  }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
@@ -210,9 +279,16 @@ ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
   const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
   const size_t per_pass = per_sample * B;
   RoundKey key = next ? make_round_key(next->seed, ROLE_X, next->index, step) : RoundKey{0, 0};
-  normalize_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(
-      b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext, xq_next, b.absmax + FF_A_XNEXT_POS,
-      next ? next->round_x : 0, key);
+  {
+    ProfScope prof(ctx, FF_K_NORMALIZE, st);
+    const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
+    if (!next || next->round_x == FF_ROUND_NEAREST_EVEN)
+      normalize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
+                                                                  xq_next, b.absmax + FF_A_XNEXT_POS, key);
+    else
+      normalize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
+                                                                     xq_next, b.absmax + FF_A_XNEXT_POS, key);
+  }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
@@ -225,12 +301,26 @@ ff_status loss_grad_impl(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
     later.G[j] = G_later[j];
     later.theta[j] = theta_later[j];
   }
-  loss_coef_kernel<<<1, LOSS_THREADS, 0, st>>>(b.G, L.theta, later, lambda, B, b.rowmax, b.absmax, b.coef, b.loss);
+  int loss_blocks = (2 * B + LOSS_THREADS - 1) / LOSS_THREADS;
+  if (loss_blocks > LOSS_MAX_BLOCKS) loss_blocks = LOSS_MAX_BLOCKS;
+  {
+    ProfScope prof(ctx, FF_K_LOSS, st);
+    loss_coef_kernel<<<loss_blocks, LOSS_THREADS, 0, st>>>(
+        b.G, L.theta, later, lambda, B, b.rowmax, b.absmax, b.coef, b.loss,
+        reinterpret_cast<LossScratch*>(static_cast<char*>(ctx->workspace) + WS_LOSS_OFFSET));
+  }
   FF_LAUNCH_CHECK(ctx);
   const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
   const size_t per_pass = per_sample * B;
-  dh_quantize_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(
-      b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, L.round_dh, make_round_key(L.seed, ROLE_DH, L.index, step));
+  {
+    ProfScope prof(ctx, FF_K_DH_QUANTIZE, st);
+    const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
+    const RoundKey key = make_round_key(L.seed, ROLE_DH, L.index, step);
+    if (L.round_dh == FF_ROUND_NEAREST_EVEN)
+      dh_quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key);
+    else
+      dh_quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key);
+  }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
@@ -259,19 +349,26 @@ ff_status ff_create(ff_ctx** out, int device) {
 }
 
 ff_status ff_destroy(ff_ctx* ctx) {
+  if (ctx) {
+    for (auto& r : ctx->prof_recs) {
+      cudaEventDestroy(r.a);
+      cudaEventDestroy(r.b);
+    }
+    for (auto e : ctx->prof_pool) cudaEventDestroy(e);
+  }
   delete ctx;
   return FF_OK;
 }
 
 ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, size_t* out_bytes) {
   if (!layers || n_layers <= 0 || B <= 0 || !out_bytes) return FF_ERR_ARG;
-  *out_bytes = WS_STATUS_BYTES;
+  *out_bytes = WS_BYTES;
   return FF_OK;
 }
 
 ff_status ff_set_workspace(ff_ctx* ctx, void* dev_ptr, size_t bytes) {
   if (!ctx) return FF_ERR_ARG;
-  if (!dev_ptr || bytes < WS_STATUS_BYTES) return fail(ctx, FF_ERR_WORKSPACE, "workspace too small");
+  if (!dev_ptr || bytes < WS_BYTES) return fail(ctx, FF_ERR_WORKSPACE, "workspace too small");
   if (reinterpret_cast<uintptr_t>(dev_ptr) & 255) return fail(ctx, FF_ERR_ALIGN, "workspace must be 256-byte aligned");
   ctx->workspace = dev_ptr;
   ctx->workspace_bytes = bytes;
@@ -283,6 +380,13 @@ ff_status ff_set_gemm_path(ff_ctx* ctx, int path) {
   if (!ctx) return FF_ERR_ARG;
   if (path != FF_GEMM_AUTO && path != FF_GEMM_SIMT && path != FF_GEMM_TENSOR) return fail(ctx, FF_ERR_ARG, "unknown gemm path");
   ctx->gemm_path = path;
+  return FF_OK;
+}
+
+ff_status ff_set_tensor_form(ff_ctx* ctx, int ctas_per_tile) {
+  if (!ctx) return FF_ERR_ARG;
+  if (ctas_per_tile < 0 || ctas_per_tile > 2) return fail(ctx, FF_ERR_ARG, "ctas_per_tile must be 0, 1 or 2");
+  ctx->tc.force_ncta = ctas_per_tile;
   return FF_OK;
 }
 
@@ -383,6 +487,38 @@ ff_status ff_poll_status(ff_ctx* ctx, void* cuda_stream) {
   return FF_OK;
 }
 
+ff_status ff_profile_start(ff_ctx* ctx) {
+  if (!ctx) return FF_ERR_ARG;
+  for (auto& r : ctx->prof_recs) {
+    ctx->prof_pool.push_back(r.a);
+    ctx->prof_pool.push_back(r.b);
+  }
+  ctx->prof_recs.clear();
+  ctx->profiling = true;
+  return FF_OK;
+}
+
+ff_status ff_profile_stop(ff_ctx* ctx, void* cuda_stream, float* ms_per_kernel, uint32_t* launches_per_kernel) {
+  if (!ctx) return FF_ERR_ARG;
+  if (!ms_per_kernel || !launches_per_kernel) return fail(ctx, FF_ERR_ARG, "output arrays are NULL");
+  ctx->profiling = false;
+  FF_CUDA(ctx, cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)));
+  for (int k = 0; k < FF_K_COUNT; ++k) {
+    ms_per_kernel[k] = 0.0f;
+    launches_per_kernel[k] = 0;
+  }
+  for (auto& r : ctx->prof_recs) {
+    float ms = 0.0f;
+    FF_CUDA(ctx, cudaEventElapsedTime(&ms, r.a, r.b));
+    ms_per_kernel[r.kid] += ms;
+    launches_per_kernel[r.kid] += 1;
+    ctx->prof_pool.push_back(r.a);
+    ctx->prof_pool.push_back(r.b);
+  }
+  ctx->prof_recs.clear();
+  return FF_OK;
+}
+
 const char* ff_last_error(const ff_ctx* ctx) { return ctx ? ctx->err : "context is NULL"; }
 
 uint64_t ff_launch_count(const ff_ctx* ctx) { return ctx ? ctx->launches : 0; }
@@ -399,6 +535,7 @@ ff_status ff_int8_gemm(ff_ctx* ctx, const int8_t* A, const int8_t* Bm, int32_t* 
   bool tc_ok = tc_gemm_supported(M, N, K, trans);
   if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core gemm");
   if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT) {
+    ProfScope prof(ctx, FF_K_RAW_GEMM, st);
     s = tc_gemm(ctx->tc, A, Bm, C, M, N, K, trans, status_ptr(ctx), st);
     if (s != FF_OK) return fail(ctx, s, "tensor-core gemm launch failed: %s", ctx->tc.err);
     ctx->launches++;

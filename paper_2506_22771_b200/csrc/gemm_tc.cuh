@@ -4,7 +4,12 @@
 //   weight gradient   accW_p[n,k] = sum_{m in set p} dHq[m,n] * Xq[m,k]        (Sec. IV-B, g^W)
 // Persistent kernel, one CTA per SM, 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer
 // (one elected lane each), warps 2..5 = epilogue (one TMEM lane quadrant each).
-// Output tile 128 x 256, contraction block 128 bytes (4 MMAs of K = 32), 4-stage smem ring.
+// NCTA = 1: output tile 128 x 256 per CTA, 4-stage smem ring of 48 KiB stages.
+// NCTA = 2: two CTAs of a cluster share a 256 x 256 tile (tcgen05 cta_group::2): each CTA stages
+// its own 128 rows of A and one half (128 columns) of B, 6-stage ring of 32 KiB stages; the CTA
+// of cluster rank 0 issues the MMAs for both and holds the barriers the pair synchronises on.
+// The pair halves the B-operand traffic per MMA, which is what bounds the 1-CTA kernel.
+// Contraction block 128 bytes (4 MMAs of K = 32).
 // The forward operands are K-major (contraction contiguous); the weight-gradient operands are
 // read in their natural row-major layout as MN-major operands, so no transposed copy of dHq or Xq
 // is ever written.  The forward double-buffers the accumulator (2 x 256 TMEM columns) so that the
@@ -23,14 +28,17 @@
 namespace ffi8 {
 
 constexpr int TC_BM = 128, TC_BN = 256, TC_BKB = 128;  // tile rows, tile cols, contraction bytes per block
-constexpr int TC_STAGES = 4;
 constexpr int TC_THREADS = 192;
-constexpr uint32_t TC_A_BYTES = TC_BM * TC_BKB;      // 16 KiB
-constexpr uint32_t TC_B_BYTES = TC_BN * TC_BKB;      // 32 KiB
-constexpr uint32_t TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
+constexpr int TC_MAX_STAGES = 8;
+constexpr uint32_t TC_A_BYTES = TC_BM * TC_BKB;      // 16 KiB: 128 rows of this CTA
+__host__ __device__ constexpr int tc_stages(int ncta) { return ncta == 2 ? 6 : 4; }
+__host__ __device__ constexpr uint32_t tc_b_bytes(int ncta) { return (uint32_t)(TC_BN / ncta) * TC_BKB; }  // 32 / 16 KiB
+__host__ __device__ constexpr uint32_t tc_stage_bytes(int ncta) { return TC_A_BYTES + tc_b_bytes(ncta); }
 constexpr int TC_STG_PITCH = 36;                       // floats per staged row (32 + 4: 16-byte aligned, conflict-free)
 constexpr uint32_t TC_STG_BYTES = 32 * TC_STG_PITCH * 4;  // one 32 x 32 FP32 staging patch per epilogue warp
-constexpr uint32_t TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 4 * TC_STG_BYTES;
+__host__ __device__ constexpr uint32_t tc_smem_bytes(int ncta) {
+  return tc_stages(ncta) * tc_stage_bytes(ncta) + 1024 /*align*/ + 256 /*barriers*/ + 4 * TC_STG_BYTES;
+}
 constexpr int TC_PREFETCH_KB = 8;                      // W tile is prefetched into L2 this many k-blocks before the epilogue
 constexpr int TC_GROUP_M = 16;                          // tile rows per rasterisation group (L2 reuse)
 constexpr uint32_t TC_TMEM_COLS = 512;
@@ -79,17 +87,49 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Waits that may be released by the other CTA of a pair use cluster-scope acquire.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in the CTA of cluster rank `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
 // Bounded wait: false when the time limit ran out or another role already gave up.
+template <bool CLUSTER = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
+  auto poll = [&]() { return CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+  if (poll()) return true;
   const unsigned long long t0 = globaltimer_ns();
   uint32_t spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
+  while (!poll()) {
     if ((++spins & 0xFFu) == 0) {
       if (*abort_flag) return false;
       if (globaltimer_ns() - t0 > TC_WAIT_NS) return false;
@@ -97,29 +137,60 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
   return true;
 }
+// Tiled TMA loads into this CTA's shared memory.  NCTA = 2: `bar` is a shared::cluster address and may
+// name a barrier of the other CTA of the pair (the cta_group::2 form allows that); no multicast.
+template <int NCTA>
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-               "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y)
-               : "memory");
+  if (NCTA == 1)
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y)
+                 : "memory");
+  else
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y)
+                 : "memory");
 }
+template <int NCTA>
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y, int z) {
-  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
-               "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "r"(z)
-               : "memory");
+  if (NCTA == 1)
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "r"(z)
+                 : "memory");
+  else
+    asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "r"(z)
+                 : "memory");
 }
 __device__ __forceinline__ void l2_prefetch(const void* gptr, uint32_t bytes) {  // 16-byte aligned, multiple of 16
   asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Arrive on `bar` once all MMAs issued so far by this thread have completed.  NCTA = 2: the arrival is
+// delivered to the barrier at the same shared-memory offset in both CTAs of the pair.
+template <int NCTA>
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  if (NCTA == 1) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  } else {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                 "h"(mask)
+                 : "memory");
+  }
 }
+template <int NCTA>
 __device__ __forceinline__ void tc_mma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
+  if (NCTA == 1)
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 // Load 32 consecutive accumulator columns of this thread's TMEM lane and wait for them.
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, int (&r)[32]) {
@@ -149,10 +220,10 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
   d |= 2ull << 61;  // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: INT8 x INT8 -> INT32, dense, M = 128, N = 256.
-__host__ __device__ constexpr uint32_t make_idesc_i8(bool a_mn_major, bool b_mn_major) {
+// Instruction descriptor: INT8 x INT8 -> INT32, dense, M = 128 per CTA of the group, N = 256.
+__host__ __device__ constexpr uint32_t make_idesc_i8(bool a_mn_major, bool b_mn_major, int ncta) {
   return (2u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
-         ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+         ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)((TC_BM * ncta) >> 4) << 24);
 }
 
 // Tile order: groups of TC_GROUP_M tile rows, column by column inside a group, so that the CTAs
@@ -166,104 +237,125 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 }
 
 // ---- kernel --------------------------------------------------------------------------------
-template <int MODE, bool MN_MAJOR>
+template <int MODE, bool MN_MAJOR, int NCTA>
 __global__ void __launch_bounds__(TC_THREADS, 1)
     tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  constexpr int STAGES = tc_stages(NCTA);
+  constexpr uint32_t STAGE_BYTES = tc_stage_bytes(NCTA);
+  constexpr bool PAIR = NCTA == 2;
   extern __shared__ uint8_t smem_raw[];
-  // 1024-byte aligned operand ring, then the barriers
+  // 1024-byte aligned operand ring, then the barriers (identical offsets in both CTAs of a pair)
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t ring = (raw + 1023u) & ~1023u;
   uint8_t* ring_ptr = smem_raw + (ring - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ring_ptr + TC_STAGES * TC_STAGE_BYTES);
-  const uint32_t bar_full = smem_u32(bars);                      // [TC_STAGES]
-  const uint32_t bar_empty = bar_full + 8 * TC_STAGES;           // [TC_STAGES]
-  const uint32_t bar_tfull = bar_empty + 8 * TC_STAGES;          // [2]
-  const uint32_t bar_tempty = bar_tfull + 16;                    // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_STAGES + 4);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring_ptr + STAGES * STAGE_BYTES);
+  const uint32_t bar_full = smem_u32(bars);                      // [STAGES]  used in the leader CTA
+  const uint32_t bar_empty = bar_full + 8 * TC_MAX_STAGES;       // [STAGES]  one set per CTA
+  const uint32_t bar_tfull = bar_empty + 8 * TC_MAX_STAGES;      // [2]       one set per CTA
+  const uint32_t bar_tempty = bar_tfull + 16;                    // [2]       used in the leader CTA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_MAX_STAGES + 4);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  float* stage_all = reinterpret_cast<float*>(ring_ptr + TC_STAGES * TC_STAGE_BYTES + 256);
+  float* stage_all = reinterpret_cast<float*>(ring_ptr + STAGES * STAGE_BYTES + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = leader of the pair
+  const int group = blockIdx.x / NCTA, n_groups = gridDim.x / NCTA;
   constexpr int ACC_STAGES = (MODE == TC_MODE_UPD || MN_MAJOR) ? 1 : 2;
-  const int total_tiles = p.tiles_m * p.tiles_n;
+  const int total_tiles = p.tiles_m * p.tiles_n;                 // tiles of (128*NCTA) x 256
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < TC_STAGES; ++s) {
+    for (int s = 0; s < STAGES; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar_tfull + 8 * s, 1);
-      mbar_init(bar_tempty + 8 * s, 4);  // one arrive per epilogue warp
+      mbar_init(bar_tempty + 8 * s, 4 * NCTA);  // one arrive per epilogue warp of every CTA of the group
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TC_TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (warp == 1) {  // one warp of every CTA of the group takes part in the allocation
+    if (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TC_TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TC_TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();  // the other CTA's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // barriers of the leader CTA as seen from this CTA
+  const uint32_t lead_full = PAIR ? map_to_cta(bar_full, 0) : bar_full;
+  const uint32_t lead_tempty = PAIR ? map_to_cta(bar_tempty, 0) : bar_tempty;
+  auto raise_abort = [&]() {
+    atomicOr(p.status, ST_TIMEOUT);
+    *abort_flag = 1;
+    if (PAIR) st_cluster_u32(map_to_cta(smem_u32(const_cast<uint32_t*>(abort_flag)), rank ^ 1u), 1u);
+  };
 
   if (warp == 0) {
-    // ------------------------------- TMA producer -------------------------------------------
+    // ------------------------------- TMA producer (every CTA loads its own operand parts) ----
     if (lane == 0) {
       uint32_t it = 0;  // running k-block counter (ring position)
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int a_rows0 = (int)rank * TC_BM;            // this CTA's rows inside the group's tile
+      const int b_cols0 = (int)rank * (TC_BN / NCTA);   // this CTA's share of the tile's columns
+      for (int tile = group; tile < total_tiles && ok; tile += n_groups) {
         int tm, tn;
         tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+        const int row0 = tm * (TC_BM * NCTA) + a_rows0, col0 = tn * TC_BN + b_cols0;
         for (int pass = 0; pass < p.npass && ok; ++pass) {
           for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-            const uint32_t s = it % TC_STAGES, ph = (it / TC_STAGES) & 1u;
-            if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) {
+            const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+            if (!mbar_wait<PAIR>(bar_empty + 8 * s, ph ^ 1u, abort_flag)) {
               ok = false;
               break;
             }
-            const uint32_t a_dst = ring + s * TC_STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
+            const uint32_t a_dst = ring + s * STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
             if (MODE == TC_MODE_UPD && pass == p.npass - 1 && kb == max(0, p.kblocks - TC_PREFETCH_KB)) {
-              // pull this tile's W rows into L2 shortly before the epilogue's read-modify-write
+              // pull this CTA's W rows of the tile into L2 shortly before the epilogue's read-modify-write
               const int c0w = tn * TC_BN;
               const int ncols = min(TC_BN, p.out_cols - c0w);
               if ((p.out_cols & 3) == 0 && ncols > 0) {
-                const int nrows = min(TC_BM, p.out_rows - tm * TC_BM);
+                const int nrows = min(TC_BM, p.out_rows - row0);
                 for (int r = 0; r < nrows; ++r)
-                  l2_prefetch(p.W + (size_t)(tm * TC_BM + r) * p.out_cols + c0w, (uint32_t)ncols * 4u);
+                  l2_prefetch(p.W + (size_t)(row0 + r) * p.out_cols + c0w, (uint32_t)ncols * 4u);
               }
             }
-            mbar_expect_tx(bar_full + 8 * s, TC_STAGE_BYTES);
+            if (rank == 0) mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES * NCTA);
+            const uint32_t fb = lead_full + 8 * s;
             if (!MN_MAJOR) {
-              tma_load_2d(a_dst, &tmA, bar_full + 8 * s, kb * TC_BKB, tm * TC_BM);
-              tma_load_2d(b_dst, &tmB, bar_full + 8 * s, kb * TC_BKB, tn * TC_BN);
+              tma_load_2d<NCTA>(a_dst, &tmA, fb, kb * TC_BKB, row0);
+              tma_load_2d<NCTA>(b_dst, &tmB, fb, kb * TC_BKB, col0);
             } else {
-              // tile of 128 contraction rows x 128 output indices; B takes two such boxes
-              tma_load_3d(a_dst, &tmA, bar_full + 8 * s, tm * TC_BM, kb * 128, pass);
-              tma_load_3d(b_dst, &tmB, bar_full + 8 * s, tn * TC_BN, kb * 128, pass);
-              tma_load_3d(b_dst + 16384, &tmB, bar_full + 8 * s, tn * TC_BN + 128, kb * 128, pass);
+              // boxes of 128 contraction rows x 128 output indices
+              tma_load_3d<NCTA>(a_dst, &tmA, fb, row0, kb * 128, pass);
+              tma_load_3d<NCTA>(b_dst, &tmB, fb, col0, kb * 128, pass);
+              if (!PAIR) tma_load_3d<NCTA>(b_dst + 16384, &tmB, fb, col0 + 128, kb * 128, pass);
             }
           }
         }
       }
-      if (!ok) {
-        atomicOr(p.status, ST_TIMEOUT);
-        *abort_flag = 1;
-      }
+      if (!ok) raise_abort();
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------- MMA issuer ---------------------------------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_i8(MN_MAJOR, MN_MAJOR);
+    // ------------------------------- MMA issuer (leader CTA only) ----------------------------
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc_i8(MN_MAJOR, MN_MAJOR, NCTA);
       uint32_t it = 0, tile_it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+      for (int tile = group; tile < total_tiles && ok; tile += n_groups, ++tile_it) {
         const uint32_t as = tile_it % ACC_STAGES, aph = (tile_it / ACC_STAGES) & 1u;
-        if (!mbar_wait(bar_tempty + 8 * as, aph ^ 1u, abort_flag)) {
+        if (!mbar_wait<PAIR>(bar_tempty + 8 * as, aph ^ 1u, abort_flag)) {
           ok = false;
           break;
         }
@@ -271,13 +363,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         for (int pass = 0; pass < p.npass && ok; ++pass) {
           const uint32_t d_tmem = tmem_base + (MODE == TC_MODE_UPD ? pass * TC_BN : as * TC_BN);
           for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
-            const uint32_t s = it % TC_STAGES, ph = (it / TC_STAGES) & 1u;
-            if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) {
+            const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+            if (!mbar_wait<PAIR>(bar_full + 8 * s, ph, abort_flag)) {
               ok = false;
               break;
             }
             tc_fence_after();
-            const uint32_t a_src = ring + s * TC_STAGE_BYTES, b_src = a_src + TC_A_BYTES;
+            const uint32_t a_src = ring + s * STAGE_BYTES, b_src = a_src + TC_A_BYTES;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               uint64_t ad, bd;
@@ -288,21 +380,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
                 ad = make_smem_desc(a_src + k * 4096, 16384, 1024);
                 bd = make_smem_desc(b_src + k * 4096, 16384, 1024);
               }
-              tc_mma_i8(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+              tc_mma_i8<NCTA>(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
             }
-            tc_commit(bar_empty + 8 * s);  // frees the smem stage once these MMAs have read it
+            tc_commit<NCTA>(bar_empty + 8 * s);  // frees the smem stage (in every CTA) once these MMAs have read it
           }
         }
-        if (ok) tc_commit(bar_tfull + 8 * as);  // accumulator complete
+        if (ok) tc_commit<NCTA>(bar_tfull + 8 * as);  // accumulator complete (signalled in every CTA)
       }
-      if (!ok) {
-        atomicOr(p.status, ST_TIMEOUT);
-        *abort_flag = 1;
-      }
+      if (!ok) raise_abort();
     }
     __syncwarp();
   } else {
-    // ------------------------------- epilogue (warps 2..5) ----------------------------------
+    // ------------------------------- epilogue (warps 2..5 of every CTA) -----------------------
     const int quad = warp & 3;  // TMEM lane quadrant this warp may read
     float* stg = stage_all + (warp - 2) * (32 * TC_STG_PITCH);
     uint32_t tile_it = 0;
@@ -317,16 +406,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       cP = __fmul_rn(scale_of(p.absmax[3]), scale_of(p.absmax[0]));
       cN = __fmul_rn(scale_of(p.absmax[4]), scale_of(p.absmax[1]));
     }
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+    for (int tile = group; tile < total_tiles && ok; tile += n_groups, ++tile_it) {
       int tm, tn;
       tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
       const uint32_t as = tile_it % ACC_STAGES, aph = (tile_it / ACC_STAGES) & 1u;
-      if (!mbar_wait(bar_tfull + 8 * as, aph, abort_flag)) {
+      if (!mbar_wait<PAIR>(bar_tfull + 8 * as, aph, abort_flag)) {
         ok = false;
         break;
       }
       tc_fence_after();
-      const int row = tm * TC_BM + quad * 32 + lane;
+      const int wrow0 = tm * (TC_BM * NCTA) + (int)rank * TC_BM + quad * 32;  // first output row of this warp
+      const int row = wrow0 + lane;
       const bool row_ok = row < p.out_rows;
       const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
       const int col0 = tn * TC_BN;
@@ -351,7 +441,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         const float c = row < p.rows_per_pass ? c0 : c1;
         unsigned long long ssum = 0ull;
         int mx = 0;
-        const int wrow0 = tm * TC_BM + quad * 32;  // first output row of this warp
         for (int cb = 0; cb < TC_BN; cb += 32) {
           if (col0 + cb >= p.out_cols) break;  // uniform across the warp
           int v[32];
@@ -406,7 +495,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       } else {  // TC_MODE_UPD
         // thread = one accumulator row computes d = lr*(float(accP)*cP + float(accN)*cN); d is staged
         // through smem so that the read-modify-write of W is row-contiguous
-        const int wrow0 = tm * TC_BM + quad * 32;
         const size_t plane = (size_t)p.out_rows * p.out_cols;
         for (int cb = 0; cb < TC_BN; cb += 32) {
           if (col0 + cb >= p.out_cols) break;
@@ -468,15 +556,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           __syncwarp();
         }
       }
-      // accumulator stage drained: hand it back to the MMA issuer
+      // accumulator stage drained: hand it back to the MMA issuer (in the leader CTA)
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty + 8 * as);
+      if (lane == 0) {
+        if (PAIR)
+          mbar_arrive_cluster(lead_tempty + 8 * as);
+        else
+          mbar_arrive(bar_tempty + 8 * as);
+      }
     }
-    if (!ok && lane == 0) {
-      atomicOr(p.status, ST_TIMEOUT);
-      *abort_flag = 1;
-    }
+    if (!ok && lane == 0) raise_abort();
   }
 
   // ---- teardown: everyone meets, outstanding copies are waited for, TMEM is released ---------
@@ -487,10 +577,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     while (globaltimer_ns() - t0 < 2000000ull) {
     }
   }
+  tc_fence_before();
   __syncthreads();
+  // neither CTA of a pair leaves (or frees its tensor memory) while the other may still use it
+  if (PAIR) cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+    if (PAIR)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
   }
 }
 
@@ -501,8 +597,10 @@ typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_
 
 struct TcState {
   int sm_count = 148;
+  int force_ncta = 0;  // 0: choose by problem size; 1 / 2: always that CTA-group size
   PFN_encodeTiled encode = nullptr;
-  bool attr_set[3][2] = {{false, false}, {false, false}, {false, false}};
+  bool attr_set[3][2][2] = {};
+  int max_groups[3][2][2] = {};  // CTA groups that can be resident at one time, per kernel instance
   char err[256] = {0};
 };
 
@@ -540,20 +638,55 @@ inline ff_status tc_make_map(TcState& t, CUtensorMap* tm, const int8_t* base, ui
   return FF_OK;
 }
 
-template <int MODE, bool MN_MAJOR>
-inline ff_status tc_launch(TcState& t, const CUtensorMap& a, const CUtensorMap& b, TcParams p, cudaStream_t st) {
-  if (!t.attr_set[MODE][MN_MAJOR]) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<MODE, MN_MAJOR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES);
+inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+// CTA-group size for an output of out_rows x out_cols: pairs once there are at least two 128-row
+// blocks and enough 256 x 256 tiles to occupy every SM pair; single CTAs for small problems.
+inline int tc_pick_ncta(const TcState& t, long long out_rows, long long out_cols) {
+  if (t.force_ncta == 1 || t.force_ncta == 2) return t.force_ncta;
+  const long long pair_tiles = (long long)cdiv(out_rows, 2 * TC_BM) * cdiv(out_cols, TC_BN);
+  return (out_rows > TC_BM && pair_tiles >= t.sm_count / 2) ? 2 : 1;
+}
+
+template <int MODE, bool MN_MAJOR, int NCTA>
+inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap& b, TcParams p, cudaStream_t st) {
+  constexpr uint32_t SMEM = tc_smem_bytes(NCTA);
+  auto kern = tc_gemm_kernel<MODE, MN_MAJOR, NCTA>;
+  if (!t.attr_set[MODE][MN_MAJOR][NCTA - 1]) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM);
     if (e != cudaSuccess) {
       snprintf(t.err, sizeof(t.err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
       return FF_ERR_CUDA;
     }
-    t.attr_set[MODE][MN_MAJOR] = true;
+    t.attr_set[MODE][MN_MAJOR][NCTA - 1] = true;
   }
+  p.tiles_m = cdiv(p.out_rows, TC_BM * NCTA);
+  p.tiles_n = cdiv(p.out_cols, TC_BN);
   const int tiles = p.tiles_m * p.tiles_n;
-  const int grid = tiles < t.sm_count ? tiles : t.sm_count;
-  tc_gemm_kernel<MODE, MN_MAJOR><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(a, b, p);
-  cudaError_t e = cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(TC_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SMEM;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = NCTA;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int& max_groups = t.max_groups[MODE][MN_MAJOR][NCTA - 1];
+  if (max_groups == 0) {
+    // a persistent grid must be resident as a whole: ask how many CTA groups fit on the device
+    max_groups = t.sm_count / NCTA;
+    if (NCTA > 1) {
+      cfg.gridDim = dim3(t.sm_count / NCTA * NCTA, 1, 1);
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0 && n < max_groups) max_groups = n;
+    }
+  }
+  const int groups = tiles < max_groups ? tiles : max_groups;
+  cfg.gridDim = dim3(groups * NCTA, 1, 1);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a, b, p);
   if (e != cudaSuccess) {
     snprintf(t.err, sizeof(t.err), "launch: %s", cudaGetErrorString(e));
     return FF_ERR_CUDA;
@@ -561,7 +694,11 @@ inline ff_status tc_launch(TcState& t, const CUtensorMap& a, const CUtensorMap& 
   return FF_OK;
 }
 
-inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
+template <int MODE, bool MN_MAJOR>
+inline ff_status tc_launch(TcState& t, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, cudaStream_t st) {
+  if (tc_pick_ncta(t, p.out_rows, p.out_cols) == 2) return tc_launch_n<MODE, MN_MAJOR, 2>(t, a, b, p, st);
+  return tc_launch_n<MODE, MN_MAJOR, 1>(t, a, b, p, st);
+}
 
 // K-major ("NT") problem: A [M,K], B [N,K]; K % 16 == 0 (TMA row pitch), everything else ragged.
 inline bool tc_nt_ok(long long M, long long N, long long K) { return K % 16 == 0 && K >= 16 && M >= 1 && N >= 1; }
@@ -572,6 +709,11 @@ inline bool tc_gemm_supported(int M, int N, int K, int trans) { return trans ? t
 inline bool tc_forward_supported(const ff_layer_desc& L, int B) { return L.kind == FF_LINEAR && tc_nt_ok(2LL * B, L.N, L.K); }
 inline bool tc_update_supported(const ff_layer_desc& L, int B) { return L.kind == FF_LINEAR && tc_tn_ok(L.N, L.K, B); }
 
+// Box rows of the B operand: all 256 tile columns for a single CTA, this CTA's 128 for a pair.
+inline uint32_t tc_b_box_rows(const TcState& t, long long out_rows, long long out_cols) {
+  return (uint32_t)(TC_BN / tc_pick_ncta(t, out_rows, out_cols));
+}
+
 inline ff_status tc_gemm(TcState& t, const int8_t* A, const int8_t* Bm, int32_t* C, int M, int N, int K, int trans,
                          uint32_t* status, cudaStream_t st) {
   ff_status s = tc_init(t);
@@ -580,15 +722,13 @@ inline ff_status tc_gemm(TcState& t, const int8_t* A, const int8_t* Bm, int32_t*
   TcParams p = {};
   p.out_rows = M;
   p.out_cols = N;
-  p.tiles_m = cdiv(M, TC_BM);
-  p.tiles_n = cdiv(N, TC_BN);
   p.npass = 1;
   p.status = status;
   p.C = C;
   if (!trans) {
     p.kblocks = cdiv(K, TC_BKB);
     if ((s = tc_make_map(t, &ta, A, K, M, 0, TC_BKB, TC_BM)) != FF_OK) return s;
-    if ((s = tc_make_map(t, &tb, Bm, K, N, 0, TC_BKB, TC_BN)) != FF_OK) return s;
+    if ((s = tc_make_map(t, &tb, Bm, K, N, 0, TC_BKB, tc_b_box_rows(t, M, N))) != FF_OK) return s;
     return tc_launch<TC_MODE_RAW, false>(t, ta, tb, p, st);
   }
   p.kblocks = cdiv(K, 128);
@@ -605,8 +745,6 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   TcParams p = {};
   p.out_rows = M;
   p.out_cols = L.N;
-  p.tiles_m = cdiv(M, TC_BM);
-  p.tiles_n = cdiv(L.N, TC_BN);
   p.kblocks = cdiv(L.K, TC_BKB);
   p.npass = 1;
   p.status = status;
@@ -618,7 +756,7 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   p.rows_per_pass = B;
   p.rows_per_sample = 1;
   if ((s = tc_make_map(t, &ta, b.Xq, L.K, M, 0, TC_BKB, TC_BM)) != FF_OK) return s;
-  if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, TC_BKB, TC_BN)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, TC_BKB, tc_b_box_rows(t, M, L.N))) != FF_OK) return s;
   return tc_launch<TC_MODE_FWD, false>(t, ta, tb, p, st);
 }
 
@@ -629,8 +767,6 @@ inline ff_status tc_update(TcState& t, const ff_layer_desc& L, const ff_layer_bu
   TcParams p = {};
   p.out_rows = L.N;
   p.out_cols = L.K;
-  p.tiles_m = cdiv(L.N, TC_BM);
-  p.tiles_n = cdiv(L.K, TC_BN);
   p.kblocks = cdiv(B, 128);
   p.npass = 2;
   p.status = status;

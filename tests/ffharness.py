@@ -28,6 +28,9 @@ class GpuNet:
         self.B = B
         self.descs = descs
         self.ctx = ffb.Context(descs, B, 0)
+        if isinstance(gemm_path, tuple):
+            gemm_path, form = gemm_path
+            ffb.ff_set_tensor_form(self.ctx.ctx, form)
         ffb.ff_set_gemm_path(self.ctx.ctx, gemm_path)
         self.bufs = [ffb.LayerBuffers(d, B, self.dev, dumps=dumps, xnext=xnext, own_x=(i == 0 or not chain))
                      for i, d in enumerate(descs)]

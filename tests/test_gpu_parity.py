@@ -12,14 +12,17 @@ from tests.ffharness import GpuNet, compare_layer, specs_and_descs
 
 pytestmark = pytest.mark.gpu
 
-PATHS = [ffb.FF_GEMM_SIMT, ffb.FF_GEMM_AUTO]
+# (contraction path, CTAs per tensor-core tile: 0 = by problem size, 1 = single CTA, 2 = CTA pair)
+PATHS = [(ffb.FF_GEMM_SIMT, 0), (ffb.FF_GEMM_AUTO, 1), (ffb.FF_GEMM_AUTO, 2)]
+TENSOR_FORMS = [1, 2]
 
 
-def _gemm_case(M, N, K, trans, path):
+def _gemm_case(M, N, K, trans, path, form=0):
     import torch
     g = np.random.default_rng(M * 7 + N * 3 + K + trans)
     ctx = ffb.Context([ffb.ff_layer_desc(0, 16, 16, 1, 1, 0, 0, 0, 0, 0, 1.0, 0.1, 1.0, 1e-8, 0)], 1, 0)
     ffb.ff_set_gemm_path(ctx.ctx, path)
+    ffb.ff_set_tensor_form(ctx.ctx, form)
     if not trans:
         a = g.integers(-127, 128, size=(M, K)).astype(np.int8)
         b = g.integers(-127, 128, size=(N, K)).astype(np.int8)
@@ -45,14 +48,16 @@ def test_int8_gemm_simt(M, N, K, trans):
 
 @pytest.mark.parametrize("M,N,K", [(128, 256, 128), (128, 256, 512), (256, 512, 1024), (200, 300, 784),
                                    (1000, 2000, 2000), (16, 16, 16), (4096, 2048, 4096)])
-def test_int8_gemm_tensor_forward_orientation(M, N, K):
-    _gemm_case(M, N, K, 0, ffb.FF_GEMM_TENSOR)
+@pytest.mark.parametrize("form", TENSOR_FORMS)
+def test_int8_gemm_tensor_forward_orientation(M, N, K, form):
+    _gemm_case(M, N, K, 0, ffb.FF_GEMM_TENSOR, form)
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 256, 128), (128, 256, 512), (256, 512, 1000), (208, 304, 77),
                                    (2000, 784, 1024), (16, 16, 3), (2048, 4096, 4096)])
-def test_int8_gemm_tensor_weight_gradient_orientation(M, N, K):
-    _gemm_case(M, N, K, 1, ffb.FF_GEMM_TENSOR)
+@pytest.mark.parametrize("form", TENSOR_FORMS)
+def test_int8_gemm_tensor_weight_gradient_orientation(M, N, K, form):
+    _gemm_case(M, N, K, 1, ffb.FF_GEMM_TENSOR, form)
 
 
 def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), chain=True, check_every=1):
