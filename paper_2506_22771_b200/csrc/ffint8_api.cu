@@ -42,7 +42,12 @@ namespace {
 // workspace layout: [0, 256) status word (+ padding), then the loss kernel's partial-sum scratch
 constexpr size_t WS_STATUS_BYTES = 256;
 constexpr size_t WS_LOSS_OFFSET = WS_STATUS_BYTES;
-constexpr size_t WS_BYTES = (WS_LOSS_OFFSET + sizeof(LossScratch) + 255) / 256 * 256;
+constexpr size_t WS_BYTES = (WS_LOSS_OFFSET + sizeof(LossScratch) + 255) / 256 * 256;  // fixed header
+// After the header: INT32 partial-sum slabs of a split weight-gradient contraction,
+// [splits][2 sets][N][K].  Splitting is used where the output N x K alone has too few tiles to
+// occupy the device (convolutions contract over every output position of the batch).
+constexpr size_t WS_SLAB_CAP = (size_t)64 << 20;  // never ask for more than this per layer
+constexpr int WS_TARGET_ITEMS = 296;               // tiles x splits aimed at (two per SM of a 148-SM device)
 
 ff_status fail(ff_ctx* ctx, ff_status st, const char* fmt, const char* a = "", long long b = 0) {
   if (ctx) snprintf(ctx->err, sizeof(ctx->err), fmt, a, b);
@@ -156,10 +161,13 @@ inline int ew_blocks(ff_ctx* ctx, size_t work_items, int per_thread = 4) {
 
 // ---- contraction dispatch ----------------------------------------------------------------
 template <class LA, class LB, bool TRANS, int NPASS, class Epi>
-ff_status launch_simt(ff_ctx* ctx, LA la, LB lb, int out_rows, int out_cols, int clen, Epi epi, cudaStream_t st) {
-  dim3 grid((out_cols + SG_BN - 1) / SG_BN, (out_rows + SG_BM - 1) / SG_BM);
+ff_status launch_simt(ff_ctx* ctx, LA la, LB lb, int out_rows, int out_cols, int clen, Epi epi, cudaStream_t st,
+                      int splits = 1) {
+  // contraction elements per split, a multiple of the kernel's contraction block
+  const int csplit = splits > 1 ? ((clen + splits - 1) / splits + SG_BK - 1) / SG_BK * SG_BK : clen;
+  dim3 grid((out_cols + SG_BN - 1) / SG_BN, (out_rows + SG_BM - 1) / SG_BM, splits > 1 ? (clen + csplit - 1) / csplit : 1);
   ProfScope prof(ctx, std::is_same<Epi, ForwardEpilogue>::value ? FF_K_FWD_GEMM : std::is_same<Epi, UpdateEpilogue>::value ? FF_K_UPD_GEMM : FF_K_RAW_GEMM, st);
-  gemm_simt_kernel<LA, LB, TRANS, NPASS, Epi><<<grid, SG_THREADS, 0, st>>>(la, lb, clen, epi);
+  gemm_simt_kernel<LA, LB, TRANS, NPASS, Epi><<<grid, SG_THREADS, 0, st>>>(la, lb, clen, csplit, epi);
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
@@ -170,6 +178,38 @@ inline DenseView dense(const int8_t* p, int rows, int cols) {
 inline Im2colView im2col(const int8_t* p, const ff_layer_desc& L, int samples) {
   return Im2colView{p, samples * L.H * L.Wd, 9 * L.Cin, L.H, L.Wd, L.Cin,
                     (L.Cin % 8 == 0) && ((reinterpret_cast<uintptr_t>(p) & 7) == 0)};
+}
+
+// ---- split weight gradient ------------------------------------------------------------------
+inline long long simt_tiles(const ff_layer_desc& L) {
+  return (long long)((L.N + SG_BM - 1) / SG_BM) * ((L.K + SG_BN - 1) / SG_BN);
+}
+// Number of splits the SIMT weight gradient asks for (1 = none): enough that tiles x splits reaches
+// WS_TARGET_ITEMS, at least 1024 contraction elements per split, slabs within WS_SLAB_CAP and within
+// the workspace actually set (`ws_bytes`; pass SIZE_MAX to get the wish).
+inline int simt_wgrad_splits(const ff_layer_desc& L, int B, size_t ws_bytes) {
+  const long long clen = (long long)B * rows_per_sample(L);
+  const long long tiles = simt_tiles(L);
+  long long splits = (WS_TARGET_ITEMS + tiles - 1) / tiles;
+  if (splits > clen / 1024) splits = clen / 1024;
+  const size_t per_split = (size_t)2 * L.N * L.K * sizeof(int32_t);
+  const size_t room = ws_bytes > WS_BYTES ? ws_bytes - WS_BYTES : 0;
+  const size_t cap = room < WS_SLAB_CAP ? room : WS_SLAB_CAP;
+  if ((size_t)splits * per_split > cap) splits = (long long)(cap / per_split);
+  return splits < 2 ? 1 : (int)splits;
+}
+// grid.z the split launch really uses (the last splits can be empty after rounding to blocks)
+inline int simt_split_count(int clen, int splits) {
+  const int csplit = ((clen + splits - 1) / splits + SG_BK - 1) / SG_BK * SG_BK;
+  return (clen + csplit - 1) / csplit;
+}
+
+ff_status launch_slab_update(ff_ctx* ctx, const int32_t* slabs, int splits, const ff_layer_desc& L, const ff_layer_bufs& b,
+                             cudaStream_t st) {
+  const size_t plane = (size_t)L.N * L.K;
+  slab_update_kernel<<<ew_blocks(ctx, plane, 1), 256, 0, st>>>(slabs, splits, plane, b.W, b.absmax, L.lr, b.accW_dump);
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
 }
 
 // Forward contraction + fused epilogue.
@@ -204,10 +244,30 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     ctx->launches++;
     return FF_OK;
   }
+  const int clen = B * R;
+  const int splits = simt_wgrad_splits(L, B, ctx->workspace_bytes);
+  if (splits > 1) {
+    // few output tiles, long contraction: split it, keep INT32 partial sums in the workspace, add them exactly
+    int32_t* slabs = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
+    SlabEpilogue epi{slabs, L.N, L.K};
+    ff_status s;
+    {
+      ProfScope prof(ctx, FF_K_UPD_GEMM, st);
+      const bool was = ctx->profiling;
+      ctx->profiling = false;  // one event pair around both launches
+      if (L.kind == FF_LINEAR)
+        s = launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st, splits);
+      else
+        s = launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st, splits);
+      if (s == FF_OK) s = launch_slab_update(ctx, slabs, simt_split_count(clen, splits), L, b, st);
+      ctx->profiling = was;
+    }
+    return s;
+  }
   UpdateEpilogue epi{b.W, b.accW_dump, b.absmax, L.lr, L.N, L.K};
   if (L.kind == FF_LINEAR)
-    return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, B * R, epi, st);
-  return launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, B * R, epi, st);
+    return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st);
+  return launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st);
 }
 
 // ---- step pieces --------------------------------------------------------------------------
@@ -362,7 +422,14 @@ ff_status ff_destroy(ff_ctx* ctx) {
 
 ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, size_t* out_bytes) {
   if (!layers || n_layers <= 0 || B <= 0 || !out_bytes) return FF_ERR_ARG;
-  *out_bytes = WS_BYTES;
+  size_t slab = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    if (layers[l].K <= 0 || layers[l].N <= 0) return FF_ERR_ARG;
+    const int sp = simt_wgrad_splits(layers[l], B, SIZE_MAX);
+    const size_t need = sp > 1 ? (size_t)sp * 2 * layers[l].N * layers[l].K * sizeof(int32_t) : 0;
+    if (need > slab) slab = need;
+  }
+  *out_bytes = WS_BYTES + (slab + 255) / 256 * 256;
   return FF_OK;
 }
 

@@ -160,13 +160,59 @@ struct UpdateEpilogue {
   }
 };
 
+// Split weight-gradient epilogue: the contraction is divided over gridDim.z; every split stores
+// its INT32 partial sums of both sets to its own slab [split][set][rows][cols] (plain stores;
+// slab_update_kernel adds the slabs, which is exact in integers, and applies the update).
+struct SlabEpilogue {
+  int32_t* slabs;
+  int rows, cols;  // N, K
+  __device__ __forceinline__ void operator()(int i0, int j0, const int (&acc)[2][4][4]) const {
+    const size_t plane = (size_t)rows * cols;
+    int32_t* base = slabs + (size_t)blockIdx.z * 2 * plane;
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int i = i0 + r, j = j0 + c;
+        if (i < rows && j < cols) {
+          const size_t o = (size_t)i * cols + j;
+          base[o] = acc[0][r][c];
+          base[plane + o] = acc[1][r][c];
+        }
+      }
+  }
+};
+
+// Adds the `splits` INT32 slabs of both sets and applies the dequantised SGD update (Sec. IV-B;
+// Alg. 1 line 9): W <- W - lr*(float(accP)*cP + float(accN)*cN).  plane = N*K elements.
+__global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane,
+                                                          float* __restrict__ W, const float* __restrict__ absmax, float lr,
+                                                          int32_t* __restrict__ accW_dump) {
+  const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
+  const float cN = __fmul_rn(scale_of(absmax[4]), scale_of(absmax[1]));
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < plane; e += (size_t)gridDim.x * blockDim.x) {
+    int aP = 0, aN = 0;
+    for (int z = 0; z < splits; ++z) {
+      aP += slabs[((size_t)z * 2) * plane + e];
+      aN += slabs[((size_t)z * 2 + 1) * plane + e];
+    }
+    const float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
+    W[e] = __fsub_rn(W[e], __fmul_rn(lr, g));
+    if (accW_dump) {
+      accW_dump[e] = aP;
+      accW_dump[plane + e] = aN;
+    }
+  }
+}
+
 // ---- kernel ------------------------------------------------------------------------------
 // !TRANS: C[i,j] = sum_c LA(i,c) * LB(j,c)          (operands contraction-contiguous)
 //  TRANS: C[i,j] = sum_c LA(c,i) * LB(c,j)          (operands contraction-strided)
 // The contraction index runs over NPASS consecutive ranges of `clen` each (one accumulator set
-// per range: the positive and the negative set of the weight gradient).
+// per range: the positive and the negative set of the weight gradient).  Block z of the grid
+// takes the part [z*csplit, (z+1)*csplit) of every range (csplit = clen: no split).
 template <class LA, class LB, bool TRANS, int NPASS, class Epi>
-__global__ void __launch_bounds__(SG_THREADS) gemm_simt_kernel(LA la, LB lb, int clen, Epi epi) {
+__global__ void __launch_bounds__(SG_THREADS) gemm_simt_kernel(LA la, LB lb, int clen, int csplit, Epi epi) {
   __shared__ __align__(16) int8_t As[SG_BM * SG_PITCH];
   __shared__ __align__(16) int8_t Bs[SG_BN * SG_PITCH];
   const int tid = threadIdx.x;
@@ -182,7 +228,7 @@ __global__ void __launch_bounds__(SG_THREADS) gemm_simt_kernel(LA la, LB lb, int
 
 #pragma unroll
   for (int pass = 0; pass < NPASS; ++pass) {
-    const int cbeg = pass * clen, cend = cbeg + clen;
+    const int cbeg = pass * clen + (int)blockIdx.z * csplit, cend = min(pass * clen + clen, cbeg + csplit);
     for (int c0 = cbeg; c0 < cend; c0 += SG_BK) {
       int8_t va[8], vb[8];
       if (!TRANS) {
