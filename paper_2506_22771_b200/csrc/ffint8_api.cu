@@ -237,12 +237,33 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
   const int rows = 2 * B * R;
   bool tc_ok = tc_update_supported(L, B);
   if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core weight gradient");
-  if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT) {
+  if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT && L.kind == FF_LINEAR) {
     ProfScope prof(ctx, FF_K_UPD_GEMM, st);
     ff_status s = tc_update(ctx->tc, L, b, B, status_ptr(ctx), st);
     if (s != FF_OK) return fail(ctx, s, "tensor-core weight-gradient launch failed: %s", ctx->tc.err);
     ctx->launches++;
     return FF_OK;
+  }
+  if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT) {
+    // convolution: split implicit-GEMM contraction into INT32 slabs in the workspace, then reduce + update
+    int splits = tc_conv_update_splits(L, B, ctx->sm_count, ctx->tc.force_ncta);
+    const size_t room = ctx->workspace_bytes > WS_BYTES ? ctx->workspace_bytes - WS_BYTES : 0;
+    const size_t per_split = tc_conv_update_slab_bytes(L, 1);
+    if ((size_t)splits * per_split > room) splits = (int)(room / per_split);
+    if (splits >= 1) {
+      int32_t* slabs = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
+      ProfScope prof(ctx, FF_K_UPD_GEMM, st);
+      int used = 0;
+      ff_status s = tc_conv_update(ctx->tc, L, b, B, slabs, splits, &used, status_ptr(ctx), st);
+      if (s != FF_OK) return fail(ctx, s, "tensor-core convolution weight-gradient launch failed: %s", ctx->tc.err);
+      ctx->launches++;
+      const bool was = ctx->profiling;
+      ctx->profiling = false;
+      s = launch_slab_update(ctx, slabs, used, L, b, st);
+      ctx->profiling = was;
+      return s;
+    }
+    if (ctx->gemm_path == FF_GEMM_TENSOR) return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the weight-gradient slabs");
   }
   const int clen = B * R;
   const int splits = simt_wgrad_splits(L, B, ctx->workspace_bytes);
@@ -426,7 +447,13 @@ ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, s
   for (int l = 0; l < n_layers; ++l) {
     if (layers[l].K <= 0 || layers[l].N <= 0) return FF_ERR_ARG;
     const int sp = simt_wgrad_splits(layers[l], B, SIZE_MAX);
-    const size_t need = sp > 1 ? (size_t)sp * 2 * layers[l].N * layers[l].K * sizeof(int32_t) : 0;
+    size_t need = sp > 1 ? (size_t)sp * 2 * layers[l].N * layers[l].K * sizeof(int32_t) : 0;
+    if (tc_update_supported(layers[l], B) && layers[l].kind == FF_CONV3X3) {
+      // the larger of the single-CTA and CTA-pair split counts, so that either form finds room
+      const int s1 = tc_conv_update_splits(layers[l], B, 0, 1), s2 = tc_conv_update_splits(layers[l], B, 0, 2);
+      const size_t tc_need = tc_conv_update_slab_bytes(layers[l], s1 > s2 ? s1 : s2);
+      if (tc_need > need) need = tc_need;
+    }
     if (need > slab) slab = need;
   }
   *out_bytes = WS_BYTES + (slab + 255) / 256 * 256;

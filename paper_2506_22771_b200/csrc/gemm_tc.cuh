@@ -2,55 +2,73 @@
 // (tcgen05.mma kind::i8, accumulators in tensor memory, operands staged by TMA):
 //   forward           acc[m,n]    = sum_k Xq[m,k] * Wq[n,k]                    (Sec. IV-B, INT8 MAC)
 //   weight gradient   accW_p[n,k] = sum_{m in set p} dHq[m,n] * Xq[m,k]        (Sec. IV-B, g^W)
-// Persistent kernel, one CTA per SM, 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer
-// (one elected lane each), warps 2..5 = epilogue (one TMEM lane quadrant each).
-// NCTA = 1: output tile 128 x 256 per CTA, 4-stage smem ring of 48 KiB stages.
-// NCTA = 2: two CTAs of a cluster share a 256 x 256 tile (tcgen05 cta_group::2): each CTA stages
-// its own 128 rows of A and one half (128 columns) of B, 6-stage ring of 32 KiB stages; the CTA
-// of cluster rank 0 issues the MMAs for both and holds the barriers the pair synchronises on.
-// The pair halves the B-operand traffic per MMA, which is what bounds the 1-CTA kernel.
-// Contraction block 128 bytes (4 MMAs of K = 32).
-// The forward operands are K-major (contraction contiguous); the weight-gradient operands are
-// read in their natural row-major layout as MN-major operands, so no transposed copy of dHq or Xq
-// is ever written.  The forward double-buffers the accumulator (2 x 256 TMEM columns) so that the
-// epilogue of tile i overlaps the MMAs of tile i+1; the weight gradient holds the accumulators
-// of the positive and the negative set side by side (2 x 256 columns) and applies the update
-// W <- W - lr*(float(accP)*cP + float(accN)*cN) (Alg. 1 line 9) in its epilogue.
+// for dense layers and, as implicit GEMMs, for 3x3 / stride 1 / zero-pad 1 convolutions over NHWC
+// tensors ("dense or convolution layers", Sec. IV-B): the im2col matrix is never written; the
+// producer fetches, per filter tap, a box of the input shifted by the tap offset with a 4-D TMA
+// copy whose out-of-image part is zero-filled (zero is exact in the symmetric quantiser).
+//
+// One kernel template.  192 threads: warp 0 = TMA producer, warp 1 = MMA issuer (one elected lane
+// each), warps 2..5 = epilogue (one TMEM lane quadrant each).
+// NCTA = 1: output tile 128 x 256 per CTA.  NCTA = 2: the two CTAs of a cluster share a 256 x 256
+// tile (tcgen05 cta_group::2): each stages its own 128 rows of A and one half (128 columns) of B;
+// the CTA of cluster rank 0 issues the MMAs for both and holds the barriers the pair synchronises
+// on.  The pair halves the B-operand traffic per MMA.
+// Forward operands are K-major (contraction contiguous), CH = 128 or 64 contraction bytes per
+// block (64: convolution with 64 input channels; 64-byte swizzle).  Weight-gradient operands are
+// read in their natural row-major layout as MN-major operands (contraction block = 128 rows), so no
+// transposed copy of dHq or Xq is ever written; CH is then the width of one B box in bytes.
+// The forward double-buffers the accumulator (2 x 256 TMEM columns) so that the epilogue of tile
+// i overlaps the MMAs of tile i+1; the weight gradient holds the accumulators of the positive and
+// the negative set side by side (2 x 256 columns) and either applies the update
+// W <- W - lr*(float(accP)*cP + float(accN)*cN) (Alg. 1 line 9) in its epilogue (dense layers) or,
+// when the contraction is split over several CTAs because the output has few tiles
+// (convolutions), stores INT32 partial sums to slabs that slab_update_kernel adds exactly.
 // Every wait is bounded: when one runs out the CTA raises ST_TIMEOUT, drains and returns.
 #pragma once
 #include <cuda.h>
 
 #include <cstdio>
+#include <unordered_map>
 
 #include "../../include/ffint8.h"
 #include "common.cuh"
 
 namespace ffi8 {
 
-constexpr int TC_BM = 128, TC_BN = 256, TC_BKB = 128;  // tile rows, tile cols, contraction bytes per block
+constexpr int TC_BM = 128, TC_BN = 256;  // tile rows per CTA, tile columns
 constexpr int TC_THREADS = 192;
 constexpr int TC_MAX_STAGES = 8;
-constexpr uint32_t TC_A_BYTES = TC_BM * TC_BKB;      // 16 KiB: 128 rows of this CTA
-__host__ __device__ constexpr int tc_stages(int ncta) { return ncta == 2 ? 6 : 4; }
-__host__ __device__ constexpr uint32_t tc_b_bytes(int ncta) { return (uint32_t)(TC_BN / ncta) * TC_BKB; }  // 32 / 16 KiB
-__host__ __device__ constexpr uint32_t tc_stage_bytes(int ncta) { return TC_A_BYTES + tc_b_bytes(ncta); }
-constexpr int TC_STG_PITCH = 36;                       // floats per staged row (32 + 4: 16-byte aligned, conflict-free)
+constexpr int TC_STG_PITCH = 36;                          // floats per staged row (32 + 4: 16-byte aligned, conflict-free)
 constexpr uint32_t TC_STG_BYTES = 32 * TC_STG_PITCH * 4;  // one 32 x 32 FP32 staging patch per epilogue warp
-__host__ __device__ constexpr uint32_t tc_smem_bytes(int ncta) {
-  return tc_stages(ncta) * tc_stage_bytes(ncta) + 1024 /*align*/ + 256 /*barriers*/ + 4 * TC_STG_BYTES;
-}
-constexpr int TC_PREFETCH_KB = 8;                      // W tile is prefetched into L2 this many k-blocks before the epilogue
-constexpr int TC_GROUP_M = 16;                          // tile rows per rasterisation group (L2 reuse)
+constexpr uint32_t TC_RING_BYTES = 192 * 1024;            // operand ring budget
+constexpr int TC_PREFETCH_KB = 8;                         // W tile is prefetched into L2 this many k-blocks before the epilogue
+constexpr int TC_GROUP_M = 16;                            // tile rows per rasterisation group (L2 reuse)
 constexpr uint32_t TC_TMEM_COLS = 512;
 constexpr unsigned long long TC_WAIT_NS = 2000000000ull;  // 2 s bound on every wait
 
-enum { TC_MODE_RAW = 0, TC_MODE_FWD = 1, TC_MODE_UPD = 2 };
+// Shared-memory geometry of one pipeline stage.
+template <bool MN_MAJOR, int NCTA, int CH>
+struct TcGeom {
+  // K-major: A = 128 rows x CH bytes, B = (256/NCTA) rows x CH bytes.
+  // MN-major: A = 128 contraction rows x 128 bytes, B = 128 contraction rows x (256/NCTA) bytes in boxes of CH bytes.
+  static constexpr uint32_t A_BYTES = MN_MAJOR ? 128u * 128u : 128u * CH;
+  static constexpr uint32_t B_BYTES = MN_MAJOR ? 128u * (TC_BN / NCTA) : (uint32_t)(TC_BN / NCTA) * CH;
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = (int)(TC_RING_BYTES / STAGE_BYTES) < TC_MAX_STAGES ? (int)(TC_RING_BYTES / STAGE_BYTES) : TC_MAX_STAGES;
+  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 4 * TC_STG_BYTES;
+  static constexpr int MMAS = MN_MAJOR ? 4 : CH / 32;            // MMAs (K = 32) per contraction block
+  static constexpr int B_BOXES = MN_MAJOR ? (TC_BN / NCTA) / CH : 1;  // TMA boxes of the B operand per stage
+  static constexpr uint32_t SWZ = CH == 128 ? 2u : 4u;             // descriptor swizzle code: 128-byte / 64-byte
+};
+
+enum { TC_MODE_RAW = 0, TC_MODE_FWD = 1, TC_MODE_UPD = 2, TC_MODE_SLAB = 3 };
 
 struct TcParams {
   int out_rows, out_cols;   // extent of the output matrix
   int tiles_m, tiles_n;
   int kblocks;              // contraction blocks per pass
   int npass;                // 1, or 2 for the weight gradient (positive / negative set)
+  int splits, kb_per_split; // the contraction blocks of a pass are divided over `splits` work items
   uint32_t* status;
   // raw
   int32_t* C;
@@ -65,6 +83,11 @@ struct TcParams {
   float* W;
   int32_t* accW_dump;
   float lr;
+  // split weight gradient
+  int32_t* slabs;
+  // convolution geometry (conv_W = 0: dense layer).  A 128-row block of positions is conv_TH image
+  // rows of conv_W pixels; conv_cpt = channel chunks of CH bytes per filter tap; images per set.
+  int conv_W, conv_H, conv_TH, conv_cin, conv_cpt, conv_imgs_per_pass;
 };
 
 // ---- PTX wrappers --------------------------------------------------------------------------
@@ -161,6 +184,17 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
                  "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "r"(z)
                  : "memory");
 }
+template <int NCTA>
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y, int z, int w) {
+  if (NCTA == 1)
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
+                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w)
+                 : "memory");
+  else
+    asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(dst),
+                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w)
+                 : "memory");
+}
 __device__ __forceinline__ void l2_prefetch(const void* gptr, uint32_t bytes) {  // 16-byte aligned, multiple of 16
   asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
 }
@@ -207,17 +241,17 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, int (&r)[32]) {
 }
 // (the wait for the load is part of tc_ld32, so the registers are valid when it returns)
 
-// Shared-memory matrix descriptor for a 128-byte-swizzled operand tile (rows of 128 bytes, groups
-// of 8 rows = 1024 bytes).  K-major: rows are M/N indices, SBO = 1024 between 8-row groups, LBO
-// unused.  MN-major: rows are contraction indices, SBO = 1024 between groups of 8 contraction
-// rows, LBO = distance between successive 128-element chunks along M/N.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+// Shared-memory matrix descriptor for a swizzled operand tile whose rows are CH = 128 (swz = 2) or
+// 64 (swz = 4) bytes long; 8 rows form one swizzle atom.  K-major: rows are M/N indices, SBO = 8 rows
+// between atoms, LBO unused.  MN-major: rows are contraction indices, SBO = 8 contraction rows,
+// LBO = distance between successive CH-element chunks along M/N.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swz) {
   uint64_t d = 0;
   d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
   d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
   d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
   d |= 1ull << 46;  // descriptor version of this architecture
-  d |= 2ull << 61;  // 128-byte swizzle
+  d |= (uint64_t)swz << 61;
   return d;
 }
 // Instruction descriptor: INT8 x INT8 -> INT32, dense, M = 128 per CTA of the group, N = 256.
@@ -237,11 +271,12 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 }
 
 // ---- kernel --------------------------------------------------------------------------------
-template <int MODE, bool MN_MAJOR, int NCTA>
+template <int MODE, bool MN_MAJOR, int NCTA, int CH>
 __global__ void __launch_bounds__(TC_THREADS, 1)
     tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
-  constexpr int STAGES = tc_stages(NCTA);
-  constexpr uint32_t STAGE_BYTES = tc_stage_bytes(NCTA);
+  using G = TcGeom<MN_MAJOR, NCTA, CH>;
+  constexpr int STAGES = G::STAGES;
+  constexpr uint32_t STAGE_BYTES = G::STAGE_BYTES;
   constexpr bool PAIR = NCTA == 2;
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte aligned operand ring, then the barriers (identical offsets in both CTAs of a pair)
@@ -260,8 +295,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = leader of the pair
   const int group = blockIdx.x / NCTA, n_groups = gridDim.x / NCTA;
-  constexpr int ACC_STAGES = (MODE == TC_MODE_UPD || MN_MAJOR) ? 1 : 2;
-  const int total_tiles = p.tiles_m * p.tiles_n;                 // tiles of (128*NCTA) x 256
+  constexpr bool TWO_SETS = MODE == TC_MODE_UPD || MODE == TC_MODE_SLAB;  // accumulators of both sets side by side
+  constexpr int ACC_STAGES = (TWO_SETS || MN_MAJOR) ? 1 : 2;
+  const int total_items = p.tiles_m * p.tiles_n * p.splits;      // work item = (tile of (128*NCTA) x 256, split)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -308,19 +344,32 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       bool ok = true;
       const int a_rows0 = (int)rank * TC_BM;            // this CTA's rows inside the group's tile
       const int b_cols0 = (int)rank * (TC_BN / NCTA);   // this CTA's share of the tile's columns
-      for (int tile = group; tile < total_tiles && ok; tile += n_groups) {
+      const int hw = p.conv_H * p.conv_W;
+      const int blocks_per_img = p.conv_W ? p.conv_H / p.conv_TH : 1;
+      for (int item = group; item < total_items && ok; item += n_groups) {
+        const int tile = item / p.splits, split = item - tile * p.splits;
+        const int kb0 = split * p.kb_per_split, kb1 = min(p.kblocks, kb0 + p.kb_per_split);
         int tm, tn;
         tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
         const int row0 = tm * (TC_BM * NCTA) + a_rows0, col0 = tn * TC_BN + b_cols0;
+        // forward convolution: image and first image row of this CTA's 128 output positions
+        const int f_img = (!MN_MAJOR && p.conv_W) ? row0 / hw : 0;
+        const int f_h0 = (!MN_MAJOR && p.conv_W) ? (row0 - f_img * hw) / p.conv_W : 0;
+        // bytes the leader's barrier expects per stage from all CTAs of the group
+        uint32_t stage_tx = STAGE_BYTES * NCTA;
+        if (MN_MAJOR && p.conv_W) {
+          const int valid_cols = min(TC_BN, p.out_cols - tn * TC_BN);  // a multiple of CH
+          stage_tx = G::A_BYTES * NCTA + (uint32_t)valid_cols * 128u;
+        }
         for (int pass = 0; pass < p.npass && ok; ++pass) {
-          for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+          for (int kb = kb0; kb < kb1; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
             if (!mbar_wait<PAIR>(bar_empty + 8 * s, ph ^ 1u, abort_flag)) {
               ok = false;
               break;
             }
-            const uint32_t a_dst = ring + s * STAGE_BYTES, b_dst = a_dst + TC_A_BYTES;
-            if (MODE == TC_MODE_UPD && pass == p.npass - 1 && kb == max(0, p.kblocks - TC_PREFETCH_KB)) {
+            const uint32_t a_dst = ring + s * STAGE_BYTES, b_dst = a_dst + G::A_BYTES;
+            if (MODE == TC_MODE_UPD && pass == p.npass - 1 && kb == max(kb0, kb1 - TC_PREFETCH_KB)) {
               // pull this CTA's W rows of the tile into L2 shortly before the epilogue's read-modify-write
               const int c0w = tn * TC_BN;
               const int ncols = min(TC_BN, p.out_cols - c0w);
@@ -330,16 +379,40 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
                   l2_prefetch(p.W + (size_t)(row0 + r) * p.out_cols + c0w, (uint32_t)ncols * 4u);
               }
             }
-            if (rank == 0) mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES * NCTA);
+            if (rank == 0) mbar_expect_tx(bar_full + 8 * s, stage_tx);
             const uint32_t fb = lead_full + 8 * s;
             if (!MN_MAJOR) {
-              tma_load_2d<NCTA>(a_dst, &tmA, fb, kb * TC_BKB, row0);
-              tma_load_2d<NCTA>(b_dst, &tmB, fb, kb * TC_BKB, col0);
+              if (p.conv_W) {
+                // k-block = CH channels of one filter tap (r, s): the input box shifted by (r-1, s-1)
+                const int tap = kb / p.conv_cpt, cc = kb - tap * p.conv_cpt;
+                const int r = tap / 3, sx = tap - r * 3;
+                tma_load_4d<NCTA>(a_dst, &tmA, fb, cc * CH, sx - 1, f_h0 + r - 1, f_img);
+              } else {
+                tma_load_2d<NCTA>(a_dst, &tmA, fb, kb * CH, row0);
+              }
+              tma_load_2d<NCTA>(b_dst, &tmB, fb, kb * CH, col0);
             } else {
-              // boxes of 128 contraction rows x 128 output indices
+              // boxes of 128 contraction rows x 128 (A) or CH (B) output indices
               tma_load_3d<NCTA>(a_dst, &tmA, fb, row0, kb * 128, pass);
-              tma_load_3d<NCTA>(b_dst, &tmB, fb, col0, kb * 128, pass);
-              if (!PAIR) tma_load_3d<NCTA>(b_dst + 16384, &tmB, fb, col0 + 128, kb * 128, pass);
+              if (p.conv_W) {
+                // contraction block kb of set `pass` = conv_TH rows of one image; B column chunk q of the
+                // tile = CH channels of one filter tap, fetched from the shifted input box
+                const int img = pass * p.conv_imgs_per_pass + kb / blocks_per_img;
+                const int h0 = (kb % blocks_per_img) * p.conv_TH;
+#pragma unroll
+                for (int q = 0; q < G::B_BOXES; ++q) {
+                  const int c = col0 + q * CH;
+                  if (c < p.out_cols) {
+                    const int tap = c / p.conv_cin, ci0 = c - tap * p.conv_cin;
+                    const int r = tap / 3, sx = tap - r * 3;
+                    tma_load_4d<NCTA>(b_dst + q * (128 * CH), &tmB, fb, ci0, sx - 1, h0 + r - 1, img);
+                  }
+                }
+              } else {
+#pragma unroll
+                for (int q = 0; q < G::B_BOXES; ++q)
+                  tma_load_3d<NCTA>(b_dst + q * (128 * CH), &tmB, fb, col0 + q * CH, kb * 128, pass);
+              }
             }
           }
         }
@@ -353,7 +426,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       constexpr uint32_t idesc = make_idesc_i8(MN_MAJOR, MN_MAJOR, NCTA);
       uint32_t it = 0, tile_it = 0;
       bool ok = true;
-      for (int tile = group; tile < total_tiles && ok; tile += n_groups, ++tile_it) {
+      for (int item = group; item < total_items && ok; item += n_groups, ++tile_it) {
+        const int split = item % p.splits;
+        const int kb0 = split * p.kb_per_split, kb1 = min(p.kblocks, kb0 + p.kb_per_split);
         const uint32_t as = tile_it % ACC_STAGES, aph = (tile_it / ACC_STAGES) & 1u;
         if (!mbar_wait<PAIR>(bar_tempty + 8 * as, aph ^ 1u, abort_flag)) {
           ok = false;
@@ -361,26 +436,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         }
         tc_fence_after();
         for (int pass = 0; pass < p.npass && ok; ++pass) {
-          const uint32_t d_tmem = tmem_base + (MODE == TC_MODE_UPD ? pass * TC_BN : as * TC_BN);
-          for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+          const uint32_t d_tmem = tmem_base + (TWO_SETS ? pass * TC_BN : as * TC_BN);
+          for (int kb = kb0; kb < kb1; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
             if (!mbar_wait<PAIR>(bar_full + 8 * s, ph, abort_flag)) {
               ok = false;
               break;
             }
             tc_fence_after();
-            const uint32_t a_src = ring + s * STAGE_BYTES, b_src = a_src + TC_A_BYTES;
+            const uint32_t a_src = ring + s * STAGE_BYTES, b_src = a_src + G::A_BYTES;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < G::MMAS; ++k) {
               uint64_t ad, bd;
               if (!MN_MAJOR) {
-                ad = make_smem_desc(a_src + k * 32, 16, 1024);
-                bd = make_smem_desc(b_src + k * 32, 16, 1024);
+                ad = make_smem_desc(a_src + k * 32, 16, 8 * CH, G::SWZ);
+                bd = make_smem_desc(b_src + k * 32, 16, 8 * CH, G::SWZ);
               } else {
-                ad = make_smem_desc(a_src + k * 4096, 16384, 1024);
-                bd = make_smem_desc(b_src + k * 4096, 16384, 1024);
+                ad = make_smem_desc(a_src + k * 4096, 16384, 1024, 2u);
+                bd = make_smem_desc(b_src + k * (32 * CH), 128 * CH, 8 * CH, G::SWZ);
               }
-              tc_mma_i8<NCTA>(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+              tc_mma_i8<NCTA>(d_tmem, ad, bd, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
             }
             tc_commit<NCTA>(bar_empty + 8 * s);  // frees the smem stage (in every CTA) once these MMAs have read it
           }
@@ -406,7 +481,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       cP = __fmul_rn(scale_of(p.absmax[3]), scale_of(p.absmax[0]));
       cN = __fmul_rn(scale_of(p.absmax[4]), scale_of(p.absmax[1]));
     }
-    for (int tile = group; tile < total_tiles && ok; tile += n_groups, ++tile_it) {
+    for (int item = group; item < total_items && ok; item += n_groups, ++tile_it) {
+      const int tile = item / p.splits, split = item - tile * p.splits;
+      (void)split;
       int tm, tn;
       tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
       const uint32_t as = tile_it % ACC_STAGES, aph = (tile_it / ACC_STAGES) & 1u;
@@ -487,10 +564,45 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           }
           __syncwarp();
         }
-        if (row_ok && mx > 0) {
+        if ((p.rows_per_sample & 31) == 0) {
+          // the warp's 32 rows belong to one sample (convolution: a sample has H*W rows): one atomic
+          // per warp; rows past the end hold zero accumulators and add nothing
+          ssum += __shfl_xor_sync(0xffffffffu, ssum, 16);
+          ssum += __shfl_xor_sync(0xffffffffu, ssum, 8);
+          ssum += __shfl_xor_sync(0xffffffffu, ssum, 4);
+          ssum += __shfl_xor_sync(0xffffffffu, ssum, 2);
+          ssum += __shfl_xor_sync(0xffffffffu, ssum, 1);
+          mx = __reduce_max_sync(0xffffffffu, mx);
+          if (lane == 0 && wrow0 < p.out_rows && mx > 0) {
+            const int sample = wrow0 / p.rows_per_sample;
+            atomicAdd(p.S + sample, ssum);
+            atomicMax(p.rowmax + sample, mx);
+          }
+        } else if (row_ok && mx > 0) {
           const int sample = row / p.rows_per_sample;
           atomicAdd(p.S + sample, ssum);
           atomicMax(p.rowmax + sample, mx);
+        }
+      } else if (MODE == TC_MODE_SLAB) {
+        // raw INT32 partial sums of both sets to this split's slab [split][set][rows][cols]
+        for (int pass = 0; pass < 2; ++pass) {
+          int32_t* slab = p.slabs + (size_t)(split * 2 + pass) * p.out_rows * p.out_cols;
+          for (int cb = 0; cb < TC_BN; cb += 32) {
+            if (col0 + cb >= p.out_cols) break;
+            int v[32];
+            tc_ld32(t_row + pass * TC_BN + cb, v);
+            if (row_ok) {
+              int32_t* dst = slab + (size_t)row * p.out_cols + col0 + cb;
+              if (col0 + cb + 32 <= p.out_cols && (p.out_cols & 3) == 0) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) *reinterpret_cast<int4*>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (col0 + cb + j < p.out_cols) dst[j] = v[j];
+              }
+            }
+          }
         }
       } else {  // TC_MODE_UPD
         // thread = one accumulator row computes d = lr*(float(accP)*cP + float(accN)*cN); d is staged
@@ -599,8 +711,7 @@ struct TcState {
   int sm_count = 148;
   int force_ncta = 0;  // 0: choose by problem size; 1 / 2: always that CTA-group size
   PFN_encodeTiled encode = nullptr;
-  bool attr_set[3][2][2] = {};
-  int max_groups[3][2][2] = {};  // CTA groups that can be resident at one time, per kernel instance
+  std::unordered_map<const void*, int> max_groups;  // CTA groups resident at one time, per kernel instance
   char err[256] = {0};
 };
 
@@ -617,55 +728,66 @@ inline ff_status tc_init(TcState& t) {
   return FF_OK;
 }
 
-// INT8 row-major matrix [rows, cols] viewed as `passes` stacked matrices of rows_per_pass rows;
-// box = box_cols x box_rows (x 1), 128-byte swizzle, zero fill outside.
-inline ff_status tc_make_map(TcState& t, CUtensorMap* tm, const int8_t* base, uint64_t cols, uint64_t rows_per_pass, uint64_t passes,
-                             uint32_t box_cols, uint32_t box_rows) {
-  cuuint64_t dims[3] = {cols, rows_per_pass, passes};
-  cuuint64_t strides[2] = {cols, cols * rows_per_pass};
-  cuuint32_t box[3] = {box_cols, box_rows, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  const cuuint32_t rank = passes > 0 ? 3 : 2;
-  if (rank == 2) dims[2] = 1;
+inline ff_status tc_encode(TcState& t, CUtensorMap* tm, const int8_t* base, cuuint32_t rank, const cuuint64_t* dims,
+                           const cuuint64_t* strides, const cuuint32_t* box, int swizzle_bytes) {
+  cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = t.encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, rank, const_cast<int8_t*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
-    snprintf(t.err, sizeof(t.err), "cuTensorMapEncodeTiled failed (%d) cols=%llu rows=%llu", (int)r, (unsigned long long)cols,
-             (unsigned long long)rows_per_pass);
+    snprintf(t.err, sizeof(t.err), "cuTensorMapEncodeTiled failed (%d) rank=%u dims=%llu,%llu box=%u,%u", (int)r, rank,
+             (unsigned long long)dims[0], (unsigned long long)dims[1], box[0], box[1]);
     return FF_ERR_CUDA;
   }
   return FF_OK;
+}
+
+// INT8 row-major matrix [rows, cols] viewed as `passes` stacked matrices of rows_per_pass rows (passes = 0:
+// a plain 2-D map); box = box_cols x box_rows (x 1), swizzle = box_cols bytes (128 or 64), zero fill outside.
+inline ff_status tc_make_map(TcState& t, CUtensorMap* tm, const int8_t* base, uint64_t cols, uint64_t rows_per_pass, uint64_t passes,
+                             uint32_t box_cols, uint32_t box_rows) {
+  cuuint64_t dims[3] = {cols, rows_per_pass, passes ? passes : 1};
+  cuuint64_t strides[2] = {cols, cols * rows_per_pass};
+  cuuint32_t box[3] = {box_cols, box_rows, 1};
+  return tc_encode(t, tm, base, passes > 0 ? 3 : 2, dims, strides, box, (int)box_cols);
+}
+// NHWC INT8 tensor [imgs, H, W, C]; box = ch_box channels x W pixels x th rows x 1 image.
+inline ff_status tc_make_map_nhwc(TcState& t, CUtensorMap* tm, const int8_t* base, uint64_t C, uint64_t W, uint64_t H, uint64_t imgs,
+                                  uint32_t ch_box, uint32_t th) {
+  cuuint64_t dims[4] = {C, W, H, imgs};
+  cuuint64_t strides[3] = {C, C * W, C * W * H};
+  cuuint32_t box[4] = {ch_box, (cuuint32_t)W, th, 1};
+  return tc_encode(t, tm, base, 4, dims, strides, box, (int)ch_box);
 }
 
 inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 // CTA-group size for an output of out_rows x out_cols: pairs once there are at least two 128-row
 // blocks and enough 256 x 256 tiles to occupy every SM pair; single CTAs for small problems.
-inline int tc_pick_ncta(const TcState& t, long long out_rows, long long out_cols) {
+inline int tc_pick_ncta(const TcState& t, long long out_rows, long long out_cols, long long splits = 1) {
   if (t.force_ncta == 1 || t.force_ncta == 2) return t.force_ncta;
-  const long long pair_tiles = (long long)cdiv(out_rows, 2 * TC_BM) * cdiv(out_cols, TC_BN);
-  return (out_rows > TC_BM && pair_tiles >= t.sm_count / 2) ? 2 : 1;
+  const long long pair_items = (long long)cdiv(out_rows, 2 * TC_BM) * cdiv(out_cols, TC_BN) * splits;
+  return (out_rows > TC_BM && pair_items >= t.sm_count / 2) ? 2 : 1;
 }
 
-template <int MODE, bool MN_MAJOR, int NCTA>
+template <int MODE, bool MN_MAJOR, int NCTA, int CH>
 inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap& b, TcParams p, cudaStream_t st) {
-  constexpr uint32_t SMEM = tc_smem_bytes(NCTA);
-  auto kern = tc_gemm_kernel<MODE, MN_MAJOR, NCTA>;
-  if (!t.attr_set[MODE][MN_MAJOR][NCTA - 1]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM);
-    if (e != cudaSuccess) {
-      snprintf(t.err, sizeof(t.err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-      return FF_ERR_CUDA;
-    }
-    t.attr_set[MODE][MN_MAJOR][NCTA - 1] = true;
+  using G = TcGeom<MN_MAJOR, NCTA, CH>;
+  auto kern = tc_gemm_kernel<MODE, MN_MAJOR, NCTA, CH>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::SMEM_BYTES);
+  if (e != cudaSuccess) {
+    snprintf(t.err, sizeof(t.err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    return FF_ERR_CUDA;
   }
   p.tiles_m = cdiv(p.out_rows, TC_BM * NCTA);
   p.tiles_n = cdiv(p.out_cols, TC_BN);
-  const int tiles = p.tiles_m * p.tiles_n;
+  if (p.splits < 1) p.splits = 1;
+  p.kb_per_split = cdiv(p.kblocks, p.splits);
+  p.splits = cdiv(p.kblocks, p.kb_per_split);  // no empty split
+  const int items = p.tiles_m * p.tiles_n * p.splits;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(TC_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = SMEM;
+  cfg.dynamicSmemBytes = G::SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -674,7 +796,7 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  int& max_groups = t.max_groups[MODE][MN_MAJOR][NCTA - 1];
+  int& max_groups = t.max_groups[reinterpret_cast<const void*>(kern)];
   if (max_groups == 0) {
     // a persistent grid must be resident as a whole: ask how many CTA groups fit on the device
     max_groups = t.sm_count / NCTA;
@@ -684,9 +806,9 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
       if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0 && n < max_groups) max_groups = n;
     }
   }
-  const int groups = tiles < max_groups ? tiles : max_groups;
+  const int groups = items < max_groups ? items : max_groups;
   cfg.gridDim = dim3(groups * NCTA, 1, 1);
-  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a, b, p);
+  e = cudaLaunchKernelEx(&cfg, kern, a, b, p);
   if (e != cudaSuccess) {
     snprintf(t.err, sizeof(t.err), "launch: %s", cudaGetErrorString(e));
     return FF_ERR_CUDA;
@@ -694,10 +816,10 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
   return FF_OK;
 }
 
-template <int MODE, bool MN_MAJOR>
-inline ff_status tc_launch(TcState& t, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, cudaStream_t st) {
-  if (tc_pick_ncta(t, p.out_rows, p.out_cols) == 2) return tc_launch_n<MODE, MN_MAJOR, 2>(t, a, b, p, st);
-  return tc_launch_n<MODE, MN_MAJOR, 1>(t, a, b, p, st);
+template <int MODE, bool MN_MAJOR, int CH>
+inline ff_status tc_launch(TcState& t, int ncta, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, cudaStream_t st) {
+  if (ncta == 2) return tc_launch_n<MODE, MN_MAJOR, 2, CH>(t, a, b, p, st);
+  return tc_launch_n<MODE, MN_MAJOR, 1, CH>(t, a, b, p, st);
 }
 
 // K-major ("NT") problem: A [M,K], B [N,K]; K % 16 == 0 (TMA row pitch), everything else ragged.
@@ -706,12 +828,35 @@ inline bool tc_nt_ok(long long M, long long N, long long K) { return K % 16 == 0
 inline bool tc_tn_ok(long long M, long long N, long long Kc) { return M % 16 == 0 && N % 16 == 0 && Kc >= 1; }
 
 inline bool tc_gemm_supported(int M, int N, int K, int trans) { return trans ? tc_tn_ok(M, N, K) : tc_nt_ok(M, N, K); }
-inline bool tc_forward_supported(const ff_layer_desc& L, int B) { return L.kind == FF_LINEAR && tc_nt_ok(2LL * B, L.N, L.K); }
-inline bool tc_update_supported(const ff_layer_desc& L, int B) { return L.kind == FF_LINEAR && tc_tn_ok(L.N, L.K, B); }
+// 3x3 convolution as an implicit GEMM: whole 128-byte (or 64-byte) channel chunks per filter tap, image
+// width a power of two up to 128 so that 128 consecutive output positions are whole image rows.
+inline bool tc_conv_ok(const ff_layer_desc& L) {
+  if (L.kind != FF_CONV3X3 || L.Cin % 64 != 0) return false;
+  const int W = L.Wd;
+  if (W < 8 || W > 128 || (W & (W - 1)) != 0) return false;
+  return L.H % (128 / W) == 0;
+}
+inline bool tc_forward_supported(const ff_layer_desc& L, int B) {
+  return L.kind == FF_LINEAR ? tc_nt_ok(2LL * B, L.N, L.K) : tc_conv_ok(L);
+}
+inline bool tc_update_supported(const ff_layer_desc& L, int B) {
+  return L.kind == FF_LINEAR ? tc_tn_ok(L.N, L.K, B) : (tc_conv_ok(L) && L.N % 16 == 0);
+}
 
-// Box rows of the B operand: all 256 tile columns for a single CTA, this CTA's 128 for a pair.
-inline uint32_t tc_b_box_rows(const TcState& t, long long out_rows, long long out_cols) {
-  return (uint32_t)(TC_BN / tc_pick_ncta(t, out_rows, out_cols));
+// Split count of the convolution weight gradient (its output N x 9*Cin has few tiles, its contraction
+// runs over every output position of a set): as many splits as keep every SM (pair) busy with one
+// work item, at least 8 contraction blocks each.  sm_count <= 0: assume 148.
+inline int tc_conv_update_splits(const ff_layer_desc& L, int B, int sm_count, int force_ncta) {
+  if (sm_count <= 0) sm_count = 148;
+  const int ncta = force_ncta ? force_ncta : (L.N > TC_BM ? 2 : 1);
+  const long long tiles = (long long)cdiv(L.N, TC_BM * ncta) * cdiv(L.K, TC_BN);
+  const long long kblocks = (long long)B * L.H * L.Wd / 128;
+  long long splits = (sm_count / ncta) / tiles;
+  if (splits > kblocks / 8) splits = kblocks / 8;
+  return splits < 1 ? 1 : (int)splits;
+}
+inline size_t tc_conv_update_slab_bytes(const ff_layer_desc& L, int splits) {
+  return (size_t)splits * 2 * L.N * L.K * sizeof(int32_t);
 }
 
 inline ff_status tc_gemm(TcState& t, const int8_t* A, const int8_t* Bm, int32_t* C, int M, int N, int K, int trans,
@@ -723,43 +868,64 @@ inline ff_status tc_gemm(TcState& t, const int8_t* A, const int8_t* Bm, int32_t*
   p.out_rows = M;
   p.out_cols = N;
   p.npass = 1;
+  p.splits = 1;
   p.status = status;
   p.C = C;
+  const int ncta = tc_pick_ncta(t, M, N);
   if (!trans) {
-    p.kblocks = cdiv(K, TC_BKB);
-    if ((s = tc_make_map(t, &ta, A, K, M, 0, TC_BKB, TC_BM)) != FF_OK) return s;
-    if ((s = tc_make_map(t, &tb, Bm, K, N, 0, TC_BKB, tc_b_box_rows(t, M, N))) != FF_OK) return s;
-    return tc_launch<TC_MODE_RAW, false>(t, ta, tb, p, st);
+    p.kblocks = cdiv(K, 128);
+    if ((s = tc_make_map(t, &ta, A, K, M, 0, 128, TC_BM)) != FF_OK) return s;
+    if ((s = tc_make_map(t, &tb, Bm, K, N, 0, 128, TC_BN / ncta)) != FF_OK) return s;
+    return tc_launch<TC_MODE_RAW, false, 128>(t, ncta, ta, tb, p, st);
   }
   p.kblocks = cdiv(K, 128);
   if ((s = tc_make_map(t, &ta, A, M, K, 1, 128, 128)) != FF_OK) return s;
   if ((s = tc_make_map(t, &tb, Bm, N, K, 1, 128, 128)) != FF_OK) return s;
-  return tc_launch<TC_MODE_RAW, true>(t, ta, tb, p, st);
+  return tc_launch<TC_MODE_RAW, true, 128>(t, ncta, ta, tb, p, st);
 }
 
 inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint32_t* status, cudaStream_t st) {
   ff_status s = tc_init(t);
   if (s != FF_OK) return s;
-  const int M = 2 * B;
+  const bool conv = L.kind == FF_CONV3X3;
+  const int R = conv ? L.H * L.Wd : 1;
+  const int M = 2 * B * R;
   CUtensorMap ta, tb;
   TcParams p = {};
   p.out_rows = M;
   p.out_cols = L.N;
-  p.kblocks = cdiv(L.K, TC_BKB);
   p.npass = 1;
+  p.splits = 1;
   p.status = status;
   p.Y = b.Y;
   p.acc_dump = b.acc_dump;
   p.S = reinterpret_cast<unsigned long long*>(b.S);
   p.rowmax = b.rowmax;
   p.absmax = b.absmax;
-  p.rows_per_pass = B;
-  p.rows_per_sample = 1;
-  if ((s = tc_make_map(t, &ta, b.Xq, L.K, M, 0, TC_BKB, TC_BM)) != FF_OK) return s;
-  if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, TC_BKB, tc_b_box_rows(t, M, L.N))) != FF_OK) return s;
-  return tc_launch<TC_MODE_FWD, false>(t, ta, tb, p, st);
+  p.rows_per_pass = B * R;
+  p.rows_per_sample = R;
+  const int ncta = tc_pick_ncta(t, M, L.N);
+  if (!conv) {
+    p.kblocks = cdiv(L.K, 128);
+    if ((s = tc_make_map(t, &ta, b.Xq, L.K, M, 0, 128, TC_BM)) != FF_OK) return s;
+    if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, 128, TC_BN / ncta)) != FF_OK) return s;
+    return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st);
+  }
+  const int ch = L.Cin % 128 == 0 ? 128 : 64;
+  p.conv_W = L.Wd;
+  p.conv_H = L.H;
+  p.conv_TH = 128 / L.Wd;
+  p.conv_cin = L.Cin;
+  p.conv_cpt = L.Cin / ch;
+  p.conv_imgs_per_pass = B;
+  p.kblocks = 9 * p.conv_cpt;
+  if ((s = tc_make_map_nhwc(t, &ta, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_TH)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, ch, TC_BN / ncta)) != FF_OK) return s;
+  if (ch == 128) return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st);
+  return tc_launch<TC_MODE_FWD, false, 64>(t, ncta, ta, tb, p, st);
 }
 
+// Dense weight gradient + update in one kernel.
 inline ff_status tc_update(TcState& t, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint32_t* status, cudaStream_t st) {
   ff_status s = tc_init(t);
   if (s != FF_OK) return s;
@@ -769,6 +935,7 @@ inline ff_status tc_update(TcState& t, const ff_layer_desc& L, const ff_layer_bu
   p.out_cols = L.K;
   p.kblocks = cdiv(B, 128);
   p.npass = 2;
+  p.splits = 1;
   p.status = status;
   p.W = b.W;
   p.accW_dump = b.accW_dump;
@@ -776,7 +943,39 @@ inline ff_status tc_update(TcState& t, const ff_layer_desc& L, const ff_layer_bu
   p.lr = L.lr;
   if ((s = tc_make_map(t, &ta, b.dHq, L.N, B, 2, 128, 128)) != FF_OK) return s;
   if ((s = tc_make_map(t, &tb, b.Xq, L.K, B, 2, 128, 128)) != FF_OK) return s;
-  return tc_launch<TC_MODE_UPD, true>(t, ta, tb, p, st);
+  return tc_launch<TC_MODE_UPD, true, 128>(t, tc_pick_ncta(t, L.N, L.K), ta, tb, p, st);
+}
+
+// Convolution weight gradient: split contraction, INT32 partial sums of both sets to `slabs`
+// ([splits][2][N][K]); the caller adds the slabs and applies the update.  *splits_out = slabs written.
+inline ff_status tc_conv_update(TcState& t, const ff_layer_desc& L, const ff_layer_bufs& b, int B, int32_t* slabs, int splits,
+                                int* splits_out, uint32_t* status, cudaStream_t st) {
+  ff_status s = tc_init(t);
+  if (s != FF_OK) return s;
+  CUtensorMap ta, tb;
+  TcParams p = {};
+  const int ch = L.Cin % 128 == 0 ? 128 : 64;
+  const int pos_per_pass = B * L.H * L.Wd;
+  p.out_rows = L.N;
+  p.out_cols = L.K;
+  p.kblocks = pos_per_pass / 128;
+  p.npass = 2;
+  p.splits = splits;
+  p.status = status;
+  p.slabs = slabs;
+  p.conv_W = L.Wd;
+  p.conv_H = L.H;
+  p.conv_TH = 128 / L.Wd;
+  p.conv_cin = L.Cin;
+  p.conv_cpt = L.Cin / ch;
+  p.conv_imgs_per_pass = B;
+  const int kb_per_split = cdiv(p.kblocks, splits);
+  *splits_out = cdiv(p.kblocks, kb_per_split);
+  const int ncta = t.force_ncta ? t.force_ncta : (L.N > TC_BM ? 2 : 1);
+  if ((s = tc_make_map(t, &ta, b.dHq, L.N, pos_per_pass, 2, 128, 128)) != FF_OK) return s;
+  if ((s = tc_make_map_nhwc(t, &tb, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_TH)) != FF_OK) return s;
+  if (ch == 128) return tc_launch<TC_MODE_SLAB, true, 128>(t, ncta, ta, tb, p, st);
+  return tc_launch<TC_MODE_SLAB, true, 64>(t, ncta, ta, tb, p, st);
 }
 
 }  // namespace ffi8

@@ -66,7 +66,9 @@ def workload(name: str) -> Workload:
                         "kaiming_uniform", 200, lam_per_step=0.001)
     if name == "cnn":               # config 4
         chans = [3, 64, 128, 256]
-        layers = [LayerCfg(1, 9 * ci, co, float(co * 1024), 0.03, float(np.sqrt(co * 1024)),
+        # theta = number of outputs per sample (goodness is a sum over C_out*H*W activities); the
+        # step size is the MLP one divided by the H*W positions a filter's gradient sums over
+        layers = [LayerCfg(1, 9 * ci, co, float(co * 1024), 0.03 / 1024.0, float(np.sqrt(co * 1024)),
                            H=32, Wd=32, Cin=ci) for ci, co in zip(chans[:-1], chans[1:])]
         return Workload(name, 256, layers, (32, 32, 3), "normal", "kaiming_uniform", 50)
     if name == "roofline":          # config 5

@@ -126,6 +126,27 @@ def test_config4_cnn_scaled(path):
     _run_and_compare(w, seed=21, steps=2, lam_per_step=0.0, path=path)
 
 
+def _conv_workload(chans, H, Wd, B):
+    layers = [synth.LayerCfg(1, 9 * ci, co, float(co * H * Wd) / 2, 0.03, float(np.sqrt(co * H * Wd)), H=H, Wd=Wd, Cin=ci)
+              for ci, co in zip(chans[:-1], chans[1:])]
+    return synth.Workload("conv_case", B, layers, (H, Wd, chans[0]), "normal", "kaiming_uniform", 2)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("chans,H,Wd,B", [((3, 64, 128, 64), 32, 32, 2),     # config 4's channel widths: 64- and 128-byte taps
+                                          ((3, 64, 256, 128), 8, 16, 3),     # 8 image rows per 128-position block, odd batch
+                                          ((3, 128, 80), 16, 64, 1)])        # ragged Cout, 2 rows per block
+def test_conv_tensor_core_shapes(path, chans, H, Wd, B):
+    _run_and_compare(_conv_workload(chans, H, Wd, B), seed=31, steps=2, lam_per_step=0.1, path=path)
+
+
+@pytest.mark.parametrize("form", TENSOR_FORMS)
+@pytest.mark.parametrize("chans", [(64, 128), (128, 256)])
+def test_conv_layer_forced_tensor_path(chans, form):
+    # FF_GEMM_TENSOR fails instead of falling back, so this proves the tcgen05 implicit-GEMM kernels ran
+    _run_and_compare(_conv_workload(chans, 32, 32, 2), seed=33, steps=2, lam_per_step=0.0, path=(ffb.FF_GEMM_TENSOR, form))
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_config5_roofline_scaled(path):
     w = synth.scaled(synth.workload("roofline"), B=256, width_div=8)   # 8192 -> 1024, theta = N/2
