@@ -189,6 +189,37 @@ ff_status ff_profile_stop(ff_ctx* ctx, void* cuda_stream, float* ms_per_kernel, 
 ff_status ff_int8_gemm(ff_ctx* ctx, const int8_t* A, const int8_t* B, int32_t* C, int M, int N,
                        int K, int trans, void* cuda_stream);
 
+/* Loss, per-sample coefficient and g^Y range of one layer without any caller-provided scratch.
+ * (The paper has no counterpart: this is a packaging variant of the loss step of
+ * ff_layer_loss_grad, not a different computation.)
+ *
+ * Who it is for: code that runs where device memory cannot be allocated -- a plug-in called inside
+ * another framework's stream callback or memory-pool critical section, a process whose memory was
+ * handed out in full at start-up, a caller that holds no ff_ctx and no workspace.  Everything else
+ * in this library keeps its partial sums in the workspace the caller allocates; here they live in a
+ * small array (about 4 KiB) built into the library image, which every GPU that loads the library
+ * keeps until the process ends.  The call allocates nothing: no cudaMalloc, no cudaFree, no
+ * workspace, no context.
+ *
+ * Same arithmetic and same outputs as the loss kernel behind ff_layer_loss_grad: reads G [2B],
+ * rowmax [2B] and absmax[FF_A_X_POS..FF_A_W]; writes coef [2B], loss [1] and
+ * absmax[FF_A_DH_POS..FF_A_DH_NEG].  It does not quantise g^Y.  All pointers are device pointers
+ * on the CURRENT device; G_later / theta_later are host arrays as in ff_layer_loss_grad.
+ *
+ * Limits and rules:
+ *  - 2*B <= FF_STATIC_LOSS_MAX_SAMPLES (the array is laid out for that many samples); larger
+ *    batches are refused with FF_ERR_RANGE.
+ *  - The first call on each device looks up the array's device address (a synchronous runtime
+ *    query); make that first call before starting any stream capture on that device.
+ *  - All calls share the one array per device.  It keeps the previous call's contents; the call
+ *    clears the one word that must start at zero.  Two calls whose kernels can run at the same time
+ *    on one device (different streams) race on it: keep calls on a device in stream order.
+ *  - `err` (nullable) receives a short text when the return value is not FF_OK. */
+#define FF_STATIC_LOSS_MAX_SAMPLES 65536
+ff_status ff_loss_coef_static(const float* G, float theta, const float* const* G_later, const float* theta_later,
+                              int n_later, float lambda, int B, const int32_t* rowmax, float* absmax, float* coef,
+                              float* loss, void* cuda_stream, char* err, size_t err_len);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,8 @@ FF_ABSMAX_LEN = 8
 EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", "ff_set_gemm_path", "ff_set_tensor_form",
            "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step",
            "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
-           "ff_profile_start", "ff_profile_stop"]
+           "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static"]
+FF_STATIC_LOSS_MAX_SAMPLES = 65536
 FF_K_NAMES = ["absmax", "quantize", "zero_stats", "fwd_gemm", "finalize", "normalize", "loss", "dh_quantize",
               "upd_gemm", "raw_gemm"]
 
@@ -82,6 +83,8 @@ def load(build_if_missing: bool = True):
     lib.ff_launch_count.restype = u64
     lib.ff_int8_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ff_profile_start.argtypes = [vp]
+    lib.ff_loss_coef_static.argtypes = [vp, f32, C.POINTER(vp), C.POINTER(f32), i32, f32, i32, vp, vp, vp, vp, vp,
+                                        C.c_char_p, C.c_size_t]
     lib.ff_profile_stop.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(C.c_uint32)]
     for name in EXPORTS:
         if name not in ("ff_last_error", "ff_launch_count"):
@@ -167,6 +170,20 @@ def ff_profile_stop(ctx, stream: int = 0):
     cnt = (C.c_uint32 * n)()
     _check(ctx, load().ff_profile_stop(ctx, stream, ms, cnt))
     return {FF_K_NAMES[i]: (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i]}
+
+
+def ff_loss_coef_static(G: int, theta: float, G_later: Sequence[int], theta_later: Sequence[float], lam: float, B: int,
+                        rowmax: int, absmax: int, coef: int, loss: int, stream: int = 0):
+    """Loss / coefficient step with the library's built-in scratch array: needs no context and no
+    workspace and allocates nothing (for callers that cannot allocate device memory).  Arguments
+    are device addresses on the current device."""
+    n = len(G_later)
+    gp = (C.c_void_p * max(n, 1))(*G_later)
+    th = (C.c_float * max(n, 1))(*theta_later)
+    buf = C.create_string_buffer(256)
+    code = load().ff_loss_coef_static(G, theta, gp, th, n, lam, B, rowmax, absmax, coef, loss, stream, buf, len(buf))
+    if code != FF_OK:
+        raise FFError(code, buf.value.decode())
 
 
 def ff_int8_gemm(ctx, A: int, B: int, Cptr: int, M: int, N: int, K: int, trans: int, stream: int = 0):

@@ -640,4 +640,88 @@ ff_status ff_int8_gemm(ff_ctx* ctx, const int8_t* A, const int8_t* Bm, int32_t* 
   return launch_simt<DenseView, DenseView, true, 1>(ctx, dense(A, K, M), dense(Bm, K, N), M, N, K, epi, st);
 }
 
+// ------------------------------------------------------------------------------------------------
+// ff_loss_coef_static: the loss / coefficient kernel with its partial-sum scratch in a fixed device
+// array instead of the caller's workspace.
+//
+// The array below is part of the library image: every GPU that loads the library holds these few
+// kilobytes until the process exits.  In host code the name `g_static_loss_scratch` is only a handle;
+// the device address the kernel needs comes from cudaGetSymbolAddress, asked for once per device
+// while that device is current.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_loss_scratch[sizeof(LossScratch)];
+static_assert(FF_STATIC_LOSS_MAX_SAMPLES == LOSS_MAX_BLOCKS * LOSS_THREADS, "one scratch slot per block of LOSS_THREADS samples");
+
+namespace {
+constexpr int STATIC_MAX_DEVICES = 64;
+LossScratch* g_static_loss_ptr[STATIC_MAX_DEVICES] = {nullptr};
+
+void static_err(char* err, size_t err_len, const char* msg, const char* detail = "") {
+  if (err && err_len) snprintf(err, err_len, "%s%s", msg, detail);
+}
+}  // namespace
+
+ff_status ff_loss_coef_static(const float* G, float theta, const float* const* G_later, const float* theta_later, int n_later,
+                              float lambda, int B, const int32_t* rowmax, float* absmax, float* coef, float* loss,
+                              void* cuda_stream, char* err, size_t err_len) {
+  if (!G || !rowmax || !absmax || !coef || !loss) {
+    static_err(err, err_len, "a required device pointer is NULL");
+    return FF_ERR_ARG;
+  }
+  if (B <= 0) {
+    static_err(err, err_len, "B must be positive");
+    return FF_ERR_ARG;
+  }
+  if (2LL * B > FF_STATIC_LOSS_MAX_SAMPLES) {
+    static_err(err, err_len, "2*B exceeds FF_STATIC_LOSS_MAX_SAMPLES, the size the built-in scratch array was laid out for");
+    return FF_ERR_RANGE;
+  }
+  if (n_later < 0 || n_later > FF_MAX_LATER || (n_later > 0 && (!G_later || !theta_later))) {
+    static_err(err, err_len, "bad list of later layers");
+    return FF_ERR_ARG;
+  }
+  LaterLayers later;
+  later.n = n_later;
+  for (int j = 0; j < n_later; ++j) {
+    if (!G_later[j]) {
+      static_err(err, err_len, "a G_later pointer is NULL");
+      return FF_ERR_ARG;
+    }
+    later.G[j] = G_later[j];
+    later.theta[j] = theta_later[j];
+  }
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) {
+    static_err(err, err_len, "cudaGetDevice: ", e != cudaSuccess ? cudaGetErrorString(e) : "device index out of range");
+    return FF_ERR_CUDA;
+  }
+  if (!g_static_loss_ptr[dev]) {
+    // first call on this device: turn the symbol into the address of this device's copy of the array
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_loss_scratch);
+    if (e != cudaSuccess || !ptr) {
+      static_err(err, err_len, "cudaGetSymbolAddress: ", cudaGetErrorString(e));
+      return FF_ERR_CUDA;
+    }
+    g_static_loss_ptr[dev] = static_cast<LossScratch*>(ptr);
+  }
+  LossScratch* scratch = g_static_loss_ptr[dev];
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // the array keeps whatever the last call left: the block-completion ticket has to start at zero
+  e = cudaMemsetAsync(&scratch->ticket, 0, sizeof(scratch->ticket), st);
+  if (e != cudaSuccess) {
+    static_err(err, err_len, "cudaMemsetAsync: ", cudaGetErrorString(e));
+    return FF_ERR_CUDA;
+  }
+  const int blocks = (2 * B + LOSS_THREADS - 1) / LOSS_THREADS;  // <= LOSS_MAX_BLOCKS by the size check above
+  loss_coef_kernel<<<blocks, LOSS_THREADS, 0, st>>>(G, theta, later, lambda, B, rowmax, absmax, coef, loss, scratch);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    static_err(err, err_len, "launch: ", cudaGetErrorString(e));
+    return FF_ERR_CUDA;
+  }
+  return FF_OK;
+}
+
 }  // extern "C"
