@@ -205,9 +205,11 @@ inline int simt_split_count(int clen, int splits) {
 }
 
 ff_status launch_slab_update(ff_ctx* ctx, const int32_t* slabs, int splits, const ff_layer_desc& L, const ff_layer_bufs& b,
-                             cudaStream_t st) {
+                             cudaStream_t st, int pitch = 0) {
   const size_t plane = (size_t)L.N * L.K;
-  slab_update_kernel<<<ew_blocks(ctx, plane, 1), 256, 0, st>>>(slabs, splits, plane, b.W, b.absmax, L.lr, b.accW_dump);
+  const size_t want = (plane + 31) / 32, cap = (size_t)ctx->sm_count * 8;
+  slab_update_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, L.K, pitch ? pitch : L.K, b.W,
+                                                                          b.absmax, L.lr, b.accW_dump);
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }

@@ -184,25 +184,86 @@ struct SlabEpilogue {
 };
 
 // Adds the `splits` INT32 slabs of both sets and applies the dequantised SGD update (Sec. IV-B;
-// Alg. 1 line 9): W <- W - lr*(float(accP)*cP + float(accN)*cN).  plane = N*K elements.
-__global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane,
-                                                          float* __restrict__ W, const float* __restrict__ absmax, float lr,
-                                                          int32_t* __restrict__ accW_dump) {
+// Alg. 1 line 9): W <- W - lr*(float(accP)*cP + float(accN)*cN).  plane = rows*cols elements of W;
+// the slabs may have a wider row pitch (cols <= pitch).  A block covers 32 consecutive elements; its
+// 8 warps take the splits round-robin (coalesced along the elements) and their integer partial
+// sums meet in shared memory.
+__global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane, int cols,
+                                                          int pitch, float* __restrict__ W, const float* __restrict__ absmax,
+                                                          float lr, int32_t* __restrict__ accW_dump) {
+  __shared__ int part[2][8][32];
+  const int lane = threadIdx.x & 31, zl = threadIdx.x >> 5;
   const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
   const float cN = __fmul_rn(scale_of(absmax[4]), scale_of(absmax[1]));
-  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < plane; e += (size_t)gridDim.x * blockDim.x) {
+  const size_t splane = plane / cols * pitch;  // elements of one slab
+  for (size_t e0 = (size_t)blockIdx.x * 32; e0 < plane; e0 += (size_t)gridDim.x * 32) {
+    const size_t e = e0 + lane;
     int aP = 0, aN = 0;
-    for (int z = 0; z < splits; ++z) {
-      aP += slabs[((size_t)z * 2) * plane + e];
-      aN += slabs[((size_t)z * 2 + 1) * plane + e];
+    if (e < plane) {
+      const size_t se = pitch == cols ? e : e / cols * pitch + e % cols;
+      for (int z = zl; z < splits; z += 8) {
+        aP += __ldg(slabs + ((size_t)z * 2) * splane + se);
+        aN += __ldg(slabs + ((size_t)z * 2 + 1) * splane + se);
+      }
     }
-    const float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
-    W[e] = __fsub_rn(W[e], __fmul_rn(lr, g));
-    if (accW_dump) {
-      accW_dump[e] = aP;
-      accW_dump[plane + e] = aN;
+    part[0][zl][lane] = aP;
+    part[1][zl][lane] = aN;
+    __syncthreads();
+    if (zl == 0 && e < plane) {
+#pragma unroll
+      for (int k = 1; k < 8; ++k) {
+        aP += part[0][k][lane];
+        aN += part[1][k][lane];
+      }
+      const float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
+      W[e] = __fsub_rn(W[e], __fmul_rn(lr, g));
+      if (accW_dump) {
+        accW_dump[e] = aP;
+        accW_dump[plane + e] = aN;
+      }
     }
+    __syncthreads();
   }
+}
+
+// Explicit INT8 im2col for 3x3 / stride 1 / zero-pad 1 convolutions with few input channels (the
+// first layer of an image network: 9*Cin <= 128): row = output position, column (r*3+s)*Cin + ci,
+// zero beyond 9*Cin up to the padded width KPAD (a multiple of 16).  The padded matrix feeds the
+// dense tensor-core kernels.  One thread per output position.
+template <int KPAD>
+__global__ void __launch_bounds__(256) im2col3x3_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ out, int rows, int H,
+                                                        int W, int Cin) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= rows) return;
+  const int w = row % W, t = row / W;
+  const int h = t % H, b = t / H;
+  __align__(16) int8_t v[KPAD];
+#pragma unroll
+  for (int i = 0; i < KPAD; ++i) v[i] = 0;
+  int k = 0;
+  for (int r = 0; r < 3; ++r)
+    for (int s = 0; s < 3; ++s) {
+      const int hh = h + r - 1, ww = w + s - 1;
+      const bool in = hh >= 0 && hh < H && ww >= 0 && ww < W;
+      const int8_t* src = x + ((size_t)(b * H + hh) * W + ww) * Cin;
+      for (int ci = 0; ci < Cin; ++ci, ++k) {
+        const int8_t val = in ? src[ci] : (int8_t)0;
+#pragma unroll
+        for (int i = 0; i < KPAD; ++i)  // static indexing keeps v in registers
+          if (i == k) v[i] = val;
+      }
+    }
+  uint4* dst = reinterpret_cast<uint4*>(out + (size_t)row * KPAD);
+#pragma unroll
+  for (int i = 0; i < KPAD / 16; ++i) dst[i] = reinterpret_cast<const uint4*>(v)[i];
+}
+// Rows of an INT8 matrix [rows, cols] copied to a zero-padded pitch.
+__global__ void __launch_bounds__(256) pad_rows_kernel(const int8_t* __restrict__ in, int8_t* __restrict__ out, int rows, int cols,
+                                                       int pitch) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * pitch) return;
+  const int r = i / pitch, c = i - r * pitch;
+  out[i] = c < cols ? in[(size_t)r * cols + c] : (int8_t)0;
 }
 
 // ---- kernel ------------------------------------------------------------------------------

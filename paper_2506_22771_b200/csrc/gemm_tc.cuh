@@ -7,8 +7,8 @@
 // producer fetches, per filter tap, a box of the input shifted by the tap offset with a 4-D TMA
 // copy whose out-of-image part is zero-filled (zero is exact in the symmetric quantiser).
 //
-// One kernel template.  192 threads: warp 0 = TMA producer, warp 1 = MMA issuer (one elected lane
-// each), warps 2..5 = epilogue (one TMEM lane quadrant each).
+// One kernel template.  320 threads: warp 0 = TMA producer, warp 1 = MMA issuer (one elected lane
+// each), warps 2..9 = epilogue (two warps per TMEM lane quadrant; they share the tile's columns).
 // NCTA = 1: output tile 128 x 256 per CTA.  NCTA = 2: the two CTAs of a cluster share a 256 x 256
 // tile (tcgen05 cta_group::2): each stages its own 128 rows of A and one half (128 columns) of B;
 // the CTA of cluster rank 0 issues the MMAs for both and holds the barriers the pair synchronises
@@ -28,6 +28,7 @@
 #include <cuda.h>
 
 #include <cstdio>
+#include <cstring>
 #include <unordered_map>
 
 #include "../../include/ffint8.h"
@@ -36,10 +37,11 @@
 namespace ffi8 {
 
 constexpr int TC_BM = 128, TC_BN = 256;  // tile rows per CTA, tile columns
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;
+constexpr int TC_EPI_WARPS = 8;                           // two per TMEM lane quadrant
+constexpr int TC_EPI_COLS = TC_BN / 2;                    // most accumulator columns one epilogue warp takes
 constexpr int TC_MAX_STAGES = 8;
-constexpr int TC_STG_PITCH = 36;                          // floats per staged row (32 + 4: 16-byte aligned, conflict-free)
-constexpr uint32_t TC_STG_BYTES = 32 * TC_STG_PITCH * 4;  // one 32 x 32 FP32 staging patch per epilogue warp
+constexpr uint32_t TC_PATCH_BYTES = 32 * 32 * 4;          // one 32 x 32 FP32 staging patch per epilogue warp (128-byte swizzle)
 constexpr uint32_t TC_RING_BYTES = 192 * 1024;            // operand ring budget
 constexpr int TC_PREFETCH_KB = 8;                         // W tile is prefetched into L2 this many k-blocks before the epilogue
 constexpr int TC_GROUP_M = 16;                            // tile rows per rasterisation group (L2 reuse)
@@ -55,7 +57,7 @@ struct TcGeom {
   static constexpr uint32_t B_BYTES = MN_MAJOR ? 128u * (TC_BN / NCTA) : (uint32_t)(TC_BN / NCTA) * CH;
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (int)(TC_RING_BYTES / STAGE_BYTES) < TC_MAX_STAGES ? (int)(TC_RING_BYTES / STAGE_BYTES) : TC_MAX_STAGES;
-  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + 4 * TC_STG_BYTES;
+  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + TC_EPI_WARPS * TC_PATCH_BYTES + 1024 /*align*/ + 256 /*barriers*/;
   static constexpr int MMAS = MN_MAJOR ? 4 : CH / 32;            // MMAs (K = 32) per contraction block
   static constexpr int B_BOXES = MN_MAJOR ? (TC_BN / NCTA) / CH : 1;  // TMA boxes of the B operand per stage
   static constexpr uint32_t SWZ = CH == 128 ? 2u : 4u;             // descriptor swizzle code: 128-byte / 64-byte
@@ -79,6 +81,7 @@ struct TcParams {
   int32_t* rowmax;
   const float* absmax;
   int rows_per_pass, rows_per_sample;
+  int y_tma;                // Y leaves through TMA stores (needs N % 4 == 0); else plain stores
   // update epilogue
   float* W;
   int32_t* accW_dump;
@@ -240,6 +243,27 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, int (&r)[32]) {
       : "memory");
 }
 // (the wait for the load is part of tc_ld32, so the registers are valid when it returns)
+// The same load without the wait: the registers are valid after the next tc_wait_ld().
+__device__ __forceinline__ void tc_ld32_async(uint32_t taddr, int (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// TMA store of one staged box to global memory (clipped at the tensor's edge), bulk async-group completion.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(reinterpret_cast<uint64_t>(tm)),
+               "r"(src), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // Shared-memory matrix descriptor for a swizzled operand tile whose rows are CH = 128 (swz = 2) or
 // 64 (swz = 4) bytes long; 8 rows form one swizzle atom.  K-major: rows are M/N indices, SBO = 8 rows
@@ -273,24 +297,26 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 // ---- kernel --------------------------------------------------------------------------------
 template <int MODE, bool MN_MAJOR, int NCTA, int CH>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-    tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+    tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                   const __grid_constant__ CUtensorMap tmY, const TcParams p) {
   using G = TcGeom<MN_MAJOR, NCTA, CH>;
   constexpr int STAGES = G::STAGES;
   constexpr uint32_t STAGE_BYTES = G::STAGE_BYTES;
   constexpr bool PAIR = NCTA == 2;
   extern __shared__ uint8_t smem_raw[];
-  // 1024-byte aligned operand ring, then the barriers (identical offsets in both CTAs of a pair)
+  // 1024-byte aligned operand ring, then the epilogue patches, then the barriers (identical offsets in
+  // both CTAs of a pair)
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t ring = (raw + 1023u) & ~1023u;
   uint8_t* ring_ptr = smem_raw + (ring - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ring_ptr + STAGES * STAGE_BYTES);
+  uint8_t* patch_all = ring_ptr + STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(patch_all + TC_EPI_WARPS * TC_PATCH_BYTES);
   const uint32_t bar_full = smem_u32(bars);                      // [STAGES]  used in the leader CTA
   const uint32_t bar_empty = bar_full + 8 * TC_MAX_STAGES;       // [STAGES]  one set per CTA
   const uint32_t bar_tfull = bar_empty + 8 * TC_MAX_STAGES;      // [2]       one set per CTA
   const uint32_t bar_tempty = bar_tfull + 16;                    // [2]       used in the leader CTA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_MAX_STAGES + 4);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  float* stage_all = reinterpret_cast<float*>(ring_ptr + STAGES * STAGE_BYTES + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = leader of the pair
@@ -306,7 +332,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar_tfull + 8 * s, 1);
-      mbar_init(bar_tempty + 8 * s, 4 * NCTA);  // one arrive per epilogue warp of every CTA of the group
+      mbar_init(bar_tempty + 8 * s, TC_EPI_WARPS * NCTA);  // one arrive per epilogue warp of every CTA of the group
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -357,11 +383,35 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         const int f_h0 = (!MN_MAJOR && p.conv_W) ? (row0 - f_img * hw) / p.conv_W : 0;
         // bytes the leader's barrier expects per stage from all CTAs of the group
         uint32_t stage_tx = STAGE_BYTES * NCTA;
+        // weight-gradient convolution: filter tap and first channel of each of this CTA's B boxes
+        int b_ci0[G::B_BOXES], b_r[G::B_BOXES], b_s[G::B_BOXES];
         if (MN_MAJOR && p.conv_W) {
           const int valid_cols = min(TC_BN, p.out_cols - tn * TC_BN);  // a multiple of CH
           stage_tx = G::A_BYTES * NCTA + (uint32_t)valid_cols * 128u;
+#pragma unroll
+          for (int q = 0; q < G::B_BOXES; ++q) {
+            const int c = col0 + q * CH, tap = c / p.conv_cin;
+            b_ci0[q] = c - tap * p.conv_cin;
+            b_r[q] = tap / 3;
+            b_s[q] = tap - b_r[q] * 3;
+          }
         }
         for (int pass = 0; pass < p.npass && ok; ++pass) {
+          // forward convolution: (filter row, filter column, channel chunk) of k-block kb, kept by counting
+          int f_r = 0, f_s = 0, f_cc = 0;
+          if (!MN_MAJOR && p.conv_W) {
+            const int tap = kb0 / p.conv_cpt;
+            f_cc = kb0 - tap * p.conv_cpt;
+            f_r = tap / 3;
+            f_s = tap - f_r * 3;
+          }
+          // weight-gradient convolution: image and block of image rows of contraction block kb
+          int g_img = 0, g_blk = 0;
+          if (MN_MAJOR && p.conv_W) {
+            g_img = kb0 / blocks_per_img;
+            g_blk = kb0 - g_img * blocks_per_img;
+            g_img += pass * p.conv_imgs_per_pass;
+          }
           for (int kb = kb0; kb < kb1; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
             if (!mbar_wait<PAIR>(bar_empty + 8 * s, ph ^ 1u, abort_flag)) {
@@ -384,9 +434,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             if (!MN_MAJOR) {
               if (p.conv_W) {
                 // k-block = CH channels of one filter tap (r, s): the input box shifted by (r-1, s-1)
-                const int tap = kb / p.conv_cpt, cc = kb - tap * p.conv_cpt;
-                const int r = tap / 3, sx = tap - r * 3;
-                tma_load_4d<NCTA>(a_dst, &tmA, fb, cc * CH, sx - 1, f_h0 + r - 1, f_img);
+                tma_load_4d<NCTA>(a_dst, &tmA, fb, f_cc * CH, f_s - 1, f_h0 + f_r - 1, f_img);
+                if (++f_cc == p.conv_cpt) {
+                  f_cc = 0;
+                  if (++f_s == 3) {
+                    f_s = 0;
+                    ++f_r;
+                  }
+                }
               } else {
                 tma_load_2d<NCTA>(a_dst, &tmA, fb, kb * CH, row0);
               }
@@ -397,16 +452,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               if (p.conv_W) {
                 // contraction block kb of set `pass` = conv_TH rows of one image; B column chunk q of the
                 // tile = CH channels of one filter tap, fetched from the shifted input box
-                const int img = pass * p.conv_imgs_per_pass + kb / blocks_per_img;
-                const int h0 = (kb % blocks_per_img) * p.conv_TH;
+                const int h0 = g_blk * p.conv_TH;
 #pragma unroll
-                for (int q = 0; q < G::B_BOXES; ++q) {
-                  const int c = col0 + q * CH;
-                  if (c < p.out_cols) {
-                    const int tap = c / p.conv_cin, ci0 = c - tap * p.conv_cin;
-                    const int r = tap / 3, sx = tap - r * 3;
-                    tma_load_4d<NCTA>(b_dst + q * (128 * CH), &tmB, fb, ci0, sx - 1, h0 + r - 1, img);
-                  }
+                for (int q = 0; q < G::B_BOXES; ++q)
+                  if (col0 + q * CH < p.out_cols)
+                    tma_load_4d<NCTA>(b_dst + q * (128 * CH), &tmB, fb, b_ci0[q], b_s[q] - 1, h0 + b_r[q] - 1, g_img);
+                if (++g_blk == blocks_per_img) {
+                  g_blk = 0;
+                  ++g_img;
                 }
               } else {
 #pragma unroll
@@ -466,9 +519,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     }
     __syncwarp();
   } else {
-    // ------------------------------- epilogue (warps 2..5 of every CTA) -----------------------
-    const int quad = warp & 3;  // TMEM lane quadrant this warp may read
-    float* stg = stage_all + (warp - 2) * (32 * TC_STG_PITCH);
+    // ------------------------------- epilogue (warps 2..9 of every CTA) -----------------------
+    const int quad = warp & 3;                           // TMEM lane quadrant this warp may read
+    const int half = (warp - 2) >> 2;                    // which of the quadrant's two warps
+    uint8_t* patch = patch_all + (warp - 2) * TC_PATCH_BYTES;
+    const uint32_t patch_u32 = smem_u32(patch);
+    (void)patch_u32;
     uint32_t tile_it = 0;
     bool ok = true;
     float c0 = 0.f, c1 = 0.f, cP = 0.f, cN = 0.f;
@@ -497,8 +553,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       const bool row_ok = row < p.out_rows;
       const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
       const int col0 = tn * TC_BN;
+      // the quadrant's two warps share the tile's valid 32-column chunks (a narrow last tile keeps both busy)
+      const int chunks = (min(TC_BN, p.out_cols - col0) + 31) >> 5;
+      const int cbeg = half ? ((chunks + 1) >> 1) * 32 : 0;
+      const int cend = half ? chunks * 32 : ((chunks + 1) >> 1) * 32;
       if (MODE == TC_MODE_RAW) {
-        for (int cb = 0; cb < TC_BN; cb += 32) {
+#pragma unroll 1
+        for (int cb = cbeg; cb < cend; cb += 32) {
           int v[32];
           tc_ld32(t_row + as * TC_BN + cb, v);
           if (row_ok) {
@@ -514,59 +575,73 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           }
         }
       } else if (MODE == TC_MODE_FWD) {
-        // thread = one accumulator row; y staged through smem so that global stores are row-contiguous
+        // thread = one accumulator row.  Rows and columns outside the output hold zero accumulators (their
+        // operand rows were zero-filled by TMA), so the goodness statistics need no masks.  y is staged in
+        // a swizzled 32 x 32 patch and leaves with one TMA store per patch (clipped at the output's edge);
+        // the TMEM load of the next 32 columns is in flight while this chunk is processed.
         const float c = row < p.rows_per_pass ? c0 : c1;
         unsigned long long ssum = 0ull;
         int mx = 0;
-        for (int cb = 0; cb < TC_BN; cb += 32) {
-          if (col0 + cb >= p.out_cols) break;  // uniform across the warp
-          int v[32];
-          tc_ld32(t_row + as * TC_BN + cb, v);
-          const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
+        int v[2][32];
+        if (cbeg < cend) tc_ld32_async(t_row + as * TC_BN + cbeg, v[0]);
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            float y[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const int a = v[j + q];
-              y[q] = dequant_relu(a, c);
-              if (full || col0 + cb + j + q < p.out_cols) {
-                const int rl = max(a, 0);
-                ssum += (unsigned long long)((long long)rl * (long long)rl);
-                mx = max(mx, rl);
-              }
+        for (int i = 0; i < TC_EPI_COLS / 32; ++i) {
+          const int cb = cbeg + i * 32;
+          tc_wait_ld();
+          if (i + 1 < TC_EPI_COLS / 32 && cb + 32 < cend) tc_ld32_async(t_row + as * TC_BN + cb + 32, v[(i + 1) & 1]);
+          if (cb < cend) {  // uniform across the warp
+            const int(&a)[32] = v[i & 1];
+            if (p.y_tma) {  // the previous store of this warp must have read the patch
+              if (lane == 0) bulk_wait_read0();
+              __syncwarp();
             }
-            *reinterpret_cast<float4*>(stg + lane * TC_STG_PITCH + j) = make_float4(y[0], y[1], y[2], y[3]);
-          }
-          __syncwarp();
-          // lanes 0..7 of each quarter-warp cover one staged row: 4 rows x 128 bytes per store instruction
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int r = i * 4 + (lane >> 3), cc = (lane & 7) * 4;
-            const int grow = wrow0 + r, gcol = col0 + cb + cc;
-            if (grow < p.out_rows) {
-              const float4 yv = *reinterpret_cast<const float4*>(stg + r * TC_STG_PITCH + cc);
-              float* dst = p.Y + (size_t)grow * p.out_cols + gcol;
-              if (full) {
-                *reinterpret_cast<float4*>(dst) = yv;
-              } else {
-                const float yy[4] = {yv.x, yv.y, yv.z, yv.w};
+            for (int j = 0; j < 32; j += 4) {
+              float y[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                  if (gcol + q < p.out_cols) dst[q] = yy[q];
+              for (int q = 0; q < 4; ++q) {
+                // relu on the integer first: float(max(acc,0))*c equals max(0, float(acc)*c) bit for bit (c >= 0)
+                const unsigned rl = (unsigned)max(a[j + q], 0);
+                y[q] = __fmul_rn(__uint2float_rn(rl), c);
+                ssum += (unsigned long long)rl * rl;  // one 32x32+64 multiply-add
+                mx = max(mx, (int)rl);
               }
+              *reinterpret_cast<float4*>(patch + lane * 128 + (((j >> 2) ^ (lane & 7)) << 4)) = make_float4(y[0], y[1], y[2], y[3]);
+            }
+            if (p.y_tma) {
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+              __syncwarp();
+              if (lane == 0 && wrow0 < p.out_rows) {  // a box that starts inside the output; its overhang is clipped
+                tma_store_2d(&tmY, patch_u32, col0 + cb, wrow0);
+                bulk_commit();
+              }
+            } else {
+              __syncwarp();
+              // lanes 0..7 of each quarter-warp cover one staged row: 4 rows x 128 bytes per store instruction
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const int r = k * 4 + (lane >> 3), cc = lane & 7;
+                const int grow = wrow0 + r, gcol = col0 + cb + cc * 4;
+                if (grow < p.out_rows) {
+                  const float4 yv = *reinterpret_cast<const float4*>(patch + r * 128 + ((cc ^ (r & 7)) << 4));
+                  float* dst = p.Y + (size_t)grow * p.out_cols + gcol;
+                  const float yy[4] = {yv.x, yv.y, yv.z, yv.w};
+#pragma unroll
+                  for (int q = 0; q < 4; ++q)
+                    if (gcol + q < p.out_cols) dst[q] = yy[q];
+                }
+              }
+              __syncwarp();
+            }
+            if (p.acc_dump && row_ok) {  // parity dump: plain per-row stores
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + cb + j < p.out_cols) p.acc_dump[(size_t)row * p.out_cols + col0 + cb + j] = a[j];
             }
           }
-          if (p.acc_dump && row_ok) {  // parity dump: plain per-row stores
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + cb + j < p.out_cols) p.acc_dump[(size_t)row * p.out_cols + col0 + cb + j] = v[j];
-          }
-          __syncwarp();
         }
         if ((p.rows_per_sample & 31) == 0) {
-          // the warp's 32 rows belong to one sample (convolution: a sample has H*W rows): one atomic
-          // per warp; rows past the end hold zero accumulators and add nothing
+          // the warp's 32 rows belong to one sample (convolution: a sample has H*W rows): one atomic per warp
           ssum += __shfl_xor_sync(0xffffffffu, ssum, 16);
           ssum += __shfl_xor_sync(0xffffffffu, ssum, 8);
           ssum += __shfl_xor_sync(0xffffffffu, ssum, 4);
@@ -587,8 +662,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         // raw INT32 partial sums of both sets to this split's slab [split][set][rows][cols]
         for (int pass = 0; pass < 2; ++pass) {
           int32_t* slab = p.slabs + (size_t)(split * 2 + pass) * p.out_rows * p.out_cols;
-          for (int cb = 0; cb < TC_BN; cb += 32) {
-            if (col0 + cb >= p.out_cols) break;
+#pragma unroll 1
+          for (int cb = cbeg; cb < cend; cb += 32) {
             int v[32];
             tc_ld32(t_row + pass * TC_BN + cb, v);
             if (row_ok) {
@@ -608,8 +683,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         // thread = one accumulator row computes d = lr*(float(accP)*cP + float(accN)*cN); d is staged
         // through smem so that the read-modify-write of W is row-contiguous
         const size_t plane = (size_t)p.out_rows * p.out_cols;
-        for (int cb = 0; cb < TC_BN; cb += 32) {
-          if (col0 + cb >= p.out_cols) break;
+#pragma unroll 1
+        for (int cb = cbeg; cb < cend; cb += 32) {
           const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
           // issue the (row-contiguous) W loads first so that they are in flight during the TMEM reads
           float4 wv[8];
@@ -622,8 +697,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             }
           }
           int vp[32], vn[32];
-          tc_ld32(t_row + cb, vp);
-          tc_ld32(t_row + TC_BN + cb, vn);
+          tc_ld32_async(t_row + cb, vp);
+          tc_ld32_async(t_row + TC_BN + cb, vn);
+          tc_wait_ld();
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             float d[4];
@@ -632,15 +708,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               const float g = __fadd_rn(__fmul_rn(__int2float_rn(vp[j + q]), cP), __fmul_rn(__int2float_rn(vn[j + q]), cN));
               d[q] = __fmul_rn(p.lr, g);
             }
-            *reinterpret_cast<float4*>(stg + lane * TC_STG_PITCH + j) = make_float4(d[0], d[1], d[2], d[3]);
+            *reinterpret_cast<float4*>(patch + lane * 128 + (((j >> 2) ^ (lane & 7)) << 4)) = make_float4(d[0], d[1], d[2], d[3]);
           }
           __syncwarp();
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const int r = i * 4 + (lane >> 3), cc = (lane & 7) * 4;
-            const int grow = wrow0 + r, gcol = col0 + cb + cc;
+            const int r = i * 4 + (lane >> 3), cc = lane & 7;
+            const int grow = wrow0 + r, gcol = col0 + cb + cc * 4;
             if (grow < p.out_rows) {
-              const float4 dv = *reinterpret_cast<const float4*>(stg + r * TC_STG_PITCH + cc);
+              const float4 dv = *reinterpret_cast<const float4*>(patch + r * 128 + ((cc ^ (r & 7)) << 4));
               float* dst = p.W + (size_t)grow * p.out_cols + gcol;
               if (full) {
                 float4 w = wv[i];
@@ -678,6 +754,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           mbar_arrive(bar_tempty + 8 * as);
       }
     }
+    if (MODE == TC_MODE_FWD && lane == 0) bulk_wait_read0();  // the last stores have read their patches
     if (!ok && lane == 0) raise_abort();
   }
 
@@ -770,8 +847,25 @@ inline int tc_pick_ncta(const TcState& t, long long out_rows, long long out_cols
   return (out_rows > TC_BM && pair_items >= t.sm_count / 2) ? 2 : 1;
 }
 
+// FP32 row-major matrix [rows, cols] for the forward epilogue's TMA stores: boxes of 32 x 32, 128-byte swizzle.
+inline ff_status tc_make_store_map(TcState& t, CUtensorMap* tm, float* base, uint64_t cols, uint64_t rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * sizeof(float)};
+  cuuint32_t box[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = t.encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(t.err, sizeof(t.err), "cuTensorMapEncodeTiled (store map) failed (%d) cols=%llu rows=%llu", (int)r,
+             (unsigned long long)cols, (unsigned long long)rows);
+    return FF_ERR_CUDA;
+  }
+  return FF_OK;
+}
+
 template <int MODE, bool MN_MAJOR, int NCTA, int CH>
-inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap& b, TcParams p, cudaStream_t st) {
+inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& y, TcParams p,
+                             cudaStream_t st) {
   using G = TcGeom<MN_MAJOR, NCTA, CH>;
   auto kern = tc_gemm_kernel<MODE, MN_MAJOR, NCTA, CH>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::SMEM_BYTES);
@@ -808,7 +902,7 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
   }
   const int groups = items < max_groups ? items : max_groups;
   cfg.gridDim = dim3(groups * NCTA, 1, 1);
-  e = cudaLaunchKernelEx(&cfg, kern, a, b, p);
+  e = cudaLaunchKernelEx(&cfg, kern, a, b, y, p);
   if (e != cudaSuccess) {
     snprintf(t.err, sizeof(t.err), "launch: %s", cudaGetErrorString(e));
     return FF_ERR_CUDA;
@@ -817,9 +911,13 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
 }
 
 template <int MODE, bool MN_MAJOR, int CH>
-inline ff_status tc_launch(TcState& t, int ncta, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, cudaStream_t st) {
-  if (ncta == 2) return tc_launch_n<MODE, MN_MAJOR, 2, CH>(t, a, b, p, st);
-  return tc_launch_n<MODE, MN_MAJOR, 1, CH>(t, a, b, p, st);
+inline ff_status tc_launch(TcState& t, int ncta, const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, cudaStream_t st,
+                           const CUtensorMap* y = nullptr) {
+  CUtensorMap none;
+  memset(&none, 0, sizeof(none));
+  const CUtensorMap& ym = y ? *y : none;
+  if (ncta == 2) return tc_launch_n<MODE, MN_MAJOR, 2, CH>(t, a, b, ym, p, st);
+  return tc_launch_n<MODE, MN_MAJOR, 1, CH>(t, a, b, ym, p, st);
 }
 
 // K-major ("NT") problem: A [M,K], B [N,K]; K % 16 == 0 (TMA row pitch), everything else ragged.
@@ -905,11 +1003,15 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   p.rows_per_pass = B * R;
   p.rows_per_sample = R;
   const int ncta = tc_pick_ncta(t, M, L.N);
+  CUtensorMap ty;
+  p.y_tma = (L.N % 4 == 0) ? 1 : 0;
+  if (p.y_tma && (s = tc_make_store_map(t, &ty, b.Y, L.N, M)) != FF_OK) return s;
+  const CUtensorMap* typ = p.y_tma ? &ty : nullptr;
   if (!conv) {
     p.kblocks = cdiv(L.K, 128);
     if ((s = tc_make_map(t, &ta, b.Xq, L.K, M, 0, 128, TC_BM)) != FF_OK) return s;
     if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, 128, TC_BN / ncta)) != FF_OK) return s;
-    return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st);
+    return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st, typ);
   }
   const int ch = L.Cin % 128 == 0 ? 128 : 64;
   p.conv_W = L.Wd;
@@ -921,8 +1023,8 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   p.kblocks = 9 * p.conv_cpt;
   if ((s = tc_make_map_nhwc(t, &ta, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_TH)) != FF_OK) return s;
   if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, ch, TC_BN / ncta)) != FF_OK) return s;
-  if (ch == 128) return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st);
-  return tc_launch<TC_MODE_FWD, false, 64>(t, ncta, ta, tb, p, st);
+  if (ch == 128) return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st, typ);
+  return tc_launch<TC_MODE_FWD, false, 64>(t, ncta, ta, tb, p, st, typ);
 }
 
 // Dense weight gradient + update in one kernel.
