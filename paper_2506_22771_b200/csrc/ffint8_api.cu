@@ -214,11 +214,76 @@ ff_status launch_slab_update(ff_ctx* ctx, const int32_t* slabs, int splits, cons
   return FF_OK;
 }
 
+// ---- explicit-im2col route for convolutions with few input channels -------------------------
+// Transient workspace after the header: [ xi: rows x kpad | wi: N x kpad | slabs ], each 256-byte aligned.
+struct Im2colPlan {
+  int kpad;
+  size_t xi_off, wi_off, slab_off, slab_bytes_per_split;
+  int max_splits;   // that fit the workspace (the wish when ws_bytes = SIZE_MAX); -1: xi / wi do not fit
+};
+inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
+inline Im2colPlan im2col_plan(const ff_layer_desc& L, int B, size_t ws_bytes, int sm_count) {
+  Im2colPlan pl;
+  pl.kpad = tc_im2col_kpad(L);
+  const size_t rows = (size_t)2 * B * L.H * L.Wd;
+  pl.xi_off = WS_BYTES;
+  pl.wi_off = pl.xi_off + up256(rows * pl.kpad);
+  pl.slab_off = pl.wi_off + up256((size_t)L.N * pl.kpad);
+  pl.slab_bytes_per_split = (size_t)2 * L.N * pl.kpad * sizeof(int32_t);
+  const int wish = tc_dense_slab_splits(L.N, pl.kpad, (long long)B * L.H * L.Wd, sm_count);
+  const size_t room = ws_bytes > pl.slab_off ? ws_bytes - pl.slab_off : 0;
+  const size_t fit = room / pl.slab_bytes_per_split;
+  pl.max_splits = ws_bytes < pl.slab_off ? -1 : (int)(fit < (size_t)wish ? fit : (size_t)wish);
+  return pl;
+}
+inline bool im2col_route(ff_ctx* ctx, const ff_layer_desc& L, int B) {
+  if (ctx->gemm_path == FF_GEMM_SIMT || !tc_im2col_ok(L)) return false;
+  return im2col_plan(L, B, ctx->workspace_bytes, ctx->sm_count).max_splits >= 1;
+}
+// Writes xi (and wi) for layer L from its Xq (and Wq).
+ff_status launch_im2col(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, const Im2colPlan& pl, bool weights,
+                        cudaStream_t st) {
+  char* ws = static_cast<char*>(ctx->workspace);
+  int8_t* xi = reinterpret_cast<int8_t*>(ws + pl.xi_off);
+  const int rows = 2 * B * L.H * L.Wd;
+  const int blocks = (rows + 255) / 256;
+  switch (pl.kpad) {
+    case 16: im2col3x3_kernel<16><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
+    case 32: im2col3x3_kernel<32><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
+    case 48: im2col3x3_kernel<48><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
+    case 64: im2col3x3_kernel<64><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
+    case 96: im2col3x3_kernel<96><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
+    default: im2col3x3_kernel<128><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
+  }
+  FF_LAUNCH_CHECK(ctx);
+  if (weights) {
+    int8_t* wi = reinterpret_cast<int8_t*>(ws + pl.wi_off);
+    pad_rows_kernel<<<(L.N * pl.kpad + 255) / 256, 256, 0, st>>>(b.Wq, wi, L.N, L.K, pl.kpad);
+    FF_LAUNCH_CHECK(ctx);
+  }
+  return FF_OK;
+}
+
 // Forward contraction + fused epilogue.
 ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
   const int R = rows_per_sample(L);
   const int rows = 2 * B * R;
   bool tc_ok = tc_forward_supported(L, B);
+  if (!tc_ok && im2col_route(ctx, L, B)) {
+    const Im2colPlan pl = im2col_plan(L, B, ctx->workspace_bytes, ctx->sm_count);
+    ProfScope prof(ctx, FF_K_FWD_GEMM, st);
+    const bool was = ctx->profiling;
+    ctx->profiling = false;  // one event pair around the whole route
+    ff_status s = launch_im2col(ctx, L, b, B, pl, true, st);
+    ctx->profiling = was;
+    if (s != FF_OK) return s;
+    const char* ws = static_cast<const char*>(ctx->workspace);
+    s = tc_forward(ctx->tc, L, b, B, status_ptr(ctx), st, reinterpret_cast<const int8_t*>(ws + pl.xi_off),
+                   reinterpret_cast<const int8_t*>(ws + pl.wi_off), pl.kpad);
+    if (s != FF_OK) return fail(ctx, s, "tensor-core forward launch failed: %s", ctx->tc.err);
+    ctx->launches++;
+    return FF_OK;
+  }
   if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core forward");
   if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT) {
     ProfScope prof(ctx, FF_K_FWD_GEMM, st);
@@ -238,6 +303,29 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
   const int R = rows_per_sample(L);
   const int rows = 2 * B * R;
   bool tc_ok = tc_update_supported(L, B);
+  if (!tc_ok && L.N % 16 == 0 && im2col_route(ctx, L, B)) {
+    // explicit im2col (rebuilt from Xq: the workspace is transient), dense split contraction into slabs, reduce + update
+    const Im2colPlan pl = im2col_plan(L, B, ctx->workspace_bytes, ctx->sm_count);
+    ProfScope prof(ctx, FF_K_UPD_GEMM, st);
+    const bool was = ctx->profiling;
+    ctx->profiling = false;
+    ff_status s = launch_im2col(ctx, L, b, B, pl, false, st);
+    if (s == FF_OK) {
+      char* ws = static_cast<char*>(ctx->workspace);
+      int32_t* slabs = reinterpret_cast<int32_t*>(ws + pl.slab_off);
+      int used = 0;
+      s = tc_dense_update_slab(ctx->tc, b.dHq, L.N, reinterpret_cast<const int8_t*>(ws + pl.xi_off), pl.kpad, B * R, slabs,
+                               pl.max_splits, &used, status_ptr(ctx), st);
+      if (s != FF_OK) {
+        ctx->profiling = was;
+        return fail(ctx, s, "tensor-core weight-gradient launch failed: %s", ctx->tc.err);
+      }
+      ctx->launches++;
+      s = launch_slab_update(ctx, slabs, used, L, b, st, pl.kpad);
+    }
+    ctx->profiling = was;
+    return s;
+  }
   if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core weight gradient");
   if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT && L.kind == FF_LINEAR) {
     ProfScope prof(ctx, FF_K_UPD_GEMM, st);
@@ -455,6 +543,11 @@ ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, s
       const int s1 = tc_conv_update_splits(layers[l], B, 0, 1), s2 = tc_conv_update_splits(layers[l], B, 0, 2);
       const size_t tc_need = tc_conv_update_slab_bytes(layers[l], s1 > s2 ? s1 : s2);
       if (tc_need > need) need = tc_need;
+    }
+    if (tc_im2col_ok(layers[l])) {
+      const Im2colPlan pl = im2col_plan(layers[l], B, SIZE_MAX, 0);
+      const size_t im_need = pl.slab_off - WS_BYTES + (size_t)pl.max_splits * pl.slab_bytes_per_split;
+      if (im_need > need) need = im_need;
     }
     if (need > slab) slab = need;
   }

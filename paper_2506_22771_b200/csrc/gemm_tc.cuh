@@ -982,12 +982,26 @@ inline ff_status tc_gemm(TcState& t, const int8_t* A, const int8_t* Bm, int32_t*
   return tc_launch<TC_MODE_RAW, true, 128>(t, ncta, ta, tb, p, st);
 }
 
-inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint32_t* status, cudaStream_t st) {
+// A convolution whose 9*Cin contraction fits one 128-byte block is run through an explicit, zero-padded
+// INT8 im2col matrix (xi [rows, kpad], weights wi [N, kpad]) and the dense kernels.
+inline int tc_im2col_kpad(const ff_layer_desc& L) { return (9 * L.Cin + 15) / 16 * 16; }
+inline bool tc_im2col_ok(const ff_layer_desc& L) {
+  if (L.kind != FF_CONV3X3 || tc_conv_ok(L)) return false;
+  const int kp = tc_im2col_kpad(L);
+  return kp == 16 || kp == 32 || kp == 48 || kp == 64 || kp == 96 || kp == 128;
+}
+
+// xi / wi / kpad: explicit-im2col operands (nullptr / 0: use the layer's Xq and Wq directly).
+inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint32_t* status, cudaStream_t st,
+                            const int8_t* xi = nullptr, const int8_t* wi = nullptr, int kpad = 0) {
   ff_status s = tc_init(t);
   if (s != FF_OK) return s;
-  const bool conv = L.kind == FF_CONV3X3;
-  const int R = conv ? L.H * L.Wd : 1;
+  const bool conv = L.kind == FF_CONV3X3 && !xi;
+  const int R = L.kind == FF_CONV3X3 ? L.H * L.Wd : 1;
   const int M = 2 * B * R;
+  const int K = xi ? kpad : L.K;
+  const int8_t* A = xi ? xi : b.Xq;
+  const int8_t* Bw = xi ? wi : b.Wq;
   CUtensorMap ta, tb;
   TcParams p = {};
   p.out_rows = M;
@@ -1008,9 +1022,9 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   if (p.y_tma && (s = tc_make_store_map(t, &ty, b.Y, L.N, M)) != FF_OK) return s;
   const CUtensorMap* typ = p.y_tma ? &ty : nullptr;
   if (!conv) {
-    p.kblocks = cdiv(L.K, 128);
-    if ((s = tc_make_map(t, &ta, b.Xq, L.K, M, 0, 128, TC_BM)) != FF_OK) return s;
-    if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, 128, TC_BN / ncta)) != FF_OK) return s;
+    p.kblocks = cdiv(K, 128);
+    if ((s = tc_make_map(t, &ta, A, K, M, 0, 128, TC_BM)) != FF_OK) return s;
+    if ((s = tc_make_map(t, &tb, Bw, K, L.N, 0, 128, TC_BN / ncta)) != FF_OK) return s;
     return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st, typ);
   }
   const int ch = L.Cin % 128 == 0 ? 128 : 64;
@@ -1078,6 +1092,36 @@ inline ff_status tc_conv_update(TcState& t, const ff_layer_desc& L, const ff_lay
   if ((s = tc_make_map_nhwc(t, &tb, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_TH)) != FF_OK) return s;
   if (ch == 128) return tc_launch<TC_MODE_SLAB, true, 128>(t, ncta, ta, tb, p, st);
   return tc_launch<TC_MODE_SLAB, true, 64>(t, ncta, ta, tb, p, st);
+}
+
+// Dense split weight gradient into slabs: A = dHq [rows_per_pass x 2, N], B = xi [rows_per_pass x 2, kcols]
+// (kcols % 16 == 0); slabs [splits][2][N][kcols].
+inline int tc_dense_slab_splits(int N, int kcols, long long rows_per_pass, int sm_count) {
+  if (sm_count <= 0) sm_count = 148;
+  const long long tiles = (long long)cdiv(N, TC_BM) * cdiv(kcols, TC_BN);
+  const long long kblocks = (rows_per_pass + 127) / 128;
+  long long splits = sm_count / tiles;
+  if (splits > kblocks / 8) splits = kblocks / 8;
+  return splits < 1 ? 1 : (int)splits;
+}
+inline ff_status tc_dense_update_slab(TcState& t, const int8_t* dHq, int N, const int8_t* xi, int kcols, int rows_per_pass,
+                                      int32_t* slabs, int splits, int* splits_out, uint32_t* status, cudaStream_t st) {
+  ff_status s = tc_init(t);
+  if (s != FF_OK) return s;
+  CUtensorMap ta, tb;
+  TcParams p = {};
+  p.out_rows = N;
+  p.out_cols = kcols;
+  p.kblocks = cdiv(rows_per_pass, 128);
+  p.npass = 2;
+  p.splits = splits;
+  p.status = status;
+  p.slabs = slabs;
+  const int kb_per_split = cdiv(p.kblocks, splits);
+  *splits_out = cdiv(p.kblocks, kb_per_split);
+  if ((s = tc_make_map(t, &ta, dHq, N, rows_per_pass, 2, 128, 128)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &tb, xi, kcols, rows_per_pass, 2, 128, 128)) != FF_OK) return s;
+  return tc_launch<TC_MODE_SLAB, true, 128>(t, 1, ta, tb, p, st);
 }
 
 }  // namespace ffi8
