@@ -41,8 +41,9 @@ constexpr int TC_THREADS = 320;
 constexpr int TC_EPI_WARPS = 8;                           // two per TMEM lane quadrant
 constexpr int TC_EPI_COLS = TC_BN / 2;                    // most accumulator columns one epilogue warp takes
 constexpr int TC_MAX_STAGES = 8;
-constexpr uint32_t TC_PATCH_BYTES = 32 * 32 * 4;          // one 32 x 32 FP32 staging patch per epilogue warp (128-byte swizzle)
-constexpr uint32_t TC_RING_BYTES = 192 * 1024;            // operand ring budget
+constexpr uint32_t TC_PATCH_BYTES = 32 * 32 * 4;          // one 32 x 32 FP32 staging patch (128-byte swizzle)
+constexpr int TC_PATCHES = 2;                             // patches per epilogue warp: a store may still be reading one while the next fills
+constexpr uint32_t TC_RING_BYTES = 160 * 1024;            // operand ring budget
 constexpr int TC_PREFETCH_KB = 8;                         // W tile is prefetched into L2 this many k-blocks before the epilogue
 constexpr int TC_GROUP_M = 16;                            // tile rows per rasterisation group (L2 reuse)
 constexpr uint32_t TC_TMEM_COLS = 512;
@@ -57,7 +58,7 @@ struct TcGeom {
   static constexpr uint32_t B_BYTES = MN_MAJOR ? 128u * (TC_BN / NCTA) : (uint32_t)(TC_BN / NCTA) * CH;
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (int)(TC_RING_BYTES / STAGE_BYTES) < TC_MAX_STAGES ? (int)(TC_RING_BYTES / STAGE_BYTES) : TC_MAX_STAGES;
-  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + TC_EPI_WARPS * TC_PATCH_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + TC_EPI_WARPS * TC_PATCHES * TC_PATCH_BYTES + 1024 /*align*/ + 256 /*barriers*/;
   static constexpr int MMAS = MN_MAJOR ? 4 : CH / 32;            // MMAs (K = 32) per contraction block
   static constexpr int B_BOXES = MN_MAJOR ? (TC_BN / NCTA) / CH : 1;  // TMA boxes of the B operand per stage
   static constexpr uint32_t SWZ = CH == 128 ? 2u : 4u;             // descriptor swizzle code: 128-byte / 64-byte
@@ -264,6 +265,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 
 // Shared-memory matrix descriptor for a swizzled operand tile whose rows are CH = 128 (swz = 2) or
 // 64 (swz = 4) bytes long; 8 rows form one swizzle atom.  K-major: rows are M/N indices, SBO = 8 rows
@@ -310,7 +312,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   const uint32_t ring = (raw + 1023u) & ~1023u;
   uint8_t* ring_ptr = smem_raw + (ring - raw);
   uint8_t* patch_all = ring_ptr + STAGES * STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(patch_all + TC_EPI_WARPS * TC_PATCH_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(patch_all + TC_EPI_WARPS * TC_PATCHES * TC_PATCH_BYTES);
   const uint32_t bar_full = smem_u32(bars);                      // [STAGES]  used in the leader CTA
   const uint32_t bar_empty = bar_full + 8 * TC_MAX_STAGES;       // [STAGES]  one set per CTA
   const uint32_t bar_tfull = bar_empty + 8 * TC_MAX_STAGES;      // [2]       one set per CTA
@@ -522,9 +524,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     // ------------------------------- epilogue (warps 2..9 of every CTA) -----------------------
     const int quad = warp & 3;                           // TMEM lane quadrant this warp may read
     const int half = (warp - 2) >> 2;                    // which of the quadrant's two warps
-    uint8_t* patch = patch_all + (warp - 2) * TC_PATCH_BYTES;
-    const uint32_t patch_u32 = smem_u32(patch);
-    (void)patch_u32;
+    uint8_t* patch0 = patch_all + (warp - 2) * TC_PATCHES * TC_PATCH_BYTES;
+    uint32_t pflip = 0;  // which of the warp's two patches the next chunk fills (forward epilogue)
+    (void)pflip;
     uint32_t tile_it = 0;
     bool ok = true;
     float c0 = 0.f, c1 = 0.f, cP = 0.f, cN = 0.f;
@@ -591,8 +593,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           if (i + 1 < TC_EPI_COLS / 32 && cb + 32 < cend) tc_ld32_async(t_row + as * TC_BN + cb + 32, v[(i + 1) & 1]);
           if (cb < cend) {  // uniform across the warp
             const int(&a)[32] = v[i & 1];
-            if (p.y_tma) {  // the previous store of this warp must have read the patch
-              if (lane == 0) bulk_wait_read0();
+            uint8_t* patch = patch0 + pflip * TC_PATCH_BYTES;
+            pflip ^= 1u;
+            if (p.y_tma) {  // the store issued two chunks ago must have read this patch
+              if (lane == 0) bulk_wait_read1();
               __syncwarp();
             }
 #pragma unroll
@@ -612,7 +616,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
               __syncwarp();
               if (lane == 0 && wrow0 < p.out_rows) {  // a box that starts inside the output; its overhang is clipped
-                tma_store_2d(&tmY, patch_u32, col0 + cb, wrow0);
+                tma_store_2d(&tmY, smem_u32(patch), col0 + cb, wrow0);
                 bulk_commit();
               }
             } else {
@@ -683,6 +687,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         // thread = one accumulator row computes d = lr*(float(accP)*cP + float(accN)*cN); d is staged
         // through smem so that the read-modify-write of W is row-contiguous
         const size_t plane = (size_t)p.out_rows * p.out_cols;
+        uint8_t* patch = patch0;
 #pragma unroll 1
         for (int cb = cbeg; cb < cend; cb += 32) {
           const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
