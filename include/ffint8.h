@@ -119,7 +119,7 @@ ff_status ff_set_gemm_path(ff_ctx* ctx, int path);
 
 /* The tensor-core kernels run either one CTA per 128 x 256 output tile or a pair of CTAs (tcgen05
  * cta_group::2) per 256 x 256 tile.  ctas_per_tile = 0 chooses by problem size (pairs once the
- * output has enough tiles to occupy every SM pair), 1 / 2 force one form.  Identical bits. */
+ * output has more than 128 rows), 1 / 2 force one form.  Identical bits. */
 ff_status ff_set_tensor_form(ff_ctx* ctx, int ctas_per_tile);
 
 /* Forward of one layer (Sec. IV-B: quantise A and W, INT8 MAC with INT32 accumulation; Sec. III /
@@ -167,8 +167,7 @@ uint64_t ff_launch_count(const ff_ctx* ctx);
  * device time in milliseconds and the number of launches (host arrays of FF_K_COUNT entries). */
 enum {
   FF_K_ABSMAX = 0,   /* per-tensor max|x| (Sec. IV, SUQ range)                                   */
-  FF_K_QUANTIZE,     /* SUQ of A or W to INT8                                                    */
-  FF_K_ZERO_STATS,   /* clears S and rowmax                                                      */
+  FF_K_QUANTIZE,     /* SUQ of A or W to INT8 (the W call also clears S and rowmax)              */
   FF_K_FWD_GEMM,     /* forward INT8 MAC + dequantise/ReLU/goodness epilogue                     */
   FF_K_FINALIZE,     /* G from S, range of the normalised output                                 */
   FF_K_NORMALIZE,    /* length normalisation (+ next layer's SUQ)                                */
@@ -197,7 +196,7 @@ ff_status ff_int8_gemm(ff_ctx* ctx, const int8_t* A, const int8_t* B, int32_t* C
  * another framework's stream callback or memory-pool critical section, a process whose memory was
  * handed out in full at start-up, a caller that holds no ff_ctx and no workspace.  Everything else
  * in this library keeps its partial sums in the workspace the caller allocates; here they live in a
- * small array (about 4 KiB) built into the library image, which every GPU that loads the library
+ * small array (about 16 KiB) built into the library image, which every GPU that loads the library
  * keeps until the process ends.  The call allocates nothing: no cudaMalloc, no cudaFree, no
  * workspace, no context.
  *

@@ -23,7 +23,7 @@ EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", 
            "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
            "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static"]
 FF_STATIC_LOSS_MAX_SAMPLES = 65536
-FF_K_NAMES = ["absmax", "quantize", "zero_stats", "fwd_gemm", "finalize", "normalize", "loss", "dh_quantize",
+FF_K_NAMES = ["absmax", "quantize", "fwd_gemm", "finalize", "normalize", "loss", "dh_quantize",
               "upd_gemm", "raw_gemm"]
 
 

@@ -62,10 +62,18 @@ __global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restr
 // Linear element index (over the whole tensor) keys the stochastic rounding.
 // grid = (blocks, passes)
 // ---------------------------------------------------------------------------------------------
+// zero_S / zero_rowmax (nullable, zero_n entries): per-sample accumulators of the forward epilogue that
+// the weight quantiser clears on the side, sparing a launch.
 template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __restrict__ x, int8_t* __restrict__ q,
                                                               size_t n_per_pass, const float* __restrict__ a,
-                                                              RoundKey key) {
+                                                              RoundKey key, unsigned long long* __restrict__ zero_S = nullptr,
+                                                              int32_t* __restrict__ zero_rowmax = nullptr, int zero_n = 0) {
+  if (zero_S && blockIdx.y == 0)
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < zero_n; i += gridDim.x * blockDim.x) {
+      zero_S[i] = 0ull;
+      zero_rowmax[i] = 0;
+    }
   const size_t base = (size_t)blockIdx.y * n_per_pass;
   const float* xp = x + base;
   int8_t* qp = q + base;
@@ -219,6 +227,13 @@ __device__ __forceinline__ double sigmoid_spec(double x) {
   return x >= 0.0 ? __ddiv_rn(1.0, d) : __ddiv_rn(e, d);
 }
 
+// log(1 + e^z) for the reported loss value only (it feeds no state and is compared at 1e-5): the
+// correction term in FP32, which keeps the long FP64 library chains out of the kernel's critical path.
+__device__ __forceinline__ double softplus_value(double z) {
+  const float az = fabsf((float)z);
+  return fmax(z, 0.0) + (double)log1pf(expf(-az));
+}
+
 constexpr int FF_MAX_LATER = 31;
 struct LaterLayers {
   const float* G[FF_MAX_LATER];
@@ -234,8 +249,8 @@ struct LaterLayers {
 // finishes last (ticket counter) combines them in block order, so the loss is reproducible and
 // nothing has to be zeroed beforehand.  scratch: LossScratch, ticket zero on entry and on exit.
 // ---------------------------------------------------------------------------------------------
-constexpr int LOSS_THREADS = 256;
-constexpr int LOSS_MAX_BLOCKS = 256;
+constexpr int LOSS_THREADS = 64;      // small blocks: the FP64 work of a few thousand samples spreads over many SMs
+constexpr int LOSS_MAX_BLOCKS = 1024;
 struct LossScratch {
   unsigned int ticket;
   unsigned int pad[3];
@@ -261,12 +276,12 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
     const double sign = p ? 1.0 : -1.0;
     double arg = __dmul_rn(sign, __dsub_rn((double)G[m], (double)theta));
     double g0 = __dmul_rn(sign, sigmoid_spec(arg));
-    double L0 = fmax(arg, 0.0) + log1p(exp(-fabs(arg)));
+    double L0 = softplus_value(arg);
     double gsum = 0.0, Lsum = 0.0;
     for (int j = 0; j < later.n; ++j) {
       double aj = __dmul_rn(sign, __dsub_rn((double)later.G[j][m], (double)later.theta[j]));
       gsum = __dadd_rn(gsum, __dmul_rn(sign, sigmoid_spec(aj)));
-      Lsum += fmax(aj, 0.0) + log1p(exp(-fabs(aj)));
+      Lsum += softplus_value(aj);
     }
     float cf = __double2float_rn(__dmul_rn(__dadd_rn(g0, __dmul_rn(lam, gsum)), inv_m));
     coef[m] = cf;
@@ -353,15 +368,6 @@ __global__ void __launch_bounds__(EW_THREADS) dh_quantize_kernel(const float* __
       float k2 = __fmul_rn(2.0f, coef[(uint32_t)e / (uint32_t)per_sample]);
       dHq[e] = (int8_t)quant_one<MODE>(__fmul_rn(k2, Y[e]), inv, (uint32_t)e, key);
     }
-  }
-}
-
-// Zero the per-sample integer accumulators of the forward epilogue (S: u64 sum, rowmax: i32 max).
-__global__ void __launch_bounds__(EW_THREADS) zero_sample_stats_kernel(unsigned long long* S, int32_t* rowmax, int M) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < M) {
-    S[i] = 0ull;
-    rowmax[i] = 0;
   }
 }
 

@@ -396,17 +396,11 @@ ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     ProfScope prof(ctx, FF_K_QUANTIZE, st);
     const dim3 grid(ew_blocks(ctx, nW / 4 + 1), 1);
     const RoundKey key = make_round_key(L.seed, ROLE_W, L.index, step);
+    unsigned long long* S = reinterpret_cast<unsigned long long*>(b.S);  // cleared on the side for the forward epilogue
     if (L.round_w == FF_ROUND_NEAREST_EVEN)
-      quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, key);
+      quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, key, S, b.rowmax, 2 * B);
     else
-      quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, key);
-  }
-  FF_LAUNCH_CHECK(ctx);
-  const int M = 2 * B;
-  {
-    ProfScope prof(ctx, FF_K_ZERO_STATS, st);
-    zero_sample_stats_kernel<<<(M + EW_THREADS - 1) / EW_THREADS, EW_THREADS, 0, st>>>(
-        reinterpret_cast<unsigned long long*>(b.S), b.rowmax, M);
+      quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, key, S, b.rowmax, 2 * B);
   }
   FF_LAUNCH_CHECK(ctx);
   ff_status s = run_forward_gemm(ctx, L, b, B, st);

@@ -844,12 +844,14 @@ inline ff_status tc_make_map_nhwc(TcState& t, CUtensorMap* tm, const int8_t* bas
 
 inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
 
-// CTA-group size for an output of out_rows x out_cols: pairs once there are at least two 128-row
-// blocks and enough 256 x 256 tiles to occupy every SM pair; single CTAs for small problems.
+// CTA-group size for an output of out_rows x out_cols: a pair whenever the output has at least two
+// 128-row blocks (the pair halves the B-operand traffic per MMA; measured at least as fast as single
+// CTAs from one wave of tiles upwards), single CTAs for outputs of at most 128 rows.
 inline int tc_pick_ncta(const TcState& t, long long out_rows, long long out_cols, long long splits = 1) {
+  (void)out_cols;
+  (void)splits;
   if (t.force_ncta == 1 || t.force_ncta == 2) return t.force_ncta;
-  const long long pair_items = (long long)cdiv(out_rows, 2 * TC_BM) * cdiv(out_cols, TC_BN) * splits;
-  return (out_rows > TC_BM && pair_items >= t.sm_count / 2) ? 2 : 1;
+  return out_rows > TC_BM ? 2 : 1;
 }
 
 // FP32 row-major matrix [rows, cols] for the forward epilogue's TMA stores: boxes of 32 x 32, 128-byte swizzle.
