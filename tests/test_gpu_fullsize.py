@@ -1,0 +1,86 @@
+"""Full-size parity: the CUDA path at the task's full configuration sizes, in the launch configuration
+bench.py times (no parity dumps, no FP32 copy of the normalised output, layers chained on device),
+against SHA-256 digests of the CPU oracle's tensors (tests/golden/fullsize_digests.json, written by
+tests/golden/make_fullsize_digests.py from oracle/ alone).  Every INT8 tensor, accumulator statistic
+and FP32 tensor is compared bit for bit through its digest; the loss scalar at 1e-5 relative."""
+import ctypes as C
+import hashlib
+import json
+import os
+
+import numpy as np
+import pytest
+
+from paper_2506_22771_b200 import binding as ffb
+from paper_2506_22771_b200 import synth
+from tests.ffharness import GpuNet, REL_TOL
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "fullsize_digests.json")
+DIG = json.load(open(GOLDEN)) if os.path.exists(GOLDEN) else {}
+TENSORS = ["Xq", "Wq", "Y", "S", "rowmax", "G", "coef", "dHq"]
+
+
+def _sha(t):
+    return hashlib.sha256(t.detach().cpu().contiguous().numpy().tobytes()).hexdigest()
+
+
+def _check_layer(b, want, tag):
+    am = b.absmax.detach().cpu().numpy()
+    got_am = [float(np.float32(v)).hex() for v in am[:5]]
+    assert got_am == want["absmax"], (tag, "absmax", got_am, want["absmax"])
+    for name in TENSORS:
+        assert _sha(getattr(b, name)) == want[name], (tag, name, "digest differs from the oracle's")
+    assert _sha(b.W) == want["W_new"], (tag, "W_new", "digest differs from the oracle's")
+    got = float(b.loss[0])
+    assert abs(got - want["loss"]) <= REL_TOL * max(abs(want["loss"]), 1e-30), (tag, "loss", got, want["loss"])
+
+
+def _descs(w, seed):
+    return [ffb.make_desc(l, i, seed) for i, l in enumerate(w.layers)]
+
+
+@pytest.mark.parametrize("name", ["tiny_mlp", "mlp_lookahead", "cnn", "roofline"])
+def test_fullsize_train_steps_match_oracle_digests(name):
+    if name not in DIG:
+        pytest.skip("no digests for this workload in tests/golden/fullsize_digests.json")
+    d = DIG[name]
+    w = synth.workload(name)
+    assert d["B"] == w.B and not d["greedy"]
+    net = GpuNet(_descs(w, d["seed"]), w.B, synth.make_weights(w, d["seed"]), dumps=False, xnext=False, chain=True)
+    net.set_input(synth.make_batch(w, d["seed"]))
+    for step, layers in enumerate(d["steps"]):
+        net.train_step(w.lam_per_step * step, step)
+        for l, want in enumerate(layers):
+            _check_layer(net.bufs[l], want, f"{name}/step{step}/layer{l}")
+    net.close()
+
+
+def test_fullsize_greedy_phases_match_oracle_digests():
+    name = "mlp_greedy"
+    if name not in DIG:
+        pytest.skip("no digests for this workload in tests/golden/fullsize_digests.json")
+    import torch
+    d = DIG[name]
+    w = synth.workload(name)
+    assert d["B"] == w.B and d["greedy"]
+    descs = _descs(w, d["seed"])
+    W0 = synth.make_weights(w, d["seed"])
+    X = synth.make_batch(w, d["seed"])
+    for l, phase in enumerate(d["steps"]):
+        # layer l trained alone on the INT8 forward of the frozen earlier layers, from the initial weights
+        net = GpuNet(descs[:l + 1], w.B, W0[:l + 1], dumps=False, xnext=True, chain=False)
+        one_d = (ffb.ff_layer_desc * 1)(descs[l])
+        one_b = (ffb.ff_layer_bufs * 1)(net.bufs[l].struct)
+        for step, want in enumerate(phase):
+            net.set_input(X)
+            for j in range(l):
+                ffb.ff_layer_forward(net.ctx.ctx, descs[j], net.bufs[j].struct, w.B, step, 0)
+                net.bufs[j + 1].X.copy_(net.bufs[j].Xnext)
+            ffb.ff_train_step(net.ctx.ctx, one_d, one_b, 1, w.B, 0.0, step, 0)
+            ffb.ff_poll_status(net.ctx.ctx, 0)
+            _check_layer(net.bufs[l], want, f"{name}/layer{l}/step{step}")
+        net.close()
+        del net
+        torch.cuda.empty_cache()
