@@ -36,6 +36,28 @@ UNIT = "samples/s"
 INT8_TO_BF16 = 2.0          # nominal dense tensor ratio (4.5 : 2.25 PFLOP/s)
 BURST_SECONDS = 2.0         # timed regions shorter than this are compared with the burst GEMM peak
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one ncu capture of the
+# roofline workload at its full size (profiles/tc_gemm_kernel_roofline_layer.md).  They are reported
+# only while the kernel source is the one that was profiled (hash below) and the workload matches.
+NCU_TRAFFIC = {
+    "source": "paper_2506_22771_b200/csrc/gemm_tc.cuh",
+    "sha256": "304b8c4a1a2868774875060fedebe886acbc33c888b18769f7aad80bc97d1df3",
+    "workload": "roofline", "B": 16384,
+    "bytes_per_launch": {"fwd_gemm": 2428.4e6, "upd_gemm": 3086.2e6},
+}
+
+
+def _ncu_traffic(kind: str, workload: str, B: int):
+    import hashlib
+    t = NCU_TRAFFIC
+    try:
+        sha = hashlib.sha256(open(os.path.join(ROOT, t["source"]), "rb").read()).hexdigest()
+    except OSError:
+        return None
+    if sha != t["sha256"] or workload != t["workload"] or B != t["B"]:
+        return None
+    return t["bytes_per_launch"].get(kind)
+
 
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -324,7 +346,7 @@ def main():
                                         f"{ms * 1e-3:.2f} s",
                          "frac_of_sustained_x2": per_kernel[dom]["achieved"] / (INT8_TO_BF16 * peaks["bf16_sustained"]),
                          "frac_of_nominal_4500": per_kernel[dom]["achieved"] / 4500.0,
-                         "traffic": None},
+                         "traffic": _ncu_traffic(dom, args.workload, B)},
             "kernels": per_kernel,
         }
         if not args.no_cpu_baseline and world == 1:
