@@ -64,19 +64,29 @@ __device__ __forceinline__ uint32_t pair_hash(uint32_t pair, RoundKey key) {
   return h;
 }
 // u in [0,1) with 16 random bits: low half of the pair hash for even indices, high half for odd.
-// u = half16 * 2^-16, formed without an integer-to-float conversion: the float 1.m with the 16 bits
-// at the top of the mantissa is 1 + half16*2^-16, and subtracting 1 is exact.
-__device__ __forceinline__ float u_from_half(uint32_t half16) {
-  return __fsub_rn(__uint_as_float(0x3F800000u | (half16 << 7)), 1.0f);
+// u = half16 * 2^-16, formed without shifts or an integer-to-float conversion: floats in [128, 256)
+// have an ulp of 2^-16, so the bit pattern 0x4300hhhh is 128 + half16*2^-16 and subtracting 128 is
+// exact.  One byte permute places the half (HI = 0: bytes 0-1 of h, HI = 1: bytes 2-3).
+template <int HI>
+__device__ __forceinline__ float u_from_hash(uint32_t h) {
+  const uint32_t bits = __byte_perm(h, 0x43000000u, HI ? 0x7632 : 0x7610);
+  return __fsub_rn(__uint_as_float(bits), 128.0f);
 }
 
-// rint(t) (ties to even) or floor(t+u), then clip to [-127, 127].  The float-to-int conversion does
-// the rounding (|t| stays far inside the int range: |x| <= a gives |t| <= 127 up to one rounding).
-// MODE is a compile-time constant so that only one conversion is issued per element.
+// rint(t) (ties to even) or floor(t+u), then clip to [-127, 127], as one saturating float-to-int8
+// conversion.  |x| <= a gives |t| <= 127 up to one rounding, so: nearest never reaches -128; for
+// floor, clamping t at -127 first gives the same result as clipping afterwards (u >= 0), and the
+// conversion's saturation at +127 is the upper clip.  MODE is a compile-time constant.
 template <int MODE>
 __device__ __forceinline__ int round_clip(float t, float u) {
-  const int r = (MODE == ROUND_NEAREST) ? __float2int_rn(t) : __float2int_rd(__fadd_rn(t, u));
-  return min(max(r, -127), 127);
+  int r;
+  if (MODE == ROUND_NEAREST) {
+    asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(r) : "f"(t));
+  } else {
+    const float v = __fadd_rn(fmaxf(t, -127.0f), u);
+    asm("cvt.rmi.sat.s8.f32 %0, %1;" : "=r"(r) : "f"(v));
+  }
+  return r;
 }
 
 // Quantise two neighbouring elements (even linear index idx_even and idx_even+1).
@@ -85,8 +95,8 @@ __device__ __forceinline__ void quant_pair(float x0, float x1, float inv, uint32
   float u0 = 0.0f, u1 = 0.0f;
   if (MODE != ROUND_NEAREST) {
     const uint32_t h = pair_hash(idx_even >> 1, key);
-    u0 = u_from_half(h & 0xFFFFu);
-    u1 = u_from_half(h >> 16);
+    u0 = u_from_hash<0>(h);
+    u1 = u_from_hash<1>(h);
   }
   q0 = round_clip<MODE>(__fmul_rn(x0, inv), u0);
   q1 = round_clip<MODE>(__fmul_rn(x1, inv), u1);
@@ -97,7 +107,7 @@ __device__ __forceinline__ int quant_one(float x, float inv, uint32_t idx, Round
   float u = 0.0f;
   if (MODE != ROUND_NEAREST) {
     const uint32_t h = pair_hash(idx >> 1, key);
-    u = u_from_half((idx & 1u) ? (h >> 16) : (h & 0xFFFFu));
+    u = (idx & 1u) ? u_from_hash<1>(h) : u_from_hash<0>(h);
   }
   return round_clip<MODE>(__fmul_rn(x, inv), u);
 }
