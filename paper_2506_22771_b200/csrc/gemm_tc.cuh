@@ -45,7 +45,11 @@ constexpr uint32_t TC_PATCH_BYTES = 32 * 32 * 4;          // one 32 x 32 FP32 st
 constexpr int TC_PATCHES = 2;                             // patches per epilogue warp: a store may still be reading one while the next fills
 constexpr uint32_t TC_RING_BYTES = 160 * 1024;            // operand ring budget
 constexpr int TC_PREFETCH_KB = 8;                         // W tile is prefetched into L2 this many k-blocks before the epilogue
-constexpr int TC_GROUP_M = 16;                            // tile rows per rasterisation group (L2 reuse)
+// Tile rows per rasterisation group.  K-major forward: the group's A row panels stay in L2 while the B
+// column panels stream past once per group, so a tall group pays.  MN-major weight gradient: the
+// contraction is so long that panels are only shared by tiles running at the same time; a group of
+// 8 makes a wave of 74 CTA pairs nearly square (8 x 9 panels instead of 16 x 5).
+constexpr int TC_GROUP_M_KMAJOR = 16, TC_GROUP_M_MNMAJOR = 8;
 constexpr uint32_t TC_TMEM_COLS = 512;
 constexpr unsigned long long TC_WAIT_NS = 2000000000ull;  // 2 s bound on every wait
 
@@ -69,6 +73,7 @@ enum { TC_MODE_RAW = 0, TC_MODE_FWD = 1, TC_MODE_UPD = 2, TC_MODE_SLAB = 3 };
 struct TcParams {
   int out_rows, out_cols;   // extent of the output matrix
   int tiles_m, tiles_n;
+  int group_m;              // tile rows per rasterisation group
   int kblocks;              // contraction blocks per pass
   int npass;                // 1, or 2 for the weight gradient (positive / negative set)
   int splits, kb_per_split; // the contraction blocks of a pass are divided over `splits` work items
@@ -167,15 +172,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // Tiled TMA loads into this CTA's shared memory.  NCTA = 2: `bar` is a shared::cluster address and may
 // name a barrier of the other CTA of the pair (the cta_group::2 form allows that); no multicast.
 template <int NCTA>
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y) {
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y, uint64_t policy) {
   if (NCTA == 1)
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y)
-                 : "memory");
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "l"(policy)
+        : "memory");
   else
-    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y)
-                 : "memory");
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(x), "r"(y), "l"(policy)
+        : "memory");
 }
 template <int NCTA>
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y, int z) {
@@ -258,10 +265,23 @@ __device__ __forceinline__ void tc_ld32_async(uint32_t taddr, int (&r)[32]) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // TMA store of one staged box to global memory (clipped at the tensor's edge), bulk async-group completion.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(reinterpret_cast<uint64_t>(tm)),
-               "r"(src), "r"(x), "r"(y)
+// `policy`: an L2 eviction policy (l2_policy_evict_first: the stored lines are the first to leave L2, so a
+// stream of output written once does not push the operand panels out).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y, uint64_t policy) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;" ::"l"(
+                   reinterpret_cast<uint64_t>(tm)),
+               "r"(src), "r"(x), "r"(y), "l"(policy)
                : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
@@ -288,11 +308,11 @@ __host__ __device__ constexpr uint32_t make_idesc_i8(bool a_mn_major, bool b_mn_
 
 // Tile order: groups of TC_GROUP_M tile rows, column by column inside a group, so that the CTAs
 // running at one time share a small set of operand row / column panels in L2.
-__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
-  const int per_group = TC_GROUP_M * tiles_n;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int group_m, int& tm, int& tn) {
+  const int per_group = group_m * tiles_n;
   const int g = tile / per_group, r = tile - g * per_group;
-  const int rows = min(TC_GROUP_M, tiles_m - g * TC_GROUP_M);
-  tm = g * TC_GROUP_M + r % rows;
+  const int rows = min(group_m, tiles_m - g * group_m);
+  tm = g * group_m + r % rows;
   tn = r / rows;
 }
 
@@ -372,13 +392,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       bool ok = true;
       const int a_rows0 = (int)rank * TC_BM;            // this CTA's rows inside the group's tile
       const int b_cols0 = (int)rank * (TC_BN / NCTA);   // this CTA's share of the tile's columns
+      // L2 policies of the K-major loads.  Dense forward: the group's row panels of A are reused by every
+      // tile column of the rasterisation group (keep), a column panel of B only by the tiles in flight
+      // (stream).  Convolution: the small weight matrix is reused by every tile (keep).
+      const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
       const int hw = p.conv_H * p.conv_W;
       const int blocks_per_img = p.conv_W ? p.conv_H / p.conv_TH : 1;
       for (int item = group; item < total_items && ok; item += n_groups) {
         const int tile = item / p.splits, split = item - tile * p.splits;
         const int kb0 = split * p.kb_per_split, kb1 = min(p.kblocks, kb0 + p.kb_per_split);
         int tm, tn;
-        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+        tile_coords(tile, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
         const int row0 = tm * (TC_BM * NCTA) + a_rows0, col0 = tn * TC_BN + b_cols0;
         // forward convolution: image and first image row of this CTA's 128 output positions
         const int f_img = (!MN_MAJOR && p.conv_W) ? row0 / hw : 0;
@@ -445,9 +469,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
                   }
                 }
               } else {
-                tma_load_2d<NCTA>(a_dst, &tmA, fb, kb * CH, row0);
+                tma_load_2d<NCTA>(a_dst, &tmA, fb, kb * CH, row0, pol_keep);
               }
-              tma_load_2d<NCTA>(b_dst, &tmB, fb, kb * CH, col0);
+              tma_load_2d<NCTA>(b_dst, &tmB, fb, kb * CH, col0, p.conv_W ? pol_keep : pol_stream);
             } else {
               // boxes of 128 contraction rows x 128 (A) or CH (B) output indices
               tma_load_3d<NCTA>(a_dst, &tmA, fb, row0, kb * 128, pass);
@@ -527,6 +551,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     uint8_t* patch0 = patch_all + (warp - 2) * TC_PATCHES * TC_PATCH_BYTES;
     uint32_t pflip = 0;  // which of the warp's two patches the next chunk fills (forward epilogue)
     (void)pflip;
+    const uint64_t y_policy = l2_policy_evict_first();
+    (void)y_policy;
     uint32_t tile_it = 0;
     bool ok = true;
     float c0 = 0.f, c1 = 0.f, cP = 0.f, cN = 0.f;
@@ -543,7 +569,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       const int tile = item / p.splits, split = item - tile * p.splits;
       (void)split;
       int tm, tn;
-      tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      tile_coords(tile, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
       const uint32_t as = tile_it % ACC_STAGES, aph = (tile_it / ACC_STAGES) & 1u;
       if (!mbar_wait<PAIR>(bar_tfull + 8 * as, aph, abort_flag)) {
         ok = false;
@@ -616,7 +642,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
               __syncwarp();
               if (lane == 0 && wrow0 < p.out_rows) {  // a box that starts inside the output; its overhang is clipped
-                tma_store_2d(&tmY, smem_u32(patch), col0 + cb, wrow0);
+                tma_store_2d(&tmY, smem_u32(patch), col0 + cb, wrow0, y_policy);
                 bulk_commit();
               }
             } else {
@@ -882,6 +908,7 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
   }
   p.tiles_m = cdiv(p.out_rows, TC_BM * NCTA);
   p.tiles_n = cdiv(p.out_cols, TC_BN);
+  p.group_m = MN_MAJOR ? TC_GROUP_M_MNMAJOR : TC_GROUP_M_KMAJOR;
   if (p.splits < 1) p.splits = 1;
   p.kb_per_split = cdiv(p.kblocks, p.splits);
   p.splits = cdiv(p.kblocks, p.kb_per_split);  // no empty split
@@ -1026,6 +1053,7 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   const int ncta = tc_pick_ncta(t, M, L.N);
   CUtensorMap ty;
   p.y_tma = (L.N % 4 == 0) ? 1 : 0;
+
   if (p.y_tma && (s = tc_make_store_map(t, &ty, b.Y, L.N, M)) != FF_OK) return s;
   const CUtensorMap* typ = p.y_tma ? &ty : nullptr;
   if (!conv) {
