@@ -199,6 +199,64 @@ def run_reference(args):
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+def run_predict(args, w, world, rank, local, dev):
+    """Classification by goodness: every sample is forwarded once per candidate label (10 labels); the
+    candidate batch has about as many rows as the workload's training batch."""
+    import torch
+    import torch.distributed as dist
+    from paper_2506_22771_b200 import binding as ffb
+    n_classes = 10
+    Bp = args.B or (2 * w.B) // n_classes
+    half = n_classes * Bp // 2
+    seed = 1 + rank
+    descs = [ffb.make_desc(l, i, seed) for i, l in enumerate(w.layers)]
+    ctx = ffb.Context(descs, half, local)
+    bufs = [ffb.LayerBuffers(d, half, dev, dumps=False, xnext=False, own_x=(i == 0)) for i, d in enumerate(descs)]
+    for b, W in zip(bufs, synth.make_weights(w, seed)):
+        b.W.copy_(torch.from_numpy(W))
+    Xc, _ = synth.make_candidates(w, seed, Bp, n_classes)
+    bufs[0].X.copy_(torch.from_numpy(Xc).reshape(bufs[0].X.shape))
+    descs_arr = (ffb.ff_layer_desc * len(descs))(*descs)
+    bufs_arr = (ffb.ff_layer_bufs * len(descs))(*[b.struct for b in bufs])
+    scores = torch.zeros(n_classes * Bp, dtype=torch.float32, device=dev)
+    pred = torch.zeros(Bp, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def step(i):
+        ffb.ff_predict(ctx.ctx, descs_arr, bufs_arr, len(descs), Bp, n_classes, 0, scores.data_ptr(), pred.data_ptr(), i, stream)
+
+    for i in range(args.warmup):
+        step(i)
+    ffb.ff_poll_status(ctx.ctx, stream)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ffb.ff_profile_start(ctx.ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    kernel_ms = ffb.ff_profile_stop(ctx.ctx, stream)
+    ffb.ff_poll_status(ctx.ctx, stream)
+    ms, value = whole_job_throughput(e0.elapsed_time(e1), Bp * args.steps, dev)
+    if rank == 0:
+        print(json.dumps({
+            "metric": "FF-INT8 classified samples/s (10 candidate labels per sample)", "value": value, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": args.workload, "mode": "predict", "samples": Bp, "candidate_rows": n_classes * Bp,
+                       "layers": [[x.K, x.N] for x in w.layers]},
+            "kernels": {k: {"ms_per_step": t / args.steps, "launches_per_step": n / args.steps}
+                        for k, (t, n) in kernel_ms.items()}}))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -211,6 +269,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--B", type=int, default=0, help="override positives per batch (profiling runs on a smaller case)")
     ap.add_argument("--tensor-form", type=int, default=0, help="CTAs per tensor-core tile: 0 auto, 1, 2")
+    ap.add_argument("--predict", action="store_true",
+                    help="time classification by goodness (ff_predict, 10 candidate labels) instead of the train step")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -231,6 +291,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     w = synth.workload(args.workload)
+    if args.predict:
+        return run_predict(args, w, world, rank, local, dev)
     B = args.B or w.B
     seed = 1 + rank
     descs = [ffb.make_desc(l, i, seed) for i, l in enumerate(w.layers)]

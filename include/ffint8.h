@@ -151,6 +151,23 @@ ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_laye
 ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs,
                         int n_layers, int B, float lambda, uint64_t step, void* cuda_stream);
 
+/* Classification of B samples by goodness with the current weights.  The paper reports accuracy but
+ * does not describe the procedure; this is the Forward-Forward one its Sec. III builds on ("make
+ * each layer excited about positive samples"): every sample is presented once per candidate label,
+ * label written one-hot into the input exactly as for the positive set; each candidate runs through
+ * the same INT8 forward as training (Sec. IV-B; Alg. 1 line 5-6); the goodness of the layers
+ * first_counted_layer .. n_layers-1 is added per candidate (FP32, in layer order) and the label with
+ * the largest total wins (lowest label on ties).
+ * Layout: the caller builds the candidate batch [n_classes*B, ...] in bufs[0].X, row c*B + b = sample
+ * b with candidate label c, already length-normalised.  It is quantised like a training batch, with
+ * one range for the first and one for the second half of its rows, so n_classes must be even and
+ * every buffer of `bufs` must be sized for n_classes*B rows (i.e. as for a batch of n_classes*B/2
+ * positives + negatives).  Writes scores [n_classes*B] (row c*B + b) and pred [B] (device, 16-byte
+ * aligned) and, as a side effect, the forward outputs of every layer.  No weights change. */
+ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
+                     int n_classes, int first_counted_layer, float* scores, int32_t* pred, uint64_t step,
+                     void* cuda_stream);
+
 /* Synchronises `cuda_stream`, reads the device status word and clears it.  Returns FF_OK,
  * FF_ERR_NONFINITE, FF_ERR_DEVICE_TIMEOUT or FF_ERR_CUDA. */
 ff_status ff_poll_status(ff_ctx* ctx, void* cuda_stream);
@@ -175,6 +192,7 @@ enum {
   FF_K_DH_QUANTIZE,  /* g^Y to INT8                                                              */
   FF_K_UPD_GEMM,     /* g^W INT8 MAC + SGD update epilogue                                       */
   FF_K_RAW_GEMM,     /* ff_int8_gemm                                                             */
+  FF_K_CLASSIFY,     /* ff_predict: per-candidate goodness totals and their argmax               */
   FF_K_COUNT
 };
 ff_status ff_profile_start(ff_ctx* ctx);

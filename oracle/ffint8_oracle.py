@@ -438,6 +438,37 @@ def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: i
 
 
 # --------------------------------------------------------------------------------------
+# Classification with a trained network  (Sec. III: goodness is high for positive data)
+# --------------------------------------------------------------------------------------
+def predict(specs: List[LayerSpec], Ws: List[np.ndarray], X_cand: np.ndarray, B: int, n_classes: int,
+            step: int, first_counted: int = 0):
+    """Label of each of B samples by goodness.  The paper reports accuracy but does not spell the
+    procedure out; this is the Forward-Forward one its Sec. III builds on: a sample is presented
+    once per candidate label (label written one-hot into the input, exactly as for the positive
+    set), every candidate runs through the INT8 forward of all layers, the goodness of the layers
+    from `first_counted` on is added up, and the label with the largest total wins (lowest label
+    on ties).  X_cand [n_classes*B, ...]: row c*B + b is sample b with candidate label c, already
+    length-normalised.  The candidate batch is quantised like a training batch: per-tensor ranges
+    for its first and second half of the rows (labels 0..n/2-1 | n/2..n-1), so n_classes is even.
+    Returns (pred [B] int32, scores [n_classes, B] float32, per-layer LayerStates)."""
+    if n_classes % 2 or n_classes <= 0:
+        raise ValueError("n_classes must be even and positive")
+    half = n_classes * B // 2
+    x = np.asarray(X_cand, dtype=F32)
+    states = []
+    for spec, W in zip(specs, Ws):
+        st = layer_forward(spec, x, W, half, step)
+        states.append(st)
+        x = st.Xnext
+    total = np.zeros(n_classes * B, dtype=F32)
+    for st in states[first_counted:]:
+        total = total + st.G.astype(F32)          # float32 additions in layer order
+    scores = total.reshape(n_classes, B)
+    pred = np.argmax(scores, axis=0).astype(np.int32)   # first maximum = lowest label
+    return pred, scores, states
+
+
+# --------------------------------------------------------------------------------------
 # Unquantised float64 model of one layer (for the finite-difference pin only)
 # --------------------------------------------------------------------------------------
 def fp64_layer_loss(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int) -> float:

@@ -21,10 +21,10 @@ FF_ABSMAX_LEN = 8
 EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", "ff_set_gemm_path", "ff_set_tensor_form",
            "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step",
            "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
-           "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static"]
+           "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict"]
 FF_STATIC_LOSS_MAX_SAMPLES = 65536
 FF_K_NAMES = ["absmax", "quantize", "fwd_gemm", "finalize", "normalize", "loss", "dh_quantize",
-              "upd_gemm", "raw_gemm"]
+              "upd_gemm", "raw_gemm", "classify"]
 
 
 class ff_layer_desc(C.Structure):
@@ -83,6 +83,7 @@ def load(build_if_missing: bool = True):
     lib.ff_launch_count.restype = u64
     lib.ff_int8_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ff_profile_start.argtypes = [vp]
+    lib.ff_predict.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, i32, i32, i32, vp, vp, u64, vp]
     lib.ff_loss_coef_static.argtypes = [vp, f32, C.POINTER(vp), C.POINTER(f32), i32, f32, i32, vp, vp, vp, vp, vp,
                                         C.c_char_p, C.c_size_t]
     lib.ff_profile_stop.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(C.c_uint32)]
@@ -149,6 +150,13 @@ def ff_layer_update(ctx, desc, bufs, B: int, stream: int = 0):
 def ff_train_step(ctx, descs_arr, bufs_arr, n_layers: int, B: int, lam: float, step: int, stream: int = 0):
     """descs_arr / bufs_arr: ctypes arrays (ff_layer_desc * n), (ff_layer_bufs * n)."""
     _check(ctx, load().ff_train_step(ctx, descs_arr, bufs_arr, n_layers, B, lam, step, stream))
+
+
+def ff_predict(ctx, descs_arr, bufs_arr, n_layers: int, B: int, n_classes: int, first_counted_layer: int, scores: int,
+               pred: int, step: int, stream: int = 0):
+    """descs_arr / bufs_arr as for ff_train_step; scores / pred are device addresses."""
+    _check(ctx, load().ff_predict(ctx, descs_arr, bufs_arr, n_layers, B, n_classes, first_counted_layer, scores, pred,
+                                  step, stream))
 
 
 def ff_poll_status(ctx, stream: int = 0):

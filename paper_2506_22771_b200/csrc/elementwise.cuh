@@ -338,6 +338,29 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
 }
 
 // ---------------------------------------------------------------------------------------------
+// Classification by goodness (Sec. III): sample b was presented once per candidate label c (row c*B + b);
+// its score for c is the sum over the counted layers of that row's goodness (FP32 additions in layer
+// order), its label the candidate with the largest score (lowest label on ties).  One thread per sample.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) classify_kernel(LaterLayers layers, int B, int n_classes,
+                                                              float* __restrict__ scores, int32_t* __restrict__ pred) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  float best = 0.0f;
+  int best_c = 0;
+  for (int c = 0; c < n_classes; ++c) {
+    float total = 0.0f;
+    for (int j = 0; j < layers.n; ++j) total = __fadd_rn(total, layers.G[j][(size_t)c * B + b]);
+    scores[(size_t)c * B + b] = total;
+    if (c == 0 || total > best) {
+      best = total;
+      best_c = c;
+    }
+  }
+  pred[b] = best_c;
+}
+
+// ---------------------------------------------------------------------------------------------
 // dHq = clip(round((2*coef_m * y) * 127/a_dh[p])).  grid = (blocks, 2)
 // ---------------------------------------------------------------------------------------------
 template <int MODE>

@@ -490,6 +490,40 @@ ff_status loss_grad_impl(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
   return FF_OK;
 }
 
+ff_status check_layer_list(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B) {
+  if (!layers || !bufs || n_layers <= 0 || n_layers > FF_MAX_LATER + 1) return fail(ctx, FF_ERR_ARG, "bad layer list");
+  ff_status s;
+  for (int l = 0; l < n_layers; ++l) {
+    if ((s = check_layer(ctx, &layers[l], B)) != FF_OK) return s;
+    if ((s = check_bufs(ctx, &bufs[l], l == 0)) != FF_OK) return s;
+    if (l > 0 && !bufs[l].X) {
+      const ff_layer_desc &p = layers[l - 1], &c = layers[l];
+      if ((long long)rows_per_sample(p) * p.N != (long long)rows_per_sample(c) * in_features(c))
+        return fail(ctx, FF_ERR_ARG, "layer output / next layer input sizes differ");
+    }
+  }
+  return FF_OK;
+}
+
+// INT8 forward through all layers with the current weights (Alg. 1 line 5-6): layer 0 reads bufs[0].X,
+// layer l > 0 reads bufs[l].X if given, else the previous layer's normalised output, quantised on the fly.
+ff_status forward_all(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B, uint64_t step,
+                      cudaStream_t st) {
+  ff_status s;
+  for (int l = 0; l < n_layers; ++l) FF_CUDA(ctx, cudaMemsetAsync(bufs[l].absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
+  for (int l = 0; l < n_layers; ++l) {
+    const bool chained = l > 0 && !bufs[l].X;
+    if (!chained && (s = quantize_input(ctx, layers[l], bufs[l], B, step, st)) != FF_OK) return s;
+    const bool feeds_next = l + 1 < n_layers && !bufs[l + 1].X;
+    if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, step, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st)) != FF_OK)
+      return s;
+    if ((s = normalize_output(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].Xq : nullptr,
+                              feeds_next ? &layers[l + 1] : nullptr, step, st)) != FF_OK)
+      return s;
+  }
+  return FF_OK;
+}
+
 }  // namespace
 
 // ================================================================================================
@@ -617,30 +651,11 @@ ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
                         float lambda, uint64_t step, void* cuda_stream) {
   ff_status s = check_ctx(ctx);
   if (s != FF_OK) return s;
-  if (!layers || !bufs || n_layers <= 0 || n_layers > FF_MAX_LATER + 1) return fail(ctx, FF_ERR_ARG, "bad layer list");
-  for (int l = 0; l < n_layers; ++l) {
-    if ((s = check_layer(ctx, &layers[l], B)) != FF_OK) return s;
-    if ((s = check_bufs(ctx, &bufs[l], l == 0)) != FF_OK) return s;
-    if (l > 0 && !bufs[l].X) {
-      const ff_layer_desc &p = layers[l - 1], &c = layers[l];
-      if ((long long)rows_per_sample(p) * p.N != (long long)rows_per_sample(c) * in_features(c))
-        return fail(ctx, FF_ERR_ARG, "layer output / next layer input sizes differ");
-    }
-  }
+  if ((s = check_layer_list(ctx, layers, bufs, n_layers, B)) != FF_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
-  for (int l = 0; l < n_layers; ++l) FF_CUDA(ctx, cudaMemsetAsync(bufs[l].absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
   // Alg. 1 line 5-6: one forward through all layers with the pre-update weights
-  for (int l = 0; l < n_layers; ++l) {
-    const bool chained = l > 0 && !bufs[l].X;
-    if (!chained && (s = quantize_input(ctx, layers[l], bufs[l], B, step, st)) != FF_OK) return s;
-    const bool feeds_next = l + 1 < n_layers && !bufs[l + 1].X;
-    if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, step, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st)) != FF_OK)
-      return s;
-    if ((s = normalize_output(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].Xq : nullptr,
-                              feeds_next ? &layers[l + 1] : nullptr, step, st)) != FF_OK)
-      return s;
-  }
+  if ((s = forward_all(ctx, layers, bufs, n_layers, B, step, st)) != FF_OK) return s;
   // Alg. 1 line 7-9: per layer, loss from the G's (Eq. 3), INT8 gradient and update
   for (int l = 0; l < n_layers; ++l) {
     const float* Gl[FF_MAX_LATER];
@@ -653,6 +668,35 @@ ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
     if ((s = loss_grad_impl(ctx, layers[l], bufs[l], B, Gl, th, n_later, lambda, step, st)) != FF_OK) return s;
     if ((s = run_update_gemm(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
   }
+  return FF_OK;
+}
+
+ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B, int n_classes,
+                     int first_counted_layer, float* scores, int32_t* pred, uint64_t step, void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if (n_classes <= 0 || (n_classes & 1)) return fail(ctx, FF_ERR_ARG, "n_classes must be even and positive");
+  if (B <= 0) return fail(ctx, FF_ERR_ARG, "B must be positive");
+  if (!scores || !pred) return fail(ctx, FF_ERR_ARG, "scores / pred is NULL");
+  if (!aligned16(scores) || !aligned16(pred)) return fail(ctx, FF_ERR_ALIGN, "scores / pred must be 16-byte aligned");
+  if ((long long)n_classes * B / 2 >= (1LL << 30)) return fail(ctx, FF_ERR_RANGE, "too many candidate rows");
+  const int half = n_classes * B / 2;  // rows of each of the two quantisation sets of the candidate batch
+  if ((s = check_layer_list(ctx, layers, bufs, n_layers, half)) != FF_OK) return s;
+  if (first_counted_layer < 0 || first_counted_layer >= n_layers) return fail(ctx, FF_ERR_ARG, "first_counted_layer out of range");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  if ((s = forward_all(ctx, layers, bufs, n_layers, half, step, st)) != FF_OK) return s;
+  LaterLayers gs;
+  gs.n = n_layers - first_counted_layer;
+  for (int j = 0; j < gs.n; ++j) {
+    gs.G[j] = bufs[first_counted_layer + j].G;
+    gs.theta[j] = 0.0f;
+  }
+  {
+    ProfScope prof(ctx, FF_K_CLASSIFY, st);
+    classify_kernel<<<(B + EW_THREADS - 1) / EW_THREADS, EW_THREADS, 0, st>>>(gs, B, n_classes, scores, pred);
+  }
+  FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
 

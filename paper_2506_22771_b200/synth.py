@@ -137,3 +137,30 @@ def make_batch(w: Workload, seed: int, batch_index: int = 0, B: int = None) -> n
     norm = np.sqrt((flat ** 2).sum(axis=1, keepdims=True))
     flat *= np.sqrt(float(n_in)) / (norm + 1e-8)
     return np.ascontiguousarray(x.astype(F32))
+
+
+def make_candidates(w: Workload, seed: int, B: int, n_classes: int = 10, batch_index: int = 0):
+    """Candidate batch for classification [n_classes*B, *in_shape] FP32: row c*B + b is sample b with
+    candidate label c written one-hot into it (same places as make_batch), each row scaled to length
+    sqrt(number of input values).  Also returns the B drawn labels (random: the data carry no class
+    structure, they only have the right shape)."""
+    g = _rng(seed, 3000 + batch_index)
+    n_in = int(np.prod(w.in_shape))
+    if w.data == "uniform01":
+        base = g.random((B, n_in), dtype=np.float64)
+    else:
+        base = g.normal(0.0, 1.0, size=(B, n_in))
+    label = g.integers(0, n_classes, size=B)
+    x = np.tile(base, (n_classes, 1)).reshape((n_classes * B,) + tuple(w.in_shape))
+    for c in range(n_classes):
+        rows = np.arange(B) + c * B
+        if len(w.in_shape) == 1:
+            x[rows, :n_classes] = 0.0
+            x[rows, c] = 1.0
+        else:
+            x[rows, 0, :n_classes, 0] = 0.0
+            x[rows, 0, c, 0] = 1.0
+    flat = x.reshape(n_classes * B, -1)
+    norm = np.sqrt((flat ** 2).sum(axis=1, keepdims=True))
+    flat *= np.sqrt(float(n_in)) / (norm + 1e-8)
+    return np.ascontiguousarray(x.astype(F32)), label.astype(np.int32)

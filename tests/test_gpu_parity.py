@@ -214,3 +214,35 @@ def test_host_side_argument_errors():
         ffb.ff_layer_forward(net.ctx.ctx, descs[0], bufs, w.B, 0, 0)
     assert e.value.code == ffb.FF_ERR_ALIGN
     net.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("first_counted", [0, 1])
+def test_predict_matches_oracle(path, first_counted):
+    import torch
+    n_classes, B = 10, 52                       # 520 candidate rows: several tiles and a ragged tail
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=n_classes * B // 2, width_div=4)
+    w.layers = w.layers[:3]
+    specs, descs = specs_and_descs(w.layers, 6)
+    Ws = synth.make_weights(w, 6)
+    Xc, _ = synth.make_candidates(w, 6, B, n_classes)
+    net = GpuNet(descs, n_classes * B // 2, Ws, dumps=False, xnext=False, chain=True, gemm_path=path)
+    net.set_input(Xc)
+    scores = torch.zeros(n_classes * B, dtype=torch.float32, device="cuda")
+    pred = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    ffb.ff_predict(net.ctx.ctx, net.descs_arr, net.bufs_arr, len(descs), B, n_classes, first_counted,
+                   scores.data_ptr(), pred.data_ptr(), 3, 0)
+    ffb.ff_poll_status(net.ctx.ctx, 0)
+    want_pred, want_scores, states = O.predict(specs, Ws, Xc, B, n_classes, 3, first_counted)
+    for l, st in enumerate(states):
+        assert np.array_equal(net.bufs[l].G.cpu().numpy().view(np.uint32), st.G.view(np.uint32)), f"G of layer {l}"
+        assert np.array_equal(net.bufs[l].Xq.cpu().numpy().reshape(-1), st.Xq.reshape(-1)), f"Xq of layer {l}"
+    assert np.array_equal(scores.cpu().numpy().view(np.uint32), want_scores.reshape(-1).view(np.uint32))
+    assert np.array_equal(pred.cpu().numpy(), want_pred)
+    # weights untouched
+    for b, W in zip(net.bufs, Ws):
+        assert torch.equal(b.W.cpu(), torch.from_numpy(W))
+    with pytest.raises(ffb.FFError) as e:
+        ffb.ff_predict(net.ctx.ctx, net.descs_arr, net.bufs_arr, len(descs), B, 9, 0, scores.data_ptr(), pred.data_ptr(), 0, 0)
+    assert e.value.code == ffb.FF_ERR_ARG
+    net.close()

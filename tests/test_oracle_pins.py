@@ -486,3 +486,69 @@ def test_tiny_range_is_treated_as_zero_tensor():
     b = F32(2.0 ** -99)
     s, inv = O.scale_pair(b)
     assert np.isfinite(inv) and s == b / F32(127.0)
+
+
+# --------------------------------------------------------------------------------------
+# Classification by goodness, and the direction of learning
+# --------------------------------------------------------------------------------------
+def test_predict_hand_example_and_tie_rule():
+    # one linear layer with identity-like weights, nearest rounding, B = 2 samples, 2 candidate labels:
+    # sample 0 is longer along unit 0 under label 0, sample 1 gives both labels the same goodness (tie -> 0)
+    spec = O.LayerSpec(O.KIND_LINEAR, 2, 2, theta=1.0, lr=0.0, tau=1.0, round_x=0, round_w=0, round_dh=0)
+    W = np.eye(2, dtype=np.float32)
+    X = np.array([[1.0, 0.0],     # label 0, sample 0
+                  [1.0, 1.0],     # label 0, sample 1
+                  [0.5, 0.0],     # label 1, sample 0
+                  [1.0, 1.0]],    # label 1, sample 1  (both halves have range 1, so the tie is exact)
+                 dtype=np.float32)
+    pred, scores, states = O.predict([spec], [W], X, B=2, n_classes=2, step=0)
+    assert scores.shape == (2, 2)
+    assert scores[0, 0] > scores[1, 0] and scores[0, 1] == scores[1, 1]
+    assert pred.tolist() == [0, 0]
+    # scores are the goodness of the only layer
+    assert np.array_equal(scores.reshape(-1), states[0].G)
+    # with two layers and first_counted = 1 only the second layer counts
+    spec2 = O.LayerSpec(O.KIND_LINEAR, 2, 2, theta=1.0, lr=0.0, tau=1.0, round_x=0, round_w=0, round_dh=0, index=1)
+    _, s2, st2 = O.predict([spec, spec2], [W, W], X, 2, 2, 0, first_counted=1)
+    assert np.array_equal(s2.reshape(-1), st2[1].G)
+    _, s01, st01 = O.predict([spec, spec2], [W, W], X, 2, 2, 0, first_counted=0)
+    assert np.array_equal(s01.reshape(-1), (st01[0].G + st01[1].G).astype(np.float32))
+
+
+def test_int8_ff_training_learns_and_predicts_separable_classes():
+    """End-to-end direction check of the whole oracle: FF-INT8 training (positive set = true label, negative
+    set = wrong label, Eq. 1 / Eq. 2, INT8 gradients) followed by classification by goodness must learn
+    class-dependent synthetic data: a flipped sign anywhere (loss, gradient, update, argmax) keeps the
+    accuracy at chance."""
+    K, N, C, B = 64, 64, 10, 64
+    g = np.random.default_rng(0)
+    patterns = g.normal(size=(C, K))
+
+    def draw(gen, n):
+        lab = gen.integers(0, C, size=n)
+        return patterns[lab] + 0.5 * gen.normal(size=(n, K)), lab
+
+    def embed(base, lab):
+        x = base.copy()
+        x[:, :C] = 0.0
+        x[np.arange(len(lab)), lab] = 1.0
+        return (x * np.sqrt(K) / np.sqrt((x ** 2).sum(1, keepdims=True))).astype(np.float32)
+
+    specs = [O.LayerSpec(O.KIND_LINEAR, K, N, theta=float(N), lr=0.03, tau=float(np.sqrt(N)), seed=3, index=0),
+             O.LayerSpec(O.KIND_LINEAR, N, N, theta=float(N), lr=0.03, tau=float(np.sqrt(N)), seed=3, index=1)]
+    Ws = [(g.uniform(-1, 1, size=(N, K)) * np.sqrt(6 / K)).astype(np.float32),
+          (g.uniform(-1, 1, size=(N, N)) * np.sqrt(6 / N)).astype(np.float32)]
+
+    def accuracy(weights):
+        base, lab = draw(np.random.default_rng(999), 200)
+        Xc = np.concatenate([embed(base, np.full(200, c)) for c in range(C)])
+        pred, _, _ = O.predict(specs, weights, Xc, 200, C, step=0)
+        return float((pred == lab).mean())
+
+    assert accuracy(Ws) < 0.3
+    for step in range(40):
+        base, lab = draw(g, B)
+        wrong = (lab + g.integers(1, C, size=B)) % C
+        X = np.concatenate([embed(base, lab), embed(base, wrong)])
+        Ws = [st.W_new for st in O.train_step(specs, Ws, X, B, 0.0, step)]
+    assert accuracy(Ws) > 0.9
