@@ -323,7 +323,7 @@ def main():
         for b, W in zip(bufs, W0):
             b.W.copy_(W)
 
-    # ---------------- device-resident timing (value), per-kernel events inside the same region --------
+    # ---------------- device-resident timing (value) ----------------
     for i in range(args.warmup):
         step(i)
     ffb.ff_poll_status(ctx.ctx, stream)
@@ -334,7 +334,6 @@ def main():
         time.sleep(0.3)
     barrier()
     l0 = ffb.ff_launch_count(ctx.ctx)
-    ffb.ff_profile_start(ctx.ctx)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_begin = time.time()
     e0.record()
@@ -342,14 +341,28 @@ def main():
         step(i)
     e1.record()
     barrier()
-    t_end = time.time()
-    kernel_ms = ffb.ff_profile_stop(ctx.ctx, stream)
     launches = ffb.ff_launch_count(ctx.ctx) - l0
     ms_local = e0.elapsed_time(e1)
-    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     ffb.ff_poll_status(ctx.ctx, stream)
     loss_last = float(bufs[last].loss[0].item())
     ms, value = whole_job_throughput(ms_local, B * args.steps, dev)
+
+    # ---------------- the same K steps again with a CUDA-event pair around every kernel ----------------
+    # (a second region, so that the events' cost stays out of `value`; same steps, same state of the device)
+    reset_weights()
+    barrier()
+    ffb.ff_profile_start(ctx.ctx)
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    for i in range(args.steps):
+        step(i)
+    e3.record()
+    barrier()
+    t_end = time.time()
+    kernel_ms = ffb.ff_profile_stop(ctx.ctx, stream)
+    ms_profiled = e2.elapsed_time(e3)
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
+    ffb.ff_poll_status(ctx.ctx, stream)
 
     # ---------------- end to end: host buffers, H2D of the batch + D2H of the loss every step ---------
     # The batch of step i+1 is copied (pinned host -> second device buffer, copy stream) while step i
@@ -398,13 +411,13 @@ def main():
     if rank == 0:
         peaks = _peaks()
         work = algorithmic_work(w, B)
-        burst = ms * 1e-3 < BURST_SECONDS
+        burst = (ms + ms_profiled) * 1e-3 < BURST_SECONDS
         bf16 = peaks["bf16_burst"] if burst else peaks["bf16_sustained"]
         int8_peak = INT8_TO_BF16 * bf16
         per_kernel = {}
         for k, (tot_ms, n) in kernel_ms.items():
             ent = {"launches_per_step": n / args.steps, "ms_per_step": tot_ms / args.steps,
-                   "share": tot_ms / ms_local}
+                   "share": tot_ms / ms_profiled}
             if k in work and work[k] > 0 and tot_ms > 0:
                 rate = work[k] * args.steps / (tot_ms * 1e-3)
                 if k.endswith("gemm"):
@@ -426,11 +439,12 @@ def main():
                        "l2": "inputs larger than L2 (no flush needed)"
                        if 2 * B * l.H * l.Wd * l.K * 4 > 126e6 else "inputs smaller than L2, not flushed"},
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "loss_last": loss_last,
+            "ms_per_step_with_kernel_events": ms_profiled / args.steps,
             "roofline": {"bound": "tensor", "kernel": names[dom], "achieved": per_kernel[dom]["achieved"],
                          "peak": int8_peak, "unit": "TOP/s", "frac": per_kernel[dom]["frac"],
                          "peak_source": f"{INT8_TO_BF16:g} x {peaks['source']} bf16 cuBLAS "
-                                        f"{'burst' if burst else 'sustained'} ({bf16} TF/s): the timed region lasted "
-                                        f"{ms * 1e-3:.2f} s",
+                                        f"{'burst' if burst else 'sustained'} ({bf16} TF/s): the two timed regions lasted "
+                                        f"{(ms + ms_profiled) * 1e-3:.2f} s",
                          "frac_of_sustained_x2": per_kernel[dom]["achieved"] / (INT8_TO_BF16 * peaks["bf16_sustained"]),
                          "frac_of_nominal_4500": per_kernel[dom]["achieved"] / 4500.0,
                          "traffic": _ncu_traffic(dom, args.workload, B)},
