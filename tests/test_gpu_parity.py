@@ -246,3 +246,48 @@ def test_predict_matches_oracle(path, first_counted):
         ffb.ff_predict(net.ctx.ctx, net.descs_arr, net.bufs_arr, len(descs), B, 9, 0, scores.data_ptr(), pred.data_ptr(), 0, 0)
     assert e.value.code == ffb.FF_ERR_ARG
     net.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("B,K,N", [(1, 1, 1), (1, 16, 16), (3, 5, 7), (2, 33, 500), (129, 144, 272), (65, 784, 16)])
+def test_edge_shapes_dense(path, B, K, N):
+    # smallest and ragged shapes: one sample per set, single features, sizes that are no multiple of any tile
+    layers = [synth.LayerCfg(0, K, N, float(N) / 2, 0.03, float(np.sqrt(N))),
+              synth.LayerCfg(0, N, 24, 12.0, 0.03, float(np.sqrt(24)))]
+    w = synth.Workload("edge", B, layers, (K,), "normal", "kaiming_uniform", 2)
+    specs, descs = specs_and_descs(w.layers, 41)
+    Ws = synth.make_weights(w, 41)
+    g = np.random.default_rng(B * 1000 + K)
+    X = g.normal(size=(2 * B, K))
+    X = (X * np.sqrt(K) / (np.sqrt((X ** 2).sum(1, keepdims=True)) + 1e-8)).astype(np.float32)
+    net = GpuNet(descs, B, Ws, gemm_path=path)
+    net.set_input(X)
+    for step in range(2):
+        net.train_step(0.5, step)
+        states = O.train_step(specs, Ws, X, B, 0.5, step)
+        for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
+            compare_layer(st, b, sp, B, tag=f"step{step}/layer{l}/")
+        Ws = [st.W_new for st in states]
+    net.close()
+
+
+def test_dead_layer_and_vanishing_gradient():
+    # all-negative weights on a non-negative input: every accumulator <= 0, so Y = 0, G = 0, dH = 0 and its
+    # range is 0 (all-zero codes); the weights must come back unchanged and the next layer sees zeros
+    import torch
+    B, K, N = 40, 64, 48
+    layers = [synth.LayerCfg(0, K, N, float(N), 0.03, float(np.sqrt(N))), synth.LayerCfg(0, N, 32, 32.0, 0.03, float(np.sqrt(32)))]
+    w = synth.Workload("dead", B, layers, (K,), "uniform01", "kaiming_uniform", 1)
+    specs, descs = specs_and_descs(w.layers, 2)
+    Ws = synth.make_weights(w, 2)
+    Ws[0] = -np.abs(Ws[0])
+    X = np.abs(synth.make_batch(w, 2))
+    net = GpuNet(descs, B, Ws)
+    net.set_input(X)
+    net.train_step(0.3, 0)
+    states = O.train_step(specs, Ws, X, B, 0.3, 0)
+    for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
+        compare_layer(st, b, sp, B, tag=f"layer{l}/")
+    assert not net.bufs[0].Y.any() and not net.bufs[0].G.any() and not net.bufs[0].dHq.any()
+    assert torch.equal(net.bufs[0].W.cpu(), torch.from_numpy(Ws[0]))
+    net.close()
