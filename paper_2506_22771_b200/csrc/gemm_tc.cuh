@@ -88,6 +88,7 @@ struct TcParams {
   const float* absmax;
   int rows_per_pass, rows_per_sample;
   int y_tma;                // Y leaves through TMA stores (needs N % 4 == 0); else plain stores
+  int y_stream;             // Y is larger than what L2 can usefully hold for the kernels that follow
   // update epilogue
   float* W;
   int32_t* accW_dump;
@@ -551,7 +552,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     uint8_t* patch0 = patch_all + (warp - 2) * TC_PATCHES * TC_PATCH_BYTES;
     uint32_t pflip = 0;  // which of the warp's two patches the next chunk fills (forward epilogue)
     (void)pflip;
-    const uint64_t y_policy = l2_policy_evict_first();
+    // A large Y is written once and read much later: let it leave L2 first.  A small one is read back by
+    // the next kernels (normalisation, dH quantiser) while it still sits in L2: keep it.
+    const uint64_t y_policy = p.y_stream ? l2_policy_evict_first() : l2_policy_evict_last();
     (void)y_policy;
     uint32_t tile_it = 0;
     bool ok = true;
@@ -1053,6 +1056,7 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   const int ncta = tc_pick_ncta(t, M, L.N);
   CUtensorMap ty;
   p.y_tma = (L.N % 4 == 0) ? 1 : 0;
+  p.y_stream = (size_t)M * L.N * sizeof(float) > ((size_t)80 << 20) ? 1 : 0;
 
   if (p.y_tma && (s = tc_make_store_map(t, &ty, b.Y, L.N, M)) != FF_OK) return s;
   const CUtensorMap* typ = p.y_tma ? &ty : nullptr;
