@@ -52,7 +52,7 @@ typedef enum {
   FF_ERR_UNSUPPORTED_ARCH = -8 /* the device is not compute capability 10.x                    */
 } ff_status;
 
-enum { FF_LINEAR = 0, FF_CONV3X3 = 1 };                  /* ff_layer_desc.kind      */
+enum { FF_LINEAR = 0, FF_CONV3X3 = 1, FF_CONV1X1 = 2 };  /* ff_layer_desc.kind      */
 enum { FF_ROUND_NEAREST_EVEN = 0, FF_ROUND_STOCHASTIC = 1 }; /* rounding modes (Sec. IV-B) */
 enum { FF_GEMM_AUTO = 0, FF_GEMM_SIMT = 1, FF_GEMM_TENSOR = 2 }; /* ff_set_gemm_path       */
 
@@ -67,11 +67,13 @@ enum {
 
 /* One FF layer (host struct).  linear: X[M,K] -> Y[M,N], W[N,K].
  * conv3x3 (stride 1, zero padding 1, NHWC): X[M,H,Wd,Cin] -> Y[M,H,Wd,N], W[N,3,3,Cin] stored as
- * [N,K] with K = 9*Cin and k = (r*3+s)*Cin + ci. */
+ * [N,K] with K = 9*Cin and k = (r*3+s)*Cin + ci.
+ * conv1x1 (pointwise, NHWC): X[M,H,Wd,Cin] -> Y[M,H,Wd,N], W[N,Cin], K = Cin: the dense MAC applied
+ * at every position; goodness and normalisation over all H*Wd*N values of a sample. */
 typedef struct {
   int32_t kind;
   int32_t K, N;
-  int32_t H, Wd, Cin;   /* conv only; 1,1,0 for linear                                        */
+  int32_t H, Wd, Cin;   /* conv3x3 / conv1x1 only; 1,1,0 for linear                           */
   int32_t index;        /* position of the layer in the network (keys the rounding hash)      */
   int32_t round_x, round_w, round_dh; /* rounding of A, W, g^Y (paper: stochastic for A)      */
   float theta;          /* threshold of Eq. 1 / Eq. 2                                         */

@@ -40,6 +40,7 @@ ROLE_DH = 2  # hash stream of the output-gradient quantiser
 
 KIND_LINEAR = 0
 KIND_CONV3X3 = 1
+KIND_CONV1X1 = 2
 
 _M64 = (1 << 64) - 1
 
@@ -50,7 +51,8 @@ _M64 = (1 << 64) - 1
 @dataclass
 class LayerSpec:
     """One FF layer.  linear: X [2B,K] -> Y [2B,N].  conv3x3 (stride 1, zero pad 1, NHWC):
-    X [2B,H,W,Cin] -> Y [2B,H,W,N] with K = 9*Cin and weights [N,3,3,Cin] flattened to [N,K]."""
+    X [2B,H,W,Cin] -> Y [2B,H,W,N] with K = 9*Cin and weights [N,3,3,Cin] flattened to [N,K].
+    conv1x1 (pointwise, NHWC): X [2B,H,W,Cin] -> Y [2B,H,W,N] with K = Cin and weights [N,Cin]."""
     kind: int
     K: int
     N: int
@@ -69,7 +71,7 @@ class LayerSpec:
 
     @property
     def rows_per_sample(self) -> int:
-        return self.H * self.Wd if self.kind == KIND_CONV3X3 else 1
+        return self.H * self.Wd if self.kind != KIND_LINEAR else 1
 
 
 # --------------------------------------------------------------------------------------
@@ -376,6 +378,9 @@ def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: i
     st.Wq = quantize(W, st.a_w, spec.round_w, rounding_key(spec.seed, ROLE_W, spec.index, step))
     if spec.kind == KIND_LINEAR:
         st.acc = int8_gemm_nt(st.Xq, st.Wq)
+    elif spec.kind == KIND_CONV1X1:
+        # pointwise convolution: the dense MAC applied at every position ('dense or convolution layers', Sec. IV-B)
+        st.acc = int8_gemm_nt(st.Xq.reshape(-1, spec.K), st.Wq).reshape(st.Xq.shape[:3] + (spec.N,))
     else:
         st.acc = int8_conv3x3(st.Xq, st.Wq.reshape(spec.N, 3, 3, spec.Cin))
     s_w, _ = scale_pair(st.a_w)
@@ -407,6 +412,8 @@ def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int) -> Laye
         sl = slice(p * B, (p + 1) * B)
         if spec.kind == KIND_LINEAR:
             accW.append(int8_gemm_tn(st.dHq[sl], st.Xq[sl]))
+        elif spec.kind == KIND_CONV1X1:
+            accW.append(int8_gemm_tn(st.dHq[sl].reshape(-1, spec.N), st.Xq[sl].reshape(-1, spec.K)))
         else:
             accW.append(int8_conv3x3_wgrad(st.dHq[sl], st.Xq[sl]).reshape(spec.N, spec.K))
     st.accW = np.stack(accW)
@@ -475,7 +482,7 @@ def fp64_layer_loss(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int) -> fl
     """Mean over the 2B samples of Eq. 1 / Eq. 2 with G = ||relu(X W^T)||^2, no quantisation."""
     X = np.asarray(X, dtype=F64)
     W = np.asarray(W, dtype=F64)
-    if spec.kind == KIND_LINEAR:
+    if spec.kind in (KIND_LINEAR, KIND_CONV1X1):
         Y = np.maximum(X @ W.T, 0.0)
     else:
         xp = np.pad(X, ((0, 0), (1, 1), (1, 1), (0, 0)))

@@ -12,7 +12,7 @@ from . import build as _build
 FF_OK = 0
 FF_ERR_ARG, FF_ERR_ALIGN, FF_ERR_WORKSPACE, FF_ERR_NONFINITE = -1, -2, -3, -4
 FF_ERR_RANGE, FF_ERR_DEVICE_TIMEOUT, FF_ERR_CUDA, FF_ERR_UNSUPPORTED_ARCH = -5, -6, -7, -8
-FF_LINEAR, FF_CONV3X3 = 0, 1
+FF_LINEAR, FF_CONV3X3, FF_CONV1X1 = 0, 1, 2
 FF_ROUND_NEAREST_EVEN, FF_ROUND_STOCHASTIC = 0, 1
 FF_GEMM_AUTO, FF_GEMM_SIMT, FF_GEMM_TENSOR = 0, 1, 2
 FF_A_X_POS, FF_A_X_NEG, FF_A_W, FF_A_DH_POS, FF_A_DH_NEG, FF_A_XNEXT_POS, FF_A_XNEXT_NEG = range(7)
@@ -214,8 +214,8 @@ class LayerBuffers:
     def __init__(self, desc: ff_layer_desc, B: int, device, dumps: bool = False, xnext: bool = True,
                  own_x: bool = True):
         import torch
-        R = desc.H * desc.Wd if desc.kind == FF_CONV3X3 else 1
-        kin = desc.Cin if desc.kind == FF_CONV3X3 else desc.K
+        R = desc.H * desc.Wd if desc.kind != FF_LINEAR else 1
+        kin = desc.Cin if desc.kind != FF_LINEAR else desc.K
         rows = 2 * B * R
         z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)
         self.W = z((desc.N, desc.K), torch.float32)

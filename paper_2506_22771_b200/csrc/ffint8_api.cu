@@ -6,6 +6,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <type_traits>
 #include <vector>
@@ -96,13 +97,15 @@ struct ProfScope {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-inline int rows_per_sample(const ff_layer_desc& L) { return L.kind == FF_CONV3X3 ? L.H * L.Wd : 1; }
+inline int rows_per_sample(const ff_layer_desc& L) { return L.kind != FF_LINEAR ? L.H * L.Wd : 1; }
 inline int in_features(const ff_layer_desc& L) { return L.kind == FF_CONV3X3 ? L.Cin : L.K; }
 
 ff_status check_layer(ff_ctx* ctx, const ff_layer_desc* L, int B) {
   if (!L) return fail(ctx, FF_ERR_ARG, "layer descriptor is NULL");
   if (B <= 0) return fail(ctx, FF_ERR_ARG, "B must be positive");
-  if (L->kind != FF_LINEAR && L->kind != FF_CONV3X3) return fail(ctx, FF_ERR_ARG, "unknown layer kind");
+  if (L->kind != FF_LINEAR && L->kind != FF_CONV3X3 && L->kind != FF_CONV1X1) return fail(ctx, FF_ERR_ARG, "unknown layer kind");
+  if (L->kind == FF_CONV1X1 && (L->H <= 0 || L->Wd <= 0 || L->Cin <= 0 || L->K != L->Cin))
+    return fail(ctx, FF_ERR_ARG, "conv1x1 needs H, Wd, Cin > 0 and K = Cin");
   if (L->K <= 0 || L->N <= 0) return fail(ctx, FF_ERR_ARG, "K and N must be positive");
   if (L->kind == FF_CONV3X3 && (L->H <= 0 || L->Wd <= 0 || L->Cin <= 0 || L->K != 9 * L->Cin))
     return fail(ctx, FF_ERR_ARG, "conv3x3 needs H, Wd, Cin > 0 and K = 9*Cin");
@@ -293,7 +296,7 @@ ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
     return FF_OK;
   }
   ForwardEpilogue epi{b.Y, b.acc_dump, reinterpret_cast<unsigned long long*>(b.S), b.rowmax, b.absmax, rows, L.N, B * R, R};
-  if (L.kind == FF_LINEAR)
+  if (L.kind != FF_CONV3X3)
     return launch_simt<DenseView, DenseView, false, 1>(ctx, dense(b.Xq, rows, L.K), dense(b.Wq, L.N, L.K), rows, L.N, L.K, epi, st);
   return launch_simt<Im2colView, DenseView, false, 1>(ctx, im2col(b.Xq, L, 2 * B), dense(b.Wq, L.N, L.K), rows, L.N, L.K, epi, st);
 }
@@ -327,9 +330,30 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     return s;
   }
   if (ctx->gemm_path == FF_GEMM_TENSOR && !tc_ok) return fail(ctx, FF_ERR_ARG, "shape not supported by the tensor-core weight gradient");
-  if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT && L.kind == FF_LINEAR) {
+  if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT && L.kind == FF_CONV1X1) {
+    // pointwise convolution: a dense contraction over every position of a set.  With few output tiles it is
+    // split into INT32 slabs like the 3x3 case; otherwise the fused dense kernel below takes it.
+    int splits = tc_dense_slab_splits(L.N, L.K, (long long)B * R, ctx->sm_count);
+    const size_t room = ctx->workspace_bytes > WS_BYTES ? ctx->workspace_bytes - WS_BYTES : 0;
+    const size_t per_split = (size_t)2 * L.N * L.K * sizeof(int32_t);
+    if ((size_t)splits * per_split > room) splits = (int)(room / per_split);
+    if (splits >= 2) {
+      int32_t* slabs = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
+      ProfScope prof(ctx, FF_K_UPD_GEMM, st);
+      int used = 0;
+      ff_status s = tc_dense_update_slab(ctx->tc, b.dHq, L.N, b.Xq, L.K, B * R, slabs, splits, &used, status_ptr(ctx), st);
+      if (s != FF_OK) return fail(ctx, s, "tensor-core weight-gradient launch failed: %s", ctx->tc.err);
+      ctx->launches++;
+      const bool was = ctx->profiling;
+      ctx->profiling = false;
+      s = launch_slab_update(ctx, slabs, used, L, b, st);
+      ctx->profiling = was;
+      return s;
+    }
+  }
+  if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT && L.kind != FF_CONV3X3) {
     ProfScope prof(ctx, FF_K_UPD_GEMM, st);
-    ff_status s = tc_update(ctx->tc, L, b, B, status_ptr(ctx), st);
+    ff_status s = tc_update(ctx->tc, L, b, B * R, status_ptr(ctx), st);
     if (s != FF_OK) return fail(ctx, s, "tensor-core weight-gradient launch failed: %s", ctx->tc.err);
     ctx->launches++;
     return FF_OK;
@@ -366,7 +390,7 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
       ProfScope prof(ctx, FF_K_UPD_GEMM, st);
       const bool was = ctx->profiling;
       ctx->profiling = false;  // one event pair around both launches
-      if (L.kind == FF_LINEAR)
+      if (L.kind != FF_CONV3X3)
         s = launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st, splits);
       else
         s = launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st, splits);
@@ -376,7 +400,7 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     return s;
   }
   UpdateEpilogue epi{b.W, b.accW_dump, b.absmax, L.lr, L.N, L.K};
-  if (L.kind == FF_LINEAR)
+  if (L.kind != FF_CONV3X3)
     return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st);
   return launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st);
 }
@@ -571,6 +595,11 @@ ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, s
       const int s1 = tc_conv_update_splits(layers[l], B, 0, 1), s2 = tc_conv_update_splits(layers[l], B, 0, 2);
       const size_t tc_need = tc_conv_update_slab_bytes(layers[l], s1 > s2 ? s1 : s2);
       if (tc_need > need) need = tc_need;
+    }
+    if (layers[l].kind == FF_CONV1X1 && tc_update_supported(layers[l], B)) {
+      const int sp1 = tc_dense_slab_splits(layers[l].N, layers[l].K, (long long)B * layers[l].H * layers[l].Wd, 0);
+      const size_t n1 = sp1 >= 2 ? (size_t)sp1 * 2 * layers[l].N * layers[l].K * sizeof(int32_t) : 0;
+      if (n1 > need) need = n1;
     }
     if (tc_im2col_ok(layers[l])) {
       const Im2colPlan pl = im2col_plan(layers[l], B, SIZE_MAX, 0);
@@ -788,6 +817,7 @@ static_assert(FF_STATIC_LOSS_MAX_SAMPLES == LOSS_MAX_BLOCKS * LOSS_THREADS, "one
 namespace {
 constexpr int STATIC_MAX_DEVICES = 64;
 LossScratch* g_static_loss_ptr[STATIC_MAX_DEVICES] = {nullptr};
+std::mutex g_static_loss_mutex;  // guards the table above (first calls from several host threads)
 
 void static_err(char* err, size_t err_len, const char* msg, const char* detail = "") {
   if (err && err_len) snprintf(err, err_len, "%s%s", msg, detail);
@@ -829,17 +859,21 @@ ff_status ff_loss_coef_static(const float* G, float theta, const float* const* G
     static_err(err, err_len, "cudaGetDevice: ", e != cudaSuccess ? cudaGetErrorString(e) : "device index out of range");
     return FF_ERR_CUDA;
   }
-  if (!g_static_loss_ptr[dev]) {
-    // first call on this device: turn the symbol into the address of this device's copy of the array
-    void* ptr = nullptr;
-    e = cudaGetSymbolAddress(&ptr, g_static_loss_scratch);
-    if (e != cudaSuccess || !ptr) {
-      static_err(err, err_len, "cudaGetSymbolAddress: ", cudaGetErrorString(e));
-      return FF_ERR_CUDA;
+  LossScratch* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_loss_mutex);
+    if (!g_static_loss_ptr[dev]) {
+      // first call on this device: turn the symbol into the address of this device's copy of the array
+      void* ptr = nullptr;
+      e = cudaGetSymbolAddress(&ptr, g_static_loss_scratch);
+      if (e != cudaSuccess || !ptr) {
+        static_err(err, err_len, "cudaGetSymbolAddress: ", cudaGetErrorString(e));
+        return FF_ERR_CUDA;
+      }
+      g_static_loss_ptr[dev] = static_cast<LossScratch*>(ptr);
     }
-    g_static_loss_ptr[dev] = static_cast<LossScratch*>(ptr);
+    scratch = g_static_loss_ptr[dev];
   }
-  LossScratch* scratch = g_static_loss_ptr[dev];
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   // the array keeps whatever the last call left: the block-completion ticket has to start at zero
   e = cudaMemsetAsync(&scratch->ticket, 0, sizeof(scratch->ticket), st);

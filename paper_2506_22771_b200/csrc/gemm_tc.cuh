@@ -972,10 +972,12 @@ inline bool tc_conv_ok(const ff_layer_desc& L) {
   return L.H % (128 / W) == 0;
 }
 inline bool tc_forward_supported(const ff_layer_desc& L, int B) {
-  return L.kind == FF_LINEAR ? tc_nt_ok(2LL * B, L.N, L.K) : tc_conv_ok(L);
+  if (L.kind == FF_CONV3X3) return tc_conv_ok(L);
+  return tc_nt_ok(2LL * B * (L.kind == FF_LINEAR ? 1 : L.H * L.Wd), L.N, L.K);
 }
 inline bool tc_update_supported(const ff_layer_desc& L, int B) {
-  return L.kind == FF_LINEAR ? tc_tn_ok(L.N, L.K, B) : (tc_conv_ok(L) && L.N % 16 == 0);
+  if (L.kind == FF_CONV3X3) return tc_conv_ok(L) && L.N % 16 == 0;
+  return tc_tn_ok(L.N, L.K, (long long)B * (L.kind == FF_LINEAR ? 1 : L.H * L.Wd));
 }
 
 // Split count of the convolution weight gradient (its output N x 9*Cin has few tiles, its contraction
@@ -1034,7 +1036,7 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   ff_status s = tc_init(t);
   if (s != FF_OK) return s;
   const bool conv = L.kind == FF_CONV3X3 && !xi;
-  const int R = L.kind == FF_CONV3X3 ? L.H * L.Wd : 1;
+  const int R = L.kind != FF_LINEAR ? L.H * L.Wd : 1;
   const int M = 2 * B * R;
   const int K = xi ? kpad : L.K;
   const int8_t* A = xi ? xi : b.Xq;
@@ -1080,7 +1082,7 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   return tc_launch<TC_MODE_FWD, false, 64>(t, ncta, ta, tb, p, st, typ);
 }
 
-// Dense weight gradient + update in one kernel.
+// Dense weight gradient + update in one kernel.  B = rows of one set (samples x positions per sample).
 inline ff_status tc_update(TcState& t, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint32_t* status, cudaStream_t st) {
   ff_status s = tc_init(t);
   if (s != FF_OK) return s;

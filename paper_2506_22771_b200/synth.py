@@ -18,7 +18,7 @@ F32 = np.float32
 
 @dataclass
 class LayerCfg:
-    kind: int          # 0 linear, 1 conv3x3 (stride 1, pad 1, NHWC)
+    kind: int          # 0 linear, 1 conv3x3 (stride 1, pad 1, NHWC), 2 conv1x1 (pointwise, NHWC)
     K: int
     N: int
     theta: float

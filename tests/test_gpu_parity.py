@@ -291,3 +291,22 @@ def test_dead_layer_and_vanishing_gradient():
     assert not net.bufs[0].Y.any() and not net.bufs[0].G.any() and not net.bufs[0].dHq.any()
     assert torch.equal(net.bufs[0].W.cpu(), torch.from_numpy(Ws[0]))
     net.close()
+
+
+def _mixed_conv_workload(kinds_chans, H, Wd, B):
+    """kinds_chans: list of (kind, Cin, Cout); kind 1 = 3x3, 2 = pointwise."""
+    layers = []
+    for kind, ci, co in kinds_chans:
+        K = 9 * ci if kind == 1 else ci
+        layers.append(synth.LayerCfg(kind, K, co, float(co * H * Wd) / 2, 0.03 / (H * Wd), float(np.sqrt(co * H * Wd)),
+                                     H=H, Wd=Wd, Cin=ci))
+    return synth.Workload("mixed_conv", B, layers, (H, Wd, kinds_chans[0][1]), "normal", "kaiming_uniform", 2)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("stack,H,Wd,B", [
+    ([(1, 3, 64), (2, 64, 128), (1, 128, 64), (2, 64, 48)], 32, 32, 2),   # 3x3 and pointwise layers alternating
+    ([(2, 16, 32), (2, 32, 20)], 8, 16, 3),                                # narrow pointwise layers, ragged Cout
+    ([(2, 12, 10)], 4, 12, 5)])                                            # Cin not a multiple of 16: dp4a path
+def test_pointwise_convolution_layers(path, stack, H, Wd, B):
+    _run_and_compare(_mixed_conv_workload(stack, H, Wd, B), seed=51, steps=2, lam_per_step=0.2, path=path)

@@ -552,3 +552,52 @@ def test_int8_ff_training_learns_and_predicts_separable_classes():
         X = np.concatenate([embed(base, lab), embed(base, wrong)])
         Ws = [st.W_new for st in O.train_step(specs, Ws, X, B, 0.0, step)]
     assert accuracy(Ws) > 0.9
+
+
+# --------------------------------------------------------------------------------------
+# Pointwise convolution
+# --------------------------------------------------------------------------------------
+def test_conv1x1_equals_centre_tap_of_conv3x3():
+    """A 1x1 convolution is a 3x3 convolution whose only non-zero tap is the centre one: the whole train
+    step of the pointwise layer must reproduce the (brute-force-pinned) 3x3 layer with embedded weights,
+    and its weight gradient must equal the centre tap of the 3x3 one."""
+    g = np.random.default_rng(11)
+    B, H, Wd, Cin, N = 2, 5, 6, 7, 9
+    X = g.normal(size=(2 * B, H, Wd, Cin)).astype(F32)
+    W1 = g.normal(size=(N, Cin)).astype(F32) * 0.3
+    W3 = np.zeros((N, 3, 3, Cin), dtype=F32)
+    W3[:, 1, 1, :] = W1
+    theta, tau = float(N * H * Wd) / 2, float(np.sqrt(N * H * Wd))
+    s1 = O.LayerSpec(O.KIND_CONV1X1, Cin, N, theta, 0.05, tau, H=H, Wd=Wd, Cin=Cin, seed=4)
+    s3 = O.LayerSpec(O.KIND_CONV3X3, 9 * Cin, N, theta, 0.05, tau, H=H, Wd=Wd, Cin=Cin, seed=4)
+    a = O.train_step([s1], [W1], X, B, 0.0, 5)[0]
+    b = O.train_step([s3], [W3.reshape(N, -1)], X, B, 0.0, 5)[0]
+    assert np.array_equal(a.Xq, b.Xq) and a.a_w == b.a_w
+    assert np.array_equal(a.Wq, b.Wq.reshape(N, 3, 3, Cin)[:, 1, 1, :])
+    assert np.array_equal(a.acc, b.acc) and np.array_equal(a.Y, b.Y) and np.array_equal(a.G, b.G)
+    assert np.array_equal(a.coef, b.coef) and np.array_equal(a.dHq, b.dHq) and a.loss == b.loss
+    assert np.array_equal(a.accW, b.accW.reshape(2, N, 3, 3, Cin)[:, :, 1, 1, :])
+    assert np.array_equal(a.W_new, b.W_new.reshape(N, 3, 3, Cin)[:, 1, 1, :])
+    assert a.Y.shape == (2 * B, H, Wd, N) and s1.rows_per_sample == H * Wd
+
+
+def test_conv1x1_gradient_matches_finite_differences():
+    g = np.random.default_rng(12)
+    B, H, Wd, Cin, N = 2, 3, 3, 4, 5
+    X = g.normal(size=(2 * B, H, Wd, Cin))
+    W = g.normal(size=(N, Cin)) * 0.4
+    spec = O.LayerSpec(O.KIND_CONV1X1, Cin, N, float(N * H * Wd) / 2, 0.0, 1.0, H=H, Wd=Wd, Cin=Cin)
+    # analytic dL/dW of the unquantised layer: dH = 2*coef*Y with coef = dL/dG / (2B), dW = dH^T X over positions
+    Y = np.maximum(X @ W.T, 0.0)
+    G = (Y.reshape(2 * B, -1) ** 2).sum(1)
+    _, gp = O.ff_loss_terms(G.astype(F32), spec.theta, B)
+    coef = gp / (2 * B)
+    dH = 2.0 * coef[:, None, None, None] * Y
+    dW = dH.reshape(-1, N).T @ X.reshape(-1, Cin)
+    eps = 1e-6
+    for (n, k) in [(0, 0), (2, 3), (4, 1)]:
+        Wp, Wm = W.copy(), W.copy()
+        Wp[n, k] += eps
+        Wm[n, k] -= eps
+        fd = (O.fp64_layer_loss(spec, X, Wp, B) - O.fp64_layer_loss(spec, X, Wm, B)) / (2 * eps)
+        assert abs(fd - dW[n, k]) <= 1e-4 * max(1.0, abs(fd)), (n, k, fd, dW[n, k])
