@@ -264,7 +264,17 @@ __device__ __forceinline__ void tc_ld32_async(uint32_t taddr, int (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Waits for this thread's outstanding TMEM loads.  The loaded registers are passed through as read-write
+// operands so that the compiler cannot schedule a use of them above the wait.
+__device__ __forceinline__ void tc_wait_ld(int (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                 "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                 "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
 // TMA store of one staged box to global memory (clipped at the tensor's edge), bulk async-group completion.
 // `policy`: an L2 eviction policy (l2_policy_evict_first: the stored lines are the first to leave L2, so a
 // stream of output written once does not push the operand panels out).
@@ -618,7 +628,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 #pragma unroll
         for (int i = 0; i < TC_EPI_COLS / 32; ++i) {
           const int cb = cbeg + i * 32;
-          tc_wait_ld();
+          if (cb < cend) tc_wait_ld(v[i & 1]);
           if (i + 1 < TC_EPI_COLS / 32 && cb + 32 < cend) tc_ld32_async(t_row + as * TC_BN + cb + 32, v[(i + 1) & 1]);
           if (cb < cend) {  // uniform across the warp
             const int(&a)[32] = v[i & 1];
@@ -733,7 +743,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           int vp[32], vn[32];
           tc_ld32_async(t_row + cb, vp);
           tc_ld32_async(t_row + TC_BN + cb, vn);
-          tc_wait_ld();
+          tc_wait_ld(vp);
+          tc_wait_ld(vn);
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             float d[4];
