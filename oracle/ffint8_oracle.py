@@ -261,7 +261,7 @@ def goodness(acc: np.ndarray, c_rows: np.ndarray):
 
 def length_normalise(y: np.ndarray, G: np.ndarray, tau: float, eps: float) -> np.ndarray:
     """Next layer's input x = y * tau/(||y|| + eps) with ||y|| = sqrt(G) (FF length
-    normalisation; the paper is silent, the benchmark spec asks for it).  One sqrt, one add,
+    normalisation of Forward-Forward, Hinton 2022; the paper itself is silent on it).  One sqrt, one add,
     one divide per sample; one multiply per element."""
     r = F32(tau) / (np.sqrt(G.astype(F32)) + F32(eps))
     return y * r.reshape((-1,) + (1,) * (y.ndim - 1)).astype(F32)

@@ -55,7 +55,7 @@ def _mlp(widths, theta=None, lr=0.03):
 
 
 def workload(name: str) -> Workload:
-    """The five configurations of the benchmark spec (sizes only; data are drawn by make_*)."""
+    """The five benchmark configurations (sizes only; data are drawn by make_*)."""
     if name == "tiny_mlp":          # config 1
         return Workload(name, 64, _mlp([784, 500, 500]), (784,), "uniform01", "kaiming_uniform", 10)
     if name == "mlp_greedy":        # config 2

@@ -8,7 +8,7 @@ import numpy as np
 from oracle import ffint8_oracle as O
 from paper_2506_22771_b200 import binding as ffb
 
-REL_TOL = 1e-5   # tolerance of the benchmark spec for FP32 goodness / loss / weights
+REL_TOL = 1e-5   # relative tolerance for order-dependent FP32 scalars (the loss value)
 
 
 def specs_and_descs(layers, seed, round_x=1, round_w=0, round_dh=1):

@@ -1,6 +1,6 @@
 #!/usr/bin/env python
 """Writes tests/golden/fullsize_digests.json: SHA-256 digests of every tensor the CPU oracle produces
-for train steps at the FULL sizes of the task's configurations (the sizes bench.py times).
+for train steps at the FULL sizes of the five benchmark configurations (the sizes bench.py times).
 
 Calls only oracle/ and the seeded input generators; nothing here comes from the CUDA path.  The GPU
 test tests/test_gpu_fullsize.py recomputes the same digests from the device buffers, so a full-size

@@ -1,4 +1,4 @@
-"""Full-size parity: the CUDA path at the task's full configuration sizes, in the launch configuration
+"""Full-size parity: the CUDA path at the full sizes of the five benchmark configurations, in the launch configuration
 bench.py times (no parity dumps, no FP32 copy of the normalised output, layers chained on device),
 against SHA-256 digests of the CPU oracle's tensors (tests/golden/fullsize_digests.json, written by
 tests/golden/make_fullsize_digests.py from oracle/ alone).  Every INT8 tensor, accumulator statistic

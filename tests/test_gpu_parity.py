@@ -1,6 +1,6 @@
 """GPU parity tests: the CUDA path (through the C ABI) against the CPU oracle, element by element.
 Bit-exact for INT8 / INT32 / index work and, by the arithmetic contract, for every FP32 state
-tensor too (which is tighter than the 1e-5 relative tolerance the task allows); the loss scalar
+tensor too (tighter than a 1e-5 relative tolerance would be); the loss scalar
 is compared at 1e-5 relative."""
 import numpy as np
 import pytest
