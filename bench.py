@@ -161,8 +161,8 @@ def algorithmic_work(w, B: int):
 def _oracle_step_time(w, B_sample: int, steps: int, seed: int = 1):
     """Time the CPU oracle, as it stands, on a bounded sample (B_sample positives + negatives)."""
     from oracle import ffint8_oracle as O
-    specs = [O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, l.eps, l.H, l.Wd, l.Cin, seed=seed, index=i)
-             for i, l in enumerate(w.layers)]
+    specs = [O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, l.eps, l.H, l.Wd, l.Cin, seed=seed, index=i,
+                         stride=l.stride) for i, l in enumerate(w.layers)]
     Ws = synth.make_weights(w, seed)
     X = synth.make_batch(w, seed, B=B_sample)
     times = []

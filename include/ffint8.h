@@ -15,8 +15,8 @@
  *    aligned, valid on the device the context was created for.  Pointers to ff_layer_desc /
  *    ff_layer_bufs structs and all by-value scalars are HOST data.
  *  - Batch layout: B positive samples followed by B negative samples ("positive and negative
- *    sets", Alg. 1 line 3).  M = 2B.  R = rows per sample: 1 for a linear layer, H*Wd for a
- *    convolution (one row per output position, NHWC).
+ *    sets", Alg. 1 line 3).  M = 2B.  R = rows per sample: 1 for a linear layer, Ho*Wo for a
+ *    convolution (one row per output position, NHWC); the input of a convolution has H*Wd rows.
  *  - Calls are asynchronous on the given CUDA stream (a cudaStream_t passed as void*; NULL =
  *    the legacy default stream) and never synchronise.  Host-detectable errors are returned
  *    before anything is launched.  Device-detected conditions (non-finite input, a bounded wait
@@ -66,8 +66,8 @@ enum {
 };
 
 /* One FF layer (host struct).  linear: X[M,K] -> Y[M,N], W[N,K].
- * conv3x3 (stride 1, zero padding 1, NHWC): X[M,H,Wd,Cin] -> Y[M,H,Wd,N], W[N,3,3,Cin] stored as
- * [N,K] with K = 9*Cin and k = (r*3+s)*Cin + ci.
+ * conv3x3 (stride 1 or 2, zero padding 1, NHWC): X[M,H,Wd,Cin] -> Y[M,Ho,Wo,N], W[N,3,3,Cin] stored
+ * as [N,K] with K = 9*Cin and k = (r*3+s)*Cin + ci; Ho = H, Wo = Wd at stride 1.
  * conv1x1 (pointwise, NHWC): X[M,H,Wd,Cin] -> Y[M,H,Wd,N], W[N,Cin], K = Cin: the dense MAC applied
  * at every position; goodness and normalisation over all H*Wd*N values of a sample. */
 typedef struct {
@@ -80,18 +80,22 @@ typedef struct {
   float lr;             /* SGD step size of the update (Alg. 1 line 9)                        */
   float tau, eps;       /* length normalisation of the output: x = y*tau/(sqrt(G)+eps), eps>0 */
   uint64_t seed;        /* keys the stochastic-rounding hash                                  */
+  int32_t stride;       /* conv3x3 only: 0 or 1 = every position, 2 = every second row and column; */
+                        /* the output then has Ho = (H-1)/2 + 1 rows of Wo = (Wd-1)/2 + 1 positions */
+  int32_t reserved;     /* zero                                                                */
 } ff_layer_desc;
 
 /* Device buffers of one layer (host struct of device pointers; caller-owned). */
 typedef struct {
   float* W;          /* [N,K] FP32 master weights; ff_layer_update rewrites them in place      */
-  const float* X;    /* [M*R,Kin] FP32 input, already length-normalised (Kin = K, conv: Cin).   */
+  const float* X;    /* [M*Rin,Kin] FP32 input, already length-normalised (Kin = K, conv: Cin;  */
+                     /* Rin = input rows per sample: 1, conv: H*Wd).                            */
                      /* In ff_train_step it may be NULL for layers > 0: the layer then takes   */
                      /* the previous layer's normalised output without materialising it.      */
   float* Y;          /* [M*R,N] FP32 out: max(0, float(acc)*s_x*s_w)                           */
   float* G;          /* [M] FP32 out: goodness per sample                                      */
   float* Xnext;      /* [M*R,N] FP32 out, nullable: Y*tau/(sqrt(G)+eps)                         */
-  int8_t* Xq;        /* [M*R,Kin] INT8 out                                                     */
+  int8_t* Xq;        /* [M*Rin,Kin] INT8 out                                                   */
   int8_t* Wq;        /* [N,K] INT8 out                                                         */
   int8_t* dHq;       /* [M*R,N] INT8 out (ff_layer_loss_grad)                                  */
   float* absmax;     /* [FF_ABSMAX_LEN] FP32 out, see FF_A_*                                   */

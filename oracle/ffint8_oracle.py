@@ -68,10 +68,21 @@ class LayerSpec:
     round_dh: int = ROUND_STOCHASTIC
     seed: int = 0
     index: int = 0        # position of the layer in the network (feeds the rounding hash)
+    stride: int = 1       # conv3x3 only: 1 or 2 (output (H-1)//stride + 1 by (Wd-1)//stride + 1)
+
+    @property
+    def out_hw(self):
+        if self.kind == KIND_CONV3X3:
+            return (self.H - 1) // self.stride + 1, (self.Wd - 1) // self.stride + 1
+        return self.H, self.Wd
 
     @property
     def rows_per_sample(self) -> int:
-        return self.H * self.Wd if self.kind != KIND_LINEAR else 1
+        """Output positions per sample."""
+        if self.kind == KIND_LINEAR:
+            return 1
+        ho, wo = self.out_hw
+        return ho * wo
 
 
 # --------------------------------------------------------------------------------------
@@ -203,31 +214,32 @@ def _pad_hw(xq: np.ndarray) -> np.ndarray:
     return np.pad(xq, ((0, 0), (1, 1), (1, 1), (0, 0)))
 
 
-def int8_conv3x3(xq: np.ndarray, wq: np.ndarray) -> np.ndarray:
-    """acc[b,h,w,co] = sum_{r,s,ci} xq[b,h+r-1,w+s-1,ci]*wq[co,r,s,ci], zero padding
+def int8_conv3x3(xq: np.ndarray, wq: np.ndarray, stride: int = 1) -> np.ndarray:
+    """acc[b,i,j,co] = sum_{r,s,ci} xq[b,stride*i+r-1,stride*j+s-1,ci]*wq[co,r,s,ci], zero padding 1
     ('dense or convolution layers', Sec. IV-B).  xq NHWC int8, wq [Cout,3,3,Cin] int8."""
     Bn, H, Wd, Cin = xq.shape
     Cout = wq.shape[0]
+    Ho, Wo = (H - 1) // stride + 1, (Wd - 1) // stride + 1
     xp = _pad_hw(xq)
-    acc = np.zeros((Bn * H * Wd, Cout), dtype=F64)
+    acc = np.zeros((Bn * Ho * Wo, Cout), dtype=F64)
     for r in range(3):
         for s in range(3):
-            win = xp[:, r:r + H, s:s + Wd, :].reshape(-1, Cin)
+            win = xp[:, r:r + stride * (Ho - 1) + 1:stride, s:s + stride * (Wo - 1) + 1:stride, :].reshape(-1, Cin)
             acc += _matmul_exact(win, wq[:, r, s, :].T)
-    return _check_i32(acc).reshape(Bn, H, Wd, Cout)
+    return _check_i32(acc).reshape(Bn, Ho, Wo, Cout)
 
 
-def int8_conv3x3_wgrad(dhq: np.ndarray, xq: np.ndarray) -> np.ndarray:
-    """accW[co,r,s,ci] = sum_{b,h,w} dhq[b,h,w,co]*xq[b,h+r-1,w+s-1,ci] (weight gradient of the
-    convolution above; there is no input gradient in FF, Sec. IV-B)."""
+def int8_conv3x3_wgrad(dhq: np.ndarray, xq: np.ndarray, stride: int = 1) -> np.ndarray:
+    """accW[co,r,s,ci] = sum_{b,i,j} dhq[b,i,j,co]*xq[b,stride*i+r-1,stride*j+s-1,ci] (weight gradient of
+    the convolution above; there is no input gradient in FF, Sec. IV-B)."""
     Bn, H, Wd, Cin = xq.shape
-    Cout = dhq.shape[-1]
+    _, Ho, Wo, Cout = dhq.shape
     xp = _pad_hw(xq)
     d2 = dhq.reshape(-1, Cout)
     out = np.empty((Cout, 3, 3, Cin), dtype=np.int32)
     for r in range(3):
         for s in range(3):
-            win = xp[:, r:r + H, s:s + Wd, :].reshape(-1, Cin)
+            win = xp[:, r:r + stride * (Ho - 1) + 1:stride, s:s + stride * (Wo - 1) + 1:stride, :].reshape(-1, Cin)
             out[:, r, s, :] = _check_i32(_matmul_exact(d2.T, win))
     return out
 
@@ -382,7 +394,7 @@ def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: i
         # pointwise convolution: the dense MAC applied at every position ('dense or convolution layers', Sec. IV-B)
         st.acc = int8_gemm_nt(st.Xq.reshape(-1, spec.K), st.Wq).reshape(st.Xq.shape[:3] + (spec.N,))
     else:
-        st.acc = int8_conv3x3(st.Xq, st.Wq.reshape(spec.N, 3, 3, spec.Cin))
+        st.acc = int8_conv3x3(st.Xq, st.Wq.reshape(spec.N, 3, 3, spec.Cin), spec.stride)
     s_w, _ = scale_pair(st.a_w)
     c_rows = _pass_rows(scale_pair(st.a_x[0])[0] * s_w, scale_pair(st.a_x[1])[0] * s_w, B)
     st.Y = dequant_relu(st.acc, c_rows)
@@ -415,7 +427,7 @@ def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int) -> Laye
         elif spec.kind == KIND_CONV1X1:
             accW.append(int8_gemm_tn(st.dHq[sl].reshape(-1, spec.N), st.Xq[sl].reshape(-1, spec.K)))
         else:
-            accW.append(int8_conv3x3_wgrad(st.dHq[sl], st.Xq[sl]).reshape(spec.N, spec.K))
+            accW.append(int8_conv3x3_wgrad(st.dHq[sl], st.Xq[sl], spec.stride).reshape(spec.N, spec.K))
     st.accW = np.stack(accW)
     cP = scale_pair(st.a_dh[0])[0] * scale_pair(st.a_x[0])[0]
     cN = scale_pair(st.a_dh[1])[0] * scale_pair(st.a_x[1])[0]
@@ -487,10 +499,12 @@ def fp64_layer_loss(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int) -> fl
     else:
         xp = np.pad(X, ((0, 0), (1, 1), (1, 1), (0, 0)))
         w4 = W.reshape(spec.N, 3, 3, spec.Cin)
-        Y = np.zeros(X.shape[:3] + (spec.N,))
+        Ho, Wo = spec.out_hw
+        st = spec.stride
+        Y = np.zeros((X.shape[0], Ho, Wo, spec.N))
         for r in range(3):
             for s in range(3):
-                Y += xp[:, r:r + spec.H, s:s + spec.Wd, :] @ w4[:, r, s, :].T
+                Y += xp[:, r:r + st * (Ho - 1) + 1:st, s:s + st * (Wo - 1) + 1:st, :] @ w4[:, r, s, :].T
         Y = np.maximum(Y, 0.0)
     G = (Y.reshape(2 * B, -1) ** 2).sum(axis=1)
     z = G - spec.theta

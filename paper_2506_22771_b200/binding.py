@@ -32,7 +32,7 @@ class ff_layer_desc(C.Structure):
                 ("Wd", C.c_int32), ("Cin", C.c_int32), ("index", C.c_int32),
                 ("round_x", C.c_int32), ("round_w", C.c_int32), ("round_dh", C.c_int32),
                 ("theta", C.c_float), ("lr", C.c_float), ("tau", C.c_float), ("eps", C.c_float),
-                ("seed", C.c_uint64)]
+                ("seed", C.c_uint64), ("stride", C.c_int32), ("reserved", C.c_int32)]
 
 
 class ff_layer_bufs(C.Structure):
@@ -205,7 +205,7 @@ def make_desc(cfg, index: int, seed: int, round_x=FF_ROUND_STOCHASTIC, round_w=F
               round_dh=FF_ROUND_STOCHASTIC) -> ff_layer_desc:
     """cfg: an object with kind, K, N, H, Wd, Cin, theta, lr, tau, eps (e.g. synth.LayerCfg)."""
     return ff_layer_desc(cfg.kind, cfg.K, cfg.N, cfg.H, cfg.Wd, cfg.Cin, index, round_x, round_w, round_dh,
-                         cfg.theta, cfg.lr, cfg.tau, cfg.eps, seed)
+                         cfg.theta, cfg.lr, cfg.tau, cfg.eps, seed, getattr(cfg, "stride", 1), 0)
 
 
 class LayerBuffers:
@@ -214,16 +214,18 @@ class LayerBuffers:
     def __init__(self, desc: ff_layer_desc, B: int, device, dumps: bool = False, xnext: bool = True,
                  own_x: bool = True):
         import torch
-        R = desc.H * desc.Wd if desc.kind != FF_LINEAR else 1
+        st = 2 if (desc.kind == FF_CONV3X3 and desc.stride == 2) else 1
+        Rin = desc.H * desc.Wd if desc.kind != FF_LINEAR else 1                    # input rows per sample
+        R = ((desc.H - 1) // st + 1) * ((desc.Wd - 1) // st + 1) if desc.kind != FF_LINEAR else 1   # output rows
         kin = desc.Cin if desc.kind != FF_LINEAR else desc.K
-        rows = 2 * B * R
+        rows, rows_in = 2 * B * R, 2 * B * Rin
         z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)
         self.W = z((desc.N, desc.K), torch.float32)
-        self.X = z((rows, kin), torch.float32) if own_x else None
+        self.X = z((rows_in, kin), torch.float32) if own_x else None
         self.Y = z((rows, desc.N), torch.float32)
         self.G = z((2 * B,), torch.float32)
         self.Xnext = z((rows, desc.N), torch.float32) if xnext else None
-        self.Xq = z((rows, kin), torch.int8)
+        self.Xq = z((rows_in, kin), torch.int8)
         self.Wq = z((desc.N, desc.K), torch.int8)
         self.dHq = z((rows, desc.N), torch.int8)
         self.absmax = z((FF_ABSMAX_LEN,), torch.float32)

@@ -97,7 +97,9 @@ struct ProfScope {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-inline int rows_per_sample(const ff_layer_desc& L) { return L.kind != FF_LINEAR ? L.H * L.Wd : 1; }
+// output rows (positions) per sample, and input rows per sample (they differ for a strided convolution)
+inline int rows_per_sample(const ff_layer_desc& L) { return L.kind != FF_LINEAR ? tc_out_h(L) * tc_out_w(L) : 1; }
+inline int in_rows_per_sample(const ff_layer_desc& L) { return L.kind != FF_LINEAR ? L.H * L.Wd : 1; }
 inline int in_features(const ff_layer_desc& L) { return L.kind == FF_CONV3X3 ? L.Cin : L.K; }
 
 ff_status check_layer(ff_ctx* ctx, const ff_layer_desc* L, int B) {
@@ -109,13 +111,16 @@ ff_status check_layer(ff_ctx* ctx, const ff_layer_desc* L, int B) {
   if (L->K <= 0 || L->N <= 0) return fail(ctx, FF_ERR_ARG, "K and N must be positive");
   if (L->kind == FF_CONV3X3 && (L->H <= 0 || L->Wd <= 0 || L->Cin <= 0 || L->K != 9 * L->Cin))
     return fail(ctx, FF_ERR_ARG, "conv3x3 needs H, Wd, Cin > 0 and K = 9*Cin");
+  if (L->stride < 0 || L->stride > 2 || (L->stride == 2 && L->kind != FF_CONV3X3))
+    return fail(ctx, FF_ERR_ARG, "stride must be 0 / 1, or 2 for a conv3x3 layer");
   for (int r : {L->round_x, L->round_w, L->round_dh})
     if (r != FF_ROUND_NEAREST_EVEN && r != FF_ROUND_STOCHASTIC) return fail(ctx, FF_ERR_ARG, "unknown rounding mode");
   if (!(L->eps > 0.0f)) return fail(ctx, FF_ERR_ARG, "eps must be > 0");
   const long long R = rows_per_sample(*L);
   const long long rows = 2LL * B * R;
   // 32-bit rounding counters and element indices
-  if (rows * L->N >= (1LL << 32) || rows * in_features(*L) >= (1LL << 32) || (long long)L->N * L->K >= (1LL << 32))
+  const long long rows_in = 2LL * B * in_rows_per_sample(*L);
+  if (rows * L->N >= (1LL << 32) || rows_in * in_features(*L) >= (1LL << 32) || (long long)L->N * L->K >= (1LL << 32))
     return fail(ctx, FF_ERR_RANGE, "tensor has 2^32 or more elements");
   if (rows >= (1LL << 31)) return fail(ctx, FF_ERR_RANGE, "too many rows");
   // worst-case INT32 accumulator range: 127*127*contraction length < 2^31  (Sec. IV-B: INT32 accumulation)
@@ -179,8 +184,8 @@ inline DenseView dense(const int8_t* p, int rows, int cols) {
   return DenseView{p, rows, cols, (cols % 8 == 0) && ((reinterpret_cast<uintptr_t>(p) & 7) == 0)};
 }
 inline Im2colView im2col(const int8_t* p, const ff_layer_desc& L, int samples) {
-  return Im2colView{p, samples * L.H * L.Wd, 9 * L.Cin, L.H, L.Wd, L.Cin,
-                    (L.Cin % 8 == 0) && ((reinterpret_cast<uintptr_t>(p) & 7) == 0)};
+  return Im2colView{p, samples * tc_out_h(L) * tc_out_w(L), 9 * L.Cin, L.H, L.Wd, L.Cin, tc_out_h(L), tc_out_w(L),
+                    tc_conv_stride(L), (L.Cin % 8 == 0) && ((reinterpret_cast<uintptr_t>(p) & 7) == 0)};
 }
 
 // ---- split weight gradient ------------------------------------------------------------------
@@ -228,12 +233,12 @@ inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 inline Im2colPlan im2col_plan(const ff_layer_desc& L, int B, size_t ws_bytes, int sm_count) {
   Im2colPlan pl;
   pl.kpad = tc_im2col_kpad(L);
-  const size_t rows = (size_t)2 * B * L.H * L.Wd;
+  const size_t rows = (size_t)2 * B * tc_out_h(L) * tc_out_w(L);
   pl.xi_off = WS_BYTES;
   pl.wi_off = pl.xi_off + up256(rows * pl.kpad);
   pl.slab_off = pl.wi_off + up256((size_t)L.N * pl.kpad);
   pl.slab_bytes_per_split = (size_t)2 * L.N * pl.kpad * sizeof(int32_t);
-  const int wish = tc_dense_slab_splits(L.N, pl.kpad, (long long)B * L.H * L.Wd, sm_count);
+  const int wish = tc_dense_slab_splits(L.N, pl.kpad, (long long)B * tc_out_h(L) * tc_out_w(L), sm_count);
   const size_t room = ws_bytes > pl.slab_off ? ws_bytes - pl.slab_off : 0;
   const size_t fit = room / pl.slab_bytes_per_split;
   pl.max_splits = ws_bytes < pl.slab_off ? -1 : (int)(fit < (size_t)wish ? fit : (size_t)wish);
@@ -248,15 +253,16 @@ ff_status launch_im2col(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs
                         cudaStream_t st) {
   char* ws = static_cast<char*>(ctx->workspace);
   int8_t* xi = reinterpret_cast<int8_t*>(ws + pl.xi_off);
-  const int rows = 2 * B * L.H * L.Wd;
+  const int Ho = tc_out_h(L), Wo = tc_out_w(L), sd = tc_conv_stride(L);
+  const int rows = 2 * B * Ho * Wo;
   const int blocks = (rows + 255) / 256;
   switch (pl.kpad) {
-    case 16: im2col3x3_kernel<16><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
-    case 32: im2col3x3_kernel<32><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
-    case 48: im2col3x3_kernel<48><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
-    case 64: im2col3x3_kernel<64><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
-    case 96: im2col3x3_kernel<96><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
-    default: im2col3x3_kernel<128><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin); break;
+    case 16: im2col3x3_kernel<16><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin, Ho, Wo, sd); break;
+    case 32: im2col3x3_kernel<32><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin, Ho, Wo, sd); break;
+    case 48: im2col3x3_kernel<48><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin, Ho, Wo, sd); break;
+    case 64: im2col3x3_kernel<64><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin, Ho, Wo, sd); break;
+    case 96: im2col3x3_kernel<96><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin, Ho, Wo, sd); break;
+    default: im2col3x3_kernel<128><<<blocks, 256, 0, st>>>(b.Xq, xi, rows, L.H, L.Wd, L.Cin, Ho, Wo, sd); break;
   }
   FF_LAUNCH_CHECK(ctx);
   if (weights) {
@@ -440,7 +446,7 @@ ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
 }
 
 ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint64_t step, cudaStream_t st) {
-  const size_t per_pass = (size_t)B * rows_per_sample(L) * in_features(L);
+  const size_t per_pass = (size_t)B * in_rows_per_sample(L) * in_features(L);
   {
     ProfScope prof(ctx, FF_K_ABSMAX, st);
     absmax_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(b.X, per_pass, b.absmax + FF_A_X_POS,
@@ -522,7 +528,7 @@ ff_status check_layer_list(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
     if ((s = check_bufs(ctx, &bufs[l], l == 0)) != FF_OK) return s;
     if (l > 0 && !bufs[l].X) {
       const ff_layer_desc &p = layers[l - 1], &c = layers[l];
-      if ((long long)rows_per_sample(p) * p.N != (long long)rows_per_sample(c) * in_features(c))
+      if ((long long)rows_per_sample(p) * p.N != (long long)in_rows_per_sample(c) * in_features(c))
         return fail(ctx, FF_ERR_ARG, "layer output / next layer input sizes differ");
     }
   }

@@ -32,12 +32,13 @@ struct DenseView {
     }
   }
 };
-// im2col view of an NHWC INT8 tensor for a 3x3 / stride 1 / pad 1 convolution:
-// row = (b*H + h)*W + w, col = (r*3 + s)*Cin + ci  ->  x[b, h+r-1, w+s-1, ci].
+// im2col view of an NHWC INT8 tensor for a 3x3 / pad 1 convolution of stride 1 or 2:
+// row = (b*Ho + i)*Wo + j, col = (r*3 + s)*Cin + ci  ->  x[b, stride*i+r-1, stride*j+s-1, ci].
 struct Im2colView {
   const int8_t* p;
-  int rows, cols;  // rows = Bn*H*W, cols = 9*Cin
-  int H, W, Cin;
+  int rows, cols;  // rows = Bn*Ho*Wo, cols = 9*Cin
+  int H, W, Cin;   // input geometry
+  int Ho, Wo, stride;
   bool vec8;  // Cin % 8 == 0 and p 8-byte aligned
   __device__ __forceinline__ void load8(int row, int col0, int8_t* out) const {
     if (row >= rows) {
@@ -45,8 +46,10 @@ struct Im2colView {
       for (int i = 0; i < 8; ++i) out[i] = 0;
       return;
     }
-    int w = row % W, t = row / W;
-    int h = t % H, b = t / H;
+    int w = row % Wo, t = row / Wo;
+    int h = t % Ho, b = t / Ho;
+    w *= stride;
+    h *= stride;
     if (vec8 && col0 + 8 <= cols) {
       int tap = col0 / Cin, ci = col0 - tap * Cin;
       int hh = h + tap / 3 - 1, ww = w + tap % 3 - 1;
@@ -232,11 +235,12 @@ __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restr
 // dense tensor-core kernels.  One thread per output position.
 template <int KPAD>
 __global__ void __launch_bounds__(256) im2col3x3_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ out, int rows, int H,
-                                                        int W, int Cin) {
+                                                        int W, int Cin, int Ho, int Wo, int stride) {
   const int row = blockIdx.x * blockDim.x + threadIdx.x;
   if (row >= rows) return;
-  const int w = row % W, t = row / W;
-  const int h = t % H, b = t / H;
+  const int t = row / Wo;
+  const int w = (row - t * Wo) * stride;
+  const int h = (t % Ho) * stride, b = t / Ho;
   __align__(16) int8_t v[KPAD];
 #pragma unroll
   for (int i = 0; i < KPAD; ++i) v[i] = 0;

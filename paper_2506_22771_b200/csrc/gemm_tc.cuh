@@ -97,7 +97,9 @@ struct TcParams {
   int32_t* slabs;
   // convolution geometry (conv_W = 0: dense layer).  A 128-row block of positions is conv_TH image
   // rows of conv_W pixels; conv_cpt = channel chunks of CH bytes per filter tap; images per set.
-  int conv_W, conv_H, conv_TH, conv_cin, conv_cpt, conv_imgs_per_pass;
+  // conv_W / conv_H are the OUTPUT extents; the input box of an output position starts conv_stride
+  // input pixels further per output pixel (the tensor map steps through the input with that stride).
+  int conv_W, conv_H, conv_TH, conv_cin, conv_cpt, conv_imgs_per_pass, conv_stride;
 };
 
 // ---- PTX wrappers --------------------------------------------------------------------------
@@ -471,7 +473,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             if (!MN_MAJOR) {
               if (p.conv_W) {
                 // k-block = CH channels of one filter tap (r, s): the input box shifted by (r-1, s-1)
-                tma_load_4d<NCTA>(a_dst, &tmA, fb, f_cc * CH, f_s - 1, f_h0 + f_r - 1, f_img);
+                tma_load_4d<NCTA>(a_dst, &tmA, fb, f_cc * CH, f_s - 1, f_h0 * p.conv_stride + f_r - 1, f_img);
                 if (++f_cc == p.conv_cpt) {
                   f_cc = 0;
                   if (++f_s == 3) {
@@ -489,7 +491,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               if (p.conv_W) {
                 // contraction block kb of set `pass` = conv_TH rows of one image; B column chunk q of the
                 // tile = CH channels of one filter tap, fetched from the shifted input box
-                const int h0 = g_blk * p.conv_TH;
+                const int h0 = g_blk * p.conv_TH * p.conv_stride;
 #pragma unroll
                 for (int q = 0; q < G::B_BOXES; ++q)
                   if (col0 + q * CH < p.out_cols)
@@ -851,8 +853,10 @@ inline ff_status tc_init(TcState& t) {
 }
 
 inline ff_status tc_encode(TcState& t, CUtensorMap* tm, const int8_t* base, cuuint32_t rank, const cuuint64_t* dims,
-                           const cuuint64_t* strides, const cuuint32_t* box, int swizzle_bytes) {
-  cuuint32_t estr[4] = {1, 1, 1, 1};
+                           const cuuint64_t* strides, const cuuint32_t* box, int swizzle_bytes,
+                           const cuuint32_t* element_strides = nullptr) {
+  cuuint32_t ones[4] = {1, 1, 1, 1};
+  const cuuint32_t* estr = element_strides ? element_strides : ones;
   CUresult r = t.encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, rank, const_cast<int8_t*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -873,14 +877,20 @@ inline ff_status tc_make_map(TcState& t, CUtensorMap* tm, const int8_t* base, ui
   cuuint32_t box[3] = {box_cols, box_rows, 1};
   return tc_encode(t, tm, base, passes > 0 ? 3 : 2, dims, strides, box, (int)box_cols);
 }
-// NHWC INT8 tensor [imgs, H, W, C]; box = ch_box channels x W pixels x th rows x 1 image.
+// NHWC INT8 tensor [imgs, H, W, C] stepped through with `stride` pixels in both image directions;
+// one copy brings ch_box channels of wo x th positions of one image (the box spans stride times as
+// many input pixels).
 inline ff_status tc_make_map_nhwc(TcState& t, CUtensorMap* tm, const int8_t* base, uint64_t C, uint64_t W, uint64_t H, uint64_t imgs,
-                                  uint32_t ch_box, uint32_t th) {
+                                  uint32_t ch_box, uint32_t wo, uint32_t th, uint32_t stride) {
   cuuint64_t dims[4] = {C, W, H, imgs};
   cuuint64_t strides[3] = {C, C * W, C * W * H};
-  cuuint32_t box[4] = {ch_box, (cuuint32_t)W, th, 1};
-  return tc_encode(t, tm, base, 4, dims, strides, box, (int)ch_box);
+  cuuint32_t box[4] = {ch_box, wo * stride, th * stride, 1};
+  cuuint32_t estr[4] = {1, stride, stride, 1};
+  return tc_encode(t, tm, base, 4, dims, strides, box, (int)ch_box, estr);
 }
+inline int tc_conv_stride(const ff_layer_desc& L) { return (L.kind == FF_CONV3X3 && L.stride == 2) ? 2 : 1; }
+inline int tc_out_h(const ff_layer_desc& L) { return (L.H - 1) / tc_conv_stride(L) + 1; }
+inline int tc_out_w(const ff_layer_desc& L) { return (L.Wd - 1) / tc_conv_stride(L) + 1; }
 
 inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
 
@@ -978,17 +988,17 @@ inline bool tc_gemm_supported(int M, int N, int K, int trans) { return trans ? t
 // width a power of two up to 128 so that 128 consecutive output positions are whole image rows.
 inline bool tc_conv_ok(const ff_layer_desc& L) {
   if (L.kind != FF_CONV3X3 || L.Cin % 64 != 0) return false;
-  const int W = L.Wd;
+  const int W = tc_out_w(L);   // 128 consecutive OUTPUT positions must be whole output rows
   if (W < 8 || W > 128 || (W & (W - 1)) != 0) return false;
-  return L.H % (128 / W) == 0;
+  return tc_out_h(L) % (128 / W) == 0;
 }
 inline bool tc_forward_supported(const ff_layer_desc& L, int B) {
   if (L.kind == FF_CONV3X3) return tc_conv_ok(L);
-  return tc_nt_ok(2LL * B * (L.kind == FF_LINEAR ? 1 : L.H * L.Wd), L.N, L.K);
+  return tc_nt_ok(2LL * B * (L.kind == FF_LINEAR ? 1 : tc_out_h(L) * tc_out_w(L)), L.N, L.K);
 }
 inline bool tc_update_supported(const ff_layer_desc& L, int B) {
   if (L.kind == FF_CONV3X3) return tc_conv_ok(L) && L.N % 16 == 0;
-  return tc_tn_ok(L.N, L.K, (long long)B * (L.kind == FF_LINEAR ? 1 : L.H * L.Wd));
+  return tc_tn_ok(L.N, L.K, (long long)B * (L.kind == FF_LINEAR ? 1 : tc_out_h(L) * tc_out_w(L)));
 }
 
 // Split count of the convolution weight gradient (its output N x 9*Cin has few tiles, its contraction
@@ -998,7 +1008,7 @@ inline int tc_conv_update_splits(const ff_layer_desc& L, int B, int sm_count, in
   if (sm_count <= 0) sm_count = 148;
   const int ncta = force_ncta ? force_ncta : (L.N > TC_BM ? 2 : 1);
   const long long tiles = (long long)cdiv(L.N, TC_BM * ncta) * cdiv(L.K, TC_BN);
-  const long long kblocks = (long long)B * L.H * L.Wd / 128;
+  const long long kblocks = (long long)B * tc_out_h(L) * tc_out_w(L) / 128;
   long long splits = (sm_count / ncta) / tiles;
   if (splits > kblocks / 8) splits = kblocks / 8;
   return splits < 1 ? 1 : (int)splits;
@@ -1047,7 +1057,7 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   ff_status s = tc_init(t);
   if (s != FF_OK) return s;
   const bool conv = L.kind == FF_CONV3X3 && !xi;
-  const int R = L.kind != FF_LINEAR ? L.H * L.Wd : 1;
+  const int R = L.kind != FF_LINEAR ? tc_out_h(L) * tc_out_w(L) : 1;
   const int M = 2 * B * R;
   const int K = xi ? kpad : L.K;
   const int8_t* A = xi ? xi : b.Xq;
@@ -1080,14 +1090,15 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
     return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st, typ);
   }
   const int ch = L.Cin % 128 == 0 ? 128 : 64;
-  p.conv_W = L.Wd;
-  p.conv_H = L.H;
-  p.conv_TH = 128 / L.Wd;
+  p.conv_W = tc_out_w(L);
+  p.conv_H = tc_out_h(L);
+  p.conv_TH = 128 / p.conv_W;
+  p.conv_stride = tc_conv_stride(L);
   p.conv_cin = L.Cin;
   p.conv_cpt = L.Cin / ch;
   p.conv_imgs_per_pass = B;
   p.kblocks = 9 * p.conv_cpt;
-  if ((s = tc_make_map_nhwc(t, &ta, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_TH)) != FF_OK) return s;
+  if ((s = tc_make_map_nhwc(t, &ta, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_W, p.conv_TH, p.conv_stride)) != FF_OK) return s;
   if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, ch, TC_BN / ncta)) != FF_OK) return s;
   if (ch == 128) return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st, typ);
   return tc_launch<TC_MODE_FWD, false, 64>(t, ncta, ta, tb, p, st, typ);
@@ -1123,7 +1134,7 @@ inline ff_status tc_conv_update(TcState& t, const ff_layer_desc& L, const ff_lay
   CUtensorMap ta, tb;
   TcParams p = {};
   const int ch = L.Cin % 128 == 0 ? 128 : 64;
-  const int pos_per_pass = B * L.H * L.Wd;
+  const int pos_per_pass = B * tc_out_h(L) * tc_out_w(L);
   p.out_rows = L.N;
   p.out_cols = L.K;
   p.kblocks = pos_per_pass / 128;
@@ -1131,9 +1142,10 @@ inline ff_status tc_conv_update(TcState& t, const ff_layer_desc& L, const ff_lay
   p.splits = splits;
   p.status = status;
   p.slabs = slabs;
-  p.conv_W = L.Wd;
-  p.conv_H = L.H;
-  p.conv_TH = 128 / L.Wd;
+  p.conv_W = tc_out_w(L);
+  p.conv_H = tc_out_h(L);
+  p.conv_TH = 128 / p.conv_W;
+  p.conv_stride = tc_conv_stride(L);
   p.conv_cin = L.Cin;
   p.conv_cpt = L.Cin / ch;
   p.conv_imgs_per_pass = B;
@@ -1141,7 +1153,7 @@ inline ff_status tc_conv_update(TcState& t, const ff_layer_desc& L, const ff_lay
   *splits_out = cdiv(p.kblocks, kb_per_split);
   const int ncta = t.force_ncta ? t.force_ncta : (L.N > TC_BM ? 2 : 1);
   if ((s = tc_make_map(t, &ta, b.dHq, L.N, pos_per_pass, 2, 128, 128)) != FF_OK) return s;
-  if ((s = tc_make_map_nhwc(t, &tb, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_TH)) != FF_OK) return s;
+  if ((s = tc_make_map_nhwc(t, &tb, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_W, p.conv_TH, p.conv_stride)) != FF_OK) return s;
   if (ch == 128) return tc_launch<TC_MODE_SLAB, true, 128>(t, ncta, ta, tb, p, st);
   return tc_launch<TC_MODE_SLAB, true, 64>(t, ncta, ta, tb, p, st);
 }

@@ -28,6 +28,7 @@ class LayerCfg:
     Wd: int = 1
     Cin: int = 0
     eps: float = 1e-8
+    stride: int = 1    # conv3x3 only
 
 
 @dataclass

@@ -15,7 +15,7 @@ def specs_and_descs(layers, seed, round_x=1, round_w=0, round_dh=1):
     specs, descs = [], []
     for i, l in enumerate(layers):
         specs.append(O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, l.eps, l.H, l.Wd, l.Cin,
-                                 round_x, round_w, round_dh, seed, i))
+                                 round_x, round_w, round_dh, seed, i, getattr(l, "stride", 1)))
         descs.append(ffb.make_desc(l, i, seed, round_x, round_w, round_dh))
     return specs, descs
 

@@ -23,8 +23,13 @@ from paper_2506_22771_b200 import synth        # noqa: E402
 
 OUT = os.path.join(os.path.dirname(os.path.abspath(__file__)), "fullsize_digests.json")
 SEED = 1
-# workload -> number of consecutive steps digested (weights carried from step to step)
-CASES = {"tiny_mlp": 10, "mlp_greedy": 2, "mlp_lookahead": 2, "cnn": 1, "roofline": 1}
+# workload -> number of consecutive steps run (weights carried from step to step).  Every step of a short
+# run is digested; of a long run the first two steps and every tenth (out["digested"] lists them).
+CASES = {"tiny_mlp": 10, "mlp_greedy": 3, "mlp_lookahead": 50, "cnn": 3, "roofline": 2}
+
+
+def digested_steps(steps: int):
+    return [s for s in range(steps) if steps <= 10 or s < 2 or s % 10 == 9]
 
 
 def digest(a) -> str:
@@ -47,7 +52,8 @@ def run(name: str, steps: int) -> dict:
              for i, l in enumerate(w.layers)]
     Ws = synth.make_weights(w, SEED)
     X = synth.make_batch(w, SEED)
-    out = {"B": w.B, "seed": SEED, "greedy": bool(w.greedy), "steps": []}
+    out = {"B": w.B, "seed": SEED, "greedy": bool(w.greedy), "n_steps": steps, "digested": digested_steps(steps),
+           "steps": []}
     if w.greedy:
         # layers trained one after another (Sec. III): phase l trains layer l alone on the INT8 forward of
         # the earlier layers; here every phase starts from the initial weights so that it can be checked on
@@ -69,7 +75,8 @@ def run(name: str, steps: int) -> dict:
     for step in range(steps):
         t0 = time.time()
         states = O.train_step(specs, Ws, X, w.B, w.lam_per_step * step, step)
-        out["steps"].append([layer_digests(st, w.B) for st in states])
+        if step in out["digested"]:
+            out["steps"].append([layer_digests(st, w.B) for st in states])
         Ws = [st.W_new for st in states]
         print(f"{name} step {step}: {time.time() - t0:.1f} s", flush=True)
     return out

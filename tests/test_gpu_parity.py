@@ -294,12 +294,18 @@ def test_dead_layer_and_vanishing_gradient():
 
 
 def _mixed_conv_workload(kinds_chans, H, Wd, B):
-    """kinds_chans: list of (kind, Cin, Cout); kind 1 = 3x3, 2 = pointwise."""
+    """kinds_chans: list of (kind, Cin, Cout[, stride]); kind 1 = 3x3, 2 = pointwise.  A stride-2 layer
+    halves the image for the layers after it."""
     layers = []
-    for kind, ci, co in kinds_chans:
+    h, w_ = H, Wd
+    for spec in kinds_chans:
+        kind, ci, co = spec[:3]
+        stride = spec[3] if len(spec) > 3 else 1
         K = 9 * ci if kind == 1 else ci
-        layers.append(synth.LayerCfg(kind, K, co, float(co * H * Wd) / 2, 0.03 / (H * Wd), float(np.sqrt(co * H * Wd)),
-                                     H=H, Wd=Wd, Cin=ci))
+        ho, wo = ((h - 1) // stride + 1, (w_ - 1) // stride + 1) if kind == 1 else (h, w_)
+        layers.append(synth.LayerCfg(kind, K, co, float(co * ho * wo) / 2, 0.03 / (ho * wo), float(np.sqrt(co * ho * wo)),
+                                     H=h, Wd=w_, Cin=ci, stride=stride))
+        h, w_ = ho, wo
     return synth.Workload("mixed_conv", B, layers, (H, Wd, kinds_chans[0][1]), "normal", "kaiming_uniform", 2)
 
 
@@ -310,3 +316,56 @@ def _mixed_conv_workload(kinds_chans, H, Wd, B):
     ([(2, 12, 10)], 4, 12, 5)])                                            # Cin not a multiple of 16: dp4a path
 def test_pointwise_convolution_layers(path, stack, H, Wd, B):
     _run_and_compare(_mixed_conv_workload(stack, H, Wd, B), seed=51, steps=2, lam_per_step=0.2, path=path)
+
+
+def _fuzz_cases(n, seed):
+    g = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        n_layers = int(g.integers(1, 4))
+        widths = [int(g.choice([16, 24, 48, 100, 128, 130, 256, 272, 500, 512]))] + \
+                 [int(g.choice([8, 16, 33, 64, 96, 128, 144, 256, 300])) for _ in range(n_layers)]
+        B = int(g.choice([1, 2, 7, 32, 64, 100, 128, 129, 200]))
+        rounding = tuple(int(x) for x in g.integers(0, 2, size=3))
+        lam = float(g.choice([0.0, 0.25, 1.0]))
+        out.append((i, B, widths, rounding, lam))
+    return out
+
+
+@pytest.mark.parametrize("case", _fuzz_cases(24, 2024), ids=lambda c: f"fuzz{c[0]}")
+def test_fuzz_dense_networks(case):
+    """Seeded random layer stacks: widths on both sides of every tile and alignment boundary (so both the
+    tensor-core and the dp4a kernels and their hand-overs between layers are hit), all rounding modes."""
+    i, B, widths, rounding, lam = case
+    layers = [synth.LayerCfg(0, K, N, float(N) / 2, 0.03, float(np.sqrt(N))) for K, N in zip(widths[:-1], widths[1:])]
+    w = synth.Workload("fuzz", B, layers, (widths[0],), "uniform01", "kaiming_uniform", 1)
+    path = PATHS[i % len(PATHS)]
+    _run_and_compare(w, seed=100 + i, steps=2, lam_per_step=lam, path=path, rounding=rounding)
+
+
+@pytest.mark.parametrize("case", list(range(8)), ids=lambda c: f"convfuzz{c}")
+def test_fuzz_conv_networks(case):
+    g = np.random.default_rng(500 + case)
+    H, Wd = [(8, 16), (16, 16), (4, 32), (32, 32), (6, 12), (16, 64), (5, 10), (8, 128)][case]
+    chans = [int(g.choice([3, 8, 16]))] + [int(g.choice([16, 48, 64, 128])) for _ in range(int(g.integers(1, 4)))]
+    kinds = [1] + [int(g.choice([1, 2])) for _ in chans[2:]]
+    stack = [(k, ci, co) for k, ci, co in zip(kinds, chans[:-1], chans[1:])]
+    B = int(g.choice([1, 2, 3]))
+    _run_and_compare(_mixed_conv_workload(stack, H, Wd, B), seed=600 + case, steps=2, lam_per_step=0.3,
+                     path=PATHS[case % len(PATHS)])
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("stack,H,Wd,B", [
+    ([(1, 3, 64, 2), (1, 64, 128, 2), (1, 128, 64, 1)], 32, 32, 2),   # 32x32 -> 16x16 -> 8x8: im2col route, then 64- and 128-byte taps
+    ([(1, 64, 128, 2)], 64, 64, 1),                                    # one strided layer on the tensor cores, forced below
+    ([(1, 16, 32, 2), (2, 32, 24)], 9, 11, 3),                         # odd extents (5x6 outputs): dp4a path, then pointwise
+    ([(1, 3, 16, 1), (1, 16, 16, 2)], 16, 16, 2)])
+def test_strided_convolution_layers(path, stack, H, Wd, B):
+    _run_and_compare(_mixed_conv_workload(stack, H, Wd, B), seed=61, steps=2, lam_per_step=0.2, path=path)
+
+
+@pytest.mark.parametrize("form", TENSOR_FORMS)
+def test_strided_conv_forced_tensor_path(form):
+    w = _mixed_conv_workload([(1, 64, 128, 2)], 64, 64, 1)
+    _run_and_compare(w, seed=62, steps=2, lam_per_step=0.0, path=(ffb.FF_GEMM_TENSOR, form))

@@ -601,3 +601,66 @@ def test_conv1x1_gradient_matches_finite_differences():
         Wm[n, k] -= eps
         fd = (O.fp64_layer_loss(spec, X, Wp, B) - O.fp64_layer_loss(spec, X, Wm, B)) / (2 * eps)
         assert abs(fd - dW[n, k]) <= 1e-4 * max(1.0, abs(fd)), (n, k, fd, dW[n, k])
+
+
+# --------------------------------------------------------------------------------------
+# Strided 3x3 convolution
+# --------------------------------------------------------------------------------------
+def test_strided_conv_is_the_subsampled_stride1_conv_and_matches_brute_force():
+    g = np.random.default_rng(21)
+    for (H, Wd) in [(6, 8), (5, 7)]:                      # even and odd extents
+        x = g.integers(-127, 128, size=(2, H, Wd, 3)).astype(np.int8)
+        w = g.integers(-127, 128, size=(4, 3, 3, 3)).astype(np.int8)
+        full = O.int8_conv3x3(x, w)                      # pinned by brute force above
+        half = O.int8_conv3x3(x, w, stride=2)
+        assert half.shape == (2, (H - 1) // 2 + 1, (Wd - 1) // 2 + 1, 4)
+        assert np.array_equal(half, full[:, ::2, ::2, :])
+        # weight gradient: brute force over the strided windows
+        d = g.integers(-127, 128, size=half.shape).astype(np.int8)
+        got = O.int8_conv3x3_wgrad(d, x, stride=2)
+        want = np.zeros((4, 3, 3, 3), dtype=np.int64)
+        Ho, Wo = half.shape[1:3]
+        for b in range(2):
+            for i in range(Ho):
+                for j in range(Wo):
+                    for r in range(3):
+                        for t in range(3):
+                            hh, ww = 2 * i + r - 1, 2 * j + t - 1
+                            if 0 <= hh < H and 0 <= ww < Wd:
+                                want[:, r, t, :] += np.outer(d[b, i, j].astype(np.int64), x[b, hh, ww].astype(np.int64))
+        assert np.array_equal(got, want)
+
+
+def test_strided_conv_gradient_matches_finite_differences():
+    g = np.random.default_rng(22)
+    B, H, Wd, Cin, N = 1, 5, 6, 2, 3
+    spec = O.LayerSpec(O.KIND_CONV3X3, 9 * Cin, N, 10.0, 0.0, 1.0, H=H, Wd=Wd, Cin=Cin, stride=2)
+    X = g.normal(size=(2 * B, H, Wd, Cin))
+    W = g.normal(size=(N, 9 * Cin)) * 0.3
+    Ho, Wo = spec.out_hw
+    assert (Ho, Wo) == (3, 3) and spec.rows_per_sample == 9
+    # analytic gradient of the unquantised layer through the oracle's own integer routines is not possible;
+    # use the float formula: dW[n,r,s,ci] = sum dH[b,i,j,n] * xpad[b,2i+r,2j+s,ci]
+    xp = np.pad(X, ((0, 0), (1, 1), (1, 1), (0, 0)))
+    w4 = W.reshape(N, 3, 3, Cin)
+    Y = np.zeros((2 * B, Ho, Wo, N))
+    for r in range(3):
+        for s in range(3):
+            Y += xp[:, r:r + 2 * (Ho - 1) + 1:2, s:s + 2 * (Wo - 1) + 1:2, :] @ w4[:, r, s, :].T
+    Y = np.maximum(Y, 0.0)
+    G = (Y.reshape(2 * B, -1) ** 2).sum(1)
+    _, gp = O.ff_loss_terms(G.astype(F32), spec.theta, B)
+    dH = 2.0 * (gp / (2 * B))[:, None, None, None] * Y
+    dW = np.zeros((N, 3, 3, Cin))
+    for r in range(3):
+        for s in range(3):
+            win = xp[:, r:r + 2 * (Ho - 1) + 1:2, s:s + 2 * (Wo - 1) + 1:2, :]
+            dW[:, r, s, :] = dH.reshape(-1, N).T @ win.reshape(-1, Cin)
+    dW = dW.reshape(N, -1)
+    eps = 1e-6
+    for (n, k) in [(0, 0), (1, 7), (2, 17)]:
+        Wp, Wm = W.copy(), W.copy()
+        Wp[n, k] += eps
+        Wm[n, k] -= eps
+        fd = (O.fp64_layer_loss(spec, X, Wp, B) - O.fp64_layer_loss(spec, X, Wm, B)) / (2 * eps)
+        assert abs(fd - dW[n, k]) <= 1e-4 * max(1.0, abs(fd)), (n, k, fd, dW[n, k])
