@@ -269,6 +269,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--B", type=int, default=0, help="override positives per batch (profiling runs on a smaller case)")
     ap.add_argument("--tensor-form", type=int, default=0, help="CTAs per tensor-core tile: 0 auto, 1, 2")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="launch every kernel of a step one by one instead of replaying the captured launch sequence")
     ap.add_argument("--predict", action="store_true",
                     help="time classification by goodness (ff_predict, 10 candidate labels) instead of the train step")
     args = ap.parse_args()
@@ -298,6 +300,7 @@ def main():
     descs = [ffb.make_desc(l, i, seed) for i, l in enumerate(w.layers)]
     ctx = ffb.Context(descs, B, local)
     ffb.ff_set_tensor_form(ctx.ctx, args.tensor_form)
+    ffb.ff_set_graph_mode(ctx.ctx, not args.no_graph)
     bufs = [ffb.LayerBuffers(d, B, dev, dumps=False, xnext=False, own_x=(i == 0)) for i, d in enumerate(descs)]
     Ws = synth.make_weights(w, seed)
     for b, W in zip(bufs, Ws):
@@ -378,6 +381,9 @@ def main():
             st0 = ffb.ff_layer_bufs.from_buffer_copy(bufs[0].struct)
             st0.X = xd.data_ptr()
             arrs.append((ffb.ff_layer_bufs * len(descs))(st0, *[b.struct for b in bufs[1:]]))
+        for k in (0, 1, 0, 1):     # untimed: both buffer sets reach their steady launch form
+            ffb.ff_train_step(ctx.ctx, descs_arr, arrs[k], n_layers, B, 0.0, k, stream)
+        reset_weights()
         copy_stream = torch.cuda.Stream()
         main = torch.cuda.current_stream()
         ready = [torch.cuda.Event(), torch.cuda.Event()]     # batch landed in x_dev[k]
@@ -436,6 +442,8 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": {"workload": args.workload, "B_pos": B, "B_neg": B,
                        "layers": [[x.K, x.N] for x in w.layers],
+                       "launch": "kernel by kernel" if args.no_graph else
+                       f"captured launch sequence, {ffb.ff_graph_replay_count(ctx.ctx)} graph replays in this run",
                        "l2": "inputs larger than L2 (no flush needed)"
                        if 2 * B * l.H * l.Wd * l.K * 4 > 126e6 else "inputs smaller than L2, not flushed"},
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "loss_last": loss_last,

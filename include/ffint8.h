@@ -128,6 +128,22 @@ ff_status ff_set_gemm_path(ff_ctx* ctx, int path);
  * output has more than 128 rows), 1 / 2 force one form.  Identical bits. */
 ff_status ff_set_tensor_form(ff_ctx* ctx, int ctas_per_tile);
 
+/* Launch-sequence replay for ff_train_step (the paper's edge setting, batch 32 in Sec. V, makes a step a
+ * chain of short kernels whose cost is launch overhead; it states no counterpart of this switch).
+ * on = 1: the first ff_train_step call of a call shape runs its kernels one by one, the second is
+ * captured into a CUDA graph, and every later one is a single graph launch; the step counter and
+ * lambda are read from device memory, so they may change from call to call.  A call shape is the byte
+ * content of the layer and buffer arrays (zero any padding), n_layers, B, the workspace and the
+ * contraction route (the stream may change, the legacy default stream included); another shape gets a graph of its own (16 are kept, least recently used
+ * dropped), so a value inside a descriptor that changes every step (lr, theta) defeats the replay.
+ * Results are bit-identical to on = 0.  Replay is bypassed while ff_profile_start is active or the stream
+ * is already being captured by the caller.  on = 0 (default) drops the graphs.  Host state only: no
+ * device memory is allocated by the library beyond what graph instantiation itself takes. */
+ff_status ff_set_graph_mode(ff_ctx* ctx, int on);
+/* ff_train_step calls served by a graph launch so far (0 while the mode is off).  A call shape whose
+ * capture fails keeps running kernel by kernel and says why through ff_last_error. */
+uint64_t ff_graph_replay_count(const ff_ctx* ctx);
+
 /* Forward of one layer (Sec. IV-B: quantise A and W, INT8 MAC with INT32 accumulation; Sec. III /
  * Alg. 1 line 6: goodness).  Reads X, W.  Writes Xq, Wq, absmax[X,W,XNEXT], Y, S, rowmax, G,
  * Xnext (if non-NULL), acc_dump (if non-NULL).  `step` keys the stochastic rounding. */

@@ -19,6 +19,7 @@ FF_A_X_POS, FF_A_X_NEG, FF_A_W, FF_A_DH_POS, FF_A_DH_NEG, FF_A_XNEXT_POS, FF_A_X
 FF_ABSMAX_LEN = 8
 
 EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", "ff_set_gemm_path", "ff_set_tensor_form",
+           "ff_set_graph_mode", "ff_graph_replay_count",
            "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step",
            "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
            "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict"]
@@ -71,6 +72,7 @@ def load(build_if_missing: bool = True):
     lib.ff_set_workspace.argtypes = [vp, vp, C.c_size_t]
     lib.ff_set_gemm_path.argtypes = [vp, i32]
     lib.ff_set_tensor_form.argtypes = [vp, i32]
+    lib.ff_set_graph_mode.argtypes = [vp, i32]
     lib.ff_layer_forward.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, u64, vp]
     lib.ff_layer_loss_grad.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32,
                                        C.POINTER(vp), C.POINTER(f32), i32, f32, u64, vp]
@@ -81,6 +83,8 @@ def load(build_if_missing: bool = True):
     lib.ff_last_error.restype = C.c_char_p
     lib.ff_launch_count.argtypes = [vp]
     lib.ff_launch_count.restype = u64
+    lib.ff_graph_replay_count.argtypes = [vp]
+    lib.ff_graph_replay_count.restype = u64
     lib.ff_int8_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ff_profile_start.argtypes = [vp]
     lib.ff_predict.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, i32, i32, i32, vp, vp, u64, vp]
@@ -88,7 +92,7 @@ def load(build_if_missing: bool = True):
                                         C.c_char_p, C.c_size_t]
     lib.ff_profile_stop.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(C.c_uint32)]
     for name in EXPORTS:
-        if name not in ("ff_last_error", "ff_launch_count"):
+        if name not in ("ff_last_error", "ff_launch_count", "ff_graph_replay_count"):
             getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -131,6 +135,10 @@ def ff_set_tensor_form(ctx, ctas_per_tile: int):
     _check(ctx, load().ff_set_tensor_form(ctx, ctas_per_tile))
 
 
+def ff_set_graph_mode(ctx, on: bool):
+    _check(ctx, load().ff_set_graph_mode(ctx, 1 if on else 0))
+
+
 def ff_layer_forward(ctx, desc, bufs, B: int, step: int, stream: int = 0):
     _check(ctx, load().ff_layer_forward(ctx, C.byref(desc), C.byref(bufs), B, step, stream))
 
@@ -165,6 +173,14 @@ def ff_poll_status(ctx, stream: int = 0):
 
 def ff_launch_count(ctx) -> int:
     return int(load().ff_launch_count(ctx))
+
+
+def ff_last_error(ctx) -> str:
+    return load().ff_last_error(ctx).decode()
+
+
+def ff_graph_replay_count(ctx) -> int:
+    return int(load().ff_graph_replay_count(ctx))
 
 
 def ff_profile_start(ctx):

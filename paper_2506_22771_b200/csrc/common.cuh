@@ -23,8 +23,8 @@ struct RoundKey {
   uint32_t k0, k1;
 };
 
-// SplitMix64 output function (host side key derivation).
-__host__ inline uint64_t splitmix64(uint64_t x) {
+// SplitMix64 output function (key derivation).
+__host__ __device__ inline uint64_t splitmix64(uint64_t x) {
   x += 0x9E3779B97F4A7C15ull;
   uint64_t z = x;
   z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
@@ -32,14 +32,38 @@ __host__ inline uint64_t splitmix64(uint64_t x) {
   return z ^ (z >> 31);
 }
 
-__host__ inline RoundKey make_round_key(uint64_t seed, int role, int layer, uint64_t step) {
+// The values of a train step that change from call to call.  They live in device memory (written by
+// set_step_kernel before the step's kernels) instead of kernel arguments, so that the launch sequence
+// of a step is the same every time and can be replayed from a captured CUDA graph.
+struct StepState {
+  unsigned long long step;  // keys the stochastic rounding
+  float lambda;             // look-ahead weight of Eq. 3
+  float pad;
+};
+
+// Key of one quantiser call: the step-independent part (seed, tensor role, layer) is folded on the host,
+// the step is folded in on the device.
+struct KeySpec {
+  unsigned long long s1;
+  const StepState* ss;
+};
+__host__ inline KeySpec make_key_spec(uint64_t seed, int role, int layer, const StepState* ss) {
   uint64_t s0 = splitmix64(seed);
-  uint64_t s1 = splitmix64(s0 ^ (uint64_t)((uint32_t)(role & 0xFF) | ((uint32_t)(layer & 0xFFFFFF) << 8)));
-  uint64_t s2 = splitmix64(s1 ^ step);
+  KeySpec k;
+  k.s1 = splitmix64(s0 ^ (uint64_t)((uint32_t)(role & 0xFF) | ((uint32_t)(layer & 0xFFFFFF) << 8)));
+  k.ss = ss;
+  return k;
+}
+__device__ __forceinline__ RoundKey derive_key(KeySpec ks) {
+  const uint64_t s2 = splitmix64(ks.s1 ^ ks.ss->step);
   RoundKey k;
   k.k0 = (uint32_t)(s2 & 0xFFFFFFFFull);
   k.k1 = (uint32_t)(s2 >> 32);
   return k;
+}
+__global__ void set_step_kernel(StepState* ss, unsigned long long step, float lambda, int set_lambda) {
+  ss->step = step;
+  if (set_lambda) ss->lambda = lambda;
 }
 
 // s = a/127, inv = 127/a.  A zero tensor, or one whose range is below 2^-100 (127/a would leave

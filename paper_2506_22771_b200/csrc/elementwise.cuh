@@ -67,8 +67,9 @@ __global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restr
 template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __restrict__ x, int8_t* __restrict__ q,
                                                               size_t n_per_pass, const float* __restrict__ a,
-                                                              RoundKey key, unsigned long long* __restrict__ zero_S = nullptr,
+                                                              KeySpec ks, unsigned long long* __restrict__ zero_S = nullptr,
                                                               int32_t* __restrict__ zero_rowmax = nullptr, int zero_n = 0) {
+  const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
   if (zero_S && blockIdx.y == 0)
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < zero_n; i += gridDim.x * blockDim.x) {
       zero_S[i] = 0ull;
@@ -161,7 +162,8 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
                                                                float tau, float eps, size_t per_sample,
                                                                size_t per_pass, float* __restrict__ xnext,
                                                                int8_t* __restrict__ xq, const float* __restrict__ a,
-                                                               RoundKey key) {
+                                                               KeySpec ks) {
+  const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
   const size_t base = (size_t)blockIdx.y * per_pass;
   const float inv = xq ? inv_of(a[blockIdx.y]) : 0.0f;
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) &&
@@ -260,7 +262,9 @@ struct LossScratch {
 __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __restrict__ G, float theta, LaterLayers later,
                                                                  float lambda, int B, const int32_t* __restrict__ rowmax,
                                                                  float* __restrict__ absmax, float* __restrict__ coef,
-                                                                 float* __restrict__ loss, LossScratch* __restrict__ scratch) {
+                                                                 float* __restrict__ loss, LossScratch* __restrict__ scratch,
+                                                                 const StepState* __restrict__ ss = nullptr) {
+  if (ss) lambda = ss->lambda;  // a step run through the library's own launch sequence keeps lambda in device memory
   __shared__ double red[LOSS_THREADS / 32];
   __shared__ uint32_t redmax[2][LOSS_THREADS / 32];
   __shared__ bool is_last;
@@ -366,7 +370,8 @@ __global__ void __launch_bounds__(EW_THREADS) classify_kernel(LaterLayers layers
 template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) dh_quantize_kernel(const float* __restrict__ Y, const float* __restrict__ coef,
                                                                  const float* __restrict__ absmax, size_t per_sample,
-                                                                 size_t per_pass, int8_t* __restrict__ dHq, RoundKey key) {
+                                                                 size_t per_pass, int8_t* __restrict__ dHq, KeySpec ks) {
+  const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
   const size_t base = (size_t)blockIdx.y * per_pass;
   const float inv = inv_of(absmax[3 + blockIdx.y]);
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)dHq) & 3) == 0);

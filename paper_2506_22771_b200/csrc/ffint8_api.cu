@@ -35,6 +35,19 @@ struct ff_ctx {
   };
   std::vector<ProfRec> prof_recs;
   std::vector<cudaEvent_t> prof_pool;
+  // captured launch sequences of ff_train_step (ff_set_graph_mode)
+  bool graph_mode = false;
+  struct GraphEntry {
+    std::vector<unsigned char> key;  // everything the launch sequence depends on, compared byte by byte
+    cudaGraphExec_t exec = nullptr;
+    uint64_t launches = 0;           // kernel launches one replay stands for
+    bool eager_only = false;         // capture failed once: this call shape stays on the eager path
+    uint64_t last_use = 0;
+  };
+  std::vector<GraphEntry> graphs;
+  uint64_t graph_clock = 0;
+  uint64_t graph_replays = 0;
+  cudaStream_t capture_stream = nullptr;  // captures are recorded here (the caller's may be the legacy stream, which cannot capture)
   char err[512] = {0};
 };
 
@@ -42,6 +55,7 @@ namespace {
 
 // workspace layout: [0, 256) status word (+ padding), then the loss kernel's partial-sum scratch
 constexpr size_t WS_STATUS_BYTES = 256;
+constexpr size_t WS_STEP_OFFSET = 64;   // StepState inside the status block
 constexpr size_t WS_LOSS_OFFSET = WS_STATUS_BYTES;
 constexpr size_t WS_BYTES = (WS_LOSS_OFFSET + sizeof(LossScratch) + 255) / 256 * 256;  // fixed header
 // After the header: INT32 partial-sum slabs of a split weight-gradient contraction,
@@ -151,6 +165,15 @@ ff_status check_ctx(ff_ctx* ctx) {
 }
 
 inline uint32_t* status_ptr(ff_ctx* ctx) { return reinterpret_cast<uint32_t*>(ctx->workspace); }
+inline StepState* step_ptr(ff_ctx* ctx) {
+  return reinterpret_cast<StepState*>(static_cast<char*>(ctx->workspace) + WS_STEP_OFFSET);
+}
+// Publishes the step counter (and lambda) to the kernels of the calls that follow on `st`.
+ff_status set_step(ff_ctx* ctx, uint64_t step, float lambda, bool with_lambda, cudaStream_t st) {
+  set_step_kernel<<<1, 1, 0, st>>>(step_ptr(ctx), step, lambda, with_lambda ? 1 : 0);
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
 
 ff_status ensure_status(ff_ctx* ctx, cudaStream_t st) {
   if (!ctx->status_zeroed) {
@@ -414,7 +437,7 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
 // ---- step pieces --------------------------------------------------------------------------
 // Quantise the weights and run the forward contraction; the layer input is already in Xq and
 // its ranges in absmax[X_POS..X_NEG].
-ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint64_t step,
+ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B,
                           float* a_next2, cudaStream_t st) {
   const size_t nW = (size_t)L.N * L.K;
   {
@@ -425,7 +448,7 @@ ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
   {
     ProfScope prof(ctx, FF_K_QUANTIZE, st);
     const dim3 grid(ew_blocks(ctx, nW / 4 + 1), 1);
-    const RoundKey key = make_round_key(L.seed, ROLE_W, L.index, step);
+    const KeySpec key = make_key_spec(L.seed, ROLE_W, L.index, step_ptr(ctx));
     unsigned long long* S = reinterpret_cast<unsigned long long*>(b.S);  // cleared on the side for the forward epilogue
     if (L.round_w == FF_ROUND_NEAREST_EVEN)
       quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, key, S, b.rowmax, 2 * B);
@@ -445,7 +468,7 @@ ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
   return FF_OK;
 }
 
-ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, uint64_t step, cudaStream_t st) {
+ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
   const size_t per_pass = (size_t)B * in_rows_per_sample(L) * in_features(L);
   {
     ProfScope prof(ctx, FF_K_ABSMAX, st);
@@ -456,7 +479,7 @@ ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
   {
     ProfScope prof(ctx, FF_K_QUANTIZE, st);
     const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
-    const RoundKey key = make_round_key(L.seed, ROLE_X, L.index, step);
+    const KeySpec key = make_key_spec(L.seed, ROLE_X, L.index, step_ptr(ctx));
     if (L.round_x == FF_ROUND_NEAREST_EVEN)
       quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, key);
     else
@@ -469,11 +492,11 @@ ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
 // Normalised output of layer `L` as FP32 (b.Xnext, if non-NULL) and / or as the INT8 input of the
 // next layer (xq_next, nullable; rounding keyed by the next layer).
 ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, int8_t* xq_next,
-                           const ff_layer_desc* next, uint64_t step, cudaStream_t st) {
+                           const ff_layer_desc* next, cudaStream_t st) {
   if (!b.Xnext && !xq_next) return FF_OK;
   const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
   const size_t per_pass = per_sample * B;
-  RoundKey key = next ? make_round_key(next->seed, ROLE_X, next->index, step) : RoundKey{0, 0};
+  const KeySpec key = next ? make_key_spec(next->seed, ROLE_X, next->index, step_ptr(ctx)) : KeySpec{0ull, step_ptr(ctx)};
   {
     ProfScope prof(ctx, FF_K_NORMALIZE, st);
     const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
@@ -489,7 +512,7 @@ ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
 }
 
 ff_status loss_grad_impl(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, const float* const* G_later,
-                         const float* theta_later, int n_later, float lambda, uint64_t step, cudaStream_t st) {
+                         const float* theta_later, int n_later, float lambda, cudaStream_t st) {
   LaterLayers later;
   later.n = n_later;
   for (int j = 0; j < n_later; ++j) {
@@ -502,7 +525,7 @@ ff_status loss_grad_impl(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
     ProfScope prof(ctx, FF_K_LOSS, st);
     loss_coef_kernel<<<loss_blocks, LOSS_THREADS, 0, st>>>(
         b.G, L.theta, later, lambda, B, b.rowmax, b.absmax, b.coef, b.loss,
-        reinterpret_cast<LossScratch*>(static_cast<char*>(ctx->workspace) + WS_LOSS_OFFSET));
+        reinterpret_cast<LossScratch*>(static_cast<char*>(ctx->workspace) + WS_LOSS_OFFSET), step_ptr(ctx));
   }
   FF_LAUNCH_CHECK(ctx);
   const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
@@ -510,7 +533,7 @@ ff_status loss_grad_impl(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
   {
     ProfScope prof(ctx, FF_K_DH_QUANTIZE, st);
     const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
-    const RoundKey key = make_round_key(L.seed, ROLE_DH, L.index, step);
+    const KeySpec key = make_key_spec(L.seed, ROLE_DH, L.index, step_ptr(ctx));
     if (L.round_dh == FF_ROUND_NEAREST_EVEN)
       dh_quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key);
     else
@@ -537,20 +560,140 @@ ff_status check_layer_list(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
 
 // INT8 forward through all layers with the current weights (Alg. 1 line 5-6): layer 0 reads bufs[0].X,
 // layer l > 0 reads bufs[l].X if given, else the previous layer's normalised output, quantised on the fly.
-ff_status forward_all(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B, uint64_t step,
+ff_status forward_all(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
                       cudaStream_t st) {
   ff_status s;
   for (int l = 0; l < n_layers; ++l) FF_CUDA(ctx, cudaMemsetAsync(bufs[l].absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
   for (int l = 0; l < n_layers; ++l) {
     const bool chained = l > 0 && !bufs[l].X;
-    if (!chained && (s = quantize_input(ctx, layers[l], bufs[l], B, step, st)) != FF_OK) return s;
+    if (!chained && (s = quantize_input(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
     const bool feeds_next = l + 1 < n_layers && !bufs[l + 1].X;
-    if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, step, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st)) != FF_OK)
+    if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st)) != FF_OK)
       return s;
     if ((s = normalize_output(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].Xq : nullptr,
-                              feeds_next ? &layers[l + 1] : nullptr, step, st)) != FF_OK)
+                              feeds_next ? &layers[l + 1] : nullptr, st)) != FF_OK)
       return s;
   }
+  return FF_OK;
+}
+
+// Everything of one train step after the step counter and lambda have been published (Alg. 1, epoch body).
+ff_status train_step_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
+                          float lambda, cudaStream_t st) {
+  ff_status s;
+  // Alg. 1 line 5-6: one forward through all layers with the pre-update weights
+  if ((s = forward_all(ctx, layers, bufs, n_layers, B, st)) != FF_OK) return s;
+  // Alg. 1 line 7-9: per layer, loss from the G's (Eq. 3), INT8 gradient and update
+  for (int l = 0; l < n_layers; ++l) {
+    const float* Gl[FF_MAX_LATER];
+    float th[FF_MAX_LATER];
+    int n_later = n_layers - 1 - l;
+    for (int j = 0; j < n_later; ++j) {
+      Gl[j] = bufs[l + 1 + j].G;
+      th[j] = layers[l + 1 + j].theta;
+    }
+    if ((s = loss_grad_impl(ctx, layers[l], bufs[l], B, Gl, th, n_later, lambda, st)) != FF_OK) return s;
+    if ((s = run_update_gemm(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
+  }
+  return FF_OK;
+}
+
+constexpr size_t FF_MAX_GRAPHS = 16;
+
+void drop_graphs(ff_ctx* ctx) {
+  for (auto& g : ctx->graphs)
+    if (g.exec) cudaGraphExecDestroy(g.exec);
+  ctx->graphs.clear();
+}
+
+// Notes why a call shape stays on the eager path; readable through ff_last_error, no call fails because of it.
+void graph_gave_up(ff_ctx* ctx, ff_ctx::GraphEntry* ent, const char* what, cudaError_t e) {
+  ent->eager_only = true;
+  snprintf(ctx->err, sizeof(ctx->err), "graph mode: %s (%s); this call shape runs kernel by kernel", what,
+           cudaGetErrorString(e));
+  cudaGetLastError();
+}
+
+// Train step through a captured launch sequence.  The sequence of a step depends on the layer list, the
+// buffer pointers, the batch size, the workspace and the contraction route, but not on the step counter
+// or lambda (those are read from device memory), so one captured graph serves every later step of the
+// same call shape.  First call of a shape: eager (it also fills the per-kernel attribute and occupancy
+// caches, which must not happen inside a capture).  Second call: captured, instantiated and launched.
+// Later calls: one graph launch.  A shape whose capture fails stays on the eager path.
+ff_status train_step_graph(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
+                           float lambda, cudaStream_t st) {
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+    cudaGetLastError();
+    return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);  // the caller is capturing already
+  }
+  std::vector<unsigned char> key;
+  auto put = [&key](const void* p, size_t n) {
+    const unsigned char* c = static_cast<const unsigned char*>(p);
+    key.insert(key.end(), c, c + n);
+  };
+  const int route[3] = {ctx->gemm_path, ctx->tc.force_ncta, B};
+  put(route, sizeof(route));
+  put(&ctx->workspace, sizeof(void*));
+  put(&ctx->workspace_bytes, sizeof(size_t));
+  put(layers, sizeof(ff_layer_desc) * n_layers);
+  put(bufs, sizeof(ff_layer_bufs) * n_layers);
+
+  ff_ctx::GraphEntry* ent = nullptr;
+  for (auto& g : ctx->graphs)
+    if (g.key == key) ent = &g;
+  if (!ent) {
+    if (ctx->graphs.size() >= FF_MAX_GRAPHS) {  // drop the entry unused for longest
+      size_t old = 0;
+      for (size_t i = 1; i < ctx->graphs.size(); ++i)
+        if (ctx->graphs[i].last_use < ctx->graphs[old].last_use) old = i;
+      if (ctx->graphs[old].exec) cudaGraphExecDestroy(ctx->graphs[old].exec);
+      ctx->graphs.erase(ctx->graphs.begin() + old);
+    }
+    ctx->graphs.emplace_back();
+    ctx->graphs.back().key = std::move(key);
+    ctx->graphs.back().last_use = ++ctx->graph_clock;
+    return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+  }
+  ent->last_use = ++ctx->graph_clock;
+  if (ent->eager_only) return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+  if (!ent->exec) {
+    cudaError_t e;
+    if (!ctx->capture_stream &&
+        (e = cudaStreamCreateWithFlags(&ctx->capture_stream, cudaStreamNonBlocking)) != cudaSuccess) {
+      ctx->capture_stream = nullptr;
+      graph_gave_up(ctx, ent, "no capture stream", e);
+      return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+    }
+    const uint64_t before = ctx->launches;
+    if ((e = cudaStreamBeginCapture(ctx->capture_stream, cudaStreamCaptureModeThreadLocal)) != cudaSuccess) {
+      graph_gave_up(ctx, ent, "capture did not start", e);
+      return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+    }
+    // nothing runs while capturing: the launches are recorded on the library's own stream and replayed on the caller's
+    const ff_status body = train_step_body(ctx, layers, bufs, n_layers, B, lambda, ctx->capture_stream);
+    cudaGraph_t graph = nullptr;
+    e = cudaStreamEndCapture(ctx->capture_stream, &graph);
+    const uint64_t captured = ctx->launches - before;
+    ctx->launches = before;
+    cudaGraphExec_t exec = nullptr;
+    if (body == FF_OK && e == cudaSuccess && graph) e = cudaGraphInstantiate(&exec, graph, 0);
+    if (graph) cudaGraphDestroy(graph);
+    if (body != FF_OK) {  // an argument the body rejects: nothing was launched
+      ent->eager_only = true;
+      cudaGetLastError();
+      return body;
+    }
+    if (e != cudaSuccess || !exec) {
+      graph_gave_up(ctx, ent, "capture or instantiation failed", e);
+      return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+    }
+    ent->exec = exec;
+    ent->launches = captured;
+  }
+  FF_CUDA(ctx, cudaGraphLaunch(ent->exec, st));
+  ctx->launches += ent->launches;
+  ctx->graph_replays++;
   return FF_OK;
 }
 
@@ -584,6 +727,8 @@ ff_status ff_destroy(ff_ctx* ctx) {
       cudaEventDestroy(r.b);
     }
     for (auto e : ctx->prof_pool) cudaEventDestroy(e);
+    drop_graphs(ctx);
+    if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
   }
   delete ctx;
   return FF_OK;
@@ -625,6 +770,7 @@ ff_status ff_set_workspace(ff_ctx* ctx, void* dev_ptr, size_t bytes) {
   ctx->workspace = dev_ptr;
   ctx->workspace_bytes = bytes;
   ctx->status_zeroed = false;
+  drop_graphs(ctx);
   return FF_OK;
 }
 
@@ -651,9 +797,10 @@ ff_status ff_layer_forward(ff_ctx* ctx, const ff_layer_desc* layer, const ff_lay
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
   FF_CUDA(ctx, cudaMemsetAsync(bufs->absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
-  if ((s = quantize_input(ctx, *layer, *bufs, B, step, st)) != FF_OK) return s;
-  if ((s = forward_from_xq(ctx, *layer, *bufs, B, step, nullptr, st)) != FF_OK) return s;
-  return normalize_output(ctx, *layer, *bufs, B, nullptr, nullptr, step, st);
+  if ((s = set_step(ctx, step, 0.0f, false, st)) != FF_OK) return s;
+  if ((s = quantize_input(ctx, *layer, *bufs, B, st)) != FF_OK) return s;
+  if ((s = forward_from_xq(ctx, *layer, *bufs, B, nullptr, st)) != FF_OK) return s;
+  return normalize_output(ctx, *layer, *bufs, B, nullptr, nullptr, st);
 }
 
 ff_status ff_layer_loss_grad(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs, int B,
@@ -669,7 +816,8 @@ ff_status ff_layer_loss_grad(ff_ctx* ctx, const ff_layer_desc* layer, const ff_l
     if (!G_later[j]) return fail(ctx, FF_ERR_ARG, "a G_later pointer is NULL");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
-  return loss_grad_impl(ctx, *layer, *bufs, B, G_later, theta_later, n_later, lambda, step, st);
+  if ((s = set_step(ctx, step, lambda, true, st)) != FF_OK) return s;
+  return loss_grad_impl(ctx, *layer, *bufs, B, G_later, theta_later, n_later, lambda, st);
 }
 
 ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs, int B, void* cuda_stream) {
@@ -689,20 +837,16 @@ ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
   if ((s = check_layer_list(ctx, layers, bufs, n_layers, B)) != FF_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
-  // Alg. 1 line 5-6: one forward through all layers with the pre-update weights
-  if ((s = forward_all(ctx, layers, bufs, n_layers, B, step, st)) != FF_OK) return s;
-  // Alg. 1 line 7-9: per layer, loss from the G's (Eq. 3), INT8 gradient and update
-  for (int l = 0; l < n_layers; ++l) {
-    const float* Gl[FF_MAX_LATER];
-    float th[FF_MAX_LATER];
-    int n_later = n_layers - 1 - l;
-    for (int j = 0; j < n_later; ++j) {
-      Gl[j] = bufs[l + 1 + j].G;
-      th[j] = layers[l + 1 + j].theta;
-    }
-    if ((s = loss_grad_impl(ctx, layers[l], bufs[l], B, Gl, th, n_later, lambda, step, st)) != FF_OK) return s;
-    if ((s = run_update_gemm(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
-  }
+  if ((s = set_step(ctx, step, lambda, true, st)) != FF_OK) return s;
+  if (ctx->graph_mode && !ctx->profiling) return train_step_graph(ctx, layers, bufs, n_layers, B, lambda, st);
+  return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+}
+
+ff_status ff_set_graph_mode(ff_ctx* ctx, int on) {
+  if (!ctx) return FF_ERR_ARG;
+  if (on != 0 && on != 1) return fail(ctx, FF_ERR_ARG, "graph mode must be 0 or 1");
+  ctx->graph_mode = on != 0;
+  if (!on) drop_graphs(ctx);
   return FF_OK;
 }
 
@@ -720,7 +864,8 @@ ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bu
   if (first_counted_layer < 0 || first_counted_layer >= n_layers) return fail(ctx, FF_ERR_ARG, "first_counted_layer out of range");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
-  if ((s = forward_all(ctx, layers, bufs, n_layers, half, step, st)) != FF_OK) return s;
+  if ((s = set_step(ctx, step, 0.0f, false, st)) != FF_OK) return s;
+  if ((s = forward_all(ctx, layers, bufs, n_layers, half, st)) != FF_OK) return s;
   LaterLayers gs;
   gs.n = n_layers - first_counted_layer;
   for (int j = 0; j < gs.n; ++j) {
@@ -784,6 +929,8 @@ ff_status ff_profile_stop(ff_ctx* ctx, void* cuda_stream, float* ms_per_kernel, 
 const char* ff_last_error(const ff_ctx* ctx) { return ctx ? ctx->err : "context is NULL"; }
 
 uint64_t ff_launch_count(const ff_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+uint64_t ff_graph_replay_count(const ff_ctx* ctx) { return ctx ? ctx->graph_replays : 0; }
 
 ff_status ff_int8_gemm(ff_ctx* ctx, const int8_t* A, const int8_t* Bm, int32_t* C, int M, int N, int K, int trans,
                        void* cuda_stream) {

@@ -60,11 +60,11 @@ def test_int8_gemm_tensor_weight_gradient_orientation(M, N, K, form):
     _gemm_case(M, N, K, 1, ffb.FF_GEMM_TENSOR, form)
 
 
-def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), chain=True, check_every=1):
+def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), chain=True, check_every=1, graph=False):
     specs, descs = specs_and_descs(w.layers, seed, *rounding)
     Ws = synth.make_weights(w, seed)
     X = synth.make_batch(w, seed)
-    net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path)
+    net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path, graph=graph)
     net.set_input(X)
     for step in range(steps):
         lam = lam_per_step * step
@@ -369,3 +369,85 @@ def test_strided_convolution_layers(path, stack, H, Wd, B):
 def test_strided_conv_forced_tensor_path(form):
     w = _mixed_conv_workload([(1, 64, 128, 2)], 64, 64, 1)
     _run_and_compare(w, seed=62, steps=2, lam_per_step=0.0, path=(ffb.FF_GEMM_TENSOR, form))
+
+
+# ---- launch-sequence replay (CUDA graph) of the train step ---------------------------------------
+# step 0 runs eagerly, step 1 is captured, steps 2.. are graph launches; the step counter (rounding
+# keys) and lambda change every step and must reach the replayed kernels through device memory.
+@pytest.mark.parametrize("path", PATHS)
+def test_graph_replay_dense_lookahead(path):
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=72, width_div=8)
+    _run_and_compare(w, seed=31, steps=6, lam_per_step=0.125, path=path, graph=True)
+
+
+def test_graph_replay_tiny_mlp_all_stochastic():
+    _run_and_compare(synth.workload("tiny_mlp"), seed=12, steps=8, lam_per_step=0.0, path=(ffb.FF_GEMM_AUTO, 0),
+                     rounding=(1, 1, 1), graph=True)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_graph_replay_cnn(path):
+    w = synth.scaled(synth.workload("cnn"), B=2, width_div=4)
+    _run_and_compare(w, seed=22, steps=4, lam_per_step=0.0, path=path, graph=True)
+
+
+def test_graph_replay_counts_launches_and_yields_to_profiling():
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=40, width_div=8)
+    specs, descs = specs_and_descs(w.layers, 4)
+    Ws = synth.make_weights(w, 4)
+    X = synth.make_batch(w, 4)
+    net = GpuNet(descs, w.B, Ws, graph=True)
+    net.set_input(X)
+    counts = []
+    for step in range(7):
+        if step == 4:
+            ffb.ff_profile_start(net.ctx.ctx)          # profiled steps run kernel by kernel
+        before = ffb.ff_launch_count(net.ctx.ctx)
+        net.train_step(0.5, step)
+        counts.append(ffb.ff_launch_count(net.ctx.ctx) - before)
+        if step == 4:
+            timed = sum(v[1] for v in ffb.ff_profile_stop(net.ctx.ctx, 0).values())
+            assert 0 < timed < counts[-1]               # the step-counter store is launched but not timed
+        states = O.train_step(specs, Ws, X, w.B, 0.5, step)
+        Ws = [st.W_new for st in states]
+    assert len(set(counts)) == 1 and counts[0] > 0, counts   # a replay stands for the same launches
+    # steps 0 (first sight) and 1 (capture + first replay) aside, every unprofiled step was a graph launch
+    assert ffb.ff_graph_replay_count(net.ctx.ctx) == 5, ffb.ff_last_error(net.ctx.ctx)
+    for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
+        compare_layer(st, b, sp, w.B, tag=f"layer{l}/")
+    # switching the mode off drops the graphs; the eager path continues the same trajectory
+    ffb.ff_set_graph_mode(net.ctx.ctx, False)
+    net.train_step(0.5, 7)
+    states = O.train_step(specs, Ws, X, w.B, 0.5, 7)
+    for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
+        compare_layer(st, b, sp, w.B, tag=f"eager/layer{l}/")
+    net.close()
+
+
+def test_graph_replay_two_call_shapes_share_a_context():
+    # two networks' worth of buffers driven through ONE context, alternating: each call shape gets its own graph
+    import torch
+    w = synth.scaled(synth.workload("tiny_mlp"), B=16, width_div=2)
+    specs, descs = specs_and_descs(w.layers, 8)
+    net = GpuNet(descs, w.B, synth.make_weights(w, 8), graph=True)
+    other = [ffb.LayerBuffers(d, w.B, net.dev, dumps=True, xnext=True, own_x=(i == 0)) for i, d in enumerate(descs)]
+    other_arr = (ffb.ff_layer_bufs * len(descs))(*[b.struct for b in other])
+    Wa, Wb = synth.make_weights(w, 8), synth.make_weights(w, 9)
+    Xa, Xb = synth.make_batch(w, 8), synth.make_batch(w, 9)
+    for b, W in zip(other, Wb):
+        b.W.copy_(torch.from_numpy(W))
+    net.set_input(Xa)
+    other[0].X.copy_(torch.from_numpy(np.ascontiguousarray(Xb)).reshape(other[0].X.shape))
+    for step in range(5):
+        net.train_step(0.0, step)
+        ffb.ff_train_step(net.ctx.ctx, net.descs_arr, other_arr, len(descs), w.B, 0.0, step + 100, 0)
+        ffb.ff_poll_status(net.ctx.ctx, 0)
+        sa = O.train_step(specs, Wa, Xa, w.B, 0.0, step)
+        sb = O.train_step(specs, Wb, Xb, w.B, 0.0, step + 100)
+        for l in range(len(specs)):
+            compare_layer(sa[l], net.bufs[l], specs[l], w.B, tag=f"a/step{step}/layer{l}/")
+            compare_layer(sb[l], other[l], specs[l], w.B, tag=f"b/step{step}/layer{l}/")
+        Wa = [st.W_new for st in sa]
+        Wb = [st.W_new for st in sb]
+    assert ffb.ff_graph_replay_count(net.ctx.ctx) == 8, ffb.ff_last_error(net.ctx.ctx)
+    net.close()
