@@ -271,6 +271,9 @@ def main():
     ap.add_argument("--tensor-form", type=int, default=0, help="CTAs per tensor-core tile: 0 auto, 1, 2")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every kernel of a step one by one instead of replaying the captured launch sequence")
+    ap.add_argument("--data-parallel", action="store_true",
+                    help="split ONE batch by rows over the ranks (ff_dp_train_phase + NCCL all-reduce between the phases) "
+                         "instead of independent replicas; strong scaling, no end-to-end leg")
     ap.add_argument("--predict", action="store_true",
                     help="time classification by goodness (ff_predict, 10 candidate labels) instead of the train step")
     args = ap.parse_args()
@@ -289,23 +292,39 @@ def main():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    if world > 1 or args.data_parallel:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+        dist.init_process_group("nccl", device_id=dev, rank=rank, world_size=world)
 
     w = synth.workload(args.workload)
     if args.predict:
         return run_predict(args, w, world, rank, local, dev)
     B = args.B or w.B
     seed = 1 + rank
+    dpar = args.data_parallel
+    if dpar:
+        # one batch of B_total rows per set, this rank holds rows [row_off, row_off + B); identical replicas
+        from paper_2506_22771_b200 import data_parallel as dp
+        B_total, seed = B, 1
+        row_off, B = dp.shard_rows(B_total, world, rank)
+        args.no_e2e = args.no_graph = True
     descs = [ffb.make_desc(l, i, seed) for i, l in enumerate(w.layers)]
     ctx = ffb.Context(descs, B, local)
     ffb.ff_set_tensor_form(ctx.ctx, args.tensor_form)
     ffb.ff_set_graph_mode(ctx.ctx, not args.no_graph)
-    bufs = [ffb.LayerBuffers(d, B, dev, dumps=False, xnext=False, own_x=(i == 0)) for i, d in enumerate(descs)]
+    bufs = [ffb.LayerBuffers(d, B, dev, dumps=False, xnext=False, own_x=(i == 0), accw=dpar) for i, d in enumerate(descs)]
     Ws = synth.make_weights(w, seed)
     for b, W in zip(bufs, Ws):
         b.W.copy_(torch.from_numpy(W))
-    X_host = torch.from_numpy(synth.make_batch(w, seed, B=B)).reshape(bufs[0].X.shape).pin_memory()
+    if dpar:
+        table = dp.PointerTable()
+        table.add_layer_buffers(bufs)
+        X_all = torch.from_numpy(synth.make_batch(w, seed, B=B_total)).reshape(2 * B_total, -1)
+        X_host = dp.shard_batch(X_all, B_total, row_off, B).reshape(bufs[0].X.shape).pin_memory()
+        del X_all
+    else:
+        X_host = torch.from_numpy(synth.make_batch(w, seed, B=B)).reshape(bufs[0].X.shape).pin_memory()
     bufs[0].X.copy_(X_host)
     W0 = [b.W.clone() for b in bufs]
     descs_arr = (ffb.ff_layer_desc * len(descs))(*descs)
@@ -315,7 +334,11 @@ def main():
     last = n_layers - 1
 
     def step(i):
-        ffb.ff_train_step(ctx.ctx, descs_arr, bufs_arr, n_layers, B, w.lam_per_step * i, i, stream)
+        if dpar:
+            dp.dp_train_step(ctx.ctx, descs_arr, bufs_arr, n_layers, B, B_total, row_off, w.lam_per_step * i, i,
+                             lambda entries: dp.all_reduce_entries(entries, table), stream)
+        else:
+            ffb.ff_train_step(ctx.ctx, descs_arr, bufs_arr, n_layers, B, w.lam_per_step * i, i, stream)
 
     def barrier():
         if world > 1:
@@ -439,9 +462,12 @@ def main():
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "scaling": "strong" if dpar else "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": {"workload": args.workload, "B_pos": B, "B_neg": B,
                        "layers": [[x.K, x.N] for x in w.layers],
+                       "parallelism": f"one batch of {B_total} + {B_total} rows split over {world} rank(s), all-reduce of "
+                                      "ranges, loss and INT32 weight-gradient sums between phases" if dpar else
+                                      "independent replicas",
                        "launch": "kernel by kernel" if args.no_graph else
                        f"captured launch sequence, {ffb.ff_graph_replay_count(ctx.ctx)} graph replays in this run",
                        "l2": "inputs larger than L2 (no flush needed)"

@@ -128,6 +128,44 @@ ff_status ff_set_gemm_path(ff_ctx* ctx, int path);
  * output has more than 128 rows), 1 / 2 force one form.  Identical bits. */
 ff_status ff_set_tensor_form(ff_ctx* ctx, int ctas_per_tile);
 
+/* ---- data-parallel train step --------------------------------------------------------------
+ * The batch of one step split by rows over several devices, each holding a replica of the weights:
+ * forward, goodness, loss coefficient and output gradient are per sample (Sec. III, Sec. IV-B), so a
+ * shard computes them alone; what couples the shards are (1) the per-tensor ranges of the symmetric
+ * quantiser (a maximum over the whole batch), (2) the batch mean of the loss, (3) the INT32
+ * weight-gradient sums g^W = g^Y^T A (Sec. IV-B), which add exactly in integers.  With those
+ * three combined over the shards every replica applies the same update, bit-identical to
+ * ff_train_step on the whole batch on one device (the stochastic-rounding counters are the element
+ * indices of the unsplit tensors).  The paper trains on one device and describes no such split.
+ *
+ * The step is cut at the points where shards must exchange data.  The caller runs phases
+ * 0 .. ff_dp_phase_count(n_layers)-1 in order, on every shard; after each phase it combines, in place
+ * and over all shards, the n_reduce device arrays listed in `reduce` (element type and operation given
+ * per entry; any all-reduce will do, e.g. NCCL's, ordered after the phase on the stream) before the
+ * next phase starts.  The library itself performs no communication.
+ *   phase 0: ranges of the network input            -> MAX of 2 floats
+ *   phase 1+l: forward of layer l                   -> MAX of the output / next-input ranges
+ *   phase n+1: losses and coefficients, all layers  -> MAX of the dH ranges, SUM of the loss shares
+ *   phase n+2: INT8 dH and local g^W sums, all layers -> SUM of INT32 accW_dump [2][N][K] per layer
+ *   phase n+3: update of every layer from the combined sums
+ * B_local rows per set are rows [row_offset, row_offset + B_local) of the B_total rows per set of the
+ * whole batch.  Layers must be chained (X of layers > 0 NULL), accW_dump of every layer non-NULL (it
+ * carries the sums), and every shard must pass the same descriptors (seed included), lambda and step.
+ * `reduce` has room for FF_DP_MAX_REDUCE entries.  Errors as ff_train_step. */
+#define FF_DP_MAX_REDUCE 96
+enum { FF_DP_F32 = 0, FF_DP_I32 = 1 };
+enum { FF_DP_MAX = 0, FF_DP_SUM = 1 };
+typedef struct ff_dp_reduce {
+  void* dev_ptr;   /* device array to combine in place over the shards */
+  uint64_t count;  /* elements */
+  int32_t dtype;   /* FF_DP_F32 / FF_DP_I32 */
+  int32_t op;      /* FF_DP_MAX / FF_DP_SUM */
+} ff_dp_reduce;
+int ff_dp_phase_count(int n_layers);
+ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B_local,
+                            int B_total, int row_offset, int phase, float lambda, uint64_t step, void* cuda_stream,
+                            ff_dp_reduce* reduce, int* n_reduce);
+
 /* Launch-sequence replay for ff_train_step (the paper's edge setting, batch 32 in Sec. V, makes a step a
  * chain of short kernels whose cost is launch overhead; it states no counterpart of this switch).
  * on = 1: the first ff_train_step call of a call shape runs its kernels one by one, the second is

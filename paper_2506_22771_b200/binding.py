@@ -19,7 +19,7 @@ FF_A_X_POS, FF_A_X_NEG, FF_A_W, FF_A_DH_POS, FF_A_DH_NEG, FF_A_XNEXT_POS, FF_A_X
 FF_ABSMAX_LEN = 8
 
 EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", "ff_set_gemm_path", "ff_set_tensor_form",
-           "ff_set_graph_mode", "ff_graph_replay_count",
+           "ff_set_graph_mode", "ff_graph_replay_count", "ff_dp_phase_count", "ff_dp_train_phase",
            "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step",
            "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
            "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict"]
@@ -40,6 +40,15 @@ class ff_layer_bufs(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
                 ("W", "X", "Y", "G", "Xnext", "Xq", "Wq", "dHq", "absmax", "S", "rowmax", "coef",
                  "loss", "acc_dump", "accW_dump")]
+
+
+FF_DP_MAX_REDUCE = 96
+FF_DP_F32, FF_DP_I32 = 0, 1
+FF_DP_MAX, FF_DP_SUM = 0, 1
+
+
+class ff_dp_reduce(C.Structure):
+    _fields_ = [("dev_ptr", C.c_void_p), ("count", C.c_uint64), ("dtype", C.c_int32), ("op", C.c_int32)]
 
 
 class FFError(RuntimeError):
@@ -73,6 +82,9 @@ def load(build_if_missing: bool = True):
     lib.ff_set_gemm_path.argtypes = [vp, i32]
     lib.ff_set_tensor_form.argtypes = [vp, i32]
     lib.ff_set_graph_mode.argtypes = [vp, i32]
+    lib.ff_dp_phase_count.argtypes = [i32]
+    lib.ff_dp_train_phase.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, i32, i32, i32, i32, f32,
+                                      u64, vp, C.POINTER(ff_dp_reduce), C.POINTER(i32)]
     lib.ff_layer_forward.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, u64, vp]
     lib.ff_layer_loss_grad.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32,
                                        C.POINTER(vp), C.POINTER(f32), i32, f32, u64, vp]
@@ -92,7 +104,7 @@ def load(build_if_missing: bool = True):
                                         C.c_char_p, C.c_size_t]
     lib.ff_profile_stop.argtypes = [vp, vp, C.POINTER(f32), C.POINTER(C.c_uint32)]
     for name in EXPORTS:
-        if name not in ("ff_last_error", "ff_launch_count", "ff_graph_replay_count"):
+        if name not in ("ff_last_error", "ff_launch_count", "ff_graph_replay_count", "ff_dp_phase_count"):
             getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -158,6 +170,21 @@ def ff_layer_update(ctx, desc, bufs, B: int, stream: int = 0):
 def ff_train_step(ctx, descs_arr, bufs_arr, n_layers: int, B: int, lam: float, step: int, stream: int = 0):
     """descs_arr / bufs_arr: ctypes arrays (ff_layer_desc * n), (ff_layer_bufs * n)."""
     _check(ctx, load().ff_train_step(ctx, descs_arr, bufs_arr, n_layers, B, lam, step, stream))
+
+
+def ff_dp_phase_count(n_layers: int) -> int:
+    return int(load().ff_dp_phase_count(n_layers))
+
+
+def ff_dp_train_phase(ctx, descs_arr, bufs_arr, n_layers: int, B_local: int, B_total: int, row_offset: int, phase: int,
+                      lam: float, step: int, stream: int = 0):
+    """One phase of the data-parallel step.  Returns the arrays to combine over the shards before the
+    next phase as a list of (device address, element count, FF_DP_F32 | FF_DP_I32, FF_DP_MAX | FF_DP_SUM)."""
+    red = (ff_dp_reduce * FF_DP_MAX_REDUCE)()
+    n = C.c_int(0)
+    _check(ctx, load().ff_dp_train_phase(ctx, descs_arr, bufs_arr, n_layers, B_local, B_total, row_offset, phase, lam,
+                                         step, stream, red, C.byref(n)))
+    return [(int(red[i].dev_ptr), int(red[i].count), int(red[i].dtype), int(red[i].op)) for i in range(n.value)]
 
 
 def ff_predict(ctx, descs_arr, bufs_arr, n_layers: int, B: int, n_classes: int, first_counted_layer: int, scores: int,
@@ -228,7 +255,7 @@ class LayerBuffers:
     """Torch-allocated device tensors of one layer plus the ff_layer_bufs struct pointing at them."""
 
     def __init__(self, desc: ff_layer_desc, B: int, device, dumps: bool = False, xnext: bool = True,
-                 own_x: bool = True):
+                 own_x: bool = True, accw: bool = False):
         import torch
         st = 2 if (desc.kind == FF_CONV3X3 and desc.stride == 2) else 1
         Rin = desc.H * desc.Wd if desc.kind != FF_LINEAR else 1                    # input rows per sample
@@ -250,7 +277,7 @@ class LayerBuffers:
         self.coef = z((2 * B,), torch.float32)
         self.loss = z((4,), torch.float32)
         self.acc_dump = z((rows, desc.N), torch.int32) if dumps else None
-        self.accW_dump = z((2, desc.N, desc.K), torch.int32) if dumps else None
+        self.accW_dump = z((2, desc.N, desc.K), torch.int32) if (dumps or accw) else None
         p = lambda t: t.data_ptr() if t is not None else None
         self.struct = ff_layer_bufs(p(self.W), p(self.X), p(self.Y), p(self.G), p(self.Xnext), p(self.Xq),
                                     p(self.Wq), p(self.dHq), p(self.absmax), p(self.S), p(self.rowmax),

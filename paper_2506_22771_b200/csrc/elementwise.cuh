@@ -59,7 +59,9 @@ __global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restr
 
 // ---------------------------------------------------------------------------------------------
 // q = clip(round(x * 127/a_p)) for `passes` slices, a_p read from device memory (absmax[p]).
-// Linear element index (over the whole tensor) keys the stochastic rounding.
+// Linear element index (over the whole tensor) keys the stochastic rounding.  When the tensor is one
+// shard of a batch split by rows over several devices, ctr_bias.x / .y (passes 0 / 1) is added to the
+// local index so that the counter is the element's index in the unsplit tensor.
 // grid = (blocks, passes)
 // ---------------------------------------------------------------------------------------------
 // zero_S / zero_rowmax (nullable, zero_n entries): per-sample accumulators of the forward epilogue that
@@ -68,8 +70,10 @@ template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __restrict__ x, int8_t* __restrict__ q,
                                                               size_t n_per_pass, const float* __restrict__ a,
                                                               KeySpec ks, unsigned long long* __restrict__ zero_S = nullptr,
-                                                              int32_t* __restrict__ zero_rowmax = nullptr, int zero_n = 0) {
+                                                              int32_t* __restrict__ zero_rowmax = nullptr, int zero_n = 0,
+                                                              uint2 ctr_bias = uint2{0u, 0u}) {
   const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
+  const uint32_t bias = blockIdx.y ? ctr_bias.y : ctr_bias.x;
   if (zero_S && blockIdx.y == 0)
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < zero_n; i += gridDim.x * blockDim.x) {
       zero_S[i] = 0ull;
@@ -79,7 +83,8 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __res
   const float* xp = x + base;
   int8_t* qp = q + base;
   const float inv = inv_of(a[blockIdx.y]);
-  const bool vec = ((n_per_pass & 3) == 0) && ((((uintptr_t)xp) & 15) == 0) && ((((uintptr_t)qp) & 3) == 0);
+  // (an odd bias would split the element pairs that share one hash differently from the unsplit tensor)
+  const bool vec = ((n_per_pass & 3) == 0) && ((((uintptr_t)xp) & 15) == 0) && ((((uintptr_t)qp) & 3) == 0) && !(bias & 1u);
   size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   size_t stride = (size_t)gridDim.x * blockDim.x;
   if (vec) {
@@ -89,7 +94,7 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __res
 #pragma unroll 4
     for (size_t i = tid; i < n4; i += stride) {
       float4 v = __ldg(x4 + i);
-      uint32_t idx = (uint32_t)(base + (i << 2));
+      uint32_t idx = (uint32_t)(base + (i << 2)) + bias;
       int q0, q1, q2, q3;
       quant_pair<MODE>(v.x, v.y, inv, idx, key, q0, q1);
       quant_pair<MODE>(v.z, v.w, inv, idx + 2, key, q2, q3);
@@ -97,7 +102,7 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __res
     }
   } else {
     for (size_t i = tid; i < n_per_pass; i += stride)
-      qp[i] = (int8_t)quant_one<MODE>(xp[i], inv, (uint32_t)(base + i), key);
+      qp[i] = (int8_t)quant_one<MODE>(xp[i], inv, (uint32_t)(base + i) + bias, key);
   }
 }
 
@@ -162,8 +167,9 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
                                                                float tau, float eps, size_t per_sample,
                                                                size_t per_pass, float* __restrict__ xnext,
                                                                int8_t* __restrict__ xq, const float* __restrict__ a,
-                                                               KeySpec ks) {
+                                                               KeySpec ks, uint2 ctr_bias = uint2{0u, 0u}) {
   const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
+  const uint32_t bias = blockIdx.y ? ctr_bias.y : ctr_bias.x;
   const size_t base = (size_t)blockIdx.y * per_pass;
   const float inv = xq ? inv_of(a[blockIdx.y]) : 0.0f;
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) &&
@@ -185,8 +191,8 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
       if (xnext) *reinterpret_cast<float4*>(xnext + e) = v;
       if (xq) {
         int q0, q1, q2, q3;
-        quant_pair<MODE>(v.x, v.y, inv, (uint32_t)e, key, q0, q1);
-        quant_pair<MODE>(v.z, v.w, inv, (uint32_t)e + 2, key, q2, q3);
+        quant_pair<MODE>(v.x, v.y, inv, (uint32_t)e + bias, key, q0, q1);
+        quant_pair<MODE>(v.z, v.w, inv, (uint32_t)e + bias + 2, key, q2, q3);
         *reinterpret_cast<uint32_t*>(xq + e) = pack4(q0, q1, q2, q3);
       }
     }
@@ -197,7 +203,7 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
       float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(g), eps));
       float v = __fmul_rn(Y[e], r);
       if (xnext) xnext[e] = v;
-      if (xq) xq[e] = (int8_t)quant_one<MODE>(v, inv, (uint32_t)e, key);
+      if (xq) xq[e] = (int8_t)quant_one<MODE>(v, inv, (uint32_t)e + bias, key);
     }
   }
 }
@@ -263,14 +269,16 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
                                                                  float lambda, int B, const int32_t* __restrict__ rowmax,
                                                                  float* __restrict__ absmax, float* __restrict__ coef,
                                                                  float* __restrict__ loss, LossScratch* __restrict__ scratch,
-                                                                 const StepState* __restrict__ ss = nullptr) {
+                                                                 const StepState* __restrict__ ss = nullptr,
+                                                                 int m_total = 0) {
   if (ss) lambda = ss->lambda;  // a step run through the library's own launch sequence keeps lambda in device memory
   __shared__ double red[LOSS_THREADS / 32];
   __shared__ uint32_t redmax[2][LOSS_THREADS / 32];
   __shared__ bool is_last;
   const int M = 2 * B;
   const double lam = (double)lambda;
-  const double inv_m = __ddiv_rn(1.0, (double)M);
+  // the mean of Eq. 1 / Eq. 2 runs over the whole batch: m_total samples when these 2B are one shard of it
+  const double inv_m = __ddiv_rn(1.0, (double)(m_total > 0 ? m_total : M));
   const float s_w = scale_of(absmax[2]);
   const float cpass[2] = {__fmul_rn(scale_of(absmax[0]), s_w), __fmul_rn(scale_of(absmax[1]), s_w)};
   double lsum = 0.0;
@@ -370,8 +378,10 @@ __global__ void __launch_bounds__(EW_THREADS) classify_kernel(LaterLayers layers
 template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) dh_quantize_kernel(const float* __restrict__ Y, const float* __restrict__ coef,
                                                                  const float* __restrict__ absmax, size_t per_sample,
-                                                                 size_t per_pass, int8_t* __restrict__ dHq, KeySpec ks) {
+                                                                 size_t per_pass, int8_t* __restrict__ dHq, KeySpec ks,
+                                                                 uint2 ctr_bias = uint2{0u, 0u}) {
   const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
+  const uint32_t bias = blockIdx.y ? ctr_bias.y : ctr_bias.x;
   const size_t base = (size_t)blockIdx.y * per_pass;
   const float inv = inv_of(absmax[3 + blockIdx.y]);
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)dHq) & 3) == 0);
@@ -386,15 +396,15 @@ __global__ void __launch_bounds__(EW_THREADS) dh_quantize_kernel(const float* __
       const float k2 = __fmul_rn(2.0f, __ldg(cp + cur.sample));
       const float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
       int q0, q1, q2, q3;
-      quant_pair<MODE>(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, (uint32_t)e, key, q0, q1);
-      quant_pair<MODE>(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, (uint32_t)e + 2, key, q2, q3);
+      quant_pair<MODE>(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, (uint32_t)e + bias, key, q0, q1);
+      quant_pair<MODE>(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, (uint32_t)e + bias + 2, key, q2, q3);
       *reinterpret_cast<uint32_t*>(dHq + e) = pack4(q0, q1, q2, q3);
     }
   } else {
     for (size_t i = tid; i < per_pass; i += stride) {
       size_t e = base + i;
       float k2 = __fmul_rn(2.0f, coef[(uint32_t)e / (uint32_t)per_sample]);
-      dHq[e] = (int8_t)quant_one<MODE>(__fmul_rn(k2, Y[e]), inv, (uint32_t)e, key);
+      dHq[e] = (int8_t)quant_one<MODE>(__fmul_rn(k2, Y[e]), inv, (uint32_t)e + bias, key);
     }
   }
 }

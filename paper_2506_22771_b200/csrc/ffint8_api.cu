@@ -35,6 +35,13 @@ struct ff_ctx {
   };
   std::vector<ProfRec> prof_recs;
   std::vector<cudaEvent_t> prof_pool;
+  // set for the duration of a data-parallel phase call: the 2B rows at hand are rows [row_off, row_off + B)
+  // of each set of a batch of B_total rows per set (B_total == 0: the batch is not split)
+  struct Shard {
+    int B_total = 0;
+    int row_off = 0;
+  } shard;
+  bool accumulate_only = false;  // weight-gradient contractions leave their INT32 sums in accW_dump, no update
   // captured launch sequences of ff_train_step (ff_set_graph_mode)
   bool graph_mode = false;
   struct GraphEntry {
@@ -183,6 +190,14 @@ ff_status ensure_status(ff_ctx* ctx, cudaStream_t st) {
   return FF_OK;
 }
 
+// Offsets that turn a shard's local element index into the index in the unsplit [2][B_total][per_sample]
+// tensor (the stochastic-rounding counter), for the positive and the negative pass.
+inline uint2 ctr_bias(const ff_ctx* ctx, size_t per_sample, int B) {
+  if (!ctx->shard.B_total) return uint2{0u, 0u};
+  const uint32_t off = (uint32_t)((size_t)ctx->shard.row_off * per_sample);
+  return uint2{off, (uint32_t)((size_t)(ctx->shard.B_total - B) * per_sample) + off};
+}
+
 inline int ew_blocks(ff_ctx* ctx, size_t work_items, int per_thread = 4) {
   size_t need = (work_items + (size_t)EW_THREADS * per_thread - 1) / ((size_t)EW_THREADS * per_thread);
   size_t cap = (size_t)ctx->sm_count * 8;
@@ -238,9 +253,17 @@ inline int simt_split_count(int clen, int splits) {
 ff_status launch_slab_update(ff_ctx* ctx, const int32_t* slabs, int splits, const ff_layer_desc& L, const ff_layer_bufs& b,
                              cudaStream_t st, int pitch = 0) {
   const size_t plane = (size_t)L.N * L.K;
-  const size_t want = (plane + 31) / 32, cap = (size_t)ctx->sm_count * 8;
-  slab_update_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, L.K, pitch ? pitch : L.K, b.W,
-                                                                          b.absmax, L.lr, b.accW_dump);
+  float* W = ctx->accumulate_only ? nullptr : b.W;
+  int32_t* dump = b.accW_dump == slabs ? nullptr : b.accW_dump;  // the sums already are where they would be copied to
+  if (!W && !dump) return FF_OK;
+  if (splits <= 2 && (pitch == 0 || pitch == L.K) && (plane & 3) == 0 && plane >= ((size_t)1 << 18)) {
+    const size_t want = (plane / 4 + 255) / 256, cap = (size_t)ctx->sm_count * 8;
+    slab_update_flat_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, W, b.absmax, L.lr, dump);
+  } else {
+    const size_t want = (plane + 31) / 32, cap = (size_t)ctx->sm_count * 8;
+    slab_update_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, L.K, pitch ? pitch : L.K, W,
+                                                                            b.absmax, L.lr, dump);
+  }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
@@ -382,7 +405,11 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
   }
   if (tc_ok && ctx->gemm_path != FF_GEMM_SIMT && L.kind != FF_CONV3X3) {
     ProfScope prof(ctx, FF_K_UPD_GEMM, st);
-    ff_status s = tc_update(ctx->tc, L, b, B * R, status_ptr(ctx), st);
+    int used = 0;
+    // accumulate only: one unsplit contraction whose single slab [2][N][K] is accW_dump itself
+    ff_status s = ctx->accumulate_only ? tc_dense_update_slab(ctx->tc, b.dHq, L.N, b.Xq, L.K, B * R, b.accW_dump, 1, &used,
+                                                              status_ptr(ctx), st)
+                                       : tc_update(ctx->tc, L, b, B * R, status_ptr(ctx), st);
     if (s != FF_OK) return fail(ctx, s, "tensor-core weight-gradient launch failed: %s", ctx->tc.err);
     ctx->launches++;
     return FF_OK;
@@ -428,6 +455,12 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     }
     return s;
   }
+  if (ctx->accumulate_only) {
+    SlabEpilogue epi{b.accW_dump, L.N, L.K};
+    if (L.kind != FF_CONV3X3)
+      return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st);
+    return launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st);
+  }
   UpdateEpilogue epi{b.W, b.accW_dump, b.absmax, L.lr, L.N, L.K};
   if (L.kind != FF_CONV3X3)
     return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st);
@@ -468,22 +501,28 @@ ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
   return FF_OK;
 }
 
-ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
-  const size_t per_pass = (size_t)B * in_rows_per_sample(L) * in_features(L);
-  {
+ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st,
+                         bool do_absmax = true, bool do_quantize = true) {
+  const size_t per_sample = (size_t)in_rows_per_sample(L) * in_features(L);
+  const size_t per_pass = (size_t)B * per_sample;
+  if (do_absmax) {
     ProfScope prof(ctx, FF_K_ABSMAX, st);
     absmax_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(b.X, per_pass, b.absmax + FF_A_X_POS,
                                                                                  status_ptr(ctx));
   }
-  FF_LAUNCH_CHECK(ctx);
+  if (do_absmax) FF_LAUNCH_CHECK(ctx);
+  if (!do_quantize) return FF_OK;
   {
     ProfScope prof(ctx, FF_K_QUANTIZE, st);
     const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
     const KeySpec key = make_key_spec(L.seed, ROLE_X, L.index, step_ptr(ctx));
+    const uint2 bias = ctr_bias(ctx, per_sample, B);
     if (L.round_x == FF_ROUND_NEAREST_EVEN)
-      quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, key);
+      quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, key, nullptr,
+                                                                 nullptr, 0, bias);
     else
-      quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, key);
+      quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, key, nullptr,
+                                                                    nullptr, 0, bias);
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -500,19 +539,21 @@ ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
   {
     ProfScope prof(ctx, FF_K_NORMALIZE, st);
     const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
+    const uint2 bias = ctr_bias(ctx, per_sample, B);
     if (!next || next->round_x == FF_ROUND_NEAREST_EVEN)
       normalize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
-                                                                  xq_next, b.absmax + FF_A_XNEXT_POS, key);
+                                                                  xq_next, b.absmax + FF_A_XNEXT_POS, key, bias);
     else
       normalize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
-                                                                     xq_next, b.absmax + FF_A_XNEXT_POS, key);
+                                                                     xq_next, b.absmax + FF_A_XNEXT_POS, key, bias);
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
 
 ff_status loss_grad_impl(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, const float* const* G_later,
-                         const float* theta_later, int n_later, float lambda, cudaStream_t st) {
+                         const float* theta_later, int n_later, float lambda, cudaStream_t st, bool do_loss = true,
+                         bool do_dh = true) {
   LaterLayers later;
   later.n = n_later;
   for (int j = 0; j < n_later; ++j) {
@@ -521,23 +562,27 @@ ff_status loss_grad_impl(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
   }
   int loss_blocks = (2 * B + LOSS_THREADS - 1) / LOSS_THREADS;
   if (loss_blocks > LOSS_MAX_BLOCKS) loss_blocks = LOSS_MAX_BLOCKS;
-  {
+  if (do_loss) {
     ProfScope prof(ctx, FF_K_LOSS, st);
     loss_coef_kernel<<<loss_blocks, LOSS_THREADS, 0, st>>>(
         b.G, L.theta, later, lambda, B, b.rowmax, b.absmax, b.coef, b.loss,
-        reinterpret_cast<LossScratch*>(static_cast<char*>(ctx->workspace) + WS_LOSS_OFFSET), step_ptr(ctx));
+        reinterpret_cast<LossScratch*>(static_cast<char*>(ctx->workspace) + WS_LOSS_OFFSET), step_ptr(ctx),
+        2 * ctx->shard.B_total);
   }
-  FF_LAUNCH_CHECK(ctx);
+  if (do_loss) FF_LAUNCH_CHECK(ctx);
+  if (!do_dh) return FF_OK;
   const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
   const size_t per_pass = per_sample * B;
   {
     ProfScope prof(ctx, FF_K_DH_QUANTIZE, st);
     const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
     const KeySpec key = make_key_spec(L.seed, ROLE_DH, L.index, step_ptr(ctx));
+    const uint2 bias = ctr_bias(ctx, per_sample, B);
     if (L.round_dh == FF_ROUND_NEAREST_EVEN)
-      dh_quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key);
+      dh_quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key, bias);
     else
-      dh_quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key);
+      dh_quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key,
+                                                                       bias);
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -595,6 +640,73 @@ ff_status train_step_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_lay
     if ((s = loss_grad_impl(ctx, layers[l], bufs[l], B, Gl, th, n_later, lambda, st)) != FF_OK) return s;
     if ((s = run_update_gemm(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
   }
+  return FF_OK;
+}
+
+// One phase of the data-parallel step (see ff_dp_train_phase); ctx->shard is set by the caller.
+ff_status dp_phase_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n, int B, int phase,
+                        float lambda, cudaStream_t st, ff_dp_reduce* red, int* n_red) {
+  ff_status s;
+  int nr = 0;
+  auto want = [&](void* p, uint64_t count, int dtype, int op) {
+    red[nr].dev_ptr = p;
+    red[nr].count = count;
+    red[nr].dtype = dtype;
+    red[nr].op = op;
+    ++nr;
+  };
+  if (phase == 0) {
+    // ranges of the network input: local maxima now, the maximum over the shards before phase 1
+    for (int l = 0; l < n; ++l) FF_CUDA(ctx, cudaMemsetAsync(bufs[l].absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
+    if ((s = quantize_input(ctx, layers[0], bufs[0], B, st, true, false)) != FF_OK) return s;
+    want(bufs[0].absmax + FF_A_X_POS, 2, FF_DP_F32, FF_DP_MAX);
+  } else if (phase <= n) {
+    // forward of layer l; its input range is global by now, the range of its normalised output becomes so after the phase
+    const int l = phase - 1;
+    if (l == 0)
+      s = quantize_input(ctx, layers[0], bufs[0], B, st, false, true);
+    else
+      s = normalize_output(ctx, layers[l - 1], bufs[l - 1], B, bufs[l].Xq, &layers[l], st);
+    if (s != FF_OK) return s;
+    const bool feeds_next = l + 1 < n;
+    if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st)) != FF_OK)
+      return s;
+    want(bufs[l].absmax + FF_A_XNEXT_POS, 2, FF_DP_F32, FF_DP_MAX);
+    if (feeds_next) want(bufs[l + 1].absmax + FF_A_X_POS, 2, FF_DP_F32, FF_DP_MAX);
+  } else if (phase == n + 1) {
+    // FP32 output of the last layer (if asked for); losses and coefficients of all layers from the local G's
+    if ((s = normalize_output(ctx, layers[n - 1], bufs[n - 1], B, nullptr, nullptr, st)) != FF_OK) return s;
+    for (int l = 0; l < n; ++l) {
+      const float* Gl[FF_MAX_LATER];
+      float th[FF_MAX_LATER];
+      const int n_later = n - 1 - l;
+      for (int j = 0; j < n_later; ++j) {
+        Gl[j] = bufs[l + 1 + j].G;
+        th[j] = layers[l + 1 + j].theta;
+      }
+      if ((s = loss_grad_impl(ctx, layers[l], bufs[l], B, Gl, th, n_later, lambda, st, true, false)) != FF_OK) return s;
+      want(bufs[l].absmax + FF_A_DH_POS, 2, FF_DP_F32, FF_DP_MAX);   // range of dH over the whole batch
+      want(bufs[l].loss, 1, FF_DP_F32, FF_DP_SUM);                    // each shard holds its share of the batch mean
+    }
+  } else if (phase == n + 2) {
+    // INT8 output gradient and the local INT32 weight-gradient sums of every layer
+    ctx->accumulate_only = true;
+    for (int l = 0; l < n; ++l) {
+      s = loss_grad_impl(ctx, layers[l], bufs[l], B, nullptr, nullptr, 0, lambda, st, false, true);
+      if (s == FF_OK) s = run_update_gemm(ctx, layers[l], bufs[l], B, st);
+      if (s != FF_OK) break;
+      want(bufs[l].accW_dump, (uint64_t)2 * layers[l].N * layers[l].K, FF_DP_I32, FF_DP_SUM);
+    }
+    ctx->accumulate_only = false;
+    if (s != FF_OK) return s;
+  } else {
+    // the sums are those of the whole batch now: the same update on every device keeps the weights identical
+    for (int l = 0; l < n; ++l) {
+      ProfScope prof(ctx, FF_K_UPD_GEMM, st);
+      if ((s = launch_slab_update(ctx, bufs[l].accW_dump, 1, layers[l], bufs[l], st)) != FF_OK) return s;
+    }
+  }
+  *n_red = nr;
   return FF_OK;
 }
 
@@ -840,6 +952,37 @@ ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
   if ((s = set_step(ctx, step, lambda, true, st)) != FF_OK) return s;
   if (ctx->graph_mode && !ctx->profiling) return train_step_graph(ctx, layers, bufs, n_layers, B, lambda, st);
   return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+}
+
+int ff_dp_phase_count(int n_layers) { return n_layers > 0 ? n_layers + 4 : 0; }
+
+ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B_local,
+                            int B_total, int row_offset, int phase, float lambda, uint64_t step, void* cuda_stream,
+                            ff_dp_reduce* reduce, int* n_reduce) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if (!reduce || !n_reduce) return fail(ctx, FF_ERR_ARG, "reduce / n_reduce is NULL");
+  *n_reduce = 0;
+  if ((s = check_layer_list(ctx, layers, bufs, n_layers, B_local)) != FF_OK) return s;
+  if (B_total < B_local || row_offset < 0 || row_offset > B_total - B_local)
+    return fail(ctx, FF_ERR_ARG, "rows [row_offset, row_offset + B_local) do not lie inside the batch of B_total");
+  if (phase < 0 || phase >= ff_dp_phase_count(n_layers)) return fail(ctx, FF_ERR_ARG, "phase out of range");
+  for (int l = 0; l < n_layers; ++l) {
+    // counters, row counts and the INT32 weight-gradient range are those of the whole batch
+    if ((s = check_layer(ctx, &layers[l], B_total)) != FF_OK) return s;
+    if (l > 0 && bufs[l].X) return fail(ctx, FF_ERR_ARG, "a data-parallel step takes chained layers (X of layers > 0 NULL)");
+    if (!bufs[l].accW_dump) return fail(ctx, FF_ERR_ARG, "a data-parallel step needs accW_dump of every layer");
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  if ((s = set_step(ctx, step, lambda, true, st)) != FF_OK) return s;
+  ctx->shard.B_total = B_total;
+  ctx->shard.row_off = row_offset;
+  s = dp_phase_body(ctx, layers, bufs, n_layers, B_local, phase, lambda, st, reduce, n_reduce);
+  ctx->shard.B_total = 0;
+  ctx->shard.row_off = 0;
+  ctx->accumulate_only = false;
+  return s;
 }
 
 ff_status ff_set_graph_mode(ff_ctx* ctx, int on) {

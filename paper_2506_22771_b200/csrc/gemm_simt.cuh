@@ -190,7 +190,8 @@ struct SlabEpilogue {
 // Alg. 1 line 9): W <- W - lr*(float(accP)*cP + float(accN)*cN).  plane = rows*cols elements of W;
 // the slabs may have a wider row pitch (cols <= pitch).  A block covers 32 consecutive elements; its
 // 8 warps take the splits round-robin (coalesced along the elements) and their integer partial
-// sums meet in shared memory.
+// sums meet in shared memory.  W == NULL: no update, only the sums are written to accW_dump (dense
+// [2][rows][cols]) - the buffer a data-parallel step adds up over the devices before it updates.
 __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane, int cols,
                                                           int pitch, float* __restrict__ W, const float* __restrict__ absmax,
                                                           float lr, int32_t* __restrict__ accW_dump) {
@@ -218,14 +219,48 @@ __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restr
         aP += part[0][k][lane];
         aN += part[1][k][lane];
       }
-      const float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
-      W[e] = __fsub_rn(W[e], __fmul_rn(lr, g));
+      if (W) {
+        const float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
+        W[e] = __fsub_rn(W[e], __fmul_rn(lr, g));
+      }
       if (accW_dump) {
         accW_dump[e] = aP;
         accW_dump[plane + e] = aN;
       }
     }
     __syncthreads();
+  }
+}
+
+// The same for one or two slabs of a large output (dense rows, cols % 4 == 0): nothing to share between
+// warps, so every thread takes four consecutive elements with 128-bit accesses.
+__global__ void __launch_bounds__(256) slab_update_flat_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane,
+                                                               float* __restrict__ W, const float* __restrict__ absmax, float lr,
+                                                               int32_t* __restrict__ accW_dump) {
+  const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
+  const float cN = __fmul_rn(scale_of(absmax[4]), scale_of(absmax[1]));
+  const size_t n4 = plane >> 2, stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    int4 aP = __ldcs(reinterpret_cast<const int4*>(slabs) + i);
+    int4 aN = __ldcs(reinterpret_cast<const int4*>(slabs + plane) + i);
+    for (int z = 1; z < splits; ++z) {
+      const int4 bP = __ldcs(reinterpret_cast<const int4*>(slabs + (size_t)z * 2 * plane) + i);
+      const int4 bN = __ldcs(reinterpret_cast<const int4*>(slabs + ((size_t)z * 2 + 1) * plane) + i);
+      aP.x += bP.x, aP.y += bP.y, aP.z += bP.z, aP.w += bP.w;
+      aN.x += bN.x, aN.y += bN.y, aN.z += bN.z, aN.w += bN.w;
+    }
+    if (W) {
+      float4 w = reinterpret_cast<const float4*>(W)[i];
+      w.x = __fsub_rn(w.x, __fmul_rn(lr, __fadd_rn(__fmul_rn(__int2float_rn(aP.x), cP), __fmul_rn(__int2float_rn(aN.x), cN))));
+      w.y = __fsub_rn(w.y, __fmul_rn(lr, __fadd_rn(__fmul_rn(__int2float_rn(aP.y), cP), __fmul_rn(__int2float_rn(aN.y), cN))));
+      w.z = __fsub_rn(w.z, __fmul_rn(lr, __fadd_rn(__fmul_rn(__int2float_rn(aP.z), cP), __fmul_rn(__int2float_rn(aN.z), cN))));
+      w.w = __fsub_rn(w.w, __fmul_rn(lr, __fadd_rn(__fmul_rn(__int2float_rn(aP.w), cP), __fmul_rn(__int2float_rn(aN.w), cN))));
+      reinterpret_cast<float4*>(W)[i] = w;
+    }
+    if (accW_dump) {
+      reinterpret_cast<int4*>(accW_dump)[i] = aP;
+      reinterpret_cast<int4*>(accW_dump + plane)[i] = aN;
+    }
   }
 }
 

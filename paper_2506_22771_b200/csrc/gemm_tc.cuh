@@ -704,22 +704,40 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           atomicMax(p.rowmax + sample, mx);
         }
       } else if (MODE == TC_MODE_SLAB) {
-        // raw INT32 partial sums of both sets to this split's slab [split][set][rows][cols]
+        // raw INT32 partial sums of both sets to this split's slab [split][set][rows][cols].  A thread
+        // holds one accumulator row; the 32 x 32 chunk is turned through a swizzled smem patch so that each
+        // store instruction of the warp writes four whole 128-byte row segments.
+        uint8_t* patch = patch0;
         for (int pass = 0; pass < 2; ++pass) {
           int32_t* slab = p.slabs + (size_t)(split * 2 + pass) * p.out_rows * p.out_cols;
-#pragma unroll 1
-          for (int cb = cbeg; cb < cend; cb += 32) {
-            int v[32];
-            tc_ld32(t_row + pass * TC_BN + cb, v);
-            if (row_ok) {
-              int32_t* dst = slab + (size_t)row * p.out_cols + col0 + cb;
+          int v[2][32];
+          if (cbeg < cend) tc_ld32_async(t_row + pass * TC_BN + cbeg, v[0]);
+#pragma unroll
+          for (int i = 0; i < TC_EPI_COLS / 32; ++i) {
+            const int cb = cbeg + i * 32;
+            if (cb < cend) tc_wait_ld(v[i & 1]);
+            if (i + 1 < TC_EPI_COLS / 32 && cb + 32 < cend) tc_ld32_async(t_row + pass * TC_BN + cb + 32, v[(i + 1) & 1]);
+            if (cb < cend) {  // uniform across the warp
+              const int(&a)[32] = v[i & 1];
               if (col0 + cb + 32 <= p.out_cols && (p.out_cols & 3) == 0) {
 #pragma unroll
-                for (int j = 0; j < 32; j += 4) *reinterpret_cast<int4*>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-              } else {
+                for (int j = 0; j < 32; j += 4)
+                  *reinterpret_cast<int4*>(patch + lane * 128 + (((j >> 2) ^ (lane & 7)) << 4)) =
+                      make_int4(a[j], a[j + 1], a[j + 2], a[j + 3]);
+                __syncwarp();
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                  const int r = q * 4 + (lane >> 3), cc = lane & 7;
+                  if (wrow0 + r < p.out_rows)
+                    *reinterpret_cast<int4*>(slab + (size_t)(wrow0 + r) * p.out_cols + col0 + cb + cc * 4) =
+                        *reinterpret_cast<const int4*>(patch + r * 128 + ((cc ^ (r & 7)) << 4));
+                }
+                __syncwarp();
+              } else if (row_ok) {
+                int32_t* dst = slab + (size_t)row * p.out_cols + col0 + cb;
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
-                  if (col0 + cb + j < p.out_cols) dst[j] = v[j];
+                  if (col0 + cb + j < p.out_cols) dst[j] = a[j];
               }
             }
           }
@@ -1185,7 +1203,9 @@ inline ff_status tc_dense_update_slab(TcState& t, const int8_t* dHq, int N, cons
   *splits_out = cdiv(p.kblocks, kb_per_split);
   if ((s = tc_make_map(t, &ta, dHq, N, rows_per_pass, 2, 128, 128)) != FF_OK) return s;
   if ((s = tc_make_map(t, &tb, xi, kcols, rows_per_pass, 2, 128, 128)) != FF_OK) return s;
-  return tc_launch<TC_MODE_SLAB, true, 128>(t, 1, ta, tb, p, st);
+  // one split: a large output with tiles for every SM, where CTA pairs pay; several: a small output, single CTAs
+  const int ncta = t.force_ncta ? t.force_ncta : (splits == 1 ? tc_pick_ncta(t, N, kcols) : 1);
+  return tc_launch<TC_MODE_SLAB, true, 128>(t, ncta, ta, tb, p, st);
 }
 
 }  // namespace ffi8

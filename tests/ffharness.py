@@ -75,7 +75,8 @@ def compare_layer(st: O.LayerState, b, spec, B, check_dumps=True, tag=""):
     eq("G", _np(b.G), st.G)
     if b.Xnext is not None:
         eq("Xnext", _np(b.Xnext).reshape(-1), st.Xnext.reshape(-1))
-        eq("a_xnext", am[5:7], np.array([O.absmax(st.Xnext[:B]), O.absmax(st.Xnext[B:])], dtype=np.float32))
+        a_xn = getattr(st, "a_xnext_full", None) or (O.absmax(st.Xnext[:B]), O.absmax(st.Xnext[B:]))
+        eq("a_xnext", am[5:7], np.array(a_xn, dtype=np.float32))
     if st.coef is not None:
         eq("coef", _np(b.coef), st.coef)
         eq("a_dh", am[3:5], np.array(st.a_dh, dtype=np.float32))
@@ -102,3 +103,22 @@ def _assert_equal(name, got, want):
         i = int(bad[0])
         raise AssertionError(f"{name}: {bad.size} of {same.size} elements differ; first at {i}: "
                              f"got {np.atleast_1d(got)[i]!r} want {np.atleast_1d(want)[i]!r}")
+
+
+def shard_state(st: O.LayerState, B_total, row_off, B_local):
+    """The part of a whole-batch LayerState that the shard holding samples [row_off, row_off + B_local)
+    of each set must reproduce: per-sample arrays (first axis = sample) cut to those samples; ranges,
+    loss, weight-gradient sums and new weights are those of the whole batch."""
+    import copy
+
+    def cut(a):
+        if a is None:
+            return None
+        a = np.asarray(a)
+        return np.concatenate([a[row_off:row_off + B_local], a[B_total + row_off:B_total + row_off + B_local]], 0)
+
+    out = copy.copy(st)
+    for name in ("Xq", "acc", "Y", "Xnext", "dHq", "S", "rowmax", "G", "coef"):
+        setattr(out, name, cut(getattr(st, name)))
+    out.a_xnext_full = (O.absmax(st.Xnext[:B_total]), O.absmax(st.Xnext[B_total:]))
+    return out

@@ -62,3 +62,72 @@ def test_algorithmic_work_of_the_roofline_workload():
     assert work["fwd_gemm"] == 2.0 * M * N * K and work["upd_gemm"] == 2.0 * M * N * K
     assert work["absmax"] == 4.0 * (M * K + N * K) and work["quantize"] == 5.0 * (M * K + N * K)
     assert work["dh_quantize"] == 5.0 * M * N and work["normalize"] == 0.0
+
+
+# ---- data-parallel step: the plumbing around the library's phases -----------------------------------
+def _dp_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2506_22771_b200 import binding as ffb
+    from paper_2506_22771_b200 import data_parallel as dp
+    # stand-ins for one layer's buffers on this rank: a range vector, a loss share, INT32 weight-gradient sums
+    absmax = torch.tensor([0.5 + rank, 3.0 - rank, 0.0, 1.0 + 2 * rank, 0.25, 0.0, 0.0, 0.0])
+    loss = torch.tensor([0.125 * (rank + 1), 0.0, 0.0, 0.0])
+    accw = torch.arange(24, dtype=torch.int32).reshape(2, 3, 4) * (1 if rank == 0 else -3)
+    table = dp.PointerTable([absmax, loss, accw])
+    entries = [(absmax.data_ptr(), 2, ffb.FF_DP_F32, ffb.FF_DP_MAX),           # input ranges
+               (absmax.data_ptr() + 12, 2, ffb.FF_DP_F32, ffb.FF_DP_MAX),      # dH ranges (elements 3, 4)
+               (loss.data_ptr(), 1, ffb.FF_DP_F32, ffb.FF_DP_SUM),
+               (accw.data_ptr(), 24, ffb.FF_DP_I32, ffb.FF_DP_SUM)]
+    dp.all_reduce_entries(entries, table)
+    out[rank] = (absmax.tolist(), loss.tolist(), accw.reshape(-1).tolist())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_dp_reductions_over_two_ranks():
+    world = 2
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_dp_worker, args=(world, _free_port(), out), nprocs=world, join=True)
+        res = dict(out)
+    for rank in range(world):
+        absmax, loss, accw = res[rank]
+        assert absmax[:2] == [1.5, 3.0] and absmax[3:5] == [3.0, 0.25]
+        assert absmax[2] == 0.0 and absmax[5:] == [0.0, 0.0, 0.0]          # untouched neighbours
+        assert loss == [0.375, 0.0, 0.0, 0.0]
+        assert accw == [-2 * i for i in range(24)]
+
+
+def test_shard_rows_cover_the_batch_once():
+    from paper_2506_22771_b200 import data_parallel as dp
+    for B, world in [(16384, 8), (200, 3), (5, 5), (7, 2)]:
+        spans = [dp.shard_rows(B, world, r) for r in range(world)]
+        assert spans[0][0] == 0 and sum(n for _, n in spans) == B
+        for (o0, n0), (o1, _) in zip(spans, spans[1:]):
+            assert o0 + n0 == o1
+        assert max(n for _, n in spans) - min(n for _, n in spans) <= 1
+
+
+def test_shard_batch_takes_the_same_rows_of_both_sets():
+    import numpy as np
+    from paper_2506_22771_b200 import data_parallel as dp
+    B, per, K = 6, 2, 3                       # 2 rows per sample (e.g. positions of a convolution input)
+    X = np.arange(2 * B * per * K, dtype=np.float32).reshape(2 * B * per, K)
+    got = dp.shard_batch(X, B, 4, 2)
+    want = np.concatenate([X[8:12], X[B * per + 8:B * per + 12]], 0)
+    assert np.array_equal(got, want)
+    assert torch.equal(dp.shard_batch(torch.from_numpy(X), B, 4, 2), torch.from_numpy(want))
+
+
+def test_pointer_table_rejects_foreign_addresses_and_types():
+    import pytest
+    from paper_2506_22771_b200 import binding as ffb
+    from paper_2506_22771_b200 import data_parallel as dp
+    t = torch.zeros(8, dtype=torch.float32)
+    table = dp.PointerTable([t])
+    assert table.view(t.data_ptr() + 8, 3, ffb.FF_DP_F32).data_ptr() == t.data_ptr() + 8
+    with pytest.raises(KeyError):
+        table.view(t.data_ptr() + 24, 4, ffb.FF_DP_F32)      # runs past the end
+    with pytest.raises(TypeError):
+        table.view(t.data_ptr(), 2, ffb.FF_DP_I32)
