@@ -128,6 +128,22 @@ ff_status ff_set_gemm_path(ff_ctx* ctx, int path);
  * output has more than 128 rows), 1 / 2 force one form.  Identical bits. */
 ff_status ff_set_tensor_form(ff_ctx* ctx, int ctas_per_tile);
 
+/* Positive / negative / candidate batches by label embedding (Sec. III: the true label makes a
+ * positive sample, a wrong one a negative; Alg. 1 line 3).  x [B, n] FP32 raw samples (device),
+ * labels [sets, B] INT32 (device; the wrong labels of a negative set are drawn by the caller).
+ * out [sets*B, n] FP32 (device): row s*B + b = sample b with labels[s, b] written one-hot over its
+ * label places - flat positions 0, label_stride, ..., (n_classes-1)*label_stride hold on_value at the
+ * label and zero elsewhere (label_stride = 1 for a vector, = channels for a channels-last image whose
+ * first pixels of channel 0 carry the label).  tau0 > 0: every row is then scaled to length tau0,
+ * r = tau0 / (float(sqrt(sum of squares, FP64)) + eps), one FP32 multiply per element (the sum's
+ * order is free, so rows agree with a reference to FP32 rounding, not always bit for bit); tau0 <= 0:
+ * no scaling.  sets = 2 with (true, wrong) labels gives a training batch for ff_train_step, sets =
+ * n_classes with labels[c, b] = c the candidate batch for ff_predict.  x and out must not overlap.
+ * A label outside [0, n_classes) leaves its row without a hot place and makes the next ff_poll_status
+ * return FF_ERR_RANGE.  Asynchronous on the stream; nothing is allocated. */
+ff_status ff_embed_labels(ff_ctx* ctx, const float* x, const int32_t* labels, int B, int n, int sets, int n_classes,
+                          int label_stride, float on_value, float tau0, float eps, float* out, void* cuda_stream);
+
 /* ---- data-parallel train step --------------------------------------------------------------
  * The batch of one step split by rows over several devices, each holding a replica of the weights:
  * forward, goodness, loss coefficient and output gradient are per sample (Sec. III, Sec. IV-B), so a

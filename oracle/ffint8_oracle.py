@@ -488,6 +488,43 @@ def predict(specs: List[LayerSpec], Ws: List[np.ndarray], X_cand: np.ndarray, B:
 
 
 # --------------------------------------------------------------------------------------
+# Positive / negative (and candidate) batches by label embedding  (Sec. III; Alg. 1 line 3)
+# --------------------------------------------------------------------------------------
+def embed_labels(x: np.ndarray, labels: np.ndarray, n_classes: int, label_stride: int = 1, on_value: float = 1.0,
+                 tau0: float = 0.0, eps: float = 1e-8) -> np.ndarray:
+    """Batches made from B raw samples by writing a label into each (Sec. III: the true label gives the
+    positive sample, a wrong one the negative; Alg. 1 line 3).  x [B, n] float32, labels [sets, B]:
+    output row s*B + b is sample b with labels[s, b] written one-hot over its n_classes label places
+    (flat positions 0, label_stride, 2*label_stride, ...: the place of the label holds on_value, the
+    others zero).  The wrong labels are drawn by the caller and passed in.  With tau0 > 0 every row is
+    then scaled to length tau0: r = tau0 / (float32(sqrt(sum of squares in float64)) + eps), one
+    float32 multiply per element (the first layer's input arrives length-normalised like every other
+    layer's).  Labels outside [0, n_classes) are an error."""
+    x = np.asarray(x, dtype=F32)
+    labels = np.asarray(labels)
+    B, n = x.shape
+    sets = labels.shape[0]
+    if labels.shape != (sets, B):
+        raise ValueError("labels must be [sets, B]")
+    if (labels < 0).any() or (labels >= n_classes).any():
+        raise ValueError("label outside [0, n_classes)")
+    if n_classes <= 0 or label_stride <= 0 or (n_classes - 1) * label_stride >= n:
+        raise ValueError("label places do not fit the sample")
+    out = np.empty((sets * B, n), dtype=F32)
+    for s_ in range(sets):
+        for b_ in range(B):
+            v = x[b_].copy()
+            v[0:n_classes * label_stride:label_stride] = F32(0.0)
+            v[int(labels[s_, b_]) * label_stride] = F32(on_value)
+            if tau0 > 0.0:
+                ss = np.sum(v.astype(F64) * v.astype(F64))
+                r = F32(tau0) / (F32(np.sqrt(ss)) + F32(eps))
+                v = v * F32(r)
+            out[s_ * B + b_] = v
+    return out
+
+
+# --------------------------------------------------------------------------------------
 # Unquantised float64 model of one layer (for the finite-difference pin only)
 # --------------------------------------------------------------------------------------
 def fp64_layer_loss(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int) -> float:

@@ -20,6 +20,7 @@ FF_ABSMAX_LEN = 8
 
 EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", "ff_set_gemm_path", "ff_set_tensor_form",
            "ff_set_graph_mode", "ff_graph_replay_count", "ff_dp_phase_count", "ff_dp_train_phase",
+           "ff_embed_labels",
            "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step",
            "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
            "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict"]
@@ -82,6 +83,7 @@ def load(build_if_missing: bool = True):
     lib.ff_set_gemm_path.argtypes = [vp, i32]
     lib.ff_set_tensor_form.argtypes = [vp, i32]
     lib.ff_set_graph_mode.argtypes = [vp, i32]
+    lib.ff_embed_labels.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, f32, vp, vp]
     lib.ff_dp_phase_count.argtypes = [i32]
     lib.ff_dp_train_phase.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, i32, i32, i32, i32, f32,
                                       u64, vp, C.POINTER(ff_dp_reduce), C.POINTER(i32)]
@@ -170,6 +172,13 @@ def ff_layer_update(ctx, desc, bufs, B: int, stream: int = 0):
 def ff_train_step(ctx, descs_arr, bufs_arr, n_layers: int, B: int, lam: float, step: int, stream: int = 0):
     """descs_arr / bufs_arr: ctypes arrays (ff_layer_desc * n), (ff_layer_bufs * n)."""
     _check(ctx, load().ff_train_step(ctx, descs_arr, bufs_arr, n_layers, B, lam, step, stream))
+
+
+def ff_embed_labels(ctx, x: int, labels: int, B: int, n: int, sets: int, n_classes: int, label_stride: int,
+                    on_value: float, tau0: float, eps: float, out: int, stream: int = 0):
+    """x / labels / out are device addresses (see include/ffint8.h)."""
+    _check(ctx, load().ff_embed_labels(ctx, x, labels, B, n, sets, n_classes, label_stride, on_value, tau0, eps, out,
+                                       stream))
 
 
 def ff_dp_phase_count(n_layers: int) -> int:

@@ -11,6 +11,7 @@ namespace ffi8 {
 // device status word bits (OR-ed by kernels, read by ff_poll_status)
 constexpr uint32_t ST_NONFINITE = 1u;
 constexpr uint32_t ST_TIMEOUT = 2u;
+constexpr uint32_t ST_BADLABEL = 4u;   // a label outside [0, n_classes) met by the label-embedding kernel
 
 constexpr int ROUND_NEAREST = 0;
 constexpr int ROUND_STOCHASTIC = 1;

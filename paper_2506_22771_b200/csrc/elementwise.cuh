@@ -409,4 +409,85 @@ __global__ void __launch_bounds__(EW_THREADS) dh_quantize_kernel(const float* __
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Positive / negative / candidate batches by label embedding (Sec. III; Alg. 1 line 3).
+// x [B, n] raw samples, labels [sets, B]; out row s*B + b = sample b with labels[s, b] written
+// one-hot over the label places (flat positions j*label_stride, j < n_classes: on_value at the label,
+// zero elsewhere), then, if tau0 > 0, scaled to length tau0 with
+// r = tau0 / (float(sqrt(sum of squares in FP64)) + eps).  The squares of the data entries are summed
+// once per sample and shared by all sets.  One block per sample (grid-stride).
+// ---------------------------------------------------------------------------------------------
+constexpr int EMBED_THREADS = 256;
+__global__ void __launch_bounds__(EMBED_THREADS) embed_labels_kernel(const float* __restrict__ x, const int32_t* __restrict__ labels,
+                                                                     int B, int n, int sets, int n_classes, int label_stride,
+                                                                     float on_value, float tau0, float eps,
+                                                                     float* __restrict__ out, uint32_t* __restrict__ status) {
+  __shared__ double red[EMBED_THREADS / 32];
+  __shared__ double total;
+  const int span = (n_classes - 1) * label_stride + 1;      // flat positions below this may be label places
+  const int head = min(n, (span + 3) & ~3);                  // handled element by element
+  const bool vec = ((n & 3) == 0) && ((((uintptr_t)x) & 15) == 0) && ((((uintptr_t)out) & 15) == 0);
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  for (int b = blockIdx.x; b < B; b += gridDim.x) {
+    const float* xr = x + (size_t)b * n;
+    double ss = 0.0;
+    if (tau0 > 0.0f) {
+      for (int k = threadIdx.x; k < head; k += EMBED_THREADS) {
+        const bool place = k < span && (k % label_stride) == 0;
+        const double v = place ? 0.0 : (double)xr[k];
+        ss = fma(v, v, ss);  // the square of a float is exact in double: the fused form rounds once like the sum
+      }
+      if (vec) {
+        for (int k = head + 4 * threadIdx.x; k < n; k += 4 * EMBED_THREADS) {
+          const float4 v = __ldg(reinterpret_cast<const float4*>(xr + k));
+          ss += (double)v.x * v.x + (double)v.y * v.y + (double)v.z * v.z + (double)v.w * v.w;
+        }
+      } else {
+        for (int k = head + threadIdx.x; k < n; k += EMBED_THREADS) ss += (double)xr[k] * xr[k];
+      }
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_down_sync(0xffffffffu, ss, o);
+      if (lane == 0) red[wid] = ss;
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int i = 0; i < EMBED_THREADS / 32; ++i) t += red[i];
+        total = t;
+      }
+      __syncthreads();
+    }
+    for (int s = 0; s < sets; ++s) {
+      int lab = labels[(size_t)s * B + b];
+      const bool good = lab >= 0 && lab < n_classes;
+      if (!good && threadIdx.x == 0) atomicOr(status, ST_BADLABEL);
+      const int hot = good ? lab * label_stride : -1;
+      float r = 1.0f;
+      if (tau0 > 0.0f) {
+        const double sq = total + (good ? (double)on_value * (double)on_value : 0.0);
+        r = __fdiv_rn(tau0, __fadd_rn(__double2float_rn(sqrt(sq)), eps));
+      }
+      float* orow = out + ((size_t)s * B + b) * n;
+      for (int k = threadIdx.x; k < head; k += EMBED_THREADS) {
+        const bool place = k < span && (k % label_stride) == 0;
+        const float v = place ? (k == hot ? on_value : 0.0f) : xr[k];
+        orow[k] = tau0 > 0.0f ? __fmul_rn(v, r) : v;
+      }
+      if (vec) {
+        for (int k = head + 4 * threadIdx.x; k < n; k += 4 * EMBED_THREADS) {
+          float4 v = __ldg(reinterpret_cast<const float4*>(xr + k));
+          if (tau0 > 0.0f) {
+            v.x = __fmul_rn(v.x, r);
+            v.y = __fmul_rn(v.y, r);
+            v.z = __fmul_rn(v.z, r);
+            v.w = __fmul_rn(v.w, r);
+          }
+          __stcs(reinterpret_cast<float4*>(orow + k), v);
+        }
+      } else {
+        for (int k = head + threadIdx.x; k < n; k += EMBED_THREADS) orow[k] = tau0 > 0.0f ? __fmul_rn(xr[k], r) : xr[k];
+      }
+    }
+    __syncthreads();  // `total` is rewritten for the next sample
+  }
+}
+
 }  // namespace ffi8

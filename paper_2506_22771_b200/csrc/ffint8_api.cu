@@ -1023,6 +1023,26 @@ ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bu
   return FF_OK;
 }
 
+ff_status ff_embed_labels(ff_ctx* ctx, const float* x, const int32_t* labels, int B, int n, int sets, int n_classes,
+                          int label_stride, float on_value, float tau0, float eps, float* out, void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if (!x || !labels || !out) return fail(ctx, FF_ERR_ARG, "x / labels / out is NULL");
+  if (B <= 0 || n <= 0 || sets <= 0 || n_classes <= 0 || label_stride <= 0) return fail(ctx, FF_ERR_ARG, "sizes must be positive");
+  if ((long long)(n_classes - 1) * label_stride >= n) return fail(ctx, FF_ERR_ARG, "the label places do not fit a sample");
+  if (tau0 > 0.0f && !(eps >= 0.0f)) return fail(ctx, FF_ERR_ARG, "eps must be >= 0");
+  if ((long long)sets * B * n >= (1LL << 40)) return fail(ctx, FF_ERR_RANGE, "output too large");
+  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(labels)) & 3)
+    return fail(ctx, FF_ERR_ALIGN, "x / labels / out must be 4-byte aligned");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  const int cap = ctx->sm_count * 8;
+  embed_labels_kernel<<<B < cap ? B : cap, EMBED_THREADS, 0, st>>>(x, labels, B, n, sets, n_classes, label_stride, on_value,
+                                                                  tau0, eps, out, status_ptr(ctx));
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
+
 ff_status ff_poll_status(ff_ctx* ctx, void* cuda_stream) {
   ff_status s = check_ctx(ctx);
   if (s != FF_OK) return s;
@@ -1034,6 +1054,7 @@ ff_status ff_poll_status(ff_ctx* ctx, void* cuda_stream) {
   FF_CUDA(ctx, cudaStreamSynchronize(st));
   if (h & ST_TIMEOUT) return fail(ctx, FF_ERR_DEVICE_TIMEOUT, "a bounded in-kernel wait ran out");
   if (h & ST_NONFINITE) return fail(ctx, FF_ERR_NONFINITE, "a tensor to be quantised held Inf or NaN");
+  if (h & ST_BADLABEL) return fail(ctx, FF_ERR_RANGE, "a label lay outside [0, n_classes)");
   return FF_OK;
 }
 

@@ -664,3 +664,40 @@ def test_strided_conv_gradient_matches_finite_differences():
         Wm[n, k] -= eps
         fd = (O.fp64_layer_loss(spec, X, Wp, B) - O.fp64_layer_loss(spec, X, Wm, B)) / (2 * eps)
         assert abs(fd - dW[n, k]) <= 1e-4 * max(1.0, abs(fd)), (n, k, fd, dW[n, k])
+
+
+# ---- label embedding (positive / negative / candidate batches; Sec. III, Alg. 1 line 3) ------------
+def test_embed_labels_hand_example():
+    x = np.array([[9.0, 9.0, 9.0, 3.0, 4.0]], dtype=np.float32)          # 3 label places, then the data
+    got = O.embed_labels(x, np.array([[2], [0]]), n_classes=3)
+    assert np.array_equal(got, np.array([[0, 0, 1, 3, 4], [1, 0, 0, 3, 4]], dtype=np.float32))
+    # scaled to length 13: |(0,0,12,3,4)| = 13 exactly, so r = 13/(13+0) = 1 and nothing changes
+    got = O.embed_labels(x, np.array([[2]]), n_classes=3, on_value=12.0, tau0=13.0, eps=0.0)
+    assert np.array_equal(got, np.array([[0, 0, 12, 3, 4]], dtype=np.float32))
+    # label places two apart (a channels-last image: channel 0 of the first pixels)
+    x = np.arange(1, 9, dtype=np.float32).reshape(1, 8)
+    got = O.embed_labels(x, np.array([[1]]), n_classes=3, label_stride=2, on_value=5.0)
+    assert np.array_equal(got, np.array([[0, 2, 5, 4, 0, 6, 7, 8]], dtype=np.float32))
+
+
+def test_embed_labels_matches_the_batch_generator_and_has_unit_invariants():
+    from paper_2506_22771_b200 import synth
+    # the input generator builds its batches the same way from its own base samples (float64, then cast):
+    # rebuild one of its batches from those base samples and compare
+    w = synth.workload("tiny_mlp")
+    B, n = 16, int(np.prod(w.in_shape))
+    g = synth._rng(7, 2000)
+    base = g.random((B, n), dtype=np.float64)
+    label = g.integers(0, 10, size=B)
+    wrong = (label + g.integers(1, 10, size=B)) % 10
+    want = synth.make_batch(w, 7, B=B).reshape(2 * B, n)
+    got = O.embed_labels(base.astype(np.float32), np.stack([label, wrong]), 10, tau0=float(np.sqrt(n)))
+    assert np.allclose(got, want, rtol=2e-6, atol=0.0)
+    # invariants: length tau0, label places one-hot, data entries of both sets parallel to the raw sample
+    assert np.allclose(np.sqrt((got.astype(np.float64) ** 2).sum(1)), np.sqrt(n), rtol=1e-6)
+    hot = got[:, :10] != 0
+    assert (hot.sum(1) == 1).all() and (hot.argmax(1) == np.concatenate([label, wrong])).all()
+    ratio = got[:, 10:] / np.concatenate([base, base])[:, 10:].astype(np.float32)
+    assert np.allclose(ratio, ratio[:, :1], rtol=1e-6)
+    with pytest.raises(ValueError):
+        O.embed_labels(base.astype(np.float32), np.full((1, B), 10), 10)
