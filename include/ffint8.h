@@ -82,7 +82,8 @@ typedef struct {
   uint64_t seed;        /* keys the stochastic-rounding hash                                  */
   int32_t stride;       /* conv3x3 only: 0 or 1 = every position, 2 = every second row and column; */
                         /* the output then has Ho = (H-1)/2 + 1 rows of Wo = (Wd-1)/2 + 1 positions */
-  int32_t reserved;     /* zero                                                                */
+  float momentum;       /* update rule: 0 = plain SGD (W -= lr*g); mu > 0 = heavy-ball SGD on the   */
+                        /* buffer Mom: m = mu*m + g, W -= lr*m (the paper names no optimiser)       */
 } ff_layer_desc;
 
 /* Device buffers of one layer (host struct of device pointers; caller-owned). */
@@ -105,6 +106,7 @@ typedef struct {
   float* loss;       /* [1] out: L_new averaged over the M samples (Eq. 3)                     */
   int32_t* acc_dump; /* [M*R,N] INT32 out, nullable: the forward accumulators                  */
   int32_t* accW_dump;/* [2,N,K] INT32 out, nullable: g^W accumulators of the two sets          */
+  float* Mom;        /* [N,K] FP32 in/out momentum buffer; needed (and touched) only if momentum != 0 */
 } ff_layer_bufs;
 
 /* Create / destroy a context for CUDA device `device` (must be compute capability 10.x).

@@ -69,6 +69,7 @@ class LayerSpec:
     seed: int = 0
     index: int = 0        # position of the layer in the network (feeds the rounding hash)
     stride: int = 1       # conv3x3 only: 1 or 2 (output (H-1)//stride + 1 by (Wd-1)//stride + 1)
+    momentum: float = 0.0 # heavy-ball coefficient of the update; 0 = plain SGD
 
     @property
     def out_hw(self):
@@ -373,6 +374,7 @@ class LayerState:
     accW: np.ndarray = None    # [2, N, K] int32, pass-separated
     W_new: np.ndarray = None
     dW: np.ndarray = None      # dequantised weight gradient (float32)
+    M_new: np.ndarray = None   # momentum buffer after the update (None for plain SGD)
 
 
 def _pass_rows(v_pos, v_neg, B):
@@ -415,9 +417,18 @@ def layer_loss_grad(spec: LayerSpec, st: LayerState, B: int, G_later: Sequence[n
     return st
 
 
-def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int) -> LayerState:
+def sgd_momentum(W: np.ndarray, M: np.ndarray, g: np.ndarray, lr: float, mu: float):
+    """Heavy-ball SGD (Polyak): m <- mu*m + g, W <- W - lr*m, each operation one float32 rounding.
+    The paper names no optimiser for 'updated to current weights' (Sec. IV-B; Alg. 1 line 9); plain
+    SGD is mu = 0, this is the usual next choice.  Returns (W_new, M_new)."""
+    M_new = F32(mu) * np.asarray(M, dtype=F32) + np.asarray(g, dtype=F32)
+    return np.asarray(W, dtype=F32) - F32(lr) * M_new, M_new
+
+
+def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int, M: Optional[np.ndarray] = None) -> LayerState:
     """g^W per pass as an INT8 MAC, dequantised and applied as plain SGD (Sec. IV-B; Alg. 1
-    line 9):  g = float(accP)*cP + float(accN)*cN,  W <- W - lr*g."""
+    line 9):  g = float(accP)*cP + float(accN)*cN,  W <- W - lr*g.  With spec.momentum != 0 the
+    update is heavy-ball SGD on the momentum buffer M (zeros when None), see sgd_momentum."""
     W = np.asarray(W, dtype=F32)
     accW = []
     for p in range(2):
@@ -432,16 +443,20 @@ def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int) -> Laye
     cP = scale_pair(st.a_dh[0])[0] * scale_pair(st.a_x[0])[0]
     cN = scale_pair(st.a_dh[1])[0] * scale_pair(st.a_x[1])[0]
     st.dW = st.accW[0].astype(F32) * cP + st.accW[1].astype(F32) * cN
-    st.W_new = W - F32(spec.lr) * st.dW
+    if spec.momentum != 0.0:
+        st.W_new, st.M_new = sgd_momentum(W, np.zeros_like(W) if M is None else M, st.dW, spec.lr, spec.momentum)
+    else:
+        st.W_new = W - F32(spec.lr) * st.dW
     return st
 
 
 def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: int, lam: float,
-               step: int) -> List[LayerState]:
+               step: int, Ms: Optional[List[np.ndarray]] = None) -> List[LayerState]:
     """Body of Algorithm 1's epoch loop: one INT8 forward through all k layers with the
     pre-update weights (line 5), goodness of every layer (line 6), then for each layer its
     loss from the G's (line 8) and its INT8 gradient and update (line 9).  lambda is the
-    caller's (lines 2 and 11).  With one layer and lambda = 0 this is the vanilla step."""
+    caller's (lines 2 and 11).  With one layer and lambda = 0 this is the vanilla step.  Ms: the
+    layers' momentum buffers (only read by layers with momentum != 0)."""
     states = []
     x = X
     for spec, W in zip(specs, Ws):
@@ -452,7 +467,7 @@ def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: i
         later = list(range(l + 1, len(specs)))
         layer_loss_grad(spec, states[l], B, [states[j].G for j in later],
                         [specs[j].theta for j in later], lam, step)
-        layer_update(spec, states[l], W, B)
+        layer_update(spec, states[l], W, B, None if Ms is None else Ms[l])
     return states
 
 

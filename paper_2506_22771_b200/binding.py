@@ -34,13 +34,13 @@ class ff_layer_desc(C.Structure):
                 ("Wd", C.c_int32), ("Cin", C.c_int32), ("index", C.c_int32),
                 ("round_x", C.c_int32), ("round_w", C.c_int32), ("round_dh", C.c_int32),
                 ("theta", C.c_float), ("lr", C.c_float), ("tau", C.c_float), ("eps", C.c_float),
-                ("seed", C.c_uint64), ("stride", C.c_int32), ("reserved", C.c_int32)]
+                ("seed", C.c_uint64), ("stride", C.c_int32), ("momentum", C.c_float)]
 
 
 class ff_layer_bufs(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
                 ("W", "X", "Y", "G", "Xnext", "Xq", "Wq", "dHq", "absmax", "S", "rowmax", "coef",
-                 "loss", "acc_dump", "accW_dump")]
+                 "loss", "acc_dump", "accW_dump", "Mom")]
 
 
 FF_DP_MAX_REDUCE = 96
@@ -257,7 +257,7 @@ def make_desc(cfg, index: int, seed: int, round_x=FF_ROUND_STOCHASTIC, round_w=F
               round_dh=FF_ROUND_STOCHASTIC) -> ff_layer_desc:
     """cfg: an object with kind, K, N, H, Wd, Cin, theta, lr, tau, eps (e.g. synth.LayerCfg)."""
     return ff_layer_desc(cfg.kind, cfg.K, cfg.N, cfg.H, cfg.Wd, cfg.Cin, index, round_x, round_w, round_dh,
-                         cfg.theta, cfg.lr, cfg.tau, cfg.eps, seed, getattr(cfg, "stride", 1), 0)
+                         cfg.theta, cfg.lr, cfg.tau, cfg.eps, seed, getattr(cfg, "stride", 1), getattr(cfg, "momentum", 0.0))
 
 
 class LayerBuffers:
@@ -287,10 +287,11 @@ class LayerBuffers:
         self.loss = z((4,), torch.float32)
         self.acc_dump = z((rows, desc.N), torch.int32) if dumps else None
         self.accW_dump = z((2, desc.N, desc.K), torch.int32) if (dumps or accw) else None
+        self.Mom = z((desc.N, desc.K), torch.float32) if desc.momentum != 0.0 else None
         p = lambda t: t.data_ptr() if t is not None else None
         self.struct = ff_layer_bufs(p(self.W), p(self.X), p(self.Y), p(self.G), p(self.Xnext), p(self.Xq),
                                     p(self.Wq), p(self.dHq), p(self.absmax), p(self.S), p(self.rowmax),
-                                    p(self.coef), p(self.loss), p(self.acc_dump), p(self.accW_dump))
+                                    p(self.coef), p(self.loss), p(self.acc_dump), p(self.accW_dump), p(self.Mom))
 
 
 class Context:

@@ -137,6 +137,7 @@ ff_status check_layer(ff_ctx* ctx, const ff_layer_desc* L, int B) {
   for (int r : {L->round_x, L->round_w, L->round_dh})
     if (r != FF_ROUND_NEAREST_EVEN && r != FF_ROUND_STOCHASTIC) return fail(ctx, FF_ERR_ARG, "unknown rounding mode");
   if (!(L->eps > 0.0f)) return fail(ctx, FF_ERR_ARG, "eps must be > 0");
+  if (!(L->momentum >= 0.0f && L->momentum < 1.0f)) return fail(ctx, FF_ERR_ARG, "momentum must lie in [0, 1)");
   const long long R = rows_per_sample(*L);
   const long long rows = 2LL * B * R;
   // 32-bit rounding counters and element indices
@@ -159,7 +160,7 @@ ff_status check_bufs(ff_ctx* ctx, const ff_layer_bufs* b, bool need_x) {
     if (!p) return fail(ctx, FF_ERR_ARG, "a required device pointer is NULL");
   if (need_x && !b->X) return fail(ctx, FF_ERR_ARG, "X is NULL");
   const void* all[] = {b->W, b->X, b->Y, b->G, b->Xnext, b->Xq, b->Wq, b->dHq, b->absmax, b->S, b->rowmax, b->coef,
-                       b->loss, b->acc_dump, b->accW_dump};
+                       b->loss, b->acc_dump, b->accW_dump, b->Mom};
   for (const void* p : all)
     if (p && !aligned16(p)) return fail(ctx, FF_ERR_ALIGN, "a device pointer is not 16-byte aligned");
   return FF_OK;
@@ -255,14 +256,16 @@ ff_status launch_slab_update(ff_ctx* ctx, const int32_t* slabs, int splits, cons
   const size_t plane = (size_t)L.N * L.K;
   float* W = ctx->accumulate_only ? nullptr : b.W;
   int32_t* dump = b.accW_dump == slabs ? nullptr : b.accW_dump;  // the sums already are where they would be copied to
+  float* Mom = L.momentum != 0.0f ? b.Mom : nullptr;
   if (!W && !dump) return FF_OK;
   if (splits <= 2 && (pitch == 0 || pitch == L.K) && (plane & 3) == 0 && plane >= ((size_t)1 << 18)) {
     const size_t want = (plane / 4 + 255) / 256, cap = (size_t)ctx->sm_count * 8;
-    slab_update_flat_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, W, b.absmax, L.lr, dump);
+    slab_update_flat_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, W, b.absmax, L.lr, dump,
+                                                                                 Mom, L.momentum);
   } else {
     const size_t want = (plane + 31) / 32, cap = (size_t)ctx->sm_count * 8;
     slab_update_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, L.K, pitch ? pitch : L.K, W,
-                                                                            b.absmax, L.lr, dump);
+                                                                            b.absmax, L.lr, dump, Mom, L.momentum);
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -355,6 +358,7 @@ ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
 
 // Weight-gradient contraction + fused update.
 ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  if (L.momentum != 0.0f && !b.Mom) return fail(ctx, FF_ERR_ARG, "momentum != 0 needs the buffer Mom");
   const int R = rows_per_sample(L);
   const int rows = 2 * B * R;
   bool tc_ok = tc_update_supported(L, B);
@@ -461,7 +465,7 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
       return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st);
     return launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st);
   }
-  UpdateEpilogue epi{b.W, b.accW_dump, b.absmax, L.lr, L.N, L.K};
+  UpdateEpilogue epi{b.W, b.accW_dump, b.absmax, L.lr, L.N, L.K, L.momentum != 0.0f ? b.Mom : nullptr, L.momentum};
   if (L.kind != FF_CONV3X3)
     return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st);
   return launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st);
@@ -972,6 +976,7 @@ ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_l
     if ((s = check_layer(ctx, &layers[l], B_total)) != FF_OK) return s;
     if (l > 0 && bufs[l].X) return fail(ctx, FF_ERR_ARG, "a data-parallel step takes chained layers (X of layers > 0 NULL)");
     if (!bufs[l].accW_dump) return fail(ctx, FF_ERR_ARG, "a data-parallel step needs accW_dump of every layer");
+    if (layers[l].momentum != 0.0f && !bufs[l].Mom) return fail(ctx, FF_ERR_ARG, "momentum != 0 needs the buffer Mom");
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;

@@ -142,6 +142,8 @@ struct UpdateEpilogue {
   const float* absmax;
   float lr;
   int rows, cols;  // N, K
+  float* Mom;      // nullable: heavy-ball buffer, m = mu*m + g, W -= lr*m
+  float mu;
   __device__ __forceinline__ void operator()(int i0, int j0, const int (&acc)[2][4][4]) const {
     const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
     const float cN = __fmul_rn(scale_of(absmax[4]), scale_of(absmax[1]));
@@ -152,7 +154,8 @@ struct UpdateEpilogue {
         const int i = i0 + r, j = j0 + c;
         if (i < rows && j < cols) {
           const size_t o = (size_t)i * cols + j;
-          const float g = __fadd_rn(__fmul_rn(__int2float_rn(acc[0][r][c]), cP), __fmul_rn(__int2float_rn(acc[1][r][c]), cN));
+          float g = __fadd_rn(__fmul_rn(__int2float_rn(acc[0][r][c]), cP), __fmul_rn(__int2float_rn(acc[1][r][c]), cN));
+          if (Mom) Mom[o] = g = __fadd_rn(__fmul_rn(mu, Mom[o]), g);
           W[o] = __fsub_rn(W[o], __fmul_rn(lr, g));
           if (accW_dump) {
             accW_dump[o] = acc[0][r][c];
@@ -194,7 +197,8 @@ struct SlabEpilogue {
 // [2][rows][cols]) - the buffer a data-parallel step adds up over the devices before it updates.
 __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane, int cols,
                                                           int pitch, float* __restrict__ W, const float* __restrict__ absmax,
-                                                          float lr, int32_t* __restrict__ accW_dump) {
+                                                          float lr, int32_t* __restrict__ accW_dump,
+                                                          float* __restrict__ Mom = nullptr, float mu = 0.0f) {
   __shared__ int part[2][8][32];
   const int lane = threadIdx.x & 31, zl = threadIdx.x >> 5;
   const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
@@ -220,7 +224,8 @@ __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restr
         aN += part[1][k][lane];
       }
       if (W) {
-        const float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
+        float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
+        if (Mom) Mom[e] = g = __fadd_rn(__fmul_rn(mu, Mom[e]), g);
         W[e] = __fsub_rn(W[e], __fmul_rn(lr, g));
       }
       if (accW_dump) {
@@ -236,7 +241,8 @@ __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restr
 // warps, so every thread takes four consecutive elements with 128-bit accesses.
 __global__ void __launch_bounds__(256) slab_update_flat_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane,
                                                                float* __restrict__ W, const float* __restrict__ absmax, float lr,
-                                                               int32_t* __restrict__ accW_dump) {
+                                                               int32_t* __restrict__ accW_dump, float* __restrict__ Mom = nullptr,
+                                                               float mu = 0.0f) {
   const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
   const float cN = __fmul_rn(scale_of(absmax[4]), scale_of(absmax[1]));
   const size_t n4 = plane >> 2, stride = (size_t)gridDim.x * blockDim.x;
@@ -251,10 +257,23 @@ __global__ void __launch_bounds__(256) slab_update_flat_kernel(const int32_t* __
     }
     if (W) {
       float4 w = reinterpret_cast<const float4*>(W)[i];
-      w.x = __fsub_rn(w.x, __fmul_rn(lr, __fadd_rn(__fmul_rn(__int2float_rn(aP.x), cP), __fmul_rn(__int2float_rn(aN.x), cN))));
-      w.y = __fsub_rn(w.y, __fmul_rn(lr, __fadd_rn(__fmul_rn(__int2float_rn(aP.y), cP), __fmul_rn(__int2float_rn(aN.y), cN))));
-      w.z = __fsub_rn(w.z, __fmul_rn(lr, __fadd_rn(__fmul_rn(__int2float_rn(aP.z), cP), __fmul_rn(__int2float_rn(aN.z), cN))));
-      w.w = __fsub_rn(w.w, __fmul_rn(lr, __fadd_rn(__fmul_rn(__int2float_rn(aP.w), cP), __fmul_rn(__int2float_rn(aN.w), cN))));
+      float4 g;
+      g.x = __fadd_rn(__fmul_rn(__int2float_rn(aP.x), cP), __fmul_rn(__int2float_rn(aN.x), cN));
+      g.y = __fadd_rn(__fmul_rn(__int2float_rn(aP.y), cP), __fmul_rn(__int2float_rn(aN.y), cN));
+      g.z = __fadd_rn(__fmul_rn(__int2float_rn(aP.z), cP), __fmul_rn(__int2float_rn(aN.z), cN));
+      g.w = __fadd_rn(__fmul_rn(__int2float_rn(aP.w), cP), __fmul_rn(__int2float_rn(aN.w), cN));
+      if (Mom) {
+        const float4 m = reinterpret_cast<const float4*>(Mom)[i];
+        g.x = __fadd_rn(__fmul_rn(mu, m.x), g.x);
+        g.y = __fadd_rn(__fmul_rn(mu, m.y), g.y);
+        g.z = __fadd_rn(__fmul_rn(mu, m.z), g.z);
+        g.w = __fadd_rn(__fmul_rn(mu, m.w), g.w);
+        reinterpret_cast<float4*>(Mom)[i] = g;
+      }
+      w.x = __fsub_rn(w.x, __fmul_rn(lr, g.x));
+      w.y = __fsub_rn(w.y, __fmul_rn(lr, g.y));
+      w.z = __fsub_rn(w.z, __fmul_rn(lr, g.z));
+      w.w = __fsub_rn(w.w, __fmul_rn(lr, g.w));
       reinterpret_cast<float4*>(W)[i] = w;
     }
     if (accW_dump) {

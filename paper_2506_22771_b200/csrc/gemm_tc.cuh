@@ -93,6 +93,8 @@ struct TcParams {
   float* W;
   int32_t* accW_dump;
   float lr;
+  float* mom;               // nullable heavy-ball buffer [out_rows, out_cols]: m = mu*m + g, W -= lr*m
+  float mu;
   // split weight gradient
   int32_t* slabs;
   // convolution geometry (conv_W = 0: dense layer).  A 128-row block of positions is conv_TH image
@@ -743,8 +745,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           }
         }
       } else {  // TC_MODE_UPD
-        // thread = one accumulator row computes d = lr*(float(accP)*cP + float(accN)*cN); d is staged
-        // through smem so that the read-modify-write of W is row-contiguous
+        // thread = one accumulator row computes g = float(accP)*cP + float(accN)*cN; g is staged
+        // through smem so that the read-modify-write of W (and of the momentum buffer) is row-contiguous
         const size_t plane = (size_t)p.out_rows * p.out_cols;
         uint8_t* patch = patch0;
 #pragma unroll 1
@@ -769,10 +771,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           for (int j = 0; j < 32; j += 4) {
             float d[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float g = __fadd_rn(__fmul_rn(__int2float_rn(vp[j + q]), cP), __fmul_rn(__int2float_rn(vn[j + q]), cN));
-              d[q] = __fmul_rn(p.lr, g);
-            }
+            for (int q = 0; q < 4; ++q)
+              d[q] = __fadd_rn(__fmul_rn(__int2float_rn(vp[j + q]), cP), __fmul_rn(__int2float_rn(vn[j + q]), cN));
             *reinterpret_cast<float4*>(patch + lane * 128 + (((j >> 2) ^ (lane & 7)) << 4)) = make_float4(d[0], d[1], d[2], d[3]);
           }
           __syncwarp();
@@ -781,8 +781,28 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             const int r = i * 4 + (lane >> 3), cc = lane & 7;
             const int grow = wrow0 + r, gcol = col0 + cb + cc * 4;
             if (grow < p.out_rows) {
-              const float4 dv = *reinterpret_cast<const float4*>(patch + r * 128 + ((cc ^ (r & 7)) << 4));
+              float4 dv = *reinterpret_cast<const float4*>(patch + r * 128 + ((cc ^ (r & 7)) << 4));
               float* dst = p.W + (size_t)grow * p.out_cols + gcol;
+              if (p.mom) {  // heavy ball: the step is taken along m = mu*m + g
+                float* mp = p.mom + (size_t)grow * p.out_cols + gcol;
+                if (full) {
+                  const float4 m = *reinterpret_cast<const float4*>(mp);
+                  dv.x = __fadd_rn(__fmul_rn(p.mu, m.x), dv.x);
+                  dv.y = __fadd_rn(__fmul_rn(p.mu, m.y), dv.y);
+                  dv.z = __fadd_rn(__fmul_rn(p.mu, m.z), dv.z);
+                  dv.w = __fadd_rn(__fmul_rn(p.mu, m.w), dv.w);
+                  *reinterpret_cast<float4*>(mp) = dv;
+                } else {
+                  float* dd = reinterpret_cast<float*>(&dv);
+#pragma unroll
+                  for (int q = 0; q < 4; ++q)
+                    if (gcol + q < p.out_cols) mp[q] = dd[q] = __fadd_rn(__fmul_rn(p.mu, mp[q]), dd[q]);
+                }
+              }
+              dv.x = __fmul_rn(p.lr, dv.x);
+              dv.y = __fmul_rn(p.lr, dv.y);
+              dv.z = __fmul_rn(p.lr, dv.z);
+              dv.w = __fmul_rn(p.lr, dv.w);
               if (full) {
                 float4 w = wv[i];
                 w.x = __fsub_rn(w.x, dv.x);
@@ -1138,6 +1158,8 @@ inline ff_status tc_update(TcState& t, const ff_layer_desc& L, const ff_layer_bu
   p.accW_dump = b.accW_dump;
   p.absmax = b.absmax;
   p.lr = L.lr;
+  p.mom = L.momentum != 0.0f ? b.Mom : nullptr;
+  p.mu = L.momentum;
   if ((s = tc_make_map(t, &ta, b.dHq, L.N, B, 2, 128, 128)) != FF_OK) return s;
   if ((s = tc_make_map(t, &tb, b.Xq, L.K, B, 2, 128, 128)) != FF_OK) return s;
   return tc_launch<TC_MODE_UPD, true, 128>(t, tc_pick_ncta(t, L.N, L.K), ta, tb, p, st);

@@ -29,6 +29,7 @@ class LayerCfg:
     Cin: int = 0
     eps: float = 1e-8
     stride: int = 1    # conv3x3 only
+    momentum: float = 0.0   # heavy-ball coefficient of the update (0: plain SGD)
 
 
 @dataclass

@@ -15,7 +15,8 @@ def specs_and_descs(layers, seed, round_x=1, round_w=0, round_dh=1):
     specs, descs = [], []
     for i, l in enumerate(layers):
         specs.append(O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, l.eps, l.H, l.Wd, l.Cin,
-                                 round_x, round_w, round_dh, seed, i, getattr(l, "stride", 1)))
+                                 round_x, round_w, round_dh, seed, i, getattr(l, "stride", 1),
+                                 getattr(l, "momentum", 0.0)))
         descs.append(ffb.make_desc(l, i, seed, round_x, round_w, round_dh))
     return specs, descs
 
@@ -87,6 +88,8 @@ def compare_layer(st: O.LayerState, b, spec, B, check_dumps=True, tag=""):
         if check_dumps and b.accW_dump is not None:
             eq("accW", _np(b.accW_dump).reshape(-1), st.accW.reshape(-1))
         eq("W_new", _np(b.W).reshape(-1), st.W_new.reshape(-1))
+        if st.M_new is not None:
+            eq("M_new", _np(b.Mom).reshape(-1), st.M_new.reshape(-1))
 
 
 def _assert_equal(name, got, want):

@@ -51,6 +51,7 @@ def _run_dp(w, seed, steps, lam_per_step, world, path, rounding=(1, 0, 1)):
     n = len(descs)
     for sh in shards:
         sh.net.set_input(dp.shard_batch(np.ascontiguousarray(X).reshape(2 * w.B, -1), w.B, sh.off, sh.B))
+    Ms = None
     for step in range(steps):
         lam = lam_per_step * step
         for phase in range(ffb.ff_dp_phase_count(n)):
@@ -59,11 +60,12 @@ def _run_dp(w, seed, steps, lam_per_step, world, path, rounding=(1, 0, 1)):
             _combine(shards, entries)
         for sh in shards:
             ffb.ff_poll_status(sh.net.ctx.ctx, 0)
-        states = O.train_step(specs, Ws, X, w.B, lam, step)
+        states = O.train_step(specs, Ws, X, w.B, lam, step, Ms)
         for r, sh in enumerate(shards):
             for l, (st, b, sp) in enumerate(zip(states, sh.net.bufs, specs)):
                 compare_layer(shard_state(st, w.B, sh.off, sh.B), b, sp, sh.B, tag=f"step{step}/shard{r}/layer{l}/")
         Ws = [st.W_new for st in states]
+        Ms = [st.M_new for st in states]
     for sh in shards:
         sh.net.close()
 
@@ -108,6 +110,13 @@ def test_dp_wide_layers_take_the_flat_update():
     w = synth.scaled(synth.workload("mlp_lookahead"), B=160, width_div=4)
     _run_dp(w, seed=13, steps=2, lam_per_step=0.5, world=2, path=(ffb.FF_GEMM_AUTO, 0))
     _run_dp(w, seed=13, steps=1, lam_per_step=0.5, world=2, path=(ffb.FF_GEMM_AUTO, 1))
+
+
+def test_dp_with_momentum():
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=90, width_div=8)
+    for l in w.layers:
+        l.momentum = 0.9
+    _run_dp(w, seed=14, steps=3, lam_per_step=0.5, world=3, path=(ffb.FF_GEMM_AUTO, 0))
 
 
 def test_dp_single_shard_equals_train_step():

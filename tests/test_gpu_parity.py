@@ -66,14 +66,16 @@ def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), cha
     X = synth.make_batch(w, seed)
     net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path, graph=graph)
     net.set_input(X)
+    Ms = None
     for step in range(steps):
         lam = lam_per_step * step
         net.train_step(lam, step)
-        states = O.train_step(specs, Ws, X, w.B, lam, step)
+        states = O.train_step(specs, Ws, X, w.B, lam, step, Ms)
         if step % check_every == 0 or step == steps - 1:
             for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
                 compare_layer(st, b, sp, w.B, tag=f"step{step}/layer{l}/")
         Ws = [st.W_new for st in states]
+        Ms = [st.M_new for st in states]
     net.close()
 
 
@@ -450,4 +452,47 @@ def test_graph_replay_two_call_shapes_share_a_context():
         Wa = [st.W_new for st in sa]
         Wb = [st.W_new for st in sb]
     assert ffb.ff_graph_replay_count(net.ctx.ctx) == 8, ffb.ff_last_error(net.ctx.ctx)
+    net.close()
+
+
+# ---- heavy-ball variant of the update: every weight-gradient route carries the momentum buffer ----------
+def _with_momentum(w, mu):
+    for i, l in enumerate(w.layers):
+        l.momentum = mu if i != 1 else 0.0        # one plain layer in between: its buffer must stay untouched / absent
+    return w
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_momentum_dense_lookahead(path):
+    w = _with_momentum(synth.scaled(synth.workload("mlp_lookahead"), B=136, width_div=8), 0.875)
+    _run_and_compare(w, seed=17, steps=4, lam_per_step=0.25, path=path)
+    _run_and_compare(w, seed=17, steps=4, lam_per_step=0.25, path=path, graph=True)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_momentum_cnn_and_pointwise(path):
+    w = _with_momentum(synth.scaled(synth.workload("cnn"), B=2, width_div=4), 0.5)     # im2col, dp4a / slab routes
+    _run_and_compare(w, seed=27, steps=3, lam_per_step=0.0, path=path)
+    layers = [synth.LayerCfg(1, 9 * 64, 128, float(128 * 16 * 16) / 2, 0.03 / 1024, float(np.sqrt(128 * 256)), H=16, Wd=16,
+                             Cin=64, momentum=0.9),                                   # implicit-GEMM split slabs
+              synth.LayerCfg(2, 128, 64, float(64 * 16 * 16) / 2, 0.03 / 256, float(np.sqrt(64 * 256)), H=16, Wd=16, Cin=128,
+                             momentum=0.9)]
+    w = synth.Workload("conv_mom", 2, layers, (16, 16, 64), "normal", "kaiming_uniform", 2)
+    _run_and_compare(w, seed=28, steps=3, lam_per_step=0.0, path=path)
+
+
+def test_momentum_wide_layer_and_argument_errors():
+    # 784 x 1000 weights through the fused tensor-core update (pairs), ragged last column tile
+    w = _with_momentum(synth.scaled(synth.workload("mlp_lookahead"), B=130, width_div=2), 0.75)
+    w.layers = w.layers[:2]
+    w.layers[1].momentum = 0.75
+    _run_and_compare(w, seed=19, steps=3, lam_per_step=0.0, path=(ffb.FF_GEMM_AUTO, 0))
+    specs, descs = specs_and_descs(w.layers, 1)
+    net = GpuNet(descs, w.B, synth.make_weights(w, 1))
+    net.bufs_arr[0].Mom = None
+    with pytest.raises(ffb.FFError):
+        net.train_step(0.0, 0)
+    net.descs_arr[0].momentum = 1.5
+    with pytest.raises(ffb.FFError):
+        net.train_step(0.0, 0)
     net.close()

@@ -701,3 +701,47 @@ def test_embed_labels_matches_the_batch_generator_and_has_unit_invariants():
     assert np.allclose(ratio, ratio[:, :1], rtol=1e-6)
     with pytest.raises(ValueError):
         O.embed_labels(base.astype(np.float32), np.full((1, B), 10), 10)
+
+
+# ---- heavy-ball variant of the update (Alg. 1 line 9 names no optimiser) ----------------------------
+def test_sgd_momentum_hand_example_and_closed_form():
+    # powers of two: every product and sum is exact in float32
+    W, M = np.array([1.0, -2.0], np.float32), np.array([0.5, 0.0], np.float32)
+    g = np.array([0.25, 1.0], np.float32)
+    W1, M1 = O.sgd_momentum(W, M, g, lr=0.5, mu=0.5)
+    assert np.array_equal(M1, np.array([0.5, 1.0], np.float32))          # 0.5*0.5 + 0.25 ; 0 + 1
+    assert np.array_equal(W1, np.array([0.75, -2.5], np.float32))        # 1 - 0.5*0.5 ; -2 - 0.5*1
+    W2, M2 = O.sgd_momentum(W1, M1, g, lr=0.5, mu=0.5)
+    assert np.array_equal(M2, np.array([0.5, 1.5], np.float32)) and np.array_equal(W2, np.array([0.5, -3.25], np.float32))
+    # constant gradient from m = 0: m_t = g (1 - mu^t)/(1 - mu), W_t = W_0 - lr * sum_{i<=t} m_i
+    mu, lr, gg = 0.9, 0.01, np.float32(0.3)
+    Wt, Mt = np.zeros(1, np.float32), np.zeros(1, np.float32)
+    for t in range(1, 51):
+        Wt, Mt = O.sgd_momentum(Wt, Mt, np.array([gg]), lr, mu)
+        m_closed = 0.3 * (1 - mu ** t) / (1 - mu)
+        w_closed = -lr * 0.3 * (t - mu * (1 - mu ** t) / (1 - mu)) / (1 - mu)
+        assert abs(Mt[0] - m_closed) < 1e-5 and abs(Wt[0] - w_closed) < 1e-5
+    # mu = 0 is plain SGD bit for bit
+    g3 = np.random.default_rng(0).normal(size=7).astype(np.float32)
+    W3 = np.random.default_rng(1).normal(size=7).astype(np.float32)
+    assert np.array_equal(O.sgd_momentum(W3, np.ones(7, np.float32), g3, 0.03, 0.0)[0], W3 - np.float32(0.03) * g3)
+
+
+def test_layer_update_with_momentum_carries_the_buffer():
+    from paper_2506_22771_b200 import synth
+    w = synth.scaled(synth.workload("tiny_mlp"), B=8, width_div=8)
+    l = w.layers[0]
+    plain = O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, seed=3)
+    heavy = O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, seed=3, momentum=0.75)
+    W0 = synth.make_weights(w, 3)[0]
+    X = synth.make_batch(w, 3)
+    a = O.train_step([plain], [W0], X, w.B, 0.0, 0)[0]
+    b = O.train_step([heavy], [W0], X, w.B, 0.0, 0)[0]
+    # from a zero buffer the first heavy-ball step is the plain step and leaves m = g
+    assert np.array_equal(a.W_new, b.W_new) and np.array_equal(b.M_new, b.dW) and a.M_new is None
+    b2 = O.train_step([heavy], [b.W_new], X, w.B, 0.0, 1, Ms=[b.M_new])[0]
+    a2 = O.train_step([plain], [b.W_new], X, w.B, 0.0, 1)[0]
+    assert np.array_equal(b2.dW, a2.dW)                                   # same gradient, different step
+    assert np.array_equal(b2.M_new, np.float32(0.75) * b.dW + b2.dW)
+    assert np.array_equal(b2.W_new, b.W_new - np.float32(l.lr) * b2.M_new)
+    assert not np.array_equal(b2.W_new, a2.W_new)
