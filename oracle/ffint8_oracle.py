@@ -41,6 +41,7 @@ ROLE_DH = 2  # hash stream of the output-gradient quantiser
 KIND_LINEAR = 0
 KIND_CONV3X3 = 1
 KIND_CONV1X1 = 2
+KIND_DWCONV3X3 = 3
 
 _M64 = (1 << 64) - 1
 
@@ -52,7 +53,9 @@ _M64 = (1 << 64) - 1
 class LayerSpec:
     """One FF layer.  linear: X [2B,K] -> Y [2B,N].  conv3x3 (stride 1, zero pad 1, NHWC):
     X [2B,H,W,Cin] -> Y [2B,H,W,N] with K = 9*Cin and weights [N,3,3,Cin] flattened to [N,K].
-    conv1x1 (pointwise, NHWC): X [2B,H,W,Cin] -> Y [2B,H,W,N] with K = Cin and weights [N,Cin]."""
+    conv1x1 (pointwise, NHWC): X [2B,H,W,Cin] -> Y [2B,H,W,N] with K = Cin and weights [N,Cin].
+    dwconv3x3 (depthwise: every channel has its own 3x3 filter; stride 1 or 2, zero pad 1, NHWC):
+    X [2B,H,W,C] -> Y [2B,Ho,Wo,C] with N = Cin = C, K = 9 and weights [C,3,3] flattened to [C,9]."""
     kind: int
     K: int
     N: int
@@ -73,7 +76,7 @@ class LayerSpec:
 
     @property
     def out_hw(self):
-        if self.kind == KIND_CONV3X3:
+        if self.kind in (KIND_CONV3X3, KIND_DWCONV3X3):
             return (self.H - 1) // self.stride + 1, (self.Wd - 1) // self.stride + 1
         return self.H, self.Wd
 
@@ -245,6 +248,36 @@ def int8_conv3x3_wgrad(dhq: np.ndarray, xq: np.ndarray, stride: int = 1) -> np.n
     return out
 
 
+def int8_dwconv3x3(xq: np.ndarray, wq: np.ndarray, stride: int = 1) -> np.ndarray:
+    """Depthwise 3x3 MAC: acc[b,i,j,c] = sum_{r,s} xq[b,stride*i+r-1,stride*j+s-1,c]*wq[c,r,s], zero
+    padding 1 - the convolution of Sec. IV-B's 'dense or convolution layers' with one filter per
+    channel and no sum over channels (the depthwise layers of the paper's MobileNetV2 / EfficientNet
+    models, Table II).  xq NHWC int8, wq [C,3,3] int8; exact in int64, checked against INT32."""
+    Bn, H, Wd, C = xq.shape
+    Ho, Wo = (H - 1) // stride + 1, (Wd - 1) // stride + 1
+    xp = _pad_hw(xq).astype(np.int64)
+    acc = np.zeros((Bn, Ho, Wo, C), dtype=np.int64)
+    for r in range(3):
+        for s in range(3):
+            acc += xp[:, r:r + stride * (Ho - 1) + 1:stride, s:s + stride * (Wo - 1) + 1:stride, :] * wq[:, r, s].astype(np.int64)
+    return _check_i32(acc)
+
+
+def int8_dwconv3x3_wgrad(dhq: np.ndarray, xq: np.ndarray, stride: int = 1) -> np.ndarray:
+    """accW[c,r,s] = sum_{b,i,j} dhq[b,i,j,c]*xq[b,stride*i+r-1,stride*j+s-1,c] (weight gradient of the
+    depthwise MAC; no input gradient, Sec. IV-B)."""
+    Bn, H, Wd, C = xq.shape
+    _, Ho, Wo, _ = dhq.shape
+    xp = _pad_hw(xq).astype(np.int64)
+    d = dhq.astype(np.int64)
+    out = np.empty((C, 3, 3), dtype=np.int64)
+    for r in range(3):
+        for s in range(3):
+            win = xp[:, r:r + stride * (Ho - 1) + 1:stride, s:s + stride * (Wo - 1) + 1:stride, :]
+            out[:, r, s] = (d * win).sum(axis=(0, 1, 2))
+    return _check_i32(out)
+
+
 # --------------------------------------------------------------------------------------
 # Epilogue: dequantise, ReLU, goodness, length normalisation  (Sec. III; Alg. 1 line 6)
 # --------------------------------------------------------------------------------------
@@ -395,6 +428,8 @@ def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: i
     elif spec.kind == KIND_CONV1X1:
         # pointwise convolution: the dense MAC applied at every position ('dense or convolution layers', Sec. IV-B)
         st.acc = int8_gemm_nt(st.Xq.reshape(-1, spec.K), st.Wq).reshape(st.Xq.shape[:3] + (spec.N,))
+    elif spec.kind == KIND_DWCONV3X3:
+        st.acc = int8_dwconv3x3(st.Xq, st.Wq.reshape(spec.N, 3, 3), spec.stride)
     else:
         st.acc = int8_conv3x3(st.Xq, st.Wq.reshape(spec.N, 3, 3, spec.Cin), spec.stride)
     s_w, _ = scale_pair(st.a_w)
@@ -437,6 +472,8 @@ def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int, M: Opti
             accW.append(int8_gemm_tn(st.dHq[sl], st.Xq[sl]))
         elif spec.kind == KIND_CONV1X1:
             accW.append(int8_gemm_tn(st.dHq[sl].reshape(-1, spec.N), st.Xq[sl].reshape(-1, spec.K)))
+        elif spec.kind == KIND_DWCONV3X3:
+            accW.append(int8_dwconv3x3_wgrad(st.dHq[sl], st.Xq[sl], spec.stride).reshape(spec.N, 9))
         else:
             accW.append(int8_conv3x3_wgrad(st.dHq[sl], st.Xq[sl], spec.stride).reshape(spec.N, spec.K))
     st.accW = np.stack(accW)
@@ -548,6 +585,16 @@ def fp64_layer_loss(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int) -> fl
     W = np.asarray(W, dtype=F64)
     if spec.kind in (KIND_LINEAR, KIND_CONV1X1):
         Y = np.maximum(X @ W.T, 0.0)
+    elif spec.kind == KIND_DWCONV3X3:
+        xp = np.pad(X, ((0, 0), (1, 1), (1, 1), (0, 0)))
+        w3 = W.reshape(spec.N, 3, 3)
+        Ho, Wo = spec.out_hw
+        st = spec.stride
+        Y = np.zeros((X.shape[0], Ho, Wo, spec.N))
+        for r in range(3):
+            for s in range(3):
+                Y += xp[:, r:r + st * (Ho - 1) + 1:st, s:s + st * (Wo - 1) + 1:st, :] * w3[:, r, s]
+        Y = np.maximum(Y, 0.0)
     else:
         xp = np.pad(X, ((0, 0), (1, 1), (1, 1), (0, 0)))
         w4 = W.reshape(spec.N, 3, 3, spec.Cin)

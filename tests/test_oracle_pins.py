@@ -745,3 +745,86 @@ def test_layer_update_with_momentum_carries_the_buffer():
     assert np.array_equal(b2.M_new, np.float32(0.75) * b.dW + b2.dW)
     assert np.array_equal(b2.W_new, b.W_new - np.float32(l.lr) * b2.M_new)
     assert not np.array_equal(b2.W_new, a2.W_new)
+
+
+# --------------------------------------------------------------------------------------
+# Depthwise 3x3 convolution
+# --------------------------------------------------------------------------------------
+def test_depthwise_conv_is_the_full_conv_with_one_filter_per_channel():
+    g = np.random.default_rng(31)
+    for stride, (H, Wd) in [(1, (5, 6)), (2, (5, 6)), (2, (4, 7))]:
+        C = 5
+        x = g.integers(-127, 128, size=(3, H, Wd, C)).astype(np.int8)
+        w = g.integers(-127, 128, size=(C, 3, 3)).astype(np.int8)
+        # the full convolution (pinned by brute force) whose filter for output channel c looks at input channel c only
+        wfull = np.zeros((C, 3, 3, C), dtype=np.int8)
+        for c in range(C):
+            wfull[c, :, :, c] = w[c]
+        got = O.int8_dwconv3x3(x, w, stride)
+        assert np.array_equal(got, O.int8_conv3x3(x, wfull, stride))
+        # weight gradient: the matching entries of the full convolution's gradient
+        d = g.integers(-127, 128, size=got.shape).astype(np.int8)
+        full_grad = O.int8_conv3x3_wgrad(d, x, stride)                   # [C,3,3,C]
+        want = np.stack([full_grad[c, :, :, c] for c in range(C)])
+        assert np.array_equal(O.int8_dwconv3x3_wgrad(d, x, stride), want)
+
+
+def test_depthwise_conv_brute_force_single_output():
+    x = np.zeros((1, 3, 3, 2), dtype=np.int8)
+    x[0, :, :, 0] = np.arange(1, 10).reshape(3, 3)
+    x[0, :, :, 1] = -1
+    w = np.zeros((2, 3, 3), dtype=np.int8)
+    w[0] = np.arange(9, 0, -1).reshape(3, 3)
+    w[1, 1, 1] = 7
+    acc = O.int8_dwconv3x3(x, w)
+    assert acc[0, 1, 1, 0] == sum((i + 1) * (9 - i) for i in range(9))   # centre: all nine taps
+    assert acc[0, 0, 0, 0] == 1 * 5 + 2 * 4 + 4 * 2 + 5 * 1              # corner: the four taps inside the image
+    assert np.all(acc[0, :, :, 1] == -7)                                  # channel 1 never sees channel 0
+
+
+def test_depthwise_gradient_matches_finite_differences():
+    g = np.random.default_rng(32)
+    for stride in (1, 2):
+        B, H, Wd, C = 1, 4, 5, 3
+        spec = O.LayerSpec(O.KIND_DWCONV3X3, 9, C, 6.0, 0.0, 1.0, H=H, Wd=Wd, Cin=C, stride=stride)
+        X = g.normal(size=(2 * B, H, Wd, C))
+        W = g.normal(size=(C, 9)) * 0.5
+        Ho, Wo = spec.out_hw
+        xp = np.pad(X, ((0, 0), (1, 1), (1, 1), (0, 0)))
+        w3 = W.reshape(C, 3, 3)
+        wins = {(r, s): xp[:, r:r + stride * (Ho - 1) + 1:stride, s:s + stride * (Wo - 1) + 1:stride, :]
+                for r in range(3) for s in range(3)}
+        Y = np.maximum(sum(wins[r, s] * w3[:, r, s] for r in range(3) for s in range(3)), 0.0)
+        G = (Y.reshape(2 * B, -1) ** 2).sum(1)
+        _, gp = O.ff_loss_terms(G.astype(F32), spec.theta, B)
+        dH = 2.0 * (gp / (2 * B))[:, None, None, None] * Y
+        eps = 1e-6
+        for (c, r, s) in [(0, 0, 0), (1, 1, 1), (2, 2, 0), (1, 0, 2)]:
+            dW = (dH * wins[r, s])[..., c].sum()
+            Wp, Wm = W.copy(), W.copy()
+            Wp[c, r * 3 + s] += eps
+            Wm[c, r * 3 + s] -= eps
+            fd = (O.fp64_layer_loss(spec, X, Wp, B) - O.fp64_layer_loss(spec, X, Wm, B)) / (2 * eps)
+            assert abs(fd - dW) <= 1e-4 * max(1.0, abs(fd)), (stride, c, r, s, fd, dW)
+
+
+def test_depthwise_layer_step_descends_and_chains():
+    # a depthwise layer between two pointwise layers (the separable block of the paper's mobile models): the INT8
+    # gradient of the depthwise layer correlates with the float64 gradient of the unquantised loss
+    g = np.random.default_rng(33)
+    B, H, Wd, C = 4, 6, 6, 8
+    spec = O.LayerSpec(O.KIND_DWCONV3X3, 9, C, float(C * H * Wd) / 2, 0.01, float(np.sqrt(C * H * Wd)), H=H, Wd=Wd, Cin=C,
+                       seed=5)
+    X = g.normal(size=(2 * B, H, Wd, C)).astype(F32)
+    W = (g.normal(size=(C, 9)) * 0.5).astype(F32)
+    st = O.train_step([spec], [W], X, B, 0.0, 0)[0]
+    assert st.acc.shape == (2 * B, H, Wd, C) and st.accW.shape == (2, C, 9) and st.W_new.shape == (C, 9)
+    fd = np.zeros_like(W, dtype=np.float64)
+    eps = 1e-5
+    for idx in np.ndindex(*W.shape):
+        Wp, Wm = W.astype(np.float64), W.astype(np.float64)
+        Wp[idx] += eps
+        Wm[idx] -= eps
+        fd[idx] = (O.fp64_layer_loss(spec, X, Wp, B) - O.fp64_layer_loss(spec, X, Wm, B)) / (2 * eps)
+    cos = float((st.dW * fd).sum() / (np.linalg.norm(st.dW) * np.linalg.norm(fd)))
+    assert cos > 0.98, cos
