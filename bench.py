@@ -140,19 +140,23 @@ def algorithmic_work(w, B: int):
     """Algorithmic bytes (memory-bound kernels) and INT8 ops (contractions) of ONE train step, per
     kernel kind, from the layer shapes: absmax reads 4 B/element, the quantisers read 4 B and write
     1 B per element, a contraction does 2*rows*N*K operations."""
-    out = {k: 0.0 for k in ("absmax", "quantize", "normalize", "dh_quantize", "fwd_gemm", "upd_gemm")}
+    out = {k: 0.0 for k in ("absmax", "quantize", "normalize", "dh_quantize", "fwd_gemm", "upd_gemm", "dw_fwd", "dw_upd")}
     for i, l in enumerate(w.layers):
-        R = l.H * l.Wd
-        rows = 2 * B * R
-        kin = l.Cin if l.kind == 1 else l.K
+        st = getattr(l, "stride", 1) if l.kind in (1, 3) else 1
+        rows = 2 * B * ((l.H - 1) // st + 1) * ((l.Wd - 1) // st + 1)      # output positions of both sets
+        kin = l.Cin if l.kind in (1, 3) else l.K
         n_w = l.N * l.K
-        n_x = rows * kin
+        n_x = 2 * B * l.H * l.Wd * kin
         n_y = rows * l.N
         out["absmax"] += 4.0 * n_w + (4.0 * n_x if i == 0 else 0.0)
         out["quantize"] += 5.0 * n_w + (5.0 * n_x if i == 0 else 0.0)
         if i + 1 < len(w.layers):
             out["normalize"] += 5.0 * n_y            # reads Y, writes the next layer's INT8 input
         out["dh_quantize"] += 5.0 * n_y
+        if l.kind == 3:       # depthwise: streaming kernels, bytes not operations
+            out["dw_fwd"] += 1.0 * n_x + 4.0 * n_y
+            out["dw_upd"] += 1.0 * n_x + 1.0 * n_y
+            continue
         out["fwd_gemm"] += 2.0 * rows * l.N * l.K
         out["upd_gemm"] += 2.0 * rows * l.N * l.K
     return out

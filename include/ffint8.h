@@ -52,7 +52,7 @@ typedef enum {
   FF_ERR_UNSUPPORTED_ARCH = -8 /* the device is not compute capability 10.x                    */
 } ff_status;
 
-enum { FF_LINEAR = 0, FF_CONV3X3 = 1, FF_CONV1X1 = 2 };  /* ff_layer_desc.kind      */
+enum { FF_LINEAR = 0, FF_CONV3X3 = 1, FF_CONV1X1 = 2, FF_DWCONV3X3 = 3 };  /* ff_layer_desc.kind */
 enum { FF_ROUND_NEAREST_EVEN = 0, FF_ROUND_STOCHASTIC = 1 }; /* rounding modes (Sec. IV-B) */
 enum { FF_GEMM_AUTO = 0, FF_GEMM_SIMT = 1, FF_GEMM_TENSOR = 2 }; /* ff_set_gemm_path       */
 
@@ -69,7 +69,9 @@ enum {
  * conv3x3 (stride 1 or 2, zero padding 1, NHWC): X[M,H,Wd,Cin] -> Y[M,Ho,Wo,N], W[N,3,3,Cin] stored
  * as [N,K] with K = 9*Cin and k = (r*3+s)*Cin + ci; Ho = H, Wo = Wd at stride 1.
  * conv1x1 (pointwise, NHWC): X[M,H,Wd,Cin] -> Y[M,H,Wd,N], W[N,Cin], K = Cin: the dense MAC applied
- * at every position; goodness and normalisation over all H*Wd*N values of a sample. */
+ * at every position; goodness and normalisation over all H*Wd*N values of a sample.
+ * dwconv3x3 (depthwise: one 3x3 filter per channel, no sum over channels; stride 1 or 2, zero padding 1,
+ * NHWC): X[M,H,Wd,C] -> Y[M,Ho,Wo,C] with N = Cin = C, K = 9, W[C,3,3] stored as [C,9] (k = r*3+s). */
 typedef struct {
   int32_t kind;
   int32_t K, N;
@@ -80,7 +82,7 @@ typedef struct {
   float lr;             /* SGD step size of the update (Alg. 1 line 9)                        */
   float tau, eps;       /* length normalisation of the output: x = y*tau/(sqrt(G)+eps), eps>0 */
   uint64_t seed;        /* keys the stochastic-rounding hash                                  */
-  int32_t stride;       /* conv3x3 only: 0 or 1 = every position, 2 = every second row and column; */
+  int32_t stride;       /* conv3x3 / dwconv3x3 only: 0 or 1 = every position, 2 = every second row and column; */
                         /* the output then has Ho = (H-1)/2 + 1 rows of Wo = (Wd-1)/2 + 1 positions */
   float momentum;       /* update rule: 0 = plain SGD (W -= lr*g); mu > 0 = heavy-ball SGD on the   */
                         /* buffer Mom: m = mu*m + g, W -= lr*m (the paper names no optimiser)       */
@@ -271,6 +273,8 @@ enum {
   FF_K_UPD_GEMM,     /* g^W INT8 MAC + SGD update epilogue                                       */
   FF_K_RAW_GEMM,     /* ff_int8_gemm                                                             */
   FF_K_CLASSIFY,     /* ff_predict: per-candidate goodness totals and their argmax               */
+  FF_K_DW_FWD,       /* depthwise 3x3 forward MAC + dequantise/ReLU/goodness                     */
+  FF_K_DW_UPD,       /* depthwise 3x3 g^W sums + update                                          */
   FF_K_COUNT
 };
 ff_status ff_profile_start(ff_ctx* ctx);

@@ -12,7 +12,7 @@ from . import build as _build
 FF_OK = 0
 FF_ERR_ARG, FF_ERR_ALIGN, FF_ERR_WORKSPACE, FF_ERR_NONFINITE = -1, -2, -3, -4
 FF_ERR_RANGE, FF_ERR_DEVICE_TIMEOUT, FF_ERR_CUDA, FF_ERR_UNSUPPORTED_ARCH = -5, -6, -7, -8
-FF_LINEAR, FF_CONV3X3, FF_CONV1X1 = 0, 1, 2
+FF_LINEAR, FF_CONV3X3, FF_CONV1X1, FF_DWCONV3X3 = 0, 1, 2, 3
 FF_ROUND_NEAREST_EVEN, FF_ROUND_STOCHASTIC = 0, 1
 FF_GEMM_AUTO, FF_GEMM_SIMT, FF_GEMM_TENSOR = 0, 1, 2
 FF_A_X_POS, FF_A_X_NEG, FF_A_W, FF_A_DH_POS, FF_A_DH_NEG, FF_A_XNEXT_POS, FF_A_XNEXT_NEG = range(7)
@@ -26,7 +26,7 @@ EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", 
            "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict"]
 FF_STATIC_LOSS_MAX_SAMPLES = 65536
 FF_K_NAMES = ["absmax", "quantize", "fwd_gemm", "finalize", "normalize", "loss", "dh_quantize",
-              "upd_gemm", "raw_gemm", "classify"]
+              "upd_gemm", "raw_gemm", "classify", "dw_fwd", "dw_upd"]
 
 
 class ff_layer_desc(C.Structure):
@@ -266,7 +266,7 @@ class LayerBuffers:
     def __init__(self, desc: ff_layer_desc, B: int, device, dumps: bool = False, xnext: bool = True,
                  own_x: bool = True, accw: bool = False):
         import torch
-        st = 2 if (desc.kind == FF_CONV3X3 and desc.stride == 2) else 1
+        st = 2 if (desc.kind in (FF_CONV3X3, FF_DWCONV3X3) and desc.stride == 2) else 1
         Rin = desc.H * desc.Wd if desc.kind != FF_LINEAR else 1                    # input rows per sample
         R = ((desc.H - 1) // st + 1) * ((desc.Wd - 1) // st + 1) if desc.kind != FF_LINEAR else 1   # output rows
         kin = desc.Cin if desc.kind != FF_LINEAR else desc.K

@@ -15,6 +15,7 @@
 #include "elementwise.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "dwconv.cuh"
 
 using namespace ffi8;
 
@@ -121,19 +122,22 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // output rows (positions) per sample, and input rows per sample (they differ for a strided convolution)
 inline int rows_per_sample(const ff_layer_desc& L) { return L.kind != FF_LINEAR ? tc_out_h(L) * tc_out_w(L) : 1; }
 inline int in_rows_per_sample(const ff_layer_desc& L) { return L.kind != FF_LINEAR ? L.H * L.Wd : 1; }
-inline int in_features(const ff_layer_desc& L) { return L.kind == FF_CONV3X3 ? L.Cin : L.K; }
+inline int in_features(const ff_layer_desc& L) { return (L.kind == FF_CONV3X3 || L.kind == FF_DWCONV3X3) ? L.Cin : L.K; }
 
 ff_status check_layer(ff_ctx* ctx, const ff_layer_desc* L, int B) {
   if (!L) return fail(ctx, FF_ERR_ARG, "layer descriptor is NULL");
   if (B <= 0) return fail(ctx, FF_ERR_ARG, "B must be positive");
-  if (L->kind != FF_LINEAR && L->kind != FF_CONV3X3 && L->kind != FF_CONV1X1) return fail(ctx, FF_ERR_ARG, "unknown layer kind");
+  if (L->kind != FF_LINEAR && L->kind != FF_CONV3X3 && L->kind != FF_CONV1X1 && L->kind != FF_DWCONV3X3)
+    return fail(ctx, FF_ERR_ARG, "unknown layer kind");
+  if (L->kind == FF_DWCONV3X3 && (L->H <= 0 || L->Wd <= 0 || L->Cin <= 0 || L->N != L->Cin || L->K != 9))
+    return fail(ctx, FF_ERR_ARG, "dwconv3x3 needs H, Wd, Cin > 0, N = Cin and K = 9");
   if (L->kind == FF_CONV1X1 && (L->H <= 0 || L->Wd <= 0 || L->Cin <= 0 || L->K != L->Cin))
     return fail(ctx, FF_ERR_ARG, "conv1x1 needs H, Wd, Cin > 0 and K = Cin");
   if (L->K <= 0 || L->N <= 0) return fail(ctx, FF_ERR_ARG, "K and N must be positive");
   if (L->kind == FF_CONV3X3 && (L->H <= 0 || L->Wd <= 0 || L->Cin <= 0 || L->K != 9 * L->Cin))
     return fail(ctx, FF_ERR_ARG, "conv3x3 needs H, Wd, Cin > 0 and K = 9*Cin");
-  if (L->stride < 0 || L->stride > 2 || (L->stride == 2 && L->kind != FF_CONV3X3))
-    return fail(ctx, FF_ERR_ARG, "stride must be 0 / 1, or 2 for a conv3x3 layer");
+  if (L->stride < 0 || L->stride > 2 || (L->stride == 2 && L->kind != FF_CONV3X3 && L->kind != FF_DWCONV3X3))
+    return fail(ctx, FF_ERR_ARG, "stride must be 0 / 1, or 2 for a conv3x3 / dwconv3x3 layer");
   for (int r : {L->round_x, L->round_w, L->round_dh})
     if (r != FF_ROUND_NEAREST_EVEN && r != FF_ROUND_STOCHASTIC) return fail(ctx, FF_ERR_ARG, "unknown rounding mode");
   if (!(L->eps > 0.0f)) return fail(ctx, FF_ERR_ARG, "eps must be > 0");
@@ -323,7 +327,84 @@ ff_status launch_im2col(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs
 }
 
 // Forward contraction + fused epilogue.
+// ---- depthwise layers: streaming kernels of their own (no contraction) ------------------------------
+inline DwGeom dw_geom(const ff_layer_desc& L, int B) {
+  DwGeom g;
+  g.H = L.H, g.W = L.Wd, g.C = L.Cin, g.Ho = tc_out_h(L), g.Wo = tc_out_w(L), g.stride = tc_conv_stride(L);
+  g.rows_per_sample = g.Ho * g.Wo;
+  g.rows_per_pass = B * g.rows_per_sample;
+  g.rows = 2 * g.rows_per_pass;
+  g.imgs_per_pass = B;
+  g.wblocks = (g.Wo + DW_WB - 1) / DW_WB;
+  return g;
+}
+// four channels per thread need whole words; the per-channel weight table must fit the default shared memory
+inline bool dw_vec(const ff_layer_desc& L) { return L.Cin % 4 == 0 && (size_t)L.Cin * 36 <= 40 * 1024; }
+
+ff_status dw_forward(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  const DwGeom g = dw_geom(L, B);
+  ProfScope prof(ctx, FF_K_DW_FWD, st);
+  unsigned long long* S = reinterpret_cast<unsigned long long*>(b.S);
+  if (dw_vec(L)) {
+    const size_t items = (size_t)2 * B * g.Ho * g.wblocks * (g.C / 4);
+    const int grid = ew_blocks(ctx, items, 1);
+    if (g.stride == 2)
+      dwconv3x3_fwd_kernel<2><<<grid, DW_THREADS, (size_t)g.C * 36, st>>>(b.Xq, b.Wq, b.Y, b.acc_dump, S, b.rowmax, b.absmax, g);
+    else
+      dwconv3x3_fwd_kernel<1><<<grid, DW_THREADS, (size_t)g.C * 36, st>>>(b.Xq, b.Wq, b.Y, b.acc_dump, S, b.rowmax, b.absmax, g);
+  } else {
+    const int grid = ew_blocks(ctx, (size_t)g.rows * g.C, 1);
+    dwconv3x3_fwd_scalar_kernel<<<grid, DW_THREADS, 0, st>>>(b.Xq, b.Wq, b.Y, b.acc_dump, S, b.rowmax, b.absmax, g);
+  }
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
+
+// INT32 sums of both sets into the workspace ([2][C][9], cleared first), then the common reduce / update kernel.
+ff_status dw_update(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  const DwGeom g = dw_geom(L, B);
+  const size_t bytes = (size_t)2 * g.C * 9 * sizeof(int32_t);
+  if (ctx->workspace_bytes < WS_BYTES + bytes)
+    return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the depthwise weight-gradient sums");
+  int32_t* accW = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
+  ProfScope prof(ctx, FF_K_DW_UPD, st);
+  const bool was = ctx->profiling;
+  ctx->profiling = false;  // one event pair around the whole route
+  cudaError_t e = cudaMemsetAsync(accW, 0, bytes, st);
+  if (e != cudaSuccess) {
+    ctx->profiling = was;
+    return fail(ctx, FF_ERR_CUDA, "%s", cudaGetErrorString(e));
+  }
+  if (L.Cin % 4 == 0) {
+    const int tiles = (g.C / 4 + 31) / 32;
+    const int pb_total = B * g.Ho * g.wblocks;
+    // enough chunks to occupy the device several times over, at least 32 position blocks each
+    int chunks = (ctx->sm_count * 8 + 2 * tiles - 1) / (2 * tiles);
+    const int max_chunks = (pb_total + 31) / 32;
+    if (chunks > max_chunks) chunks = max_chunks;
+    const int per = (pb_total + chunks - 1) / chunks;
+    const dim3 grid((pb_total + per - 1) / per, tiles, 2);
+    if (g.stride == 2)
+      dwconv3x3_wgrad_kernel<2><<<grid, DW_THREADS, 0, st>>>(b.dHq, b.Xq, accW, g, per);
+    else
+      dwconv3x3_wgrad_kernel<1><<<grid, DW_THREADS, 0, st>>>(b.dHq, b.Xq, accW, g, per);
+  } else {
+    int chunks = ctx->sm_count * 4;
+    const int max_chunks = (g.rows_per_pass + 63) / 64;
+    if (chunks > max_chunks) chunks = max_chunks;
+    const int per = (g.rows_per_pass + chunks - 1) / chunks;
+    dwconv3x3_wgrad_scalar_kernel<<<dim3((g.rows_per_pass + per - 1) / per, 1, 2), DW_THREADS, 0, st>>>(b.dHq, b.Xq, accW, g, per);
+  }
+  ctx->launches++;
+  ff_status s = FF_OK;
+  if ((e = cudaGetLastError()) != cudaSuccess) s = fail(ctx, FF_ERR_CUDA, "launch: %s", cudaGetErrorString(e));
+  if (s == FF_OK) s = launch_slab_update(ctx, accW, 1, L, b, st, 0);
+  ctx->profiling = was;
+  return s;
+}
+
 ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  if (L.kind == FF_DWCONV3X3) return dw_forward(ctx, L, b, B, st);
   const int R = rows_per_sample(L);
   const int rows = 2 * B * R;
   bool tc_ok = tc_forward_supported(L, B);
@@ -359,6 +440,7 @@ ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
 // Weight-gradient contraction + fused update.
 ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
   if (L.momentum != 0.0f && !b.Mom) return fail(ctx, FF_ERR_ARG, "momentum != 0 needs the buffer Mom");
+  if (L.kind == FF_DWCONV3X3) return dw_update(ctx, L, b, B, st);
   const int R = rows_per_sample(L);
   const int rows = 2 * B * R;
   bool tc_ok = tc_update_supported(L, B);
@@ -868,6 +950,7 @@ ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, s
       const size_t n1 = sp1 >= 2 ? (size_t)sp1 * 2 * layers[l].N * layers[l].K * sizeof(int32_t) : 0;
       if (n1 > need) need = n1;
     }
+    if (layers[l].kind == FF_DWCONV3X3) need = (size_t)2 * layers[l].N * 9 * sizeof(int32_t);
     if (tc_im2col_ok(layers[l])) {
       const Im2colPlan pl = im2col_plan(layers[l], B, SIZE_MAX, 0);
       const size_t im_need = pl.slab_off - WS_BYTES + (size_t)pl.max_splits * pl.slab_bytes_per_split;

@@ -926,7 +926,9 @@ inline ff_status tc_make_map_nhwc(TcState& t, CUtensorMap* tm, const int8_t* bas
   cuuint32_t estr[4] = {1, stride, stride, 1};
   return tc_encode(t, tm, base, 4, dims, strides, box, (int)ch_box, estr);
 }
-inline int tc_conv_stride(const ff_layer_desc& L) { return (L.kind == FF_CONV3X3 && L.stride == 2) ? 2 : 1; }
+inline int tc_conv_stride(const ff_layer_desc& L) {
+  return ((L.kind == FF_CONV3X3 || L.kind == FF_DWCONV3X3) && L.stride == 2) ? 2 : 1;
+}
 inline int tc_out_h(const ff_layer_desc& L) { return (L.H - 1) / tc_conv_stride(L) + 1; }
 inline int tc_out_w(const ff_layer_desc& L) { return (L.Wd - 1) / tc_conv_stride(L) + 1; }
 

@@ -73,6 +73,13 @@ def workload(name: str) -> Workload:
         layers = [LayerCfg(1, 9 * ci, co, float(co * 1024), 0.03 / 1024.0, float(np.sqrt(co * 1024)),
                            H=32, Wd=32, Cin=ci) for ci, co in zip(chans[:-1], chans[1:])]
         return Workload(name, 256, layers, (32, 32, 3), "normal", "kaiming_uniform", 50)
+    if name == "separable":         # beyond the five configurations: one inverted-residual-style block (without the
+        # skip connection) of the paper's mobile models at CIFAR size: pointwise 32 -> 192, depthwise 3x3 on 192
+        # channels, pointwise 192 -> 64, all 32 x 32; theta and step size as for the CNN workload
+        hw = 32 * 32
+        mk = lambda kind, K, N, cin: LayerCfg(kind, K, N, float(N * hw), 0.03 / hw, float(np.sqrt(N * hw)), H=32, Wd=32, Cin=cin)
+        layers = [mk(2, 32, 192, 32), mk(3, 9, 192, 192), mk(2, 192, 64, 192)]
+        return Workload(name, 256, layers, (32, 32, 32), "normal", "kaiming_uniform", 50)
     if name == "roofline":          # config 5
         return Workload(name, 16384, [LayerCfg(0, 8192, 8192, 4096.0, 0.03, float(np.sqrt(8192)))],
                         (8192,), "normal", "normal_1_over_k", 100)
