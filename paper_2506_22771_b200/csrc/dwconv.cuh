@@ -29,17 +29,60 @@ struct DwWindow {
   static constexpr int NW = (DW_WB - 1) * STRIDE + 3;
   uint32_t w[3][NW];
   __device__ __forceinline__ void load(const int8_t* __restrict__ xq, int img, int hh0, int ww0, int cg, const DwGeom& g) {
+    const size_t pix = (size_t)g.C, line = (size_t)g.W * pix;
+    if (hh0 >= 0 && hh0 + 3 <= g.H && ww0 >= 0 && ww0 + NW <= g.W) {
+      // the whole window lies inside the image: one base address, constant offsets, no tests
+      const int8_t* base = xq + (((size_t)img * g.H + hh0) * g.W + ww0) * pix + 4 * (size_t)cg;
+#pragma unroll
+      for (int r = 0; r < 3; ++r)
+#pragma unroll
+        for (int i = 0; i < NW; ++i) w[r][i] = __ldg(reinterpret_cast<const uint32_t*>(base + r * line + i * pix));
+      return;
+    }
 #pragma unroll
     for (int r = 0; r < 3; ++r) {
       const int hh = hh0 + r;
       const bool row_in = hh >= 0 && hh < g.H;
-      const int8_t* rowp = xq + (((size_t)img * g.H + (row_in ? hh : 0)) * g.W) * g.C + 4 * (size_t)cg;
+      const int8_t* rowp = xq + ((size_t)img * g.H + (row_in ? hh : 0)) * line + 4 * (size_t)cg;
 #pragma unroll
       for (int i = 0; i < NW; ++i) {
         const int ww = ww0 + i;
-        w[r][i] = (row_in && ww >= 0 && ww < g.W) ? __ldg(reinterpret_cast<const uint32_t*>(rowp + (size_t)ww * g.C)) : 0u;
+        w[r][i] = (row_in && ww >= 0 && ww < g.W) ? __ldg(reinterpret_cast<const uint32_t*>(rowp + (size_t)ww * pix)) : 0u;
       }
     }
+  }
+};
+
+// Position of a work item (four channels cg of output block wb in output row ho of image img) that is
+// advanced by a fixed number of items per loop trip with carries instead of divisions.
+struct DwCursor {
+  int cg, wb, ho, img;
+  int d_cg, d_wb, d_ho, d_img;
+  int CG, WBK, Ho;
+  __device__ __forceinline__ DwCursor(uint32_t item, uint32_t step, int CG_, int WBK_, int Ho_) : CG(CG_), WBK(WBK_), Ho(Ho_) {
+    split(item, cg, wb, ho, img);
+    split(step, d_cg, d_wb, d_ho, d_img);
+  }
+  __device__ __forceinline__ void split(uint32_t v, int& c, int& w, int& h, int& i) const {
+    uint32_t q = v / (uint32_t)CG;
+    c = (int)(v - q * CG);
+    uint32_t q2 = q / (uint32_t)WBK;
+    w = (int)(q - q2 * WBK);
+    uint32_t q3 = q2 / (uint32_t)Ho;
+    h = (int)(q2 - q3 * Ho);
+    i = (int)q3;
+  }
+  __device__ __forceinline__ void advance() {
+    cg += d_cg;
+    int c = cg >= CG;
+    cg -= c ? CG : 0;
+    wb += d_wb + c;
+    c = wb >= WBK;
+    wb -= c ? WBK : 0;
+    ho += d_ho + c;
+    c = ho >= Ho;
+    ho -= c ? Ho : 0;
+    img += d_img + c;
   }
 };
 
@@ -54,8 +97,6 @@ __global__ void __launch_bounds__(DW_THREADS) dwconv3x3_fwd_kernel(const int8_t*
                                                                   unsigned long long* __restrict__ S, int32_t* __restrict__ rowmax,
                                                                   const float* __restrict__ absmax, DwGeom g) {
   extern __shared__ uint32_t dw_tab[];  // [C/4][9][4] words
-  __shared__ unsigned long long red_s[DW_THREADS / 32];
-  __shared__ int red_m[DW_THREADS / 32], red_id[DW_THREADS / 32];
   const uint32_t CG = (uint32_t)g.C >> 2;
   for (uint32_t i = threadIdx.x; i < CG * 36; i += DW_THREADS) {
     const uint32_t cg = i / 36, rem = i - cg * 36, t = rem >> 2, j = rem & 3;
@@ -65,99 +106,86 @@ __global__ void __launch_bounds__(DW_THREADS) dwconv3x3_fwd_kernel(const int8_t*
   const float s_w = scale_of(absmax[2]);
   const float c0 = __fmul_rn(scale_of(absmax[0]), s_w), c1 = __fmul_rn(scale_of(absmax[1]), s_w);
   const uint32_t total = (uint32_t)(2 * g.imgs_per_pass) * g.Ho * g.wblocks * CG;  // < 2^32: fewer items than outputs
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  // whole blocks iterate together: the reductions below synchronise
-  for (uint32_t base = blockIdx.x * DW_THREADS; base < total; base += gridDim.x * DW_THREADS) {
-    const uint32_t item = base + threadIdx.x;
-    const bool valid = item < total;
+  const int lane = threadIdx.x & 31;
+  // a block takes a contiguous range of items, so that a warp stays inside one sample for many trips and its
+  // goodness statistics can ride in registers until the sample changes
+  const uint32_t per_block = ((total + gridDim.x - 1) / gridDim.x + DW_THREADS - 1) / DW_THREADS * DW_THREADS;
+  const uint32_t begin = min(total, blockIdx.x * per_block), end = min(total, begin + per_block);
+  DwCursor cur(begin + threadIdx.x, DW_THREADS, (int)CG, g.wblocks, g.Ho);
+  int held = -1;  // sample whose statistics the warp is holding (warp-uniform), -1: none
+  unsigned long long ssum = 0ull;
+  int mx = 0;
+  auto flush = [&]() {
+    if (held >= 0) {
+      for (int o = 16; o > 0; o >>= 1) ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
+      mx = __reduce_max_sync(0xffffffffu, mx);
+      if (lane == 0 && mx > 0) {
+        atomicAdd(S + held, ssum);
+        atomicMax(rowmax + held, mx);
+      }
+    }
+    held = -1;
+    ssum = 0ull;
+    mx = 0;
+  };
+  for (uint32_t base = begin + (threadIdx.x & ~31u); base < end; base += DW_THREADS, cur.advance()) {
+    const bool valid = base + lane < end;
+    const int img = valid ? cur.img : -1;
+    const int first = __shfl_sync(0xffffffffu, img, 0), last = __shfl_sync(0xffffffffu, img, 31);
+    const bool uniform = first == last;  // every lane valid and in the same sample
+    if (!uniform || first != held) flush();
+    if (uniform) held = first;
+    if (!valid) continue;
+    const int ho = cur.ho, wo0 = cur.wb * DW_WB, cg = cur.cg;
     int acc[DW_WB][4];
 #pragma unroll
     for (int o = 0; o < DW_WB; ++o)
 #pragma unroll
       for (int j = 0; j < 4; ++j) acc[o][j] = 0;
-    int img = -1, ho = 0, wo0 = 0;
-    uint32_t cg = 0;
-    if (valid) {
-      const uint32_t pb = item / CG;
-      cg = item - pb * CG;
-      const uint32_t t = pb / g.wblocks;
-      wo0 = (int)(pb - t * g.wblocks) * DW_WB;
-      img = (int)(t / g.Ho);
-      ho = (int)(t - (uint32_t)img * g.Ho);
-      DwWindow<STRIDE> win;
-      win.load(xq, img, ho * STRIDE - 1, wo0 * STRIDE - 1, (int)cg, g);
+    DwWindow<STRIDE> win;
+    win.load(xq, img, ho * STRIDE - 1, wo0 * STRIDE - 1, cg, g);
 #pragma unroll
-      for (int r = 0; r < 3; ++r)
+    for (int r = 0; r < 3; ++r)
 #pragma unroll
-        for (int s = 0; s < 3; ++s) {
-          const uint4 tw = *reinterpret_cast<const uint4*>(dw_tab + (cg * 9 + r * 3 + s) * 4);
+      for (int s = 0; s < 3; ++s) {
+        const uint4 tw = *reinterpret_cast<const uint4*>(dw_tab + (cg * 9 + r * 3 + s) * 4);
 #pragma unroll
-          for (int o = 0; o < DW_WB; ++o) {
-            const int xw = (int)win.w[r][o * STRIDE + s];
-            acc[o][0] = __dp4a(xw, (int)tw.x, acc[o][0]);
-            acc[o][1] = __dp4a(xw, (int)tw.y, acc[o][1]);
-            acc[o][2] = __dp4a(xw, (int)tw.z, acc[o][2]);
-            acc[o][3] = __dp4a(xw, (int)tw.w, acc[o][3]);
-          }
+        for (int o = 0; o < DW_WB; ++o) {
+          const int xw = (int)win.w[r][o * STRIDE + s];
+          acc[o][0] = __dp4a(xw, (int)tw.x, acc[o][0]);
+          acc[o][1] = __dp4a(xw, (int)tw.y, acc[o][1]);
+          acc[o][2] = __dp4a(xw, (int)tw.z, acc[o][2]);
+          acc[o][3] = __dp4a(xw, (int)tw.w, acc[o][3]);
         }
-    }
+      }
     const float c = img < g.imgs_per_pass ? c0 : c1;
-    unsigned long long ssum = 0ull;
-    int mx = 0;
+    unsigned long long ts = 0ull;
+    int tm = 0;
+    const size_t off0 = (((size_t)img * g.Ho + ho) * g.Wo + wo0) * g.C + 4 * (size_t)cg;
 #pragma unroll
     for (int o = 0; o < DW_WB; ++o) {
-      if (!valid || wo0 + o >= g.Wo) continue;
+      if (wo0 + o >= g.Wo) break;
       float y[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int a = max(acc[o][j], 0);
         y[j] = __fmul_rn(__uint2float_rn((unsigned)a), c);
-        ssum += (unsigned long long)a * (unsigned long long)a;
-        mx = max(mx, a);
+        ts += (unsigned long long)(unsigned)a * (unsigned long long)(unsigned)a;  // up to (9*127*127)^2: needs 64 bits
+        tm = max(tm, a);
       }
-      const size_t off = (((size_t)img * g.Ho + ho) * g.Wo + wo0 + o) * g.C + 4 * (size_t)cg;
+      const size_t off = off0 + (size_t)o * g.C;
       __stcs(reinterpret_cast<float4*>(Y + off), make_float4(y[0], y[1], y[2], y[3]));
       if (acc_dump) *reinterpret_cast<int4*>(acc_dump + off) = make_int4(acc[o][0], acc[o][1], acc[o][2], acc[o][3]);
     }
-    // goodness statistics: reduced over the warp, then over the block, wherever the values belong to one sample
-    const int sample = valid ? img : -1;
-    const int s_first = __shfl_sync(0xffffffffu, sample, 0), s_last = __shfl_sync(0xffffffffu, sample, 31);
-    int warp_id = -2;  // -2: this warp's lanes have gone to the atomics themselves
-    if (s_first == s_last) {
-      for (int o = 16; o > 0; o >>= 1) ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
-      mx = __reduce_max_sync(0xffffffffu, mx);
-      warp_id = s_first;  // -1: nothing valid
-    } else if (valid && mx > 0) {
-      atomicAdd(S + sample, ssum);
-      atomicMax(rowmax + sample, mx);
+    if (uniform) {
+      ssum += ts;
+      mx = max(mx, tm);
+    } else if (tm > 0) {  // a warp that straddles two samples (or the end of the range): every lane for itself
+      atomicAdd(S + img, ts);
+      atomicMax(rowmax + img, tm);
     }
-    if (lane == 0) {
-      red_s[wid] = ssum;
-      red_m[wid] = mx;
-      red_id[wid] = warp_id;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int i = 0;
-      while (i < DW_THREADS / 32) {  // runs of equal sample ids among the warps' results
-        const int id = red_id[i];
-        unsigned long long ts = red_s[i];
-        int tm = red_m[i];
-        int k = i + 1;
-        while (k < DW_THREADS / 32 && red_id[k] == id) {
-          ts += red_s[k];
-          tm = max(tm, red_m[k]);
-          ++k;
-        }
-        if (id >= 0 && tm > 0) {
-          atomicAdd(S + id, ts);
-          atomicMax(rowmax + id, tm);
-        }
-        i = k;
-      }
-    }
-    __syncthreads();
   }
+  flush();
 }
 
 // Forward for any channel count: one thread per output value (slow path for C % 4 != 0).
@@ -215,11 +243,12 @@ __global__ void __launch_bounds__(DW_THREADS) dwconv3x3_wgrad_kernel(const int8_
   const int pb_total = g.imgs_per_pass * g.Ho * g.wblocks;  // position blocks of one set
   const int pb_begin = blockIdx.x * pb_per_block;
   const int pb_end = min(pb_total, pb_begin + pb_per_block);
-  if (cg < CG) {
-    for (int pb = pb_begin + slot; pb < pb_end; pb += DW_THREADS / 32) {
-      const int t = pb / g.wblocks, wo0 = (pb - t * g.wblocks) * DW_WB;
-      const int img_l = t / g.Ho, ho = t - img_l * g.Ho;
-      const int img = p * g.imgs_per_pass + img_l;
+  if (cg < CG && pb_begin + slot < pb_end) {
+    // (cg = 0, step in position blocks: the cursor's channel digit stays put)
+    DwCursor cur((uint32_t)(pb_begin + slot), DW_THREADS / 32, 1, g.wblocks, g.Ho);
+    for (int pb = pb_begin + slot; pb < pb_end; pb += DW_THREADS / 32, cur.advance()) {
+      const int wo0 = cur.wb * DW_WB, ho = cur.ho;
+      const int img = p * g.imgs_per_pass + cur.img;
       uint32_t dh[DW_WB];
       uint32_t any = 0u;
       const int8_t* dp = dhq + ((((size_t)img * g.Ho + ho) * g.Wo + wo0) * g.C) + 4 * (size_t)cg;
