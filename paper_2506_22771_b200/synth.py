@@ -120,11 +120,8 @@ def make_weights(w: Workload, seed: int) -> List[np.ndarray]:
     return out
 
 
-def make_batch(w: Workload, seed: int, batch_index: int = 0, B: int = None) -> np.ndarray:
-    """One batch [2B, *in_shape] FP32: rows 0..B-1 positive (true label), B..2B-1 negative (a
-    random wrong label), label written one-hot into the first 10 entries (CNN: channel 0, row 0,
-    pixels 0..9), each sample scaled to length tau0 = sqrt(number of input values)."""
-    B = B or w.B
+def _draw_labelled(w: Workload, seed: int, batch_index: int, B: int):
+    """B raw samples (float64), their labels and one wrong label each."""
     g = _rng(seed, 2000 + batch_index)
     n_in = int(np.prod(w.in_shape))
     if w.data == "uniform01":
@@ -133,6 +130,25 @@ def make_batch(w: Workload, seed: int, batch_index: int = 0, B: int = None) -> n
         base = g.normal(0.0, 1.0, size=(B, n_in))
     label = g.integers(0, 10, size=B)
     wrong = (label + g.integers(1, 10, size=B)) % 10
+    return base, label, wrong
+
+
+def make_raw(w: Workload, seed: int, batch_index: int = 0, B: int = None):
+    """The labelled samples make_batch builds its batch from: (samples [B, n_in] FP32, labels [2, B] INT32 with
+    row 0 the true and row 1 the wrong label, label stride = distance in values between two label places)."""
+    B = B or w.B
+    base, label, wrong = _draw_labelled(w, seed, batch_index, B)
+    stride = 1 if len(w.in_shape) == 1 else int(w.in_shape[-1])
+    return np.ascontiguousarray(base.astype(F32)), np.stack([label, wrong]).astype(np.int32), stride
+
+
+def make_batch(w: Workload, seed: int, batch_index: int = 0, B: int = None) -> np.ndarray:
+    """One batch [2B, *in_shape] FP32: rows 0..B-1 positive (true label), B..2B-1 negative (a
+    random wrong label), label written one-hot into the first 10 entries (CNN: channel 0, row 0,
+    pixels 0..9), each sample scaled to length tau0 = sqrt(number of input values)."""
+    B = B or w.B
+    base, label, wrong = _draw_labelled(w, seed, batch_index, B)
+    n_in = base.shape[1]
     x = np.concatenate([base, base], axis=0).reshape((2 * B,) + tuple(w.in_shape))
     for p, lab in enumerate((label, wrong)):
         rows = np.arange(B) + p * B

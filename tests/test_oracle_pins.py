@@ -686,12 +686,10 @@ def test_embed_labels_matches_the_batch_generator_and_has_unit_invariants():
     # rebuild one of its batches from those base samples and compare
     w = synth.workload("tiny_mlp")
     B, n = 16, int(np.prod(w.in_shape))
-    g = synth._rng(7, 2000)
-    base = g.random((B, n), dtype=np.float64)
-    label = g.integers(0, 10, size=B)
-    wrong = (label + g.integers(1, 10, size=B)) % 10
+    raw, labels, stride = synth.make_raw(w, 7, B=B)
+    base, (label, wrong) = raw.astype(np.float64), labels
     want = synth.make_batch(w, 7, B=B).reshape(2 * B, n)
-    got = O.embed_labels(base.astype(np.float32), np.stack([label, wrong]), 10, tau0=float(np.sqrt(n)))
+    got = O.embed_labels(raw, labels, 10, label_stride=stride, tau0=float(np.sqrt(n)))
     assert np.allclose(got, want, rtol=2e-6, atol=0.0)
     # invariants: length tau0, label places one-hot, data entries of both sets parallel to the raw sample
     assert np.allclose(np.sqrt((got.astype(np.float64) ** 2).sum(1)), np.sqrt(n), rtol=1e-6)
