@@ -1,6 +1,7 @@
 #!/usr/bin/env python
 """Writes tests/golden/fullsize_digests.json: SHA-256 digests of every tensor the CPU oracle produces
-for train steps at the FULL sizes of the five benchmark configurations (the sizes bench.py times).
+for train steps at the FULL sizes of the five benchmark configurations (the sizes bench.py times) and of
+the separable-convolution block.
 
 Calls only oracle/ and the seeded input generators; nothing here comes from the CUDA path.  The GPU
 test tests/test_gpu_fullsize.py recomputes the same digests from the device buffers, so a full-size
@@ -25,7 +26,7 @@ OUT = os.path.join(os.path.dirname(os.path.abspath(__file__)), "fullsize_digests
 SEED = 1
 # workload -> number of consecutive steps run (weights carried from step to step).  Every step of a short
 # run is digested; of a long run the first two steps and every tenth (out["digested"] lists them).
-CASES = {"tiny_mlp": 10, "mlp_greedy": 3, "mlp_lookahead": 50, "cnn": 3, "roofline": 2}
+CASES = {"tiny_mlp": 10, "mlp_greedy": 3, "mlp_lookahead": 50, "cnn": 3, "roofline": 2, "separable": 2}
 
 
 def digested_steps(steps: int):
@@ -48,8 +49,8 @@ def layer_digests(st: O.LayerState, B: int) -> dict:
 
 def run(name: str, steps: int) -> dict:
     w = synth.workload(name)
-    specs = [O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, l.eps, l.H, l.Wd, l.Cin, seed=SEED, index=i)
-             for i, l in enumerate(w.layers)]
+    specs = [O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, l.eps, l.H, l.Wd, l.Cin, seed=SEED, index=i,
+                         stride=l.stride, momentum=l.momentum) for i, l in enumerate(w.layers)]
     Ws = synth.make_weights(w, SEED)
     X = synth.make_batch(w, SEED)
     out = {"B": w.B, "seed": SEED, "greedy": bool(w.greedy), "n_steps": steps, "digested": digested_steps(steps),

@@ -41,14 +41,16 @@ def _descs(w, seed):
     return [ffb.make_desc(l, i, seed) for i, l in enumerate(w.layers)]
 
 
-@pytest.mark.parametrize("name", ["tiny_mlp", "mlp_lookahead", "cnn", "roofline"])
-def test_fullsize_train_steps_match_oracle_digests(name):
+@pytest.mark.parametrize("name,graph", [("tiny_mlp", False), ("mlp_lookahead", False), ("cnn", False), ("roofline", False),
+                                        ("separable", False), ("tiny_mlp", True), ("mlp_lookahead", True)])
+def test_fullsize_train_steps_match_oracle_digests(name, graph):
     if name not in DIG:
         pytest.skip("no digests for this workload in tests/golden/fullsize_digests.json")
     d = DIG[name]
     w = synth.workload(name)
     assert d["B"] == w.B and not d["greedy"]
-    net = GpuNet(_descs(w, d["seed"]), w.B, synth.make_weights(w, d["seed"]), dumps=False, xnext=False, chain=True)
+    net = GpuNet(_descs(w, d["seed"]), w.B, synth.make_weights(w, d["seed"]), dumps=False, xnext=False, chain=True,
+                 graph=graph)             # graph: steps 2.. are replays of the launch sequence captured at step 1
     net.set_input(synth.make_batch(w, d["seed"]))
     digested = d.get("digested", list(range(len(d["steps"]))))
     for step in range(d.get("n_steps", len(d["steps"]))):
