@@ -72,7 +72,10 @@ class LayerSpec:
     seed: int = 0
     index: int = 0        # position of the layer in the network (feeds the rounding hash)
     stride: int = 1       # conv3x3 only: 1 or 2 (output (H-1)//stride + 1 by (Wd-1)//stride + 1)
-    momentum: float = 0.0 # heavy-ball coefficient of the update; 0 = plain SGD
+    momentum: float = 0.0 # heavy-ball coefficient of the update; 0 = plain SGD (Adam: beta1)
+    optimizer: int = 0    # 0 = SGD / heavy ball, 1 = Adam
+    beta2: float = 0.999  # Adam only
+    adam_eps: float = 1e-8
 
     @property
     def out_hw(self):
@@ -408,6 +411,7 @@ class LayerState:
     W_new: np.ndarray = None
     dW: np.ndarray = None      # dequantised weight gradient (float32)
     M_new: np.ndarray = None   # momentum buffer after the update (None for plain SGD)
+    V_new: np.ndarray = None   # Adam's second-moment buffer after the update
 
 
 def _pass_rows(v_pos, v_neg, B):
@@ -460,7 +464,38 @@ def sgd_momentum(W: np.ndarray, M: np.ndarray, g: np.ndarray, lr: float, mu: flo
     return np.asarray(W, dtype=F32) - F32(lr) * M_new, M_new
 
 
-def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int, M: Optional[np.ndarray] = None) -> LayerState:
+def _pow_int(x: float, n: int) -> float:
+    """x**n for n >= 0 by square-and-multiply from the low bit up, every product one float64 rounding
+    (a fixed order, so that any two implementations agree bit for bit)."""
+    r, p = F64(1.0), F64(x)
+    while n > 0:
+        if n & 1:
+            r = r * p
+        n >>= 1
+        if n:
+            p = p * p
+    return r
+
+
+def adam_update(W, M, V, g, lr: float, beta1: float, beta2: float, eps: float, t: int):
+    """Adam (Kingma & Ba 2015, Algorithm 1) for update number t >= 1, the other usual choice where the paper
+    says only 'updated to current weights' (Sec. IV-B; Alg. 1 line 9):
+        m = beta1*m + (1-beta1)*g;  v = beta2*v + (1-beta2)*g*g;
+        W -= lr * (m*c1) / (sqrt(v*c2) + eps),   c_i = float32(1/(1 - beta_i^t)).
+    float32 throughout, one rounding per operation in the order written (1-beta_i is one float32
+    subtraction); the bias corrections come from float64 powers by _pow_int.  Returns (W_new, M_new, V_new)."""
+    b1, b2 = F32(beta1), F32(beta2)
+    g = np.asarray(g, dtype=F32)
+    M_new = b1 * np.asarray(M, dtype=F32) + (F32(1.0) - b1) * g
+    V_new = b2 * np.asarray(V, dtype=F32) + (F32(1.0) - b2) * (g * g)
+    c1 = F32(F64(1.0) / (F64(1.0) - _pow_int(F64(b1), t)))
+    c2 = F32(F64(1.0) / (F64(1.0) - _pow_int(F64(b2), t)))
+    upd = (M_new * c1) / (np.sqrt(V_new * c2) + F32(eps))
+    return np.asarray(W, dtype=F32) - F32(lr) * upd, M_new, V_new
+
+
+def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int, M: Optional[np.ndarray] = None,
+                 V: Optional[np.ndarray] = None, step: int = 0) -> LayerState:
     """g^W per pass as an INT8 MAC, dequantised and applied as plain SGD (Sec. IV-B; Alg. 1
     line 9):  g = float(accP)*cP + float(accN)*cN,  W <- W - lr*g.  With spec.momentum != 0 the
     update is heavy-ball SGD on the momentum buffer M (zeros when None), see sgd_momentum."""
@@ -480,7 +515,11 @@ def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int, M: Opti
     cP = scale_pair(st.a_dh[0])[0] * scale_pair(st.a_x[0])[0]
     cN = scale_pair(st.a_dh[1])[0] * scale_pair(st.a_x[1])[0]
     st.dW = st.accW[0].astype(F32) * cP + st.accW[1].astype(F32) * cN
-    if spec.momentum != 0.0:
+    if spec.optimizer == 1:   # Adam; update number t = step + 1
+        z = np.zeros_like(W)
+        st.W_new, st.M_new, st.V_new = adam_update(W, z if M is None else M, z if V is None else V, st.dW, spec.lr,
+                                                   spec.momentum, spec.beta2, spec.adam_eps, step + 1)
+    elif spec.momentum != 0.0:
         st.W_new, st.M_new = sgd_momentum(W, np.zeros_like(W) if M is None else M, st.dW, spec.lr, spec.momentum)
     else:
         st.W_new = W - F32(spec.lr) * st.dW
@@ -488,7 +527,7 @@ def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int, M: Opti
 
 
 def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: int, lam: float,
-               step: int, Ms: Optional[List[np.ndarray]] = None) -> List[LayerState]:
+               step: int, Ms: Optional[List[np.ndarray]] = None, Vs: Optional[List[np.ndarray]] = None) -> List[LayerState]:
     """Body of Algorithm 1's epoch loop: one INT8 forward through all k layers with the
     pre-update weights (line 5), goodness of every layer (line 6), then for each layer its
     loss from the G's (line 8) and its INT8 gradient and update (line 9).  lambda is the
@@ -504,7 +543,7 @@ def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: i
         later = list(range(l + 1, len(specs)))
         layer_loss_grad(spec, states[l], B, [states[j].G for j in later],
                         [specs[j].theta for j in later], lam, step)
-        layer_update(spec, states[l], W, B, None if Ms is None else Ms[l])
+        layer_update(spec, states[l], W, B, None if Ms is None else Ms[l], None if Vs is None else Vs[l], step)
     return states
 
 

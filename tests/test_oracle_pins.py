@@ -826,3 +826,49 @@ def test_depthwise_layer_step_descends_and_chains():
         fd[idx] = (O.fp64_layer_loss(spec, X, Wp, B) - O.fp64_layer_loss(spec, X, Wm, B)) / (2 * eps)
     cos = float((st.dW * fd).sum() / (np.linalg.norm(st.dW) * np.linalg.norm(fd)))
     assert cos > 0.98, cos
+
+
+# ---- Adam variant of the update ------------------------------------------------------------------------
+def test_pow_int_and_adam_hand_example():
+    assert O._pow_int(0.5, 0) == 1.0 and O._pow_int(0.5, 10) == 2.0 ** -10 and O._pow_int(3.0, 5) == 243.0
+    assert abs(O._pow_int(0.999, 1000) - 0.999 ** 1000) < 1e-13      # ten roundings of relative size 2^-53, amplified by the squarings
+    # first update from zero buffers: m*c1 = g and v*c2 = g*g, so the step is lr*g/(|g|+eps) whatever the betas.
+    # Powers of two keep every operation exact: beta1 = 0.5, beta2 = 0.75, g = 2, eps = 2 -> step = lr*2/4
+    W1, M1, V1 = O.adam_update(np.array([1.0], np.float32), np.zeros(1, np.float32), np.zeros(1, np.float32),
+                               np.array([2.0], np.float32), lr=0.5, beta1=0.5, beta2=0.75, eps=2.0, t=1)
+    assert M1[0] == 1.0 and V1[0] == 1.0 and W1[0] == 0.75
+    # second update with the same gradient: m = 1.5, v = 1.75, c1 = 1/(1-0.25) = 4/3, c2 = 1/(1-0.5625) = 16/7
+    W2, M2, V2 = O.adam_update(W1, M1, V1, np.array([2.0], np.float32), lr=0.5, beta1=0.5, beta2=0.75, eps=2.0, t=2)
+    assert M2[0] == 1.5 and V2[0] == 1.75
+    want = 0.75 - 0.5 * (1.5 * (4.0 / 3.0)) / (np.sqrt(1.75 * 16.0 / 7.0) + 2.0)      # = 0.75 - 0.5*2/4
+    assert abs(W2[0] - want) < 1e-6 and abs(want - 0.5) < 1e-12
+
+
+def test_adam_constant_gradient_and_sign_invariance():
+    # constant gradient: bias-corrected moments equal g and g^2 at every step, so W moves by lr*g/(|g|+eps) per step
+    g = np.array([0.3, -0.02, 5.0], np.float32)
+    W, M, V = np.zeros(3, np.float32), np.zeros(3, np.float32), np.zeros(3, np.float32)
+    for t in range(1, 41):
+        W, M, V = O.adam_update(W, M, V, g, lr=0.01, beta1=0.9, beta2=0.999, eps=1e-8, t=t)
+        assert np.allclose(W, -0.01 * t * np.sign(g), rtol=2e-5, atol=0.0), (t, W)
+    # the step does not depend on the gradient's scale (up to eps), unlike SGD's
+    Wa = O.adam_update(np.zeros(1, np.float32), np.zeros(1, np.float32), np.zeros(1, np.float32), np.array([1e-3], np.float32),
+                       0.1, 0.9, 0.999, 1e-12, 1)[0]
+    Wb = O.adam_update(np.zeros(1, np.float32), np.zeros(1, np.float32), np.zeros(1, np.float32), np.array([1e+3], np.float32),
+                       0.1, 0.9, 0.999, 1e-12, 1)[0]
+    assert np.allclose(Wa, Wb, rtol=1e-6) and np.allclose(Wa, -0.1, rtol=1e-6)
+
+
+def test_layer_update_with_adam_carries_both_buffers():
+    from paper_2506_22771_b200 import synth
+    w = synth.scaled(synth.workload("tiny_mlp"), B=8, width_div=8)
+    l = w.layers[0]
+    spec = O.LayerSpec(l.kind, l.K, l.N, l.theta, 0.001, l.tau, seed=3, momentum=0.9, optimizer=1, beta2=0.99, adam_eps=1e-6)
+    W0 = synth.make_weights(w, 3)[0]
+    X = synth.make_batch(w, 3)
+    a = O.train_step([spec], [W0], X, w.B, 0.0, 0)[0]
+    nz = a.dW != 0
+    assert np.allclose((W0 - a.W_new)[nz], 0.001 * np.sign(a.dW[nz]), rtol=1e-2)       # first step: lr * sign(g)
+    b = O.train_step([spec], [a.W_new], X, w.B, 0.0, 1, Ms=[a.M_new], Vs=[a.V_new])[0]
+    Wn, Mn, Vn = O.adam_update(a.W_new, a.M_new, a.V_new, b.dW, 0.001, 0.9, 0.99, 1e-6, 2)
+    assert np.array_equal(b.W_new, Wn) and np.array_equal(b.M_new, Mn) and np.array_equal(b.V_new, Vn)
