@@ -52,6 +52,7 @@ typedef enum {
   FF_ERR_UNSUPPORTED_ARCH = -8 /* the device is not compute capability 10.x                    */
 } ff_status;
 
+enum { FF_OPT_SGD = 0, FF_OPT_ADAM = 1 };  /* ff_layer_desc.optimizer */
 enum { FF_LINEAR = 0, FF_CONV3X3 = 1, FF_CONV1X1 = 2, FF_DWCONV3X3 = 3 };  /* ff_layer_desc.kind */
 enum { FF_ROUND_NEAREST_EVEN = 0, FF_ROUND_STOCHASTIC = 1 }; /* rounding modes (Sec. IV-B) */
 enum { FF_GEMM_AUTO = 0, FF_GEMM_SIMT = 1, FF_GEMM_TENSOR = 2 }; /* ff_set_gemm_path       */
@@ -86,6 +87,14 @@ typedef struct {
                         /* the output then has Ho = (H-1)/2 + 1 rows of Wo = (Wd-1)/2 + 1 positions */
   float momentum;       /* update rule: 0 = plain SGD (W -= lr*g); mu > 0 = heavy-ball SGD on the   */
                         /* buffer Mom: m = mu*m + g, W -= lr*m (the paper names no optimiser)       */
+  int32_t optimizer;    /* FF_OPT_SGD (the two forms above) or FF_OPT_ADAM: m = b1*m + (1-b1)*g,    */
+                        /* v = b2*v + (1-b2)*g*g, W -= lr*(m*c1)/(sqrt(v*c2) + adam_eps) with       */
+                        /* b1 = momentum, b2 = beta2, c_i = 1/(1 - b_i^t), t = step + 1; buffers   */
+                        /* Mom and Var; the weight-gradient sums pass through accW_dump if given,  */
+                        /* else through the workspace                                              */
+  float beta2;          /* Adam only, in [0, 1)                                                    */
+  float adam_eps;       /* Adam only, >= 0                                                         */
+  int32_t reserved;     /* zero                                                                    */
 } ff_layer_desc;
 
 /* Device buffers of one layer (host struct of device pointers; caller-owned). */
@@ -109,6 +118,8 @@ typedef struct {
   int32_t* acc_dump; /* [M*R,N] INT32 out, nullable: the forward accumulators                  */
   int32_t* accW_dump;/* [2,N,K] INT32 out, nullable: g^W accumulators of the two sets          */
   float* Mom;        /* [N,K] FP32 in/out momentum buffer; needed (and touched) only if momentum != 0 */
+                     /* or the optimiser is Adam (first moment)                                */
+  float* Var;        /* [N,K] FP32 in/out second-moment buffer; Adam only                      */
 } ff_layer_bufs;
 
 /* Create / destroy a context for CUDA device `device` (must be compute capability 10.x).

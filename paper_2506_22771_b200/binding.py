@@ -14,6 +14,7 @@ FF_ERR_ARG, FF_ERR_ALIGN, FF_ERR_WORKSPACE, FF_ERR_NONFINITE = -1, -2, -3, -4
 FF_ERR_RANGE, FF_ERR_DEVICE_TIMEOUT, FF_ERR_CUDA, FF_ERR_UNSUPPORTED_ARCH = -5, -6, -7, -8
 FF_LINEAR, FF_CONV3X3, FF_CONV1X1, FF_DWCONV3X3 = 0, 1, 2, 3
 FF_ROUND_NEAREST_EVEN, FF_ROUND_STOCHASTIC = 0, 1
+FF_OPT_SGD, FF_OPT_ADAM = 0, 1
 FF_GEMM_AUTO, FF_GEMM_SIMT, FF_GEMM_TENSOR = 0, 1, 2
 FF_A_X_POS, FF_A_X_NEG, FF_A_W, FF_A_DH_POS, FF_A_DH_NEG, FF_A_XNEXT_POS, FF_A_XNEXT_NEG = range(7)
 FF_ABSMAX_LEN = 8
@@ -34,13 +35,14 @@ class ff_layer_desc(C.Structure):
                 ("Wd", C.c_int32), ("Cin", C.c_int32), ("index", C.c_int32),
                 ("round_x", C.c_int32), ("round_w", C.c_int32), ("round_dh", C.c_int32),
                 ("theta", C.c_float), ("lr", C.c_float), ("tau", C.c_float), ("eps", C.c_float),
-                ("seed", C.c_uint64), ("stride", C.c_int32), ("momentum", C.c_float)]
+                ("seed", C.c_uint64), ("stride", C.c_int32), ("momentum", C.c_float),
+                ("optimizer", C.c_int32), ("beta2", C.c_float), ("adam_eps", C.c_float), ("reserved", C.c_int32)]
 
 
 class ff_layer_bufs(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
                 ("W", "X", "Y", "G", "Xnext", "Xq", "Wq", "dHq", "absmax", "S", "rowmax", "coef",
-                 "loss", "acc_dump", "accW_dump", "Mom")]
+                 "loss", "acc_dump", "accW_dump", "Mom", "Var")]
 
 
 FF_DP_MAX_REDUCE = 96
@@ -257,7 +259,8 @@ def make_desc(cfg, index: int, seed: int, round_x=FF_ROUND_STOCHASTIC, round_w=F
               round_dh=FF_ROUND_STOCHASTIC) -> ff_layer_desc:
     """cfg: an object with kind, K, N, H, Wd, Cin, theta, lr, tau, eps (e.g. synth.LayerCfg)."""
     return ff_layer_desc(cfg.kind, cfg.K, cfg.N, cfg.H, cfg.Wd, cfg.Cin, index, round_x, round_w, round_dh,
-                         cfg.theta, cfg.lr, cfg.tau, cfg.eps, seed, getattr(cfg, "stride", 1), getattr(cfg, "momentum", 0.0))
+                         cfg.theta, cfg.lr, cfg.tau, cfg.eps, seed, getattr(cfg, "stride", 1), getattr(cfg, "momentum", 0.0),
+                         getattr(cfg, "optimizer", 0), getattr(cfg, "beta2", 0.999), getattr(cfg, "adam_eps", 1e-8), 0)
 
 
 class LayerBuffers:
@@ -287,11 +290,12 @@ class LayerBuffers:
         self.loss = z((4,), torch.float32)
         self.acc_dump = z((rows, desc.N), torch.int32) if dumps else None
         self.accW_dump = z((2, desc.N, desc.K), torch.int32) if (dumps or accw) else None
-        self.Mom = z((desc.N, desc.K), torch.float32) if desc.momentum != 0.0 else None
+        self.Mom = z((desc.N, desc.K), torch.float32) if (desc.momentum != 0.0 or desc.optimizer == FF_OPT_ADAM) else None
+        self.Var = z((desc.N, desc.K), torch.float32) if desc.optimizer == FF_OPT_ADAM else None
         p = lambda t: t.data_ptr() if t is not None else None
         self.struct = ff_layer_bufs(p(self.W), p(self.X), p(self.Y), p(self.G), p(self.Xnext), p(self.Xq),
                                     p(self.Wq), p(self.dHq), p(self.absmax), p(self.S), p(self.rowmax),
-                                    p(self.coef), p(self.loss), p(self.acc_dump), p(self.accW_dump), p(self.Mom))
+                                    p(self.coef), p(self.loss), p(self.acc_dump), p(self.accW_dump), p(self.Mom), p(self.Var))
 
 
 class Context:

@@ -62,6 +62,53 @@ __device__ __forceinline__ RoundKey derive_key(KeySpec ks) {
   k.k1 = (uint32_t)(s2 >> 32);
   return k;
 }
+// How a dequantised weight gradient g becomes a weight change (Alg. 1 line 9 names no optimiser):
+// kind 0: plain SGD, or heavy ball when Mom is given (m = mu*m + g, W -= lr*m);
+// kind 1: Adam - m = b1*m + (1-b1)*g, v = b2*v + (1-b2)*g*g, W -= lr*(m*c1)/(sqrt(v*c2) + eps), with the
+// bias corrections c_i = float(1/(1 - b_i^t)), t = step + 1, from FP64 powers taken by square-and-multiply
+// from the low bit up (a fixed order of correctly rounded products).  Every FP32 operation is rounded once.
+struct UpdateRule {
+  int kind;
+  float lr, mu, beta2, eps;  // mu: heavy-ball coefficient or Adam's b1
+  float* Mom;
+  float* Var;
+  const StepState* ss;       // Adam reads the step counter here
+};
+__device__ __forceinline__ double pow_int_rn(double x, unsigned long long n) {
+  double r = 1.0, p = x;
+  while (n) {
+    if (n & 1ull) r = __dmul_rn(r, p);
+    n >>= 1;
+    if (n) p = __dmul_rn(p, p);
+  }
+  return r;
+}
+struct UpdateCoefs {
+  float c1, c2, omb1, omb2;
+};
+__device__ __forceinline__ UpdateCoefs update_coefs(const UpdateRule& r) {
+  UpdateCoefs c = {1.0f, 1.0f, 0.0f, 0.0f};
+  if (r.kind == 1) {
+    const unsigned long long t = r.ss->step + 1ull;
+    c.c1 = __double2float_rn(__ddiv_rn(1.0, __dsub_rn(1.0, pow_int_rn((double)r.mu, t))));
+    c.c2 = __double2float_rn(__ddiv_rn(1.0, __dsub_rn(1.0, pow_int_rn((double)r.beta2, t))));
+    c.omb1 = __fsub_rn(1.0f, r.mu);
+    c.omb2 = __fsub_rn(1.0f, r.beta2);
+  }
+  return c;
+}
+// New weight for gradient g; m / v are the element's buffer values, rewritten when the rule uses them.
+__device__ __forceinline__ float apply_update(const UpdateRule& r, const UpdateCoefs& c, float w, float g, float& m, float& v) {
+  if (r.kind == 1) {
+    m = __fadd_rn(__fmul_rn(r.mu, m), __fmul_rn(c.omb1, g));
+    v = __fadd_rn(__fmul_rn(r.beta2, v), __fmul_rn(c.omb2, __fmul_rn(g, g)));
+    const float upd = __fdiv_rn(__fmul_rn(m, c.c1), __fadd_rn(__fsqrt_rn(__fmul_rn(v, c.c2)), r.eps));
+    return __fsub_rn(w, __fmul_rn(r.lr, upd));
+  }
+  if (r.Mom) g = m = __fadd_rn(__fmul_rn(r.mu, m), g);
+  return __fsub_rn(w, __fmul_rn(r.lr, g));
+}
+
 __global__ void set_step_kernel(StepState* ss, unsigned long long step, float lambda, int set_lambda) {
   ss->step = step;
   if (set_lambda) ss->lambda = lambda;

@@ -142,6 +142,9 @@ ff_status check_layer(ff_ctx* ctx, const ff_layer_desc* L, int B) {
     if (r != FF_ROUND_NEAREST_EVEN && r != FF_ROUND_STOCHASTIC) return fail(ctx, FF_ERR_ARG, "unknown rounding mode");
   if (!(L->eps > 0.0f)) return fail(ctx, FF_ERR_ARG, "eps must be > 0");
   if (!(L->momentum >= 0.0f && L->momentum < 1.0f)) return fail(ctx, FF_ERR_ARG, "momentum must lie in [0, 1)");
+  if (L->optimizer != FF_OPT_SGD && L->optimizer != FF_OPT_ADAM) return fail(ctx, FF_ERR_ARG, "unknown optimizer");
+  if (L->optimizer == FF_OPT_ADAM && (!(L->beta2 >= 0.0f && L->beta2 < 1.0f) || !(L->adam_eps >= 0.0f)))
+    return fail(ctx, FF_ERR_ARG, "Adam needs beta2 in [0, 1) and adam_eps >= 0");
   const long long R = rows_per_sample(*L);
   const long long rows = 2LL * B * R;
   // 32-bit rounding counters and element indices
@@ -164,7 +167,7 @@ ff_status check_bufs(ff_ctx* ctx, const ff_layer_bufs* b, bool need_x) {
     if (!p) return fail(ctx, FF_ERR_ARG, "a required device pointer is NULL");
   if (need_x && !b->X) return fail(ctx, FF_ERR_ARG, "X is NULL");
   const void* all[] = {b->W, b->X, b->Y, b->G, b->Xnext, b->Xq, b->Wq, b->dHq, b->absmax, b->S, b->rowmax, b->coef,
-                       b->loss, b->acc_dump, b->accW_dump, b->Mom};
+                       b->loss, b->acc_dump, b->accW_dump, b->Mom, b->Var};
   for (const void* p : all)
     if (p && !aligned16(p)) return fail(ctx, FF_ERR_ALIGN, "a device pointer is not 16-byte aligned");
   return FF_OK;
@@ -260,16 +263,20 @@ ff_status launch_slab_update(ff_ctx* ctx, const int32_t* slabs, int splits, cons
   const size_t plane = (size_t)L.N * L.K;
   float* W = ctx->accumulate_only ? nullptr : b.W;
   int32_t* dump = b.accW_dump == slabs ? nullptr : b.accW_dump;  // the sums already are where they would be copied to
-  float* Mom = L.momentum != 0.0f ? b.Mom : nullptr;
+  UpdateRule rule;
+  rule.kind = L.optimizer == FF_OPT_ADAM ? 1 : 0;
+  rule.lr = L.lr, rule.mu = L.momentum, rule.beta2 = L.beta2, rule.eps = L.adam_eps;
+  rule.Mom = (rule.kind == 1 || L.momentum != 0.0f) ? b.Mom : nullptr;
+  rule.Var = rule.kind == 1 ? b.Var : nullptr;
+  rule.ss = step_ptr(ctx);
   if (!W && !dump) return FF_OK;
   if (splits <= 2 && (pitch == 0 || pitch == L.K) && (plane & 3) == 0 && plane >= ((size_t)1 << 18)) {
     const size_t want = (plane / 4 + 255) / 256, cap = (size_t)ctx->sm_count * 8;
-    slab_update_flat_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, W, b.absmax, L.lr, dump,
-                                                                                 Mom, L.momentum);
+    slab_update_flat_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, W, b.absmax, rule, dump);
   } else {
     const size_t want = (plane + 31) / 32, cap = (size_t)ctx->sm_count * 8;
     slab_update_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, L.K, pitch ? pitch : L.K, W,
-                                                                            b.absmax, L.lr, dump, Mom, L.momentum);
+                                                                            b.absmax, rule, dump);
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -437,8 +444,43 @@ ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
   return launch_simt<Im2colView, DenseView, false, 1>(ctx, im2col(b.Xq, L, 2 * B), dense(b.Wq, L.N, L.K), rows, L.N, L.K, epi, st);
 }
 
+ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st);
+
+inline size_t adam_plane_bytes(const ff_layer_desc& L) { return up256((size_t)2 * L.N * L.K * sizeof(int32_t)); }
+
+// Adam layers: the weight-gradient routes only accumulate (INT32 sums of both sets into one dense plane: the
+// caller's accW_dump if given, else the tail of the workspace, which the routes are kept out of meanwhile),
+// then the common update kernel applies the rule.  The fused update epilogues stay as they are.
+ff_status run_update_adam(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  if (!b.Mom || !b.Var) return fail(ctx, FF_ERR_ARG, "the Adam update needs the buffers Mom and Var");
+  if (ctx->accumulate_only) {  // data-parallel phase: sums go to accW_dump (checked by the caller), update comes later
+    ff_layer_desc plain = L;
+    plain.optimizer = FF_OPT_SGD;
+    return run_update_gemm(ctx, plain, b, B, st);
+  }
+  ff_layer_bufs b2 = b;
+  const size_t saved = ctx->workspace_bytes;
+  if (!b2.accW_dump) {
+    const size_t bytes = adam_plane_bytes(L);
+    if (saved < WS_BYTES + bytes) return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the Adam layer's weight-gradient sums");
+    const size_t off = (saved - bytes) / 256 * 256;
+    b2.accW_dump = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + off);
+    ctx->workspace_bytes = off;
+  }
+  ff_layer_desc plain = L;
+  plain.optimizer = FF_OPT_SGD;
+  ctx->accumulate_only = true;
+  ff_status s = run_update_gemm(ctx, plain, b2, B, st);
+  ctx->accumulate_only = false;
+  ctx->workspace_bytes = saved;
+  if (s != FF_OK) return s;
+  ProfScope prof(ctx, FF_K_UPD_GEMM, st);
+  return launch_slab_update(ctx, b2.accW_dump, 1, L, b2, st);
+}
+
 // Weight-gradient contraction + fused update.
 ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  if (L.optimizer == FF_OPT_ADAM) return run_update_adam(ctx, L, b, B, st);
   if (L.momentum != 0.0f && !b.Mom) return fail(ctx, FF_ERR_ARG, "momentum != 0 needs the buffer Mom");
   if (L.kind == FF_DWCONV3X3) return dw_update(ctx, L, b, B, st);
   const int R = rows_per_sample(L);
@@ -956,6 +998,7 @@ ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, s
       const size_t im_need = pl.slab_off - WS_BYTES + (size_t)pl.max_splits * pl.slab_bytes_per_split;
       if (im_need > need) need = im_need;
     }
+    if (layers[l].optimizer == FF_OPT_ADAM) need = up256(need) + adam_plane_bytes(layers[l]) + 256;  // sums plane at the tail
     if (need > slab) slab = need;
   }
   *out_bytes = WS_BYTES + (slab + 255) / 256 * 256;
@@ -1060,6 +1103,8 @@ ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_l
     if (l > 0 && bufs[l].X) return fail(ctx, FF_ERR_ARG, "a data-parallel step takes chained layers (X of layers > 0 NULL)");
     if (!bufs[l].accW_dump) return fail(ctx, FF_ERR_ARG, "a data-parallel step needs accW_dump of every layer");
     if (layers[l].momentum != 0.0f && !bufs[l].Mom) return fail(ctx, FF_ERR_ARG, "momentum != 0 needs the buffer Mom");
+    if (layers[l].optimizer == FF_OPT_ADAM && (!bufs[l].Mom || !bufs[l].Var))
+      return fail(ctx, FF_ERR_ARG, "the Adam update needs the buffers Mom and Var");
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;

@@ -197,8 +197,8 @@ struct SlabEpilogue {
 // [2][rows][cols]) - the buffer a data-parallel step adds up over the devices before it updates.
 __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane, int cols,
                                                           int pitch, float* __restrict__ W, const float* __restrict__ absmax,
-                                                          float lr, int32_t* __restrict__ accW_dump,
-                                                          float* __restrict__ Mom = nullptr, float mu = 0.0f) {
+                                                          UpdateRule rule, int32_t* __restrict__ accW_dump) {
+  const UpdateCoefs uc = update_coefs(rule);
   __shared__ int part[2][8][32];
   const int lane = threadIdx.x & 31, zl = threadIdx.x >> 5;
   const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
@@ -224,9 +224,11 @@ __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restr
         aN += part[1][k][lane];
       }
       if (W) {
-        float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
-        if (Mom) Mom[e] = g = __fadd_rn(__fmul_rn(mu, Mom[e]), g);
-        W[e] = __fsub_rn(W[e], __fmul_rn(lr, g));
+        const float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
+        float m = rule.Mom ? rule.Mom[e] : 0.0f, v = rule.Var ? rule.Var[e] : 0.0f;
+        W[e] = apply_update(rule, uc, W[e], g, m, v);
+        if (rule.Mom) rule.Mom[e] = m;
+        if (rule.Var) rule.Var[e] = v;
       }
       if (accW_dump) {
         accW_dump[e] = aP;
@@ -240,9 +242,9 @@ __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restr
 // The same for one or two slabs of a large output (dense rows, cols % 4 == 0): nothing to share between
 // warps, so every thread takes four consecutive elements with 128-bit accesses.
 __global__ void __launch_bounds__(256) slab_update_flat_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane,
-                                                               float* __restrict__ W, const float* __restrict__ absmax, float lr,
-                                                               int32_t* __restrict__ accW_dump, float* __restrict__ Mom = nullptr,
-                                                               float mu = 0.0f) {
+                                                               float* __restrict__ W, const float* __restrict__ absmax,
+                                                               UpdateRule rule, int32_t* __restrict__ accW_dump) {
+  const UpdateCoefs uc = update_coefs(rule);
   const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
   const float cN = __fmul_rn(scale_of(absmax[4]), scale_of(absmax[1]));
   const size_t n4 = plane >> 2, stride = (size_t)gridDim.x * blockDim.x;
@@ -262,18 +264,14 @@ __global__ void __launch_bounds__(256) slab_update_flat_kernel(const int32_t* __
       g.y = __fadd_rn(__fmul_rn(__int2float_rn(aP.y), cP), __fmul_rn(__int2float_rn(aN.y), cN));
       g.z = __fadd_rn(__fmul_rn(__int2float_rn(aP.z), cP), __fmul_rn(__int2float_rn(aN.z), cN));
       g.w = __fadd_rn(__fmul_rn(__int2float_rn(aP.w), cP), __fmul_rn(__int2float_rn(aN.w), cN));
-      if (Mom) {
-        const float4 m = reinterpret_cast<const float4*>(Mom)[i];
-        g.x = __fadd_rn(__fmul_rn(mu, m.x), g.x);
-        g.y = __fadd_rn(__fmul_rn(mu, m.y), g.y);
-        g.z = __fadd_rn(__fmul_rn(mu, m.z), g.z);
-        g.w = __fadd_rn(__fmul_rn(mu, m.w), g.w);
-        reinterpret_cast<float4*>(Mom)[i] = g;
-      }
-      w.x = __fsub_rn(w.x, __fmul_rn(lr, g.x));
-      w.y = __fsub_rn(w.y, __fmul_rn(lr, g.y));
-      w.z = __fsub_rn(w.z, __fmul_rn(lr, g.z));
-      w.w = __fsub_rn(w.w, __fmul_rn(lr, g.w));
+      float4 m = rule.Mom ? reinterpret_cast<const float4*>(rule.Mom)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 v = rule.Var ? reinterpret_cast<const float4*>(rule.Var)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+      w.x = apply_update(rule, uc, w.x, g.x, m.x, v.x);
+      w.y = apply_update(rule, uc, w.y, g.y, m.y, v.y);
+      w.z = apply_update(rule, uc, w.z, g.z, m.z, v.z);
+      w.w = apply_update(rule, uc, w.w, g.w, m.w, v.w);
+      if (rule.Mom) reinterpret_cast<float4*>(rule.Mom)[i] = m;
+      if (rule.Var) reinterpret_cast<float4*>(rule.Var)[i] = v;
       reinterpret_cast<float4*>(W)[i] = w;
     }
     if (accW_dump) {

@@ -29,7 +29,10 @@ class LayerCfg:
     Cin: int = 0
     eps: float = 1e-8
     stride: int = 1    # conv3x3 only
-    momentum: float = 0.0   # heavy-ball coefficient of the update (0: plain SGD)
+    momentum: float = 0.0   # heavy-ball coefficient of the update (0: plain SGD); Adam: beta1
+    optimizer: int = 0      # 0 SGD / heavy ball, 1 Adam
+    beta2: float = 0.999
+    adam_eps: float = 1e-8
 
 
 @dataclass

@@ -16,7 +16,8 @@ def specs_and_descs(layers, seed, round_x=1, round_w=0, round_dh=1):
     for i, l in enumerate(layers):
         specs.append(O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, l.eps, l.H, l.Wd, l.Cin,
                                  round_x, round_w, round_dh, seed, i, getattr(l, "stride", 1),
-                                 getattr(l, "momentum", 0.0)))
+                                 getattr(l, "momentum", 0.0), getattr(l, "optimizer", 0), getattr(l, "beta2", 0.999),
+                                 getattr(l, "adam_eps", 1e-8)))
         descs.append(ffb.make_desc(l, i, seed, round_x, round_w, round_dh))
     return specs, descs
 
@@ -90,6 +91,8 @@ def compare_layer(st: O.LayerState, b, spec, B, check_dumps=True, tag=""):
         eq("W_new", _np(b.W).reshape(-1), st.W_new.reshape(-1))
         if st.M_new is not None:
             eq("M_new", _np(b.Mom).reshape(-1), st.M_new.reshape(-1))
+        if st.V_new is not None:
+            eq("V_new", _np(b.Var).reshape(-1), st.V_new.reshape(-1))
 
 
 def _assert_equal(name, got, want):

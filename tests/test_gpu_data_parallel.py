@@ -51,7 +51,7 @@ def _run_dp(w, seed, steps, lam_per_step, world, path, rounding=(1, 0, 1)):
     n = len(descs)
     for sh in shards:
         sh.net.set_input(dp.shard_batch(np.ascontiguousarray(X).reshape(2 * w.B, -1), w.B, sh.off, sh.B))
-    Ms = None
+    Ms = Vs = None
     for step in range(steps):
         lam = lam_per_step * step
         for phase in range(ffb.ff_dp_phase_count(n)):
@@ -60,12 +60,13 @@ def _run_dp(w, seed, steps, lam_per_step, world, path, rounding=(1, 0, 1)):
             _combine(shards, entries)
         for sh in shards:
             ffb.ff_poll_status(sh.net.ctx.ctx, 0)
-        states = O.train_step(specs, Ws, X, w.B, lam, step, Ms)
+        states = O.train_step(specs, Ws, X, w.B, lam, step, Ms, Vs)
         for r, sh in enumerate(shards):
             for l, (st, b, sp) in enumerate(zip(states, sh.net.bufs, specs)):
                 compare_layer(shard_state(st, w.B, sh.off, sh.B), b, sp, sh.B, tag=f"step{step}/shard{r}/layer{l}/")
         Ws = [st.W_new for st in states]
         Ms = [st.M_new for st in states]
+        Vs = [st.V_new for st in states]
     for sh in shards:
         sh.net.close()
 
@@ -117,6 +118,13 @@ def test_dp_with_momentum():
     for l in w.layers:
         l.momentum = 0.9
     _run_dp(w, seed=14, steps=3, lam_per_step=0.5, world=3, path=(ffb.FF_GEMM_AUTO, 0))
+
+
+def test_dp_with_adam():
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=90, width_div=8)
+    for l in w.layers:
+        l.optimizer, l.momentum, l.beta2, l.adam_eps, l.lr = 1, 0.9, 0.99, 1e-6, 1e-3
+    _run_dp(w, seed=15, steps=3, lam_per_step=0.5, world=3, path=(ffb.FF_GEMM_AUTO, 0))
 
 
 def test_dp_single_shard_equals_train_step():

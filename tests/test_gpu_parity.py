@@ -66,16 +66,17 @@ def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), cha
     X = synth.make_batch(w, seed)
     net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path, graph=graph)
     net.set_input(X)
-    Ms = None
+    Ms = Vs = None
     for step in range(steps):
         lam = lam_per_step * step
         net.train_step(lam, step)
-        states = O.train_step(specs, Ws, X, w.B, lam, step, Ms)
+        states = O.train_step(specs, Ws, X, w.B, lam, step, Ms, Vs)
         if step % check_every == 0 or step == steps - 1:
             for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
                 compare_layer(st, b, sp, w.B, tag=f"step{step}/layer{l}/")
         Ws = [st.W_new for st in states]
         Ms = [st.M_new for st in states]
+        Vs = [st.V_new for st in states]
     net.close()
 
 
@@ -495,4 +496,53 @@ def test_momentum_wide_layer_and_argument_errors():
     net.descs_arr[0].momentum = 1.5
     with pytest.raises(ffb.FFError):
         net.train_step(0.0, 0)
+    net.close()
+
+
+# ---- Adam variant of the update: sums accumulate in a plane, one update kernel applies the rule ----------
+def _with_adam(w, lr, dumps_free_layer=None):
+    for l in w.layers:
+        l.optimizer, l.momentum, l.beta2, l.adam_eps, l.lr = 1, 0.9, 0.99, 1e-6, lr
+    return w
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_adam_dense_lookahead(path):
+    w = _with_adam(synth.scaled(synth.workload("mlp_lookahead"), B=136, width_div=8), 1e-3)
+    w.layers[2].optimizer, w.layers[2].momentum = 0, 0.5              # a heavy-ball layer among the Adam ones
+    _run_and_compare(w, seed=37, steps=4, lam_per_step=0.25, path=path)
+    _run_and_compare(w, seed=37, steps=5, lam_per_step=0.25, path=path, graph=True)   # bias corrections follow the replayed step
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_adam_convolutions(path):
+    w = _with_adam(synth.scaled(synth.workload("cnn"), B=2, width_div=4), 1e-3)         # im2col, dp4a / slab routes
+    _run_and_compare(w, seed=38, steps=3, lam_per_step=0.0, path=path)
+    layers = [synth.LayerCfg(1, 9 * 64, 128, float(128 * 256), 0.0, float(np.sqrt(128 * 256)), H=16, Wd=16, Cin=64),
+              synth.LayerCfg(3, 9, 128, float(128 * 256), 0.0, float(np.sqrt(128 * 256)), H=16, Wd=16, Cin=128),
+              synth.LayerCfg(2, 128, 64, float(64 * 256), 0.0, float(np.sqrt(64 * 256)), H=16, Wd=16, Cin=128)]
+    w = _with_adam(synth.Workload("conv_adam", 2, layers, (16, 16, 64), "normal", "kaiming_uniform", 2), 1e-3)
+    _run_and_compare(w, seed=39, steps=3, lam_per_step=0.5, path=path)
+
+
+def test_adam_without_dump_buffers_uses_the_workspace():
+    # no accW_dump: the sums plane sits at the tail of the workspace; wide first layer takes the 128-bit update kernel
+    w = _with_adam(synth.scaled(synth.workload("mlp_lookahead"), B=130, width_div=4), 1e-3)
+    w.layers = w.layers[:2]
+    specs, descs = specs_and_descs(w.layers, 20)
+    Ws = synth.make_weights(w, 20)
+    X = synth.make_batch(w, 20)
+    net = GpuNet(descs, w.B, Ws, dumps=False, xnext=False)
+    net.set_input(X)
+    Ms = Vs = None
+    for step in range(3):
+        net.train_step(0.0, step)
+        states = O.train_step(specs, Ws, X, w.B, 0.0, step, Ms, Vs)
+        Ws, Ms, Vs = [s.W_new for s in states], [s.M_new for s in states], [s.V_new for s in states]
+    for st, b in zip(states, net.bufs):
+        for name, got, want in [("W", b.W, st.W_new), ("M", b.Mom, st.M_new), ("V", b.Var, st.V_new)]:
+            assert np.array_equal(got.cpu().numpy().view(np.uint32), want.view(np.uint32)), name
+    net.bufs_arr[1].Var = None
+    with pytest.raises(ffb.FFError):
+        net.train_step(0.0, 3)
     net.close()
