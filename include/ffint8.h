@@ -230,7 +230,10 @@ ff_status ff_layer_loss_grad(ff_ctx* ctx, const ff_layer_desc* layer, const ff_l
 
 /* Weight gradient and update of one layer (Sec. IV-B: g^W as an INT8 MAC, "only gradients of
  * weights are computed and updated"; Alg. 1 line 9).  Reads dHq, Xq, absmax, W.  Writes W
- * (W - lr*(float(accP)*cP + float(accN)*cN)) and accW_dump (if non-NULL). */
+ * (W - lr*(float(accP)*cP + float(accN)*cN)) and accW_dump (if non-NULL); with momentum != 0 or
+ * optimizer = FF_OPT_ADAM the step follows that rule and Mom (and Var) are rewritten.  Adam's update
+ * number t is 1 + the step of the last call on this context that took one (ff_layer_forward,
+ * ff_layer_loss_grad, ff_train_step ...), so call ff_layer_loss_grad for the same step first. */
 ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs,
                           int B, void* cuda_stream);
 
