@@ -76,6 +76,7 @@ class LayerSpec:
     optimizer: int = 0    # 0 = SGD / heavy ball, 1 = Adam
     beta2: float = 0.999  # Adam only
     adam_eps: float = 1e-8
+    pool: int = 1         # 2: the normalised output is max-pooled 2x2 (stride 2) before it feeds the next layer
 
     @property
     def out_hw(self):
@@ -316,6 +317,21 @@ def length_normalise(y: np.ndarray, G: np.ndarray, tau: float, eps: float) -> np
     return y * r.reshape((-1,) + (1,) * (y.ndim - 1)).astype(F32)
 
 
+def maxpool2x2(x: np.ndarray) -> np.ndarray:
+    """2x2 max pooling with stride 2 over the two spatial axes of an NHWC tensor (odd trailing rows /
+    columns are dropped): the down-sampling step of the convolutional models the paper trains (Table II).
+    In FF it sits between a layer's normalised output and the next layer's input; nothing is differentiated
+    through it because no input gradient exists (Sec. IV-B).  A maximum involves no rounding."""
+    n, h, w, c = x.shape
+    ho, wo = h // 2, w // 2
+    out = np.empty((n, ho, wo, c), dtype=x.dtype)
+    for i in range(ho):
+        for j in range(wo):
+            out[:, i, j, :] = np.maximum(np.maximum(x[:, 2 * i, 2 * j, :], x[:, 2 * i, 2 * j + 1, :]),
+                                         np.maximum(x[:, 2 * i + 1, 2 * j, :], x[:, 2 * i + 1, 2 * j + 1, :]))
+    return out
+
+
 # --------------------------------------------------------------------------------------
 # FF loss, sigma and the look-ahead coefficient  (Eq. 1-4; Alg. 1 lines 8-9)
 # --------------------------------------------------------------------------------------
@@ -441,6 +457,10 @@ def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: i
     st.Y = dequant_relu(st.acc, c_rows)
     st.G, st.S, st.rowmax = goodness(st.acc, c_rows)
     st.Xnext = length_normalise(st.Y, st.G, spec.tau, spec.eps)
+    if spec.pool == 2:
+        if spec.kind == KIND_LINEAR or spec.out_hw[0] % 2 or spec.out_hw[1] % 2:
+            raise ValueError("pooling needs a spatial layer with even output extents")
+        st.Xnext = maxpool2x2(st.Xnext)
     return st
 
 

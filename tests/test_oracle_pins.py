@@ -873,3 +873,40 @@ def test_layer_update_with_adam_carries_both_buffers():
     b = O.train_step([spec], [a.W_new], X, w.B, 0.0, 1, Ms=[a.M_new], Vs=[a.V_new])[0]
     Wn, Mn, Vn = O.adam_update(a.W_new, a.M_new, a.V_new, b.dW, 0.001, 0.9, 0.99, 1e-6, 2)
     assert np.array_equal(b.W_new, Wn) and np.array_equal(b.M_new, Mn) and np.array_equal(b.V_new, Vn)
+
+
+# ---- 2x2 max pooling between layers ----------------------------------------------------------------------
+def test_maxpool2x2_hand_example_and_reshape_identity():
+    x = np.arange(2 * 4 * 4 * 1, dtype=np.float32).reshape(2, 4, 4, 1)
+    x[0, 1, 0, 0] = 99.0
+    got = O.maxpool2x2(x)
+    assert got.shape == (2, 2, 2, 1)
+    assert got[0, :, :, 0].tolist() == [[99.0, 7.0], [13.0, 15.0]] and got[1, :, :, 0].tolist() == [[21.0, 23.0], [29.0, 31.0]]
+    # against the reshape form of the same definition, with odd extents (the trailing row / column is dropped)
+    g = np.random.default_rng(41)
+    y = g.normal(size=(3, 7, 9, 5)).astype(np.float32)
+    want = y[:, :6, :8, :].reshape(3, 3, 2, 4, 2, 5).max(axis=(2, 4))
+    assert np.array_equal(O.maxpool2x2(y), want)
+    # pooling commutes with a positive per-sample factor (so it can be taken before or after the normalisation)
+    r = np.float32(0.37)
+    assert np.array_equal(O.maxpool2x2(y * r), O.maxpool2x2(y) * r)
+
+
+def test_pooled_layer_output_keeps_the_range_and_feeds_a_smaller_next_layer():
+    from paper_2506_22771_b200 import synth
+    H = Wd = 12
+    specs = [O.LayerSpec(O.KIND_CONV3X3, 27, 8, float(8 * H * Wd), 0.01, float(np.sqrt(8 * H * Wd)), H=H, Wd=Wd, Cin=3, seed=2,
+                         pool=2),
+             O.LayerSpec(O.KIND_CONV3X3, 72, 4, float(4 * 36), 0.01, float(np.sqrt(4 * 36)), H=H // 2, Wd=Wd // 2, Cin=8, seed=2,
+                         index=1)]
+    w = synth.Workload("p", 3, [synth.LayerCfg(1, 27, 8, 1.0, 0.01, 1.0, H=H, Wd=Wd, Cin=3),
+                                synth.LayerCfg(1, 72, 4, 1.0, 0.01, 1.0, H=H // 2, Wd=Wd // 2, Cin=8)], (H, Wd, 3), "normal",
+                       "kaiming_uniform", 1)
+    Ws = synth.make_weights(w, 2)
+    X = synth.make_batch(w, 2)
+    st = O.train_step(specs, Ws, X, w.B, 0.5, 0)
+    full = O.length_normalise(st[0].Y, st[0].G, specs[0].tau, specs[0].eps)
+    assert st[0].Xnext.shape == (6, 6, 6, 8) and np.array_equal(st[0].Xnext, O.maxpool2x2(full))
+    # the maximum survives max pooling (outputs are >= 0), so the next layer's quantiser range is the unpooled one
+    assert st[1].a_x == (O.absmax(full[:3]), O.absmax(full[3:]))
+    assert st[1].Y.shape == (6, 6, 6, 4) and st[1].W_new.shape == (4, 72)
