@@ -94,7 +94,10 @@ typedef struct {
                         /* else through the workspace                                              */
   float beta2;          /* Adam only, in [0, 1)                                                    */
   float adam_eps;       /* Adam only, >= 0                                                         */
-  int32_t reserved;     /* zero                                                                    */
+  int32_t pool;         /* 0 or 1: none; 2: the normalised output (Xnext and the next layer's input) */
+                        /* is max-pooled 2x2 with stride 2 over the positions, [M,Ho/2,Wo/2,N]      */
+                        /* (spatial layers with even Ho, Wo; goodness, loss and g^Y stay at full    */
+                        /* resolution - no gradient passes through the pooling, Sec. IV-B)          */
 } ff_layer_desc;
 
 /* Device buffers of one layer (host struct of device pointers; caller-owned). */
@@ -106,7 +109,7 @@ typedef struct {
                      /* the previous layer's normalised output without materialising it.      */
   float* Y;          /* [M*R,N] FP32 out: max(0, float(acc)*s_x*s_w)                           */
   float* G;          /* [M] FP32 out: goodness per sample                                      */
-  float* Xnext;      /* [M*R,N] FP32 out, nullable: Y*tau/(sqrt(G)+eps)                         */
+  float* Xnext;      /* [M*R,N] FP32 out, nullable: Y*tau/(sqrt(G)+eps); [M*R/4,N] with pool = 2 */
   int8_t* Xq;        /* [M*Rin,Kin] INT8 out                                                   */
   int8_t* Wq;        /* [N,K] INT8 out                                                         */
   int8_t* dHq;       /* [M*R,N] INT8 out (ff_layer_loss_grad)                                  */

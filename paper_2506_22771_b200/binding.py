@@ -36,7 +36,7 @@ class ff_layer_desc(C.Structure):
                 ("round_x", C.c_int32), ("round_w", C.c_int32), ("round_dh", C.c_int32),
                 ("theta", C.c_float), ("lr", C.c_float), ("tau", C.c_float), ("eps", C.c_float),
                 ("seed", C.c_uint64), ("stride", C.c_int32), ("momentum", C.c_float),
-                ("optimizer", C.c_int32), ("beta2", C.c_float), ("adam_eps", C.c_float), ("reserved", C.c_int32)]
+                ("optimizer", C.c_int32), ("beta2", C.c_float), ("adam_eps", C.c_float), ("pool", C.c_int32)]
 
 
 class ff_layer_bufs(C.Structure):
@@ -260,7 +260,8 @@ def make_desc(cfg, index: int, seed: int, round_x=FF_ROUND_STOCHASTIC, round_w=F
     """cfg: an object with kind, K, N, H, Wd, Cin, theta, lr, tau, eps (e.g. synth.LayerCfg)."""
     return ff_layer_desc(cfg.kind, cfg.K, cfg.N, cfg.H, cfg.Wd, cfg.Cin, index, round_x, round_w, round_dh,
                          cfg.theta, cfg.lr, cfg.tau, cfg.eps, seed, getattr(cfg, "stride", 1), getattr(cfg, "momentum", 0.0),
-                         getattr(cfg, "optimizer", 0), getattr(cfg, "beta2", 0.999), getattr(cfg, "adam_eps", 1e-8), 0)
+                         getattr(cfg, "optimizer", 0), getattr(cfg, "beta2", 0.999), getattr(cfg, "adam_eps", 1e-8),
+                         getattr(cfg, "pool", 1))
 
 
 class LayerBuffers:
@@ -279,7 +280,7 @@ class LayerBuffers:
         self.X = z((rows_in, kin), torch.float32) if own_x else None
         self.Y = z((rows, desc.N), torch.float32)
         self.G = z((2 * B,), torch.float32)
-        self.Xnext = z((rows, desc.N), torch.float32) if xnext else None
+        self.Xnext = z((rows // 4 if desc.pool == 2 else rows, desc.N), torch.float32) if xnext else None
         self.Xq = z((rows_in, kin), torch.int8)
         self.Wq = z((desc.N, desc.K), torch.int8)
         self.dHq = z((rows, desc.N), torch.int8)

@@ -209,6 +209,55 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
 }
 
 // ---------------------------------------------------------------------------------------------
+// The same with 2x2 max pooling (stride 2) over the positions of a spatial layer before the scaling:
+// out[m, i, j, c] = max of Y[m, 2i..2i+1, 2j..2j+1, c] * tau/(sqrt(G[m])+eps)  (the maximum commutes with the
+// positive factor and needs no rounding).  Y [2B, Ho, Wo, N] -> xnext / xq [2B, Ho/2, Wo/2, N]; the rounding
+// counters are the element indices of the pooled tensor.  One thread per pooled value (V = 1) or per four
+// channels (V = 4, N % 4 == 0).   grid = (blocks, 2)
+// ---------------------------------------------------------------------------------------------
+template <int MODE, int V>
+__global__ void __launch_bounds__(EW_THREADS) normalize_pool_kernel(const float* __restrict__ Y, const float* __restrict__ G,
+                                                                    float tau, float eps, int B, int Ho, int Wo, int N,
+                                                                    float* __restrict__ xnext, int8_t* __restrict__ xq,
+                                                                    const float* __restrict__ a, KeySpec ks,
+                                                                    uint2 ctr_bias = uint2{0u, 0u}) {
+  const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
+  const uint32_t bias = blockIdx.y ? ctr_bias.y : ctr_bias.x;
+  const float inv = xq ? inv_of(a[blockIdx.y]) : 0.0f;
+  const uint32_t Hp = Ho >> 1, Wp = Wo >> 1, NG = N / V;
+  const uint32_t per_pass = (uint32_t)B * Hp * Wp * NG;          // work items of this pass
+  const size_t row = (size_t)N, line = (size_t)Wo * N;
+  for (uint32_t it = blockIdx.x * blockDim.x + threadIdx.x; it < per_pass; it += gridDim.x * blockDim.x) {
+    const uint32_t pos = it / NG, cg = it - pos * NG;
+    const uint32_t j = pos % Wp, t = pos / Wp, i = t % Hp, m = t / Hp + blockIdx.y * B;
+    const float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(__ldg(G + m)), eps));
+    const float* src = Y + (((size_t)m * Ho + 2 * i) * Wo + 2 * j) * N + (size_t)V * cg;
+    const size_t e = ((size_t)blockIdx.y * per_pass + it) * V;   // element index in the pooled tensor
+    if (V == 4) {
+      const float4 p00 = __ldg(reinterpret_cast<const float4*>(src)), p01 = __ldg(reinterpret_cast<const float4*>(src + row));
+      const float4 p10 = __ldg(reinterpret_cast<const float4*>(src + line));
+      const float4 p11 = __ldg(reinterpret_cast<const float4*>(src + line + row));
+      float4 v;
+      v.x = __fmul_rn(fmaxf(fmaxf(p00.x, p01.x), fmaxf(p10.x, p11.x)), r);
+      v.y = __fmul_rn(fmaxf(fmaxf(p00.y, p01.y), fmaxf(p10.y, p11.y)), r);
+      v.z = __fmul_rn(fmaxf(fmaxf(p00.z, p01.z), fmaxf(p10.z, p11.z)), r);
+      v.w = __fmul_rn(fmaxf(fmaxf(p00.w, p01.w), fmaxf(p10.w, p11.w)), r);
+      if (xnext) *reinterpret_cast<float4*>(xnext + e) = v;
+      if (xq) {
+        int q0, q1, q2, q3;
+        quant_pair<MODE>(v.x, v.y, inv, (uint32_t)e + bias, key, q0, q1);
+        quant_pair<MODE>(v.z, v.w, inv, (uint32_t)e + bias + 2, key, q2, q3);
+        *reinterpret_cast<uint32_t*>(xq + e) = pack4(q0, q1, q2, q3);
+      }
+    } else {
+      const float v = __fmul_rn(fmaxf(fmaxf(__ldg(src), __ldg(src + row)), fmaxf(__ldg(src + line), __ldg(src + line + row))), r);
+      if (xnext) xnext[e] = v;
+      if (xq) xq[e] = (int8_t)quant_one<MODE>(v, inv, (uint32_t)e + bias, key);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // e^v for v <= 0 in FP64 by a fixed recipe so that every implementation agrees bit for bit:
 // clamp at -700, n = rint(v*log2e), r = (v - n*LN2_HI) - n*LN2_LO, degree-13 Taylor polynomial by
 // Horner with separately rounded multiply and add, exact scaling by 2^n.

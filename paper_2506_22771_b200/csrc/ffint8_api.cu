@@ -121,6 +121,10 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 // output rows (positions) per sample, and input rows per sample (they differ for a strided convolution)
 inline int rows_per_sample(const ff_layer_desc& L) { return L.kind != FF_LINEAR ? tc_out_h(L) * tc_out_w(L) : 1; }
+// values per sample of what the layer hands to the next one (a quarter of the positions with 2x2 pooling)
+inline long long next_values_per_sample(const ff_layer_desc& L) {
+  return (long long)rows_per_sample(L) / (L.pool == 2 ? 4 : 1) * L.N;
+}
 inline int in_rows_per_sample(const ff_layer_desc& L) { return L.kind != FF_LINEAR ? L.H * L.Wd : 1; }
 inline int in_features(const ff_layer_desc& L) { return (L.kind == FF_CONV3X3 || L.kind == FF_DWCONV3X3) ? L.Cin : L.K; }
 
@@ -142,6 +146,9 @@ ff_status check_layer(ff_ctx* ctx, const ff_layer_desc* L, int B) {
     if (r != FF_ROUND_NEAREST_EVEN && r != FF_ROUND_STOCHASTIC) return fail(ctx, FF_ERR_ARG, "unknown rounding mode");
   if (!(L->eps > 0.0f)) return fail(ctx, FF_ERR_ARG, "eps must be > 0");
   if (!(L->momentum >= 0.0f && L->momentum < 1.0f)) return fail(ctx, FF_ERR_ARG, "momentum must lie in [0, 1)");
+  if (L->pool < 0 || L->pool > 2) return fail(ctx, FF_ERR_ARG, "pool must be 0, 1 or 2");
+  if (L->pool == 2 && (L->kind == FF_LINEAR || tc_out_h(*L) % 2 || tc_out_w(*L) % 2))
+    return fail(ctx, FF_ERR_ARG, "pooling needs a spatial layer with even output extents");
   if (L->optimizer != FF_OPT_SGD && L->optimizer != FF_OPT_ADAM) return fail(ctx, FF_ERR_ARG, "unknown optimizer");
   if (L->optimizer == FF_OPT_ADAM && (!(L->beta2 >= 0.0f && L->beta2 < 1.0f) || !(L->adam_eps >= 0.0f)))
     return fail(ctx, FF_ERR_ARG, "Adam needs beta2 in [0, 1) and adam_eps >= 0");
@@ -664,6 +671,29 @@ ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
   const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
   const size_t per_pass = per_sample * B;
   const KeySpec key = next ? make_key_spec(next->seed, ROLE_X, next->index, step_ptr(ctx)) : KeySpec{0ull, step_ptr(ctx)};
+  if (L.pool == 2) {
+    ProfScope prof(ctx, FF_K_NORMALIZE, st);
+    const bool stoch = next && next->round_x != FF_ROUND_NEAREST_EVEN;
+    const bool vec = L.N % 4 == 0;
+    const int Ho = tc_out_h(L), Wo = tc_out_w(L);
+    const dim3 grid(ew_blocks(ctx, per_pass / 4 / (vec ? 4 : 1) + 1, 1), 2);
+    const uint2 bias = ctr_bias(ctx, per_sample / 4, B);
+    const float* a = b.absmax + FF_A_XNEXT_POS;
+    if (vec && stoch)
+      normalize_pool_kernel<ROUND_STOCHASTIC, 4><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, B, Ho, Wo, L.N, b.Xnext,
+                                                                             xq_next, a, key, bias);
+    else if (vec)
+      normalize_pool_kernel<ROUND_NEAREST, 4><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, B, Ho, Wo, L.N, b.Xnext, xq_next,
+                                                                          a, key, bias);
+    else if (stoch)
+      normalize_pool_kernel<ROUND_STOCHASTIC, 1><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, B, Ho, Wo, L.N, b.Xnext,
+                                                                             xq_next, a, key, bias);
+    else
+      normalize_pool_kernel<ROUND_NEAREST, 1><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, B, Ho, Wo, L.N, b.Xnext, xq_next,
+                                                                          a, key, bias);
+    FF_LAUNCH_CHECK(ctx);
+    return FF_OK;
+  }
   {
     ProfScope prof(ctx, FF_K_NORMALIZE, st);
     const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
@@ -724,7 +754,7 @@ ff_status check_layer_list(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
     if ((s = check_bufs(ctx, &bufs[l], l == 0)) != FF_OK) return s;
     if (l > 0 && !bufs[l].X) {
       const ff_layer_desc &p = layers[l - 1], &c = layers[l];
-      if ((long long)rows_per_sample(p) * p.N != (long long)in_rows_per_sample(c) * in_features(c))
+      if (next_values_per_sample(p) != (long long)in_rows_per_sample(c) * in_features(c))
         return fail(ctx, FF_ERR_ARG, "layer output / next layer input sizes differ");
     }
   }

@@ -33,6 +33,7 @@ class LayerCfg:
     optimizer: int = 0      # 0 SGD / heavy ball, 1 Adam
     beta2: float = 0.999
     adam_eps: float = 1e-8
+    pool: int = 1           # 2: 2x2 max pooling of the normalised output before the next layer
 
 
 @dataclass

@@ -17,7 +17,7 @@ def specs_and_descs(layers, seed, round_x=1, round_w=0, round_dh=1):
         specs.append(O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, l.eps, l.H, l.Wd, l.Cin,
                                  round_x, round_w, round_dh, seed, i, getattr(l, "stride", 1),
                                  getattr(l, "momentum", 0.0), getattr(l, "optimizer", 0), getattr(l, "beta2", 0.999),
-                                 getattr(l, "adam_eps", 1e-8)))
+                                 getattr(l, "adam_eps", 1e-8), getattr(l, "pool", 1)))
         descs.append(ffb.make_desc(l, i, seed, round_x, round_w, round_dh))
     return specs, descs
 
