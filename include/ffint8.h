@@ -200,9 +200,9 @@ ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_l
                             int B_total, int row_offset, int phase, float lambda, uint64_t step, void* cuda_stream,
                             ff_dp_reduce* reduce, int* n_reduce);
 
-/* Launch-sequence replay for ff_train_step (the paper's edge setting, batch 32 in Sec. V, makes a step a
+/* Launch-sequence replay for ff_train_step and ff_predict (the paper's edge setting, batch 32 in Sec. V, makes a step a
  * chain of short kernels whose cost is launch overhead; it states no counterpart of this switch).
- * on = 1: the first ff_train_step call of a call shape runs its kernels one by one, the second is
+ * on = 1: the first ff_train_step (or ff_predict) call of a call shape runs its kernels one by one, the second is
  * captured into a CUDA graph, and every later one is a single graph launch; the step counter and
  * lambda are read from device memory, so they may change from call to call.  A call shape is the byte
  * content of the layer and buffer arrays (zero any padding), n_layers, B, the workspace and the
@@ -212,7 +212,7 @@ ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_l
  * is already being captured by the caller.  on = 0 (default) drops the graphs.  Host state only: no
  * device memory is allocated by the library beyond what graph instantiation itself takes. */
 ff_status ff_set_graph_mode(ff_ctx* ctx, int on);
-/* ff_train_step calls served by a graph launch so far (0 while the mode is off).  A call shape whose
+/* ff_train_step / ff_predict calls served by a graph launch so far (0 while the mode is off).  A call shape whose
  * capture fails keeps running kernel by kernel and says why through ff_last_error. */
 uint64_t ff_graph_replay_count(const ff_ctx* ctx);
 

@@ -890,12 +890,13 @@ void graph_gave_up(ff_ctx* ctx, ff_ctx::GraphEntry* ent, const char* what, cudaE
 // same call shape.  First call of a shape: eager (it also fills the per-kernel attribute and occupancy
 // caches, which must not happen inside a capture).  Second call: captured, instantiated and launched.
 // Later calls: one graph launch.  A shape whose capture fails stays on the eager path.
-ff_status train_step_graph(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
-                           float lambda, cudaStream_t st) {
+template <class Body>
+ff_status run_replayed(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
+                       const void* extra, size_t extra_bytes, cudaStream_t st, Body run_body) {
   cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
     cudaGetLastError();
-    return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);  // the caller is capturing already
+    return run_body(st);  // the caller is capturing already
   }
   std::vector<unsigned char> key;
   auto put = [&key](const void* p, size_t n) {
@@ -908,6 +909,7 @@ ff_status train_step_graph(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
   put(&ctx->workspace_bytes, sizeof(size_t));
   put(layers, sizeof(ff_layer_desc) * n_layers);
   put(bufs, sizeof(ff_layer_bufs) * n_layers);
+  put(extra, extra_bytes);   // which entry point, and its further arguments that shape the launches
 
   ff_ctx::GraphEntry* ent = nullptr;
   for (auto& g : ctx->graphs)
@@ -923,25 +925,25 @@ ff_status train_step_graph(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
     ctx->graphs.emplace_back();
     ctx->graphs.back().key = std::move(key);
     ctx->graphs.back().last_use = ++ctx->graph_clock;
-    return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+    return run_body(st);
   }
   ent->last_use = ++ctx->graph_clock;
-  if (ent->eager_only) return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+  if (ent->eager_only) return run_body(st);
   if (!ent->exec) {
     cudaError_t e;
     if (!ctx->capture_stream &&
         (e = cudaStreamCreateWithFlags(&ctx->capture_stream, cudaStreamNonBlocking)) != cudaSuccess) {
       ctx->capture_stream = nullptr;
       graph_gave_up(ctx, ent, "no capture stream", e);
-      return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+      return run_body(st);
     }
     const uint64_t before = ctx->launches;
     if ((e = cudaStreamBeginCapture(ctx->capture_stream, cudaStreamCaptureModeThreadLocal)) != cudaSuccess) {
       graph_gave_up(ctx, ent, "capture did not start", e);
-      return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+      return run_body(st);
     }
     // nothing runs while capturing: the launches are recorded on the library's own stream and replayed on the caller's
-    const ff_status body = train_step_body(ctx, layers, bufs, n_layers, B, lambda, ctx->capture_stream);
+    const ff_status body = run_body(ctx->capture_stream);
     cudaGraph_t graph = nullptr;
     e = cudaStreamEndCapture(ctx->capture_stream, &graph);
     const uint64_t captured = ctx->launches - before;
@@ -956,7 +958,7 @@ ff_status train_step_graph(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
     }
     if (e != cudaSuccess || !exec) {
       graph_gave_up(ctx, ent, "capture or instantiation failed", e);
-      return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+      return run_body(st);
     }
     ent->exec = exec;
     ent->launches = captured;
@@ -965,6 +967,14 @@ ff_status train_step_graph(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
   ctx->launches += ent->launches;
   ctx->graph_replays++;
   return FF_OK;
+}
+
+ff_status train_step_graph(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
+                           float lambda, cudaStream_t st) {
+  const int tag = 1;
+  return run_replayed(ctx, layers, bufs, n_layers, B, &tag, sizeof(tag), st, [&](cudaStream_t s) {
+    return train_step_body(ctx, layers, bufs, n_layers, B, lambda, s);
+  });
 }
 
 }  // namespace
@@ -1171,19 +1181,33 @@ ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bu
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
   if ((s = set_step(ctx, step, 0.0f, false, st)) != FF_OK) return s;
-  if ((s = forward_all(ctx, layers, bufs, n_layers, half, st)) != FF_OK) return s;
-  LaterLayers gs;
-  gs.n = n_layers - first_counted_layer;
-  for (int j = 0; j < gs.n; ++j) {
-    gs.G[j] = bufs[first_counted_layer + j].G;
-    gs.theta[j] = 0.0f;
+  auto body = [&](cudaStream_t sb) -> ff_status {
+    ff_status r = forward_all(ctx, layers, bufs, n_layers, half, sb);
+    if (r != FF_OK) return r;
+    LaterLayers gs;
+    gs.n = n_layers - first_counted_layer;
+    for (int j = 0; j < gs.n; ++j) {
+      gs.G[j] = bufs[first_counted_layer + j].G;
+      gs.theta[j] = 0.0f;
+    }
+    {
+      ProfScope prof(ctx, FF_K_CLASSIFY, sb);
+      classify_kernel<<<(B + EW_THREADS - 1) / EW_THREADS, EW_THREADS, 0, sb>>>(gs, B, n_classes, scores, pred);
+    }
+    FF_LAUNCH_CHECK(ctx);
+    return FF_OK;
+  };
+  if (ctx->graph_mode && !ctx->profiling) {
+    struct PredictKey {
+      int tag, n_classes, first;
+      float* scores;
+      int32_t* pred;
+    } extra;
+    memset(&extra, 0, sizeof(extra));  // padding bytes are part of the key
+    extra.tag = 2, extra.n_classes = n_classes, extra.first = first_counted_layer, extra.scores = scores, extra.pred = pred;
+    return run_replayed(ctx, layers, bufs, n_layers, half, &extra, sizeof(extra), st, body);
   }
-  {
-    ProfScope prof(ctx, FF_K_CLASSIFY, st);
-    classify_kernel<<<(B + EW_THREADS - 1) / EW_THREADS, EW_THREADS, 0, st>>>(gs, B, n_classes, scores, pred);
-  }
-  FF_LAUNCH_CHECK(ctx);
-  return FF_OK;
+  return body(st);
 }
 
 ff_status ff_embed_labels(ff_ctx* ctx, const float* x, const int32_t* labels, int B, int n, int sets, int n_classes,

@@ -546,3 +546,31 @@ def test_adam_without_dump_buffers_uses_the_workspace():
     with pytest.raises(ffb.FFError):
         net.train_step(0.0, 3)
     net.close()
+
+
+def test_predict_with_replayed_launches():
+    # steps 2.. of a repeated classification call are graph launches; the rounding of the candidates follows the step
+    import torch
+    n_classes, B = 10, 20
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=n_classes * B // 2, width_div=8)
+    w.layers = w.layers[:2]
+    specs, descs = specs_and_descs(w.layers, 7)
+    Ws = synth.make_weights(w, 7)
+    Xc, _ = synth.make_candidates(w, 7, B, n_classes)
+    net = GpuNet(descs, n_classes * B // 2, Ws, dumps=False, xnext=False, chain=True, graph=True)
+    net.set_input(Xc)
+    scores = torch.zeros(n_classes * B, dtype=torch.float32, device="cuda")
+    pred = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    for step in range(5):
+        ffb.ff_predict(net.ctx.ctx, net.descs_arr, net.bufs_arr, len(descs), B, n_classes, 0, scores.data_ptr(), pred.data_ptr(),
+                       step, 0)
+        ffb.ff_poll_status(net.ctx.ctx, 0)
+        want_pred, want_scores, _ = O.predict(specs, Ws, Xc, B, n_classes, step, 0)
+        assert np.array_equal(scores.cpu().numpy().view(np.uint32), want_scores.reshape(-1).view(np.uint32)), step
+        assert np.array_equal(pred.cpu().numpy(), want_pred), step
+    assert ffb.ff_graph_replay_count(net.ctx.ctx) == 4, ffb.ff_last_error(net.ctx.ctx)
+    # a train step on the same buffers is a different call shape with a graph of its own
+    for step in range(3):
+        net.train_step(0.0, step)
+    assert ffb.ff_graph_replay_count(net.ctx.ctx) == 6
+    net.close()
