@@ -10,6 +10,7 @@
 namespace ffi8 {
 
 constexpr int EW_THREADS = 256;
+constexpr int FF_MAX_LATER = 31;  // layers after the first in one call
 
 __device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) { return __reduce_max_sync(0xffffffffu, v); }
 
@@ -32,9 +33,27 @@ __device__ __forceinline__ uint32_t block_max_u32(uint32_t v) {
 // |x| compared as bit patterns (monotone for finite floats); Inf/NaN raise ST_NONFINITE.
 // grid = (blocks, passes)
 // ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void absmax_body(const float* __restrict__ xp, size_t n_per_pass, uint32_t* __restrict__ out,
+                                            uint32_t* __restrict__ status);
 __global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restrict__ x, size_t n_per_pass,
                                                             float* __restrict__ out, uint32_t* __restrict__ status) {
-  const float* xp = x + (size_t)blockIdx.y * n_per_pass;
+  absmax_body(x + (size_t)blockIdx.y * n_per_pass, n_per_pass, reinterpret_cast<uint32_t*>(out) + blockIdx.y, status);
+}
+// The same over a table of tensors in one launch (blockIdx.y = tensor): the weights of every layer and the two
+// sets of the network input are all known when a step starts.  A step of small layers is a chain of short
+// launches, so fewer launches is what counts there.
+constexpr int MT_MAX = FF_MAX_LATER + 1 + 2;
+struct AbsmaxJobs {
+  const float* x[MT_MAX];
+  unsigned long long n[MT_MAX];
+  float* out[MT_MAX];
+};
+__global__ void __launch_bounds__(EW_THREADS) absmax_multi_kernel(AbsmaxJobs jobs, uint32_t* __restrict__ status) {
+  const int t = blockIdx.y;
+  absmax_body(jobs.x[t], (size_t)jobs.n[t], reinterpret_cast<uint32_t*>(jobs.out[t]), status);
+}
+__device__ __forceinline__ void absmax_body(const float* __restrict__ xp, size_t n_per_pass, uint32_t* __restrict__ out,
+                                            uint32_t* __restrict__ status) {
   uint32_t m = 0;
   const bool vec = ((n_per_pass & 3) == 0) && ((((uintptr_t)xp) & 15) == 0);
   size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -53,7 +72,7 @@ __global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restr
   m = block_max_u32(m);
   if (threadIdx.x == 0) {
     if (m >= 0x7f800000u) atomicOr(status, ST_NONFINITE);
-    if (m) atomicMax(reinterpret_cast<uint32_t*>(out) + blockIdx.y, m);
+    if (m) atomicMax(out, m);
   }
 }
 
@@ -66,6 +85,32 @@ __global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restr
 // ---------------------------------------------------------------------------------------------
 // zero_S / zero_rowmax (nullable, zero_n entries): per-sample accumulators of the forward epilogue that
 // the weight quantiser clears on the side, sparing a launch.
+// q[i] = quantised x[i] for one tensor of n elements; ctr0 = rounding counter of element 0 (an odd one would
+// split the element pairs that share one hash differently from the unsplit tensor: scalar path then).
+template <int MODE>
+__device__ __forceinline__ void quantize_body(const float* __restrict__ xp, int8_t* __restrict__ qp, size_t n, float inv,
+                                              uint32_t ctr0, RoundKey key) {
+  const bool vec = ((n & 3) == 0) && ((((uintptr_t)xp) & 15) == 0) && ((((uintptr_t)qp) & 3) == 0) && !(ctr0 & 1u);
+  size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  size_t stride = (size_t)gridDim.x * blockDim.x;
+  if (vec) {
+    const float4* x4 = reinterpret_cast<const float4*>(xp);
+    uint32_t* q4 = reinterpret_cast<uint32_t*>(qp);
+    size_t n4 = n >> 2;
+#pragma unroll 4
+    for (size_t i = tid; i < n4; i += stride) {
+      float4 v = __ldg(x4 + i);
+      uint32_t idx = ctr0 + (uint32_t)(i << 2);
+      int q0, q1, q2, q3;
+      quant_pair<MODE>(v.x, v.y, inv, idx, key, q0, q1);
+      quant_pair<MODE>(v.z, v.w, inv, idx + 2, key, q2, q3);
+      q4[i] = pack4(q0, q1, q2, q3);
+    }
+  } else {
+    for (size_t i = tid; i < n; i += stride) qp[i] = (int8_t)quant_one<MODE>(xp[i], inv, ctr0 + (uint32_t)i, key);
+  }
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __restrict__ x, int8_t* __restrict__ q,
                                                               size_t n_per_pass, const float* __restrict__ a,
@@ -80,30 +125,48 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __res
       zero_rowmax[i] = 0;
     }
   const size_t base = (size_t)blockIdx.y * n_per_pass;
-  const float* xp = x + base;
-  int8_t* qp = q + base;
-  const float inv = inv_of(a[blockIdx.y]);
-  // (an odd bias would split the element pairs that share one hash differently from the unsplit tensor)
-  const bool vec = ((n_per_pass & 3) == 0) && ((((uintptr_t)xp) & 15) == 0) && ((((uintptr_t)qp) & 3) == 0) && !(bias & 1u);
-  size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  size_t stride = (size_t)gridDim.x * blockDim.x;
-  if (vec) {
-    const float4* x4 = reinterpret_cast<const float4*>(xp);
-    uint32_t* q4 = reinterpret_cast<uint32_t*>(qp);
-    size_t n4 = n_per_pass >> 2;
-#pragma unroll 4
-    for (size_t i = tid; i < n4; i += stride) {
-      float4 v = __ldg(x4 + i);
-      uint32_t idx = (uint32_t)(base + (i << 2)) + bias;
-      int q0, q1, q2, q3;
-      quant_pair<MODE>(v.x, v.y, inv, idx, key, q0, q1);
-      quant_pair<MODE>(v.z, v.w, inv, idx + 2, key, q2, q3);
-      q4[i] = pack4(q0, q1, q2, q3);
+  quantize_body<MODE>(x + base, q + base, n_per_pass, inv_of(a[blockIdx.y]), (uint32_t)base + bias, key);
+}
+
+// Clears the range vectors (FF_ABSMAX_LEN floats each) of up to FF_MAX_LATER + 1 layers.  <<<1, 256>>>
+struct ZeroJobs {
+  float* p[FF_MAX_LATER + 1];
+  int n;
+};
+__global__ void zero_ranges_kernel(ZeroJobs z) {
+  const int i = threadIdx.x;
+  if (i < z.n * FF_ABSMAX_LEN) z.p[i / FF_ABSMAX_LEN][i % FF_ABSMAX_LEN] = 0.0f;
+}
+
+// One launch for a table of tensors (blockIdx.y = tensor): the weights of every layer and the two sets of
+// the network input, each with its own range, rounding mode, key and first counter.  Also clears the
+// per-sample accumulators of every layer's forward epilogue.
+struct QuantJobs {
+  const float* x[MT_MAX];
+  int8_t* q[MT_MAX];
+  unsigned long long n[MT_MAX];
+  const float* a[MT_MAX];          // address of the tensor's range
+  unsigned long long s1[MT_MAX];   // step-independent part of the rounding key
+  uint32_t ctr0[MT_MAX];           // counter of the tensor's first element
+  uint8_t stochastic[MT_MAX];
+  unsigned long long* zero_S[FF_MAX_LATER + 1];
+  int32_t* zero_rowmax[FF_MAX_LATER + 1];
+  int n_zero, zero_n;              // layers whose accumulators are cleared, entries each
+  const StepState* ss;
+};
+__global__ void __launch_bounds__(EW_THREADS) quantize_multi_kernel(const QuantJobs jobs) {
+  const int t = blockIdx.y;
+  if (t < jobs.n_zero)
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < jobs.zero_n; i += gridDim.x * blockDim.x) {
+      jobs.zero_S[t][i] = 0ull;
+      jobs.zero_rowmax[t][i] = 0;
     }
-  } else {
-    for (size_t i = tid; i < n_per_pass; i += stride)
-      qp[i] = (int8_t)quant_one<MODE>(xp[i], inv, (uint32_t)(base + i) + bias, key);
-  }
+  const float inv = inv_of(*jobs.a[t]);
+  if (jobs.stochastic[t])
+    quantize_body<ROUND_STOCHASTIC>(jobs.x[t], jobs.q[t], (size_t)jobs.n[t], inv, jobs.ctr0[t],
+                                    derive_key(KeySpec{jobs.s1[t], jobs.ss}));
+  else
+    quantize_body<ROUND_NEAREST>(jobs.x[t], jobs.q[t], (size_t)jobs.n[t], inv, jobs.ctr0[t], RoundKey{0u, 0u});
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -291,7 +354,6 @@ __device__ __forceinline__ double softplus_value(double z) {
   return fmax(z, 0.0) + (double)log1pf(expf(-az));
 }
 
-constexpr int FF_MAX_LATER = 31;
 struct LaterLayers {
   const float* G[FF_MAX_LATER];
   float theta[FF_MAX_LATER];

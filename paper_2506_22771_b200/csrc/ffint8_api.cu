@@ -606,14 +606,14 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
 // Quantise the weights and run the forward contraction; the layer input is already in Xq and
 // its ranges in absmax[X_POS..X_NEG].
 ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B,
-                          float* a_next2, cudaStream_t st) {
+                          float* a_next2, cudaStream_t st, bool weights_ready = false) {
   const size_t nW = (size_t)L.N * L.K;
-  {
+  if (!weights_ready) {
     ProfScope prof(ctx, FF_K_ABSMAX, st);
     absmax_kernel<<<dim3(ew_blocks(ctx, nW / 4 + 1), 1), EW_THREADS, 0, st>>>(b.W, nW, b.absmax + FF_A_W, status_ptr(ctx));
   }
-  FF_LAUNCH_CHECK(ctx);
-  {
+  if (!weights_ready) FF_LAUNCH_CHECK(ctx);
+  if (!weights_ready) {
     ProfScope prof(ctx, FF_K_QUANTIZE, st);
     const dim3 grid(ew_blocks(ctx, nW / 4 + 1), 1);
     const KeySpec key = make_key_spec(L.seed, ROLE_W, L.index, step_ptr(ctx));
@@ -623,7 +623,7 @@ ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     else
       quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.W, b.Wq, nW, b.absmax + FF_A_W, key, S, b.rowmax, 2 * B);
   }
-  FF_LAUNCH_CHECK(ctx);
+  if (!weights_ready) FF_LAUNCH_CHECK(ctx);
   ff_status s = run_forward_gemm(ctx, L, b, B, st);
   if (s != FF_OK) return s;
   {
@@ -763,15 +763,66 @@ ff_status check_layer_list(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
 
 // INT8 forward through all layers with the current weights (Alg. 1 line 5-6): layer 0 reads bufs[0].X,
 // layer l > 0 reads bufs[l].X if given, else the previous layer's normalised output, quantised on the fly.
+// Everything a step can quantise before any layer has run, in three launches whatever the number of layers:
+// clear the range vectors, ranges of the network input (both sets) and of every layer's weights, then their
+// INT8 codes (which also clears the forward epilogues' per-sample accumulators).
+ff_status quantize_inputs_and_weights(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n, int B,
+                                      cudaStream_t st) {
+  ZeroJobs z;
+  z.n = n;
+  for (int l = 0; l < n; ++l) z.p[l] = bufs[l].absmax;
+  zero_ranges_kernel<<<1, 256, 0, st>>>(z);
+  FF_LAUNCH_CHECK(ctx);
+  AbsmaxJobs aj;
+  QuantJobs qj;
+  int t = 0;
+  size_t largest = 0;
+  const ff_layer_desc& L0 = layers[0];
+  const size_t per_sample0 = (size_t)in_rows_per_sample(L0) * in_features(L0), per_pass0 = per_sample0 * B;
+  const uint2 bias0 = ctr_bias(ctx, per_sample0, B);
+  for (int p = 0; p < 2; ++p, ++t) {
+    aj.x[t] = bufs[0].X + p * per_pass0, aj.n[t] = per_pass0, aj.out[t] = bufs[0].absmax + FF_A_X_POS + p;
+    qj.x[t] = aj.x[t], qj.q[t] = bufs[0].Xq + p * per_pass0, qj.n[t] = per_pass0, qj.a[t] = aj.out[t];
+    qj.s1[t] = make_key_spec(L0.seed, ROLE_X, L0.index, nullptr).s1;
+    qj.ctr0[t] = (uint32_t)(p * per_pass0) + (p ? bias0.y : bias0.x);
+    qj.stochastic[t] = L0.round_x != FF_ROUND_NEAREST_EVEN;
+  }
+  largest = per_pass0;
+  for (int l = 0; l < n; ++l, ++t) {
+    const size_t nW = (size_t)layers[l].N * layers[l].K;
+    aj.x[t] = bufs[l].W, aj.n[t] = nW, aj.out[t] = bufs[l].absmax + FF_A_W;
+    qj.x[t] = bufs[l].W, qj.q[t] = bufs[l].Wq, qj.n[t] = nW, qj.a[t] = aj.out[t];
+    qj.s1[t] = make_key_spec(layers[l].seed, ROLE_W, layers[l].index, nullptr).s1;
+    qj.ctr0[t] = 0u;
+    qj.stochastic[t] = layers[l].round_w != FF_ROUND_NEAREST_EVEN;
+    qj.zero_S[l] = reinterpret_cast<unsigned long long*>(bufs[l].S);
+    qj.zero_rowmax[l] = bufs[l].rowmax;
+    if (nW > largest) largest = nW;
+  }
+  qj.n_zero = n, qj.zero_n = 2 * B, qj.ss = step_ptr(ctx);
+  const dim3 grid(ew_blocks(ctx, largest / 4 + 1), t);
+  {
+    ProfScope prof(ctx, FF_K_ABSMAX, st);
+    absmax_multi_kernel<<<grid, EW_THREADS, 0, st>>>(aj, status_ptr(ctx));
+  }
+  FF_LAUNCH_CHECK(ctx);
+  {
+    ProfScope prof(ctx, FF_K_QUANTIZE, st);
+    quantize_multi_kernel<<<grid, EW_THREADS, 0, st>>>(qj);
+  }
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
+
 ff_status forward_all(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
                       cudaStream_t st) {
   ff_status s;
-  for (int l = 0; l < n_layers; ++l) FF_CUDA(ctx, cudaMemsetAsync(bufs[l].absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
+  if ((s = quantize_inputs_and_weights(ctx, layers, bufs, n_layers, B, st)) != FF_OK) return s;
   for (int l = 0; l < n_layers; ++l) {
     const bool chained = l > 0 && !bufs[l].X;
-    if (!chained && (s = quantize_input(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
+    if (l > 0 && !chained && (s = quantize_input(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
     const bool feeds_next = l + 1 < n_layers && !bufs[l + 1].X;
-    if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st)) != FF_OK)
+    if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st, true)) != FF_OK)
       return s;
     if ((s = normalize_output(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].Xq : nullptr,
                               feeds_next ? &layers[l + 1] : nullptr, st)) != FF_OK)
