@@ -376,6 +376,11 @@ struct LossScratch {
   double lsum[LOSS_MAX_BLOCKS];
   uint32_t amax[2][LOSS_MAX_BLOCKS];
 };
+__device__ __forceinline__ void loss_coef_body(const float* __restrict__ G, float theta, const float* const* later_G,
+                                               const float* later_theta, int later_n, float lambda, int B,
+                                               const int32_t* __restrict__ rowmax, float* __restrict__ absmax,
+                                               float* __restrict__ coef, float* __restrict__ loss,
+                                               LossScratch* __restrict__ scratch, int m_total);
 __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __restrict__ G, float theta, LaterLayers later,
                                                                  float lambda, int B, const int32_t* __restrict__ rowmax,
                                                                  float* __restrict__ absmax, float* __restrict__ coef,
@@ -383,6 +388,31 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
                                                                  const StepState* __restrict__ ss = nullptr,
                                                                  int m_total = 0) {
   if (ss) lambda = ss->lambda;  // a step run through the library's own launch sequence keeps lambda in device memory
+  loss_coef_body(G, theta, later.G, later.theta, later.n, lambda, B, rowmax, absmax, coef, loss, scratch, m_total);
+}
+// Every layer of a step in one launch (blockIdx.y = layer): the losses depend on the goodness values alone,
+// which are all there once the forward has run.  Layer l looks ahead at layers l+1 .. n-1 of the same table;
+// each layer has its own scratch.
+struct LossJobs {
+  const float* G[FF_MAX_LATER + 1];
+  float theta[FF_MAX_LATER + 1];
+  const int32_t* rowmax[FF_MAX_LATER + 1];
+  float* absmax[FF_MAX_LATER + 1];
+  float* coef[FF_MAX_LATER + 1];
+  float* loss[FF_MAX_LATER + 1];
+  int n;
+};
+__global__ void __launch_bounds__(LOSS_THREADS) loss_coef_multi_kernel(const LossJobs jobs, int B, LossScratch* __restrict__ scratch,
+                                                                       const StepState* __restrict__ ss, int m_total) {
+  const int l = blockIdx.y;
+  loss_coef_body(jobs.G[l], jobs.theta[l], jobs.G + l + 1, jobs.theta + l + 1, jobs.n - 1 - l, ss->lambda, B, jobs.rowmax[l],
+                 jobs.absmax[l], jobs.coef[l], jobs.loss[l], scratch + l, m_total);
+}
+__device__ __forceinline__ void loss_coef_body(const float* __restrict__ G, float theta, const float* const* later_G,
+                                               const float* later_theta, int later_n, float lambda, int B,
+                                               const int32_t* __restrict__ rowmax, float* __restrict__ absmax,
+                                               float* __restrict__ coef, float* __restrict__ loss,
+                                               LossScratch* __restrict__ scratch, int m_total) {
   __shared__ double red[LOSS_THREADS / 32];
   __shared__ uint32_t redmax[2][LOSS_THREADS / 32];
   __shared__ bool is_last;
@@ -401,8 +431,8 @@ __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_kernel(const float* __
     double g0 = __dmul_rn(sign, sigmoid_spec(arg));
     double L0 = softplus_value(arg);
     double gsum = 0.0, Lsum = 0.0;
-    for (int j = 0; j < later.n; ++j) {
-      double aj = __dmul_rn(sign, __dsub_rn((double)later.G[j][m], (double)later.theta[j]));
+    for (int j = 0; j < later_n; ++j) {
+      double aj = __dmul_rn(sign, __dsub_rn((double)later_G[j][m], (double)later_theta[j]));
       gsum = __dadd_rn(gsum, __dmul_rn(sign, sigmoid_spec(aj)));
       Lsum += softplus_value(aj);
     }
@@ -487,14 +517,44 @@ __global__ void __launch_bounds__(EW_THREADS) classify_kernel(LaterLayers layers
 // dHq = clip(round((2*coef_m * y) * 127/a_dh[p])).  grid = (blocks, 2)
 // ---------------------------------------------------------------------------------------------
 template <int MODE>
+__device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, const float* __restrict__ coef,
+                                                 const float* __restrict__ absmax, size_t per_sample, size_t per_pass,
+                                                 int8_t* __restrict__ dHq, RoundKey key, int pass, uint32_t bias);
+template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) dh_quantize_kernel(const float* __restrict__ Y, const float* __restrict__ coef,
                                                                  const float* __restrict__ absmax, size_t per_sample,
                                                                  size_t per_pass, int8_t* __restrict__ dHq, KeySpec ks,
                                                                  uint2 ctr_bias = uint2{0u, 0u}) {
   const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
-  const uint32_t bias = blockIdx.y ? ctr_bias.y : ctr_bias.x;
-  const size_t base = (size_t)blockIdx.y * per_pass;
-  const float inv = inv_of(absmax[3 + blockIdx.y]);
+  dh_quantize_body<MODE>(Y, coef, absmax, per_sample, per_pass, dHq, key, blockIdx.y, blockIdx.y ? ctr_bias.y : ctr_bias.x);
+}
+// Every layer of a step in one launch: blockIdx.y = 2*layer + set.
+struct DhJobs {
+  const float* Y[FF_MAX_LATER + 1];
+  const float* coef[FF_MAX_LATER + 1];
+  const float* absmax[FF_MAX_LATER + 1];
+  unsigned long long per_sample[FF_MAX_LATER + 1];
+  int8_t* dHq[FF_MAX_LATER + 1];
+  unsigned long long s1[FF_MAX_LATER + 1];
+  uint8_t stochastic[FF_MAX_LATER + 1];
+  const StepState* ss;
+};
+__global__ void __launch_bounds__(EW_THREADS) dh_quantize_multi_kernel(const DhJobs jobs, int B) {
+  const int l = blockIdx.y >> 1, pass = blockIdx.y & 1;
+  const size_t per_sample = (size_t)jobs.per_sample[l], per_pass = per_sample * B;
+  if (jobs.stochastic[l])
+    dh_quantize_body<ROUND_STOCHASTIC>(jobs.Y[l], jobs.coef[l], jobs.absmax[l], per_sample, per_pass, jobs.dHq[l],
+                                       derive_key(KeySpec{jobs.s1[l], jobs.ss}), pass, 0u);
+  else
+    dh_quantize_body<ROUND_NEAREST>(jobs.Y[l], jobs.coef[l], jobs.absmax[l], per_sample, per_pass, jobs.dHq[l], RoundKey{0u, 0u},
+                                    pass, 0u);
+}
+template <int MODE>
+__device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, const float* __restrict__ coef,
+                                                 const float* __restrict__ absmax, size_t per_sample, size_t per_pass,
+                                                 int8_t* __restrict__ dHq, RoundKey key, int pass, uint32_t bias) {
+  const size_t base = (size_t)pass * per_pass;
+  const float inv = inv_of(absmax[3 + pass]);
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)dHq) & 3) == 0);
   const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
   if (vec) {

@@ -65,7 +65,8 @@ namespace {
 constexpr size_t WS_STATUS_BYTES = 256;
 constexpr size_t WS_STEP_OFFSET = 64;   // StepState inside the status block
 constexpr size_t WS_LOSS_OFFSET = WS_STATUS_BYTES;
-constexpr size_t WS_BYTES = (WS_LOSS_OFFSET + sizeof(LossScratch) + 255) / 256 * 256;  // fixed header
+// one scratch per layer: the losses of all layers of a step are computed by one launch
+constexpr size_t WS_BYTES = (WS_LOSS_OFFSET + (FF_MAX_LATER + 1) * sizeof(LossScratch) + 255) / 256 * 256;  // fixed header
 // After the header: INT32 partial-sum slabs of a split weight-gradient contraction,
 // [splits][2 sets][N][K].  Splitting is used where the output N x K alone has too few tiles to
 // occupy the device (convolutions contract over every output position of the batch).
@@ -835,20 +836,40 @@ ff_status forward_all(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_b
 ff_status train_step_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
                           float lambda, cudaStream_t st) {
   ff_status s;
+  (void)lambda;  // read by the kernels from the step state
   // Alg. 1 line 5-6: one forward through all layers with the pre-update weights
   if ((s = forward_all(ctx, layers, bufs, n_layers, B, st)) != FF_OK) return s;
-  // Alg. 1 line 7-9: per layer, loss from the G's (Eq. 3), INT8 gradient and update
+  // Alg. 1 line 7-9: loss from the G's (Eq. 3) and INT8 output gradient - neither depends on an update, so all
+  // layers share one launch each - then per layer the weight gradient and update
+  LossJobs lj;
+  DhJobs dj;
+  lj.n = n_layers;
+  size_t largest = 0;
   for (int l = 0; l < n_layers; ++l) {
-    const float* Gl[FF_MAX_LATER];
-    float th[FF_MAX_LATER];
-    int n_later = n_layers - 1 - l;
-    for (int j = 0; j < n_later; ++j) {
-      Gl[j] = bufs[l + 1 + j].G;
-      th[j] = layers[l + 1 + j].theta;
-    }
-    if ((s = loss_grad_impl(ctx, layers[l], bufs[l], B, Gl, th, n_later, lambda, st)) != FF_OK) return s;
-    if ((s = run_update_gemm(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
+    lj.G[l] = bufs[l].G, lj.theta[l] = layers[l].theta, lj.rowmax[l] = bufs[l].rowmax, lj.absmax[l] = bufs[l].absmax;
+    lj.coef[l] = bufs[l].coef, lj.loss[l] = bufs[l].loss;
+    dj.Y[l] = bufs[l].Y, dj.coef[l] = bufs[l].coef, dj.absmax[l] = bufs[l].absmax, dj.dHq[l] = bufs[l].dHq;
+    dj.per_sample[l] = (unsigned long long)rows_per_sample(layers[l]) * layers[l].N;
+    dj.s1[l] = make_key_spec(layers[l].seed, ROLE_DH, layers[l].index, nullptr).s1;
+    dj.stochastic[l] = layers[l].round_dh != FF_ROUND_NEAREST_EVEN;
+    if (dj.per_sample[l] * B > largest) largest = dj.per_sample[l] * B;
   }
+  dj.ss = step_ptr(ctx);
+  int loss_blocks = (2 * B + LOSS_THREADS - 1) / LOSS_THREADS;
+  if (loss_blocks > LOSS_MAX_BLOCKS) loss_blocks = LOSS_MAX_BLOCKS;
+  {
+    ProfScope prof(ctx, FF_K_LOSS, st);
+    loss_coef_multi_kernel<<<dim3(loss_blocks, n_layers), LOSS_THREADS, 0, st>>>(
+        lj, B, reinterpret_cast<LossScratch*>(static_cast<char*>(ctx->workspace) + WS_LOSS_OFFSET), step_ptr(ctx), 0);
+  }
+  FF_LAUNCH_CHECK(ctx);
+  {
+    ProfScope prof(ctx, FF_K_DH_QUANTIZE, st);
+    dh_quantize_multi_kernel<<<dim3(ew_blocks(ctx, largest / 4 + 1), 2 * n_layers), EW_THREADS, 0, st>>>(dj, B);
+  }
+  FF_LAUNCH_CHECK(ctx);
+  for (int l = 0; l < n_layers; ++l)
+    if ((s = run_update_gemm(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
   return FF_OK;
 }
 
