@@ -557,7 +557,25 @@ __device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, co
   const float inv = inv_of(absmax[3 + pass]);
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)dHq) & 3) == 0);
   const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
-  if (vec) {
+  if (vec && per_sample >= 4 * EW_THREADS * 4 && per_pass / per_sample >= 2 * (size_t)gridDim.x) {
+    // long samples, and enough of them to keep every block busy: a block walks whole samples, so the per-sample
+    // factor is read once per sample and no sample bookkeeping rides along with the elements
+    const uint32_t g4 = (uint32_t)(per_sample >> 2), n_samples = (uint32_t)(per_pass / per_sample);
+    const float* cp = coef + (size_t)pass * n_samples;
+    for (uint32_t smp = blockIdx.x; smp < n_samples; smp += gridDim.x) {
+      const float k2 = __fmul_rn(2.0f, __ldg(cp + smp));
+      const size_t e0 = base + (size_t)smp * per_sample;
+#pragma unroll 4
+      for (uint32_t i = threadIdx.x; i < g4; i += EW_THREADS) {
+        const size_t e = e0 + ((size_t)i << 2);
+        const float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
+        int q0, q1, q2, q3;
+        quant_pair<MODE>(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, (uint32_t)e + bias, key, q0, q1);
+        quant_pair<MODE>(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, (uint32_t)e + bias + 2, key, q2, q3);
+        *reinterpret_cast<uint32_t*>(dHq + e) = pack4(q0, q1, q2, q3);
+      }
+    }
+  } else if (vec) {
     const uint32_t n4 = (uint32_t)(per_pass >> 2);
     const float* cp = coef + (uint32_t)(base / per_sample);
     SampleCursor cur(tid, stride, (uint32_t)(per_sample >> 2));

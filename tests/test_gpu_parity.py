@@ -574,3 +574,12 @@ def test_predict_with_replayed_launches():
         net.train_step(0.0, step)
     assert ffb.ff_graph_replay_count(net.ctx.ctx) == 6
     net.close()
+
+
+def test_wide_outputs_many_samples_walk_samples_in_the_dh_quantiser():
+    # 2400 + 2400 samples of 4096 outputs: the output-gradient quantiser takes its sample-walking path
+    # (long samples, more samples than blocks); checked with both rounding modes of g^Y
+    layers = [synth.LayerCfg(0, 64, 4096, 2048.0, 0.03, float(np.sqrt(4096)))]
+    w = synth.Workload("wide_out", 2400, layers, (64,), "uniform01", "kaiming_uniform", 1)
+    for rounding in [(1, 0, 1), (1, 0, 0)]:
+        _run_and_compare(w, seed=66, steps=2, lam_per_step=0.0, path=(ffb.FF_GEMM_AUTO, 0), rounding=rounding)
