@@ -11,6 +11,7 @@ namespace ffi8 {
 
 constexpr int EW_THREADS = 256;
 constexpr int FF_MAX_LATER = 31;  // layers after the first in one call
+constexpr uint32_t SAMPLE_TILE_GROUPS = 4 * EW_THREADS;  // float4 groups of one sample that a block takes at a time
 
 __device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) { return __reduce_max_sync(0xffffffffu, v); }
 
@@ -238,7 +239,36 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) &&
                    (!xnext || (((uintptr_t)xnext) & 15) == 0) && (!xq || (((uintptr_t)xq) & 3) == 0);
   const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
-  if (vec) {
+  if (vec && per_sample >= 4 * SAMPLE_TILE_GROUPS) {
+    // long samples: blocks take (sample, tile of the sample) pairs, so the per-sample factor (a square root and a
+    // division) is formed once per tile instead of once per four elements
+    const uint32_t g4 = (uint32_t)(per_sample >> 2), n_samples = (uint32_t)(per_pass / per_sample);
+    const uint32_t tps = (g4 + SAMPLE_TILE_GROUPS - 1) / SAMPLE_TILE_GROUPS;
+    const float* Gp = G + (size_t)blockIdx.y * n_samples;
+    for (uint32_t tile = blockIdx.x; tile < n_samples * tps; tile += gridDim.x) {
+      const uint32_t smp = tile / tps, g0 = (tile - smp * tps) * SAMPLE_TILE_GROUPS;
+      const float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(__ldg(Gp + smp)), eps));
+      const size_t e0 = base + (size_t)smp * per_sample;
+#pragma unroll
+      for (uint32_t k = 0; k < SAMPLE_TILE_GROUPS / EW_THREADS; ++k) {
+        const uint32_t i = g0 + k * EW_THREADS + threadIdx.x;
+        if (i >= g4) break;
+        const size_t e = e0 + ((size_t)i << 2);
+        float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
+        v.x = __fmul_rn(v.x, r);
+        v.y = __fmul_rn(v.y, r);
+        v.z = __fmul_rn(v.z, r);
+        v.w = __fmul_rn(v.w, r);
+        if (xnext) *reinterpret_cast<float4*>(xnext + e) = v;
+        if (xq) {
+          int q0, q1, q2, q3;
+          quant_pair<MODE>(v.x, v.y, inv, (uint32_t)e + bias, key, q0, q1);
+          quant_pair<MODE>(v.z, v.w, inv, (uint32_t)e + bias + 2, key, q2, q3);
+          *reinterpret_cast<uint32_t*>(xq + e) = pack4(q0, q1, q2, q3);
+        }
+      }
+    }
+  } else if (vec) {
     const uint32_t n4 = (uint32_t)(per_pass >> 2);
     const float* Gp = G + (uint32_t)(base / per_sample);
     SampleCursor cur(tid, stride, (uint32_t)(per_sample >> 2));
@@ -557,16 +587,20 @@ __device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, co
   const float inv = inv_of(absmax[3 + pass]);
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)dHq) & 3) == 0);
   const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
-  if (vec && per_sample >= 4 * EW_THREADS * 4 && per_pass / per_sample >= 2 * (size_t)gridDim.x) {
-    // long samples, and enough of them to keep every block busy: a block walks whole samples, so the per-sample
-    // factor is read once per sample and no sample bookkeeping rides along with the elements
+  if (vec && per_sample >= 4 * SAMPLE_TILE_GROUPS) {
+    // long samples: blocks take (sample, tile of the sample) pairs, so the per-sample factor is read once per
+    // tile and no sample bookkeeping rides along with the elements
     const uint32_t g4 = (uint32_t)(per_sample >> 2), n_samples = (uint32_t)(per_pass / per_sample);
+    const uint32_t tps = (g4 + SAMPLE_TILE_GROUPS - 1) / SAMPLE_TILE_GROUPS;
     const float* cp = coef + (size_t)pass * n_samples;
-    for (uint32_t smp = blockIdx.x; smp < n_samples; smp += gridDim.x) {
+    for (uint32_t tile = blockIdx.x; tile < n_samples * tps; tile += gridDim.x) {
+      const uint32_t smp = tile / tps, g0 = (tile - smp * tps) * SAMPLE_TILE_GROUPS;
       const float k2 = __fmul_rn(2.0f, __ldg(cp + smp));
       const size_t e0 = base + (size_t)smp * per_sample;
-#pragma unroll 4
-      for (uint32_t i = threadIdx.x; i < g4; i += EW_THREADS) {
+#pragma unroll
+      for (uint32_t k = 0; k < SAMPLE_TILE_GROUPS / EW_THREADS; ++k) {
+        const uint32_t i = g0 + k * EW_THREADS + threadIdx.x;
+        if (i >= g4) break;
         const size_t e = e0 + ((size_t)i << 2);
         const float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
         int q0, q1, q2, q3;

@@ -576,9 +576,9 @@ def test_predict_with_replayed_launches():
     net.close()
 
 
-def test_wide_outputs_many_samples_walk_samples_in_the_dh_quantiser():
-    # 2400 + 2400 samples of 4096 outputs: the output-gradient quantiser takes its sample-walking path
-    # (long samples, more samples than blocks); checked with both rounding modes of g^Y
+def test_wide_outputs_many_samples_take_the_per_sample_tiles():
+    # 2400 + 2400 samples of 4096 outputs: the output-gradient quantiser (and a normalisation, were there a next
+    # layer) takes (sample, tile) pairs per block - more pairs than blocks here; both rounding modes of g^Y
     layers = [synth.LayerCfg(0, 64, 4096, 2048.0, 0.03, float(np.sqrt(4096)))]
     w = synth.Workload("wide_out", 2400, layers, (64,), "uniform01", "kaiming_uniform", 1)
     for rounding in [(1, 0, 1), (1, 0, 0)]:
