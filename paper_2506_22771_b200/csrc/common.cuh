@@ -109,9 +109,17 @@ __device__ __forceinline__ float apply_update(const UpdateRule& r, const UpdateC
   return __fsub_rn(w, __fmul_rn(r.lr, g));
 }
 
-__global__ void set_step_kernel(StepState* ss, unsigned long long step, float lambda, int set_lambda) {
-  ss->step = step;
-  if (set_lambda) ss->lambda = lambda;
+// Range vectors (8 floats per layer) that the same launch clears for the step that follows.
+struct RangeTable {
+  float* p[32];
+  int n;
+};
+__global__ void set_step_kernel(StepState* ss, unsigned long long step, float lambda, int set_lambda, RangeTable ranges) {
+  if (threadIdx.x == 0) {
+    ss->step = step;
+    if (set_lambda) ss->lambda = lambda;
+  }
+  if ((int)threadIdx.x < ranges.n * 8) ranges.p[threadIdx.x >> 3][threadIdx.x & 7] = 0.0f;
 }
 
 // s = a/127, inv = 127/a.  A zero tensor, or one whose range is below 2^-100 (127/a would leave

@@ -129,16 +129,6 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __res
   quantize_body<MODE>(x + base, q + base, n_per_pass, inv_of(a[blockIdx.y]), (uint32_t)base + bias, key);
 }
 
-// Clears the range vectors (FF_ABSMAX_LEN floats each) of up to FF_MAX_LATER + 1 layers.  <<<1, 256>>>
-struct ZeroJobs {
-  float* p[FF_MAX_LATER + 1];
-  int n;
-};
-__global__ void zero_ranges_kernel(ZeroJobs z) {
-  const int i = threadIdx.x;
-  if (i < z.n * FF_ABSMAX_LEN) z.p[i / FF_ABSMAX_LEN][i % FF_ABSMAX_LEN] = 0.0f;
-}
-
 // One launch for a table of tensors (blockIdx.y = tensor): the weights of every layer and the two sets of
 // the network input, each with its own range, rounding mode, key and first counter.  Also clears the
 // per-sample accumulators of every layer's forward epilogue.

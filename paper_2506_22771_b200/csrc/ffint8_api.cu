@@ -192,8 +192,15 @@ inline StepState* step_ptr(ff_ctx* ctx) {
   return reinterpret_cast<StepState*>(static_cast<char*>(ctx->workspace) + WS_STEP_OFFSET);
 }
 // Publishes the step counter (and lambda) to the kernels of the calls that follow on `st`.
-ff_status set_step(ff_ctx* ctx, uint64_t step, float lambda, bool with_lambda, cudaStream_t st) {
-  set_step_kernel<<<1, 1, 0, st>>>(step_ptr(ctx), step, lambda, with_lambda ? 1 : 0);
+// With a layer list, the range vectors of those layers are cleared by the same launch (a whole-network call starts
+// by taking ranges; the launch is issued outside any captured sequence, so it costs the replayed step nothing).
+ff_status set_step(ff_ctx* ctx, uint64_t step, float lambda, bool with_lambda, cudaStream_t st,
+                   const ff_layer_bufs* bufs = nullptr, int n_layers = 0) {
+  static_assert(FF_MAX_LATER + 1 <= 32 && FF_ABSMAX_LEN == 8, "RangeTable holds 32 vectors of 8 floats");
+  RangeTable rt;
+  rt.n = bufs ? n_layers : 0;
+  for (int l = 0; l < rt.n; ++l) rt.p[l] = bufs[l].absmax;
+  set_step_kernel<<<1, 256, 0, st>>>(step_ptr(ctx), step, lambda, with_lambda ? 1 : 0, rt);
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
@@ -764,16 +771,11 @@ ff_status check_layer_list(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
 
 // INT8 forward through all layers with the current weights (Alg. 1 line 5-6): layer 0 reads bufs[0].X,
 // layer l > 0 reads bufs[l].X if given, else the previous layer's normalised output, quantised on the fly.
-// Everything a step can quantise before any layer has run, in three launches whatever the number of layers:
-// clear the range vectors, ranges of the network input (both sets) and of every layer's weights, then their
-// INT8 codes (which also clears the forward epilogues' per-sample accumulators).
+// Everything a step can quantise before any layer has run, in two launches whatever the number of layers:
+// ranges of the network input (both sets) and of every layer's weights, then their INT8 codes (which also
+// clears the forward epilogues' per-sample accumulators).  The range vectors were cleared by set_step.
 ff_status quantize_inputs_and_weights(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n, int B,
                                       cudaStream_t st) {
-  ZeroJobs z;
-  z.n = n;
-  for (int l = 0; l < n; ++l) z.p[l] = bufs[l].absmax;
-  zero_ranges_kernel<<<1, 256, 0, st>>>(z);
-  FF_LAUNCH_CHECK(ctx);
   AbsmaxJobs aj;
   QuantJobs qj;
   int t = 0;
@@ -1191,7 +1193,7 @@ ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
   if ((s = check_layer_list(ctx, layers, bufs, n_layers, B)) != FF_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
-  if ((s = set_step(ctx, step, lambda, true, st)) != FF_OK) return s;
+  if ((s = set_step(ctx, step, lambda, true, st, bufs, n_layers)) != FF_OK) return s;
   if (ctx->graph_mode && !ctx->profiling) return train_step_graph(ctx, layers, bufs, n_layers, B, lambda, st);
   return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
 }
@@ -1252,7 +1254,7 @@ ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bu
   if (first_counted_layer < 0 || first_counted_layer >= n_layers) return fail(ctx, FF_ERR_ARG, "first_counted_layer out of range");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
-  if ((s = set_step(ctx, step, 0.0f, false, st)) != FF_OK) return s;
+  if ((s = set_step(ctx, step, 0.0f, false, st, bufs, n_layers)) != FF_OK) return s;
   auto body = [&](cudaStream_t sb) -> ff_status {
     ff_status r = forward_all(ctx, layers, bufs, n_layers, half, sb);
     if (r != FF_OK) return r;
