@@ -59,6 +59,34 @@ def _ncu_traffic(kind: str, workload: str, B: int):
     return t["bytes_per_launch"].get(kind)
 
 
+def _library_int8_gemm(w, B: int, dev):
+    """Context for the contraction figures: the vendor library's INT8 GEMM (torch._int_mm -> cuBLASLt) on the shape of
+    the last layer's forward contraction, timed with CUDA events right after the bench's own timed regions (so at
+    about the same power state; a 20-launch burst all the same).  Not part of the product path."""
+    import torch
+    l = w.layers[-1]
+    M, N, K = 2 * B * l.H * l.Wd, l.N, l.K
+    if l.kind != 0 or M % 8 or N % 8 or K % 8 or M * N * 4 > 8e9:
+        return None
+    try:
+        a = torch.randint(-127, 128, (M, K), dtype=torch.int8, device=dev)
+        bt = torch.randint(-127, 128, (N, K), dtype=torch.int8, device=dev).t()
+        for _ in range(3):
+            torch._int_mm(a, bt)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 20
+        e0.record()
+        for _ in range(n):
+            torch._int_mm(a, bt)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / n
+        return {"shape": [M, N, K], "ms": ms, "tops": 2.0 * M * N * K / (ms * 1e-3) / 1e12,
+                "note": "torch._int_mm (cuBLASLt), INT32 output, no epilogue; for comparison only"}
+    except Exception as e:  # the comparison is optional
+        return {"unavailable": str(e)[:200]}
+
+
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -276,6 +304,7 @@ def main():
     ap.add_argument("--cpu-sample", type=int, default=256, help="positives per step of the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-library-gemm", action="store_true", help="skip the cuBLASLt INT8 GEMM timed for comparison")
     ap.add_argument("--B", type=int, default=0, help="override positives per batch (profiling runs on a smaller case)")
     ap.add_argument("--tensor-form", type=int, default=0, help="CTAs per tensor-core tile: 0 auto, 1, 2")
     ap.add_argument("--no-graph", action="store_true",
@@ -399,6 +428,9 @@ def main():
     clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     ffb.ff_poll_status(ctx.ctx, stream)
 
+    # the vendor library's INT8 GEMM of the same shape, right after the timed regions (same power state)
+    lib_gemm = _library_int8_gemm(w, B, dev) if (world == 1 and rank == 0 and not args.no_library_gemm) else None
+
     # ---------------- end to end: host buffers, H2D of the step's inputs + D2H of the loss every step ---------
     # What crosses PCIe per step is what a trainer holds on the host: the B labelled samples (FP32) and their
     # true / wrong labels.  The positive / negative batch is built from them on the device (ff_embed_labels),
@@ -510,7 +542,10 @@ def main():
                          "frac_of_nominal_4500": per_kernel[dom]["achieved"] / 4500.0,
                          "traffic": _ncu_traffic(dom, args.workload, B)},
             "kernels": per_kernel,
+            "rows_per_s": 2.0 * value,
         }
+        if lib_gemm is not None:
+            out["library_int8_gemm"] = lib_gemm
         if not args.no_cpu_baseline and world == 1:
             Bs = min(B, args.cpu_sample)
             t, cores = _oracle_step_time(w, Bs, 1)
