@@ -212,21 +212,31 @@ def _oracle_step_time(w, B_sample: int, steps: int, seed: int = 1):
 
 
 def run_reference(args):
-    """Reference arm = the CPU oracle on the host cores (bounded sample per step)."""
+    """Reference arm = the CPU oracle, as it stands, on the host cores.  Each step is a bounded sample of the
+    workload (--cpu-sample positives + negatives at full layer widths).  `--warmup` untimed and `--steps` timed steps
+    are run when they fit --cpu-budget-s seconds (projected from the first step); a step's cost is dominated by
+    quantising and updating the full-width weights, which a smaller sample would not reduce, so when they do not
+    fit, fewer steps are timed and the line says how many ("steps" = timed, "steps_requested" = asked for)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     w = synth.workload(args.workload)
+    want, warmup = max(1, args.steps), max(1, args.warmup)
     B_sample = min(w.B, args.cpu_sample)
-    _oracle_step_time(w, B_sample, 1)
-    steps = max(1, min(args.steps, 3))
+    t_first, _ = _oracle_step_time(w, B_sample, 1)                 # the first warm-up step, also the probe
+    afford = max(1, int(args.cpu_budget_s / max(t_first, 1e-6)))    # steps of any kind that fit the budget
+    warm_left = min(warmup - 1, max(0, afford - 2))
+    steps = min(want, max(1, afford - 1 - warm_left))
+    if warm_left:
+        _oracle_step_time(w, B_sample, warm_left)
     t, cores = _oracle_step_time(w, B_sample, steps)
     v = B_sample / t
     sample = f"{B_sample} positive + {B_sample} negative samples of the {args.workload} workload per step, full layer widths"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": 1, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int8", "data": "synthetic", "config": {"workload": args.workload, "B_pos": B_sample, "B_neg": B_sample},
+        "steps_requested": want, "warmup": 1 + warm_left, "ms_per_step": t * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": args.workload, "B_pos": B_sample, "B_neg": B_sample},
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
@@ -302,6 +312,8 @@ def main():
     ap.add_argument("--workload", default="roofline")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-sample", type=int, default=256, help="positives per step of the CPU-oracle sample")
+    ap.add_argument("--cpu-budget-s", type=float, default=180.0,
+                    help="--impl reference: seconds of oracle time that all warm-up and timed steps together may take")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-library-gemm", action="store_true", help="skip the cuBLASLt INT8 GEMM timed for comparison")

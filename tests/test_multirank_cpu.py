@@ -131,3 +131,30 @@ def test_pointer_table_rejects_foreign_addresses_and_types():
         table.view(t.data_ptr() + 24, 4, ffb.FF_DP_F32)      # runs past the end
     with pytest.raises(TypeError):
         table.view(t.data_ptr(), 2, ffb.FF_DP_I32)
+
+
+def test_reference_arm_prints_one_contract_line():
+    """`bench.py --impl reference` (the oracle on the host cores) on the small workload: one JSON line with the
+    metric, the exact step counts when they fit the time budget, and the oracle named as the baseline."""
+    import json
+    import subprocess
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny_mlp",
+                          "--steps", "4", "--warmup", "2", "--gpus", "1"], capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-500:]
+    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["metric"] == "FF-INT8 train samples/s" and d["unit"] == "samples/s"
+    assert d["steps"] == 4 and d["steps_requested"] == 4 and d["warmup"] == 2 and d["n_gpus"] == 1
+    assert d["higher_is_better"] is True and d["vs_baseline"] is None and d["value"] > 0
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"]
+    assert d["e2e"] == {"value": d["value"], "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert d["config"]["workload"] == "tiny_mlp"
+
+
+def test_reference_arm_other_ranks_do_nothing():
+    import subprocess
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny_mlp",
+                          "--steps", "1", "--warmup", "1", "--gpus", "2"], capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0 and out.stdout.strip() == ""
