@@ -312,7 +312,7 @@ def main():
     ap.add_argument("--workload", default="roofline")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-sample", type=int, default=256, help="positives per step of the CPU-oracle sample")
-    ap.add_argument("--cpu-budget-s", type=float, default=180.0,
+    ap.add_argument("--cpu-budget-s", type=float, default=210.0,
                     help="--impl reference: seconds of oracle time that all warm-up and timed steps together may take")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
