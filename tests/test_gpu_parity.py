@@ -583,3 +583,33 @@ def test_wide_outputs_many_samples_take_the_per_sample_tiles():
     w = synth.Workload("wide_out", 2400, layers, (64,), "uniform01", "kaiming_uniform", 1)
     for rounding in [(1, 0, 1), (1, 0, 0)]:
         _run_and_compare(w, seed=66, steps=2, lam_per_step=0.0, path=(ffb.FF_GEMM_AUTO, 0), rounding=rounding)
+
+
+def test_graph_cache_evicts_least_recently_used_shapes():
+    # 20 call shapes (the same layer with 20 different step sizes) through one context that keeps 16 graphs:
+    # every shape still computes the oracle's step, replays resume after a shape was dropped and re-captured
+    w = synth.scaled(synth.workload("tiny_mlp"), B=16, width_div=4)
+    w.layers = w.layers[:1]
+    X = synth.make_batch(w, 3)
+    W0 = synth.make_weights(w, 3)
+    specs0, descs0 = specs_and_descs(w.layers, 3)
+    net = GpuNet(descs0, w.B, W0, graph=True)
+    net.set_input(X)
+    import torch
+    for rnd in range(2):
+        for i in range(20):
+            lr = 0.01 * (i + 1)
+            w.layers[0].lr = lr
+            specs, descs = specs_and_descs(w.layers, 3)
+            net.descs_arr[0] = descs[0]
+            for b, W in zip(net.bufs, W0):
+                b.W.copy_(torch.from_numpy(W))
+            Ws = W0
+            for step in range(3):          # eager, capture, replay
+                net.train_step(0.0, step)
+                st = O.train_step(specs, Ws, X, w.B, 0.0, step)
+                Ws = [s.W_new for s in st]
+            compare_layer(st[0], net.bufs[0], specs[0], w.B, tag=f"round{rnd}/shape{i}/")
+    # per shape and round: 2 replays (steps 1 and 2); every shape was evicted before its second round (20 > 16)
+    assert ffb.ff_graph_replay_count(net.ctx.ctx) == 2 * 20 * 2, ffb.ff_last_error(net.ctx.ctx)
+    net.close()
