@@ -126,7 +126,10 @@ typedef struct {
 } ff_layer_bufs;
 
 /* Create / destroy a context for CUDA device `device` (must be compute capability 10.x).
- * ff_create makes the device current and allocates nothing on it. */
+ * ff_create makes the device current and allocates nothing on it.  A context holds host state only
+ * (route choices, the last error text, captured launch sequences) and is not thread-safe: calls on one
+ * context must not overlap in time; its kernels share the workspace, so they belong on one stream (or on
+ * streams the caller orders).  Several contexts, each with its own workspace, are independent. */
 ff_status ff_create(ff_ctx** out, int device);
 ff_status ff_destroy(ff_ctx* ctx);
 
