@@ -98,14 +98,23 @@ __device__ __forceinline__ void quantize_body(const float* __restrict__ xp, int8
     const float4* x4 = reinterpret_cast<const float4*>(xp);
     uint32_t* q4 = reinterpret_cast<uint32_t*>(qp);
     size_t n4 = n >> 2;
-#pragma unroll 4
-    for (size_t i = tid; i < n4; i += stride) {
-      float4 v = __ldg(x4 + i);
-      uint32_t idx = ctr0 + (uint32_t)(i << 2);
-      int q0, q1, q2, q3;
-      quant_pair<MODE>(v.x, v.y, inv, idx, key, q0, q1);
-      quant_pair<MODE>(v.z, v.w, inv, idx + 2, key, q2, q3);
-      q4[i] = pack4(q0, q1, q2, q3);
+    // four loads in flight per thread, then the arithmetic (the FP32 source is not read again: streaming loads)
+    for (size_t i0 = tid; i0 < n4; i0 += 4 * stride) {
+      float4 vv[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (i0 + k * stride < n4) vv[k] = __ldcs(x4 + i0 + k * stride);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const size_t i = i0 + k * stride;
+        if (i >= n4) break;
+        const float4 v = vv[k];
+        uint32_t idx = ctr0 + (uint32_t)(i << 2);
+        int q0, q1, q2, q3;
+        quant_pair<MODE>(v.x, v.y, inv, idx, key, q0, q1);
+        quant_pair<MODE>(v.z, v.w, inv, idx + 2, key, q2, q3);
+        q4[i] = pack4(q0, q1, q2, q3);
+      }
     }
   } else {
     for (size_t i = tid; i < n; i += stride) qp[i] = (int8_t)quant_one<MODE>(xp[i], inv, ctr0 + (uint32_t)i, key);
@@ -239,12 +248,18 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
       const uint32_t smp = tile / tps, g0 = (tile - smp * tps) * SAMPLE_TILE_GROUPS;
       const float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(__ldg(Gp + smp)), eps));
       const size_t e0 = base + (size_t)smp * per_sample;
+      float4 vv[SAMPLE_TILE_GROUPS / EW_THREADS];  // all loads of the tile first (Y is read again by the dH quantiser: cached loads)
+#pragma unroll
+      for (uint32_t k = 0; k < SAMPLE_TILE_GROUPS / EW_THREADS; ++k) {
+        const uint32_t i = g0 + k * EW_THREADS + threadIdx.x;
+        if (i < g4) vv[k] = __ldg(reinterpret_cast<const float4*>(Y + e0 + ((size_t)i << 2)));
+      }
 #pragma unroll
       for (uint32_t k = 0; k < SAMPLE_TILE_GROUPS / EW_THREADS; ++k) {
         const uint32_t i = g0 + k * EW_THREADS + threadIdx.x;
         if (i >= g4) break;
         const size_t e = e0 + ((size_t)i << 2);
-        float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
+        float4 v = vv[k];
         v.x = __fmul_rn(v.x, r);
         v.y = __fmul_rn(v.y, r);
         v.z = __fmul_rn(v.z, r);
@@ -587,12 +602,19 @@ __device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, co
       const uint32_t smp = tile / tps, g0 = (tile - smp * tps) * SAMPLE_TILE_GROUPS;
       const float k2 = __fmul_rn(2.0f, __ldg(cp + smp));
       const size_t e0 = base + (size_t)smp * per_sample;
+      // all loads of the tile first (Y is not read again in this step: streaming loads), then the arithmetic
+      float4 vv[SAMPLE_TILE_GROUPS / EW_THREADS];
+#pragma unroll
+      for (uint32_t k = 0; k < SAMPLE_TILE_GROUPS / EW_THREADS; ++k) {
+        const uint32_t i = g0 + k * EW_THREADS + threadIdx.x;
+        if (i < g4) vv[k] = __ldcs(reinterpret_cast<const float4*>(Y + e0 + ((size_t)i << 2)));
+      }
 #pragma unroll
       for (uint32_t k = 0; k < SAMPLE_TILE_GROUPS / EW_THREADS; ++k) {
         const uint32_t i = g0 + k * EW_THREADS + threadIdx.x;
         if (i >= g4) break;
         const size_t e = e0 + ((size_t)i << 2);
-        const float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
+        const float4 v = vv[k];
         int q0, q1, q2, q3;
         quant_pair<MODE>(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, (uint32_t)e + bias, key, q0, q1);
         quant_pair<MODE>(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, (uint32_t)e + bias + 2, key, q2, q3);
