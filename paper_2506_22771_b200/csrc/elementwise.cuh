@@ -277,21 +277,29 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
     const uint32_t n4 = (uint32_t)(per_pass >> 2);
     const float* Gp = G + (uint32_t)(base / per_sample);
     SampleCursor cur(tid, stride, (uint32_t)(per_sample >> 2));
-#pragma unroll 4
-    for (uint32_t i = tid; i < n4; i += stride, cur.advance()) {
-      const size_t e = base + ((size_t)i << 2);
-      const float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(__ldg(Gp + cur.sample)), eps));
-      float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
-      v.x = __fmul_rn(v.x, r);
-      v.y = __fmul_rn(v.y, r);
-      v.z = __fmul_rn(v.z, r);
-      v.w = __fmul_rn(v.w, r);
-      if (xnext) *reinterpret_cast<float4*>(xnext + e) = v;
-      if (xq) {
-        int q0, q1, q2, q3;
-        quant_pair<MODE>(v.x, v.y, inv, (uint32_t)e + bias, key, q0, q1);
-        quant_pair<MODE>(v.z, v.w, inv, (uint32_t)e + bias + 2, key, q2, q3);
-        *reinterpret_cast<uint32_t*>(xq + e) = pack4(q0, q1, q2, q3);
+    for (uint32_t i0 = tid; i0 < n4; i0 += 4 * stride) {  // four loads in flight, then the arithmetic
+      float4 vv[4];
+#pragma unroll
+      for (uint32_t k = 0; k < 4; ++k)
+        if (i0 + k * stride < n4) vv[k] = __ldg(reinterpret_cast<const float4*>(Y + base + ((size_t)(i0 + k * stride) << 2)));
+#pragma unroll
+      for (uint32_t k = 0; k < 4; ++k, cur.advance()) {
+        const uint32_t i = i0 + k * stride;
+        if (i >= n4) break;
+        const size_t e = base + ((size_t)i << 2);
+        const float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(__ldg(Gp + cur.sample)), eps));
+        float4 v = vv[k];
+        v.x = __fmul_rn(v.x, r);
+        v.y = __fmul_rn(v.y, r);
+        v.z = __fmul_rn(v.z, r);
+        v.w = __fmul_rn(v.w, r);
+        if (xnext) *reinterpret_cast<float4*>(xnext + e) = v;
+        if (xq) {
+          int q0, q1, q2, q3;
+          quant_pair<MODE>(v.x, v.y, inv, (uint32_t)e + bias, key, q0, q1);
+          quant_pair<MODE>(v.z, v.w, inv, (uint32_t)e + bias + 2, key, q2, q3);
+          *reinterpret_cast<uint32_t*>(xq + e) = pack4(q0, q1, q2, q3);
+        }
       }
     }
   } else {
@@ -625,15 +633,23 @@ __device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, co
     const uint32_t n4 = (uint32_t)(per_pass >> 2);
     const float* cp = coef + (uint32_t)(base / per_sample);
     SampleCursor cur(tid, stride, (uint32_t)(per_sample >> 2));
-#pragma unroll 4
-    for (uint32_t i = tid; i < n4; i += stride, cur.advance()) {
-      const size_t e = base + ((size_t)i << 2);
-      const float k2 = __fmul_rn(2.0f, __ldg(cp + cur.sample));
-      const float4 v = __ldg(reinterpret_cast<const float4*>(Y + e));
-      int q0, q1, q2, q3;
-      quant_pair<MODE>(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, (uint32_t)e + bias, key, q0, q1);
-      quant_pair<MODE>(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, (uint32_t)e + bias + 2, key, q2, q3);
-      *reinterpret_cast<uint32_t*>(dHq + e) = pack4(q0, q1, q2, q3);
+    for (uint32_t i0 = tid; i0 < n4; i0 += 4 * stride) {  // four loads in flight, then the arithmetic
+      float4 vv[4];
+#pragma unroll
+      for (uint32_t k = 0; k < 4; ++k)
+        if (i0 + k * stride < n4) vv[k] = __ldcs(reinterpret_cast<const float4*>(Y + base + ((size_t)(i0 + k * stride) << 2)));
+#pragma unroll
+      for (uint32_t k = 0; k < 4; ++k, cur.advance()) {
+        const uint32_t i = i0 + k * stride;
+        if (i >= n4) break;
+        const size_t e = base + ((size_t)i << 2);
+        const float k2 = __fmul_rn(2.0f, __ldg(cp + cur.sample));
+        const float4 v = vv[k];
+        int q0, q1, q2, q3;
+        quant_pair<MODE>(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, (uint32_t)e + bias, key, q0, q1);
+        quant_pair<MODE>(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, (uint32_t)e + bias + 2, key, q2, q3);
+        *reinterpret_cast<uint32_t*>(dHq + e) = pack4(q0, q1, q2, q3);
+      }
     }
   } else {
     for (size_t i = tid; i < per_pass; i += stride) {
