@@ -123,6 +123,10 @@ typedef struct {
   float* Mom;        /* [N,K] FP32 in/out momentum buffer; needed (and touched) only if momentum != 0 */
                      /* or the optimiser is Adam (first moment)                                */
   float* Var;        /* [N,K] FP32 in/out second-moment buffer; Adam only                      */
+  int32_t ld_xq;     /* linear layers only: row pitch of Xq in bytes, 0 = K (dense).  A pitch that is a */
+  int32_t ld_dhq;    /* multiple of 128 keeps every TMA box row of the contractions aligned when K (N  */
+                     /* for dHq) is not: >= the row length, a multiple of 16; padding bytes are never  */
+                     /* read as data and never written                                                */
 } ff_layer_bufs;
 
 /* Create / destroy a context for CUDA device `device` (must be compute capability 10.x).

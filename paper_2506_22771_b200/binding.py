@@ -42,7 +42,7 @@ class ff_layer_desc(C.Structure):
 class ff_layer_bufs(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
                 ("W", "X", "Y", "G", "Xnext", "Xq", "Wq", "dHq", "absmax", "S", "rowmax", "coef",
-                 "loss", "acc_dump", "accW_dump", "Mom", "Var")]
+                 "loss", "acc_dump", "accW_dump", "Mom", "Var")] + [("ld_xq", C.c_int32), ("ld_dhq", C.c_int32)]
 
 
 FF_DP_MAX_REDUCE = 96
@@ -268,7 +268,10 @@ class LayerBuffers:
     """Torch-allocated device tensors of one layer plus the ff_layer_bufs struct pointing at them."""
 
     def __init__(self, desc: ff_layer_desc, B: int, device, dumps: bool = False, xnext: bool = True,
-                 own_x: bool = True, accw: bool = False):
+                 own_x: bool = True, accw: bool = False, pad_rows: bool = True):
+        """pad_rows: give the INT8 tensors Xq / dHq of a linear layer whose row length is not a multiple of 128 a
+        row pitch that is (the contractions' TMA box rows are then aligned); .Xq / .dHq stay [rows, K] / [rows, N]
+        views of the padded storage."""
         import torch
         st = 2 if (desc.kind in (FF_CONV3X3, FF_DWCONV3X3) and desc.stride == 2) else 1
         Rin = desc.H * desc.Wd if desc.kind != FF_LINEAR else 1                    # input rows per sample
@@ -281,9 +284,11 @@ class LayerBuffers:
         self.Y = z((rows, desc.N), torch.float32)
         self.G = z((2 * B,), torch.float32)
         self.Xnext = z((rows // 4 if desc.pool == 2 else rows, desc.N), torch.float32) if xnext else None
-        self.Xq = z((rows_in, kin), torch.int8)
+        pad = lambda n: (n + 127) // 128 * 128 if (pad_rows and desc.kind == FF_LINEAR and n % 128 and n >= 256) else n
+        self.ld_xq, self.ld_dhq = pad(kin), pad(desc.N)
+        self._Xq_store, self._dHq_store = z((rows_in, self.ld_xq), torch.int8), z((rows, self.ld_dhq), torch.int8)
+        self.Xq, self.dHq = self._Xq_store[:, :kin], self._dHq_store[:, :desc.N]
         self.Wq = z((desc.N, desc.K), torch.int8)
-        self.dHq = z((rows, desc.N), torch.int8)
         self.absmax = z((FF_ABSMAX_LEN,), torch.float32)
         self.S = z((2 * B,), torch.int64)
         self.rowmax = z((2 * B,), torch.int32)
@@ -296,7 +301,8 @@ class LayerBuffers:
         p = lambda t: t.data_ptr() if t is not None else None
         self.struct = ff_layer_bufs(p(self.W), p(self.X), p(self.Y), p(self.G), p(self.Xnext), p(self.Xq),
                                     p(self.Wq), p(self.dHq), p(self.absmax), p(self.S), p(self.rowmax),
-                                    p(self.coef), p(self.loss), p(self.acc_dump), p(self.accW_dump), p(self.Mom), p(self.Var))
+                                    p(self.coef), p(self.loss), p(self.acc_dump), p(self.accW_dump), p(self.Mom), p(self.Var),
+                                    self.ld_xq if self.ld_xq != kin else 0, self.ld_dhq if self.ld_dhq != desc.N else 0)
 
 
 class Context:

@@ -86,17 +86,27 @@ __device__ __forceinline__ void absmax_body(const float* __restrict__ xp, size_t
 // ---------------------------------------------------------------------------------------------
 // zero_S / zero_rowmax (nullable, zero_n entries): per-sample accumulators of the forward epilogue that
 // the weight quantiser clears on the side, sparing a launch.
+// INT8 tensors of dense layers may have rows padded to a wider pitch (a multiple of 128 bytes keeps every TMA box
+// row of the contractions aligned): element e of a [rows, cols] tensor then sits at e + (e / cols) * extra with
+// extra = pitch - cols.  extra = 0: dense, no division.
+struct RowPad {
+  uint32_t cols, extra;
+};
+__device__ __forceinline__ size_t padded(size_t e, RowPad rp) { return rp.extra ? e + (e / rp.cols) * rp.extra : e; }
+
 // q[i] = quantised x[i] for one tensor of n elements; ctr0 = rounding counter of element 0 (an odd one would
 // split the element pairs that share one hash differently from the unsplit tensor: scalar path then).
-template <int MODE>
+// qp = start of the output TENSOR, e0 = dense index of xp[0] in it (rows before it are skipped with their padding).
+template <int MODE, bool PAD = false>
 __device__ __forceinline__ void quantize_body(const float* __restrict__ xp, int8_t* __restrict__ qp, size_t n, float inv,
-                                              uint32_t ctr0, RoundKey key) {
-  const bool vec = ((n & 3) == 0) && ((((uintptr_t)xp) & 15) == 0) && ((((uintptr_t)qp) & 3) == 0) && !(ctr0 & 1u);
+                                              uint32_t ctr0, RoundKey key, size_t e0 = 0, RowPad rp = RowPad{0u, 0u}) {
+  if (!PAD) rp = RowPad{0u, 0u};  // compiled without the row arithmetic
+  const bool vec = ((n & 3) == 0) && ((e0 & 3) == 0) && ((((uintptr_t)xp) & 15) == 0) && ((((uintptr_t)qp) & 3) == 0) &&
+                   !(ctr0 & 1u) && ((rp.cols | rp.extra) & 3u) == 0;
   size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   size_t stride = (size_t)gridDim.x * blockDim.x;
   if (vec) {
     const float4* x4 = reinterpret_cast<const float4*>(xp);
-    uint32_t* q4 = reinterpret_cast<uint32_t*>(qp);
     size_t n4 = n >> 2;
     // four loads in flight per thread, then the arithmetic (the FP32 source is not read again: streaming loads)
     for (size_t i0 = tid; i0 < n4; i0 += 4 * stride) {
@@ -113,11 +123,12 @@ __device__ __forceinline__ void quantize_body(const float* __restrict__ xp, int8
         int q0, q1, q2, q3;
         quant_pair<MODE>(v.x, v.y, inv, idx, key, q0, q1);
         quant_pair<MODE>(v.z, v.w, inv, idx + 2, key, q2, q3);
-        q4[i] = pack4(q0, q1, q2, q3);
+        *reinterpret_cast<uint32_t*>(qp + (PAD ? padded(e0 + (i << 2), rp) : e0 + (i << 2))) = pack4(q0, q1, q2, q3);
       }
     }
   } else {
-    for (size_t i = tid; i < n; i += stride) qp[i] = (int8_t)quant_one<MODE>(xp[i], inv, ctr0 + (uint32_t)i, key);
+    for (size_t i = tid; i < n; i += stride)
+      qp[PAD ? padded(e0 + i, rp) : e0 + i] = (int8_t)quant_one<MODE>(xp[i], inv, ctr0 + (uint32_t)i, key);
   }
 }
 
@@ -126,7 +137,7 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __res
                                                               size_t n_per_pass, const float* __restrict__ a,
                                                               KeySpec ks, unsigned long long* __restrict__ zero_S = nullptr,
                                                               int32_t* __restrict__ zero_rowmax = nullptr, int zero_n = 0,
-                                                              uint2 ctr_bias = uint2{0u, 0u}) {
+                                                              uint2 ctr_bias = uint2{0u, 0u}, RowPad rp = RowPad{0u, 0u}) {
   const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
   const uint32_t bias = blockIdx.y ? ctr_bias.y : ctr_bias.x;
   if (zero_S && blockIdx.y == 0)
@@ -135,7 +146,10 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_kernel(const float* __res
       zero_rowmax[i] = 0;
     }
   const size_t base = (size_t)blockIdx.y * n_per_pass;
-  quantize_body<MODE>(x + base, q + base, n_per_pass, inv_of(a[blockIdx.y]), (uint32_t)base + bias, key);
+  if (rp.extra)
+    quantize_body<MODE, true>(x + base, q, n_per_pass, inv_of(a[blockIdx.y]), (uint32_t)base + bias, key, base, rp);
+  else
+    quantize_body<MODE, false>(x + base, q, n_per_pass, inv_of(a[blockIdx.y]), (uint32_t)base + bias, key, base);
 }
 
 // One launch for a table of tensors (blockIdx.y = tensor): the weights of every layer and the two sets of
@@ -148,12 +162,15 @@ struct QuantJobs {
   const float* a[MT_MAX];          // address of the tensor's range
   unsigned long long s1[MT_MAX];   // step-independent part of the rounding key
   uint32_t ctr0[MT_MAX];           // counter of the tensor's first element
+  unsigned long long e0[MT_MAX];   // dense index of x[t][0] inside the output tensor q[t]
+  RowPad pad[MT_MAX];              // row padding of the output tensor
   uint8_t stochastic[MT_MAX];
   unsigned long long* zero_S[FF_MAX_LATER + 1];
   int32_t* zero_rowmax[FF_MAX_LATER + 1];
   int n_zero, zero_n;              // layers whose accumulators are cleared, entries each
   const StepState* ss;
 };
+template <bool PAD>  // PAD: some output tensor has padded rows (compiled apart so that the dense form stays lean)
 __global__ void __launch_bounds__(EW_THREADS) quantize_multi_kernel(const QuantJobs jobs) {
   const int t = blockIdx.y;
   if (t < jobs.n_zero)
@@ -163,10 +180,11 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_multi_kernel(const QuantJ
     }
   const float inv = inv_of(*jobs.a[t]);
   if (jobs.stochastic[t])
-    quantize_body<ROUND_STOCHASTIC>(jobs.x[t], jobs.q[t], (size_t)jobs.n[t], inv, jobs.ctr0[t],
-                                    derive_key(KeySpec{jobs.s1[t], jobs.ss}));
+    quantize_body<ROUND_STOCHASTIC, PAD>(jobs.x[t], jobs.q[t], (size_t)jobs.n[t], inv, jobs.ctr0[t],
+                                         derive_key(KeySpec{jobs.s1[t], jobs.ss}), (size_t)jobs.e0[t], jobs.pad[t]);
   else
-    quantize_body<ROUND_NEAREST>(jobs.x[t], jobs.q[t], (size_t)jobs.n[t], inv, jobs.ctr0[t], RoundKey{0u, 0u});
+    quantize_body<ROUND_NEAREST, PAD>(jobs.x[t], jobs.q[t], (size_t)jobs.n[t], inv, jobs.ctr0[t], RoundKey{0u, 0u},
+                                      (size_t)jobs.e0[t], jobs.pad[t]);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -225,12 +243,14 @@ struct SampleCursor {
 // and / or quantised straight to the next layer's INT8 input (xq, nullable) with per-pass range
 // a[p].  per_sample = R*N elements per sample; per_pass = B*per_sample.   grid = (blocks, 2)
 // ---------------------------------------------------------------------------------------------
-template <int MODE>
+template <int MODE, bool PAD = false>
 __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __restrict__ Y, const float* __restrict__ G,
                                                                float tau, float eps, size_t per_sample,
                                                                size_t per_pass, float* __restrict__ xnext,
                                                                int8_t* __restrict__ xq, const float* __restrict__ a,
-                                                               KeySpec ks, uint2 ctr_bias = uint2{0u, 0u}) {
+                                                               KeySpec ks, uint2 ctr_bias = uint2{0u, 0u},
+                                                               RowPad rp = RowPad{0u, 0u}) {
+  // rp: row padding of xq (dense layers only: a row is a sample, so sample index * extra is the shift)
   const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
   const uint32_t bias = blockIdx.y ? ctr_bias.y : ctr_bias.x;
   const size_t base = (size_t)blockIdx.y * per_pass;
@@ -269,13 +289,15 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
           int q0, q1, q2, q3;
           quant_pair<MODE>(v.x, v.y, inv, (uint32_t)e + bias, key, q0, q1);
           quant_pair<MODE>(v.z, v.w, inv, (uint32_t)e + bias + 2, key, q2, q3);
-          *reinterpret_cast<uint32_t*>(xq + e) = pack4(q0, q1, q2, q3);
+          *reinterpret_cast<uint32_t*>(xq + e + (PAD ? (size_t)(blockIdx.y * n_samples + smp) * rp.extra : (size_t)0)) =
+              pack4(q0, q1, q2, q3);
         }
       }
     }
   } else if (vec) {
     const uint32_t n4 = (uint32_t)(per_pass >> 2);
     const float* Gp = G + (uint32_t)(base / per_sample);
+    const uint32_t pass_row0 = (uint32_t)(base / per_sample);
     SampleCursor cur(tid, stride, (uint32_t)(per_sample >> 2));
     for (uint32_t i0 = tid; i0 < n4; i0 += 4 * stride) {  // four loads in flight, then the arithmetic
       float4 vv[4];
@@ -298,7 +320,8 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
           int q0, q1, q2, q3;
           quant_pair<MODE>(v.x, v.y, inv, (uint32_t)e + bias, key, q0, q1);
           quant_pair<MODE>(v.z, v.w, inv, (uint32_t)e + bias + 2, key, q2, q3);
-          *reinterpret_cast<uint32_t*>(xq + e) = pack4(q0, q1, q2, q3);
+          *reinterpret_cast<uint32_t*>(xq + e + (PAD ? (size_t)(pass_row0 + cur.sample) * rp.extra : (size_t)0)) =
+                pack4(q0, q1, q2, q3);
         }
       }
     }
@@ -309,7 +332,7 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
       float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(g), eps));
       float v = __fmul_rn(Y[e], r);
       if (xnext) xnext[e] = v;
-      if (xq) xq[e] = (int8_t)quant_one<MODE>(v, inv, (uint32_t)e + bias, key);
+      if (xq) xq[PAD ? padded(e, rp) : e] = (int8_t)quant_one<MODE>(v, inv, (uint32_t)e + bias, key);
     }
   }
 }
@@ -559,17 +582,21 @@ __global__ void __launch_bounds__(EW_THREADS) classify_kernel(LaterLayers layers
 // ---------------------------------------------------------------------------------------------
 // dHq = clip(round((2*coef_m * y) * 127/a_dh[p])).  grid = (blocks, 2)
 // ---------------------------------------------------------------------------------------------
-template <int MODE>
+template <int MODE, bool PAD = false>
 __device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, const float* __restrict__ coef,
                                                  const float* __restrict__ absmax, size_t per_sample, size_t per_pass,
-                                                 int8_t* __restrict__ dHq, RoundKey key, int pass, uint32_t bias);
+                                                 int8_t* __restrict__ dHq, RoundKey key, int pass, uint32_t bias,
+                                                 RowPad rp = RowPad{0u, 0u});
 template <int MODE>
 __global__ void __launch_bounds__(EW_THREADS) dh_quantize_kernel(const float* __restrict__ Y, const float* __restrict__ coef,
                                                                  const float* __restrict__ absmax, size_t per_sample,
                                                                  size_t per_pass, int8_t* __restrict__ dHq, KeySpec ks,
-                                                                 uint2 ctr_bias = uint2{0u, 0u}) {
+                                                                 uint2 ctr_bias = uint2{0u, 0u}, RowPad rp = RowPad{0u, 0u}) {
   const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
-  dh_quantize_body<MODE>(Y, coef, absmax, per_sample, per_pass, dHq, key, blockIdx.y, blockIdx.y ? ctr_bias.y : ctr_bias.x);
+  if (rp.extra)
+    dh_quantize_body<MODE, true>(Y, coef, absmax, per_sample, per_pass, dHq, key, blockIdx.y, blockIdx.y ? ctr_bias.y : ctr_bias.x, rp);
+  else
+    dh_quantize_body<MODE, false>(Y, coef, absmax, per_sample, per_pass, dHq, key, blockIdx.y, blockIdx.y ? ctr_bias.y : ctr_bias.x);
 }
 // Every layer of a step in one launch: blockIdx.y = 2*layer + set.
 struct DhJobs {
@@ -580,22 +607,25 @@ struct DhJobs {
   int8_t* dHq[FF_MAX_LATER + 1];
   unsigned long long s1[FF_MAX_LATER + 1];
   uint8_t stochastic[FF_MAX_LATER + 1];
+  RowPad pad[FF_MAX_LATER + 1];   // row padding of dHq (dense layers)
   const StepState* ss;
 };
+template <bool PAD>
 __global__ void __launch_bounds__(EW_THREADS) dh_quantize_multi_kernel(const DhJobs jobs, int B) {
   const int l = blockIdx.y >> 1, pass = blockIdx.y & 1;
   const size_t per_sample = (size_t)jobs.per_sample[l], per_pass = per_sample * B;
   if (jobs.stochastic[l])
-    dh_quantize_body<ROUND_STOCHASTIC>(jobs.Y[l], jobs.coef[l], jobs.absmax[l], per_sample, per_pass, jobs.dHq[l],
-                                       derive_key(KeySpec{jobs.s1[l], jobs.ss}), pass, 0u);
+    dh_quantize_body<ROUND_STOCHASTIC, PAD>(jobs.Y[l], jobs.coef[l], jobs.absmax[l], per_sample, per_pass, jobs.dHq[l],
+                                            derive_key(KeySpec{jobs.s1[l], jobs.ss}), pass, 0u, jobs.pad[l]);
   else
-    dh_quantize_body<ROUND_NEAREST>(jobs.Y[l], jobs.coef[l], jobs.absmax[l], per_sample, per_pass, jobs.dHq[l], RoundKey{0u, 0u},
-                                    pass, 0u);
+    dh_quantize_body<ROUND_NEAREST, PAD>(jobs.Y[l], jobs.coef[l], jobs.absmax[l], per_sample, per_pass, jobs.dHq[l],
+                                         RoundKey{0u, 0u}, pass, 0u, jobs.pad[l]);
 }
-template <int MODE>
+
+template <int MODE, bool PAD>
 __device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, const float* __restrict__ coef,
                                                  const float* __restrict__ absmax, size_t per_sample, size_t per_pass,
-                                                 int8_t* __restrict__ dHq, RoundKey key, int pass, uint32_t bias) {
+                                                 int8_t* __restrict__ dHq, RoundKey key, int pass, uint32_t bias, RowPad rp) {
   const size_t base = (size_t)pass * per_pass;
   const float inv = inv_of(absmax[3 + pass]);
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)dHq) & 3) == 0);
@@ -626,12 +656,14 @@ __device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, co
         int q0, q1, q2, q3;
         quant_pair<MODE>(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, (uint32_t)e + bias, key, q0, q1);
         quant_pair<MODE>(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, (uint32_t)e + bias + 2, key, q2, q3);
-        *reinterpret_cast<uint32_t*>(dHq + e) = pack4(q0, q1, q2, q3);
+        *reinterpret_cast<uint32_t*>(dHq + e + (PAD ? (size_t)(pass * n_samples + smp) * rp.extra : (size_t)0)) =
+            pack4(q0, q1, q2, q3);
       }
     }
   } else if (vec) {
     const uint32_t n4 = (uint32_t)(per_pass >> 2);
     const float* cp = coef + (uint32_t)(base / per_sample);
+    const uint32_t pass_row0 = (uint32_t)(base / per_sample);
     SampleCursor cur(tid, stride, (uint32_t)(per_sample >> 2));
     for (uint32_t i0 = tid; i0 < n4; i0 += 4 * stride) {  // four loads in flight, then the arithmetic
       float4 vv[4];
@@ -648,14 +680,15 @@ __device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, co
         int q0, q1, q2, q3;
         quant_pair<MODE>(__fmul_rn(k2, v.x), __fmul_rn(k2, v.y), inv, (uint32_t)e + bias, key, q0, q1);
         quant_pair<MODE>(__fmul_rn(k2, v.z), __fmul_rn(k2, v.w), inv, (uint32_t)e + bias + 2, key, q2, q3);
-        *reinterpret_cast<uint32_t*>(dHq + e) = pack4(q0, q1, q2, q3);
+        *reinterpret_cast<uint32_t*>(dHq + e + (PAD ? (size_t)(pass_row0 + cur.sample) * rp.extra : (size_t)0)) =
+              pack4(q0, q1, q2, q3);
       }
     }
   } else {
     for (size_t i = tid; i < per_pass; i += stride) {
       size_t e = base + i;
       float k2 = __fmul_rn(2.0f, coef[(uint32_t)e / (uint32_t)per_sample]);
-      dHq[e] = (int8_t)quant_one<MODE>(__fmul_rn(k2, Y[e]), inv, (uint32_t)e + bias, key);
+      dHq[PAD ? padded(e, rp) : e] = (int8_t)quant_one<MODE>(__fmul_rn(k2, Y[e]), inv, (uint32_t)e + bias, key);
     }
   }
 }

@@ -181,6 +181,15 @@ ff_status check_bufs(ff_ctx* ctx, const ff_layer_bufs* b, bool need_x) {
   return FF_OK;
 }
 
+// Row pitches of the INT8 tensors: linear layers only, at least the row length, multiples of 16 bytes.
+ff_status check_pitches(ff_ctx* ctx, const ff_layer_desc* L, const ff_layer_bufs* b) {
+  if (!b->ld_xq && !b->ld_dhq) return FF_OK;
+  if (L->kind != FF_LINEAR) return fail(ctx, FF_ERR_ARG, "row pitches are for linear layers only");
+  if (b->ld_xq && (b->ld_xq < L->K || b->ld_xq % 16)) return fail(ctx, FF_ERR_ARG, "ld_xq must be >= K and a multiple of 16");
+  if (b->ld_dhq && (b->ld_dhq < L->N || b->ld_dhq % 16)) return fail(ctx, FF_ERR_ARG, "ld_dhq must be >= N and a multiple of 16");
+  return FF_OK;
+}
+
 ff_status check_ctx(ff_ctx* ctx) {
   if (!ctx) return FF_ERR_ARG;
   if (!ctx->workspace) return fail(ctx, FF_ERR_WORKSPACE, "no workspace set");
@@ -241,9 +250,12 @@ ff_status launch_simt(ff_ctx* ctx, LA la, LB lb, int out_rows, int out_cols, int
   return FF_OK;
 }
 
-inline DenseView dense(const int8_t* p, int rows, int cols) {
-  return DenseView{p, rows, cols, (cols % 8 == 0) && ((reinterpret_cast<uintptr_t>(p) & 7) == 0)};
+inline DenseView dense(const int8_t* p, int rows, int cols, int ld = 0) {
+  if (!ld) ld = cols;
+  return DenseView{p, rows, cols, ld, (cols % 8 == 0) && (ld % 8 == 0) && ((reinterpret_cast<uintptr_t>(p) & 7) == 0)};
 }
+// row padding of a dense layer's INT8 tensor with `cols` values per row and a pitch of ld bytes (0: none)
+inline RowPad row_pad(int cols, int ld) { return RowPad{(uint32_t)cols, ld ? (uint32_t)(ld - cols) : 0u}; }
 inline Im2colView im2col(const int8_t* p, const ff_layer_desc& L, int samples) {
   return Im2colView{p, samples * tc_out_h(L) * tc_out_w(L), 9 * L.Cin, L.H, L.Wd, L.Cin, tc_out_h(L), tc_out_w(L),
                     tc_conv_stride(L), (L.Cin % 8 == 0) && ((reinterpret_cast<uintptr_t>(p) & 7) == 0)};
@@ -455,7 +467,7 @@ ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
   }
   ForwardEpilogue epi{b.Y, b.acc_dump, reinterpret_cast<unsigned long long*>(b.S), b.rowmax, b.absmax, rows, L.N, B * R, R};
   if (L.kind != FF_CONV3X3)
-    return launch_simt<DenseView, DenseView, false, 1>(ctx, dense(b.Xq, rows, L.K), dense(b.Wq, L.N, L.K), rows, L.N, L.K, epi, st);
+    return launch_simt<DenseView, DenseView, false, 1>(ctx, dense(b.Xq, rows, L.K, b.ld_xq), dense(b.Wq, L.N, L.K), rows, L.N, L.K, epi, st);
   return launch_simt<Im2colView, DenseView, false, 1>(ctx, im2col(b.Xq, L, 2 * B), dense(b.Wq, L.N, L.K), rows, L.N, L.K, epi, st);
 }
 
@@ -536,7 +548,8 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
       int32_t* slabs = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
       ProfScope prof(ctx, FF_K_UPD_GEMM, st);
       int used = 0;
-      ff_status s = tc_dense_update_slab(ctx->tc, b.dHq, L.N, b.Xq, L.K, B * R, slabs, splits, &used, status_ptr(ctx), st);
+      ff_status s = tc_dense_update_slab(ctx->tc, b.dHq, L.N, b.Xq, L.K, B * R, slabs, splits, &used, status_ptr(ctx), st,
+                                         b.ld_dhq, b.ld_xq);
       if (s != FF_OK) return fail(ctx, s, "tensor-core weight-gradient launch failed: %s", ctx->tc.err);
       ctx->launches++;
       const bool was = ctx->profiling;
@@ -551,7 +564,7 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     int used = 0;
     // accumulate only: one unsplit contraction whose single slab [2][N][K] is accW_dump itself
     ff_status s = ctx->accumulate_only ? tc_dense_update_slab(ctx->tc, b.dHq, L.N, b.Xq, L.K, B * R, b.accW_dump, 1, &used,
-                                                              status_ptr(ctx), st)
+                                                              status_ptr(ctx), st, b.ld_dhq, b.ld_xq)
                                        : tc_update(ctx->tc, L, b, B * R, status_ptr(ctx), st);
     if (s != FF_OK) return fail(ctx, s, "tensor-core weight-gradient launch failed: %s", ctx->tc.err);
     ctx->launches++;
@@ -590,7 +603,7 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
       const bool was = ctx->profiling;
       ctx->profiling = false;  // one event pair around both launches
       if (L.kind != FF_CONV3X3)
-        s = launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st, splits);
+        s = launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N, b.ld_dhq), dense(b.Xq, rows, L.K, b.ld_xq), L.N, L.K, clen, epi, st, splits);
       else
         s = launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st, splits);
       if (s == FF_OK) s = launch_slab_update(ctx, slabs, simt_split_count(clen, splits), L, b, st);
@@ -601,12 +614,12 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
   if (ctx->accumulate_only) {
     SlabEpilogue epi{b.accW_dump, L.N, L.K};
     if (L.kind != FF_CONV3X3)
-      return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st);
+      return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N, b.ld_dhq), dense(b.Xq, rows, L.K, b.ld_xq), L.N, L.K, clen, epi, st);
     return launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st);
   }
   UpdateEpilogue epi{b.W, b.accW_dump, b.absmax, L.lr, L.N, L.K, L.momentum != 0.0f ? b.Mom : nullptr, L.momentum};
   if (L.kind != FF_CONV3X3)
-    return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N), dense(b.Xq, rows, L.K), L.N, L.K, clen, epi, st);
+    return launch_simt<DenseView, DenseView, true, 2>(ctx, dense(b.dHq, rows, L.N, b.ld_dhq), dense(b.Xq, rows, L.K, b.ld_xq), L.N, L.K, clen, epi, st);
   return launch_simt<DenseView, Im2colView, true, 2>(ctx, dense(b.dHq, rows, L.N), im2col(b.Xq, L, 2 * B), L.N, L.K, clen, epi, st);
 }
 
@@ -662,10 +675,10 @@ ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
     const uint2 bias = ctr_bias(ctx, per_sample, B);
     if (L.round_x == FF_ROUND_NEAREST_EVEN)
       quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, key, nullptr,
-                                                                 nullptr, 0, bias);
+                                                                 nullptr, 0, bias, row_pad(L.K, b.ld_xq));
     else
       quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.X, b.Xq, per_pass, b.absmax + FF_A_X_POS, key, nullptr,
-                                                                    nullptr, 0, bias);
+                                                                    nullptr, 0, bias, row_pad(L.K, b.ld_xq));
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -674,8 +687,9 @@ ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
 // Normalised output of layer `L` as FP32 (b.Xnext, if non-NULL) and / or as the INT8 input of the
 // next layer (xq_next, nullable; rounding keyed by the next layer).
 ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, int8_t* xq_next,
-                           const ff_layer_desc* next, cudaStream_t st) {
+                           const ff_layer_desc* next, cudaStream_t st, int ld_next = 0) {
   if (!b.Xnext && !xq_next) return FF_OK;
+  if (ld_next && L.pool == 2) return fail(ctx, FF_ERR_ARG, "a pooled output cannot feed a layer with a padded Xq");
   const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
   const size_t per_pass = per_sample * B;
   const KeySpec key = next ? make_key_spec(next->seed, ROLE_X, next->index, step_ptr(ctx)) : KeySpec{0ull, step_ptr(ctx)};
@@ -706,12 +720,21 @@ ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
     ProfScope prof(ctx, FF_K_NORMALIZE, st);
     const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
     const uint2 bias = ctr_bias(ctx, per_sample, B);
-    if (!next || next->round_x == FF_ROUND_NEAREST_EVEN)
-      normalize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
-                                                                  xq_next, b.absmax + FF_A_XNEXT_POS, key, bias);
+    const bool nearest = !next || next->round_x == FF_ROUND_NEAREST_EVEN;
+    const RowPad rp = row_pad((int)per_sample, ld_next);
+    const float* a = b.absmax + FF_A_XNEXT_POS;
+    if (nearest && !rp.extra)
+      normalize_kernel<ROUND_NEAREST, false><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
+                                                                         xq_next, a, key, bias);
+    else if (nearest)
+      normalize_kernel<ROUND_NEAREST, true><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
+                                                                        xq_next, a, key, bias, rp);
+    else if (!rp.extra)
+      normalize_kernel<ROUND_STOCHASTIC, false><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
+                                                                            xq_next, a, key, bias);
     else
-      normalize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
-                                                                     xq_next, b.absmax + FF_A_XNEXT_POS, key, bias);
+      normalize_kernel<ROUND_STOCHASTIC, true><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
+                                                                           xq_next, a, key, bias, rp);
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -745,10 +768,11 @@ ff_status loss_grad_impl(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
     const KeySpec key = make_key_spec(L.seed, ROLE_DH, L.index, step_ptr(ctx));
     const uint2 bias = ctr_bias(ctx, per_sample, B);
     if (L.round_dh == FF_ROUND_NEAREST_EVEN)
-      dh_quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key, bias);
+      dh_quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key, bias,
+                                                                    row_pad(L.N, b.ld_dhq));
     else
       dh_quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.Y, b.coef, b.absmax, per_sample, per_pass, b.dHq, key,
-                                                                       bias);
+                                                                       bias, row_pad(L.N, b.ld_dhq));
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -760,6 +784,7 @@ ff_status check_layer_list(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
   for (int l = 0; l < n_layers; ++l) {
     if ((s = check_layer(ctx, &layers[l], B)) != FF_OK) return s;
     if ((s = check_bufs(ctx, &bufs[l], l == 0)) != FF_OK) return s;
+    if ((s = check_pitches(ctx, &layers[l], &bufs[l])) != FF_OK) return s;
     if (l > 0 && !bufs[l].X) {
       const ff_layer_desc &p = layers[l - 1], &c = layers[l];
       if (next_values_per_sample(p) != (long long)in_rows_per_sample(c) * in_features(c))
@@ -785,7 +810,8 @@ ff_status quantize_inputs_and_weights(ff_ctx* ctx, const ff_layer_desc* layers, 
   const uint2 bias0 = ctr_bias(ctx, per_sample0, B);
   for (int p = 0; p < 2; ++p, ++t) {
     aj.x[t] = bufs[0].X + p * per_pass0, aj.n[t] = per_pass0, aj.out[t] = bufs[0].absmax + FF_A_X_POS + p;
-    qj.x[t] = aj.x[t], qj.q[t] = bufs[0].Xq + p * per_pass0, qj.n[t] = per_pass0, qj.a[t] = aj.out[t];
+    qj.x[t] = aj.x[t], qj.q[t] = bufs[0].Xq, qj.e0[t] = p * per_pass0, qj.n[t] = per_pass0, qj.a[t] = aj.out[t];
+    qj.pad[t] = row_pad(L0.K, bufs[0].ld_xq);
     qj.s1[t] = make_key_spec(L0.seed, ROLE_X, L0.index, nullptr).s1;
     qj.ctr0[t] = (uint32_t)(p * per_pass0) + (p ? bias0.y : bias0.x);
     qj.stochastic[t] = L0.round_x != FF_ROUND_NEAREST_EVEN;
@@ -797,6 +823,7 @@ ff_status quantize_inputs_and_weights(ff_ctx* ctx, const ff_layer_desc* layers, 
     qj.x[t] = bufs[l].W, qj.q[t] = bufs[l].Wq, qj.n[t] = nW, qj.a[t] = aj.out[t];
     qj.s1[t] = make_key_spec(layers[l].seed, ROLE_W, layers[l].index, nullptr).s1;
     qj.ctr0[t] = 0u;
+    qj.e0[t] = 0, qj.pad[t] = RowPad{0u, 0u};
     qj.stochastic[t] = layers[l].round_w != FF_ROUND_NEAREST_EVEN;
     qj.zero_S[l] = reinterpret_cast<unsigned long long*>(bufs[l].S);
     qj.zero_rowmax[l] = bufs[l].rowmax;
@@ -811,7 +838,10 @@ ff_status quantize_inputs_and_weights(ff_ctx* ctx, const ff_layer_desc* layers, 
   FF_LAUNCH_CHECK(ctx);
   {
     ProfScope prof(ctx, FF_K_QUANTIZE, st);
-    quantize_multi_kernel<<<grid, EW_THREADS, 0, st>>>(qj);
+    if (bufs[0].ld_xq)
+      quantize_multi_kernel<true><<<grid, EW_THREADS, 0, st>>>(qj);
+    else
+      quantize_multi_kernel<false><<<grid, EW_THREADS, 0, st>>>(qj);
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -828,7 +858,7 @@ ff_status forward_all(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_b
     if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st, true)) != FF_OK)
       return s;
     if ((s = normalize_output(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].Xq : nullptr,
-                              feeds_next ? &layers[l + 1] : nullptr, st)) != FF_OK)
+                              feeds_next ? &layers[l + 1] : nullptr, st, feeds_next ? bufs[l + 1].ld_xq : 0)) != FF_OK)
       return s;
   }
   return FF_OK;
@@ -854,6 +884,7 @@ ff_status train_step_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_lay
     dj.per_sample[l] = (unsigned long long)rows_per_sample(layers[l]) * layers[l].N;
     dj.s1[l] = make_key_spec(layers[l].seed, ROLE_DH, layers[l].index, nullptr).s1;
     dj.stochastic[l] = layers[l].round_dh != FF_ROUND_NEAREST_EVEN;
+    dj.pad[l] = row_pad(layers[l].N, bufs[l].ld_dhq);
     if (dj.per_sample[l] * B > largest) largest = dj.per_sample[l] * B;
   }
   dj.ss = step_ptr(ctx);
@@ -867,7 +898,13 @@ ff_status train_step_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_lay
   FF_LAUNCH_CHECK(ctx);
   {
     ProfScope prof(ctx, FF_K_DH_QUANTIZE, st);
-    dh_quantize_multi_kernel<<<dim3(ew_blocks(ctx, largest / 4 + 1), 2 * n_layers), EW_THREADS, 0, st>>>(dj, B);
+    bool any_pad = false;
+    for (int l = 0; l < n_layers; ++l) any_pad = any_pad || bufs[l].ld_dhq != 0;
+    const dim3 grid(ew_blocks(ctx, largest / 4 + 1), 2 * n_layers);
+    if (any_pad)
+      dh_quantize_multi_kernel<true><<<grid, EW_THREADS, 0, st>>>(dj, B);
+    else
+      dh_quantize_multi_kernel<false><<<grid, EW_THREADS, 0, st>>>(dj, B);
   }
   FF_LAUNCH_CHECK(ctx);
   for (int l = 0; l < n_layers; ++l)
@@ -898,7 +935,7 @@ ff_status dp_phase_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
     if (l == 0)
       s = quantize_input(ctx, layers[0], bufs[0], B, st, false, true);
     else
-      s = normalize_output(ctx, layers[l - 1], bufs[l - 1], B, bufs[l].Xq, &layers[l], st);
+      s = normalize_output(ctx, layers[l - 1], bufs[l - 1], B, bufs[l].Xq, &layers[l], st, bufs[l].ld_xq);
     if (s != FF_OK) return s;
     const bool feeds_next = l + 1 < n;
     if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st)) != FF_OK)
@@ -1150,6 +1187,7 @@ ff_status ff_layer_forward(ff_ctx* ctx, const ff_layer_desc* layer, const ff_lay
   if (s != FF_OK) return s;
   if ((s = check_layer(ctx, layer, B)) != FF_OK) return s;
   if ((s = check_bufs(ctx, bufs, true)) != FF_OK) return s;
+  if ((s = check_pitches(ctx, layer, bufs)) != FF_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
   FF_CUDA(ctx, cudaMemsetAsync(bufs->absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
@@ -1166,6 +1204,7 @@ ff_status ff_layer_loss_grad(ff_ctx* ctx, const ff_layer_desc* layer, const ff_l
   if (s != FF_OK) return s;
   if ((s = check_layer(ctx, layer, B)) != FF_OK) return s;
   if ((s = check_bufs(ctx, bufs, false)) != FF_OK) return s;
+  if ((s = check_pitches(ctx, layer, bufs)) != FF_OK) return s;
   if (n_later < 0 || n_later > FF_MAX_LATER) return fail(ctx, FF_ERR_ARG, "n_later out of range");
   if (n_later > 0 && (!G_later || !theta_later)) return fail(ctx, FF_ERR_ARG, "G_later / theta_later is NULL");
   for (int j = 0; j < n_later; ++j)
@@ -1181,6 +1220,7 @@ ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_laye
   if (s != FF_OK) return s;
   if ((s = check_layer(ctx, layer, B)) != FF_OK) return s;
   if ((s = check_bufs(ctx, bufs, false)) != FF_OK) return s;
+  if ((s = check_pitches(ctx, layer, bufs)) != FF_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
   return run_update_gemm(ctx, *layer, *bufs, B, st);

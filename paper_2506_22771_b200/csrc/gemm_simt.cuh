@@ -19,16 +19,17 @@ constexpr int SG_PITCH = SG_BK + 4;  // bytes per smem row (36 = 9 words)
 struct DenseView {
   const int8_t* p;
   int rows, cols;
-  bool vec8;  // cols % 8 == 0 and p 8-byte aligned
+  int ld;     // bytes from one row to the next (>= cols)
+  bool vec8;  // cols % 8 == 0, ld % 8 == 0 and p 8-byte aligned
   __device__ __forceinline__ void load8(int row, int col0, int8_t* out) const {
     if (row < rows && vec8 && col0 + 8 <= cols) {
-      *reinterpret_cast<uint2*>(out) = __ldg(reinterpret_cast<const uint2*>(p + (size_t)row * cols + col0));
+      *reinterpret_cast<uint2*>(out) = __ldg(reinterpret_cast<const uint2*>(p + (size_t)row * ld + col0));
       return;
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       int c = col0 + i;
-      out[i] = (row < rows && c < cols) ? p[(size_t)row * cols + c] : (int8_t)0;
+      out[i] = (row < rows && c < cols) ? p[(size_t)row * ld + c] : (int8_t)0;
     }
   }
 };

@@ -908,10 +908,12 @@ inline ff_status tc_encode(TcState& t, CUtensorMap* tm, const int8_t* base, cuui
 
 // INT8 row-major matrix [rows, cols] viewed as `passes` stacked matrices of rows_per_pass rows (passes = 0:
 // a plain 2-D map); box = box_cols x box_rows (x 1), swizzle = box_cols bytes (128 or 64), zero fill outside.
+// pitch: bytes from one row to the next (0: rows are contiguous)
 inline ff_status tc_make_map(TcState& t, CUtensorMap* tm, const int8_t* base, uint64_t cols, uint64_t rows_per_pass, uint64_t passes,
-                             uint32_t box_cols, uint32_t box_rows) {
+                             uint32_t box_cols, uint32_t box_rows, uint64_t pitch = 0) {
+  if (!pitch) pitch = cols;
   cuuint64_t dims[3] = {cols, rows_per_pass, passes ? passes : 1};
-  cuuint64_t strides[2] = {cols, cols * rows_per_pass};
+  cuuint64_t strides[2] = {pitch, pitch * rows_per_pass};
   cuuint32_t box[3] = {box_cols, box_rows, 1};
   return tc_encode(t, tm, base, passes > 0 ? 3 : 2, dims, strides, box, (int)box_cols);
 }
@@ -1125,7 +1127,7 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   const CUtensorMap* typ = p.y_tma ? &ty : nullptr;
   if (!conv) {
     p.kblocks = cdiv(K, 128);
-    if ((s = tc_make_map(t, &ta, A, K, M, 0, 128, TC_BM)) != FF_OK) return s;
+    if ((s = tc_make_map(t, &ta, A, K, M, 0, 128, TC_BM, xi ? 0 : (uint64_t)b.ld_xq)) != FF_OK) return s;
     if ((s = tc_make_map(t, &tb, Bw, K, L.N, 0, 128, TC_BN / ncta)) != FF_OK) return s;
     return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st, typ);
   }
@@ -1162,8 +1164,8 @@ inline ff_status tc_update(TcState& t, const ff_layer_desc& L, const ff_layer_bu
   p.lr = L.lr;
   p.mom = L.momentum != 0.0f ? b.Mom : nullptr;
   p.mu = L.momentum;
-  if ((s = tc_make_map(t, &ta, b.dHq, L.N, B, 2, 128, 128)) != FF_OK) return s;
-  if ((s = tc_make_map(t, &tb, b.Xq, L.K, B, 2, 128, 128)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &ta, b.dHq, L.N, B, 2, 128, 128, (uint64_t)b.ld_dhq)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &tb, b.Xq, L.K, B, 2, 128, 128, (uint64_t)b.ld_xq)) != FF_OK) return s;
   return tc_launch<TC_MODE_UPD, true, 128>(t, tc_pick_ncta(t, L.N, L.K), ta, tb, p, st);
 }
 
@@ -1211,7 +1213,8 @@ inline int tc_dense_slab_splits(int N, int kcols, long long rows_per_pass, int s
   return splits < 1 ? 1 : (int)splits;
 }
 inline ff_status tc_dense_update_slab(TcState& t, const int8_t* dHq, int N, const int8_t* xi, int kcols, int rows_per_pass,
-                                      int32_t* slabs, int splits, int* splits_out, uint32_t* status, cudaStream_t st) {
+                                      int32_t* slabs, int splits, int* splits_out, uint32_t* status, cudaStream_t st,
+                                      int ld_dhq = 0, int ld_xi = 0) {
   ff_status s = tc_init(t);
   if (s != FF_OK) return s;
   CUtensorMap ta, tb;
@@ -1225,8 +1228,8 @@ inline ff_status tc_dense_update_slab(TcState& t, const int8_t* dHq, int N, cons
   p.slabs = slabs;
   const int kb_per_split = cdiv(p.kblocks, splits);
   *splits_out = cdiv(p.kblocks, kb_per_split);
-  if ((s = tc_make_map(t, &ta, dHq, N, rows_per_pass, 2, 128, 128)) != FF_OK) return s;
-  if ((s = tc_make_map(t, &tb, xi, kcols, rows_per_pass, 2, 128, 128)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &ta, dHq, N, rows_per_pass, 2, 128, 128, (uint64_t)ld_dhq)) != FF_OK) return s;
+  if ((s = tc_make_map(t, &tb, xi, kcols, rows_per_pass, 2, 128, 128, (uint64_t)ld_xi)) != FF_OK) return s;
   // one split: a large output with tiles for every SM, where CTA pairs pay; several: a small output, single CTAs
   const int ncta = t.force_ncta ? t.force_ncta : (splits == 1 ? tc_pick_ncta(t, N, kcols) : 1);
   return tc_launch<TC_MODE_SLAB, true, 128>(t, ncta, ta, tb, p, st);

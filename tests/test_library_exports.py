@@ -27,7 +27,7 @@ def test_struct_layouts_match_header_field_order():
     text = open(os.path.join(ROOT, "include", "ffint8.h")).read()
     body = re.search(r"typedef struct \{([^}]*)\} ff_layer_bufs;", text, flags=re.S).group(1)
     body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
-    fields = re.findall(r"\*\s*([A-Za-z_]+)\s*;", body)
+    fields = re.findall(r"(?:\*\s*|int32_t\s+)([A-Za-z_]+)\s*;", body)      # the pointers, then the INT32 row pitches
     assert fields == [f[0] for f in ffb.ff_layer_bufs._fields_]
     body = re.search(r"typedef struct \{([^}]*)\} ff_layer_desc;", text, flags=re.S).group(1)
     body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
