@@ -23,7 +23,8 @@ def specs_and_descs(layers, seed, round_x=1, round_w=0, round_dh=1):
 
 
 class GpuNet:
-    def __init__(self, descs, B, Ws, dumps=True, xnext=True, chain=True, gemm_path=ffb.FF_GEMM_AUTO, graph=False):
+    def __init__(self, descs, B, Ws, dumps=True, xnext=True, chain=True, gemm_path=ffb.FF_GEMM_AUTO, graph=False,
+                 pad_rows=True):
         import torch
         self.torch = torch
         self.dev = torch.device("cuda:0")
@@ -36,7 +37,7 @@ class GpuNet:
         ffb.ff_set_gemm_path(self.ctx.ctx, gemm_path)
         if graph:
             ffb.ff_set_graph_mode(self.ctx.ctx, True)
-        self.bufs = [ffb.LayerBuffers(d, B, self.dev, dumps=dumps, xnext=xnext, own_x=(i == 0 or not chain))
+        self.bufs = [ffb.LayerBuffers(d, B, self.dev, dumps=dumps, xnext=xnext, own_x=(i == 0 or not chain), pad_rows=pad_rows)
                      for i, d in enumerate(descs)]
         for b, W in zip(self.bufs, Ws):
             b.W.copy_(torch.from_numpy(W))

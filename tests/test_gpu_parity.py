@@ -60,11 +60,12 @@ def test_int8_gemm_tensor_weight_gradient_orientation(M, N, K, form):
     _gemm_case(M, N, K, 1, ffb.FF_GEMM_TENSOR, form)
 
 
-def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), chain=True, check_every=1, graph=False):
+def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), chain=True, check_every=1, graph=False,
+                     pad_rows=True):
     specs, descs = specs_and_descs(w.layers, seed, *rounding)
     Ws = synth.make_weights(w, seed)
     X = synth.make_batch(w, seed)
-    net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path, graph=graph)
+    net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path, graph=graph, pad_rows=pad_rows)
     net.set_input(X)
     Ms = Vs = None
     for step in range(steps):
@@ -612,4 +613,44 @@ def test_graph_cache_evicts_least_recently_used_shapes():
             compare_layer(st[0], net.bufs[0], specs[0], w.B, tag=f"round{rnd}/shape{i}/")
     # per shape and round: 2 replays (steps 1 and 2); every shape was evicted before its second round (20 > 16)
     assert ffb.ff_graph_replay_count(net.ctx.ctx) == 2 * 20 * 2, ffb.ff_last_error(net.ctx.ctx)
+    net.close()
+
+
+# ---- row pitches of the INT8 tensors -----------------------------------------------------------------------
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("pad_rows", [False, True])
+def test_unaligned_widths_with_and_without_padded_rows(path, pad_rows):
+    # widths 784 / 496 / 500: padded to 896 / 512 / 512-byte rows by default, dense rows on request; all rounding stochastic
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=136, width_div=4)
+    w.layers[0].N = w.layers[1].K = 496
+    w.layers[0].tau, w.layers[0].theta = float(np.sqrt(496)), 496.0
+    _run_and_compare(w, seed=77, steps=2, lam_per_step=0.5, path=path, rounding=(1, 1, 1), pad_rows=pad_rows)
+
+
+def test_explicit_row_pitch_and_its_checks():
+    import torch
+    w = synth.scaled(synth.workload("tiny_mlp"), B=24, width_div=2)      # 784 -> 250 -> 250
+    specs, descs = specs_and_descs(w.layers, 5)
+    Ws = synth.make_weights(w, 5)
+    X = synth.make_batch(w, 5)
+    net = GpuNet(descs, w.B, Ws, pad_rows=False)
+    # re-point layer 1 at buffers with pitches of its own choosing (the next multiples of 16 bytes and then some)
+    K, N, rows = descs[1].K, descs[1].N, 2 * w.B
+    ldx, ldd = (K + 31) // 16 * 16, (N + 63) // 16 * 16
+    xq = torch.full((rows, ldx), 99, dtype=torch.int8, device="cuda")
+    dh = torch.full((rows, ldd), 99, dtype=torch.int8, device="cuda")
+    net.bufs_arr[1].Xq, net.bufs_arr[1].ld_xq = xq.data_ptr(), ldx
+    net.bufs_arr[1].dHq, net.bufs_arr[1].ld_dhq = dh.data_ptr(), ldd
+    net.set_input(X)
+    net.train_step(0.0, 0)
+    st = O.train_step(specs, Ws, X, w.B, 0.0, 0)
+    assert np.array_equal(xq[:, :K].cpu().numpy(), st[1].Xq) and np.array_equal(dh[:, :N].cpu().numpy(), st[1].dHq)
+    assert bool((xq[:, K:] == 99).all()) and bool((dh[:, N:] == 99).all())          # padding bytes are never written
+    assert np.array_equal(net.bufs[1].W.cpu().numpy().view(np.uint32), st[1].W_new.view(np.uint32))
+    for field, bad in [("ld_xq", K // 16 * 16 - 16), ("ld_xq", ldx + 8), ("ld_dhq", ldd + 3)]:
+        old = getattr(net.bufs_arr[1], field)
+        setattr(net.bufs_arr[1], field, bad)
+        with pytest.raises(ffb.FFError):
+            net.train_step(0.0, 1)
+        setattr(net.bufs_arr[1], field, old)
     net.close()
