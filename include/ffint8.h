@@ -125,8 +125,9 @@ typedef struct {
   float* Var;        /* [N,K] FP32 in/out second-moment buffer; Adam only                      */
   int32_t ld_xq;     /* linear layers only: row pitch of Xq in bytes, 0 = K (dense).  A pitch that is a */
   int32_t ld_dhq;    /* multiple of 128 keeps every TMA box row of the contractions aligned when K (N  */
-                     /* for dHq) is not: >= the row length, a multiple of 16; padding bytes are never  */
-                     /* read as data and never written                                                */
+                     /* for dHq) is not: >= the row length, a multiple of 16.  All rows x pitch bytes  */
+                     /* belong to the buffer; the padding bytes are never written, and whatever they  */
+                     /* hold reaches no result (copies may fetch them)                                */
 } ff_layer_bufs;
 
 /* Create / destroy a context for CUDA device `device` (must be compute capability 10.x).

@@ -721,7 +721,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             if (i + 1 < TC_EPI_COLS / 32 && cb + 32 < cend) tc_ld32_async(t_row + pass * TC_BN + cb + 32, v[(i + 1) & 1]);
             if (cb < cend) {  // uniform across the warp
               const int(&a)[32] = v[i & 1];
-              if (col0 + cb + 32 <= p.out_cols && (p.out_cols & 3) == 0) {
+              if ((p.out_cols & 3) == 0) {  // groups of four columns are whole or absent, the last chunk included
 #pragma unroll
                 for (int j = 0; j < 32; j += 4)
                   *reinterpret_cast<int4*>(patch + lane * 128 + (((j >> 2) ^ (lane & 7)) << 4)) =
@@ -730,7 +730,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                   const int r = q * 4 + (lane >> 3), cc = lane & 7;
-                  if (wrow0 + r < p.out_rows)
+                  if (wrow0 + r < p.out_rows && col0 + cb + cc * 4 < p.out_cols)
                     *reinterpret_cast<int4*>(slab + (size_t)(wrow0 + r) * p.out_cols + col0 + cb + cc * 4) =
                         *reinterpret_cast<const int4*>(patch + r * 128 + ((cc ^ (r & 7)) << 4));
                 }
@@ -751,7 +751,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         uint8_t* patch = patch0;
 #pragma unroll 1
         for (int cb = cbeg; cb < cend; cb += 32) {
-          const bool full = (col0 + cb + 32 <= p.out_cols) && ((p.out_cols & 3) == 0);
+          // out_cols % 4 == 0: a lane's group of four columns is whole or absent, in the ragged last chunk too
+          const bool vec = (p.out_cols & 3) == 0;
+          const bool full = vec && col0 + cb + (lane & 7) * 4 < p.out_cols;
           // issue the (row-contiguous) W loads first so that they are in flight during the TMEM reads
           float4 wv[8];
           if (full) {
@@ -780,7 +782,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           for (int i = 0; i < 8; ++i) {
             const int r = i * 4 + (lane >> 3), cc = lane & 7;
             const int grow = wrow0 + r, gcol = col0 + cb + cc * 4;
-            if (grow < p.out_rows) {
+            if (grow < p.out_rows && (full || !vec)) {
               float4 dv = *reinterpret_cast<const float4*>(patch + r * 128 + ((cc ^ (r & 7)) << 4));
               float* dst = p.W + (size_t)grow * p.out_cols + gcol;
               if (p.mom) {  // heavy ball: the step is taken along m = mu*m + g
@@ -912,7 +914,10 @@ inline ff_status tc_encode(TcState& t, CUtensorMap* tm, const int8_t* base, cuui
 inline ff_status tc_make_map(TcState& t, CUtensorMap* tm, const int8_t* base, uint64_t cols, uint64_t rows_per_pass, uint64_t passes,
                              uint32_t box_cols, uint32_t box_rows, uint64_t pitch = 0) {
   if (!pitch) pitch = cols;
-  cuuint64_t dims[3] = {cols, rows_per_pass, passes ? passes : 1};
+  // A pitched row is mapped over its whole pitch: boxes that reach past `cols` then stay inside the map and
+  // take the plain copy path.  Whatever the padding bytes hold only meets zero-filled columns of the other
+  // operand (forward) or lands in output rows / columns that the epilogue discards (weight gradient).
+  cuuint64_t dims[3] = {pitch, rows_per_pass, passes ? passes : 1};
   cuuint64_t strides[2] = {pitch, pitch * rows_per_pass};
   cuuint32_t box[3] = {box_cols, box_rows, 1};
   return tc_encode(t, tm, base, passes > 0 ? 3 : 2, dims, strides, box, (int)box_cols);

@@ -61,11 +61,15 @@ def test_int8_gemm_tensor_weight_gradient_orientation(M, N, K, form):
 
 
 def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), chain=True, check_every=1, graph=False,
-                     pad_rows=True):
+                     pad_rows=True, pad_fill=None):
     specs, descs = specs_and_descs(w.layers, seed, *rounding)
     Ws = synth.make_weights(w, seed)
     X = synth.make_batch(w, seed)
     net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path, graph=graph, pad_rows=pad_rows)
+    if pad_fill is not None:      # whatever the padding bytes of the pitched rows hold must reach no result
+        for b in net.bufs:
+            b._Xq_store.fill_(pad_fill)
+            b._dHq_store.fill_(pad_fill)
     net.set_input(X)
     Ms = Vs = None
     for step in range(steps):
@@ -78,6 +82,10 @@ def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), cha
         Ws = [st.W_new for st in states]
         Ms = [st.M_new for st in states]
         Vs = [st.V_new for st in states]
+    if pad_fill is not None:
+        for b, d in zip(net.bufs, descs):
+            kin = b.Xq.shape[-1]
+            assert bool((b._Xq_store[:, kin:] == pad_fill).all()) and bool((b._dHq_store[:, d.N:] == pad_fill).all())
     net.close()
 
 
@@ -625,6 +633,19 @@ def test_unaligned_widths_with_and_without_padded_rows(path, pad_rows):
     w.layers[0].N = w.layers[1].K = 496
     w.layers[0].tau, w.layers[0].theta = float(np.sqrt(496)), 496.0
     _run_and_compare(w, seed=77, steps=2, lam_per_step=0.5, path=path, rounding=(1, 1, 1), pad_rows=pad_rows)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("momentum", [0.0, 0.9])
+def test_padding_bytes_reach_no_result(path, momentum):
+    # same widths with the padding of every pitched row preset to a non-zero byte: the contractions may fetch it (their
+    # copies span the pitch) but it meets zero-filled weight columns or discarded output rows / columns only
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=136, width_div=4)
+    w.layers[0].N = w.layers[1].K = 496
+    w.layers[0].tau, w.layers[0].theta = float(np.sqrt(496)), 496.0
+    for l in w.layers:
+        l.momentum = momentum
+    _run_and_compare(w, seed=78, steps=2, lam_per_step=0.5, path=path, rounding=(1, 1, 1), pad_fill=-77)
 
 
 def test_explicit_row_pitch_and_its_checks():
