@@ -62,7 +62,7 @@ struct TcGeom {
   static constexpr uint32_t B_BYTES = MN_MAJOR ? 128u * (TC_BN / NCTA) : (uint32_t)(TC_BN / NCTA) * CH;
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (int)(TC_RING_BYTES / STAGE_BYTES) < TC_MAX_STAGES ? (int)(TC_RING_BYTES / STAGE_BYTES) : TC_MAX_STAGES;
-  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + TC_EPI_WARPS * TC_PATCHES * TC_PATCH_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + TC_EPI_WARPS * TC_PATCHES * TC_PATCH_BYTES + 1024 /*align*/ + 512 /*barriers*/;
   static constexpr int MMAS = MN_MAJOR ? 4 : CH / 32;            // MMAs (K = 32) per contraction block
   static constexpr int B_BOXES = MN_MAJOR ? (TC_BN / NCTA) / CH : 1;  // TMA boxes of the B operand per stage
   static constexpr uint32_t SWZ = CH == 128 ? 2u : 4u;             // descriptor swizzle code: 128-byte / 64-byte
@@ -88,6 +88,7 @@ struct TcParams {
   const float* absmax;
   int rows_per_pass, rows_per_sample;
   int y_tma;                // Y leaves through TMA stores (needs N % 4 == 0); else plain stores
+  int w_tma;                // update epilogue: W comes and goes as 32 x 32 TMA patches (the Y map slot holds W's map)
   int y_stream;             // Y is larger than what L2 can usefully hold for the kernels that follow
   // update epilogue
   float* W;
@@ -293,6 +294,11 @@ __device__ __forceinline__ uint64_t l2_policy_evict_last() {
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
   return p;
 }
+__device__ __forceinline__ uint64_t l2_policy_evict_normal() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
   uint64_t p;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
@@ -354,6 +360,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   const uint32_t bar_tempty = bar_tfull + 16;                    // [2]       used in the leader CTA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_MAX_STAGES + 4);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  const uint32_t bar_wpatch = bar_full + 8 * (2 * TC_MAX_STAGES + 8);  // [TC_EPI_WARPS][TC_PATCHES] W patches (update epilogue)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = leader of the pair
@@ -371,6 +378,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       mbar_init(bar_tfull + 8 * s, 1);
       mbar_init(bar_tempty + 8 * s, TC_EPI_WARPS * NCTA);  // one arrive per epilogue warp of every CTA of the group
     }
+    if (MODE == TC_MODE_UPD)
+      for (int s = 0; s < TC_EPI_WARPS * TC_PATCHES; ++s) mbar_init(bar_wpatch + 8 * s, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -566,6 +575,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     uint8_t* patch0 = patch_all + (warp - 2) * TC_PATCHES * TC_PATCH_BYTES;
     uint32_t pflip = 0;  // which of the warp's two patches the next chunk fills (forward epilogue)
     (void)pflip;
+    uint32_t wuse = 0, wdone = 0;  // W patches requested / consumed so far (update epilogue): slot = count & 1, parity = count >> 1
+    (void)wuse;
+    (void)wdone;
+    const uint64_t w_policy = l2_policy_evict_normal();
+    (void)w_policy;
     // A large Y is written once and read much later: let it leave L2 first.  A small one is read back by
     // the next kernels (normalisation, dH quantiser) while it still sits in L2: keep it.
     const uint64_t y_policy = p.y_stream ? l2_policy_evict_first() : l2_policy_evict_last();
@@ -588,11 +602,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       int tm, tn;
       tile_coords(tile, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
       const uint32_t as = tile_it % ACC_STAGES, aph = (tile_it / ACC_STAGES) & 1u;
-      if (!mbar_wait<PAIR>(bar_tfull + 8 * as, aph, abort_flag)) {
-        ok = false;
-        break;
-      }
-      tc_fence_after();
       const int wrow0 = tm * (TC_BM * NCTA) + (int)rank * TC_BM + quad * 32;  // first output row of this warp
       const int row = wrow0 + lane;
       const bool row_ok = row < p.out_rows;
@@ -602,6 +611,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       const int chunks = (min(TC_BN, p.out_cols - col0) + 31) >> 5;
       const int cbeg = half ? ((chunks + 1) >> 1) * 32 : 0;
       const int cend = half ? chunks * 32 : ((chunks + 1) >> 1) * 32;
+      // Update epilogue with W patches: the 32 x 32 block of W under chunk `cb` comes into one of the warp's two
+      // swizzled patches by TMA (the box is clipped / zero-filled at the edges of W) and goes back the same way.
+      // A patch is reloaded only after the store that last left from it has read it.
+      const bool w_patches = MODE == TC_MODE_UPD && p.w_tma && wrow0 < p.out_rows;
+      auto w_patch_load = [&](int cb) {
+        if (lane == 0) {
+          const uint32_t slot = wuse & 1u;
+          bulk_wait_read0();
+          mbar_expect_tx(bar_wpatch + 8 * ((warp - 2) * TC_PATCHES + slot), TC_PATCH_BYTES);
+          tma_load_2d<1>(smem_u32(patch0 + slot * TC_PATCH_BYTES), &tmY, bar_wpatch + 8 * ((warp - 2) * TC_PATCHES + slot), col0 + cb,
+                         wrow0, w_policy);
+        }
+        ++wuse;
+      };
+      if (w_patches && cbeg < cend) w_patch_load(cbeg);  // nobody else writes this tile of W: fetch while the MMAs still run
+      if (!mbar_wait<PAIR>(bar_tfull + 8 * as, aph, abort_flag)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after();
       if (MODE == TC_MODE_RAW) {
 #pragma unroll 1
         for (int cb = cbeg; cb < cend; cb += 32) {
@@ -744,6 +773,56 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             }
           }
         }
+      } else if (MODE == TC_MODE_UPD && p.w_tma) {
+        // thread = one accumulator row: g = float(accP)*cP + float(accN)*cN stays in registers, the thread updates
+        // its own row of the W patch in shared memory, one TMA store per patch writes it back
+        if (wrow0 < p.out_rows) {
+          const size_t plane = (size_t)p.out_rows * p.out_cols;
+#pragma unroll 1
+          for (int cb = cbeg; cb < cend && ok; cb += 32) {
+            if (cb + 32 < cend) w_patch_load(cb + 32);
+            int vp[32], vn[32];
+            tc_ld32_async(t_row + cb, vp);
+            tc_ld32_async(t_row + TC_BN + cb, vn);
+            tc_wait_ld(vp);
+            tc_wait_ld(vn);
+            float d[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              d[j] = __fmul_rn(p.lr, __fadd_rn(__fmul_rn(__int2float_rn(vp[j]), cP), __fmul_rn(__int2float_rn(vn[j]), cN)));
+            const uint32_t slot = wdone & 1u, par = (wdone >> 1) & 1u;
+            ++wdone;
+            if (!mbar_wait<false>(bar_wpatch + 8 * ((warp - 2) * TC_PATCHES + slot), par, abort_flag)) {
+              ok = false;
+              break;
+            }
+            uint8_t* patch = patch0 + slot * TC_PATCH_BYTES;
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              float4* q = reinterpret_cast<float4*>(patch + lane * 128 + (((j >> 2) ^ (lane & 7)) << 4));
+              float4 w = *q;
+              w.x = __fsub_rn(w.x, d[j]);
+              w.y = __fsub_rn(w.y, d[j + 1]);
+              w.z = __fsub_rn(w.z, d[j + 2]);
+              w.w = __fsub_rn(w.w, d[j + 3]);
+              *q = w;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmY, smem_u32(patch), col0 + cb, wrow0, w_policy);
+              bulk_commit();
+            }
+            if (p.accW_dump && row_ok) {  // parity dump
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + cb + j < p.out_cols) {
+                  p.accW_dump[(size_t)row * p.out_cols + col0 + cb + j] = vp[j];
+                  p.accW_dump[plane + (size_t)row * p.out_cols + col0 + cb + j] = vn[j];
+                }
+            }
+          }
+        }
       } else {  // TC_MODE_UPD
         // thread = one accumulator row computes g = float(accP)*cP + float(accN)*cN; g is staged
         // through smem so that the read-modify-write of W (and of the momentum buffer) is row-contiguous
@@ -841,7 +920,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           mbar_arrive(bar_tempty + 8 * as);
       }
     }
-    if (MODE == TC_MODE_FWD && lane == 0) bulk_wait_read0();  // the last stores have read their patches
+    if ((MODE == TC_MODE_FWD || MODE == TC_MODE_UPD) && lane == 0) bulk_wait_read0();  // the last stores have read their patches
     if (!ok && lane == 0) raise_abort();
   }
 
@@ -1171,7 +1250,11 @@ inline ff_status tc_update(TcState& t, const ff_layer_desc& L, const ff_layer_bu
   p.mu = L.momentum;
   if ((s = tc_make_map(t, &ta, b.dHq, L.N, B, 2, 128, 128, (uint64_t)b.ld_dhq)) != FF_OK) return s;
   if ((s = tc_make_map(t, &tb, b.Xq, L.K, B, 2, 128, 128, (uint64_t)b.ld_xq)) != FF_OK) return s;
-  return tc_launch<TC_MODE_UPD, true, 128>(t, tc_pick_ncta(t, L.N, L.K), ta, tb, p, st);
+  // plain SGD: W travels through the epilogue as 32 x 32 TMA patches (K % 16 == 0 here, so its rows are 16-byte pitched)
+  CUtensorMap tw;
+  p.w_tma = (!p.mom && (reinterpret_cast<uintptr_t>(b.W) & 15) == 0) ? 1 : 0;
+  if (p.w_tma && (s = tc_make_store_map(t, &tw, b.W, L.K, L.N)) != FF_OK) return s;
+  return tc_launch<TC_MODE_UPD, true, 128>(t, tc_pick_ncta(t, L.N, L.K), ta, tb, p, st, p.w_tma ? &tw : nullptr);
 }
 
 // Convolution weight gradient: split contraction, INT32 partial sums of both sets to `slabs`
