@@ -648,6 +648,19 @@ def test_padding_bytes_reach_no_result(path, momentum):
     _run_and_compare(w, seed=78, steps=2, lam_per_step=0.5, path=path, rounding=(1, 1, 1), pad_fill=-77)
 
 
+@pytest.mark.parametrize("form", TENSOR_FORMS)
+@pytest.mark.parametrize("momentum", [0.0, 0.9])
+def test_update_epilogue_edges(form, momentum):
+    # weight matrices whose edges cut through the update epilogue's 32 x 32 patches: 144 and 272 rows (warps with 16
+    # valid rows and warps wholly outside the matrix), 784 and 272 columns (a last chunk of 16 columns), several
+    # tiles per CTA on the first layer; plain SGD moves W as TMA patches, momentum takes the load / store form
+    widths = [784, 272, 144, 48]
+    layers = [synth.LayerCfg(0, K, N, float(N) / 2, 0.03, float(np.sqrt(N)), momentum=momentum)
+              for K, N in zip(widths[:-1], widths[1:])]
+    w = synth.Workload("edges", 200, layers, (widths[0],), "uniform01", "kaiming_uniform", 1)
+    _run_and_compare(w, seed=91, steps=3, lam_per_step=0.25, path=(ffb.FF_GEMM_AUTO, form), rounding=(1, 0, 1))
+
+
 def test_explicit_row_pitch_and_its_checks():
     import torch
     w = synth.scaled(synth.workload("tiny_mlp"), B=24, width_div=2)      # 784 -> 250 -> 250
