@@ -239,14 +239,13 @@ ff_status ff_layer_loss_grad(ff_ctx* ctx, const ff_layer_desc* layer, const ff_l
                              int B, const float* const* G_later, const float* theta_later,
                              int n_later, float lambda, uint64_t step, void* cuda_stream);
 
-/* Weight gradient and update of one layer (Sec. IV-B: g^W as an INT8 MAC, "only gradients of
- * weights are computed and updated"; Alg. 1 line 9).  Reads dHq, Xq, absmax, W.  Writes W
+/* Weight gradient and update of one layer (Sec. IV-B: g^W is a second INT8 MAC and is the only
+ * gradient formed and applied; Alg. 1 line 9).  Reads dHq, Xq, absmax, W.  Writes W
  * (W - lr*(float(accP)*cP + float(accN)*cN)) and accW_dump (if non-NULL); with momentum != 0 or
- * optimizer = FF_OPT_ADAM the step follows that rule and Mom (and Var) are rewritten.  Adam's update
- * number t is 1 + the step of the last call on this context that took one (ff_layer_forward,
- * ff_layer_loss_grad, ff_train_step ...), so call ff_layer_loss_grad for the same step first. */
+ * optimizer = FF_OPT_ADAM the step follows that rule and Mom (and Var) are rewritten.  `step` is the
+ * step counter of the update (Adam's update number is t = step + 1; the other rules do not read it). */
 ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs,
-                          int B, void* cuda_stream);
+                          int B, uint64_t step, void* cuda_stream);
 
 /* Body of Algorithm 1's epoch loop for n_layers layers: one INT8 forward through all layers with
  * the pre-update weights (line 5), goodness of every layer (line 6), then per layer the loss with
@@ -255,6 +254,17 @@ ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_laye
  * With n_layers = 1 and lambda = 0 it equals forward -> loss_grad -> update. */
 ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs,
                         int n_layers, int B, float lambda, uint64_t step, void* cuda_stream);
+
+/* One step of layer-by-layer training (Sec. III: a layer is trained to the end before its successor
+ * is; Sec. IV-B trains "each layer" this way when the look-ahead of Sec. IV-C is off).  As
+ * ff_train_step, but the layers [0, first_trained) are frozen: they run the INT8 forward with their
+ * current weights and hand their normalised output on; no loss, g^Y, g^W or update is computed for
+ * them and their coef, loss, dHq, absmax[DH] and W stay untouched.  Layers first_trained .. n_layers-1
+ * are trained as in ff_train_step (each looks ahead at the layers after it).  first_trained = 0 is
+ * ff_train_step itself; first_trained = n_layers-1 with lambda = 0 is one step of the greedy schedule.
+ * Replayed like ff_train_step when ff_set_graph_mode is on (one captured sequence per first_trained). */
+ff_status ff_train_step_from(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers,
+                             int first_trained, int B, float lambda, uint64_t step, void* cuda_stream);
 
 /* Classification of B samples by goodness with the current weights.  The paper reports accuracy but
  * does not describe the procedure; this is the Forward-Forward one its Sec. III builds on ("make

@@ -547,12 +547,16 @@ def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int, M: Opti
 
 
 def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: int, lam: float,
-               step: int, Ms: Optional[List[np.ndarray]] = None, Vs: Optional[List[np.ndarray]] = None) -> List[LayerState]:
+               step: int, Ms: Optional[List[np.ndarray]] = None, Vs: Optional[List[np.ndarray]] = None,
+               first_trained: int = 0) -> List[LayerState]:
     """Body of Algorithm 1's epoch loop: one INT8 forward through all k layers with the
     pre-update weights (line 5), goodness of every layer (line 6), then for each layer its
     loss from the G's (line 8) and its INT8 gradient and update (line 9).  lambda is the
     caller's (lines 2 and 11).  With one layer and lambda = 0 this is the vanilla step.  Ms: the
-    layers' momentum buffers (only read by layers with momentum != 0)."""
+    layers' momentum buffers (only read by layers with momentum != 0).
+    first_trained > 0: the layers before it are frozen - they take part in the forward only (their
+    states carry no coef, dHq or W_new).  This is one step of the layer-by-layer schedule of Sec. III,
+    where a layer is trained on the output of the already trained layers before it."""
     states = []
     x = X
     for spec, W in zip(specs, Ws):
@@ -560,11 +564,30 @@ def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: i
         states.append(st)
         x = st.Xnext
     for l, (spec, W) in enumerate(zip(specs, Ws)):
+        if l < first_trained:
+            continue
         later = list(range(l + 1, len(specs)))
         layer_loss_grad(spec, states[l], B, [states[j].G for j in later],
                         [specs[j].theta for j in later], lam, step)
         layer_update(spec, states[l], W, B, None if Ms is None else Ms[l], None if Vs is None else Vs[l], step)
     return states
+
+
+def greedy_epoch(specs: List[LayerSpec], Ws: List[np.ndarray], batches, B: int, on_step=None) -> List[np.ndarray]:
+    """Layer-by-layer training (Sec. III: a layer is trained to the end, then its successor): phase l runs
+    over every batch once and trains layer l alone (lambda = 0) on the INT8 forward of layers 0..l-1 as
+    their own phases left them.  `batches` is a sequence of batches (anything with len() and [i]); the
+    step counter that keys the stochastic rounding runs on through the phases: t = l*len(batches) + i.
+    on_step(l, i, states) sees every step.  Returns the trained weights."""
+    Ws = [np.asarray(W, dtype=F32) for W in Ws]
+    n = len(batches)
+    for l in range(len(specs)):
+        for i in range(n):
+            states = train_step(specs[:l + 1], Ws[:l + 1], batches[i], B, 0.0, l * n + i, first_trained=l)
+            Ws[l] = states[l].W_new
+            if on_step is not None:
+                on_step(l, i, states)
+    return Ws
 
 
 # --------------------------------------------------------------------------------------

@@ -22,7 +22,7 @@ FF_ABSMAX_LEN = 8
 EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", "ff_set_gemm_path", "ff_set_tensor_form",
            "ff_set_graph_mode", "ff_graph_replay_count", "ff_dp_phase_count", "ff_dp_train_phase",
            "ff_embed_labels",
-           "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step",
+           "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step", "ff_train_step_from",
            "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
            "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict"]
 FF_STATIC_LOSS_MAX_SAMPLES = 65536
@@ -92,8 +92,9 @@ def load(build_if_missing: bool = True):
     lib.ff_layer_forward.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, u64, vp]
     lib.ff_layer_loss_grad.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32,
                                        C.POINTER(vp), C.POINTER(f32), i32, f32, u64, vp]
-    lib.ff_layer_update.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, vp]
+    lib.ff_layer_update.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, u64, vp]
     lib.ff_train_step.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, i32, f32, u64, vp]
+    lib.ff_train_step_from.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, i32, i32, f32, u64, vp]
     lib.ff_poll_status.argtypes = [vp, vp]
     lib.ff_last_error.argtypes = [vp]
     lib.ff_last_error.restype = C.c_char_p
@@ -167,13 +168,19 @@ def ff_layer_loss_grad(ctx, desc, bufs, B: int, G_later: Sequence[int], theta_la
     _check(ctx, load().ff_layer_loss_grad(ctx, C.byref(desc), C.byref(bufs), B, gp, th, n, lam, step, stream))
 
 
-def ff_layer_update(ctx, desc, bufs, B: int, stream: int = 0):
-    _check(ctx, load().ff_layer_update(ctx, C.byref(desc), C.byref(bufs), B, stream))
+def ff_layer_update(ctx, desc, bufs, B: int, step: int, stream: int = 0):
+    _check(ctx, load().ff_layer_update(ctx, C.byref(desc), C.byref(bufs), B, step, stream))
 
 
 def ff_train_step(ctx, descs_arr, bufs_arr, n_layers: int, B: int, lam: float, step: int, stream: int = 0):
     """descs_arr / bufs_arr: ctypes arrays (ff_layer_desc * n), (ff_layer_bufs * n)."""
     _check(ctx, load().ff_train_step(ctx, descs_arr, bufs_arr, n_layers, B, lam, step, stream))
+
+
+def ff_train_step_from(ctx, descs_arr, bufs_arr, n_layers: int, first_trained: int, B: int, lam: float, step: int,
+                       stream: int = 0):
+    """ff_train_step with the layers before first_trained frozen (forward only)."""
+    _check(ctx, load().ff_train_step_from(ctx, descs_arr, bufs_arr, n_layers, first_trained, B, lam, step, stream))
 
 
 def ff_embed_labels(ctx, x: int, labels: int, B: int, n: int, sets: int, n_classes: int, label_stride: int,

@@ -469,8 +469,9 @@ struct LossJobs {
   int n;
 };
 __global__ void __launch_bounds__(LOSS_THREADS) loss_coef_multi_kernel(const LossJobs jobs, int B, LossScratch* __restrict__ scratch,
-                                                                       const StepState* __restrict__ ss, int m_total) {
-  const int l = blockIdx.y;
+                                                                       const StepState* __restrict__ ss, int m_total,
+                                                                       int first = 0) {
+  const int l = blockIdx.y + first;  // layers before `first` are frozen: no loss, no gradient
   loss_coef_body(jobs.G[l], jobs.theta[l], jobs.G + l + 1, jobs.theta + l + 1, jobs.n - 1 - l, ss->lambda, B, jobs.rowmax[l],
                  jobs.absmax[l], jobs.coef[l], jobs.loss[l], scratch + l, m_total);
 }
@@ -611,8 +612,8 @@ struct DhJobs {
   const StepState* ss;
 };
 template <bool PAD>
-__global__ void __launch_bounds__(EW_THREADS) dh_quantize_multi_kernel(const DhJobs jobs, int B) {
-  const int l = blockIdx.y >> 1, pass = blockIdx.y & 1;
+__global__ void __launch_bounds__(EW_THREADS) dh_quantize_multi_kernel(const DhJobs jobs, int B, int first = 0) {
+  const int l = (blockIdx.y >> 1) + first, pass = blockIdx.y & 1;
   const size_t per_sample = (size_t)jobs.per_sample[l], per_pass = per_sample * B;
   if (jobs.stochastic[l])
     dh_quantize_body<ROUND_STOCHASTIC, PAD>(jobs.Y[l], jobs.coef[l], jobs.absmax[l], per_sample, per_pass, jobs.dHq[l],

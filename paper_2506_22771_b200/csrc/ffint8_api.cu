@@ -865,8 +865,9 @@ ff_status forward_all(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_b
 }
 
 // Everything of one train step after the step counter and lambda have been published (Alg. 1, epoch body).
+// Layers before `first` are frozen: they take part in the forward only (layer-by-layer training, Sec. III).
 ff_status train_step_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
-                          float lambda, cudaStream_t st) {
+                          float lambda, cudaStream_t st, int first = 0) {
   ff_status s;
   (void)lambda;  // read by the kernels from the step state
   // Alg. 1 line 5-6: one forward through all layers with the pre-update weights
@@ -885,29 +886,29 @@ ff_status train_step_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_lay
     dj.s1[l] = make_key_spec(layers[l].seed, ROLE_DH, layers[l].index, nullptr).s1;
     dj.stochastic[l] = layers[l].round_dh != FF_ROUND_NEAREST_EVEN;
     dj.pad[l] = row_pad(layers[l].N, bufs[l].ld_dhq);
-    if (dj.per_sample[l] * B > largest) largest = dj.per_sample[l] * B;
+    if (l >= first && dj.per_sample[l] * B > largest) largest = dj.per_sample[l] * B;
   }
   dj.ss = step_ptr(ctx);
   int loss_blocks = (2 * B + LOSS_THREADS - 1) / LOSS_THREADS;
   if (loss_blocks > LOSS_MAX_BLOCKS) loss_blocks = LOSS_MAX_BLOCKS;
   {
     ProfScope prof(ctx, FF_K_LOSS, st);
-    loss_coef_multi_kernel<<<dim3(loss_blocks, n_layers), LOSS_THREADS, 0, st>>>(
-        lj, B, reinterpret_cast<LossScratch*>(static_cast<char*>(ctx->workspace) + WS_LOSS_OFFSET), step_ptr(ctx), 0);
+    loss_coef_multi_kernel<<<dim3(loss_blocks, n_layers - first), LOSS_THREADS, 0, st>>>(
+        lj, B, reinterpret_cast<LossScratch*>(static_cast<char*>(ctx->workspace) + WS_LOSS_OFFSET), step_ptr(ctx), 0, first);
   }
   FF_LAUNCH_CHECK(ctx);
   {
     ProfScope prof(ctx, FF_K_DH_QUANTIZE, st);
     bool any_pad = false;
-    for (int l = 0; l < n_layers; ++l) any_pad = any_pad || bufs[l].ld_dhq != 0;
-    const dim3 grid(ew_blocks(ctx, largest / 4 + 1), 2 * n_layers);
+    for (int l = first; l < n_layers; ++l) any_pad = any_pad || bufs[l].ld_dhq != 0;
+    const dim3 grid(ew_blocks(ctx, largest / 4 + 1), 2 * (n_layers - first));
     if (any_pad)
-      dh_quantize_multi_kernel<true><<<grid, EW_THREADS, 0, st>>>(dj, B);
+      dh_quantize_multi_kernel<true><<<grid, EW_THREADS, 0, st>>>(dj, B, first);
     else
-      dh_quantize_multi_kernel<false><<<grid, EW_THREADS, 0, st>>>(dj, B);
+      dh_quantize_multi_kernel<false><<<grid, EW_THREADS, 0, st>>>(dj, B, first);
   }
   FF_LAUNCH_CHECK(ctx);
-  for (int l = 0; l < n_layers; ++l)
+  for (int l = first; l < n_layers; ++l)
     if ((s = run_update_gemm(ctx, layers[l], bufs[l], B, st)) != FF_OK) return s;
   return FF_OK;
 }
@@ -1081,10 +1082,10 @@ ff_status run_replayed(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_
 }
 
 ff_status train_step_graph(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
-                           float lambda, cudaStream_t st) {
-  const int tag = 1;
-  return run_replayed(ctx, layers, bufs, n_layers, B, &tag, sizeof(tag), st, [&](cudaStream_t s) {
-    return train_step_body(ctx, layers, bufs, n_layers, B, lambda, s);
+                           float lambda, cudaStream_t st, int first) {
+  const int tag[2] = {1, first};
+  return run_replayed(ctx, layers, bufs, n_layers, B, tag, sizeof(tag), st, [&](cudaStream_t s) {
+    return train_step_body(ctx, layers, bufs, n_layers, B, lambda, s, first);
   });
 }
 
@@ -1215,7 +1216,8 @@ ff_status ff_layer_loss_grad(ff_ctx* ctx, const ff_layer_desc* layer, const ff_l
   return loss_grad_impl(ctx, *layer, *bufs, B, G_later, theta_later, n_later, lambda, st);
 }
 
-ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs, int B, void* cuda_stream) {
+ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs, int B, uint64_t step,
+                          void* cuda_stream) {
   ff_status s = check_ctx(ctx);
   if (s != FF_OK) return s;
   if ((s = check_layer(ctx, layer, B)) != FF_OK) return s;
@@ -1223,19 +1225,26 @@ ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_laye
   if ((s = check_pitches(ctx, layer, bufs)) != FF_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  if ((s = set_step(ctx, step, 0.0f, false, st)) != FF_OK) return s;  // Adam's update number is step + 1
   return run_update_gemm(ctx, *layer, *bufs, B, st);
+}
+
+ff_status ff_train_step_from(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers,
+                             int first_trained, int B, float lambda, uint64_t step, void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if ((s = check_layer_list(ctx, layers, bufs, n_layers, B)) != FF_OK) return s;
+  if (first_trained < 0 || first_trained >= n_layers) return fail(ctx, FF_ERR_ARG, "first_trained out of range");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  if ((s = set_step(ctx, step, lambda, true, st, bufs, n_layers)) != FF_OK) return s;
+  if (ctx->graph_mode && !ctx->profiling) return train_step_graph(ctx, layers, bufs, n_layers, B, lambda, st, first_trained);
+  return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st, first_trained);
 }
 
 ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
                         float lambda, uint64_t step, void* cuda_stream) {
-  ff_status s = check_ctx(ctx);
-  if (s != FF_OK) return s;
-  if ((s = check_layer_list(ctx, layers, bufs, n_layers, B)) != FF_OK) return s;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
-  if ((s = set_step(ctx, step, lambda, true, st, bufs, n_layers)) != FF_OK) return s;
-  if (ctx->graph_mode && !ctx->profiling) return train_step_graph(ctx, layers, bufs, n_layers, B, lambda, st);
-  return train_step_body(ctx, layers, bufs, n_layers, B, lambda, st);
+  return ff_train_step_from(ctx, layers, bufs, n_layers, 0, B, lambda, step, cuda_stream);
 }
 
 int ff_dp_phase_count(int n_layers) { return n_layers > 0 ? n_layers + 4 : 0; }

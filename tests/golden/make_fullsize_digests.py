@@ -24,9 +24,10 @@ from paper_2506_22771_b200 import synth        # noqa: E402
 
 OUT = os.path.join(os.path.dirname(os.path.abspath(__file__)), "fullsize_digests.json")
 SEED = 1
-# workload -> number of consecutive steps run (weights carried from step to step).  Every step of a short
-# run is digested; of a long run the first two steps and every tenth (out["digested"] lists them).
-CASES = {"tiny_mlp": 10, "mlp_greedy": 3, "mlp_lookahead": 50, "cnn": 3, "roofline": 2, "separable": 2}
+# workload -> number of consecutive steps run (weights carried from step to step; mlp_greedy: batches per
+# phase of its layer-by-layer epoch).  Every step of a short run is digested; of a long run the first two
+# steps and every tenth (out["digested"] lists them).
+CASES = {"tiny_mlp": 10, "mlp_greedy": 58, "mlp_lookahead": 50, "cnn": 3, "roofline": 2, "separable": 2}
 
 
 def digested_steps(steps: int):
@@ -56,22 +57,24 @@ def run(name: str, steps: int) -> dict:
     out = {"B": w.B, "seed": SEED, "greedy": bool(w.greedy), "n_steps": steps, "digested": digested_steps(steps),
            "steps": []}
     if w.greedy:
-        # layers trained one after another (Sec. III): phase l trains layer l alone on the INT8 forward of
-        # the earlier layers; here every phase starts from the initial weights so that it can be checked on
-        # its own.  out["steps"][l][step] = digests of layer l.
-        for l, spec in enumerate(specs):
-            Wl = Ws[l]
-            phase = []
-            for step in range(steps):
-                t0 = time.time()
-                x = X
-                for j in range(l):
-                    x = O.layer_forward(specs[j], x, Ws[j], w.B, step).Xnext
-                st = O.train_step([spec], [Wl], x, w.B, 0.0, step)[0]
-                phase.append(layer_digests(st, w.B))
-                Wl = st.W_new
-                print(f"{name} layer {l} step {step}: {time.time() - t0:.1f} s", flush=True)
-            out["steps"].append(phase)
+        # the whole layer-by-layer epoch (Sec. III): `steps` distinct batches per phase, phase l trains layer l on
+        # the INT8 forward of the earlier layers as trained by their own phases, weights carried through every
+        # step.  out["steps"][l] = digests of layer l at the phase steps listed in out["digested"];
+        # out["final_W"][l] = digest of layer l's weights after its phase.
+        batches = [synth.make_batch(w, SEED, batch_index=i) for i in range(steps)]
+        dig = sorted(set(digested_steps(steps) + [steps - 1]))
+        out["digested"] = dig
+        out["steps"] = [[] for _ in specs]
+        clock = [time.time()]
+
+        def on_step(l, i, states):
+            if i in dig:
+                out["steps"][l].append(layer_digests(states[l], w.B))
+            print(f"{name} phase {l} batch {i}: {time.time() - clock[0]:.1f} s", flush=True)
+            clock[0] = time.time()
+
+        Wt = O.greedy_epoch(specs, Ws, batches, w.B, on_step)
+        out["final_W"] = [digest(W.astype(np.float32)) for W in Wt]
         return out
     for step in range(steps):
         t0 = time.time()

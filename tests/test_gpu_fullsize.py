@@ -61,30 +61,33 @@ def test_fullsize_train_steps_match_oracle_digests(name, graph):
     net.close()
 
 
-def test_fullsize_greedy_phases_match_oracle_digests():
+@pytest.mark.parametrize("graph", [False, True])
+def test_fullsize_greedy_epoch_matches_oracle_digests(graph):
+    """Configuration 2 as stated: 58 distinct batches of 1024 + 1024 samples per phase, four phases; phase l trains
+    layer l alone (ff_train_step_from with the earlier layers frozen) on the INT8 forward of the layers its
+    predecessors' phases trained, weights carried through all 232 layer-steps.  The oracle's digests of the
+    trained layer at the first two, every tenth and the last step of each phase, and of each layer's final
+    weights, are compared with the device's."""
     name = "mlp_greedy"
-    if name not in DIG:
-        pytest.skip("no digests for this workload in tests/golden/fullsize_digests.json")
+    if name not in DIG or "final_W" not in DIG[name]:
+        pytest.skip("no epoch digests for this workload in tests/golden/fullsize_digests.json")
     import torch
     d = DIG[name]
     w = synth.workload(name)
-    assert d["B"] == w.B and d["greedy"]
-    descs = _descs(w, d["seed"])
-    W0 = synth.make_weights(w, d["seed"])
-    X = synth.make_batch(w, d["seed"])
-    for l, phase in enumerate(d["steps"]):
-        # layer l trained alone on the INT8 forward of the frozen earlier layers, from the initial weights
-        net = GpuNet(descs[:l + 1], w.B, W0[:l + 1], dumps=False, xnext=True, chain=False)
-        one_d = (ffb.ff_layer_desc * 1)(descs[l])
-        one_b = (ffb.ff_layer_bufs * 1)(net.bufs[l].struct)
-        for step, want in enumerate(phase):
-            net.set_input(X)
-            for j in range(l):
-                ffb.ff_layer_forward(net.ctx.ctx, descs[j], net.bufs[j].struct, w.B, step, 0)
-                net.bufs[j + 1].X.copy_(net.bufs[j].Xnext)
-            ffb.ff_train_step(net.ctx.ctx, one_d, one_b, 1, w.B, 0.0, step, 0)
-            ffb.ff_poll_status(net.ctx.ctx, 0)
-            _check_layer(net.bufs[l], want, f"{name}/layer{l}/step{step}")
-        net.close()
-        del net
-        torch.cuda.empty_cache()
+    n_batches = d["n_steps"]
+    assert d["B"] == w.B and d["greedy"] and n_batches == w.steps
+    net = GpuNet(_descs(w, d["seed"]), w.B, synth.make_weights(w, d["seed"]), dumps=False, xnext=False, chain=True, graph=graph)
+    batches = [torch.from_numpy(synth.make_batch(w, d["seed"], batch_index=i)).cuda() for i in range(n_batches)]
+    ctx = net.ctx.ctx
+    for l in range(len(w.layers)):
+        for i in range(n_batches):
+            net.bufs[0].X.copy_(batches[i].reshape(net.bufs[0].X.shape))
+            ffb.ff_train_step_from(ctx, net.descs_arr, net.bufs_arr, l + 1, l, w.B, 0.0, l * n_batches + i, 0)
+            if i in d["digested"]:
+                ffb.ff_poll_status(ctx, 0)
+                _check_layer(net.bufs[l], d["steps"][l][d["digested"].index(i)], f"{name}/phase{l}/batch{i}")
+        ffb.ff_poll_status(ctx, 0)
+        assert _sha(net.bufs[l].W) == d["final_W"][l], (name, l, "final weights differ from the oracle's")
+    if graph:
+        assert ffb.ff_graph_replay_count(ctx) >= len(w.layers) * (n_batches - 2)
+    net.close()

@@ -133,6 +133,57 @@ def test_config2_greedy_scaled(path):
 
 
 @pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("graph", [False, True])
+def test_greedy_epoch_scaled_with_frozen_layers(path, graph):
+    # configuration 2's schedule at reduced width: three batches per phase, phase l trains layer l through
+    # ff_train_step_from on the chained INT8 forward of the layers the earlier phases trained; every tensor of the
+    # trained layer and the forward tensors of the frozen ones are compared element by element at every step
+    w = synth.scaled(synth.workload("mlp_greedy"), B=72, width_div=8)
+    specs, descs = specs_and_descs(w.layers, 9)
+    Ws = synth.make_weights(w, 9)
+    nb = 3
+    batches = [synth.make_batch(w, 9, batch_index=i) for i in range(nb)]
+    net = GpuNet(descs, w.B, Ws, gemm_path=path, graph=graph)
+    ctx = net.ctx.ctx
+    frozen_W = {}
+
+    def on_step(l, i, states):
+        net.set_input(batches[i])
+        ffb.ff_train_step_from(ctx, net.descs_arr, net.bufs_arr, l + 1, l, w.B, 0.0, l * nb + i, 0)
+        ffb.ff_poll_status(ctx, 0)
+        for j in range(l + 1):
+            compare_layer(states[j], net.bufs[j], specs[j], w.B, tag=f"phase{l}/batch{i}/layer{j}/")
+        for j in range(l):     # frozen layers keep the weights their own phase left
+            assert bool((net.bufs[j].W == frozen_W[j]).all())
+        if i == nb - 1:
+            frozen_W[l] = net.bufs[l].W.clone()
+
+    O.greedy_epoch(specs, Ws, batches, w.B, on_step)
+    net.close()
+
+
+def test_train_step_from_with_lookahead_over_the_trained_layers():
+    # layers 0 frozen, layers 1..3 trained with lambda > 0: each trained layer looks ahead at the layers after it
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=40, width_div=8)
+    specs, descs = specs_and_descs(w.layers, 6)
+    Ws = synth.make_weights(w, 6)
+    X = synth.make_batch(w, 6)
+    net = GpuNet(descs, w.B, Ws)
+    net.set_input(X)
+    for step in range(2):
+        ffb.ff_train_step_from(net.ctx.ctx, net.descs_arr, net.bufs_arr, len(descs), 1, w.B, 0.3, step, 0)
+        ffb.ff_poll_status(net.ctx.ctx, 0)
+        states = O.train_step(specs, Ws, X, w.B, 0.3, step, first_trained=1)
+        for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
+            compare_layer(st, b, sp, w.B, tag=f"step{step}/layer{l}/")
+        Ws = [Ws[0]] + [st.W_new for st in states[1:]]
+    with pytest.raises(ffb.FFError) as e:
+        ffb.ff_train_step_from(net.ctx.ctx, net.descs_arr, net.bufs_arr, len(descs), len(descs), w.B, 0.0, 0, 0)
+    assert e.value.code == ffb.FF_ERR_ARG
+    net.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
 def test_config4_cnn_scaled(path):
     w = synth.scaled(synth.workload("cnn"), B=2, width_div=4)      # 3 -> 16 -> 32 -> 64 channels, 32x32
     _run_and_compare(w, seed=21, steps=2, lam_per_step=0.0, path=path)
@@ -178,7 +229,7 @@ def test_separate_calls_equal_train_step():
     ctx, d, b = net.ctx.ctx, descs[0], net.bufs[0].struct
     ffb.ff_layer_forward(ctx, d, b, w.B, 7, 0)
     ffb.ff_layer_loss_grad(ctx, d, b, w.B, [], [], 0.0, 7, 0)
-    ffb.ff_layer_update(ctx, d, b, w.B, 0)
+    ffb.ff_layer_update(ctx, d, b, w.B, 7, 0)
     ffb.ff_poll_status(ctx, 0)
     st = O.train_step(specs, Ws, X, w.B, 0.0, 7)[0]
     compare_layer(st, net.bufs[0], specs[0], w.B)

@@ -555,6 +555,61 @@ def test_int8_ff_training_learns_and_predicts_separable_classes():
 
 
 # --------------------------------------------------------------------------------------
+# Layer-by-layer (greedy) schedule, Sec. III
+# --------------------------------------------------------------------------------------
+def test_frozen_layers_only_forward_and_the_trained_layer_sees_their_output():
+    g = np.random.default_rng(21)
+    B = 6
+    specs, Ws, X = _net(g, [20, 24, 16, 12], B)
+    for first in range(3):
+        full = O.train_step(specs, Ws, X, B, 0.25, 9)
+        part = O.train_step(specs, Ws, X, B, 0.25, 9, first_trained=first)
+        for l, (a, b) in enumerate(zip(full, part)):
+            # the forward is the same whatever is trained
+            assert np.array_equal(a.Xq, b.Xq) and np.array_equal(a.G, b.G) and np.array_equal(a.Xnext, b.Xnext)
+            if l < first:
+                assert b.coef is None and b.dHq is None and b.W_new is None and b.loss is None
+            else:  # a trained layer's step does not depend on whether earlier layers are trained too
+                assert np.array_equal(a.W_new, b.W_new) and np.array_equal(a.dHq, b.dHq) and a.loss == b.loss
+    # one trained layer at the end, lambda = 0: the stand-alone step on the frozen layers' normalised output
+    x = X
+    for l in range(2):
+        x = O.layer_forward(specs[l], x, Ws[l], B, 9).Xnext
+    alone = O.train_step([specs[2]], [Ws[2]], x, B, 0.0, 9)[0]
+    part = O.train_step(specs, Ws, X, B, 0.0, 9, first_trained=2)[2]
+    assert np.array_equal(alone.W_new, part.W_new) and np.array_equal(alone.Xq, part.Xq)
+
+
+def test_greedy_epoch_trains_one_layer_per_phase_on_trained_predecessors():
+    g = np.random.default_rng(22)
+    B, nb = 6, 3
+    specs, W0, _ = _net(g, [20, 24, 16], B)
+    batches = [g.normal(size=(2 * B, 20)).astype(F32) for _ in range(nb)]
+    seen = []
+    Wt = O.greedy_epoch(specs, W0, batches, B, lambda l, i, st: seen.append((l, i, st)))
+    assert [(l, i) for l, i, _ in seen] == [(l, i) for l in range(2) for i in range(nb)]
+    # the same schedule written out by hand: phase 0 on the raw batches, phase 1 on the forward of the TRAINED layer 0
+    W = [w.copy() for w in W0]
+    for i in range(nb):
+        W[0] = O.train_step([specs[0]], [W[0]], batches[i], B, 0.0, i)[0].W_new
+    assert np.array_equal(W[0], Wt[0]) and not np.array_equal(W0[0], Wt[0])
+    for i in range(nb):
+        x = O.layer_forward(specs[0], batches[i], W[0], B, nb + i).Xnext
+        W[1] = O.train_step([specs[1]], [W[1]], x, B, 0.0, nb + i)[0].W_new
+    assert np.array_equal(W[1], Wt[1])
+    # had phase 1 run on the untrained layer 0 the result would differ (the case the schedule must not be)
+    Wu = W0[1].copy()
+    for i in range(nb):
+        x = O.layer_forward(specs[0], batches[i], W0[0], B, nb + i).Xnext
+        Wu = O.train_step([specs[1]], [Wu], x, B, 0.0, nb + i)[0].W_new
+    assert not np.array_equal(Wu, Wt[1])
+    # layer 0 is left alone during phase 1
+    for l, i, st in seen:
+        if l == 1:
+            assert st[0].W_new is None
+
+
+# --------------------------------------------------------------------------------------
 # Pointwise convolution
 # --------------------------------------------------------------------------------------
 def test_conv1x1_equals_centre_tap_of_conv3x3():
