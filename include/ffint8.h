@@ -284,8 +284,19 @@ ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bu
                      void* cuda_stream);
 
 /* Synchronises `cuda_stream`, reads the device status word and clears it.  Returns FF_OK,
- * FF_ERR_NONFINITE, FF_ERR_DEVICE_TIMEOUT or FF_ERR_CUDA. */
+ * FF_ERR_DEVICE_TIMEOUT (a bounded wait inside a kernel ran out), FF_ERR_NONFINITE (a tensor to be quantised
+ * held Inf / NaN), FF_ERR_RANGE (a label outside its range, or a weight-gradient sum outside INT32: convolution
+ * weight gradients sum over every position of a set, are accumulated in parts that cannot wrap and added in
+ * 64 bits; a weight whose sum leaves INT32 keeps its value) or FF_ERR_CUDA. */
 ff_status ff_poll_status(ff_ctx* ctx, void* cuda_stream);
+
+/* Self-test of the library's failure reporting (the paper has no counterpart).  Every wait inside the
+ * contraction kernels is bounded: when one runs out, the kernel raises a status bit and returns instead of
+ * hanging, and ff_poll_status turns the bit into FF_ERR_DEVICE_TIMEOUT.  This call launches a one-thread kernel
+ * that runs that same wait, with a limit of limit_ns nanoseconds (1 .. 1e9), on a barrier nothing ever arrives
+ * on; the next ff_poll_status must therefore return FF_ERR_DEVICE_TIMEOUT, and the context stays usable.
+ * Nothing else is touched. */
+ff_status ff_selftest_bounded_wait(ff_ctx* ctx, uint64_t limit_ns, void* cuda_stream);
 
 /* Text of the last error returned for this context (host string, valid until the next call). */
 const char* ff_last_error(const ff_ctx* ctx);

@@ -24,7 +24,7 @@ EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", 
            "ff_embed_labels",
            "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step", "ff_train_step_from",
            "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
-           "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict"]
+           "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict", "ff_selftest_bounded_wait"]
 FF_STATIC_LOSS_MAX_SAMPLES = 65536
 FF_K_NAMES = ["absmax", "quantize", "fwd_gemm", "finalize", "normalize", "loss", "dh_quantize",
               "upd_gemm", "raw_gemm", "classify", "dw_fwd", "dw_upd"]
@@ -104,6 +104,7 @@ def load(build_if_missing: bool = True):
     lib.ff_graph_replay_count.restype = u64
     lib.ff_int8_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ff_profile_start.argtypes = [vp]
+    lib.ff_selftest_bounded_wait.argtypes = [vp, u64, vp]
     lib.ff_predict.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, i32, i32, i32, vp, vp, u64, vp]
     lib.ff_loss_coef_static.argtypes = [vp, f32, C.POINTER(vp), C.POINTER(f32), i32, f32, i32, vp, vp, vp, vp, vp,
                                         C.c_char_p, C.c_size_t]
@@ -214,6 +215,10 @@ def ff_predict(ctx, descs_arr, bufs_arr, n_layers: int, B: int, n_classes: int, 
 
 def ff_poll_status(ctx, stream: int = 0):
     _check(ctx, load().ff_poll_status(ctx, stream))
+
+
+def ff_selftest_bounded_wait(ctx, limit_ns: int, stream: int = 0):
+    _check(ctx, load().ff_selftest_bounded_wait(ctx, limit_ns, stream))
 
 
 def ff_launch_count(ctx) -> int:

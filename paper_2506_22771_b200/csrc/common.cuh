@@ -12,6 +12,12 @@ namespace ffi8 {
 constexpr uint32_t ST_NONFINITE = 1u;
 constexpr uint32_t ST_TIMEOUT = 2u;
 constexpr uint32_t ST_BADLABEL = 4u;   // a label outside [0, n_classes) met by the label-embedding kernel
+constexpr uint32_t ST_RANGE = 8u;      // a weight-gradient sum left the INT32 range (Sec. IV-B: INT32 accumulation)
+
+// Longest contraction whose INT8 x INT8 products cannot leave INT32 whatever the codes: 127*127*n <= 2^31 - 1.
+// Longer weight-gradient contractions (convolutions sum over every position of a set) are cut into parts of at
+// most this length; the parts are added in 64 bits and a sum outside INT32 raises ST_RANGE.
+constexpr long long WG_SAFE_LEN = ((1LL << 31) - 1) / (127LL * 127LL);   // 133143
 
 constexpr int ROUND_NEAREST = 0;
 constexpr int ROUND_STOCHASTIC = 1;

@@ -225,9 +225,14 @@ __global__ void __launch_bounds__(DW_THREADS) dwconv3x3_fwd_scalar_kernel(const 
 // A block takes a chunk of output-position blocks (blockIdx.x) for 32 channel groups (blockIdx.y) of one set
 // (blockIdx.z); its 8 warps stride through the chunk, every lane holding the 36 sums of its four channels, and
 // meet in shared memory.  dp4a(x word, dh word with only byte j kept) is the product for channel j alone.
+// The sums are kept in planes [plane][2][C][9]: blocks_per_plane consecutive chunks share a plane, chosen by the
+// host so that no plane sums over more than WG_SAFE_LEN positions (no INT32 sum can wrap; the update kernel adds
+// the planes in 64 bits).
 template <int STRIDE>
 __global__ void __launch_bounds__(DW_THREADS) dwconv3x3_wgrad_kernel(const int8_t* __restrict__ dhq, const int8_t* __restrict__ xq,
-                                                                    int32_t* __restrict__ accW, DwGeom g, int pb_per_block) {
+                                                                    int32_t* __restrict__ accW, DwGeom g, int pb_per_block,
+                                                                    int blocks_per_plane) {
+  accW += (size_t)(blockIdx.x / blocks_per_plane) * 2 * g.C * 9;
   __shared__ int red[32][37];
   const int CG = g.C >> 2;
   const int lane = threadIdx.x & 31, slot = threadIdx.x >> 5;
@@ -290,7 +295,9 @@ __global__ void __launch_bounds__(DW_THREADS) dwconv3x3_wgrad_kernel(const int8_
 // Weight gradient for any channel count: a block per (chunk of positions, set), a thread per channel.
 __global__ void __launch_bounds__(DW_THREADS) dwconv3x3_wgrad_scalar_kernel(const int8_t* __restrict__ dhq,
                                                                            const int8_t* __restrict__ xq,
-                                                                           int32_t* __restrict__ accW, DwGeom g, int rows_per_block) {
+                                                                           int32_t* __restrict__ accW, DwGeom g, int rows_per_block,
+                                                                           int blocks_per_plane) {
+  accW += (size_t)(blockIdx.x / blocks_per_plane) * 2 * g.C * 9;   // planes as in the kernel above
   const int p = blockIdx.z;
   const int row_begin = blockIdx.x * rows_per_block, row_end = min(g.rows_per_pass, row_begin + rows_per_block);
   for (int ch = threadIdx.x; ch < g.C; ch += DW_THREADS) {

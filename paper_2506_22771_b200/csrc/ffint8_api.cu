@@ -41,6 +41,7 @@ struct ff_ctx {
   struct Shard {
     int B_total = 0;
     int row_off = 0;
+    int B_local = 0;
   } shard;
   bool accumulate_only = false;  // weight-gradient contractions leave their INT32 sums in accW_dump, no update
   // captured launch sequences of ff_train_step (ff_set_graph_mode)
@@ -267,7 +268,20 @@ inline long long simt_tiles(const ff_layer_desc& L) {
 }
 // Number of splits the SIMT weight gradient asks for (1 = none): enough that tiles x splits reaches
 // WS_TARGET_ITEMS, at least 1024 contraction elements per split, slabs within WS_SLAB_CAP and within
-// the workspace actually set (`ws_bytes`; pass SIZE_MAX to get the wish).
+// the workspace actually set (`ws_bytes`; pass SIZE_MAX to get the wish) - but never fewer than keep every
+// split's contraction within WG_SAFE_LEN, so that no INT32 partial sum can wrap (simt_min_splits; the caller
+// refuses a workspace too small for that many).
+inline int simt_min_splits(const ff_layer_desc& L, int B) {
+  const long long clen = (long long)B * rows_per_sample(L);
+  const long long safe = WG_SAFE_LEN / SG_BK * SG_BK;  // a split's length is rounded up to contraction blocks
+  return (int)((clen + safe - 1) / safe);
+}
+// One shard of a split batch whose WHOLE contraction can leave INT32: its local sums must pass through the update
+// kernel's range check (a share of the range per shard), so the routes that would write them straight to accW_dump
+// take at least two splits.
+inline bool dp_checks_needed(const ff_ctx* ctx, const ff_layer_desc& L) {
+  return ctx->shard.B_total > 0 && (long long)ctx->shard.B_total * rows_per_sample(L) > WG_SAFE_LEN;
+}
 inline int simt_wgrad_splits(const ff_layer_desc& L, int B, size_t ws_bytes) {
   const long long clen = (long long)B * rows_per_sample(L);
   const long long tiles = simt_tiles(L);
@@ -275,8 +289,10 @@ inline int simt_wgrad_splits(const ff_layer_desc& L, int B, size_t ws_bytes) {
   if (splits > clen / 1024) splits = clen / 1024;
   const size_t per_split = (size_t)2 * L.N * L.K * sizeof(int32_t);
   const size_t room = ws_bytes > WS_BYTES ? ws_bytes - WS_BYTES : 0;
-  const size_t cap = room < WS_SLAB_CAP ? room : WS_SLAB_CAP;
-  if ((size_t)splits * per_split > cap) splits = (long long)(cap / per_split);
+  const int need = simt_min_splits(L, B);
+  if ((size_t)splits * per_split > WS_SLAB_CAP) splits = (long long)(WS_SLAB_CAP / per_split);
+  if (splits < need) splits = need;
+  if ((size_t)splits * per_split > room) splits = (long long)(room / per_split);
   return splits < 2 ? 1 : (int)splits;
 }
 // grid.z the split launch really uses (the last splits can be empty after rounding to blocks)
@@ -297,13 +313,20 @@ ff_status launch_slab_update(ff_ctx* ctx, const int32_t* slabs, int splits, cons
   rule.Var = rule.kind == 1 ? b.Var : nullptr;
   rule.ss = step_ptr(ctx);
   if (!W && !dump) return FF_OK;
+  // Largest magnitude a sum may have.  One shard of a split batch: its share of the INT32 range in proportion to
+  // its rows, so that the sums of all shards cannot wrap when the caller adds them in 32 bits (sufficient, not
+  // necessary: a shard may be refused although the whole batch would have fitted).
+  long long limit = 2147483647LL;
+  if (ctx->accumulate_only && ctx->shard.B_total > 0)
+    limit = limit / ctx->shard.B_total * ctx->shard.B_local;
   if (splits <= 2 && (pitch == 0 || pitch == L.K) && (plane & 3) == 0 && plane >= ((size_t)1 << 18)) {
     const size_t want = (plane / 4 + 255) / 256, cap = (size_t)ctx->sm_count * 8;
-    slab_update_flat_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, W, b.absmax, rule, dump);
+    slab_update_flat_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, W, b.absmax, rule, dump, limit,
+                                                                                 status_ptr(ctx));
   } else {
     const size_t want = (plane + 31) / 32, cap = (size_t)ctx->sm_count * 8;
     slab_update_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(slabs, splits, plane, L.K, pitch ? pitch : L.K, W,
-                                                                            b.absmax, rule, dump);
+                                                                            b.absmax, rule, dump, limit, status_ptr(ctx));
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -333,7 +356,9 @@ inline Im2colPlan im2col_plan(const ff_layer_desc& L, int B, size_t ws_bytes, in
 }
 inline bool im2col_route(ff_ctx* ctx, const ff_layer_desc& L, int B) {
   if (ctx->gemm_path == FF_GEMM_SIMT || !tc_im2col_ok(L)) return false;
-  return im2col_plan(L, B, ctx->workspace_bytes, ctx->sm_count).max_splits >= 1;
+  // room for xi / wi and for as many slabs as keep every split's contraction within WG_SAFE_LEN
+  const int need = tc_min_splits(((long long)B * tc_out_h(L) * tc_out_w(L) + 127) / 128);
+  return im2col_plan(L, B, ctx->workspace_bytes, ctx->sm_count).max_splits >= need;
 }
 // Writes xi (and wi) for layer L from its Xq (and Wq).
 ff_status launch_im2col(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, const Im2colPlan& pl, bool weights,
@@ -394,10 +419,18 @@ ff_status dw_forward(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b
   return FF_OK;
 }
 
-// INT32 sums of both sets into the workspace ([2][C][9], cleared first), then the common reduce / update kernel.
+// Planes of INT32 sums a depthwise layer keeps room for ([plane][2][C][9]).  No plane sums over more than
+// WG_SAFE_LEN positions of a set; a plane holds whole chunks of positions, and a chunk is at most half that
+// long, so every plane but the last is at least half full: twice the minimum, plus one, always suffices.
+inline int dw_planes(const ff_layer_desc& L, int B) {
+  const long long padded = (long long)B * tc_out_h(L) * ((tc_out_w(L) + DW_WB - 1) / DW_WB) * DW_WB;
+  return 2 * (int)((padded + WG_SAFE_LEN - 1) / WG_SAFE_LEN) + 1;
+}
+// INT32 sums of both sets into the workspace ([plane][2][C][9], cleared first), then the common reduce / update kernel.
 ff_status dw_update(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
   const DwGeom g = dw_geom(L, B);
-  const size_t bytes = (size_t)2 * g.C * 9 * sizeof(int32_t);
+  const size_t plane_bytes = (size_t)2 * g.C * 9 * sizeof(int32_t);
+  const size_t bytes = plane_bytes * dw_planes(L, B);
   if (ctx->workspace_bytes < WS_BYTES + bytes)
     return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the depthwise weight-gradient sums");
   int32_t* accW = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
@@ -409,30 +442,36 @@ ff_status dw_update(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b,
     ctx->profiling = was;
     return fail(ctx, FF_ERR_CUDA, "%s", cudaGetErrorString(e));
   }
-  if (L.Cin % 4 == 0) {
-    const int tiles = (g.C / 4 + 31) / 32;
-    const int pb_total = B * g.Ho * g.wblocks;
-    // enough chunks to occupy the device several times over, at least 32 position blocks each
-    int chunks = (ctx->sm_count * 8 + 2 * tiles - 1) / (2 * tiles);
-    const int max_chunks = (pb_total + 31) / 32;
-    if (chunks > max_chunks) chunks = max_chunks;
-    const int per = (pb_total + chunks - 1) / chunks;
-    const dim3 grid((pb_total + per - 1) / per, tiles, 2);
-    if (g.stride == 2)
-      dwconv3x3_wgrad_kernel<2><<<grid, DW_THREADS, 0, st>>>(b.dHq, b.Xq, accW, g, per);
-    else
-      dwconv3x3_wgrad_kernel<1><<<grid, DW_THREADS, 0, st>>>(b.dHq, b.Xq, accW, g, per);
-  } else {
-    int chunks = ctx->sm_count * 4;
-    const int max_chunks = (g.rows_per_pass + 63) / 64;
-    if (chunks > max_chunks) chunks = max_chunks;
-    const int per = (g.rows_per_pass + chunks - 1) / chunks;
-    dwconv3x3_wgrad_scalar_kernel<<<dim3((g.rows_per_pass + per - 1) / per, 1, 2), DW_THREADS, 0, st>>>(b.dHq, b.Xq, accW, g, per);
+  int planes = 1;
+  const bool vec = L.Cin % 4 == 0;
+  const int tiles = vec ? (g.C / 4 + 31) / 32 : 1;
+  // units of the contraction a block strides through: position blocks of DW_WB outputs (vector form) or positions
+  const int units = vec ? B * g.Ho * g.wblocks : g.rows_per_pass;
+  const long long safe_units = vec ? WG_SAFE_LEN / DW_WB : WG_SAFE_LEN, half_units = safe_units / 2;
+  // enough chunks to occupy the device several times over, not shorter than 32 (64) units - and none longer than
+  // half of what a plane may sum over
+  int chunks = vec ? (ctx->sm_count * 8 + 2 * tiles - 1) / (2 * tiles) : ctx->sm_count * 4;
+  const int max_chunks = vec ? (units + 31) / 32 : (units + 63) / 64;
+  if (chunks > max_chunks) chunks = max_chunks;
+  if (chunks < (units + half_units - 1) / half_units) chunks = (int)((units + half_units - 1) / half_units);
+  const int per = (units + chunks - 1) / chunks;
+  const int bpp = (int)(safe_units / per);   // chunks that share a plane (>= 2)
+  const dim3 grid((units + per - 1) / per, tiles, 2);
+  planes = ((int)grid.x + bpp - 1) / bpp;
+  if (planes > dw_planes(L, B)) {
+    ctx->profiling = was;
+    return fail(ctx, FF_ERR_WORKSPACE, "depthwise weight gradient: more planes than planned");
   }
+  if (vec && g.stride == 2)
+    dwconv3x3_wgrad_kernel<2><<<grid, DW_THREADS, 0, st>>>(b.dHq, b.Xq, accW, g, per, bpp);
+  else if (vec)
+    dwconv3x3_wgrad_kernel<1><<<grid, DW_THREADS, 0, st>>>(b.dHq, b.Xq, accW, g, per, bpp);
+  else
+    dwconv3x3_wgrad_scalar_kernel<<<grid, DW_THREADS, 0, st>>>(b.dHq, b.Xq, accW, g, per, bpp);
   ctx->launches++;
   ff_status s = FF_OK;
   if ((e = cudaGetLastError()) != cudaSuccess) s = fail(ctx, FF_ERR_CUDA, "launch: %s", cudaGetErrorString(e));
-  if (s == FF_OK) s = launch_slab_update(ctx, accW, 1, L, b, st, 0);
+  if (s == FF_OK) s = launch_slab_update(ctx, accW, planes, L, b, st, 0);
   ctx->profiling = was;
   return s;
 }
@@ -541,9 +580,13 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     // pointwise convolution: a dense contraction over every position of a set.  With few output tiles it is
     // split into INT32 slabs like the 3x3 case; otherwise the fused dense kernel below takes it.
     int splits = tc_dense_slab_splits(L.N, L.K, (long long)B * R, ctx->sm_count);
+    int need = tc_min_splits(((long long)B * R + 127) / 128);
+    if (dp_checks_needed(ctx, L) && need < 2) need = 2;
+    if (splits < need) splits = need;
     const size_t room = ctx->workspace_bytes > WS_BYTES ? ctx->workspace_bytes - WS_BYTES : 0;
     const size_t per_split = (size_t)2 * L.N * L.K * sizeof(int32_t);
     if ((size_t)splits * per_split > room) splits = (int)(room / per_split);
+    if (splits < need) return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the weight-gradient slabs");
     if (splits >= 2) {
       int32_t* slabs = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
       ProfScope prof(ctx, FF_K_UPD_GEMM, st);
@@ -576,7 +619,7 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     const size_t room = ctx->workspace_bytes > WS_BYTES ? ctx->workspace_bytes - WS_BYTES : 0;
     const size_t per_split = tc_conv_update_slab_bytes(L, 1);
     if ((size_t)splits * per_split > room) splits = (int)(room / per_split);
-    if (splits >= 1) {
+    if (splits >= tc_min_splits((long long)B * R / 128)) {
       int32_t* slabs = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
       ProfScope prof(ctx, FF_K_UPD_GEMM, st);
       int used = 0;
@@ -592,7 +635,13 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     if (ctx->gemm_path == FF_GEMM_TENSOR) return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the weight-gradient slabs");
   }
   const int clen = B * R;
-  const int splits = simt_wgrad_splits(L, B, ctx->workspace_bytes);
+  int splits = simt_wgrad_splits(L, B, ctx->workspace_bytes);
+  if (splits < simt_min_splits(L, B)) return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the weight-gradient slabs");
+  if (dp_checks_needed(ctx, L) && splits < 2) {
+    if (ctx->workspace_bytes < WS_BYTES + (size_t)4 * L.N * L.K * sizeof(int32_t))
+      return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the weight-gradient slabs");
+    splits = 2;
+  }
   if (splits > 1) {
     // few output tiles, long contraction: split it, keep INT32 partial sums in the workspace, add them exactly
     int32_t* slabs = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
@@ -1144,11 +1193,16 @@ ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, s
       const size_t n1 = sp1 >= 2 ? (size_t)sp1 * 2 * layers[l].N * layers[l].K * sizeof(int32_t) : 0;
       if (n1 > need) need = n1;
     }
-    if (layers[l].kind == FF_DWCONV3X3) need = (size_t)2 * layers[l].N * 9 * sizeof(int32_t);
+    if (layers[l].kind == FF_DWCONV3X3) need = (size_t)2 * layers[l].N * 9 * sizeof(int32_t) * dw_planes(layers[l], B);
     if (tc_im2col_ok(layers[l])) {
       const Im2colPlan pl = im2col_plan(layers[l], B, SIZE_MAX, 0);
       const size_t im_need = pl.slab_off - WS_BYTES + (size_t)pl.max_splits * pl.slab_bytes_per_split;
       if (im_need > need) need = im_need;
+    }
+    // a spatial layer of a split batch may be made to take two slabs so that its sums pass the range check
+    if (layers[l].kind == FF_CONV3X3 || layers[l].kind == FF_CONV1X1) {
+      const size_t two = (size_t)4 * layers[l].N * layers[l].K * sizeof(int32_t);
+      if (two > need) need = two;
     }
     if (layers[l].optimizer == FF_OPT_ADAM) need = up256(need) + adam_plane_bytes(layers[l]) + 256;  // sums plane at the tail
     if (need > slab) slab = need;
@@ -1274,9 +1328,11 @@ ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_l
   if ((s = set_step(ctx, step, lambda, true, st)) != FF_OK) return s;
   ctx->shard.B_total = B_total;
   ctx->shard.row_off = row_offset;
+  ctx->shard.B_local = B_local;
   s = dp_phase_body(ctx, layers, bufs, n_layers, B_local, phase, lambda, st, reduce, n_reduce);
   ctx->shard.B_total = 0;
   ctx->shard.row_off = 0;
+  ctx->shard.B_local = 0;
   ctx->accumulate_only = false;
   return s;
 }
@@ -1362,9 +1418,15 @@ ff_status ff_poll_status(ff_ctx* ctx, void* cuda_stream) {
   FF_CUDA(ctx, cudaMemcpyAsync(&h, ctx->workspace, sizeof(h), cudaMemcpyDeviceToHost, st));
   FF_CUDA(ctx, cudaMemsetAsync(ctx->workspace, 0, sizeof(uint32_t), st));
   FF_CUDA(ctx, cudaStreamSynchronize(st));
-  if (h & ST_TIMEOUT) return fail(ctx, FF_ERR_DEVICE_TIMEOUT, "a bounded in-kernel wait ran out");
+  if (h & ST_TIMEOUT) {
+    // a kernel that gave up may have left the loss kernels' completion tickets half counted: have the next call
+    // clear the whole workspace header again
+    ctx->status_zeroed = false;
+    return fail(ctx, FF_ERR_DEVICE_TIMEOUT, "a bounded in-kernel wait ran out");
+  }
   if (h & ST_NONFINITE) return fail(ctx, FF_ERR_NONFINITE, "a tensor to be quantised held Inf or NaN");
   if (h & ST_BADLABEL) return fail(ctx, FF_ERR_RANGE, "a label lay outside [0, n_classes)");
+  if (h & ST_RANGE) return fail(ctx, FF_ERR_RANGE, "a weight-gradient sum left the INT32 range; that weight was not updated");
   return FF_OK;
 }
 
@@ -1397,6 +1459,17 @@ ff_status ff_profile_stop(ff_ctx* ctx, void* cuda_stream, float* ms_per_kernel, 
     ctx->prof_pool.push_back(r.b);
   }
   ctx->prof_recs.clear();
+  return FF_OK;
+}
+
+ff_status ff_selftest_bounded_wait(ff_ctx* ctx, uint64_t limit_ns, void* cuda_stream) {
+  ff_status s = check_ctx(ctx);
+  if (s != FF_OK) return s;
+  if (limit_ns == 0 || limit_ns > 1000000000ull) return fail(ctx, FF_ERR_ARG, "limit_ns must lie in [1, 1e9]");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if ((s = ensure_status(ctx, st)) != FF_OK) return s;
+  bounded_wait_probe_kernel<<<1, 32, 0, st>>>(status_ptr(ctx), limit_ns);
+  FF_LAUNCH_CHECK(ctx);
   return FF_OK;
 }
 

@@ -190,24 +190,36 @@ struct SlabEpilogue {
   }
 };
 
-// Adds the `splits` INT32 slabs of both sets and applies the dequantised SGD update (Sec. IV-B;
+// Adds the `splits` INT32 slabs of both sets and applies the dequantised update (Sec. IV-B;
 // Alg. 1 line 9): W <- W - lr*(float(accP)*cP + float(accN)*cN).  plane = rows*cols elements of W;
 // the slabs may have a wider row pitch (cols <= pitch).  A block covers 32 consecutive elements; its
 // 8 warps take the splits round-robin (coalesced along the elements) and their integer partial
 // sums meet in shared memory.  W == NULL: no update, only the sums are written to accW_dump (dense
 // [2][rows][cols]) - the buffer a data-parallel step adds up over the devices before it updates.
+// No slab can have wrapped (the host keeps every part of a contraction within WG_SAFE_LEN); the slabs are
+// added in 64 bits, and a sum whose magnitude exceeds `limit` (2^31 - 1; a shard of a split batch: its share
+// of that) raises ST_RANGE: that weight is then left as it was and its dumped sums saturate.
+__device__ __forceinline__ bool wg_in_range(long long aP, long long aN, long long limit, uint32_t* status) {
+  const bool ok = aP <= limit && aP >= -limit && aN <= limit && aN >= -limit;
+  if (!ok) atomicOr(status, ST_RANGE);
+  return ok;
+}
+__device__ __forceinline__ int wg_saturate(long long a) {
+  return a > 2147483647LL ? 2147483647 : (a < -2147483647LL ? -2147483647 : (int)a);
+}
 __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane, int cols,
                                                           int pitch, float* __restrict__ W, const float* __restrict__ absmax,
-                                                          UpdateRule rule, int32_t* __restrict__ accW_dump) {
+                                                          UpdateRule rule, int32_t* __restrict__ accW_dump, long long limit,
+                                                          uint32_t* __restrict__ status) {
   const UpdateCoefs uc = update_coefs(rule);
-  __shared__ int part[2][8][32];
+  __shared__ long long part[2][8][32];
   const int lane = threadIdx.x & 31, zl = threadIdx.x >> 5;
   const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
   const float cN = __fmul_rn(scale_of(absmax[4]), scale_of(absmax[1]));
   const size_t splane = plane / cols * pitch;  // elements of one slab
   for (size_t e0 = (size_t)blockIdx.x * 32; e0 < plane; e0 += (size_t)gridDim.x * 32) {
     const size_t e = e0 + lane;
-    int aP = 0, aN = 0;
+    long long aP = 0, aN = 0;
     if (e < plane) {
       const size_t se = pitch == cols ? e : e / cols * pitch + e % cols;
       for (int z = zl; z < splits; z += 8) {
@@ -224,16 +236,17 @@ __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restr
         aP += part[0][k][lane];
         aN += part[1][k][lane];
       }
-      if (W) {
-        const float g = __fadd_rn(__fmul_rn(__int2float_rn(aP), cP), __fmul_rn(__int2float_rn(aN), cN));
+      const bool ok = wg_in_range(aP, aN, limit, status);
+      if (W && ok) {
+        const float g = __fadd_rn(__fmul_rn(__int2float_rn((int)aP), cP), __fmul_rn(__int2float_rn((int)aN), cN));
         float m = rule.Mom ? rule.Mom[e] : 0.0f, v = rule.Var ? rule.Var[e] : 0.0f;
         W[e] = apply_update(rule, uc, W[e], g, m, v);
         if (rule.Mom) rule.Mom[e] = m;
         if (rule.Var) rule.Var[e] = v;
       }
       if (accW_dump) {
-        accW_dump[e] = aP;
-        accW_dump[plane + e] = aN;
+        accW_dump[e] = wg_saturate(aP);
+        accW_dump[plane + e] = wg_saturate(aN);
       }
     }
     __syncthreads();
@@ -244,40 +257,46 @@ __global__ void __launch_bounds__(256) slab_update_kernel(const int32_t* __restr
 // warps, so every thread takes four consecutive elements with 128-bit accesses.
 __global__ void __launch_bounds__(256) slab_update_flat_kernel(const int32_t* __restrict__ slabs, int splits, size_t plane,
                                                                float* __restrict__ W, const float* __restrict__ absmax,
-                                                               UpdateRule rule, int32_t* __restrict__ accW_dump) {
+                                                               UpdateRule rule, int32_t* __restrict__ accW_dump, long long limit,
+                                                               uint32_t* __restrict__ status) {
   const UpdateCoefs uc = update_coefs(rule);
   const float cP = __fmul_rn(scale_of(absmax[3]), scale_of(absmax[0]));
   const float cN = __fmul_rn(scale_of(absmax[4]), scale_of(absmax[1]));
   const size_t n4 = plane >> 2, stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
-    int4 aP = __ldcs(reinterpret_cast<const int4*>(slabs) + i);
-    int4 aN = __ldcs(reinterpret_cast<const int4*>(slabs + plane) + i);
+    const int4 p0 = __ldcs(reinterpret_cast<const int4*>(slabs) + i);
+    const int4 n0 = __ldcs(reinterpret_cast<const int4*>(slabs + plane) + i);
+    long long sP[4] = {p0.x, p0.y, p0.z, p0.w}, sN[4] = {n0.x, n0.y, n0.z, n0.w};
     for (int z = 1; z < splits; ++z) {
       const int4 bP = __ldcs(reinterpret_cast<const int4*>(slabs + (size_t)z * 2 * plane) + i);
       const int4 bN = __ldcs(reinterpret_cast<const int4*>(slabs + ((size_t)z * 2 + 1) * plane) + i);
-      aP.x += bP.x, aP.y += bP.y, aP.z += bP.z, aP.w += bP.w;
-      aN.x += bN.x, aN.y += bN.y, aN.z += bN.z, aN.w += bN.w;
+      sP[0] += bP.x, sP[1] += bP.y, sP[2] += bP.z, sP[3] += bP.w;
+      sN[0] += bN.x, sN[1] += bN.y, sN[2] += bN.z, sN[3] += bN.w;
     }
+    bool ok[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) ok[q] = wg_in_range(sP[q], sN[q], limit, status);
     if (W) {
-      float4 w = reinterpret_cast<const float4*>(W)[i];
-      float4 g;
-      g.x = __fadd_rn(__fmul_rn(__int2float_rn(aP.x), cP), __fmul_rn(__int2float_rn(aN.x), cN));
-      g.y = __fadd_rn(__fmul_rn(__int2float_rn(aP.y), cP), __fmul_rn(__int2float_rn(aN.y), cN));
-      g.z = __fadd_rn(__fmul_rn(__int2float_rn(aP.z), cP), __fmul_rn(__int2float_rn(aN.z), cN));
-      g.w = __fadd_rn(__fmul_rn(__int2float_rn(aP.w), cP), __fmul_rn(__int2float_rn(aN.w), cN));
-      float4 m = rule.Mom ? reinterpret_cast<const float4*>(rule.Mom)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
-      float4 v = rule.Var ? reinterpret_cast<const float4*>(rule.Var)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
-      w.x = apply_update(rule, uc, w.x, g.x, m.x, v.x);
-      w.y = apply_update(rule, uc, w.y, g.y, m.y, v.y);
-      w.z = apply_update(rule, uc, w.z, g.z, m.z, v.z);
-      w.w = apply_update(rule, uc, w.w, g.w, m.w, v.w);
-      if (rule.Mom) reinterpret_cast<float4*>(rule.Mom)[i] = m;
-      if (rule.Var) reinterpret_cast<float4*>(rule.Var)[i] = v;
-      reinterpret_cast<float4*>(W)[i] = w;
+      float4 w4 = reinterpret_cast<const float4*>(W)[i];
+      float4 m4 = rule.Mom ? reinterpret_cast<const float4*>(rule.Mom)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 v4 = rule.Var ? reinterpret_cast<const float4*>(rule.Var)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+      float* w = reinterpret_cast<float*>(&w4);
+      float* m = reinterpret_cast<float*>(&m4);
+      float* v = reinterpret_cast<float*>(&v4);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (!ok[q]) continue;
+        const float g = __fadd_rn(__fmul_rn(__int2float_rn((int)sP[q]), cP), __fmul_rn(__int2float_rn((int)sN[q]), cN));
+        w[q] = apply_update(rule, uc, w[q], g, m[q], v[q]);
+      }
+      if (rule.Mom) reinterpret_cast<float4*>(rule.Mom)[i] = m4;
+      if (rule.Var) reinterpret_cast<float4*>(rule.Var)[i] = v4;
+      reinterpret_cast<float4*>(W)[i] = w4;
     }
     if (accW_dump) {
-      reinterpret_cast<int4*>(accW_dump)[i] = aP;
-      reinterpret_cast<int4*>(accW_dump + plane)[i] = aN;
+      reinterpret_cast<int4*>(accW_dump)[i] = make_int4(wg_saturate(sP[0]), wg_saturate(sP[1]), wg_saturate(sP[2]), wg_saturate(sP[3]));
+      reinterpret_cast<int4*>(accW_dump + plane)[i] =
+          make_int4(wg_saturate(sN[0]), wg_saturate(sN[1]), wg_saturate(sN[2]), wg_saturate(sN[3]));
     }
   }
 }

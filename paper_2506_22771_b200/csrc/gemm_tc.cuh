@@ -162,7 +162,8 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 }
 // Bounded wait: false when the time limit ran out or another role already gave up.
 template <bool CLUSTER = false>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          unsigned long long limit_ns = TC_WAIT_NS) {
   auto poll = [&]() { return CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
   if (poll()) return true;
   const unsigned long long t0 = globaltimer_ns();
@@ -170,10 +171,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   while (!poll()) {
     if ((++spins & 0xFFu) == 0) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > TC_WAIT_NS) return false;
+      if (globaltimer_ns() - t0 > limit_ns) return false;
     }
   }
   return true;
+}
+// Self-test of the bounded wait: one thread waits, with the limit given, on a barrier that nothing ever arrives
+// on.  The wait must give up, the thread raises ST_TIMEOUT exactly as the contraction kernels' roles do, and the
+// kernel returns normally.  No copy, no tensor memory, no other thread is involved.
+__global__ void bounded_wait_probe_kernel(uint32_t* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_word;
+  if (threadIdx.x == 0) {
+    abort_word = 0u;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait<false>(smem_u32(&bar), 0u, &abort_word, limit_ns)) atomicOr(status, ST_TIMEOUT);
+  }
 }
 // Tiled TMA loads into this CTA's shared memory.  NCTA = 2: `bar` is a shared::cluster address and may
 // name a barrier of the other CTA of the pair (the cta_group::2 form allows that); no multicast.
@@ -1127,9 +1141,14 @@ inline bool tc_update_supported(const ff_layer_desc& L, int B) {
   return tc_tn_ok(L.N, L.K, (long long)B * (L.kind == FF_LINEAR ? 1 : tc_out_h(L) * tc_out_w(L)));
 }
 
+// Fewest splits of a contraction of `kblocks` blocks of 128 such that no split is longer than WG_SAFE_LEN,
+// i.e. no INT32 partial sum can wrap whatever the codes (Sec. IV-B: INT32 accumulation).
+constexpr int TC_SAFE_KBLOCKS = (int)(WG_SAFE_LEN / 128);   // 1040 blocks = 133120 contraction elements
+inline int tc_min_splits(long long kblocks) { return (int)((kblocks + TC_SAFE_KBLOCKS - 1) / TC_SAFE_KBLOCKS); }
+
 // Split count of the convolution weight gradient (its output N x 9*Cin has few tiles, its contraction
 // runs over every output position of a set): as many splits as keep every SM (pair) busy with one
-// work item, at least 8 contraction blocks each.  sm_count <= 0: assume 148.
+// work item, at least 8 contraction blocks each, and at least tc_min_splits.  sm_count <= 0: assume 148.
 inline int tc_conv_update_splits(const ff_layer_desc& L, int B, int sm_count, int force_ncta) {
   if (sm_count <= 0) sm_count = 148;
   const int ncta = force_ncta ? force_ncta : (L.N > TC_BM ? 2 : 1);
@@ -1137,6 +1156,7 @@ inline int tc_conv_update_splits(const ff_layer_desc& L, int B, int sm_count, in
   const long long kblocks = (long long)B * tc_out_h(L) * tc_out_w(L) / 128;
   long long splits = (sm_count / ncta) / tiles;
   if (splits > kblocks / 8) splits = kblocks / 8;
+  if (splits < tc_min_splits(kblocks)) splits = tc_min_splits(kblocks);
   return splits < 1 ? 1 : (int)splits;
 }
 inline size_t tc_conv_update_slab_bytes(const ff_layer_desc& L, int splits) {
@@ -1298,6 +1318,7 @@ inline int tc_dense_slab_splits(int N, int kcols, long long rows_per_pass, int s
   const long long kblocks = (rows_per_pass + 127) / 128;
   long long splits = sm_count / tiles;
   if (splits > kblocks / 8) splits = kblocks / 8;
+  if (splits < tc_min_splits(kblocks)) splits = tc_min_splits(kblocks);
   return splits < 1 ? 1 : (int)splits;
 }
 inline ff_status tc_dense_update_slab(TcState& t, const int8_t* dHq, int N, const int8_t* xi, int kcols, int rows_per_pass,

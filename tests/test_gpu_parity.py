@@ -739,3 +739,34 @@ def test_explicit_row_pitch_and_its_checks():
             net.train_step(0.0, 1)
         setattr(net.bufs_arr[1], field, old)
     net.close()
+
+
+def test_bounded_wait_runs_out_is_reported_and_leaves_the_context_usable():
+    # the wait every role of the contraction kernels uses, run on a barrier nothing arrives on with a 1 ms limit:
+    # the kernel returns, the status word says so, and the steps before and after are bit-exact as ever
+    import time
+    w = synth.scaled(synth.workload("tiny_mlp"), B=40, width_div=2)
+    specs, descs = specs_and_descs(w.layers, 4)
+    Ws = synth.make_weights(w, 4)
+    X = synth.make_batch(w, 4)
+    net = GpuNet(descs, w.B, Ws)
+    net.set_input(X)
+    ctx = net.ctx.ctx
+    for step in range(2):
+        if step == 1:
+            t0 = time.time()
+            ffb.ff_selftest_bounded_wait(ctx, 1_000_000, 0)
+            with pytest.raises(ffb.FFError) as e:
+                ffb.ff_poll_status(ctx, 0)
+            assert e.value.code == ffb.FF_ERR_DEVICE_TIMEOUT and "wait" in str(e.value)
+            assert time.time() - t0 < 5.0
+            ffb.ff_poll_status(ctx, 0)            # reported once, then clear
+        net.train_step(0.0, step)
+        states = O.train_step(specs, Ws, X, w.B, 0.0, step)
+        for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
+            compare_layer(st, b, sp, w.B, tag=f"step{step}/layer{l}/")
+        Ws = [st.W_new for st in states]
+    with pytest.raises(ffb.FFError) as e:
+        ffb.ff_selftest_bounded_wait(ctx, 0, 0)
+    assert e.value.code == ffb.FF_ERR_ARG
+    net.close()
