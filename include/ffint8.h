@@ -98,6 +98,10 @@ typedef struct {
                         /* is max-pooled 2x2 with stride 2 over the positions, [M,Ho/2,Wo/2,N]      */
                         /* (spatial layers with even Ho, Wo; goodness, loss and g^Y stay at full    */
                         /* resolution - no gradient passes through the pooling, Sec. IV-B)          */
+  float skip_scale;     /* weight of the skip path: with ff_layer_bufs.Skip given, the layer hands         */
+                        /* z = y*tau/(sqrt(G)+eps) + skip_scale*Skip to the next layer (a residual block,   */
+                        /* Sec. IV-C / Table II; each operation rounded once).  The layer's own goodness,   */
+                        /* loss and gradient are untouched: only what the next layer sees changes.          */
 } ff_layer_desc;
 
 /* Device buffers of one layer (host struct of device pointers; caller-owned). */
@@ -123,6 +127,10 @@ typedef struct {
   float* Mom;        /* [N,K] FP32 in/out momentum buffer; needed (and touched) only if momentum != 0 */
                      /* or the optimiser is Adam (first moment)                                */
   float* Var;        /* [N,K] FP32 in/out second-moment buffer; Adam only                      */
+  const float* Skip; /* [M*R,N] FP32 in, nullable: skip path of a residual block, added (times skip_scale) to the */
+                     /* normalised output - typically the X of the block's first layer or the Xnext of the layer  */
+                     /* before it.  Needs Xnext (the sum is written there, then quantised for the next layer) and */
+                     /* no pooling.  Must not alias Xnext.                                                       */
   int32_t ld_xq;     /* linear layers only: row pitch of Xq in bytes, 0 = K (dense).  A pitch that is a */
   int32_t ld_dhq;    /* multiple of 128 keeps every TMA box row of the contractions aligned when K (N  */
                      /* for dHq) is not: >= the row length, a multiple of 16.  All rows x pitch bytes  */

@@ -77,6 +77,9 @@ class LayerSpec:
     beta2: float = 0.999  # Adam only
     adam_eps: float = 1e-8
     pool: int = 1         # 2: the normalised output is max-pooled 2x2 (stride 2) before it feeds the next layer
+    skip_from: int = -1   # >= 0: the (normalised, float32) INPUT of layer skip_from of the same call is added to this
+                          # layer's normalised output before it feeds the next layer (a residual block's skip path)
+    skip_scale: float = 1.0   # weight of the skip path
 
     @property
     def out_hw(self):
@@ -434,8 +437,24 @@ def _pass_rows(v_pos, v_neg, B):
     return np.concatenate([np.full(B, v_pos, dtype=F32), np.full(B, v_neg, dtype=F32)])
 
 
-def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: int) -> LayerState:
-    """Quantise A and W, INT8 MAC, dequantise + ReLU, goodness, normalised output."""
+def add_skip(xhat: np.ndarray, skip: np.ndarray, scale: float) -> np.ndarray:
+    """Output of a residual block: z = xhat + scale*skip, element by element (one float32 multiply, one float32 add).
+    xhat is the last layer's length-normalised output, skip the block's (length-normalised) input, so both have a
+    fixed length per sample and their sum carries no goodness of either on to the next layer.  The paper trains
+    residual networks (Sec. IV-C: the look-ahead exists so that the layers of such a block are trained together;
+    Table II) but does not say how the sum is formed in FF training; this reading keeps every layer's own goodness
+    ||y||^2 (Sec. III) untouched - the skip path changes what the NEXT layer sees, nothing else - and needs no
+    reduction whose order is free.  No gradient passes through it (there is no input gradient, Sec. IV-B)."""
+    xhat = np.asarray(xhat, dtype=F32)
+    skip = np.asarray(skip, dtype=F32)
+    if xhat.size != skip.size or xhat.shape[0] != skip.shape[0]:
+        raise ValueError("skip tensor and layer output differ in shape")
+    return xhat + F32(scale) * skip.reshape(xhat.shape)
+
+
+def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: int,
+                  skip: Optional[np.ndarray] = None) -> LayerState:
+    """Quantise A and W, INT8 MAC, dequantise + ReLU, goodness, normalised output (+ the skip path, if any)."""
     st = LayerState()
     X = np.asarray(X, dtype=F32)
     W = np.asarray(W, dtype=F32)
@@ -461,6 +480,10 @@ def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: i
         if spec.kind == KIND_LINEAR or spec.out_hw[0] % 2 or spec.out_hw[1] % 2:
             raise ValueError("pooling needs a spatial layer with even output extents")
         st.Xnext = maxpool2x2(st.Xnext)
+    if skip is not None:
+        if spec.pool == 2:
+            raise ValueError("a pooled output takes no skip path")
+        st.Xnext = add_skip(st.Xnext, skip, spec.skip_scale)
     return st
 
 
@@ -558,11 +581,14 @@ def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: i
     states carry no coef, dHq or W_new).  This is one step of the layer-by-layer schedule of Sec. III,
     where a layer is trained on the output of the already trained layers before it."""
     states = []
-    x = X
+    inputs = [X]                       # inputs[l] = float32 input of layer l (the skip paths' sources)
     for spec, W in zip(specs, Ws):
-        st = layer_forward(spec, x, W, B, step)
+        if spec.skip_from >= len(inputs):
+            raise ValueError("skip_from must name this layer or an earlier one")
+        skip = inputs[spec.skip_from] if spec.skip_from >= 0 else None
+        st = layer_forward(spec, inputs[-1], W, B, step, skip)
         states.append(st)
-        x = st.Xnext
+        inputs.append(st.Xnext)
     for l, (spec, W) in enumerate(zip(specs, Ws)):
         if l < first_trained:
             continue
@@ -607,12 +633,13 @@ def predict(specs: List[LayerSpec], Ws: List[np.ndarray], X_cand: np.ndarray, B:
     if n_classes % 2 or n_classes <= 0:
         raise ValueError("n_classes must be even and positive")
     half = n_classes * B // 2
-    x = np.asarray(X_cand, dtype=F32)
+    inputs = [np.asarray(X_cand, dtype=F32)]
     states = []
     for spec, W in zip(specs, Ws):
-        st = layer_forward(spec, x, W, half, step)
+        skip = inputs[spec.skip_from] if spec.skip_from >= 0 else None
+        st = layer_forward(spec, inputs[-1], W, half, step, skip)
         states.append(st)
-        x = st.Xnext
+        inputs.append(st.Xnext)
     total = np.zeros(n_classes * B, dtype=F32)
     for st in states[first_counted:]:
         total = total + st.G.astype(F32)          # float32 additions in layer order

@@ -36,13 +36,14 @@ class ff_layer_desc(C.Structure):
                 ("round_x", C.c_int32), ("round_w", C.c_int32), ("round_dh", C.c_int32),
                 ("theta", C.c_float), ("lr", C.c_float), ("tau", C.c_float), ("eps", C.c_float),
                 ("seed", C.c_uint64), ("stride", C.c_int32), ("momentum", C.c_float),
-                ("optimizer", C.c_int32), ("beta2", C.c_float), ("adam_eps", C.c_float), ("pool", C.c_int32)]
+                ("optimizer", C.c_int32), ("beta2", C.c_float), ("adam_eps", C.c_float), ("pool", C.c_int32),
+                ("skip_scale", C.c_float)]
 
 
 class ff_layer_bufs(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
                 ("W", "X", "Y", "G", "Xnext", "Xq", "Wq", "dHq", "absmax", "S", "rowmax", "coef",
-                 "loss", "acc_dump", "accW_dump", "Mom", "Var")] + [("ld_xq", C.c_int32), ("ld_dhq", C.c_int32)]
+                 "loss", "acc_dump", "accW_dump", "Mom", "Var", "Skip")] + [("ld_xq", C.c_int32), ("ld_dhq", C.c_int32)]
 
 
 FF_DP_MAX_REDUCE = 96
@@ -273,7 +274,7 @@ def make_desc(cfg, index: int, seed: int, round_x=FF_ROUND_STOCHASTIC, round_w=F
     return ff_layer_desc(cfg.kind, cfg.K, cfg.N, cfg.H, cfg.Wd, cfg.Cin, index, round_x, round_w, round_dh,
                          cfg.theta, cfg.lr, cfg.tau, cfg.eps, seed, getattr(cfg, "stride", 1), getattr(cfg, "momentum", 0.0),
                          getattr(cfg, "optimizer", 0), getattr(cfg, "beta2", 0.999), getattr(cfg, "adam_eps", 1e-8),
-                         getattr(cfg, "pool", 1))
+                         getattr(cfg, "pool", 1), getattr(cfg, "skip_scale", 1.0))
 
 
 class LayerBuffers:
@@ -314,7 +315,7 @@ class LayerBuffers:
         self.struct = ff_layer_bufs(p(self.W), p(self.X), p(self.Y), p(self.G), p(self.Xnext), p(self.Xq),
                                     p(self.Wq), p(self.dHq), p(self.absmax), p(self.S), p(self.rowmax),
                                     p(self.coef), p(self.loss), p(self.acc_dump), p(self.accW_dump), p(self.Mom), p(self.Var),
-                                    self.ld_xq if self.ld_xq != kin else 0, self.ld_dhq if self.ld_dhq != desc.N else 0)
+                                    None, self.ld_xq if self.ld_xq != kin else 0, self.ld_dhq if self.ld_dhq != desc.N else 0)
 
 
 class Context:

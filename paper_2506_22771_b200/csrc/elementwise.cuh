@@ -193,9 +193,12 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_multi_kernel(const QuantJ
 // max_n y*r = (float(rowmax)*c)*r because each rounded multiply by a fixed non-negative factor is
 // monotone.  a_next (and a_next2, if non-NULL) receive it by atomicMax; both must be zero before.
 // ---------------------------------------------------------------------------------------------
+// write_range = 0: only G is written (the layer's output takes a skip path, so its range is found by the kernel
+// that forms the sum).
 __global__ void __launch_bounds__(EW_THREADS) finalize_goodness_kernel(
     const unsigned long long* __restrict__ S, const int32_t* __restrict__ rowmax, const float* __restrict__ absmax,
-    int B, float tau, float eps, float* __restrict__ G, float* __restrict__ a_next, float* __restrict__ a_next2) {
+    int B, float tau, float eps, float* __restrict__ G, float* __restrict__ a_next, float* __restrict__ a_next2,
+    int write_range = 1) {
   const int p = blockIdx.y;
   const float c = __fmul_rn(scale_of(absmax[p]), scale_of(absmax[2]));
   const double c2 = __dmul_rn((double)c, (double)c);
@@ -209,7 +212,7 @@ __global__ void __launch_bounds__(EW_THREADS) finalize_goodness_kernel(
     mx = max(mx, __float_as_uint(xm));
   }
   mx = block_max_u32(mx);
-  if (threadIdx.x == 0 && mx) {
+  if (threadIdx.x == 0 && mx && write_range) {
     atomicMax(reinterpret_cast<uint32_t*>(a_next) + p, mx);
     if (a_next2) atomicMax(reinterpret_cast<uint32_t*>(a_next2) + p, mx);
   }
@@ -333,6 +336,61 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
       float v = __fmul_rn(Y[e], r);
       if (xnext) xnext[e] = v;
       if (xq) xq[PAD ? padded(e, rp) : e] = (int8_t)quant_one<MODE>(v, inv, (uint32_t)e + bias, key);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Output of a residual block: z = y*r + scale*skip per element (r = tau/(sqrt(G)+eps) of the sample; one rounding
+// per operation), written as FP32, and the per-set range max|z| (a maximum: exact, order-free) for the next
+// layer's quantiser into a_next[p] and, if given, a_next2[p] (both zero before).  The sum has no range short-cut,
+// so the next layer's INT8 input is made from xnext by the ordinary quantiser afterwards.  The paper trains
+// residual networks (Sec. IV-C, Table II) without saying how the sum is formed under FF; here the skip path only
+// changes what the next layer sees - the layer's own goodness stays ||y||^2 (Sec. III).   grid = (blocks, 2)
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS) normalize_skip_kernel(const float* __restrict__ Y, const float* __restrict__ G,
+                                                                    float tau, float eps, size_t per_sample, size_t per_pass,
+                                                                    const float* __restrict__ skip, float scale,
+                                                                    float* __restrict__ xnext, float* __restrict__ a_next,
+                                                                    float* __restrict__ a_next2, uint32_t* __restrict__ status) {
+  const size_t base = (size_t)blockIdx.y * per_pass;
+  const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)xnext) & 15) == 0) &&
+                   ((((uintptr_t)skip) & 15) == 0);
+  const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
+  uint32_t mx = 0u;
+  if (vec) {
+    const uint32_t n4 = (uint32_t)(per_pass >> 2);
+    const float* Gp = G + (uint32_t)(base / per_sample);
+    SampleCursor cur(tid, stride, (uint32_t)(per_sample >> 2));
+    for (uint32_t i = tid; i < n4; i += stride, cur.advance()) {
+      const size_t e = base + ((size_t)i << 2);
+      const float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(__ldg(Gp + cur.sample)), eps));
+      const float4 y = __ldg(reinterpret_cast<const float4*>(Y + e));
+      const float4 s = __ldcs(reinterpret_cast<const float4*>(skip + e));
+      float4 z;
+      z.x = __fadd_rn(__fmul_rn(y.x, r), __fmul_rn(scale, s.x));
+      z.y = __fadd_rn(__fmul_rn(y.y, r), __fmul_rn(scale, s.y));
+      z.z = __fadd_rn(__fmul_rn(y.z, r), __fmul_rn(scale, s.z));
+      z.w = __fadd_rn(__fmul_rn(y.w, r), __fmul_rn(scale, s.w));
+      *reinterpret_cast<float4*>(xnext + e) = z;
+      mx = max(mx, max(max(__float_as_uint(z.x) & 0x7fffffffu, __float_as_uint(z.y) & 0x7fffffffu),
+                       max(__float_as_uint(z.z) & 0x7fffffffu, __float_as_uint(z.w) & 0x7fffffffu)));
+    }
+  } else {
+    for (size_t i = tid; i < per_pass; i += stride) {
+      const size_t e = base + i;
+      const float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(G[(uint32_t)e / (uint32_t)per_sample]), eps));
+      const float z = __fadd_rn(__fmul_rn(Y[e], r), __fmul_rn(scale, skip[e]));
+      xnext[e] = z;
+      mx = max(mx, __float_as_uint(z) & 0x7fffffffu);
+    }
+  }
+  mx = block_max_u32(mx);
+  if (threadIdx.x == 0) {
+    if (mx >= 0x7f800000u) atomicOr(status, ST_NONFINITE);   // a skip tensor that held Inf / NaN
+    if (mx) {
+      atomicMax(reinterpret_cast<uint32_t*>(a_next) + blockIdx.y, mx);
+      if (a_next2) atomicMax(reinterpret_cast<uint32_t*>(a_next2) + blockIdx.y, mx);
     }
   }
 }

@@ -176,14 +176,16 @@ ff_status check_bufs(ff_ctx* ctx, const ff_layer_bufs* b, bool need_x) {
     if (!p) return fail(ctx, FF_ERR_ARG, "a required device pointer is NULL");
   if (need_x && !b->X) return fail(ctx, FF_ERR_ARG, "X is NULL");
   const void* all[] = {b->W, b->X, b->Y, b->G, b->Xnext, b->Xq, b->Wq, b->dHq, b->absmax, b->S, b->rowmax, b->coef,
-                       b->loss, b->acc_dump, b->accW_dump, b->Mom, b->Var};
+                       b->loss, b->acc_dump, b->accW_dump, b->Mom, b->Var, b->Skip};
   for (const void* p : all)
     if (p && !aligned16(p)) return fail(ctx, FF_ERR_ALIGN, "a device pointer is not 16-byte aligned");
+  if (b->Skip && (!b->Xnext || b->Skip == b->Xnext)) return fail(ctx, FF_ERR_ARG, "a skip path needs Xnext, distinct from Skip");
   return FF_OK;
 }
 
 // Row pitches of the INT8 tensors: linear layers only, at least the row length, multiples of 16 bytes.
 ff_status check_pitches(ff_ctx* ctx, const ff_layer_desc* L, const ff_layer_bufs* b) {
+  if (b->Skip && L->pool == 2) return fail(ctx, FF_ERR_ARG, "a pooled output takes no skip path");
   if (!b->ld_xq && !b->ld_dhq) return FF_OK;
   if (L->kind != FF_LINEAR) return fail(ctx, FF_ERR_ARG, "row pitches are for linear layers only");
   if (b->ld_xq && (b->ld_xq < L->K || b->ld_xq % 16)) return fail(ctx, FF_ERR_ARG, "ld_xq must be >= K and a multiple of 16");
@@ -700,7 +702,7 @@ ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     ProfScope prof(ctx, FF_K_FINALIZE, st);
     finalize_goodness_kernel<<<dim3(ew_blocks(ctx, B, 1), 2), EW_THREADS, 0, st>>>(
         reinterpret_cast<const unsigned long long*>(b.S), b.rowmax, b.absmax, B, L.tau, L.eps, b.G,
-        b.absmax + FF_A_XNEXT_POS, a_next2);
+        b.absmax + FF_A_XNEXT_POS, a_next2, b.Skip ? 0 : 1);
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -736,8 +738,33 @@ ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
 // Normalised output of layer `L` as FP32 (b.Xnext, if non-NULL) and / or as the INT8 input of the
 // next layer (xq_next, nullable; rounding keyed by the next layer).
 ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, int8_t* xq_next,
-                           const ff_layer_desc* next, cudaStream_t st, int ld_next = 0) {
+                           const ff_layer_desc* next, cudaStream_t st, int ld_next = 0, float* a_next2 = nullptr) {
   if (!b.Xnext && !xq_next) return FF_OK;
+  if (b.Skip) {
+    // residual block: the sum of the normalised output and the skip tensor goes to Xnext in FP32 together with its
+    // range (it has no short-cut), then the ordinary quantiser makes the next layer's INT8 input from it
+    if (ctx->shard.B_total) return fail(ctx, FF_ERR_ARG, "a data-parallel step takes no skip paths");
+    const size_t per_sample = (size_t)rows_per_sample(L) * L.N, per_pass = per_sample * B;
+    const dim3 grid(ew_blocks(ctx, per_pass / 4 + 1), 2);
+    {
+      ProfScope prof(ctx, FF_K_NORMALIZE, st);
+      normalize_skip_kernel<<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Skip, L.skip_scale, b.Xnext,
+                                                        b.absmax + FF_A_XNEXT_POS, a_next2, status_ptr(ctx));
+    }
+    FF_LAUNCH_CHECK(ctx);
+    if (!xq_next) return FF_OK;
+    ProfScope prof(ctx, FF_K_QUANTIZE, st);
+    const KeySpec key = make_key_spec(next->seed, ROLE_X, next->index, step_ptr(ctx));
+    const RowPad rp = row_pad((int)per_sample, ld_next);
+    if (next->round_x == FF_ROUND_NEAREST_EVEN)
+      quantize_kernel<ROUND_NEAREST><<<grid, EW_THREADS, 0, st>>>(b.Xnext, xq_next, per_pass, b.absmax + FF_A_XNEXT_POS, key, nullptr,
+                                                                 nullptr, 0, uint2{0u, 0u}, rp);
+    else
+      quantize_kernel<ROUND_STOCHASTIC><<<grid, EW_THREADS, 0, st>>>(b.Xnext, xq_next, per_pass, b.absmax + FF_A_XNEXT_POS, key, nullptr,
+                                                                    nullptr, 0, uint2{0u, 0u}, rp);
+    FF_LAUNCH_CHECK(ctx);
+    return FF_OK;
+  }
   if (ld_next && L.pool == 2) return fail(ctx, FF_ERR_ARG, "a pooled output cannot feed a layer with a padded Xq");
   const size_t per_sample = (size_t)rows_per_sample(L) * L.N;
   const size_t per_pass = per_sample * B;
@@ -907,7 +934,8 @@ ff_status forward_all(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_b
     if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st, true)) != FF_OK)
       return s;
     if ((s = normalize_output(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].Xq : nullptr,
-                              feeds_next ? &layers[l + 1] : nullptr, st, feeds_next ? bufs[l + 1].ld_xq : 0)) != FF_OK)
+                              feeds_next ? &layers[l + 1] : nullptr, st, feeds_next ? bufs[l + 1].ld_xq : 0,
+                              feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr)) != FF_OK)
       return s;
   }
   return FF_OK;
@@ -1319,6 +1347,7 @@ ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_l
     if ((s = check_layer(ctx, &layers[l], B_total)) != FF_OK) return s;
     if (l > 0 && bufs[l].X) return fail(ctx, FF_ERR_ARG, "a data-parallel step takes chained layers (X of layers > 0 NULL)");
     if (!bufs[l].accW_dump) return fail(ctx, FF_ERR_ARG, "a data-parallel step needs accW_dump of every layer");
+    if (bufs[l].Skip) return fail(ctx, FF_ERR_ARG, "a data-parallel step takes no skip paths");
     if (layers[l].momentum != 0.0f && !bufs[l].Mom) return fail(ctx, FF_ERR_ARG, "momentum != 0 needs the buffer Mom");
     if (layers[l].optimizer == FF_OPT_ADAM && (!bufs[l].Mom || !bufs[l].Var))
       return fail(ctx, FF_ERR_ARG, "the Adam update needs the buffers Mom and Var");

@@ -34,6 +34,8 @@ class LayerCfg:
     beta2: float = 0.999
     adam_eps: float = 1e-8
     pool: int = 1           # 2: 2x2 max pooling of the normalised output before the next layer
+    skip_from: int = -1     # >= 0: the input of that layer is added to this layer's normalised output (residual block)
+    skip_scale: float = 1.0
 
 
 @dataclass

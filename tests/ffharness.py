@@ -17,14 +17,17 @@ def specs_and_descs(layers, seed, round_x=1, round_w=0, round_dh=1):
         specs.append(O.LayerSpec(l.kind, l.K, l.N, l.theta, l.lr, l.tau, l.eps, l.H, l.Wd, l.Cin,
                                  round_x, round_w, round_dh, seed, i, getattr(l, "stride", 1),
                                  getattr(l, "momentum", 0.0), getattr(l, "optimizer", 0), getattr(l, "beta2", 0.999),
-                                 getattr(l, "adam_eps", 1e-8), getattr(l, "pool", 1)))
+                                 getattr(l, "adam_eps", 1e-8), getattr(l, "pool", 1), getattr(l, "skip_from", -1),
+                                 getattr(l, "skip_scale", 1.0)))
         descs.append(ffb.make_desc(l, i, seed, round_x, round_w, round_dh))
     return specs, descs
 
 
 class GpuNet:
     def __init__(self, descs, B, Ws, dumps=True, xnext=True, chain=True, gemm_path=ffb.FF_GEMM_AUTO, graph=False,
-                 pad_rows=True):
+                 pad_rows=True, skips=None):
+        """skips[l] >= 0: layer l's output takes a skip path from the FP32 input of layer skips[l] (the network input for
+        layer 0, else the Xnext of the layer before it)."""
         import torch
         self.torch = torch
         self.dev = torch.device("cuda:0")
@@ -41,6 +44,10 @@ class GpuNet:
                      for i, d in enumerate(descs)]
         for b, W in zip(self.bufs, Ws):
             b.W.copy_(torch.from_numpy(W))
+        for l, src in enumerate(skips or []):
+            if src >= 0:
+                t = self.bufs[0].X if src == 0 else self.bufs[src - 1].Xnext
+                self.bufs[l].struct.Skip = t.data_ptr()
         self.descs_arr = (ffb.ff_layer_desc * len(descs))(*descs)
         self.bufs_arr = (ffb.ff_layer_bufs * len(descs))(*[b.struct for b in self.bufs])
 

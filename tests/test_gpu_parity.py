@@ -65,7 +65,8 @@ def _run_and_compare(w, seed, steps, lam_per_step, path, rounding=(1, 0, 1), cha
     specs, descs = specs_and_descs(w.layers, seed, *rounding)
     Ws = synth.make_weights(w, seed)
     X = synth.make_batch(w, seed)
-    net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path, graph=graph, pad_rows=pad_rows)
+    net = GpuNet(descs, w.B, Ws, dumps=True, xnext=True, chain=chain, gemm_path=path, graph=graph, pad_rows=pad_rows,
+                 skips=[s.skip_from for s in specs])
     if pad_fill is not None:      # whatever the padding bytes of the pitched rows hold must reach no result
         for b in net.bufs:
             b._Xq_store.fill_(pad_fill)
@@ -768,5 +769,67 @@ def test_bounded_wait_runs_out_is_reported_and_leaves_the_context_usable():
         Ws = [st.W_new for st in states]
     with pytest.raises(ffb.FFError) as e:
         ffb.ff_selftest_bounded_wait(ctx, 0, 0)
+    assert e.value.code == ffb.FF_ERR_ARG
+    net.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("graph", [False, True])
+def test_residual_block_dense(path, graph):
+    # a look-ahead block of three layers whose last one adds the block's input to its normalised output (the skip
+    # path of a residual block), followed by a fourth layer that sees the sum; lambda > 0 so that the block's
+    # layers look ahead at the layer behind the sum
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=72, width_div=8)
+    w.layers[0].K = 256                              # the block maps 256 -> 250 -> 250 -> 256
+    w.layers[2].N = w.layers[3].K = 256
+    w.layers[2].theta, w.layers[2].tau = 256.0, 16.0
+    w.layers[2].skip_from, w.layers[2].skip_scale = 0, 0.75
+    w.in_shape = (256,)
+    specs, descs = specs_and_descs(w.layers, 12)
+    Ws = synth.make_weights(w, 12)
+    X = synth.make_batch(w, 12)
+    net = GpuNet(descs, w.B, Ws, gemm_path=path, graph=graph, skips=[s.skip_from for s in specs])
+    net.set_input(X)
+    for step in range(3):
+        net.train_step(0.3, step)
+        states = O.train_step(specs, Ws, X, w.B, 0.3, step)
+        for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
+            compare_layer(st, b, sp, w.B, tag=f"step{step}/layer{l}/")
+        Ws = [st.W_new for st in states]
+    net.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_residual_block_convolutional_with_inner_skip_source(path):
+    # conv stack 8 -> 16 -> 16 -> 16 on 12x12 images: layer 2 adds the input of layer 1 (= layer 0's normalised output)
+    chans = [8, 16, 16, 16]
+    hw = 12
+    layers = [synth.LayerCfg(1, 9 * ci, co, float(co * hw * hw), 0.03 / (hw * hw), float(np.sqrt(co * hw * hw)), H=hw, Wd=hw, Cin=ci)
+              for ci, co in zip(chans[:-1], chans[1:])]
+    layers[2].skip_from = 1
+    w = synth.Workload("res_conv", 3, layers, (hw, hw, chans[0]), "normal", "kaiming_uniform", 2)
+    specs, descs = specs_and_descs(w.layers, 5)
+    Ws = synth.make_weights(w, 5)
+    X = synth.make_batch(w, 5)
+    net = GpuNet(descs, w.B, Ws, gemm_path=path, skips=[s.skip_from for s in specs])
+    net.set_input(X)
+    for step in range(2):
+        net.train_step(0.0, step)
+        states = O.train_step(specs, Ws, X, w.B, 0.0, step)
+        for l, (st, b, sp) in enumerate(zip(states, net.bufs, specs)):
+            compare_layer(st, b, sp, w.B, tag=f"step{step}/layer{l}/")
+        Ws = [st.W_new for st in states]
+    net.close()
+
+
+def test_skip_path_argument_errors():
+    w = synth.scaled(synth.workload("tiny_mlp"), B=8, width_div=4)
+    w.layers[0].K = w.layers[0].N
+    specs, descs = specs_and_descs(w.layers, 1)
+    net = GpuNet(descs, w.B, synth.make_weights(w, 1), xnext=False)
+    net.bufs[0].struct.Skip = net.bufs[0].X.data_ptr()
+    arr = (ffb.ff_layer_bufs * len(descs))(*[b.struct for b in net.bufs])
+    with pytest.raises(ffb.FFError) as e:      # the sum has to be written somewhere
+        ffb.ff_train_step(net.ctx.ctx, net.descs_arr, arr, len(descs), w.B, 0.0, 0, 0)
     assert e.value.code == ffb.FF_ERR_ARG
     net.close()

@@ -610,6 +610,85 @@ def test_greedy_epoch_trains_one_layer_per_phase_on_trained_predecessors():
 
 
 # --------------------------------------------------------------------------------------
+# Skip path of a residual block
+# --------------------------------------------------------------------------------------
+def test_skip_path_hand_example_and_neutral_cases():
+    # z = xhat + scale*skip, one float32 multiply and one float32 add per element
+    xhat = np.array([[0.0, 1.5, 0.25], [2.0, 0.0, 0.0]], dtype=F32)
+    skip = np.array([[1.0, -0.5, 4.0], [0.125, 3.0, -1.0]], dtype=F32)
+    assert np.array_equal(O.add_skip(xhat, skip, 0.5), np.array([[0.5, 1.25, 2.25], [2.0625, 1.5, -0.5]], dtype=F32))
+    assert np.array_equal(O.add_skip(xhat, skip, 1.0), xhat + skip)
+    # each operation rounds on its own: 0.1f*3 is not 0.3f, and the sum rounds again
+    a, b = np.array([[1.0]], dtype=F32), np.array([[3.0]], dtype=F32)
+    want = F32(F32(1.0) + F32(F32(0.1) * F32(3.0)))
+    assert O.add_skip(a, b, 0.1)[0, 0] == want
+    # a zero weight or a zero tensor changes nothing, bit for bit (xhat >= 0, so no signed zero can appear)
+    assert np.array_equal(O.add_skip(xhat, skip, 0.0).view(np.uint32), xhat.view(np.uint32))
+    assert np.array_equal(O.add_skip(xhat, np.zeros_like(skip), 0.7).view(np.uint32), xhat.view(np.uint32))
+    # a spatial output takes the flat skip tensor of the same size
+    assert O.add_skip(xhat.reshape(2, 1, 1, 3), skip, 1.0).shape == (2, 1, 1, 3)
+    with pytest.raises(ValueError):
+        O.add_skip(xhat, skip[:, :2], 1.0)
+
+
+def test_residual_block_changes_only_what_the_next_layer_sees():
+    g = np.random.default_rng(31)
+    B = 6
+    specs, Ws, X = _net(g, [20, 24, 20, 12], B)           # layer 1 maps back to the width of the block's input
+    plain = O.train_step(specs, Ws, X, B, 0.25, 3)
+    specs[1].skip_from, specs[1].skip_scale = 0, 1.0      # block = layers 0..1, skip from the block's input
+    res = O.train_step(specs, Ws, X, B, 0.25, 3)
+    for l in (0, 1):   # the block's own layers: same input codes, same goodness
+        assert np.array_equal(plain[l].Xq, res[l].Xq) and np.array_equal(plain[l].G, res[l].G)
+    assert np.array_equal(plain[1].Y, res[1].Y)
+    # what leaves the block is the normalised output plus the block's input
+    assert np.array_equal(res[1].Xnext, plain[1].Xnext + X)
+    assert not np.array_equal(plain[2].Xq, res[2].Xq)
+    assert np.array_equal(res[2].Xq, O.quantize_two_pass(res[1].Xnext, B, specs[2].round_x,
+                                                         O.rounding_key(specs[2].seed, O.ROLE_X, 2, 3))[0])
+    # lengths: both summands have a fixed length per sample, so the sum lies between their difference and their sum
+    n_out = np.sqrt((res[1].Xnext.astype(np.float64) ** 2).sum(1))
+    n_a = np.sqrt((plain[1].Xnext.astype(np.float64) ** 2).sum(1))
+    n_b = np.sqrt((X.astype(np.float64) ** 2).sum(1))
+    assert np.all(n_out <= (n_a + n_b) * (1 + 1e-6)) and np.all(n_out >= np.abs(n_a - n_b) * (1 - 1e-6))
+    # weight 0 is the plain network, bit for bit
+    specs[1].skip_scale = 0.0
+    zero = O.train_step(specs, Ws, X, B, 0.25, 3)
+    for a, b in zip(plain, zero):
+        assert np.array_equal(a.W_new, b.W_new) and np.array_equal(a.Xq, b.Xq)
+    # the look-ahead coefficient of the block's layers sees the goodness of the layer AFTER the block, which the skip
+    # path changed: with lambda > 0 their gradient codes differ from the plain network's, with lambda = 0 they do not
+    specs[1].skip_scale = 1.0
+    res0 = O.train_step(specs, Ws, X, B, 0.0, 3)
+    plain0 = O.train_step([O.LayerSpec(**{**s.__dict__, "skip_from": -1}) for s in specs], Ws, X, B, 0.0, 3)
+    for l in (0, 1):
+        assert np.array_equal(res0[l].dHq, plain0[l].dHq) and np.array_equal(res0[l].W_new, plain0[l].W_new)
+    assert not np.array_equal(res[0].coef, plain[0].coef)
+    # a skip source must be this layer's input or an earlier one, and the sizes must agree
+    specs[1].skip_from = 2
+    with pytest.raises(ValueError):
+        O.train_step(specs, Ws, X, B, 0.0, 3)
+    specs[1].skip_from = 1
+    with pytest.raises(ValueError):
+        O.train_step(specs, Ws, X, B, 0.0, 3)      # layer 1's input has 24 values, its output 20
+
+
+def test_skip_path_in_a_convolutional_block():
+    g = np.random.default_rng(32)
+    B, H, C = 2, 4, 8
+    specs = [_spec(9 * C, C, kind=O.KIND_CONV3X3, H=H, Wd=H, Cin=C, rnd=O.ROUND_STOCHASTIC, index=i) for i in range(2)]
+    specs[1].skip_from = 0
+    Ws = [(g.normal(size=(C, 9 * C)) * 0.2).astype(F32) for _ in specs]
+    X = g.normal(size=(2 * B, H, H, C)).astype(F32)
+    st = O.train_step(specs, Ws, X, B, 0.0, 0)
+    no = O.layer_forward(specs[1], st[0].Xnext, Ws[1], B, 0)
+    assert st[1].Xnext.shape == X.shape and np.array_equal(st[1].Xnext, no.Xnext + X)
+    specs[1].pool = 2
+    with pytest.raises(ValueError):
+        O.train_step(specs, Ws, X, B, 0.0, 0)
+
+
+# --------------------------------------------------------------------------------------
 # Pointwise convolution
 # --------------------------------------------------------------------------------------
 def test_conv1x1_equals_centre_tap_of_conv3x3():
