@@ -370,6 +370,7 @@ def main():
     if dpar:
         table = dp.PointerTable()
         table.add_layer_buffers(bufs)
+        reducer = dp.OverlappedReducer(table, device=dev)   # INT32 sums reduced on a side stream beside later contractions
         X_all = torch.from_numpy(synth.make_batch(w, seed, B=B_total)).reshape(2 * B_total, -1)
         X_host = dp.shard_batch(X_all, B_total, row_off, B).reshape(bufs[0].X.shape).pin_memory()
         del X_all
@@ -386,7 +387,7 @@ def main():
     def step(i):
         if dpar:
             dp.dp_train_step(ctx.ctx, descs_arr, bufs_arr, n_layers, B, B_total, row_off, w.lam_per_step * i, i,
-                             lambda entries: dp.all_reduce_entries(entries, table), stream)
+                             reducer, stream)
         else:
             ffb.ff_train_step(ctx.ctx, descs_arr, bufs_arr, n_layers, B, w.lam_per_step * i, i, stream)
 

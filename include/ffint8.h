@@ -191,17 +191,24 @@ ff_status ff_embed_labels(ff_ctx* ctx, const float* x, const int32_t* labels, in
  * The step is cut at the points where shards must exchange data.  The caller runs phases
  * 0 .. ff_dp_phase_count(n_layers)-1 in order, on every shard; after each phase it combines, in place
  * and over all shards, the n_reduce device arrays listed in `reduce` (element type and operation given
- * per entry; any all-reduce will do, e.g. NCCL's, ordered after the phase on the stream) before the
- * next phase starts.  The library itself performs no communication.
- *   phase 0: ranges of the network input            -> MAX of 2 floats
- *   phase 1+l: forward of layer l                   -> MAX of the output / next-input ranges
- *   phase n+1: losses and coefficients, all layers  -> MAX of the dH ranges, SUM of the loss shares
- *   phase n+2: INT8 dH and local g^W sums, all layers -> SUM of INT32 accW_dump [2][N][K] per layer
- *   phase n+3: update of every layer from the combined sums
+ * per entry; any all-reduce will do, e.g. NCCL's, ordered after the phase on the stream).  Every entry
+ * names the first phase that reads the combined array (needed_by_phase): the reduction must have
+ * finished when that phase starts, and the library touches the array in none of the phases between.
+ * The library itself performs no communication.  With n = n_layers:
+ *   phase 0: ranges of the network input              -> MAX of 2 floats                 (needed by 1)
+ *   phase 1+l: forward of layer l                     -> MAX of the output / next-input ranges (next phase)
+ *   phase n+1: losses and coefficients, all layers    -> MAX of the dH ranges, SUM of the loss shares (n+2)
+ *   phase n+2+l: INT8 dH and local g^W sums of layer l -> SUM of INT32 accW_dump [2][N][K] (needed by 2n+2+l)
+ *   phase 2n+2+l: update of layer l from the combined sums
+ * so the large INT32 reduction of layer l can run (on a stream of its own, after an event recorded behind
+ * phase n+2+l) while the weight-gradient contractions of the layers after it still compute, and a layer's
+ * update waits for its own sums only.
  * B_local rows per set are rows [row_offset, row_offset + B_local) of the B_total rows per set of the
  * whole batch.  Layers must be chained (X of layers > 0 NULL), accW_dump of every layer non-NULL (it
  * carries the sums), and every shard must pass the same descriptors (seed included), lambda and step.
- * `reduce` has room for FF_DP_MAX_REDUCE entries.  Errors as ff_train_step. */
+ * A spatial layer whose whole-batch contraction could leave INT32 in the worst case is held to a share of
+ * the INT32 range per shard in proportion to its rows (FF_ERR_RANGE otherwise), so that the 32-bit sums of
+ * the shards cannot wrap.  `reduce` has room for FF_DP_MAX_REDUCE entries.  Errors as ff_train_step. */
 #define FF_DP_MAX_REDUCE 96
 enum { FF_DP_F32 = 0, FF_DP_I32 = 1 };
 enum { FF_DP_MAX = 0, FF_DP_SUM = 1 };
@@ -210,6 +217,8 @@ typedef struct ff_dp_reduce {
   uint64_t count;  /* elements */
   int32_t dtype;   /* FF_DP_F32 / FF_DP_I32 */
   int32_t op;      /* FF_DP_MAX / FF_DP_SUM */
+  int32_t needed_by_phase;  /* first phase that reads the combined array */
+  int32_t reserved;
 } ff_dp_reduce;
 int ff_dp_phase_count(int n_layers);
 ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B_local,

@@ -52,7 +52,8 @@ FF_DP_MAX, FF_DP_SUM = 0, 1
 
 
 class ff_dp_reduce(C.Structure):
-    _fields_ = [("dev_ptr", C.c_void_p), ("count", C.c_uint64), ("dtype", C.c_int32), ("op", C.c_int32)]
+    _fields_ = [("dev_ptr", C.c_void_p), ("count", C.c_uint64), ("dtype", C.c_int32), ("op", C.c_int32),
+                ("needed_by_phase", C.c_int32), ("reserved", C.c_int32)]
 
 
 class FFError(RuntimeError):
@@ -199,12 +200,14 @@ def ff_dp_phase_count(n_layers: int) -> int:
 def ff_dp_train_phase(ctx, descs_arr, bufs_arr, n_layers: int, B_local: int, B_total: int, row_offset: int, phase: int,
                       lam: float, step: int, stream: int = 0):
     """One phase of the data-parallel step.  Returns the arrays to combine over the shards before the
-    next phase as a list of (device address, element count, FF_DP_F32 | FF_DP_I32, FF_DP_MAX | FF_DP_SUM)."""
+    next phase as a list of (device address, element count, FF_DP_F32 | FF_DP_I32, FF_DP_MAX | FF_DP_SUM, first phase
+    that reads the combined array)."""
     red = (ff_dp_reduce * FF_DP_MAX_REDUCE)()
     n = C.c_int(0)
     _check(ctx, load().ff_dp_train_phase(ctx, descs_arr, bufs_arr, n_layers, B_local, B_total, row_offset, phase, lam,
                                          step, stream, red, C.byref(n)))
-    return [(int(red[i].dev_ptr), int(red[i].count), int(red[i].dtype), int(red[i].op)) for i in range(n.value)]
+    return [(int(red[i].dev_ptr), int(red[i].count), int(red[i].dtype), int(red[i].op), int(red[i].needed_by_phase))
+            for i in range(n.value)]
 
 
 def ff_predict(ctx, descs_arr, bufs_arr, n_layers: int, B: int, n_classes: int, first_counted_layer: int, scores: int,

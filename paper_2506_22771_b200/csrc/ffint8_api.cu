@@ -995,18 +995,20 @@ ff_status dp_phase_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
                         float lambda, cudaStream_t st, ff_dp_reduce* red, int* n_red) {
   ff_status s;
   int nr = 0;
-  auto want = [&](void* p, uint64_t count, int dtype, int op) {
+  // needed_by: the first phase that reads the combined array (the reduction may run beside the phases before it)
+  auto want = [&](void* p, uint64_t count, int dtype, int op, int needed_by) {
     red[nr].dev_ptr = p;
     red[nr].count = count;
     red[nr].dtype = dtype;
     red[nr].op = op;
+    red[nr].needed_by_phase = needed_by;
     ++nr;
   };
   if (phase == 0) {
     // ranges of the network input: local maxima now, the maximum over the shards before phase 1
     for (int l = 0; l < n; ++l) FF_CUDA(ctx, cudaMemsetAsync(bufs[l].absmax, 0, FF_ABSMAX_LEN * sizeof(float), st));
     if ((s = quantize_input(ctx, layers[0], bufs[0], B, st, true, false)) != FF_OK) return s;
-    want(bufs[0].absmax + FF_A_X_POS, 2, FF_DP_F32, FF_DP_MAX);
+    want(bufs[0].absmax + FF_A_X_POS, 2, FF_DP_F32, FF_DP_MAX, 1);
   } else if (phase <= n) {
     // forward of layer l; its input range is global by now, the range of its normalised output becomes so after the phase
     const int l = phase - 1;
@@ -1018,8 +1020,8 @@ ff_status dp_phase_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
     const bool feeds_next = l + 1 < n;
     if ((s = forward_from_xq(ctx, layers[l], bufs[l], B, feeds_next ? bufs[l + 1].absmax + FF_A_X_POS : nullptr, st)) != FF_OK)
       return s;
-    want(bufs[l].absmax + FF_A_XNEXT_POS, 2, FF_DP_F32, FF_DP_MAX);
-    if (feeds_next) want(bufs[l + 1].absmax + FF_A_X_POS, 2, FF_DP_F32, FF_DP_MAX);
+    want(bufs[l].absmax + FF_A_XNEXT_POS, 2, FF_DP_F32, FF_DP_MAX, phase + 1);
+    if (feeds_next) want(bufs[l + 1].absmax + FF_A_X_POS, 2, FF_DP_F32, FF_DP_MAX, phase + 1);
   } else if (phase == n + 1) {
     // FP32 output of the last layer (if asked for); losses and coefficients of all layers from the local G's
     if ((s = normalize_output(ctx, layers[n - 1], bufs[n - 1], B, nullptr, nullptr, st)) != FF_OK) return s;
@@ -1032,26 +1034,24 @@ ff_status dp_phase_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
         th[j] = layers[l + 1 + j].theta;
       }
       if ((s = loss_grad_impl(ctx, layers[l], bufs[l], B, Gl, th, n_later, lambda, st, true, false)) != FF_OK) return s;
-      want(bufs[l].absmax + FF_A_DH_POS, 2, FF_DP_F32, FF_DP_MAX);   // range of dH over the whole batch
-      want(bufs[l].loss, 1, FF_DP_F32, FF_DP_SUM);                    // each shard holds its share of the batch mean
+      want(bufs[l].absmax + FF_A_DH_POS, 2, FF_DP_F32, FF_DP_MAX, n + 2);   // range of dH over the whole batch
+      want(bufs[l].loss, 1, FF_DP_F32, FF_DP_SUM, n + 2);                   // each shard holds its share of the batch mean
     }
-  } else if (phase == n + 2) {
-    // INT8 output gradient and the local INT32 weight-gradient sums of every layer
+  } else if (phase < 2 * n + 2) {
+    // INT8 output gradient and the local INT32 weight-gradient sums of layer l.  Nothing reads the combined sums
+    // before the layer's own update phase, so their (large) reduction can run beside the later layers' contractions.
+    const int l = phase - (n + 2);
     ctx->accumulate_only = true;
-    for (int l = 0; l < n; ++l) {
-      s = loss_grad_impl(ctx, layers[l], bufs[l], B, nullptr, nullptr, 0, lambda, st, false, true);
-      if (s == FF_OK) s = run_update_gemm(ctx, layers[l], bufs[l], B, st);
-      if (s != FF_OK) break;
-      want(bufs[l].accW_dump, (uint64_t)2 * layers[l].N * layers[l].K, FF_DP_I32, FF_DP_SUM);
-    }
+    s = loss_grad_impl(ctx, layers[l], bufs[l], B, nullptr, nullptr, 0, lambda, st, false, true);
+    if (s == FF_OK) s = run_update_gemm(ctx, layers[l], bufs[l], B, st);
     ctx->accumulate_only = false;
     if (s != FF_OK) return s;
+    want(bufs[l].accW_dump, (uint64_t)2 * layers[l].N * layers[l].K, FF_DP_I32, FF_DP_SUM, 2 * n + 2 + l);
   } else {
     // the sums are those of the whole batch now: the same update on every device keeps the weights identical
-    for (int l = 0; l < n; ++l) {
-      ProfScope prof(ctx, FF_K_UPD_GEMM, st);
-      if ((s = launch_slab_update(ctx, bufs[l].accW_dump, 1, layers[l], bufs[l], st)) != FF_OK) return s;
-    }
+    const int l = phase - (2 * n + 2);
+    ProfScope prof(ctx, FF_K_UPD_GEMM, st);
+    if ((s = launch_slab_update(ctx, bufs[l].accW_dump, 1, layers[l], bufs[l], st)) != FF_OK) return s;
   }
   *n_red = nr;
   return FF_OK;
@@ -1329,7 +1329,7 @@ ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
   return ff_train_step_from(ctx, layers, bufs, n_layers, 0, B, lambda, step, cuda_stream);
 }
 
-int ff_dp_phase_count(int n_layers) { return n_layers > 0 ? n_layers + 4 : 0; }
+int ff_dp_phase_count(int n_layers) { return n_layers > 0 ? 3 * n_layers + 2 : 0; }
 
 ff_status ff_dp_train_phase(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B_local,
                             int B_total, int row_offset, int phase, float lambda, uint64_t step, void* cuda_stream,

@@ -63,20 +63,116 @@ class PointerTable:
         raise KeyError(f"address {ptr:#x} (+{4 * count} bytes) lies in no registered tensor")
 
 
-def all_reduce_entries(entries: List[Tuple[int, int, int, int]], table: PointerTable, group=None):
-    """Combines every listed array in place over the ranks of `group` (torch.distributed)."""
+SMALL = 64   # entries of at most this many elements are packed into one collective per (type, operation)
+
+
+def _torch_op(op: int):
     import torch.distributed as dist
-    for ptr, count, dtype, op in entries:
+    return dist.ReduceOp.MAX if op == ffb.FF_DP_MAX else dist.ReduceOp.SUM
+
+
+def all_reduce_entries(entries: List[Tuple], table: PointerTable, group=None):
+    """Combines every listed array in place over the ranks of `group` (torch.distributed), in stream order.  The
+    small entries of a phase (ranges, loss shares) share one collective per element type and operation: they are
+    packed into a staging tensor, reduced together and copied back - a phase costs one or two latencies instead of
+    one per entry."""
+    import torch
+    import torch.distributed as dist
+    packs = {}
+    for ent in entries:
+        ptr, count, dtype, op = ent[:4]
         v = table.view(ptr, count, dtype)
-        dist.all_reduce(v, op=dist.ReduceOp.MAX if op == ffb.FF_DP_MAX else dist.ReduceOp.SUM, group=group)
+        if count <= SMALL:
+            packs.setdefault((dtype, op), []).append(v)
+        else:
+            dist.all_reduce(v, op=_torch_op(op), group=group)
+    for (dtype, op), views in packs.items():
+        if len(views) == 1:
+            dist.all_reduce(views[0], op=_torch_op(op), group=group)
+            continue
+        staged = torch.cat([v.reshape(-1) for v in views])
+        dist.all_reduce(staged, op=_torch_op(op), group=group)
+        at = 0
+        for v in views:
+            v.copy_(staged[at:at + v.numel()].reshape(v.shape))
+            at += v.numel()
+
+
+class OverlappedReducer:
+    """The reductions of a data-parallel step with the large ones taken off the critical path.
+
+    now(entries): combine at once, in stream order (small entries packed as in all_reduce_entries).
+    start(entries) -> handle: begin combining on a side stream, ordered after everything enqueued so far on the
+    compute stream (an event); finish(handle): make the compute stream wait for it.  On CPU tensors (the gloo tests)
+    there are no streams: start issues the collectives with async_op=True and finish waits for them."""
+
+    def __init__(self, table: PointerTable, group=None, device=None):
+        self.table, self.group = table, group
+        self.cuda = device is not None and str(device).startswith("cuda")
+        self.side = None
+        self.log = []              # ("now" | "start" | "finish", phase tag) in call order, for the tests
+        if self.cuda:
+            import torch
+            self.side = torch.cuda.Stream(device=device)
+
+    def now(self, entries, tag=None):
+        self.log.append(("now", tag))
+        all_reduce_entries(entries, self.table, self.group)
+
+    def start(self, entries, tag=None):
+        import torch
+        import torch.distributed as dist
+        self.log.append(("start", tag))
+        views = [self.table.view(*e[:3]) for e in entries]
+        if self.cuda:
+            ready = torch.cuda.Event()
+            ready.record(torch.cuda.current_stream())
+            self.side.wait_event(ready)
+            with torch.cuda.stream(self.side):
+                for v, e in zip(views, entries):
+                    dist.all_reduce(v, op=_torch_op(e[3]), group=self.group)
+                done = torch.cuda.Event()
+                done.record(self.side)
+            return ("event", done, views)
+        works = [dist.all_reduce(v, op=_torch_op(e[3]), group=self.group, async_op=True) for v, e in zip(views, entries)]
+        return ("works", works, views)
+
+    def finish(self, handle, tag=None):
+        import torch
+        self.log.append(("finish", tag))
+        kind, obj, _views = handle
+        if kind == "event":
+            torch.cuda.current_stream().wait_event(obj)
+        else:
+            for w in obj:
+                w.wait()
 
 
 def dp_train_step(ctx, descs_arr, bufs_arr, n_layers: int, B_local: int, B_total: int, row_offset: int, lam: float,
-                  step: int, reduce: Callable[[List[Tuple[int, int, int, int]]], None], stream: int = 0):
-    """All phases of one data-parallel step on this shard; `reduce(entries)` is called between phases
-    and must combine the listed arrays over the shards, ordered after the phase on `stream`."""
+                  step: int, reduce, stream: int = 0):
+    """All phases of one data-parallel step on this shard.
+
+    `reduce` is either a callable reduce(entries) that combines the listed arrays over the shards in stream order
+    (every reduction then sits between its phase and the next), or an object with now / start / finish like
+    OverlappedReducer: a reduction whose result is needed only several phases later (the INT32 weight-gradient
+    sums of a layer, read by that layer's update phase) is started behind its phase and waited for just before
+    the phase that needs it, so it runs beside the contractions of the layers after it."""
+    overlapped = hasattr(reduce, "start")
+    pending = {}                                   # phase that needs the result -> handles
     for phase in range(ffb.ff_dp_phase_count(n_layers)):
+        for h in pending.pop(phase, []):
+            reduce.finish(h, phase)
         entries = ffb.ff_dp_train_phase(ctx, descs_arr, bufs_arr, n_layers, B_local, B_total, row_offset, phase, lam,
                                         step, stream)
-        if entries:
+        if not entries:
+            continue
+        if not overlapped:
             reduce(entries)
+            continue
+        soon = [e for e in entries if e[4] <= phase + 1]
+        later = [e for e in entries if e[4] > phase + 1]
+        if soon:
+            reduce.now(soon, phase)
+        for need in sorted({e[4] for e in later}):
+            pending.setdefault(need, []).append(reduce.start([e for e in later if e[4] == need], phase))
+    assert not pending, "a reduction was asked for by a phase that does not exist"

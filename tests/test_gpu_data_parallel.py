@@ -43,7 +43,9 @@ def _combine(shards, entries_per_shard):
             v.copy_(total)
 
 
-def _run_dp(w, seed, steps, lam_per_step, world, path, rounding=(1, 0, 1)):
+def _run_dp(w, seed, steps, lam_per_step, world, path, rounding=(1, 0, 1), defer=False):
+    """defer: an array is combined only right before the phase that needs it (the latest moment the overlapped
+    reducer allows), instead of right behind the phase that listed it."""
     specs, descs = specs_and_descs(w.layers, seed, *rounding)
     Ws = synth.make_weights(w, seed)
     X = synth.make_batch(w, seed)
@@ -54,10 +56,22 @@ def _run_dp(w, seed, steps, lam_per_step, world, path, rounding=(1, 0, 1)):
     Ms = Vs = None
     for step in range(steps):
         lam = lam_per_step * step
+        assert ffb.ff_dp_phase_count(n) == 3 * n + 2
+        waiting = {}                                  # phase that needs them -> per-shard entry lists
         for phase in range(ffb.ff_dp_phase_count(n)):
+            for ents in waiting.pop(phase, []):
+                _combine(shards, ents)
             entries = [ffb.ff_dp_train_phase(sh.net.ctx.ctx, sh.net.descs_arr, sh.net.bufs_arr, n, sh.B, w.B, sh.off,
                                              phase, lam, step, 0) for sh in shards]
-            _combine(shards, entries)
+            assert all(e[4] > phase for ent in entries for e in ent)
+            if n + 2 <= phase < 2 * n + 2:            # the INT32 sums of layer l are read by that layer's update phase
+                assert [e[4] for e in entries[0]] == [2 * n + 2 + (phase - n - 2)]
+            if not defer:
+                _combine(shards, entries)
+                continue
+            for need in sorted({e[4] for e in entries[0]}):
+                waiting.setdefault(need, []).append([[e for e in ent if e[4] == need] for ent in entries])
+        assert not waiting
         for sh in shards:
             ffb.ff_poll_status(sh.net.ctx.ctx, 0)
         states = O.train_step(specs, Ws, X, w.B, lam, step, Ms, Vs)
@@ -125,6 +139,15 @@ def test_dp_with_adam():
     for l in w.layers:
         l.optimizer, l.momentum, l.beta2, l.adam_eps, l.lr = 1, 0.9, 0.99, 1e-6, 1e-3
     _run_dp(w, seed=15, steps=3, lam_per_step=0.5, world=3, path=(ffb.FF_GEMM_AUTO, 0))
+
+
+def test_dp_deferred_reductions_equal_whole_batch():
+    # every reduction done at the last moment its needed_by_phase allows: the weight-gradient sums of layer l are
+    # combined after the contractions of all later layers have run, as with a reduction overlapped on a side stream
+    w = synth.scaled(synth.workload("mlp_lookahead"), B=120, width_div=8)
+    _run_dp(w, seed=44, steps=2, lam_per_step=0.25, world=3, path=(ffb.FF_GEMM_AUTO, 0), defer=True)
+    w = synth.scaled(synth.workload("cnn"), B=4, width_div=4)
+    _run_dp(w, seed=45, steps=2, lam_per_step=0.0, world=2, path=(ffb.FF_GEMM_AUTO, 0), defer=True)
 
 
 def test_dp_single_shard_equals_train_step():

@@ -158,3 +158,77 @@ def test_reference_arm_other_ranks_do_nothing():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny_mlp",
                           "--steps", "1", "--warmup", "1", "--gpus", "2"], capture_output=True, text=True, timeout=300, env=env)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+# ---- the overlapped form: large reductions started behind their phase, waited for where they are needed ----------
+def _dp_overlap_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2506_22771_b200 import binding as ffb
+    from paper_2506_22771_b200 import data_parallel as dp
+    n = 2                                                   # layers of the stand-in network
+    absmax = [torch.zeros(8) for _ in range(n)]
+    loss = [torch.zeros(4) for _ in range(n)]
+    accw = [torch.zeros(2, 3, 5, dtype=torch.int32) for _ in range(n)]
+    table = dp.PointerTable(absmax + loss + accw)
+    seen = {"update_saw_global_sums": [], "phases": []}
+
+    def local_sums(l, r):                                   # what rank r's contraction of layer l leaves
+        return (torch.arange(30, dtype=torch.int32).reshape(2, 3, 5) + 7 * l) * (r + 1)
+
+    def fake_phase(ctx, descs, bufs, n_layers, B_local, B_total, row_off, phase, lam, step, stream=0):
+        # the call sequence and the lists of ff_dp_train_phase, on CPU tensors
+        seen["phases"].append(phase)
+        F, I, MAX, SUM = ffb.FF_DP_F32, ffb.FF_DP_I32, ffb.FF_DP_MAX, ffb.FF_DP_SUM
+        if phase == 0:
+            absmax[0][0:2] = torch.tensor([1.0 + rank, 2.0 - rank])
+            return [(absmax[0].data_ptr(), 2, F, MAX, 1)]
+        if phase <= n:
+            l = phase - 1
+            absmax[l][5:7] = torch.tensor([0.5 * (rank + 1) + l, 3.0 - rank])
+            ent = [(absmax[l].data_ptr() + 20, 2, F, MAX, phase + 1)]
+            if l + 1 < n:
+                absmax[l + 1][0:2] = absmax[l][5:7]
+                ent.append((absmax[l + 1].data_ptr(), 2, F, MAX, phase + 1))
+            return ent
+        if phase == n + 1:
+            ent = []
+            for l in range(n):
+                absmax[l][3:5] = torch.tensor([float(rank + l), 1.0])
+                loss[l][0] = 0.25 * (rank + 1) + l
+                ent += [(absmax[l].data_ptr() + 12, 2, F, MAX, n + 2), (loss[l].data_ptr(), 1, F, SUM, n + 2)]
+            return ent
+        if phase < 2 * n + 2:
+            l = phase - (n + 2)
+            accw[l].copy_(local_sums(l, rank))
+            return [(accw[l].data_ptr(), 30, I, SUM, 2 * n + 2 + l)]
+        l = phase - (2 * n + 2)
+        want = sum(local_sums(l, r) for r in range(world))
+        seen["update_saw_global_sums"].append(bool(torch.equal(accw[l], want)))
+        return []
+
+    ffb.ff_dp_train_phase, ffb.ff_dp_phase_count = fake_phase, (lambda k: 3 * k + 2)
+    red = dp.OverlappedReducer(table)
+    dp.dp_train_step(None, None, None, n, 4, 8, 4 * rank, 0.0, 0, red)
+    out[rank] = (seen, red.log, [a.tolist() for a in absmax], [x.tolist() for x in loss])
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_dp_overlapped_reductions_over_two_ranks():
+    world, n = 2, 2
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_dp_overlap_worker, args=(world, _free_port(), out), nprocs=world, join=True)
+        res = dict(out)
+    for rank in range(world):
+        seen, log, absmax, loss = res[rank]
+        assert seen["phases"] == list(range(3 * n + 2))
+        assert seen["update_saw_global_sums"] == [True, True]          # each update found the sums of the whole batch
+        # small reductions at once, the weight-gradient sums of layer l started behind phase n+2+l and waited for
+        # right before phase 2n+2+l - i.e. the reduction of layer 0 is in flight while layer 1's sums are computed
+        assert log == [("now", 0), ("now", 1), ("now", 2), ("now", 3), ("start", 4), ("start", 5), ("finish", 6),
+                       ("finish", 7)]
+        assert absmax[0][0:2] == [2.0, 2.0] and absmax[0][5:7] == [1.0, 3.0] and absmax[1][0:2] == [1.0, 3.0]
+        assert absmax[0][3:5] == [1.0, 1.0] and absmax[1][3:5] == [2.0, 1.0]
+        assert loss[0][0] == 0.75 and loss[1][0] == 2.75
