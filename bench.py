@@ -566,7 +566,7 @@ def main():
                                    "sample": f"{Bs} positive + {Bs} negative samples, full layer widths, 1 step"}
         print(json.dumps(out))
     ctx.close()
-    if world > 1:
+    if world > 1 or args.data_parallel:
         dist.destroy_process_group()
 
 

@@ -78,6 +78,8 @@ def all_reduce_entries(entries: List[Tuple], table: PointerTable, group=None):
     one per entry."""
     import torch
     import torch.distributed as dist
+    if dist.get_world_size(group) == 1:
+        return                       # one shard: every array already is the whole batch's
     packs = {}
     for ent in entries:
         ptr, count, dtype, op = ent[:4]
@@ -123,6 +125,8 @@ class OverlappedReducer:
         import torch
         import torch.distributed as dist
         self.log.append(("start", tag))
+        if dist.get_world_size(self.group) == 1:
+            return ("none", None, None)
         views = [self.table.view(*e[:3]) for e in entries]
         if self.cuda:
             ready = torch.cuda.Event()
@@ -141,6 +145,8 @@ class OverlappedReducer:
         import torch
         self.log.append(("finish", tag))
         kind, obj, _views = handle
+        if kind == "none":
+            return
         if kind == "event":
             torch.cuda.current_stream().wait_event(obj)
         else:
