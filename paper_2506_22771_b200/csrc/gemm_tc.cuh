@@ -98,6 +98,8 @@ struct TcParams {
   float mu;
   // split weight gradient
   int32_t* slabs;
+  int splits_per_slab;      // > 1: that many consecutive splits add their partial sums into one slab with integer
+                            // atomics (exact, order-free; the slab is cleared before the launch); 1: a slab per split
   // convolution geometry (conv_W = 0: dense layer).  A 128-row block of positions is conv_TH image
   // rows of conv_W pixels; conv_cpt = channel chunks of CH bytes per filter tap; images per set.
   // conv_W / conv_H are the OUTPUT extents; the input box of an output position starts conv_stride
@@ -776,7 +778,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         // store instruction of the warp writes four whole 128-byte row segments.
         uint8_t* patch = patch0;
         for (int pass = 0; pass < 2; ++pass) {
-          int32_t* slab = p.slabs + (size_t)(split * 2 + pass) * p.out_rows * p.out_cols;
+          const bool shared_slab = p.splits_per_slab > 1;
+          int32_t* slab = p.slabs + (size_t)((shared_slab ? split / p.splits_per_slab : split) * 2 + pass) * p.out_rows * p.out_cols;
           int v[2][32];
           if (cbeg < cend) tc_ld32_async(t_row + pass * TC_BN + cbeg, v[0]);
 #pragma unroll
@@ -793,19 +796,36 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
                   *reinterpret_cast<int4*>(patch + lane * 128 + (((j >> 2) ^ (lane & 7)) << 4)) =
                       make_int4(a[j], a[j + 1], a[j + 2], a[j + 3]);
                 __syncwarp();
+                if (shared_slab) {
+                  // one staged row per instruction: the warp's 32 lanes add 32 consecutive columns (128 bytes)
+                  if (col0 + cb + lane < p.out_cols) {
+#pragma unroll 8
+                    for (int r = 0; r < 32; ++r) {
+                      const int val = *reinterpret_cast<const int*>(patch + r * 128 + ((((lane >> 2) ^ (r & 7))) << 4) + (lane & 3) * 4);
+                      if (wrow0 + r < p.out_rows && val != 0) atomicAdd(slab + (size_t)(wrow0 + r) * p.out_cols + col0 + cb + lane, val);
+                    }
+                  }
+                } else {
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                  const int r = q * 4 + (lane >> 3), cc = lane & 7;
-                  if (wrow0 + r < p.out_rows && col0 + cb + cc * 4 < p.out_cols)
-                    *reinterpret_cast<int4*>(slab + (size_t)(wrow0 + r) * p.out_cols + col0 + cb + cc * 4) =
-                        *reinterpret_cast<const int4*>(patch + r * 128 + ((cc ^ (r & 7)) << 4));
+                  for (int q = 0; q < 8; ++q) {
+                    const int r = q * 4 + (lane >> 3), cc = lane & 7;
+                    if (wrow0 + r < p.out_rows && col0 + cb + cc * 4 < p.out_cols)
+                      *reinterpret_cast<int4*>(slab + (size_t)(wrow0 + r) * p.out_cols + col0 + cb + cc * 4) =
+                          *reinterpret_cast<const int4*>(patch + r * 128 + ((cc ^ (r & 7)) << 4));
+                  }
                 }
                 __syncwarp();
               } else if (row_ok) {
                 int32_t* dst = slab + (size_t)row * p.out_cols + col0 + cb;
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
-                  if (col0 + cb + j < p.out_cols) dst[j] = a[j];
+                  if (col0 + cb + j < p.out_cols) {
+                    if (shared_slab) {
+                      if (a[j] != 0) atomicAdd(dst + j, a[j]);
+                    } else {
+                      dst[j] = a[j];
+                    }
+                  }
               }
             }
           }
@@ -1176,6 +1196,21 @@ inline int tc_conv_update_splits(const ff_layer_desc& L, int B, int sm_count, in
   if (splits < tc_min_splits(kblocks)) splits = tc_min_splits(kblocks);
   return splits < 1 ? 1 : (int)splits;
 }
+// Splits that may share one slab: as many consecutive ones as keep the slab's whole contraction within
+// TC_SAFE_KBLOCKS blocks, so that a shared INT32 sum cannot wrap either.  Sets p.splits_per_slab, clears the
+// slabs a shared accumulation adds into, and returns the number of slabs the launch will leave.
+inline int tc_plan_shared_slabs(TcParams& p, size_t plane, cudaStream_t st, cudaError_t* err) {
+  const int kb_per_split = cdiv(p.kblocks, p.splits < 1 ? 1 : p.splits);
+  const int splits = cdiv(p.kblocks, kb_per_split);
+  int per = TC_SAFE_KBLOCKS / kb_per_split;
+  if (per < 1) per = 1;
+  if (per > splits) per = splits;
+  p.splits_per_slab = per;
+  const int slabs = cdiv(splits, per);
+  *err = cudaSuccess;
+  if (per > 1) *err = cudaMemsetAsync(p.slabs, 0, (size_t)slabs * 2 * plane * sizeof(int32_t), st);
+  return slabs;
+}
 inline size_t tc_conv_update_slab_bytes(const ff_layer_desc& L, int splits) {
   return (size_t)splits * 2 * L.N * L.K * sizeof(int32_t);
 }
@@ -1318,8 +1353,12 @@ inline ff_status tc_conv_update(TcState& t, const ff_layer_desc& L, const ff_lay
   p.conv_cin = L.Cin;
   p.conv_cpt = L.Cin / ch;
   p.conv_imgs_per_pass = B;
-  const int kb_per_split = cdiv(p.kblocks, splits);
-  *splits_out = cdiv(p.kblocks, kb_per_split);
+  cudaError_t merr;
+  *splits_out = tc_plan_shared_slabs(p, (size_t)L.N * L.K, st, &merr);
+  if (merr != cudaSuccess) {
+    snprintf(t.err, sizeof(t.err), "cudaMemsetAsync: %s", cudaGetErrorString(merr));
+    return FF_ERR_CUDA;
+  }
   const int ncta = t.force_ncta ? t.force_ncta : (L.N > TC_BM ? 2 : 1);
   if ((s = tc_make_map(t, &ta, b.dHq, L.N, pos_per_pass, 2, 128, 128)) != FF_OK) return s;
   if ((s = tc_make_map_nhwc(t, &tb, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_W, p.conv_TH, p.conv_stride)) != FF_OK) return s;
@@ -1352,8 +1391,12 @@ inline ff_status tc_dense_update_slab(TcState& t, const int8_t* dHq, int N, cons
   p.splits = splits;
   p.status = status;
   p.slabs = slabs;
-  const int kb_per_split = cdiv(p.kblocks, splits);
-  *splits_out = cdiv(p.kblocks, kb_per_split);
+  cudaError_t merr;
+  *splits_out = tc_plan_shared_slabs(p, (size_t)N * kcols, st, &merr);
+  if (merr != cudaSuccess) {
+    snprintf(t.err, sizeof(t.err), "cudaMemsetAsync: %s", cudaGetErrorString(merr));
+    return FF_ERR_CUDA;
+  }
   if ((s = tc_make_map(t, &ta, dHq, N, rows_per_pass, 2, 128, 128, (uint64_t)ld_dhq)) != FF_OK) return s;
   if ((s = tc_make_map(t, &tb, xi, kcols, rows_per_pass, 2, 128, 128, (uint64_t)ld_xi)) != FF_OK) return s;
   // one split: a large output with tiles for every SM, where CTA pairs pay; several: a small output, single CTAs
