@@ -16,6 +16,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "dwconv.cuh"
+#include "conv_small.cuh"
 
 using namespace ffi8;
 
@@ -478,8 +479,43 @@ ff_status dw_update(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b,
   return s;
 }
 
+// 3x3 convolution with at most four input channels: direct dp4a kernel (conv_small.cuh)
+ff_status conv_small_forward(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  ConvSmallGeom g;
+  g.H = L.H, g.W = L.Wd, g.Ho = tc_out_h(L), g.Wo = tc_out_w(L), g.stride = tc_conv_stride(L), g.N = L.N;
+  g.rows_per_sample = g.Ho * g.Wo;
+  g.rows_per_pass = B * g.rows_per_sample;
+  g.rows = 2 * g.rows_per_pass;
+  g.y_stream = (size_t)g.rows * L.N * sizeof(float) > ((size_t)80 << 20) ? 1 : 0;
+  const int tiles = (g.rows + CS_THREADS - 1) / CS_THREADS;
+  const int cap = ctx->sm_count * 4;
+  const int grid = tiles < cap ? tiles : cap;
+  unsigned long long* S = reinterpret_cast<unsigned long long*>(b.S);
+  ProfScope prof(ctx, FF_K_FWD_GEMM, st);
+#define FF_CS_LAUNCH(CIN, LP) \
+  conv3x3_small_fwd_kernel<CIN, LP><<<grid, CS_THREADS, 0, st>>>(b.Xq, b.Wq, b.Y, b.acc_dump, S, b.rowmax, b.absmax, g)
+#define FF_CS_BY_N(CIN)                   \
+  switch (L.N) {                          \
+    case 16: FF_CS_LAUNCH(CIN, 4); break;  \
+    case 32: FF_CS_LAUNCH(CIN, 8); break;  \
+    case 64: FF_CS_LAUNCH(CIN, 16); break; \
+    default: FF_CS_LAUNCH(CIN, 32); break; \
+  }
+  switch (L.Cin) {
+    case 1: FF_CS_BY_N(1); break;
+    case 2: FF_CS_BY_N(2); break;
+    case 3: FF_CS_BY_N(3); break;
+    default: FF_CS_BY_N(4); break;
+  }
+#undef FF_CS_BY_N
+#undef FF_CS_LAUNCH
+  FF_LAUNCH_CHECK(ctx);
+  return FF_OK;
+}
+
 ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
   if (L.kind == FF_DWCONV3X3) return dw_forward(ctx, L, b, B, st);
+  if (ctx->gemm_path == FF_GEMM_AUTO && conv_small_ok(L.kind == FF_CONV3X3, L.Cin, L.N)) return conv_small_forward(ctx, L, b, B, st);
   const int R = rows_per_sample(L);
   const int rows = 2 * B * R;
   bool tc_ok = tc_forward_supported(L, B);
