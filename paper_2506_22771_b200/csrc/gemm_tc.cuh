@@ -51,6 +51,7 @@ constexpr int TC_PREFETCH_KB = 8;                         // W tile is prefetche
 // 8 makes a wave of 74 CTA pairs nearly square (8 x 9 panels instead of 16 x 5).
 constexpr int TC_GROUP_M_KMAJOR = 16, TC_GROUP_M_MNMAJOR = 8;
 constexpr uint32_t TC_TMEM_COLS = 512;
+constexpr int TC_MAX_ACC = 4;                             // most accumulator stages (narrow forward tiles)
 constexpr unsigned long long TC_WAIT_NS = 2000000000ull;  // 2 s bound on every wait
 
 // Shared-memory geometry of one pipeline stage.
@@ -77,6 +78,10 @@ struct TcParams {
   int kblocks;              // contraction blocks per pass
   int npass;                // 1, or 2 for the weight gradient (positive / negative set)
   int splits, kb_per_split; // the contraction blocks of a pass are divided over `splits` work items
+  int bn;                   // K-major kernels: tile columns (a multiple of 32, at most TC_BN) - the MMA's N and the rows of
+                            // B a stage holds follow it, so a narrow layer wastes neither, and a wide one can pick the
+                            // width that fills its last wave of tiles best; MN-major kernels always use TC_BN
+  int acc_stages;           // K-major forward: accumulator stages in tensor memory (512 / bn, at most 4)
   uint32_t* status;
   // raw
   int32_t* C;
@@ -341,9 +346,9 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
   return d;
 }
 // Instruction descriptor: INT8 x INT8 -> INT32, dense, M = 128 per CTA of the group, N = 256.
-__host__ __device__ constexpr uint32_t make_idesc_i8(bool a_mn_major, bool b_mn_major, int ncta) {
+__host__ __device__ constexpr uint32_t make_idesc_i8(bool a_mn_major, bool b_mn_major, int ncta, int n = TC_BN) {
   return (2u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
-         ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)((TC_BM * ncta) >> 4) << 24);
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)((TC_BM * ncta) >> 4) << 24);
 }
 
 // Tile order: groups of TC_GROUP_M tile rows, column by column inside a group, so that the CTAs
@@ -375,17 +380,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   uint64_t* bars = reinterpret_cast<uint64_t*>(patch_all + TC_EPI_WARPS * TC_PATCHES * TC_PATCH_BYTES);
   const uint32_t bar_full = smem_u32(bars);                      // [STAGES]  used in the leader CTA
   const uint32_t bar_empty = bar_full + 8 * TC_MAX_STAGES;       // [STAGES]  one set per CTA
-  const uint32_t bar_tfull = bar_empty + 8 * TC_MAX_STAGES;      // [2]       one set per CTA
-  const uint32_t bar_tempty = bar_tfull + 16;                    // [2]       used in the leader CTA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_MAX_STAGES + 4);
+  const uint32_t bar_tfull = bar_empty + 8 * TC_MAX_STAGES;      // [TC_MAX_ACC] one set per CTA
+  const uint32_t bar_tempty = bar_tfull + 8 * TC_MAX_ACC;        // [TC_MAX_ACC] used in the leader CTA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_MAX_STAGES + 2 * TC_MAX_ACC);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  const uint32_t bar_wpatch = bar_full + 8 * (2 * TC_MAX_STAGES + 8);  // [TC_EPI_WARPS][TC_PATCHES] W patches (update epilogue)
+  const uint32_t bar_wpatch = bar_full + 8 * (2 * TC_MAX_STAGES + 2 * TC_MAX_ACC + 4);  // [TC_EPI_WARPS][TC_PATCHES] W patches (update epilogue)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = leader of the pair
   const int group = blockIdx.x / NCTA, n_groups = gridDim.x / NCTA;
   constexpr bool TWO_SETS = MODE == TC_MODE_UPD || MODE == TC_MODE_SLAB;  // accumulators of both sets side by side
-  constexpr int ACC_STAGES = (TWO_SETS || MN_MAJOR) ? 1 : 2;
+  const int BN = MN_MAJOR ? TC_BN : p.bn;                        // tile columns
+  const uint32_t ACC_STAGES = (TWO_SETS || MN_MAJOR) ? 1u : (uint32_t)p.acc_stages;
   const int total_items = p.tiles_m * p.tiles_n * p.splits;      // work item = (tile of (128*NCTA) x 256, split)
 
   if (threadIdx.x == 0) {
@@ -393,7 +399,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 1);
     }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < TC_MAX_ACC; ++s) {
       mbar_init(bar_tfull + 8 * s, 1);
       mbar_init(bar_tempty + 8 * s, TC_EPI_WARPS * NCTA);  // one arrive per epilogue warp of every CTA of the group
     }
@@ -434,7 +440,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       uint32_t it = 0;  // running k-block counter (ring position)
       bool ok = true;
       const int a_rows0 = (int)rank * TC_BM;            // this CTA's rows inside the group's tile
-      const int b_cols0 = (int)rank * (TC_BN / NCTA);   // this CTA's share of the tile's columns
+      const int b_cols0 = (int)rank * (BN / NCTA);      // this CTA's share of the tile's columns
       // L2 policies of the K-major loads.  Dense forward: the group's row panels of A are reused by every
       // tile column of the rasterisation group (keep), a column panel of B only by the tiles in flight
       // (stream).  Convolution: the small weight matrix is reused by every tile (keep).
@@ -446,12 +452,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         const int kb0 = split * p.kb_per_split, kb1 = min(p.kblocks, kb0 + p.kb_per_split);
         int tm, tn;
         tile_coords(tile, p.tiles_m, p.tiles_n, p.group_m, tm, tn);
-        const int row0 = tm * (TC_BM * NCTA) + a_rows0, col0 = tn * TC_BN + b_cols0;
+        const int row0 = tm * (TC_BM * NCTA) + a_rows0, col0 = tn * BN + b_cols0;
         // forward convolution: image and first image row of this CTA's 128 output positions
         const int f_img = (!MN_MAJOR && p.conv_W) ? row0 / hw : 0;
         const int f_h0 = (!MN_MAJOR && p.conv_W) ? (row0 - f_img * hw) / p.conv_W : 0;
         // bytes the leader's barrier expects per stage from all CTAs of the group
-        uint32_t stage_tx = STAGE_BYTES * NCTA;
+        uint32_t stage_tx = MN_MAJOR ? STAGE_BYTES * NCTA : (G::A_BYTES + (uint32_t)(BN / NCTA) * CH) * NCTA;
         // weight-gradient convolution: filter tap and first channel of each of this CTA's B boxes
         int b_ci0[G::B_BOXES], b_r[G::B_BOXES], b_s[G::B_BOXES];
         if (MN_MAJOR && p.conv_W) {
@@ -545,7 +551,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   } else if (warp == 1) {
     // ------------------------------- MMA issuer (leader CTA only) ----------------------------
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = make_idesc_i8(MN_MAJOR, MN_MAJOR, NCTA);
+      const uint32_t idesc = make_idesc_i8(MN_MAJOR, MN_MAJOR, NCTA, BN);
       uint32_t it = 0, tile_it = 0;
       bool ok = true;
       for (int item = group; item < total_items && ok; item += n_groups, ++tile_it) {
@@ -558,7 +564,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         }
         tc_fence_after();
         for (int pass = 0; pass < p.npass && ok; ++pass) {
-          const uint32_t d_tmem = tmem_base + (TWO_SETS ? pass * TC_BN : as * TC_BN);
+          const uint32_t d_tmem = tmem_base + (TWO_SETS ? pass * TC_BN : as * BN);
           for (int kb = kb0; kb < kb1; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
             if (!mbar_wait<PAIR>(bar_full + 8 * s, ph, abort_flag)) {
@@ -625,9 +631,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       const int row = wrow0 + lane;
       const bool row_ok = row < p.out_rows;
       const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-      const int col0 = tn * TC_BN;
+      const int col0 = tn * BN;
       // the quadrant's two warps share the tile's valid 32-column chunks (a narrow last tile keeps both busy)
-      const int chunks = (min(TC_BN, p.out_cols - col0) + 31) >> 5;
+      const int chunks = (min(BN, p.out_cols - col0) + 31) >> 5;
       const int cbeg = half ? ((chunks + 1) >> 1) * 32 : 0;
       const int cend = half ? chunks * 32 : ((chunks + 1) >> 1) * 32;
       // Update epilogue with W patches: the 32 x 32 block of W under chunk `cb` comes into one of the warp's two
@@ -671,7 +677,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 #pragma unroll 1
         for (int cb = cbeg; cb < cend; cb += 32) {
           int v[32];
-          tc_ld32(t_row + as * TC_BN + cb, v);
+          tc_ld32(t_row + as * BN + cb, v);
           if (cb + 32 >= cend) release_acc();
           if (row_ok) {
             int32_t* dst = p.C + (size_t)row * p.out_cols + col0 + cb;
@@ -694,12 +700,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         unsigned long long ssum = 0ull;
         int mx = 0;
         int v[2][32];
-        if (cbeg < cend) tc_ld32_async(t_row + as * TC_BN + cbeg, v[0]);
+        if (cbeg < cend) tc_ld32_async(t_row + as * BN + cbeg, v[0]);
 #pragma unroll
         for (int i = 0; i < TC_EPI_COLS / 32; ++i) {
           const int cb = cbeg + i * 32;
           if (cb < cend) tc_wait_ld(v[i & 1]);
-          if (i + 1 < TC_EPI_COLS / 32 && cb + 32 < cend) tc_ld32_async(t_row + as * TC_BN + cb + 32, v[(i + 1) & 1]);
+          if (i + 1 < TC_EPI_COLS / 32 && cb + 32 < cend) tc_ld32_async(t_row + as * BN + cb + 32, v[(i + 1) & 1]);
           if (cb < cend && cb + 32 >= cend) release_acc();  // the tile's last chunk is in registers
           if (cb < cend) {  // uniform across the warp
             const int(&a)[32] = v[i & 1];
@@ -1107,8 +1113,10 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
     snprintf(t.err, sizeof(t.err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     return FF_ERR_CUDA;
   }
+  if (MN_MAJOR || p.bn <= 0) p.bn = TC_BN;
+  p.acc_stages = (int)TC_TMEM_COLS / p.bn < TC_MAX_ACC ? (int)TC_TMEM_COLS / p.bn : TC_MAX_ACC;
   p.tiles_m = cdiv(p.out_rows, TC_BM * NCTA);
-  p.tiles_n = cdiv(p.out_cols, TC_BN);
+  p.tiles_n = cdiv(p.out_cols, p.bn);
   p.group_m = MN_MAJOR ? TC_GROUP_M_MNMAJOR : TC_GROUP_M_KMAJOR;
   if (p.splits < 1) p.splits = 1;
   p.kb_per_split = cdiv(p.kblocks, p.splits);
@@ -1153,6 +1161,28 @@ inline ff_status tc_launch(TcState& t, int ncta, const CUtensorMap& a, const CUt
   const CUtensorMap& ym = y ? *y : none;
   if (ncta == 2) return tc_launch_n<MODE, MN_MAJOR, 2, CH>(t, a, b, ym, p, st);
   return tc_launch_n<MODE, MN_MAJOR, 1, CH>(t, a, b, ym, p, st);
+}
+
+// Tile width of a K-major contraction with out_rows x out_cols outputs on `groups` CTA groups of `rows_per_tile`
+// rows.  An output at most TC_BN wide takes its own width (rounded up to 32): the MMA and the B rows of a stage then
+// carry no padding.  A wider one takes, of 256, 224, 192, the width whose tiles fill the waves best - cost =
+// waves x (width + 32), the 32 standing for a tile's fixed overhead - and 256 unless a narrower one wins by 5 %:
+// narrower tiles re-read the A panel more often.
+inline int tc_pick_bn(long long out_rows, long long out_cols, int rows_per_tile, int groups) {
+  if (out_cols <= TC_BN) return (int)((out_cols + 31) / 32 * 32);
+  const long long tm = cdiv(out_rows, rows_per_tile);
+  auto cost = [&](int bn) { return (double)cdiv(tm * cdiv(out_cols, bn), groups) * (bn + 32); };
+  const double base = cost(TC_BN);
+  int best = TC_BN;
+  double best_cost = base;
+  for (int bn = TC_BN - 32; bn >= 192; bn -= 32) {
+    const double c = cost(bn);
+    if (c < 0.95 * base && c < best_cost) {
+      best = bn;
+      best_cost = c;
+    }
+  }
+  return best;
 }
 
 // K-major ("NT") problem: A [M,K], B [N,K]; K % 16 == 0 (TMA row pitch), everything else ragged.
@@ -1231,7 +1261,8 @@ inline ff_status tc_gemm(TcState& t, const int8_t* A, const int8_t* Bm, int32_t*
   if (!trans) {
     p.kblocks = cdiv(K, 128);
     if ((s = tc_make_map(t, &ta, A, K, M, 0, 128, TC_BM)) != FF_OK) return s;
-    if ((s = tc_make_map(t, &tb, Bm, K, N, 0, 128, TC_BN / ncta)) != FF_OK) return s;
+    p.bn = tc_pick_bn(M, N, TC_BM * ncta, t.sm_count / ncta);
+    if ((s = tc_make_map(t, &tb, Bm, K, N, 0, 128, p.bn / ncta)) != FF_OK) return s;
     return tc_launch<TC_MODE_RAW, false, 128>(t, ncta, ta, tb, p, st);
   }
   p.kblocks = cdiv(K, 128);
@@ -1284,7 +1315,8 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   if (!conv) {
     p.kblocks = cdiv(K, 128);
     if ((s = tc_make_map(t, &ta, A, K, M, 0, 128, TC_BM, xi ? 0 : (uint64_t)b.ld_xq)) != FF_OK) return s;
-    if ((s = tc_make_map(t, &tb, Bw, K, L.N, 0, 128, TC_BN / ncta)) != FF_OK) return s;
+    p.bn = tc_pick_bn(M, L.N, TC_BM * ncta, t.sm_count / ncta);
+    if ((s = tc_make_map(t, &tb, Bw, K, L.N, 0, 128, p.bn / ncta)) != FF_OK) return s;
     return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st, typ);
   }
   const int ch = L.Cin % 128 == 0 ? 128 : 64;
@@ -1297,7 +1329,8 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   p.conv_imgs_per_pass = B;
   p.kblocks = 9 * p.conv_cpt;
   if ((s = tc_make_map_nhwc(t, &ta, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_W, p.conv_TH, p.conv_stride)) != FF_OK) return s;
-  if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, ch, TC_BN / ncta)) != FF_OK) return s;
+  p.bn = tc_pick_bn(M, L.N, TC_BM * ncta, t.sm_count / ncta);
+  if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, ch, p.bn / ncta)) != FF_OK) return s;
   if (ch == 128) return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st, typ);
   return tc_launch<TC_MODE_FWD, false, 64>(t, ncta, ta, tb, p, st, typ);
 }
