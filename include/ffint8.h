@@ -247,8 +247,8 @@ uint64_t ff_graph_replay_count(const ff_ctx* ctx);
 ff_status ff_layer_forward(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs,
                            int B, uint64_t step, void* cuda_stream);
 
-/* Loss and output gradient of one layer (Eq. 1, Eq. 2; look-ahead Eq. 3, Eq. 4; Sec. IV-B "the
- * gradient g^Y is computed and quantized into INT8").  G_later[j] (device, [M] each) and
+/* Loss and output gradient of one layer (Eq. 1, Eq. 2; look-ahead Eq. 3, Eq. 4; Sec. IV-B: g^Y is formed and
+ * quantised to INT8 before the weight gradient).  G_later[j] (device, [M] each) and
  * theta_later[j] (host) are the goodness and thresholds of the n_later subsequent layers; with
  * n_later = 0 or lambda = 0 this is the vanilla FF loss.  Reads G, Y, rowmax, absmax[X,W].
  * Writes loss, coef, absmax[DH], dHq. */
@@ -273,7 +273,7 @@ ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer
                         int n_layers, int B, float lambda, uint64_t step, void* cuda_stream);
 
 /* One step of layer-by-layer training (Sec. III: a layer is trained to the end before its successor
- * is; Sec. IV-B trains "each layer" this way when the look-ahead of Sec. IV-C is off).  As
+ * is; Sec. IV-B trains every layer this way when the look-ahead of Sec. IV-C is off).  As
  * ff_train_step, but the layers [0, first_trained) are frozen: they run the INT8 forward with their
  * current weights and hand their normalised output on; no loss, g^Y, g^W or update is computed for
  * them and their coef, loss, dHq, absmax[DH] and W stay untouched.  Layers first_trained .. n_layers-1
@@ -284,8 +284,8 @@ ff_status ff_train_step_from(ff_ctx* ctx, const ff_layer_desc* layers, const ff_
                              int first_trained, int B, float lambda, uint64_t step, void* cuda_stream);
 
 /* Classification of B samples by goodness with the current weights.  The paper reports accuracy but
- * does not describe the procedure; this is the Forward-Forward one its Sec. III builds on ("make
- * each layer excited about positive samples"): every sample is presented once per candidate label,
+ * does not describe the procedure; this is the Forward-Forward one its Sec. III builds on (layers are
+ * trained to respond strongly to positive samples): every sample is presented once per candidate label,
  * label written one-hot into the input exactly as for the positive set; each candidate runs through
  * the same INT8 forward as training (Sec. IV-B; Alg. 1 line 5-6); the goodness of the layers
  * first_counted_layer .. n_layers-1 is added per candidate (FP32, in layer order) and the label with

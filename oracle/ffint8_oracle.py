@@ -179,7 +179,7 @@ def quantize(x: np.ndarray, a: np.float32, mode: int, key=None, idx0: int = 0,
 
 def quantize_two_pass(x: np.ndarray, B: int, mode: int, key):
     """Quantise the positive rows [0,B) and the negative rows [B,2B) with separate per-tensor
-    scales ('for each dataset (positive or negative)', Sec. IV-B).  Returns q, (a_pos, a_neg)."""
+    scales (Sec. IV-B runs the quantised workflow once per set).  Returns q, (a_pos, a_neg)."""
     q = np.empty(x.shape, dtype=np.int8)
     per_row = int(np.prod(x.shape[1:])) if x.ndim > 1 else 1
     a = []
@@ -227,7 +227,7 @@ def _pad_hw(xq: np.ndarray) -> np.ndarray:
 
 def int8_conv3x3(xq: np.ndarray, wq: np.ndarray, stride: int = 1) -> np.ndarray:
     """acc[b,i,j,co] = sum_{r,s,ci} xq[b,stride*i+r-1,stride*j+s-1,ci]*wq[co,r,s,ci], zero padding 1
-    ('dense or convolution layers', Sec. IV-B).  xq NHWC int8, wq [Cout,3,3,Cin] int8."""
+    (the convolutional form of Sec. IV-B's INT8 MAC).  xq NHWC int8, wq [Cout,3,3,Cin] int8."""
     Bn, H, Wd, Cin = xq.shape
     Cout = wq.shape[0]
     Ho, Wo = (H - 1) // stride + 1, (Wd - 1) // stride + 1
@@ -257,7 +257,7 @@ def int8_conv3x3_wgrad(dhq: np.ndarray, xq: np.ndarray, stride: int = 1) -> np.n
 
 def int8_dwconv3x3(xq: np.ndarray, wq: np.ndarray, stride: int = 1) -> np.ndarray:
     """Depthwise 3x3 MAC: acc[b,i,j,c] = sum_{r,s} xq[b,stride*i+r-1,stride*j+s-1,c]*wq[c,r,s], zero
-    padding 1 - the convolution of Sec. IV-B's 'dense or convolution layers' with one filter per
+    padding 1 - the convolutional MAC of Sec. IV-B with one filter per
     channel and no sum over channels (the depthwise layers of the paper's MobileNetV2 / EfficientNet
     models, Table II).  xq NHWC int8, wq [C,3,3] int8; exact in int64, checked against INT32."""
     Bn, H, Wd, C = xq.shape
@@ -297,7 +297,7 @@ def dequant_relu(acc: np.ndarray, c_rows: np.ndarray) -> np.ndarray:
 
 
 def goodness(acc: np.ndarray, c_rows: np.ndarray):
-    """G = ||y||^2 per sample ('sum of squared neural activities', Sec. III; Alg. 1 line 6),
+    """G = ||y||^2 per sample (the sum of the squared activities of the layer, Sec. III; Alg. 1 line 6),
     evaluated as the exact integer S = sum relu(acc)^2 scaled once: G = float(double(S)*c*c).
     Also returns S and the per-sample max of relu(acc) (used for the absmax short-cuts)."""
     n = acc.shape[0]
@@ -465,7 +465,7 @@ def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: i
     if spec.kind == KIND_LINEAR:
         st.acc = int8_gemm_nt(st.Xq, st.Wq)
     elif spec.kind == KIND_CONV1X1:
-        # pointwise convolution: the dense MAC applied at every position ('dense or convolution layers', Sec. IV-B)
+        # pointwise convolution: the dense MAC of Sec. IV-B applied at every position
         st.acc = int8_gemm_nt(st.Xq.reshape(-1, spec.K), st.Wq).reshape(st.Xq.shape[:3] + (spec.N,))
     elif spec.kind == KIND_DWCONV3X3:
         st.acc = int8_dwconv3x3(st.Xq, st.Wq.reshape(spec.N, 3, 3), spec.stride)
@@ -501,7 +501,7 @@ def layer_loss_grad(spec: LayerSpec, st: LayerState, B: int, G_later: Sequence[n
 
 def sgd_momentum(W: np.ndarray, M: np.ndarray, g: np.ndarray, lr: float, mu: float):
     """Heavy-ball SGD (Polyak): m <- mu*m + g, W <- W - lr*m, each operation one float32 rounding.
-    The paper names no optimiser for 'updated to current weights' (Sec. IV-B; Alg. 1 line 9); plain
+    The paper names no optimiser for its weight update (Sec. IV-B; Alg. 1 line 9); plain
     SGD is mu = 0, this is the usual next choice.  Returns (W_new, M_new)."""
     M_new = F32(mu) * np.asarray(M, dtype=F32) + np.asarray(g, dtype=F32)
     return np.asarray(W, dtype=F32) - F32(lr) * M_new, M_new
@@ -522,7 +522,7 @@ def _pow_int(x: float, n: int) -> float:
 
 def adam_update(W, M, V, g, lr: float, beta1: float, beta2: float, eps: float, t: int):
     """Adam (Kingma & Ba 2015, Algorithm 1) for update number t >= 1, the other usual choice where the paper
-    says only 'updated to current weights' (Sec. IV-B; Alg. 1 line 9):
+    only says that the weights are updated (Sec. IV-B; Alg. 1 line 9):
         m = beta1*m + (1-beta1)*g;  v = beta2*v + (1-beta2)*g*g;
         W -= lr * (m*c1) / (sqrt(v*c2) + eps),   c_i = float32(1/(1 - beta_i^t)).
     float32 throughout, one rounding per operation in the order written (1-beta_i is one float32

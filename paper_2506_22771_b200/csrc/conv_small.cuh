@@ -1,5 +1,5 @@
 // 3x3 convolution layers with very few input channels (the first layer of an image network: C_in <= 4, so the
-// contraction 9*C_in has at most 36 terms) - Sec. IV-B's INT8 MAC for a "convolution layer" whose contraction is far
+// contraction 9*C_in has at most 36 terms) - Sec. IV-B's INT8 MAC for a convolution layer whose contraction is far
 // too short for the tensor cores: the layer is bounded by writing its FP32 output, and a tile-based tensor-core
 // kernel spends its time on per-tile latencies instead.  Here a block builds the packed INT8 im2col words of 256
 // consecutive output positions in shared memory (zero padding by bounds checks; never written to global memory),

@@ -1,7 +1,7 @@
 // Memory-bound passes of the FF-INT8 step: absmax reduction, SUQ quantisation (Sec. IV) with
 // nearest / stochastic rounding (Sec. IV-B), goodness finalisation and length normalisation
 // (Sec. III; Alg. 1 line 6), the loss / look-ahead coefficient kernel (Eq. 1-4) and the output
-// gradient quantiser ("g^Y is computed and quantized into INT8", Sec. IV-B).
+// gradient quantiser (g^Y to INT8, Sec. IV-B).
 // All are coalesced 128-bit-load kernels with warp-shuffle reductions; grids are sized in
 // multiples of the SM count by the host code.
 #pragma once

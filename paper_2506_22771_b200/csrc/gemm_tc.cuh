@@ -3,7 +3,7 @@
 //   forward           acc[m,n]    = sum_k Xq[m,k] * Wq[n,k]                    (Sec. IV-B, INT8 MAC)
 //   weight gradient   accW_p[n,k] = sum_{m in set p} dHq[m,n] * Xq[m,k]        (Sec. IV-B, g^W)
 // for dense layers and, as implicit GEMMs, for 3x3 / stride 1 / zero-pad 1 convolutions over NHWC
-// tensors ("dense or convolution layers", Sec. IV-B): the im2col matrix is never written; the
+// tensors (Sec. IV-B names both layer types): the im2col matrix is never written; the
 // producer fetches, per filter tap, a box of the input shifted by the tap offset with a 4-D TMA
 // copy whose out-of-image part is zero-filled (zero is exact in the symmetric quantiser).
 //
