@@ -291,10 +291,11 @@ ff_status ff_train_step_from(ff_ctx* ctx, const ff_layer_desc* layers, const ff_
  * first_counted_layer .. n_layers-1 is added per candidate (FP32, in layer order) and the label with
  * the largest total wins (lowest label on ties).
  * Layout: the caller builds the candidate batch [n_classes*B, ...] in bufs[0].X, row c*B + b = sample
- * b with candidate label c, already length-normalised.  It is quantised like a training batch, with
- * one range for the first and one for the second half of its rows, so n_classes must be even and
- * every buffer of `bufs` must be sized for n_classes*B rows (i.e. as for a batch of n_classes*B/2
- * positives + negatives).  Writes scores [n_classes*B] (row c*B + b) and pred [B] (device, 16-byte
+ * b with candidate label c, already length-normalised.  Every layer input of the candidate batch is
+ * quantised with one per-tensor range (all candidates of a sample under the same quantisation step;
+ * both entries of absmax[X] / absmax[XNEXT] hold it).  The rows are processed as two halves, so
+ * n_classes*B must be even and every buffer of `bufs` must be sized for n_classes*B rows (i.e. as for
+ * a batch of n_classes*B/2 positives + negatives).  Writes scores [n_classes*B] (row c*B + b) and pred [B] (device, 16-byte
  * aligned) and, as a side effect, the forward outputs of every layer.  No weights change. */
 ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs, int n_layers, int B,
                      int n_classes, int first_counted_layer, float* scores, int32_t* pred, uint64_t step,

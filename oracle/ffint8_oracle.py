@@ -177,15 +177,18 @@ def quantize(x: np.ndarray, a: np.float32, mode: int, key=None, idx0: int = 0,
     return np.clip(q, -127.0, 127.0).astype(np.int8)
 
 
-def quantize_two_pass(x: np.ndarray, B: int, mode: int, key):
+def quantize_two_pass(x: np.ndarray, B: int, mode: int, key, joint: bool = False):
     """Quantise the positive rows [0,B) and the negative rows [B,2B) with separate per-tensor
-    scales (Sec. IV-B runs the quantised workflow once per set).  Returns q, (a_pos, a_neg)."""
+    scales (Sec. IV-B runs the quantised workflow once per set).  Returns q, (a_pos, a_neg).
+    joint: one range for the whole tensor (both entries of the returned pair are that range) - for batches whose
+    halves are not a positive and a negative set (the candidate batch of `predict`)."""
     q = np.empty(x.shape, dtype=np.int8)
     per_row = int(np.prod(x.shape[1:])) if x.ndim > 1 else 1
     a = []
+    whole = absmax(x) if joint else None
     for p in range(2):
         sl = slice(p * B, (p + 1) * B)
-        ap = absmax(x[sl])
+        ap = whole if joint else absmax(x[sl])
         q[sl] = quantize(x[sl], ap, mode, key, idx0=p * B * per_row)
         a.append(ap)
     return q, (a[0], a[1])
@@ -453,13 +456,14 @@ def add_skip(xhat: np.ndarray, skip: np.ndarray, scale: float) -> np.ndarray:
 
 
 def layer_forward(spec: LayerSpec, X: np.ndarray, W: np.ndarray, B: int, step: int,
-                  skip: Optional[np.ndarray] = None) -> LayerState:
-    """Quantise A and W, INT8 MAC, dequantise + ReLU, goodness, normalised output (+ the skip path, if any)."""
+                  skip: Optional[np.ndarray] = None, joint_range: bool = False) -> LayerState:
+    """Quantise A and W, INT8 MAC, dequantise + ReLU, goodness, normalised output (+ the skip path, if any).
+    joint_range: the input is quantised with one range for all 2B rows instead of one per set."""
     st = LayerState()
     X = np.asarray(X, dtype=F32)
     W = np.asarray(W, dtype=F32)
     st.Xq, st.a_x = quantize_two_pass(X, B, spec.round_x,
-                                      rounding_key(spec.seed, ROLE_X, spec.index, step))
+                                      rounding_key(spec.seed, ROLE_X, spec.index, step), joint_range)
     st.a_w = absmax(W)
     st.Wq = quantize(W, st.a_w, spec.round_w, rounding_key(spec.seed, ROLE_W, spec.index, step))
     if spec.kind == KIND_LINEAR:
@@ -627,17 +631,18 @@ def predict(specs: List[LayerSpec], Ws: List[np.ndarray], X_cand: np.ndarray, B:
     set), every candidate runs through the INT8 forward of all layers, the goodness of the layers
     from `first_counted` on is added up, and the label with the largest total wins (lowest label
     on ties).  X_cand [n_classes*B, ...]: row c*B + b is sample b with candidate label c, already
-    length-normalised.  The candidate batch is quantised like a training batch: per-tensor ranges
-    for its first and second half of the rows (labels 0..n/2-1 | n/2..n-1), so n_classes is even.
+    length-normalised.  Every layer input of the candidate batch is quantised with ONE per-tensor range (the
+    candidates of a sample must be compared under the same quantisation step, whichever label they carry); the
+    rows are still processed as two halves, so n_classes*B is even.
     Returns (pred [B] int32, scores [n_classes, B] float32, per-layer LayerStates)."""
-    if n_classes % 2 or n_classes <= 0:
-        raise ValueError("n_classes must be even and positive")
+    if n_classes <= 0 or (n_classes * B) % 2:
+        raise ValueError("n_classes must be positive and n_classes*B even")
     half = n_classes * B // 2
     inputs = [np.asarray(X_cand, dtype=F32)]
     states = []
     for spec, W in zip(specs, Ws):
         skip = inputs[spec.skip_from] if spec.skip_from >= 0 else None
-        st = layer_forward(spec, inputs[-1], W, half, step, skip)
+        st = layer_forward(spec, inputs[-1], W, half, step, skip, joint_range=True)
         states.append(st)
         inputs.append(st.Xnext)
     total = np.zeros(n_classes * B, dtype=F32)

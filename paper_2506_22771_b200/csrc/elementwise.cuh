@@ -34,11 +34,15 @@ __device__ __forceinline__ uint32_t block_max_u32(uint32_t v) {
 // |x| compared as bit patterns (monotone for finite floats); Inf/NaN raise ST_NONFINITE.
 // grid = (blocks, passes)
 // ---------------------------------------------------------------------------------------------
+// out2 (nullable): a second place that receives the same maximum - the other set's slot when both sets are to be
+// quantised with one joint range.
 __device__ __forceinline__ void absmax_body(const float* __restrict__ xp, size_t n_per_pass, uint32_t* __restrict__ out,
-                                            uint32_t* __restrict__ status);
+                                            uint32_t* __restrict__ status, uint32_t* __restrict__ out2 = nullptr);
 __global__ void __launch_bounds__(EW_THREADS) absmax_kernel(const float* __restrict__ x, size_t n_per_pass,
-                                                            float* __restrict__ out, uint32_t* __restrict__ status) {
-  absmax_body(x + (size_t)blockIdx.y * n_per_pass, n_per_pass, reinterpret_cast<uint32_t*>(out) + blockIdx.y, status);
+                                                            float* __restrict__ out, uint32_t* __restrict__ status,
+                                                            int joint = 0) {
+  uint32_t* o = reinterpret_cast<uint32_t*>(out);
+  absmax_body(x + (size_t)blockIdx.y * n_per_pass, n_per_pass, o + blockIdx.y, status, joint ? o + (blockIdx.y ^ 1) : nullptr);
 }
 // The same over a table of tensors in one launch (blockIdx.y = tensor): the weights of every layer and the two
 // sets of the network input are all known when a step starts.  A step of small layers is a chain of short
@@ -48,13 +52,15 @@ struct AbsmaxJobs {
   const float* x[MT_MAX];
   unsigned long long n[MT_MAX];
   float* out[MT_MAX];
+  float* out2[MT_MAX];   // nullable, see absmax_body
 };
 __global__ void __launch_bounds__(EW_THREADS) absmax_multi_kernel(AbsmaxJobs jobs, uint32_t* __restrict__ status) {
   const int t = blockIdx.y;
-  absmax_body(jobs.x[t], (size_t)jobs.n[t], reinterpret_cast<uint32_t*>(jobs.out[t]), status);
+  absmax_body(jobs.x[t], (size_t)jobs.n[t], reinterpret_cast<uint32_t*>(jobs.out[t]), status,
+              reinterpret_cast<uint32_t*>(jobs.out2[t]));
 }
 __device__ __forceinline__ void absmax_body(const float* __restrict__ xp, size_t n_per_pass, uint32_t* __restrict__ out,
-                                            uint32_t* __restrict__ status) {
+                                            uint32_t* __restrict__ status, uint32_t* __restrict__ out2) {
   uint32_t m = 0;
   const bool vec = ((n_per_pass & 3) == 0) && ((((uintptr_t)xp) & 15) == 0);
   size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -73,7 +79,10 @@ __device__ __forceinline__ void absmax_body(const float* __restrict__ xp, size_t
   m = block_max_u32(m);
   if (threadIdx.x == 0) {
     if (m >= 0x7f800000u) atomicOr(status, ST_NONFINITE);
-    if (m) atomicMax(out, m);
+    if (m) {
+      atomicMax(out, m);
+      if (out2) atomicMax(out2, m);
+    }
   }
 }
 
@@ -194,7 +203,7 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_multi_kernel(const QuantJ
 // monotone.  a_next (and a_next2, if non-NULL) receive it by atomicMax; both must be zero before.
 // ---------------------------------------------------------------------------------------------
 // write_range = 0: only G is written (the layer's output takes a skip path, so its range is found by the kernel
-// that forms the sum).
+// that forms the sum); 2: both sets' slots receive the maximum over both sets (one joint range).
 __global__ void __launch_bounds__(EW_THREADS) finalize_goodness_kernel(
     const unsigned long long* __restrict__ S, const int32_t* __restrict__ rowmax, const float* __restrict__ absmax,
     int B, float tau, float eps, float* __restrict__ G, float* __restrict__ a_next, float* __restrict__ a_next2,
@@ -215,6 +224,10 @@ __global__ void __launch_bounds__(EW_THREADS) finalize_goodness_kernel(
   if (threadIdx.x == 0 && mx && write_range) {
     atomicMax(reinterpret_cast<uint32_t*>(a_next) + p, mx);
     if (a_next2) atomicMax(reinterpret_cast<uint32_t*>(a_next2) + p, mx);
+    if (write_range == 2) {
+      atomicMax(reinterpret_cast<uint32_t*>(a_next) + (p ^ 1), mx);
+      if (a_next2) atomicMax(reinterpret_cast<uint32_t*>(a_next2) + (p ^ 1), mx);
+    }
   }
 }
 
@@ -352,7 +365,8 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_skip_kernel(const float*
                                                                     float tau, float eps, size_t per_sample, size_t per_pass,
                                                                     const float* __restrict__ skip, float scale,
                                                                     float* __restrict__ xnext, float* __restrict__ a_next,
-                                                                    float* __restrict__ a_next2, uint32_t* __restrict__ status) {
+                                                                    float* __restrict__ a_next2, uint32_t* __restrict__ status,
+                                                                    int joint = 0) {
   const size_t base = (size_t)blockIdx.y * per_pass;
   const bool vec = ((per_sample & 3) == 0) && ((((uintptr_t)Y) & 15) == 0) && ((((uintptr_t)xnext) & 15) == 0) &&
                    ((((uintptr_t)skip) & 15) == 0);
@@ -391,6 +405,10 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_skip_kernel(const float*
     if (mx) {
       atomicMax(reinterpret_cast<uint32_t*>(a_next) + blockIdx.y, mx);
       if (a_next2) atomicMax(reinterpret_cast<uint32_t*>(a_next2) + blockIdx.y, mx);
+      if (joint) {
+        atomicMax(reinterpret_cast<uint32_t*>(a_next) + (blockIdx.y ^ 1), mx);
+        if (a_next2) atomicMax(reinterpret_cast<uint32_t*>(a_next2) + (blockIdx.y ^ 1), mx);
+      }
     }
   }
 }

@@ -45,6 +45,8 @@ struct ff_ctx {
     int B_local = 0;
   } shard;
   bool accumulate_only = false;  // weight-gradient contractions leave their INT32 sums in accW_dump, no update
+  bool joint_range = false;      // the two halves of the batch are quantised with one range (classification: the halves
+                                 // are groups of candidate labels, not a positive and a negative set)
   // captured launch sequences of ff_train_step (ff_set_graph_mode)
   bool graph_mode = false;
   struct GraphEntry {
@@ -738,7 +740,7 @@ ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     ProfScope prof(ctx, FF_K_FINALIZE, st);
     finalize_goodness_kernel<<<dim3(ew_blocks(ctx, B, 1), 2), EW_THREADS, 0, st>>>(
         reinterpret_cast<const unsigned long long*>(b.S), b.rowmax, b.absmax, B, L.tau, L.eps, b.G,
-        b.absmax + FF_A_XNEXT_POS, a_next2, b.Skip ? 0 : 1);
+        b.absmax + FF_A_XNEXT_POS, a_next2, b.Skip ? 0 : (ctx->joint_range ? 2 : 1));
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -751,7 +753,7 @@ ff_status quantize_input(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_buf
   if (do_absmax) {
     ProfScope prof(ctx, FF_K_ABSMAX, st);
     absmax_kernel<<<dim3(ew_blocks(ctx, per_pass / 4 + 1), 2), EW_THREADS, 0, st>>>(b.X, per_pass, b.absmax + FF_A_X_POS,
-                                                                                 status_ptr(ctx));
+                                                                                 status_ptr(ctx), ctx->joint_range ? 1 : 0);
   }
   if (do_absmax) FF_LAUNCH_CHECK(ctx);
   if (!do_quantize) return FF_OK;
@@ -785,7 +787,8 @@ ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
     {
       ProfScope prof(ctx, FF_K_NORMALIZE, st);
       normalize_skip_kernel<<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Skip, L.skip_scale, b.Xnext,
-                                                        b.absmax + FF_A_XNEXT_POS, a_next2, status_ptr(ctx));
+                                                        b.absmax + FF_A_XNEXT_POS, a_next2, status_ptr(ctx),
+                                                        ctx->joint_range ? 1 : 0);
     }
     FF_LAUNCH_CHECK(ctx);
     if (!xq_next) return FF_OK;
@@ -922,6 +925,7 @@ ff_status quantize_inputs_and_weights(ff_ctx* ctx, const ff_layer_desc* layers, 
   const uint2 bias0 = ctr_bias(ctx, per_sample0, B);
   for (int p = 0; p < 2; ++p, ++t) {
     aj.x[t] = bufs[0].X + p * per_pass0, aj.n[t] = per_pass0, aj.out[t] = bufs[0].absmax + FF_A_X_POS + p;
+    aj.out2[t] = ctx->joint_range ? bufs[0].absmax + FF_A_X_POS + (p ^ 1) : nullptr;
     qj.x[t] = aj.x[t], qj.q[t] = bufs[0].Xq, qj.e0[t] = p * per_pass0, qj.n[t] = per_pass0, qj.a[t] = aj.out[t];
     qj.pad[t] = row_pad(L0.K, bufs[0].ld_xq);
     qj.s1[t] = make_key_spec(L0.seed, ROLE_X, L0.index, nullptr).s1;
@@ -931,7 +935,7 @@ ff_status quantize_inputs_and_weights(ff_ctx* ctx, const ff_layer_desc* layers, 
   largest = per_pass0;
   for (int l = 0; l < n; ++l, ++t) {
     const size_t nW = (size_t)layers[l].N * layers[l].K;
-    aj.x[t] = bufs[l].W, aj.n[t] = nW, aj.out[t] = bufs[l].absmax + FF_A_W;
+    aj.x[t] = bufs[l].W, aj.n[t] = nW, aj.out[t] = bufs[l].absmax + FF_A_W, aj.out2[t] = nullptr;
     qj.x[t] = bufs[l].W, qj.q[t] = bufs[l].Wq, qj.n[t] = nW, qj.a[t] = aj.out[t];
     qj.s1[t] = make_key_spec(layers[l].seed, ROLE_W, layers[l].index, nullptr).s1;
     qj.ctr0[t] = 0u;
@@ -1414,8 +1418,9 @@ ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bu
                      int first_counted_layer, float* scores, int32_t* pred, uint64_t step, void* cuda_stream) {
   ff_status s = check_ctx(ctx);
   if (s != FF_OK) return s;
-  if (n_classes <= 0 || (n_classes & 1)) return fail(ctx, FF_ERR_ARG, "n_classes must be even and positive");
+  if (n_classes <= 0) return fail(ctx, FF_ERR_ARG, "n_classes must be positive");
   if (B <= 0) return fail(ctx, FF_ERR_ARG, "B must be positive");
+  if (((long long)n_classes * B) & 1) return fail(ctx, FF_ERR_ARG, "n_classes * B must be even (the candidate rows are processed as two halves)");
   if (!scores || !pred) return fail(ctx, FF_ERR_ARG, "scores / pred is NULL");
   if (!aligned16(scores) || !aligned16(pred)) return fail(ctx, FF_ERR_ALIGN, "scores / pred must be 16-byte aligned");
   if ((long long)n_classes * B / 2 >= (1LL << 30)) return fail(ctx, FF_ERR_RANGE, "too many candidate rows");
@@ -1426,7 +1431,9 @@ ff_status ff_predict(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bu
   if ((s = ensure_status(ctx, st)) != FF_OK) return s;
   if ((s = set_step(ctx, step, 0.0f, false, st, bufs, n_layers)) != FF_OK) return s;
   auto body = [&](cudaStream_t sb) -> ff_status {
+    ctx->joint_range = true;    // one quantiser range per tensor for the whole candidate batch
     ff_status r = forward_all(ctx, layers, bufs, n_layers, half, sb);
+    ctx->joint_range = false;
     if (r != FF_OK) return r;
     LaterLayers gs;
     gs.n = n_layers - first_counted_layer;

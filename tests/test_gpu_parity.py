@@ -306,9 +306,12 @@ def test_predict_matches_oracle(path, first_counted):
     # weights untouched
     for b, W in zip(net.bufs, Ws):
         assert torch.equal(b.W.cpu(), torch.from_numpy(W))
+    for l, st in enumerate(states):          # one range for both halves of the candidate rows
+        am = net.bufs[l].absmax.cpu().numpy()
+        assert am[0] == am[1] == np.float32(st.a_x[0]) == np.float32(st.a_x[1])
     with pytest.raises(ffb.FFError) as e:
-        ffb.ff_predict(net.ctx.ctx, net.descs_arr, net.bufs_arr, len(descs), B, 9, 0, scores.data_ptr(), pred.data_ptr(), 0, 0)
-    assert e.value.code == ffb.FF_ERR_ARG
+        ffb.ff_predict(net.ctx.ctx, net.descs_arr, net.bufs_arr, len(descs), 1, 9, 0, scores.data_ptr(), pred.data_ptr(), 0, 0)
+    assert e.value.code == ffb.FF_ERR_ARG         # 9 candidate rows cannot be split into two halves
     net.close()
 
 

@@ -515,6 +515,33 @@ def test_predict_hand_example_and_tie_rule():
     assert np.array_equal(s01.reshape(-1), (st01[0].G + st01[1].G).astype(np.float32))
 
 
+def test_predict_compares_all_candidates_under_one_quantisation_step():
+    """The candidate batch is quantised with one range per tensor: the scores of a sample's candidates then do not
+    depend on where a candidate sits in the batch.  With nearest rounding (no element counters involved) a
+    permutation of the candidate labels permutes the scores exactly; with one range per half it would not."""
+    g = np.random.default_rng(5)
+    K, N, C, B = 24, 16, 6, 5
+    specs = [O.LayerSpec(O.KIND_LINEAR, K, N, float(N), 0.0, float(np.sqrt(N)), round_x=0, round_w=0, round_dh=0, index=0),
+             O.LayerSpec(O.KIND_LINEAR, N, N, float(N), 0.0, float(np.sqrt(N)), round_x=0, round_w=0, round_dh=0, index=1)]
+    Ws = [g.normal(size=(N, K)).astype(F32) * 0.3, g.normal(size=(N, N)).astype(F32) * 0.3]
+    X = g.normal(size=(C, B, K)).astype(F32)
+    X[3] *= 4.0                                    # one candidate with a much larger range than the others
+    _, scores, states = O.predict(specs, Ws, X.reshape(C * B, K), B, C, step=0)
+    perm = np.array([4, 0, 3, 5, 1, 2])
+    _, scores_p, _ = O.predict(specs, Ws, X[perm].reshape(C * B, K), B, C, step=0)
+    assert np.array_equal(scores_p, scores[perm])
+    assert states[0].a_x[0] == states[0].a_x[1] == O.absmax(X)
+    # the per-half ranges of a training batch do depend on the placement (the case the classification must avoid)
+    a = O.layer_forward(specs[0], X.reshape(C * B, K), Ws[0], C * B // 2, 0)
+    b = O.layer_forward(specs[0], X[perm].reshape(C * B, K), Ws[0], C * B // 2, 0)
+    assert a.a_x != b.a_x
+    # an odd number of classes is fine as long as the rows split into two halves
+    pred, sc, _ = O.predict(specs, Ws, X[:5, :4].reshape(20, K), 4, 5, step=0)
+    assert sc.shape == (5, 4) and pred.shape == (4,)
+    with pytest.raises(ValueError):
+        O.predict(specs, Ws, X[:5, :3].reshape(15, K), 3, 5, step=0)
+
+
 def test_int8_ff_training_learns_and_predicts_separable_classes():
     """End-to-end direction check of the whole oracle: FF-INT8 training (positive set = true label, negative
     set = wrong label, Eq. 1 / Eq. 2, INT8 gradients) followed by classification by goodness must learn
