@@ -82,6 +82,9 @@ struct TcParams {
                             // B a stage holds follow it, so a narrow layer wastes neither, and a wide one can pick the
                             // width that fills its last wave of tiles best; MN-major kernels always use TC_BN
   int acc_stages;           // K-major forward: accumulator stages in tensor memory (512 / bn, at most 4)
+  int b_resident;           // K-major, one tile column: the whole B operand (all contraction blocks of this CTA's rows of
+                            // B) is loaded once and stays in shared memory; the stages then hold A only.  A convolution's
+                            // weights are the same for every tile, and the loads from L2 are what bounds these kernels.
   uint32_t* status;
   // raw
   int32_t* C;
@@ -385,6 +388,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_MAX_STAGES + 2 * TC_MAX_ACC);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   const uint32_t bar_wpatch = bar_full + 8 * (2 * TC_MAX_STAGES + 2 * TC_MAX_ACC + 4);  // [TC_EPI_WARPS][TC_PATCHES] W patches (update epilogue)
+  const uint32_t bar_bres = bar_wpatch + 8 * (TC_EPI_WARPS * TC_PATCHES);               // [1] resident B operand landed (leader CTA)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = leader of the pair
@@ -405,6 +409,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     }
     if (MODE == TC_MODE_UPD)
       for (int s = 0; s < TC_EPI_WARPS * TC_PATCHES; ++s) mbar_init(bar_wpatch + 8 * s, 1);
+    mbar_init(bar_bres, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -447,6 +452,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       const uint64_t pol_keep = l2_policy_evict_last(), pol_stream = l2_policy_evict_first();
       const int hw = p.conv_H * p.conv_W;
       const int blocks_per_img = p.conv_W ? p.conv_H / p.conv_TH : 1;
+      const bool b_res = !MN_MAJOR && p.b_resident;
+      const uint32_t b_box_bytes = (uint32_t)(BN / NCTA) * CH;               // one contraction block of this CTA's B rows
+      const uint32_t bres_base = ring + STAGES * G::A_BYTES;                 // resident B: behind the (A-only) stages
+      if (b_res && group < total_items) {
+        if (rank == 0) mbar_expect_tx(bar_bres, b_box_bytes * (uint32_t)p.kblocks * NCTA);
+        const uint32_t rb = PAIR ? map_to_cta(bar_bres, 0) : bar_bres;
+        for (int kb = 0; kb < p.kblocks; ++kb) tma_load_2d<NCTA>(bres_base + kb * b_box_bytes, &tmB, rb, kb * CH, b_cols0, pol_keep);
+      }
       for (int item = group; item < total_items && ok; item += n_groups) {
         const int tile = item / p.splits, split = item - tile * p.splits;
         const int kb0 = split * p.kb_per_split, kb1 = min(p.kblocks, kb0 + p.kb_per_split);
@@ -457,7 +470,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         const int f_img = (!MN_MAJOR && p.conv_W) ? row0 / hw : 0;
         const int f_h0 = (!MN_MAJOR && p.conv_W) ? (row0 - f_img * hw) / p.conv_W : 0;
         // bytes the leader's barrier expects per stage from all CTAs of the group
-        uint32_t stage_tx = MN_MAJOR ? STAGE_BYTES * NCTA : (G::A_BYTES + (uint32_t)(BN / NCTA) * CH) * NCTA;
+        uint32_t stage_tx = MN_MAJOR ? STAGE_BYTES * NCTA : (G::A_BYTES + (b_res ? 0u : b_box_bytes)) * NCTA;
         // weight-gradient convolution: filter tap and first channel of each of this CTA's B boxes
         int b_ci0[G::B_BOXES], b_r[G::B_BOXES], b_s[G::B_BOXES];
         if (MN_MAJOR && p.conv_W) {
@@ -493,7 +506,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               ok = false;
               break;
             }
-            const uint32_t a_dst = ring + s * STAGE_BYTES, b_dst = a_dst + G::A_BYTES;
+            const uint32_t a_dst = ring + s * (b_res ? G::A_BYTES : STAGE_BYTES), b_dst = a_dst + G::A_BYTES;
             if (MODE == TC_MODE_UPD && pass == p.npass - 1 && kb == max(kb0, kb1 - TC_PREFETCH_KB)) {
               // pull this CTA's W rows of the tile into L2 shortly before the epilogue's read-modify-write
               const int c0w = tn * TC_BN;
@@ -520,7 +533,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               } else {
                 tma_load_2d<NCTA>(a_dst, &tmA, fb, kb * CH, row0, pol_keep);
               }
-              tma_load_2d<NCTA>(b_dst, &tmB, fb, kb * CH, col0, p.conv_W ? pol_keep : pol_stream);
+              if (!b_res) tma_load_2d<NCTA>(b_dst, &tmB, fb, kb * CH, col0, p.conv_W ? pol_keep : pol_stream);
             } else {
               // boxes of 128 contraction rows x 128 (A) or CH (B) output indices
               tma_load_3d<NCTA>(a_dst, &tmA, fb, row0, kb * 128, pass);
@@ -554,6 +567,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
       const uint32_t idesc = make_idesc_i8(MN_MAJOR, MN_MAJOR, NCTA, BN);
       uint32_t it = 0, tile_it = 0;
       bool ok = true;
+      const bool b_res = !MN_MAJOR && p.b_resident;
+      const uint32_t b_box_bytes = (uint32_t)(BN / NCTA) * CH, bres_base = ring + STAGES * G::A_BYTES;
+      if (b_res && group < total_items && !mbar_wait<PAIR>(bar_bres, 0u, abort_flag)) ok = false;
       for (int item = group; item < total_items && ok; item += n_groups, ++tile_it) {
         const int split = item % p.splits;
         const int kb0 = split * p.kb_per_split, kb1 = min(p.kblocks, kb0 + p.kb_per_split);
@@ -572,7 +588,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
               break;
             }
             tc_fence_after();
-            const uint32_t a_src = ring + s * STAGE_BYTES, b_src = a_src + G::A_BYTES;
+            const uint32_t a_src = ring + s * (b_res ? G::A_BYTES : STAGE_BYTES);
+            const uint32_t b_src = b_res ? bres_base + (uint32_t)kb * b_box_bytes : a_src + G::A_BYTES;
 #pragma unroll
             for (int k = 0; k < G::MMAS; ++k) {
               uint64_t ad, bd;
@@ -1117,6 +1134,11 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
   p.acc_stages = (int)TC_TMEM_COLS / p.bn < TC_MAX_ACC ? (int)TC_TMEM_COLS / p.bn : TC_MAX_ACC;
   p.tiles_m = cdiv(p.out_rows, TC_BM * NCTA);
   p.tiles_n = cdiv(p.out_cols, p.bn);
+  // one tile column, more tiles than CTA groups (some group reuses B), and all of B's contraction blocks fit where the
+  // stages' B parts were
+  p.b_resident = (!MN_MAJOR && (MODE == TC_MODE_FWD || MODE == TC_MODE_RAW) && p.tiles_n == 1 && p.splits <= 1 &&
+                  p.tiles_m > t.sm_count / NCTA &&
+                  (size_t)p.kblocks * (p.bn / NCTA) * CH <= (size_t)G::STAGES * G::B_BYTES) ? 1 : 0;
   p.group_m = MN_MAJOR ? TC_GROUP_M_MNMAJOR : TC_GROUP_M_KMAJOR;
   if (p.splits < 1) p.splits = 1;
   p.kb_per_split = cdiv(p.kblocks, p.splits);

@@ -47,7 +47,11 @@ def test_int8_gemm_simt(M, N, K, trans):
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 256, 128), (128, 256, 512), (256, 512, 1024), (200, 300, 784),
-                                   (1000, 2000, 2000), (16, 16, 16), (4096, 2048, 4096)])
+                                   (1000, 2000, 2000), (16, 16, 16), (4096, 2048, 4096),
+                                   # one tile column and more tiles than CTA groups: B stays resident in shared memory
+                                   (40000, 128, 576), (20000, 96, 1104), (39000, 256, 640),
+                                   # tile widths of 224 and 192 columns (the width that fills the last wave best)
+                                   (8192, 2000, 256), (4096, 1100, 256)])
 @pytest.mark.parametrize("form", TENSOR_FORMS)
 def test_int8_gemm_tensor_forward_orientation(M, N, K, form):
     _gemm_case(M, N, K, 0, ffb.FF_GEMM_TENSOR, form)
@@ -202,6 +206,17 @@ def _conv_workload(chans, H, Wd, B):
                                           ((3, 128, 80), 16, 64, 1)])        # ragged Cout, 2 rows per block
 def test_conv_tensor_core_shapes(path, chans, H, Wd, B):
     _run_and_compare(_conv_workload(chans, H, Wd, B), seed=31, steps=2, lam_per_step=0.1, path=path)
+
+
+@pytest.mark.parametrize("form", TENSOR_FORMS)
+def test_conv_layer_with_resident_weights(form):
+    # 64 -> 128 channels on 16 x 16 images, 80 + 80 samples: 160 (320) tiles on 74 (148) CTA groups, one tile column -
+    # the forward keeps the layer's INT8 weights in shared memory and streams the input boxes only
+    hw = 16
+    layers = [synth.LayerCfg(1, 9 * 64, 128, float(128 * hw * hw) / 2, 0.03 / (hw * hw), float(np.sqrt(128 * hw * hw)), H=hw, Wd=hw,
+                             Cin=64)]
+    w = synth.Workload("conv_res", 80, layers, (hw, hw, 64), "normal", "kaiming_uniform", 2)
+    _run_and_compare(w, seed=8, steps=2, lam_per_step=0.0, path=(ffb.FF_GEMM_TENSOR, form))
 
 
 @pytest.mark.parametrize("form", TENSOR_FORMS)
