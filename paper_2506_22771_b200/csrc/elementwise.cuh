@@ -207,7 +207,9 @@ __global__ void __launch_bounds__(EW_THREADS) quantize_multi_kernel(const QuantJ
 __global__ void __launch_bounds__(EW_THREADS) finalize_goodness_kernel(
     const unsigned long long* __restrict__ S, const int32_t* __restrict__ rowmax, const float* __restrict__ absmax,
     int B, float tau, float eps, float* __restrict__ G, float* __restrict__ a_next, float* __restrict__ a_next2,
-    int write_range = 1) {
+    int write_range = 1, float* __restrict__ Rn = nullptr) {
+  // Rn (nullable, [2B]): receives the per-sample factor tau/(sqrt(G)+eps), so that the normalisation pass of short
+  // samples reads it instead of forming a square root and a division per group of four elements
   const int p = blockIdx.y;
   const float c = __fmul_rn(scale_of(absmax[p]), scale_of(absmax[2]));
   const double c2 = __dmul_rn((double)c, (double)c);
@@ -217,6 +219,7 @@ __global__ void __launch_bounds__(EW_THREADS) finalize_goodness_kernel(
     float g = __double2float_rn(__dmul_rn(__ull2double_rn(S[m]), c2));
     G[m] = g;
     float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(g), eps));
+    if (Rn) Rn[m] = r;
     float xm = __fmul_rn(__fmul_rn(__int2float_rn(rowmax[m]), c), r);
     mx = max(mx, __float_as_uint(xm));
   }
@@ -265,8 +268,9 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
                                                                size_t per_pass, float* __restrict__ xnext,
                                                                int8_t* __restrict__ xq, const float* __restrict__ a,
                                                                KeySpec ks, uint2 ctr_bias = uint2{0u, 0u},
-                                                               RowPad rp = RowPad{0u, 0u}) {
+                                                               RowPad rp = RowPad{0u, 0u}, const float* __restrict__ Rn = nullptr) {
   // rp: row padding of xq (dense layers only: a row is a sample, so sample index * extra is the shift)
+  // Rn (nullable): the per-sample factors tau/(sqrt(G)+eps) as finalize_goodness_kernel left them (the same bits)
   const RoundKey key = (MODE == ROUND_NEAREST) ? RoundKey{0u, 0u} : derive_key(ks);
   const uint32_t bias = blockIdx.y ? ctr_bias.y : ctr_bias.x;
   const size_t base = (size_t)blockIdx.y * per_pass;
@@ -325,7 +329,7 @@ __global__ void __launch_bounds__(EW_THREADS) normalize_kernel(const float* __re
         const uint32_t i = i0 + k * stride;
         if (i >= n4) break;
         const size_t e = base + ((size_t)i << 2);
-        const float r = __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(__ldg(Gp + cur.sample)), eps));
+        const float r = Rn ? __ldg(Rn + pass_row0 + cur.sample) : __fdiv_rn(tau, __fadd_rn(__fsqrt_rn(__ldg(Gp + cur.sample)), eps));
         float4 v = vv[k];
         v.x = __fmul_rn(v.x, r);
         v.y = __fmul_rn(v.y, r);

@@ -203,6 +203,13 @@ ff_status check_ctx(ff_ctx* ctx) {
 }
 
 inline uint32_t* status_ptr(ff_ctx* ctx) { return reinterpret_cast<uint32_t*>(ctx->workspace); }
+// Per-sample normalisation factors of the layer whose forward has just run ([2B] floats at the start of the
+// transient region: written by the goodness finalisation, read by the normalisation pass that follows it, before
+// anything else uses the region); NULL when the workspace has no room, the pass then forms them itself.
+inline float* factors_ptr(ff_ctx* ctx, int B) {
+  if (ctx->workspace_bytes < WS_BYTES + (size_t)2 * B * sizeof(float)) return nullptr;
+  return reinterpret_cast<float*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
+}
 inline StepState* step_ptr(ff_ctx* ctx) {
   return reinterpret_cast<StepState*>(static_cast<char*>(ctx->workspace) + WS_STEP_OFFSET);
 }
@@ -740,7 +747,7 @@ ff_status forward_from_xq(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
     ProfScope prof(ctx, FF_K_FINALIZE, st);
     finalize_goodness_kernel<<<dim3(ew_blocks(ctx, B, 1), 2), EW_THREADS, 0, st>>>(
         reinterpret_cast<const unsigned long long*>(b.S), b.rowmax, b.absmax, B, L.tau, L.eps, b.G,
-        b.absmax + FF_A_XNEXT_POS, a_next2, b.Skip ? 0 : (ctx->joint_range ? 2 : 1));
+        b.absmax + FF_A_XNEXT_POS, a_next2, b.Skip ? 0 : (ctx->joint_range ? 2 : 1), factors_ptr(ctx, B));
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -840,16 +847,16 @@ ff_status normalize_output(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_b
     const float* a = b.absmax + FF_A_XNEXT_POS;
     if (nearest && !rp.extra)
       normalize_kernel<ROUND_NEAREST, false><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
-                                                                         xq_next, a, key, bias);
+                                                                         xq_next, a, key, bias, RowPad{0u, 0u}, factors_ptr(ctx, B));
     else if (nearest)
       normalize_kernel<ROUND_NEAREST, true><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
-                                                                        xq_next, a, key, bias, rp);
+                                                                        xq_next, a, key, bias, rp, factors_ptr(ctx, B));
     else if (!rp.extra)
       normalize_kernel<ROUND_STOCHASTIC, false><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
-                                                                            xq_next, a, key, bias);
+                                                                            xq_next, a, key, bias, RowPad{0u, 0u}, factors_ptr(ctx, B));
     else
       normalize_kernel<ROUND_STOCHASTIC, true><<<grid, EW_THREADS, 0, st>>>(b.Y, b.G, L.tau, L.eps, per_sample, per_pass, b.Xnext,
-                                                                           xq_next, a, key, bias, rp);
+                                                                           xq_next, a, key, bias, rp, factors_ptr(ctx, B));
   }
   FF_LAUNCH_CHECK(ctx);
   return FF_OK;
@@ -1272,6 +1279,7 @@ ff_status ff_workspace_bytes(const ff_layer_desc* layers, int n_layers, int B, s
       const size_t two = (size_t)4 * layers[l].N * layers[l].K * sizeof(int32_t);
       if (two > need) need = two;
     }
+    if (need < (size_t)2 * B * sizeof(float)) need = (size_t)2 * B * sizeof(float);   // per-sample normalisation factors
     if (layers[l].optimizer == FF_OPT_ADAM) need = up256(need) + adam_plane_bytes(layers[l]) + 256;  // sums plane at the tail
     if (need > slab) slab = need;
   }
