@@ -51,6 +51,7 @@ constexpr int TC_PREFETCH_KB = 8;                         // W tile is prefetche
 // 8 makes a wave of 74 CTA pairs nearly square (8 x 9 panels instead of 16 x 5).
 constexpr int TC_GROUP_M_KMAJOR = 16, TC_GROUP_M_MNMAJOR = 8;
 constexpr uint32_t TC_TMEM_COLS = 512;
+constexpr uint32_t TC_TALL_ROWS = 192;                    // rows of a tall convolution stage: (128 / W + 2) * W for W <= 32
 constexpr int TC_MAX_ACC = 4;                             // most accumulator stages (narrow forward tiles)
 constexpr unsigned long long TC_WAIT_NS = 2000000000ull;  // 2 s bound on every wait
 
@@ -82,6 +83,7 @@ struct TcParams {
                             // B a stage holds follow it, so a narrow layer wastes neither, and a wide one can pick the
                             // width that fills its last wave of tiles best; MN-major kernels always use TC_BN
   int acc_stages;           // K-major forward: accumulator stages in tensor memory (512 / bn, at most 4)
+  int tall_slots;           // stages of TC_TALL_ROWS rows that fit where the A halves of the ordinary stages were
   int b_resident;           // K-major, one tile column: the whole B operand (all contraction blocks of this CTA's rows of
                             // B) is loaded once and stays in shared memory; the stages then hold A only.  A convolution's
                             // weights are the same for every tile, and the loads from L2 are what bounds these kernels.
@@ -105,6 +107,9 @@ struct TcParams {
   float* mom;               // nullable heavy-ball buffer [out_rows, out_cols]: m = mu*m + g, W -= lr*m
   float mu;
   // split weight gradient
+  int conv_tall;            // convolution forward with resident weights, stride 1: one input box of conv_TH + 2 image rows
+                            // per horizontal tap offset and channel chunk serves the three vertical taps (the taps are the
+                            // same box shifted by whole image rows, i.e. by whole swizzle atoms): a third of the box loads
   int32_t* slabs;
   int splits_per_slab;      // > 1: that many consecutive splits add their partial sums into one slab with integer
                             // atomics (exact, order-free; the slab is cleared before the launch); 1: a slab per split
@@ -484,6 +489,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
             b_s[q] = tap - b_r[q] * 3;
           }
         }
+        if (!MN_MAJOR && p.conv_tall) {
+          // tall boxes: stage = (conv_TH + 2) image rows x conv_W pixels x CH channels for tap column s, chunk cc
+          const uint32_t tall_rows = (uint32_t)(p.conv_TH + 2) * p.conv_W, slots = (uint32_t)p.tall_slots;
+          for (int ts = 0; ts < 3 && ok; ++ts)
+            for (int cc = 0; cc < p.conv_cpt; ++cc, ++it) {
+              const uint32_t s = it % slots, ph = (it / slots) & 1u;
+              if (!mbar_wait<PAIR>(bar_empty + 8 * s, ph ^ 1u, abort_flag)) {
+                ok = false;
+                break;
+              }
+              if (rank == 0) mbar_expect_tx(bar_full + 8 * s, tall_rows * CH * NCTA);
+              tma_load_4d<NCTA>(ring + s * TC_TALL_ROWS * CH, &tmA, lead_full + 8 * s, cc * CH, ts - 1, f_h0 - 1, f_img);
+            }
+          continue;
+        }
         for (int pass = 0; pass < p.npass && ok; ++pass) {
           // forward convolution: (filter row, filter column, channel chunk) of k-block kb, kept by counting
           int f_r = 0, f_s = 0, f_cc = 0;
@@ -579,6 +599,35 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           break;
         }
         tc_fence_after();
+        if (!MN_MAJOR && p.conv_tall) {
+          const uint32_t d_tmem = tmem_base + as * BN, slots = (uint32_t)p.tall_slots;
+          const uint32_t view_bytes = (uint32_t)p.conv_W * CH;   // one image row of the box: the step between vertical taps
+          uint32_t first = 1u;
+          for (int ts = 0; ts < 3 && ok; ++ts)
+            for (int cc = 0; cc < p.conv_cpt; ++cc, ++it) {
+              const uint32_t s = it % slots, ph = (it / slots) & 1u;
+              if (!mbar_wait<PAIR>(bar_full + 8 * s, ph, abort_flag)) {
+                ok = false;
+                break;
+              }
+              tc_fence_after();
+              const uint32_t a_box = ring + s * TC_TALL_ROWS * CH;
+#pragma unroll
+              for (int tr = 0; tr < 3; ++tr) {
+                const uint32_t a_src = a_box + tr * view_bytes;
+                const uint32_t b_src = bres_base + (uint32_t)((tr * 3 + ts) * p.conv_cpt + cc) * b_box_bytes;
+#pragma unroll
+                for (int k = 0; k < G::MMAS; ++k) {
+                  tc_mma_i8<NCTA>(d_tmem, make_smem_desc(a_src + k * 32, 16, 8 * CH, G::SWZ),
+                                  make_smem_desc(b_src + k * 32, 16, 8 * CH, G::SWZ), idesc, first ? 0u : 1u);
+                  first = 0u;
+                }
+              }
+              tc_commit<NCTA>(bar_empty + 8 * s);
+            }
+          if (ok) tc_commit<NCTA>(bar_tfull + 8 * as);
+          continue;
+        }
         for (int pass = 0; pass < p.npass && ok; ++pass) {
           const uint32_t d_tmem = tmem_base + (TWO_SETS ? pass * TC_BN : as * BN);
           for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -1120,6 +1169,20 @@ inline ff_status tc_make_store_map(TcState& t, CUtensorMap* tm, float* base, uin
   return FF_OK;
 }
 
+// Shared-memory budget of the K-major kernels as the host sees it (mirrors TcGeom<false, NCTA, CH>).
+inline int tc_kmajor_stages(int ncta, int ch) {
+  const int stage = 128 * ch + (TC_BN / ncta) * ch;
+  const int n = (int)(TC_RING_BYTES / stage);
+  return n < TC_MAX_STAGES ? n : TC_MAX_STAGES;
+}
+// The B operand stays resident when the contraction has one tile column, more tiles than CTA groups (some group
+// reuses B), and all of B's contraction blocks fit where the stages' B parts were.
+inline bool tc_resident_ok(long long out_rows, long long out_cols, int bn, int kblocks, int ncta, int ch, int sm_count) {
+  if (cdiv(out_cols, bn) != 1 || cdiv(out_rows, TC_BM * ncta) <= sm_count / ncta) return false;
+  return (size_t)kblocks * (bn / ncta) * ch <= (size_t)tc_kmajor_stages(ncta, ch) * (TC_BN / ncta) * ch;
+}
+inline int tc_tall_slots(int ncta, int ch) { return (int)((size_t)tc_kmajor_stages(ncta, ch) * 128 * ch / ((size_t)TC_TALL_ROWS * ch)); }
+
 template <int MODE, bool MN_MAJOR, int NCTA, int CH>
 inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& y, TcParams p,
                              cudaStream_t st) {
@@ -1134,11 +1197,13 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
   p.acc_stages = (int)TC_TMEM_COLS / p.bn < TC_MAX_ACC ? (int)TC_TMEM_COLS / p.bn : TC_MAX_ACC;
   p.tiles_m = cdiv(p.out_rows, TC_BM * NCTA);
   p.tiles_n = cdiv(p.out_cols, p.bn);
-  // one tile column, more tiles than CTA groups (some group reuses B), and all of B's contraction blocks fit where the
-  // stages' B parts were
-  p.b_resident = (!MN_MAJOR && (MODE == TC_MODE_FWD || MODE == TC_MODE_RAW) && p.tiles_n == 1 && p.splits <= 1 &&
-                  p.tiles_m > t.sm_count / NCTA &&
-                  (size_t)p.kblocks * (p.bn / NCTA) * CH <= (size_t)G::STAGES * G::B_BYTES) ? 1 : 0;
+  p.b_resident = (!MN_MAJOR && (MODE == TC_MODE_FWD || MODE == TC_MODE_RAW) && p.splits <= 1 &&
+                  tc_resident_ok(p.out_rows, p.out_cols, p.bn, p.kblocks, NCTA, CH, t.sm_count)) ? 1 : 0;
+  p.tall_slots = tc_tall_slots(NCTA, CH);
+  if (p.conv_tall && !(p.b_resident && p.tall_slots >= 2)) {   // the caller's tensor map was made for tall boxes
+    snprintf(t.err, sizeof(t.err), "tall convolution boxes without resident weights");
+    return FF_ERR_ARG;
+  }
   p.group_m = MN_MAJOR ? TC_GROUP_M_MNMAJOR : TC_GROUP_M_KMAJOR;
   if (p.splits < 1) p.splits = 1;
   p.kb_per_split = cdiv(p.kblocks, p.splits);
@@ -1350,8 +1415,12 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   p.conv_cpt = L.Cin / ch;
   p.conv_imgs_per_pass = B;
   p.kblocks = 9 * p.conv_cpt;
-  if ((s = tc_make_map_nhwc(t, &ta, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_W, p.conv_TH, p.conv_stride)) != FF_OK) return s;
   p.bn = tc_pick_bn(M, L.N, TC_BM * ncta, t.sm_count / ncta);
+  // stride 1, rows of at most 32 pixels, weights resident: boxes of conv_TH + 2 image rows, one per horizontal tap offset
+  p.conv_tall = (p.conv_stride == 1 && p.conv_W <= 32 && p.conv_H >= p.conv_TH + 2 && tc_tall_slots(ncta, ch) >= 2 &&
+                 tc_resident_ok(M, L.N, p.bn, p.kblocks, ncta, ch, t.sm_count)) ? 1 : 0;
+  if ((s = tc_make_map_nhwc(t, &ta, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_W, p.conv_TH + (p.conv_tall ? 2 : 0), p.conv_stride)) != FF_OK)
+    return s;
   if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, ch, p.bn / ncta)) != FF_OK) return s;
   if (ch == 128) return tc_launch<TC_MODE_FWD, false, 128>(t, ncta, ta, tb, p, st, typ);
   return tc_launch<TC_MODE_FWD, false, 64>(t, ncta, ta, tb, p, st, typ);

@@ -91,7 +91,8 @@ def _residual_case(g):
         for l in range(n):
             kind = int(g.choice([1, 2, 3]))
             co = cin if (kind == 3 or l == last) else int(g.choice([8, 16, 64]))
-            if l == last and kind == 3 and cin != (c if first == 0 else layers[first].Cin):
+            block_in = c if first == 0 else (layers[first].Cin if first < len(layers) else cin)
+            if l == last and kind == 3 and cin != block_in:
                 kind = 2
             o = _rule(g)
             layers.append(synth.LayerCfg(kind, {1: 9 * cin, 2: cin, 3: 9}[kind], co, float(co * H * Wd),

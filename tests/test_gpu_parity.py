@@ -209,13 +209,14 @@ def test_conv_tensor_core_shapes(path, chans, H, Wd, B):
 
 
 @pytest.mark.parametrize("form", TENSOR_FORMS)
-def test_conv_layer_with_resident_weights(form):
-    # 64 -> 128 channels on 16 x 16 images, 80 + 80 samples: 160 (320) tiles on 74 (148) CTA groups, one tile column -
-    # the forward keeps the layer's INT8 weights in shared memory and streams the input boxes only
-    hw = 16
-    layers = [synth.LayerCfg(1, 9 * 64, 128, float(128 * hw * hw) / 2, 0.03 / (hw * hw), float(np.sqrt(128 * hw * hw)), H=hw, Wd=hw,
-                             Cin=64)]
-    w = synth.Workload("conv_res", 80, layers, (hw, hw, 64), "normal", "kaiming_uniform", 2)
+@pytest.mark.parametrize("cin,cout,hw,B", [(64, 128, 16, 80), (128, 128, 16, 80), (64, 64, 32, 24)])
+def test_conv_layer_with_resident_weights(form, cin, cout, hw, B):
+    # more tiles than CTA groups and one tile column: the forward keeps the layer's INT8 weights in shared memory and
+    # streams the input only - as boxes of (tile rows + 2) image rows that serve the three vertical taps each (64- and
+    # 128-byte channel chunks; 32- and 16-pixel rows)
+    layers = [synth.LayerCfg(1, 9 * cin, cout, float(cout * hw * hw) / 2, 0.03 / (hw * hw), float(np.sqrt(cout * hw * hw)), H=hw, Wd=hw,
+                             Cin=cin)]
+    w = synth.Workload("conv_res", B, layers, (hw, hw, cin), "normal", "kaiming_uniform", 2)
     _run_and_compare(w, seed=8, steps=2, lam_per_step=0.0, path=(ffb.FF_GEMM_TENSOR, form))
 
 
