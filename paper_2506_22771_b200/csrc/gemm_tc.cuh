@@ -83,7 +83,8 @@ struct TcParams {
                             // B a stage holds follow it, so a narrow layer wastes neither, and a wide one can pick the
                             // width that fills its last wave of tiles best; MN-major kernels always use TC_BN
   int acc_stages;           // K-major forward: accumulator stages in tensor memory (512 / bn, at most 4)
-  int tall_slots;           // stages of TC_TALL_ROWS rows that fit where the A halves of the ordinary stages were
+  int tall_slots;           // tall stages in the ring: TC_TALL_ROWS rows of A each and, when the weights are streamed, the
+  int tall_stride;          // three B boxes (vertical taps) that go with them; tall_stride = bytes from slot to slot
   int b_resident;           // K-major, one tile column: the whole B operand (all contraction blocks of this CTA's rows of
                             // B) is loaded once and stays in shared memory; the stages then hold A only.  A convolution's
                             // weights are the same for every tile, and the loads from L2 are what bounds these kernels.
@@ -499,8 +500,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
                 ok = false;
                 break;
               }
-              if (rank == 0) mbar_expect_tx(bar_full + 8 * s, tall_rows * CH * NCTA);
-              tma_load_4d<NCTA>(ring + s * TC_TALL_ROWS * CH, &tmA, lead_full + 8 * s, cc * CH, ts - 1, f_h0 - 1, f_img);
+              if (rank == 0) mbar_expect_tx(bar_full + 8 * s, (tall_rows * CH + (b_res ? 0u : 3u * b_box_bytes)) * NCTA);
+              const uint32_t slot = ring + s * (uint32_t)p.tall_stride;
+              tma_load_4d<NCTA>(slot, &tmA, lead_full + 8 * s, cc * CH, ts - 1, f_h0 - 1, f_img);
+              if (!b_res)   // the weights of the three vertical taps (tr, ts) for this channel chunk
+                for (int tr = 0; tr < 3; ++tr)
+                  tma_load_2d<NCTA>(slot + TC_TALL_ROWS * CH + tr * b_box_bytes, &tmB, lead_full + 8 * s,
+                                    ((tr * 3 + ts) * p.conv_cpt + cc) * CH, col0, pol_keep);
             }
           continue;
         }
@@ -611,11 +617,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
                 break;
               }
               tc_fence_after();
-              const uint32_t a_box = ring + s * TC_TALL_ROWS * CH;
+              const uint32_t a_box = ring + s * (uint32_t)p.tall_stride;
 #pragma unroll
               for (int tr = 0; tr < 3; ++tr) {
                 const uint32_t a_src = a_box + tr * view_bytes;
-                const uint32_t b_src = bres_base + (uint32_t)((tr * 3 + ts) * p.conv_cpt + cc) * b_box_bytes;
+                const uint32_t b_src = b_res ? bres_base + (uint32_t)((tr * 3 + ts) * p.conv_cpt + cc) * b_box_bytes
+                                             : a_box + TC_TALL_ROWS * CH + tr * b_box_bytes;
 #pragma unroll
                 for (int k = 0; k < G::MMAS; ++k) {
                   tc_mma_i8<NCTA>(d_tmem, make_smem_desc(a_src + k * 32, 16, 8 * CH, G::SWZ),
@@ -1199,9 +1206,11 @@ inline ff_status tc_launch_n(TcState& t, const CUtensorMap& a, const CUtensorMap
   p.tiles_n = cdiv(p.out_cols, p.bn);
   p.b_resident = (!MN_MAJOR && (MODE == TC_MODE_FWD || MODE == TC_MODE_RAW) && p.splits <= 1 &&
                   tc_resident_ok(p.out_rows, p.out_cols, p.bn, p.kblocks, NCTA, CH, t.sm_count)) ? 1 : 0;
-  p.tall_slots = tc_tall_slots(NCTA, CH);
-  if (p.conv_tall && !(p.b_resident && p.tall_slots >= 2)) {   // the caller's tensor map was made for tall boxes
-    snprintf(t.err, sizeof(t.err), "tall convolution boxes without resident weights");
+  p.tall_stride = (int)TC_TALL_ROWS * CH + (p.b_resident ? 0 : 3 * (p.bn / NCTA) * CH);
+  p.tall_slots = p.b_resident ? tc_tall_slots(NCTA, CH) : (int)(G::STAGES * G::STAGE_BYTES / (uint32_t)p.tall_stride);
+  if (p.tall_slots > TC_MAX_STAGES) p.tall_slots = TC_MAX_STAGES;
+  if (p.conv_tall && p.tall_slots < 2) {   // the caller's tensor map was made for tall boxes
+    snprintf(t.err, sizeof(t.err), "tall convolution boxes do not fit the operand ring");
     return FF_ERR_ARG;
   }
   p.group_m = MN_MAJOR ? TC_GROUP_M_MNMAJOR : TC_GROUP_M_KMAJOR;
@@ -1417,8 +1426,13 @@ inline ff_status tc_forward(TcState& t, const ff_layer_desc& L, const ff_layer_b
   p.kblocks = 9 * p.conv_cpt;
   p.bn = tc_pick_bn(M, L.N, TC_BM * ncta, t.sm_count / ncta);
   // stride 1, rows of at most 32 pixels, weights resident: boxes of conv_TH + 2 image rows, one per horizontal tap offset
-  p.conv_tall = (p.conv_stride == 1 && p.conv_W <= 32 && p.conv_H >= p.conv_TH + 2 && tc_tall_slots(ncta, ch) >= 2 &&
-                 tc_resident_ok(M, L.N, p.bn, p.kblocks, ncta, ch, t.sm_count)) ? 1 : 0;
+  {
+    const bool res = tc_resident_ok(M, L.N, p.bn, p.kblocks, ncta, ch, t.sm_count);
+    const int stride_bytes = (int)TC_TALL_ROWS * ch + (res ? 0 : 3 * (p.bn / ncta) * ch);
+    const int slots = res ? tc_tall_slots(ncta, ch)
+                          : tc_kmajor_stages(ncta, ch) * (128 * ch + (TC_BN / ncta) * ch) / stride_bytes;
+    p.conv_tall = (p.conv_stride == 1 && p.conv_W <= 32 && p.conv_H >= p.conv_TH + 2 && slots >= 2) ? 1 : 0;
+  }
   if ((s = tc_make_map_nhwc(t, &ta, b.Xq, L.Cin, L.Wd, L.H, 2 * B, ch, p.conv_W, p.conv_TH + (p.conv_tall ? 2 : 0), p.conv_stride)) != FF_OK)
     return s;
   if ((s = tc_make_map(t, &tb, b.Wq, L.K, L.N, 0, ch, p.bn / ncta)) != FF_OK) return s;

@@ -209,11 +209,13 @@ def test_conv_tensor_core_shapes(path, chans, H, Wd, B):
 
 
 @pytest.mark.parametrize("form", TENSOR_FORMS)
-@pytest.mark.parametrize("cin,cout,hw,B", [(64, 128, 16, 80), (128, 128, 16, 80), (64, 64, 32, 24)])
+@pytest.mark.parametrize("cin,cout,hw,B", [(64, 128, 16, 80), (128, 128, 16, 80), (64, 64, 32, 24), (128, 256, 16, 80),
+                                           (64, 512, 16, 40), (128, 288, 32, 20)])
 def test_conv_layer_with_resident_weights(form, cin, cout, hw, B):
-    # more tiles than CTA groups and one tile column: the forward keeps the layer's INT8 weights in shared memory and
-    # streams the input only - as boxes of (tile rows + 2) image rows that serve the three vertical taps each (64- and
-    # 128-byte channel chunks; 32- and 16-pixel rows)
+    # more tiles than CTA groups: the forward streams the input as boxes of (tile rows + 2) image rows that serve the
+    # three vertical taps each (64- and 128-byte channel chunks; 32- and 16-pixel rows).  The narrow layers keep their
+    # INT8 weights in shared memory; the wide ones (last three: one and two tile columns, ragged last column) load the
+    # three weight boxes of a stage beside its input box
     layers = [synth.LayerCfg(1, 9 * cin, cout, float(cout * hw * hw) / 2, 0.03 / (hw * hw), float(np.sqrt(cout * hw * hw)), H=hw, Wd=hw,
                              Cin=cin)]
     w = synth.Workload("conv_res", B, layers, (hw, hw, cin), "normal", "kaiming_uniform", 2)
