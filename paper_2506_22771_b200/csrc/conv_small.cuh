@@ -161,4 +161,184 @@ __global__ void __launch_bounds__(CS_THREADS) conv3x3_small_fwd_kernel(const int
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Weight gradient of the same layers: sums[set][n][k] = sum over the set's output positions of
+// dHq[pos][n] * x_im2col[pos][k]  (k = (r*3+s)*C_in + ci; INT8 x INT8 -> INT32, Sec. IV-B / Alg. 1 line 9).
+// The contraction runs over positions, so both operands are repacked in shared memory with four CONSECUTIVE
+// POSITIONS per word (a 4 x 4 byte transpose of dHq rows, a gather of input bytes) - which is the operand layout
+// of the warp-level INT8 matrix instruction (m16n8k32: 16 channels x 8 contraction indices x 32 positions per
+// instruction; at 9*C_in <= 36 contraction indices and a few dozen channels the tcgen05 tile sizes do not apply,
+// and dp4a issues at a fraction of this rate).  The loads of the next chunk of 256 positions are in flight while
+// the current chunk's products run.
+// A block works inside one (slab, set) plane: the planes cut each set's positions into parts of at most
+// WG_SAFE_LEN positions, so neither a register sum nor a plane's sum can leave INT32; the block's sums go to the
+// plane with integer atomics (exact, order-free; the planes are zero before) and the slab update kernel adds the
+// planes in 64 bits.  slabs [n_slabs][2][N][9*C_in].
+// ---------------------------------------------------------------------------------------------
+constexpr int CW_CHUNK = 256;            // positions per chunk (= threads per block)
+constexpr int CW_PW = CW_CHUNK / 4;      // position words per chunk
+
+struct ConvSmallWgradGeom {
+  int H, W, Ho, Wo, stride;
+  int B;                      // images per set
+  int rows_per_pass;          // output positions of one set
+  int chunks;                 // chunks per set
+  int chunks_per_slab;        // <= WG_SAFE_LEN / CW_CHUNK
+  int n_slabs;
+  int blocks_per_plane;       // gridDim.x = 2 * n_slabs * blocks_per_plane
+};
+
+// D (16 x 8, INT32) += A (16 x 32, INT8, row-major) * B (32 x 8, INT8, column-major)
+__device__ __forceinline__ void mma_s8_16x8x32(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                               uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int CIN, int N>
+__global__ void __launch_bounds__(CS_THREADS) conv3x3_small_wgrad_kernel(const int8_t* __restrict__ xq, const int8_t* __restrict__ dhq,
+                                                                         int32_t* __restrict__ slabs, ConvSmallWgradGeom g) {
+  constexpr int K = 9 * CIN, KT = (K + 7) / 8, KT8 = KT * 8;   // contraction indices; tiles of eight; padded count
+  constexpr int NG = N / 4;                                    // groups of four channels (one dHq word per position)
+  // row strides (words) of dT[pw][n] and xT[pw][k]: = 8 or 24 mod 32, so that the eight channels (indices) x four
+  // position words a fragment load touches fall into 32 different banks
+  constexpr int NS = N + 8;
+  constexpr int XS = (KT8 % 32 == 8 || KT8 % 32 == 24) ? KT8 : KT8 + 8;
+  constexpr int MT = N / 16, KGRP = 8 / MT;                    // channel tiles; warps that share a channel tile split the position words
+  constexpr int DT_WORDS = CW_PW * NS, XT_WORDS = CW_PW * XS, RED_WORDS = KGRP * N * KT8;
+  constexpr int SM_WORDS = (DT_WORDS + XT_WORDS) > RED_WORDS ? (DT_WORDS + XT_WORDS) : RED_WORDS;
+  constexpr int DTASKS = (CW_PW * NG + CS_THREADS - 1) / CS_THREADS;   // 4 x 4 transposes per thread and chunk
+  constexpr int XTASKS = CW_PW * KT8 / CS_THREADS;                     // gathered words per thread and chunk
+  __shared__ __align__(16) uint32_t sm[SM_WORDS];
+  __shared__ int4 s_pos[CW_CHUNK];   // per position of the chunk: first input row of its image, input row / column of tap (0, 0)
+  uint32_t* dT = sm;
+  uint32_t* xT = sm + DT_WORDS;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int plane = blockIdx.x / g.blocks_per_plane, bip = blockIdx.x - plane * g.blocks_per_plane;
+  const int slab = plane >> 1, set = plane & 1;
+  const int c_begin = slab * g.chunks_per_slab, c_end = min(g.chunks, c_begin + g.chunks_per_slab);
+  const bool row4 = (g.Wo & 3) == 0;   // the four positions of a word share an output row (and a set's positions are a multiple of four)
+  int acc[KT][4];
+#pragma unroll
+  for (int t = 0; t < KT; ++t)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[t][i] = 0;
+  uint32_t dw[DTASKS][4];   // the next chunk's dHq words (rows of four positions) ...
+  uint32_t xb[XTASKS][4];   // ... and input bytes
+  auto decode_chunk = [&](int ch) {
+    const int p = ch * CW_CHUNK + tid;   // position inside the set
+    const int wo = p % g.Wo, t = p / g.Wo, ho = t % g.Ho, img = t / g.Ho;
+    s_pos[tid] = p < g.rows_per_pass ? make_int4((set * g.B + img) * g.H, ho * g.stride - 1, wo * g.stride - 1, 0)
+                                     : make_int4(0, -(1 << 24), 0, 0);   // every tap out of bounds
+  };
+  auto load_chunk = [&](int ch) {   // needs decode_chunk(ch) and a barrier before
+    const int p0 = ch * CW_CHUNK;
+#pragma unroll
+    for (int q = 0; q < DTASKS; ++q) {
+      const int t = tid + q * CS_THREADS, pw = t / NG, cg = t - pw * NG;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int p = p0 + 4 * pw + j;
+        dw[q][j] = (t < CW_PW * NG && p < g.rows_per_pass)
+                       ? __ldg(reinterpret_cast<const uint32_t*>(dhq + ((size_t)set * g.rows_per_pass + p) * N) + cg)
+                       : 0u;
+      }
+    }
+    if (row4) {
+      // the four positions of a word lie in one output row: one row test and one address per word
+      const int dj = g.stride * CIN;
+#pragma unroll
+      for (int q = 0; q < XTASKS; ++q) {
+        const int t = tid + q * CS_THREADS, pw = t / KT8, k = t - pw * KT8;
+        const int tap = k / CIN, ci = k - tap * CIN, r = tap / 3, s = tap - 3 * r;
+        const int4 ps = s_pos[4 * pw];
+        const int hh = ps.y + r, w0 = ps.z + s;
+        const bool row_in = k < K && hh >= 0 && hh < g.H;
+        const int8_t* src = xq + ((long long)(ps.x + hh) * g.W + w0) * CIN + ci;   // dereferenced only where in bounds
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int ww = w0 + j * g.stride;
+          xb[q][j] = (row_in && ww >= 0 && ww < g.W) ? (uint32_t)(uint8_t)__ldg(src + j * dj) : 0u;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int q = 0; q < XTASKS; ++q) {
+        const int t = tid + q * CS_THREADS, pw = t / KT8, k = t - pw * KT8;
+        const int tap = k / CIN, ci = k - tap * CIN, r = tap / 3, s = tap - 3 * r;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int4 ps = s_pos[4 * pw + j];
+          const int hh = ps.y + r, ww = ps.z + s;
+          const bool in = k < K && hh >= 0 && hh < g.H && ww >= 0 && ww < g.W;
+          xb[q][j] = in ? (uint32_t)(uint8_t)__ldg(xq + ((size_t)(ps.x + hh) * g.W + ww) * CIN + ci) : 0u;
+        }
+      }
+    }
+  };
+  const int gq = lane >> 2, tig = lane & 3;          // fragment coordinates of this lane
+  const int m0 = (warp % MT) * 16, grp = warp / MT;  // channel tile and position-word group of this warp
+  int ch = c_begin + bip;
+  if (ch < c_end) {
+    decode_chunk(ch);
+    __syncthreads();
+    load_chunk(ch);
+  }
+  for (; ch < c_end; ch += g.blocks_per_plane) {
+    __syncthreads();   // the previous chunk's words and positions have been used
+    // ---- dT: 4 x 4 byte transposes of the dHq words;  xT: the gathered bytes as words ----
+#pragma unroll
+    for (int q = 0; q < DTASKS; ++q) {
+      const int t = tid + q * CS_THREADS, pw = t / NG, cg = t - pw * NG;
+      if (t < CW_PW * NG) {
+        const uint32_t t0 = __byte_perm(dw[q][0], dw[q][1], 0x5140), t1 = __byte_perm(dw[q][2], dw[q][3], 0x5140);
+        const uint32_t t2 = __byte_perm(dw[q][0], dw[q][1], 0x7362), t3 = __byte_perm(dw[q][2], dw[q][3], 0x7362);
+        uint4 o;
+        o.x = __byte_perm(t0, t1, 0x5410);
+        o.y = __byte_perm(t0, t1, 0x7632);
+        o.z = __byte_perm(t2, t3, 0x5410);
+        o.w = __byte_perm(t2, t3, 0x7632);
+        *reinterpret_cast<uint4*>(dT + pw * NS + 4 * cg) = o;
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < XTASKS; ++q) {
+      const int t = tid + q * CS_THREADS, pw = t / KT8, k = t - pw * KT8;
+      xT[pw * XS + k] = xb[q][0] | (xb[q][1] << 8) | (xb[q][2] << 16) | (xb[q][3] << 24);
+    }
+    const int next = ch + g.blocks_per_plane;
+    if (next < c_end) decode_chunk(next);
+    __syncthreads();
+    if (next < c_end) load_chunk(next);   // in flight during the products
+    // ---- products: A = dT (channels x positions), B = xT (positions x contraction indices) ----
+#pragma unroll 2
+    for (int ks = grp; ks < CW_PW / 8; ks += KGRP) {
+      const uint32_t* da = dT + (ks * 8 + tig) * NS + m0 + gq;
+      const uint32_t a0 = da[0], a1 = da[8], a2 = da[4 * NS], a3 = da[4 * NS + 8];
+      const uint32_t* xa = xT + (ks * 8 + tig) * XS + gq;
+#pragma unroll
+      for (int t = 0; t < KT; ++t) mma_s8_16x8x32(acc[t], a0, a1, a2, a3, xa[t * 8], xa[4 * XS + t * 8]);
+    }
+  }
+  // ---- the block's sums: add the position-word groups in shared memory, one atomic per (channel, index) ----
+  __syncthreads();
+#pragma unroll
+  for (int t = 0; t < KT; ++t) {
+    uint32_t* r0 = sm + ((grp * N + m0 + gq) * KT8 + t * 8 + 2 * tig);
+    r0[0] = (uint32_t)acc[t][0], r0[1] = (uint32_t)acc[t][1];
+    r0[8 * KT8] = (uint32_t)acc[t][2], r0[8 * KT8 + 1] = (uint32_t)acc[t][3];
+  }
+  __syncthreads();
+  int32_t* out = slabs + (size_t)plane * N * K;
+  for (int e = tid; e < N * K; e += CS_THREADS) {
+    const int n = e / K, k = e - n * K;
+    int sum = 0;
+#pragma unroll
+    for (int q = 0; q < KGRP; ++q) sum += (int)sm[(q * N + n) * KT8 + k];
+    if (sum) atomicAdd(out + e, sum);
+  }
+}
+
 }  // namespace ffi8

@@ -522,6 +522,58 @@ ff_status conv_small_forward(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer
   return FF_OK;
 }
 
+// Weight gradient of the same layers: direct dp4a kernel into (slab, set) planes of INT32 sums, then the common
+// reduce + update kernel (which also checks the INT32 range of the whole sums).
+ff_status conv_small_wgrad(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  ConvSmallWgradGeom g;
+  g.H = L.H, g.W = L.Wd, g.Ho = tc_out_h(L), g.Wo = tc_out_w(L), g.stride = tc_conv_stride(L), g.B = B;
+  g.rows_per_pass = B * g.Ho * g.Wo;
+  g.chunks = (g.rows_per_pass + CW_CHUNK - 1) / CW_CHUNK;
+  const int safe_chunks = (int)(WG_SAFE_LEN / CW_CHUNK);
+  g.n_slabs = (g.chunks + safe_chunks - 1) / safe_chunks;
+  if (dp_checks_needed(ctx, L) && g.n_slabs < 2) g.n_slabs = 2;   // a shard's sums pass through the range check
+  g.chunks_per_slab = (g.chunks + g.n_slabs - 1) / g.n_slabs;
+  const int planes = 2 * g.n_slabs;
+  g.blocks_per_plane = ctx->sm_count * 2 / planes;
+  if (g.blocks_per_plane > g.chunks_per_slab) g.blocks_per_plane = g.chunks_per_slab;
+  if (g.blocks_per_plane < 1) g.blocks_per_plane = 1;
+  const size_t bytes = (size_t)planes * L.N * L.K * sizeof(int32_t);
+  if (ctx->workspace_bytes < WS_BYTES + bytes) return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the weight-gradient slabs");
+  int32_t* slabs = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
+  ProfScope prof(ctx, FF_K_UPD_GEMM, st);
+  const bool was = ctx->profiling;
+  ctx->profiling = false;  // one event pair around the route
+  if (cudaMemsetAsync(slabs, 0, bytes, st) != cudaSuccess) {
+    ctx->profiling = was;
+    return fail(ctx, FF_ERR_CUDA, "cudaMemsetAsync failed");
+  }
+  const int grid = planes * g.blocks_per_plane;
+#define FF_CW_LAUNCH(CIN, NN) conv3x3_small_wgrad_kernel<CIN, NN><<<grid, CS_THREADS, 0, st>>>(b.Xq, b.dHq, slabs, g)
+#define FF_CW_BY_N(CIN)                  \
+  switch (L.N) {                         \
+    case 16: FF_CW_LAUNCH(CIN, 16); break; \
+    case 32: FF_CW_LAUNCH(CIN, 32); break; \
+    case 64: FF_CW_LAUNCH(CIN, 64); break; \
+    default: FF_CW_LAUNCH(CIN, 128); break; \
+  }
+  switch (L.Cin) {
+    case 1: FF_CW_BY_N(1); break;
+    case 2: FF_CW_BY_N(2); break;
+    case 3: FF_CW_BY_N(3); break;
+    default: FF_CW_BY_N(4); break;
+  }
+#undef FF_CW_BY_N
+#undef FF_CW_LAUNCH
+  ff_status s = FF_OK;
+  if (cudaPeekAtLastError() != cudaSuccess) s = fail(ctx, FF_ERR_CUDA, "weight-gradient launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  if (s == FF_OK) {
+    ctx->launches++;
+    s = launch_slab_update(ctx, slabs, g.n_slabs, L, b, st, 0);
+  }
+  ctx->profiling = was;
+  return s;
+}
+
 ff_status run_forward_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
   if (L.kind == FF_DWCONV3X3) return dw_forward(ctx, L, b, B, st);
   if (ctx->gemm_path == FF_GEMM_AUTO && conv_small_ok(L.kind == FF_CONV3X3, L.Cin, L.N)) return conv_small_forward(ctx, L, b, B, st);
@@ -598,6 +650,7 @@ ff_status run_update_gemm(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bu
   if (L.kind == FF_DWCONV3X3) return dw_update(ctx, L, b, B, st);
   const int R = rows_per_sample(L);
   const int rows = 2 * B * R;
+  if (ctx->gemm_path == FF_GEMM_AUTO && conv_small_ok(L.kind == FF_CONV3X3, L.Cin, L.N)) return conv_small_wgrad(ctx, L, b, B, st);
   bool tc_ok = tc_update_supported(L, B);
   if (!tc_ok && L.N % 16 == 0 && im2col_route(ctx, L, B)) {
     // explicit im2col (rebuilt from Xq: the workspace is transient), dense split contraction into slabs, reduce + update

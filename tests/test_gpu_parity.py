@@ -403,6 +403,39 @@ def test_pointwise_convolution_layers(path, stack, H, Wd, B):
     _run_and_compare(_mixed_conv_workload(stack, H, Wd, B), seed=51, steps=2, lam_per_step=0.2, path=path)
 
 
+SMALL_CIN = [(ci, n) for ci in (1, 2, 3, 4) for n in (16, 32, 64, 128)]
+
+
+@pytest.mark.parametrize("cin,n", SMALL_CIN)
+def test_first_layer_kernels_every_width(cin, n):
+    # 3x3 layers with at most four input channels take the direct dp4a kernels (forward and weight gradient) on the
+    # default path: every (C_in, width) instantiation, 10 x 12 images (output rows that are not a multiple of four
+    # positions only with stride 2 below), three images per set so that the last chunk of 256 positions is ragged,
+    # then a second such layer is impossible (C_in > 4) so a pointwise layer closes the stack
+    w = _mixed_conv_workload([(1, cin, n), (2, n, 16)], 10, 12, 3)
+    _run_and_compare(w, seed=900 + 10 * cin + n, steps=2, lam_per_step=0.3, path=ffb.FF_GEMM_AUTO, rounding=(1, 1, 1))
+
+
+@pytest.mark.parametrize("cin,n,H,Wd,stride,B", [(3, 64, 32, 32, 1, 5),     # whole chunks, several per block
+                                                 (3, 32, 11, 13, 2, 4),    # 6 x 7 outputs: positions of a word in two rows
+                                                 (1, 16, 28, 28, 2, 7),    # 14 x 14 outputs
+                                                 (4, 128, 9, 10, 1, 2),    # one group of threads per block
+                                                 (2, 64, 2, 10, 1, 1)])    # a single ragged chunk
+def test_first_layer_kernels_geometries(cin, n, H, Wd, stride, B):
+    w = _mixed_conv_workload([(1, cin, n, stride)], H, Wd, B)
+    _run_and_compare(w, seed=950 + H, steps=3, lam_per_step=0.0, path=ffb.FF_GEMM_AUTO, graph=(stride == 2))
+
+
+@pytest.mark.parametrize("optimizer,momentum", [(0, 0.9), (1, 0.9)])
+def test_first_layer_weight_gradient_with_optimisers(optimizer, momentum):
+    w = _mixed_conv_workload([(1, 3, 32), (1, 32, 32)], 16, 16, 3)
+    for l in w.layers:
+        l.momentum, l.optimizer = momentum, optimizer
+        if optimizer:
+            l.beta2, l.adam_eps, l.lr = 0.99, 1e-6, 1e-3
+    _run_and_compare(w, seed=970 + optimizer, steps=3, lam_per_step=0.2, path=ffb.FF_GEMM_AUTO)
+
+
 def _fuzz_cases(n, seed):
     g = np.random.default_rng(seed)
     out = []
