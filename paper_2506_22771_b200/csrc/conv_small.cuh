@@ -198,7 +198,7 @@ __device__ __forceinline__ void mma_s8_16x8x32(int (&c)[4], uint32_t a0, uint32_
 }
 
 template <int CIN, int N>
-__global__ void __launch_bounds__(CS_THREADS) conv3x3_small_wgrad_kernel(const int8_t* __restrict__ xq, const int8_t* __restrict__ dhq,
+__global__ void __launch_bounds__(CS_THREADS, (CIN <= 3 ? 2 : 1)) conv3x3_small_wgrad_kernel(const int8_t* __restrict__ xq, const int8_t* __restrict__ dhq,
                                                                          int32_t* __restrict__ slabs, ConvSmallWgradGeom g) {
   constexpr int K = 9 * CIN, KT = (K + 7) / 8, KT8 = KT * 8;   // contraction indices; tiles of eight; padded count
   constexpr int NG = N / 4;                                    // groups of four channels (one dHq word per position)
@@ -220,6 +220,7 @@ __global__ void __launch_bounds__(CS_THREADS) conv3x3_small_wgrad_kernel(const i
   const int slab = plane >> 1, set = plane & 1;
   const int c_begin = slab * g.chunks_per_slab, c_end = min(g.chunks, c_begin + g.chunks_per_slab);
   const bool row4 = (g.Wo & 3) == 0;   // the four positions of a word share an output row (and a set's positions are a multiple of four)
+  const bool run4 = row4 && g.stride == 1;
   int acc[KT][4];
 #pragma unroll
   for (int t = 0; t < KT; ++t)
@@ -246,7 +247,22 @@ __global__ void __launch_bounds__(CS_THREADS) conv3x3_small_wgrad_kernel(const i
                        : 0u;
       }
     }
-    if (row4) {
+    if (run4) {
+      // stride 1 and the four positions of a word in one output row: for filter row r the word's bytes all come
+      // from the 6 * C_in consecutive bytes of input pixels wo - 1 .. wo + 4 - one thread per (position word, r)
+      if (tid < 3 * CW_PW) {
+        const int r = tid / CW_PW, pw = tid - r * CW_PW;
+        const int4 ps = s_pos[4 * pw];
+        const int hh = ps.y + r;
+        const bool row_in = hh >= 0 && hh < g.H;
+        const int8_t* src = xq + ((long long)(ps.x + hh) * g.W + ps.z) * CIN;   // dereferenced only where in bounds
+#pragma unroll
+        for (int i = 0; i < 6 * CIN; ++i) {
+          const int ww = ps.z + i / CIN;
+          xb[i >> 2][i & 3] = (row_in && ww >= 0 && ww < g.W) ? (uint32_t)(uint8_t)__ldg(src + i) : 0u;
+        }
+      }
+    } else if (row4) {
       // the four positions of a word lie in one output row: one row test and one address per word
       const int dj = g.stride * CIN;
 #pragma unroll
@@ -280,6 +296,7 @@ __global__ void __launch_bounds__(CS_THREADS) conv3x3_small_wgrad_kernel(const i
   };
   const int gq = lane >> 2, tig = lane & 3;          // fragment coordinates of this lane
   const int m0 = (warp % MT) * 16, grp = warp / MT;  // channel tile and position-word group of this warp
+  for (int i = tid; i < XT_WORDS; i += CS_THREADS) xT[i] = 0u;   // contraction indices beyond 9 * C_in stay zero
   int ch = c_begin + bip;
   if (ch < c_end) {
     decode_chunk(ch);
@@ -303,10 +320,22 @@ __global__ void __launch_bounds__(CS_THREADS) conv3x3_small_wgrad_kernel(const i
         *reinterpret_cast<uint4*>(dT + pw * NS + 4 * cg) = o;
       }
     }
+    if (run4) {
+      if (tid < 3 * CW_PW) {
+        const int r = tid / CW_PW, pw = tid - r * CW_PW;
 #pragma unroll
-    for (int q = 0; q < XTASKS; ++q) {
-      const int t = tid + q * CS_THREADS, pw = t / KT8, k = t - pw * KT8;
-      xT[pw * XS + k] = xb[q][0] | (xb[q][1] << 8) | (xb[q][2] << 16) | (xb[q][3] << 24);
+        for (int sc = 0; sc < 3 * CIN; ++sc) {   // sc = s * C_in + ci: byte j of the word is pixel j + s, channel ci
+          const int i0 = sc, i1 = sc + CIN, i2 = sc + 2 * CIN, i3 = sc + 3 * CIN;
+          xT[pw * XS + r * 3 * CIN + sc] =
+              xb[i0 >> 2][i0 & 3] | (xb[i1 >> 2][i1 & 3] << 8) | (xb[i2 >> 2][i2 & 3] << 16) | (xb[i3 >> 2][i3 & 3] << 24);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int q = 0; q < XTASKS; ++q) {
+        const int t = tid + q * CS_THREADS, pw = t / KT8, k = t - pw * KT8;
+        xT[pw * XS + k] = xb[q][0] | (xb[q][1] << 8) | (xb[q][2] << 16) | (xb[q][3] << 24);
+      }
     }
     const int next = ch + g.blocks_per_plane;
     if (next < c_end) decode_chunk(next);
