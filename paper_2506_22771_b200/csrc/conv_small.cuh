@@ -1,11 +1,11 @@
 // 3x3 convolution layers with very few input channels (the first layer of an image network: C_in <= 4, so the
 // contraction 9*C_in has at most 36 terms) - Sec. IV-B's INT8 MAC for a convolution layer whose contraction is far
-// too short for the tensor cores: the layer is bounded by writing its FP32 output, and a tile-based tensor-core
-// kernel spends its time on per-tile latencies instead.  Here a block builds the packed INT8 im2col words of 256
-// consecutive output positions in shared memory (zero padding by bounds checks; never written to global memory),
-// every thread keeps the INT8 weights of its four output channels in registers, and the products are dp4a
-// (four INT8 MACs into INT32).  Lanes are laid out so that each store instruction of a warp writes whole rows of
-// Y (4*N bytes contiguous per position).  Same integers, same FP32 operations as every other forward route.
+// too short for the tcgen05 tiles: the layer is bounded by writing its FP32 output, and a tile-based kernel spends
+// its time on per-tile latencies instead.  Here a block builds the packed INT8 im2col words of 256 consecutive
+// output positions in shared memory (zero padding by bounds checks; never written to global memory), the layer's
+// weights sit beside them in the same packing, and the products are the warp-level INT8 matrix instruction
+// (16 positions x 8 channels x 32 contraction bytes; dp4a, used before, issues at a fraction of its rate and left
+// the kernel bound by the integer pipe).  Same integers, same FP32 operations as every other forward route.
 #pragma once
 #include "common.cuh"
 
@@ -26,32 +26,40 @@ inline bool conv_small_ok(int kind_is_conv3x3, int Cin, int N) {
   return kind_is_conv3x3 && Cin >= 1 && Cin <= 4 && (N == 16 || N == 32 || N == 64 || N == 128);
 }
 
-template <int CIN, int LP>   // LP = N / 4: lanes that share a position (4 channels each)
+// D (16 x 8, INT32) += A (16 x 32, INT8, row-major) * B (32 x 8, INT8, column-major): the warp-level INT8 matrix
+// instruction.  Lane l holds, with g = l / 4 and t = l % 4: A rows g and g + 8, bytes 4t .. 4t+3 and 16+4t .. of the
+// 32 (a0: row g low half, a1: row g+8 low, a2: row g high, a3: row g+8 high); B column g, the same bytes of its
+// 32 (b0 low, b1 high); D rows g (c0, c1) and g + 8 (c2, c3), columns 2t and 2t + 1.
+__device__ __forceinline__ void mma_s8_16x8x32(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                               uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int CIN, int N>
 __global__ void __launch_bounds__(CS_THREADS) conv3x3_small_fwd_kernel(const int8_t* __restrict__ xq, const int8_t* __restrict__ wq,
                                                                        float* __restrict__ Y, int32_t* __restrict__ acc_dump,
                                                                        unsigned long long* __restrict__ S,
                                                                        int32_t* __restrict__ rowmax,
                                                                        const float* __restrict__ absmax, ConvSmallGeom g) {
-  constexpr int K = 9 * CIN, KW = (K + 3) / 4;   // contraction bytes, packed words
-  __shared__ uint32_t xi[CS_THREADS * KW];
+  constexpr int K = 9 * CIN, KS = (K + 31) / 32, KW = KS * 8;   // contraction bytes; steps of 32; packed words per row (zero beyond K)
+  constexpr int RS = KW + 4;   // row stride in words: = 4 mod 8, so the 8 rows x 4 words of a fragment load fall into 32 banks
+  constexpr int NT = N / 8;    // channel tiles of the matrix instruction
+  static_assert(127 * 127 * K < (1 << 23), "the INT32 sums must be exact in a float's mantissa");
+  __shared__ __align__(16) uint32_t xi[CS_THREADS * RS];   // im2col words of the tile's positions
+  __shared__ __align__(16) uint32_t ws[N * RS];            // the layer's weights in the same packing
   __shared__ unsigned long long red_s[CS_THREADS / 32];
   __shared__ int red_m[CS_THREADS / 32];
   const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5;
-  constexpr int ppi = 32 / LP;                    // positions a warp takes per iteration
-  const int cg = lane % LP, ps = lane / LP;       // channel group, position slot
-  // the four channels' weights, packed like the im2col words (k = (r*3+s)*CIN + ci; bytes beyond K are zero)
-  uint32_t wr[4][KW];
+  const int gq = lane >> 2, tig = lane & 3;
+  for (int i = threadIdx.x; i < N * KW; i += CS_THREADS) {
+    const int n = i / KW, j = i - n * KW;
+    uint32_t v = 0u;
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    const int8_t* wrow = wq + (size_t)(4 * cg + c) * K;
-#pragma unroll
-    for (int j = 0; j < KW; ++j) {
-      uint32_t v = 0u;
-#pragma unroll
-      for (int b = 0; b < 4; ++b)
-        if (4 * j + b < K) v |= (uint32_t)(uint8_t)wrow[4 * j + b] << (8 * b);
-      wr[c][j] = v;
-    }
+    for (int b = 0; b < 4; ++b)
+      if (4 * j + b < K) v |= (uint32_t)(uint8_t)wq[(size_t)n * K + 4 * j + b] << (8 * b);
+    ws[n * RS + j] = v;
   }
   const float s_w = scale_of(absmax[2]);
   const float c0 = __fmul_rn(scale_of(absmax[0]), s_w), c1 = __fmul_rn(scale_of(absmax[1]), s_w);
@@ -84,54 +92,83 @@ __global__ void __launch_bounds__(CS_THREADS) conv3x3_small_fwd_kernel(const int
         }
       }
 #pragma unroll
-      for (int j = 0; j < KW; ++j) xi[threadIdx.x * KW + j] = wd[j];
+      for (int j = 0; j < KW; j += 4)
+        *reinterpret_cast<uint4*>(xi + threadIdx.x * RS + j) = make_uint4(wd[j], wd[j + 1], wd[j + 2], wd[j + 3]);
     }
-    __syncthreads();
-    // ---- MACs and epilogue: warp wv takes positions 32*wv .. 32*wv+31 of the tile, ppi per iteration ----
+    __syncthreads();   // (also orders the weights' words before their first use)
+    // ---- products and epilogue: warp wv takes positions 32*wv .. 32*wv+31 of the tile, 16 per pass ----
     unsigned long long ssum = 0ull;
     int mx = 0;
-#pragma unroll 4
-    for (int it = 0; it < LP; ++it) {
-      const int pl = 32 * wv + it * ppi + ps;
-      const int p = tile * CS_THREADS + pl;
-      int acc[4] = {0, 0, 0, 0};
+#pragma unroll 1
+    for (int half = 0; half < 2; ++half) {
+      const int pl = 32 * wv + 16 * half + gq;    // this lane's rows of the pass: pl and pl + 8
+      const uint32_t* xa = xi + pl * RS + tig;
+      uint32_t a[KS][4];
 #pragma unroll
-      for (int j = 0; j < KW; ++j) {
-        const int xw = (int)xi[pl * KW + j];
+      for (int ks = 0; ks < KS; ++ks) a[ks][0] = xa[8 * ks], a[ks][1] = xa[8 * RS + 8 * ks], a[ks][2] = xa[8 * ks + 4], a[ks][3] = xa[8 * RS + 8 * ks + 4];
+      const int pa = tile * CS_THREADS + pl, pb = pa + 8;
+      const bool oka = pa < g.rows, okb = pb < g.rows;
+      const float csa = pa < g.rows_per_pass ? c0 : c1, csb = pb < g.rows_per_pass ? c0 : c1;
+      float* ya = Y + (size_t)pa * N + 2 * tig;
+      float* yb = Y + (size_t)pb * N + 2 * tig;
+      unsigned long long sa = 0ull, sb = 0ull;
+      int ma = 0, mb = 0;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) acc[c] = __dp4a(xw, (int)wr[c][j], acc[c]);
-      }
-      unsigned long long ps_sum = 0ull;
-      int ps_max = 0;
-      if (p < g.rows) {
-        const float cs = p < g.rows_per_pass ? c0 : c1;
+      for (int nt = 0; nt < NT; ++nt) {
+        int c[4] = {0, 0, 0, 0};
+        const uint32_t* wb = ws + (nt * 8 + gq) * RS + tig;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) mma_s8_16x8x32(c, a[ks][0], a[ks][1], a[ks][2], a[ks][3], wb[8 * ks], wb[8 * ks + 4]);
+        unsigned rl[4];
         float y[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const unsigned rl = (unsigned)max(acc[c], 0);
-          y[c] = __fmul_rn(__uint2float_rn(rl), cs);
-          ps_sum += (unsigned long long)rl * rl;
-          ps_max = max(ps_max, (int)rl);
+        for (int q = 0; q < 4; ++q) {
+          rl[q] = (unsigned)max(c[q], 0);
+          // exact: rl < 2^23, so placing it in the mantissa of 2^23 and subtracting 2^23 is the integer as a float
+          y[q] = __fmul_rn(__fsub_rn(__uint_as_float(rl[q] | 0x4B000000u), 8388608.0f), q < 2 ? csa : csb);
         }
-        float4* dst = reinterpret_cast<float4*>(Y + (size_t)p * g.N + 4 * cg);
-        if (g.y_stream)
-          __stcs(dst, make_float4(y[0], y[1], y[2], y[3]));
-        else
-          *dst = make_float4(y[0], y[1], y[2], y[3]);
-        if (acc_dump) *reinterpret_cast<int4*>(acc_dump + (size_t)p * g.N + 4 * cg) = make_int4(acc[0], acc[1], acc[2], acc[3]);
+        sa += (unsigned long long)rl[0] * rl[0] + (unsigned long long)rl[1] * rl[1];
+        sb += (unsigned long long)rl[2] * rl[2] + (unsigned long long)rl[3] * rl[3];
+        ma = max(ma, (int)max(rl[0], rl[1]));
+        mb = max(mb, (int)max(rl[2], rl[3]));
+        if (oka) {
+          if (g.y_stream)
+            __stcs(reinterpret_cast<float2*>(ya + nt * 8), make_float2(y[0], y[1]));
+          else
+            *reinterpret_cast<float2*>(ya + nt * 8) = make_float2(y[0], y[1]);
+        }
+        if (okb) {
+          if (g.y_stream)
+            __stcs(reinterpret_cast<float2*>(yb + nt * 8), make_float2(y[2], y[3]));
+          else
+            *reinterpret_cast<float2*>(yb + nt * 8) = make_float2(y[2], y[3]);
+        }
+        if (acc_dump) {
+          if (oka) *reinterpret_cast<int2*>(acc_dump + (size_t)pa * N + nt * 8 + 2 * tig) = make_int2(c[0], c[1]);
+          if (okb) *reinterpret_cast<int2*>(acc_dump + (size_t)pb * N + nt * 8 + 2 * tig) = make_int2(c[2], c[3]);
+        }
       }
+      if (!oka) sa = 0ull, ma = 0;
+      if (!okb) sb = 0ull, mb = 0;
       if (tile_in_sample) {
-        ssum += ps_sum;
-        mx = max(mx, ps_max);
+        ssum += sa + sb;
+        mx = max(mx, max(ma, mb));
       } else {
-        // positions of a warp may belong to different samples: add up over the LP lanes of the position
-        for (int o = LP >> 1; o > 0; o >>= 1) {
-          ps_sum += __shfl_xor_sync(0xffffffffu, ps_sum, o);
-          ps_max = max(ps_max, __shfl_xor_sync(0xffffffffu, ps_max, o));
+        // positions of a warp may belong to different samples: add up over the four lanes of a position
+#pragma unroll
+        for (int o = 1; o <= 2; o <<= 1) {
+          sa += __shfl_xor_sync(0xffffffffu, sa, o);
+          sb += __shfl_xor_sync(0xffffffffu, sb, o);
+          ma = max(ma, __shfl_xor_sync(0xffffffffu, ma, o));
+          mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
         }
-        if (cg == 0 && p < g.rows && ps_max > 0) {
-          atomicAdd(S + p / g.rows_per_sample, ps_sum);
-          atomicMax(rowmax + p / g.rows_per_sample, ps_max);
+        if (tig == 0 && oka && ma > 0) {
+          atomicAdd(S + pa / g.rows_per_sample, sa);
+          atomicMax(rowmax + pa / g.rows_per_sample, ma);
+        }
+        if (tig == 0 && okb && mb > 0) {
+          atomicAdd(S + pb / g.rows_per_sample, sb);
+          atomicMax(rowmax + pb / g.rows_per_sample, mb);
         }
       }
     }
@@ -161,7 +198,6 @@ __global__ void __launch_bounds__(CS_THREADS) conv3x3_small_fwd_kernel(const int
   }
 }
 
-
 // ---------------------------------------------------------------------------------------------
 // Weight gradient of the same layers: sums[set][n][k] = sum over the set's output positions of
 // dHq[pos][n] * x_im2col[pos][k]  (k = (r*3+s)*C_in + ci; INT8 x INT8 -> INT32, Sec. IV-B / Alg. 1 line 9).
@@ -188,14 +224,6 @@ struct ConvSmallWgradGeom {
   int n_slabs;
   int blocks_per_plane;       // gridDim.x = 2 * n_slabs * blocks_per_plane
 };
-
-// D (16 x 8, INT32) += A (16 x 32, INT8, row-major) * B (32 x 8, INT8, column-major)
-__device__ __forceinline__ void mma_s8_16x8x32(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                               uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 
 template <int CIN, int N>
 __global__ void __launch_bounds__(CS_THREADS, (CIN <= 3 ? 2 : 1)) conv3x3_small_wgrad_kernel(const int8_t* __restrict__ xq, const int8_t* __restrict__ dhq,

@@ -501,14 +501,14 @@ ff_status conv_small_forward(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer
   const int grid = tiles < cap ? tiles : cap;
   unsigned long long* S = reinterpret_cast<unsigned long long*>(b.S);
   ProfScope prof(ctx, FF_K_FWD_GEMM, st);
-#define FF_CS_LAUNCH(CIN, LP) \
-  conv3x3_small_fwd_kernel<CIN, LP><<<grid, CS_THREADS, 0, st>>>(b.Xq, b.Wq, b.Y, b.acc_dump, S, b.rowmax, b.absmax, g)
-#define FF_CS_BY_N(CIN)                   \
-  switch (L.N) {                          \
-    case 16: FF_CS_LAUNCH(CIN, 4); break;  \
-    case 32: FF_CS_LAUNCH(CIN, 8); break;  \
-    case 64: FF_CS_LAUNCH(CIN, 16); break; \
-    default: FF_CS_LAUNCH(CIN, 32); break; \
+#define FF_CS_LAUNCH(CIN, NN) \
+  conv3x3_small_fwd_kernel<CIN, NN><<<grid, CS_THREADS, 0, st>>>(b.Xq, b.Wq, b.Y, b.acc_dump, S, b.rowmax, b.absmax, g)
+#define FF_CS_BY_N(CIN)                    \
+  switch (L.N) {                           \
+    case 16: FF_CS_LAUNCH(CIN, 16); break;  \
+    case 32: FF_CS_LAUNCH(CIN, 32); break;  \
+    case 64: FF_CS_LAUNCH(CIN, 64); break;  \
+    default: FF_CS_LAUNCH(CIN, 128); break; \
   }
   switch (L.Cin) {
     case 1: FF_CS_BY_N(1); break;
