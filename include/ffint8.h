@@ -5,9 +5,9 @@
  * The library implements the single-layer dataflow of the FF-INT8 paper (Sec. IV-B, Fig. 4):
  * symmetric uniform quantisation (Sec. IV) of the layer input A (stochastic rounding) and of
  * the weights W, an INT8 x INT8 -> INT32 MAC (dense or 3x3 convolution), goodness
- * G = ||y||^2 (Sec. III; Alg. 1 line 6), the negative-log-likelihood losses of Eq. 1 / Eq. 2
+ * G = ||y||^2 (Sec. III; Alg. 1, goodness step), the negative-log-likelihood losses of Eq. 1 / Eq. 2
  * with the look-ahead term of Eq. 3 / Eq. 4, the output gradient g^Y quantised to INT8, the
- * weight gradient g^W as a second INT8 MAC, and the weight update (Alg. 1 line 9).  No input
+ * weight gradient g^W as a second INT8 MAC, and the weight update (Alg. 1, update step).  No input
  * gradient g^A is ever formed (Sec. IV-B).
  *
  * Conventions
@@ -15,7 +15,7 @@
  *    aligned, valid on the device the context was created for.  Pointers to ff_layer_desc /
  *    ff_layer_bufs structs and all by-value scalars are HOST data.
  *  - Batch layout: B positive samples followed by B negative samples ("positive and negative
- *    sets", Alg. 1 line 3).  M = 2B.  R = rows per sample: 1 for a linear layer, Ho*Wo for a
+ *    sets", Alg. 1, sample generation).  M = 2B.  R = rows per sample: 1 for a linear layer, Ho*Wo for a
  *    convolution (one row per output position, NHWC); the input of a convolution has H*Wd rows.
  *  - Calls are asynchronous on the given CUDA stream (a cudaStream_t passed as void*; NULL =
  *    the legacy default stream) and never synchronise.  Host-detectable errors are returned
@@ -80,7 +80,7 @@ typedef struct {
   int32_t index;        /* position of the layer in the network (keys the rounding hash)      */
   int32_t round_x, round_w, round_dh; /* rounding of A, W, g^Y (paper: stochastic for A)      */
   float theta;          /* threshold of Eq. 1 / Eq. 2                                         */
-  float lr;             /* SGD step size of the update (Alg. 1 line 9)                        */
+  float lr;             /* SGD step size of the update (Alg. 1, update step)                        */
   float tau, eps;       /* length normalisation of the output: x = y*tau/(sqrt(G)+eps), eps>0 */
   uint64_t seed;        /* keys the stochastic-rounding hash                                  */
   int32_t stride;       /* conv3x3 / dwconv3x3 only: 0 or 1 = every position, 2 = every second row and column; */
@@ -163,7 +163,7 @@ ff_status ff_set_gemm_path(ff_ctx* ctx, int path);
 ff_status ff_set_tensor_form(ff_ctx* ctx, int ctas_per_tile);
 
 /* Positive / negative / candidate batches by label embedding (Sec. III: the true label makes a
- * positive sample, a wrong one a negative; Alg. 1 line 3).  x [B, n] FP32 raw samples (device),
+ * positive sample, a wrong one a negative; Alg. 1, sample generation).  x [B, n] FP32 raw samples (device),
  * labels [sets, B] INT32 (device; the wrong labels of a negative set are drawn by the caller).
  * out [sets*B, n] FP32 (device): row s*B + b = sample b with labels[s, b] written one-hot over its
  * label places - flat positions 0, label_stride, ..., (n_classes-1)*label_stride hold on_value at the
@@ -242,7 +242,7 @@ ff_status ff_set_graph_mode(ff_ctx* ctx, int on);
 uint64_t ff_graph_replay_count(const ff_ctx* ctx);
 
 /* Forward of one layer (Sec. IV-B: quantise A and W, INT8 MAC with INT32 accumulation; Sec. III /
- * Alg. 1 line 6: goodness).  Reads X, W.  Writes Xq, Wq, absmax[X,W,XNEXT], Y, S, rowmax, G,
+ * Alg. 1, goodness step: goodness).  Reads X, W.  Writes Xq, Wq, absmax[X,W,XNEXT], Y, S, rowmax, G,
  * Xnext (if non-NULL), acc_dump (if non-NULL).  `step` keys the stochastic rounding. */
 ff_status ff_layer_forward(ff_ctx* ctx, const ff_layer_desc* layer, const ff_layer_bufs* bufs,
                            int B, uint64_t step, void* cuda_stream);
@@ -257,7 +257,7 @@ ff_status ff_layer_loss_grad(ff_ctx* ctx, const ff_layer_desc* layer, const ff_l
                              int n_later, float lambda, uint64_t step, void* cuda_stream);
 
 /* Weight gradient and update of one layer (Sec. IV-B: g^W is a second INT8 MAC and is the only
- * gradient formed and applied; Alg. 1 line 9).  Reads dHq, Xq, absmax, W.  Writes W
+ * gradient formed and applied; Alg. 1, update step).  Reads dHq, Xq, absmax, W.  Writes W
  * (W - lr*(float(accP)*cP + float(accN)*cN)) and accW_dump (if non-NULL); with momentum != 0 or
  * optimizer = FF_OPT_ADAM the step follows that rule and Mom (and Var) are rewritten.  `step` is the
  * step counter of the update (Adam's update number is t = step + 1; the other rules do not read it). */
@@ -265,8 +265,8 @@ ff_status ff_layer_update(ff_ctx* ctx, const ff_layer_desc* layer, const ff_laye
                           int B, uint64_t step, void* cuda_stream);
 
 /* Body of Algorithm 1's epoch loop for n_layers layers: one INT8 forward through all layers with
- * the pre-update weights (line 5), goodness of every layer (line 6), then per layer the loss with
- * look-ahead weight `lambda` (line 8, Eq. 3) and the INT8 gradient + update (line 9).  Layer 0
+ * the pre-update weights, goodness of every layer, then per layer the loss with look-ahead
+ * weight `lambda` (Eq. 3) and the INT8 gradient + update.  Layer 0
  * reads bufs[0].X; layer l > 0 reads bufs[l].X if non-NULL, else layer l-1's normalised output.
  * With n_layers = 1 and lambda = 0 it equals forward -> loss_grad -> update. */
 ff_status ff_train_step(ff_ctx* ctx, const ff_layer_desc* layers, const ff_layer_bufs* bufs,
@@ -287,7 +287,7 @@ ff_status ff_train_step_from(ff_ctx* ctx, const ff_layer_desc* layers, const ff_
  * does not describe the procedure; this is the Forward-Forward one its Sec. III builds on (layers are
  * trained to respond strongly to positive samples): every sample is presented once per candidate label,
  * label written one-hot into the input exactly as for the positive set; each candidate runs through
- * the same INT8 forward as training (Sec. IV-B; Alg. 1 line 5-6); the goodness of the layers
+ * the same INT8 forward as training (Sec. IV-B; Alg. 1, forward pass); the goodness of the layers
  * first_counted_layer .. n_layers-1 is added per candidate (FP32, in layer order) and the label with
  * the largest total wins (lowest label on ties).
  * Layout: the caller builds the candidate batch [n_classes*B, ...] in bufs[0].X, row c*B + b = sample

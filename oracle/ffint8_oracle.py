@@ -289,7 +289,7 @@ def int8_dwconv3x3_wgrad(dhq: np.ndarray, xq: np.ndarray, stride: int = 1) -> np
 
 
 # --------------------------------------------------------------------------------------
-# Epilogue: dequantise, ReLU, goodness, length normalisation  (Sec. III; Alg. 1 line 6)
+# Epilogue: dequantise, ReLU, goodness, length normalisation  (Sec. III; Alg. 1, goodness step)
 # --------------------------------------------------------------------------------------
 def dequant_relu(acc: np.ndarray, c_rows: np.ndarray) -> np.ndarray:
     """y = max(0, float(acc) * c) with c = s_x*s_w of the row's pass; int->float conversion and
@@ -300,7 +300,7 @@ def dequant_relu(acc: np.ndarray, c_rows: np.ndarray) -> np.ndarray:
 
 
 def goodness(acc: np.ndarray, c_rows: np.ndarray):
-    """G = ||y||^2 per sample (the sum of the squared activities of the layer, Sec. III; Alg. 1 line 6),
+    """G = ||y||^2 per sample (the sum of the squared activities of the layer, Sec. III; Alg. 1, goodness step),
     evaluated as the exact integer S = sum relu(acc)^2 scaled once: G = float(double(S)*c*c).
     Also returns S and the per-sample max of relu(acc) (used for the absmax short-cuts)."""
     n = acc.shape[0]
@@ -339,7 +339,7 @@ def maxpool2x2(x: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------------------
-# FF loss, sigma and the look-ahead coefficient  (Eq. 1-4; Alg. 1 lines 8-9)
+# FF loss, sigma and the look-ahead coefficient  (Eq. 1-4; Alg. 1, loss and update steps)
 # --------------------------------------------------------------------------------------
 _LOG2E = F64(1.4426950408889634)            # nearest double to 1/ln 2
 _LN2_HI = F64(6.93147180369123816490e-01)   # ln 2 split so that n*LN2_HI is exact
@@ -505,7 +505,7 @@ def layer_loss_grad(spec: LayerSpec, st: LayerState, B: int, G_later: Sequence[n
 
 def sgd_momentum(W: np.ndarray, M: np.ndarray, g: np.ndarray, lr: float, mu: float):
     """Heavy-ball SGD (Polyak): m <- mu*m + g, W <- W - lr*m, each operation one float32 rounding.
-    The paper names no optimiser for its weight update (Sec. IV-B; Alg. 1 line 9); plain
+    The paper names no optimiser for its weight update (Sec. IV-B; Alg. 1, update step); plain
     SGD is mu = 0, this is the usual next choice.  Returns (W_new, M_new)."""
     M_new = F32(mu) * np.asarray(M, dtype=F32) + np.asarray(g, dtype=F32)
     return np.asarray(W, dtype=F32) - F32(lr) * M_new, M_new
@@ -526,7 +526,7 @@ def _pow_int(x: float, n: int) -> float:
 
 def adam_update(W, M, V, g, lr: float, beta1: float, beta2: float, eps: float, t: int):
     """Adam (Kingma & Ba 2015, Algorithm 1) for update number t >= 1, the other usual choice where the paper
-    only says that the weights are updated (Sec. IV-B; Alg. 1 line 9):
+    only says that the weights are updated (Sec. IV-B; Alg. 1, update step):
         m = beta1*m + (1-beta1)*g;  v = beta2*v + (1-beta2)*g*g;
         W -= lr * (m*c1) / (sqrt(v*c2) + eps),   c_i = float32(1/(1 - beta_i^t)).
     float32 throughout, one rounding per operation in the order written (1-beta_i is one float32
@@ -543,8 +543,8 @@ def adam_update(W, M, V, g, lr: float, beta1: float, beta2: float, eps: float, t
 
 def layer_update(spec: LayerSpec, st: LayerState, W: np.ndarray, B: int, M: Optional[np.ndarray] = None,
                  V: Optional[np.ndarray] = None, step: int = 0) -> LayerState:
-    """g^W per pass as an INT8 MAC, dequantised and applied as plain SGD (Sec. IV-B; Alg. 1
-    line 9):  g = float(accP)*cP + float(accN)*cN,  W <- W - lr*g.  With spec.momentum != 0 the
+    """g^W per pass as an INT8 MAC, dequantised and applied as plain SGD (Sec. IV-B; Alg. 1,
+    update step):  g = float(accP)*cP + float(accN)*cN,  W <- W - lr*g.  With spec.momentum != 0 the
     update is heavy-ball SGD on the momentum buffer M (zeros when None), see sgd_momentum."""
     W = np.asarray(W, dtype=F32)
     accW = []
@@ -577,9 +577,9 @@ def train_step(specs: List[LayerSpec], Ws: List[np.ndarray], X: np.ndarray, B: i
                step: int, Ms: Optional[List[np.ndarray]] = None, Vs: Optional[List[np.ndarray]] = None,
                first_trained: int = 0) -> List[LayerState]:
     """Body of Algorithm 1's epoch loop: one INT8 forward through all k layers with the
-    pre-update weights (line 5), goodness of every layer (line 6), then for each layer its
-    loss from the G's (line 8) and its INT8 gradient and update (line 9).  lambda is the
-    caller's (lines 2 and 11).  With one layer and lambda = 0 this is the vanilla step.  Ms: the
+    pre-update weights, goodness of every layer, then for each layer its loss from the G's
+    and its INT8 gradient and update.  lambda is the caller's (the algorithm starts it at zero
+    and raises it once per epoch).  With one layer and lambda = 0 this is the vanilla step.  Ms: the
     layers' momentum buffers (only read by layers with momentum != 0).
     first_trained > 0: the layers before it are frozen - they take part in the forward only (their
     states carry no coef, dHq or W_new).  This is one step of the layer-by-layer schedule of Sec. III,
@@ -654,12 +654,12 @@ def predict(specs: List[LayerSpec], Ws: List[np.ndarray], X_cand: np.ndarray, B:
 
 
 # --------------------------------------------------------------------------------------
-# Positive / negative (and candidate) batches by label embedding  (Sec. III; Alg. 1 line 3)
+# Positive / negative (and candidate) batches by label embedding  (Sec. III; Alg. 1, sample generation)
 # --------------------------------------------------------------------------------------
 def embed_labels(x: np.ndarray, labels: np.ndarray, n_classes: int, label_stride: int = 1, on_value: float = 1.0,
                  tau0: float = 0.0, eps: float = 1e-8) -> np.ndarray:
     """Batches made from B raw samples by writing a label into each (Sec. III: the true label gives the
-    positive sample, a wrong one the negative; Alg. 1 line 3).  x [B, n] float32, labels [sets, B]:
+    positive sample, a wrong one the negative; Alg. 1, sample generation).  x [B, n] float32, labels [sets, B]:
     output row s*B + b is sample b with labels[s, b] written one-hot over its n_classes label places
     (flat positions 0, label_stride, 2*label_stride, ...: the place of the label holds on_value, the
     others zero).  The wrong labels are drawn by the caller and passed in.  With tau0 > 0 every row is

@@ -68,7 +68,7 @@ __device__ __forceinline__ RoundKey derive_key(KeySpec ks) {
   k.k1 = (uint32_t)(s2 >> 32);
   return k;
 }
-// How a dequantised weight gradient g becomes a weight change (Alg. 1 line 9 names no optimiser):
+// How a dequantised weight gradient g becomes a weight change (Alg. 1, update step names no optimiser):
 // kind 0: plain SGD, or heavy ball when Mom is given (m = mu*m + g, W -= lr*m);
 // kind 1: Adam - m = b1*m + (1-b1)*g, v = b2*v + (1-b2)*g*g, W -= lr*(m*c1)/(sqrt(v*c2) + eps), with the
 // bias corrections c_i = float(1/(1 - b_i^t)), t = step + 1, from FP64 powers taken by square-and-multiply

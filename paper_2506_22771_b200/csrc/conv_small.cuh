@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(CS_THREADS) conv3x3_small_fwd_kernel(const int
 
 // ---------------------------------------------------------------------------------------------
 // Weight gradient of the same layers: sums[set][n][k] = sum over the set's output positions of
-// dHq[pos][n] * x_im2col[pos][k]  (k = (r*3+s)*C_in + ci; INT8 x INT8 -> INT32, Sec. IV-B / Alg. 1 line 9).
+// dHq[pos][n] * x_im2col[pos][k]  (k = (r*3+s)*C_in + ci; INT8 x INT8 -> INT32, Sec. IV-B / Alg. 1, update step).
 // The contraction runs over positions, so both operands are repacked in shared memory with four CONSECUTIVE
 // POSITIONS per word (a 4 x 4 byte transpose of dHq rows, a gather of input bytes) - which is the operand layout
 // of the warp-level INT8 matrix instruction (m16n8k32: 16 channels x 8 contraction indices x 32 positions per

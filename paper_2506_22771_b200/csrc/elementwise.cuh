@@ -1,6 +1,6 @@
 // Memory-bound passes of the FF-INT8 step: absmax reduction, SUQ quantisation (Sec. IV) with
 // nearest / stochastic rounding (Sec. IV-B), goodness finalisation and length normalisation
-// (Sec. III; Alg. 1 line 6), the loss / look-ahead coefficient kernel (Eq. 1-4) and the output
+// (Sec. III; Alg. 1, goodness step), the loss / look-ahead coefficient kernel (Eq. 1-4) and the output
 // gradient quantiser (g^Y to INT8, Sec. IV-B).
 // All are coalesced 128-bit-load kernels with warp-shuffle reductions; grids are sized in
 // multiples of the SM count by the host code.
@@ -775,7 +775,7 @@ __device__ __forceinline__ void dh_quantize_body(const float* __restrict__ Y, co
 }
 
 // ---------------------------------------------------------------------------------------------
-// Positive / negative / candidate batches by label embedding (Sec. III; Alg. 1 line 3).
+// Positive / negative / candidate batches by label embedding (Sec. III; Alg. 1, sample generation).
 // x [B, n] raw samples, labels [sets, B]; out row s*B + b = sample b with labels[s, b] written
 // one-hot over the label places (flat positions j*label_stride, j < n_classes: on_value at the label,
 // zero elsewhere), then, if tau0 > 0, scaled to length tau0 with

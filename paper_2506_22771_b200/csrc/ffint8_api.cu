@@ -969,7 +969,7 @@ ff_status check_layer_list(ff_ctx* ctx, const ff_layer_desc* layers, const ff_la
   return FF_OK;
 }
 
-// INT8 forward through all layers with the current weights (Alg. 1 line 5-6): layer 0 reads bufs[0].X,
+// INT8 forward through all layers with the current weights (Alg. 1, forward pass): layer 0 reads bufs[0].X,
 // layer l > 0 reads bufs[l].X if given, else the previous layer's normalised output, quantised on the fly.
 // Everything a step can quantise before any layer has run, in two launches whatever the number of layers:
 // ranges of the network input (both sets) and of every layer's weights, then their INT8 codes (which also
@@ -1047,9 +1047,9 @@ ff_status train_step_body(ff_ctx* ctx, const ff_layer_desc* layers, const ff_lay
                           float lambda, cudaStream_t st, int first = 0) {
   ff_status s;
   (void)lambda;  // read by the kernels from the step state
-  // Alg. 1 line 5-6: one forward through all layers with the pre-update weights
+  // Alg. 1, forward pass: one forward through all layers with the pre-update weights
   if ((s = forward_all(ctx, layers, bufs, n_layers, B, st)) != FF_OK) return s;
-  // Alg. 1 line 7-9: loss from the G's (Eq. 3) and INT8 output gradient - neither depends on an update, so all
+  // Alg. 1, per-layer loss and update: loss from the G's (Eq. 3) and INT8 output gradient - neither depends on an update, so all
   // layers share one launch each - then per layer the weight gradient and update
   LossJobs lj;
   DhJobs dj;

@@ -88,7 +88,7 @@ struct RawEpilogue {  // plain INT32 store
   }
 };
 
-// Forward epilogue (dequantise, ReLU, goodness statistics; Sec. III, Alg. 1 line 6).
+// Forward epilogue (dequantise, ReLU, goodness statistics; Sec. III, Alg. 1, goodness step).
 struct ForwardEpilogue {
   float* Y;
   int32_t* acc_dump;  // nullable
@@ -136,7 +136,7 @@ struct ForwardEpilogue {
   }
 };
 
-// Weight-gradient epilogue (dequantise both sets, SGD update; Sec. IV-B, Alg. 1 line 9).
+// Weight-gradient epilogue (dequantise both sets, SGD update; Sec. IV-B, Alg. 1, update step).
 struct UpdateEpilogue {
   float* W;
   int32_t* accW_dump;  // nullable, [2, rows, cols]
@@ -191,7 +191,7 @@ struct SlabEpilogue {
 };
 
 // Adds the `splits` INT32 slabs of both sets and applies the dequantised update (Sec. IV-B;
-// Alg. 1 line 9): W <- W - lr*(float(accP)*cP + float(accN)*cN).  plane = rows*cols elements of W;
+// Alg. 1, update step): W <- W - lr*(float(accP)*cP + float(accN)*cN).  plane = rows*cols elements of W;
 // the slabs may have a wider row pitch (cols <= pitch).  A block covers 32 consecutive elements; its
 // 8 warps take the splits round-robin (coalesced along the elements) and their integer partial
 // sums meet in shared memory.  W == NULL: no update, only the sums are written to accW_dump (dense

@@ -20,7 +20,7 @@
 // The forward double-buffers the accumulator (2 x 256 TMEM columns) so that the epilogue of tile
 // i overlaps the MMAs of tile i+1; the weight gradient holds the accumulators of the positive and
 // the negative set side by side (2 x 256 columns) and either applies the update
-// W <- W - lr*(float(accP)*cP + float(accN)*cN) (Alg. 1 line 9) in its epilogue (dense layers) or,
+// W <- W - lr*(float(accP)*cP + float(accN)*cN) (Alg. 1, update step) in its epilogue (dense layers) or,
 // when the contraction is split over several CTAs because the output has few tiles
 // (convolutions), stores INT32 partial sums to slabs that slab_update_kernel adds exactly.
 // Every wait is bounded: when one runs out the CTA raises ST_TIMEOUT, drains and returns.

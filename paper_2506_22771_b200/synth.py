@@ -1,7 +1,7 @@
 """Seeded synthetic inputs shaped like the paper's workloads (Sec. V-A: MNIST-style MLP data,
 CIFAR-style CNN data).  Serves the oracle tests, the GPU parity tests and the benchmark alike,
 and holds none of the method's arithmetic: it only draws numbers, writes the one-hot label
-into the input (the positive / negative set generation of Alg. 1 line 3; Sec. III) and scales
+into the input (the positive / negative set generation of Alg. 1, sample generation; Sec. III) and scales
 each sample to the length the first layer expects (the layer-1 input arrives length-normalised).
 
 Nothing here is real MNIST / CIFAR-10 data: only their shapes and value ranges are used.

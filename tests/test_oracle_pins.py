@@ -827,7 +827,7 @@ def test_strided_conv_gradient_matches_finite_differences():
         assert abs(fd - dW[n, k]) <= 1e-4 * max(1.0, abs(fd)), (n, k, fd, dW[n, k])
 
 
-# ---- label embedding (positive / negative / candidate batches; Sec. III, Alg. 1 line 3) ------------
+# ---- label embedding (positive / negative / candidate batches; Sec. III, Alg. 1, sample generation) ------------
 def test_embed_labels_hand_example():
     x = np.array([[9.0, 9.0, 9.0, 3.0, 4.0]], dtype=np.float32)          # 3 label places, then the data
     got = O.embed_labels(x, np.array([[2], [0]]), n_classes=3)
@@ -862,7 +862,7 @@ def test_embed_labels_matches_the_batch_generator_and_has_unit_invariants():
         O.embed_labels(base.astype(np.float32), np.full((1, B), 10), 10)
 
 
-# ---- heavy-ball variant of the update (Alg. 1 line 9 names no optimiser) ----------------------------
+# ---- heavy-ball variant of the update (Alg. 1, update step names no optimiser) ----------------------------
 def test_sgd_momentum_hand_example_and_closed_form():
     # powers of two: every product and sum is exact in float32
     W, M = np.array([1.0, -2.0], np.float32), np.array([0.5, 0.0], np.float32)
