@@ -41,7 +41,7 @@ BURST_SECONDS = 2.0         # timed regions shorter than this are compared with 
 # was profiled (hash below) and the workload matches; otherwise the key is null.
 NCU_TRAFFIC = {
     "source": "paper_2506_22771_b200/csrc/gemm_tc.cuh",
-    "sha256": "039ff03cf38e86c98ef04a1d620d329a1505b9c4ec2f688e67e03f181f4d5a21",
+    "sha256": "b7298b1af386290339c0bbf8f03b122d492d6423c9d81c215d84abb902aab13b",
     "workload": "roofline", "B": 16384,
     "bytes_per_launch": {"fwd_gemm": 2396.1e6, "upd_gemm": 2868.0e6},
 }
