@@ -354,6 +354,21 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
   d |= (uint64_t)swz << 61;
   return d;
 }
+// The same descriptor in halves, for the MMA issuer's inner loops (one thread issues every MMA of the CTA group, so
+// its instruction count per MMA is on the critical path of short contractions): the high word is a constant of the
+// kernel, the low word is a constant plus the start address in 16-byte units, so moving the start by `bytes` adds
+// bytes / 16 to the low word (every address is below 256 KB: the 14-bit field cannot carry).
+__device__ __forceinline__ uint32_t smem_desc_hi(uint32_t sbo_bytes, uint32_t swz) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (swz << 29);
+}
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint64_t smem_desc_join(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
 // Instruction descriptor: INT8 x INT8 -> INT32, dense, M = 128 per CTA of the group, N = 256.
 __host__ __device__ constexpr uint32_t make_idesc_i8(bool a_mn_major, bool b_mn_major, int ncta, int n = TC_BN) {
   return (2u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
@@ -449,6 +464,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     // ------------------------------- TMA producer (every CTA loads its own operand parts) ----
     if (lane == 0) {
       uint32_t it = 0;  // running k-block counter (ring position)
+      uint32_t tall_s = 0, tall_ph = 0;  // the same for the tall convolution stages, as slot and phase
       bool ok = true;
       const int a_rows0 = (int)rank * TC_BM;            // this CTA's rows inside the group's tile
       const int b_cols0 = (int)rank * (BN / NCTA);      // this CTA's share of the tile's columns
@@ -494,8 +510,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
           // tall boxes: stage = (conv_TH + 2) image rows x conv_W pixels x CH channels for tap column s, chunk cc
           const uint32_t tall_rows = (uint32_t)(p.conv_TH + 2) * p.conv_W, slots = (uint32_t)p.tall_slots;
           for (int ts = 0; ts < 3 && ok; ++ts)
-            for (int cc = 0; cc < p.conv_cpt; ++cc, ++it) {
-              const uint32_t s = it % slots, ph = (it / slots) & 1u;
+            for (int cc = 0; cc < p.conv_cpt; ++cc) {
+              const uint32_t s = tall_s, ph = tall_ph;   // ring position, kept by counting
+              if (++tall_s == slots) tall_s = 0u, tall_ph ^= 1u;
               if (!mbar_wait<PAIR>(bar_empty + 8 * s, ph ^ 1u, abort_flag)) {
                 ok = false;
                 break;
@@ -591,7 +608,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
     // ------------------------------- MMA issuer (leader CTA only) ----------------------------
     if (lane == 0 && rank == 0) {
       const uint32_t idesc = make_idesc_i8(MN_MAJOR, MN_MAJOR, NCTA, BN);
-      uint32_t it = 0, tile_it = 0;
+      uint32_t it = 0, tile_it = 0, tall_s = 0, tall_ph = 0;
       bool ok = true;
       const bool b_res = !MN_MAJOR && p.b_resident;
       const uint32_t b_box_bytes = (uint32_t)(BN / NCTA) * CH, bres_base = ring + STAGES * G::A_BYTES;
@@ -607,31 +624,35 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
         tc_fence_after();
         if (!MN_MAJOR && p.conv_tall) {
           const uint32_t d_tmem = tmem_base + as * BN, slots = (uint32_t)p.tall_slots;
-          const uint32_t view_bytes = (uint32_t)p.conv_W * CH;   // one image row of the box: the step between vertical taps
-          uint32_t first = 1u;
-          for (int ts = 0; ts < 3 && ok; ++ts)
-            for (int cc = 0; cc < p.conv_cpt; ++cc, ++it) {
-              const uint32_t s = it % slots, ph = (it / slots) & 1u;
-              if (!mbar_wait<PAIR>(bar_full + 8 * s, ph, abort_flag)) {
-                ok = false;
-                break;
-              }
-              tc_fence_after();
-              const uint32_t a_box = ring + s * (uint32_t)p.tall_stride;
-#pragma unroll
-              for (int tr = 0; tr < 3; ++tr) {
-                const uint32_t a_src = a_box + tr * view_bytes;
-                const uint32_t b_src = b_res ? bres_base + (uint32_t)((tr * 3 + ts) * p.conv_cpt + cc) * b_box_bytes
-                                             : a_box + TC_TALL_ROWS * CH + tr * b_box_bytes;
-#pragma unroll
-                for (int k = 0; k < G::MMAS; ++k) {
-                  tc_mma_i8<NCTA>(d_tmem, make_smem_desc(a_src + k * 32, 16, 8 * CH, G::SWZ),
-                                  make_smem_desc(b_src + k * 32, 16, 8 * CH, G::SWZ), idesc, first ? 0u : 1u);
-                  first = 0u;
-                }
-              }
-              tc_commit<NCTA>(bar_empty + 8 * s);
+          // descriptor low words: start addresses in 16-byte units.  One image row of the box is the step between
+          // vertical taps; a weight box follows the previous tap's box of the same (ts, cc) after 3 * cpt boxes (resident)
+          // or directly (streamed, inside the stage)
+          const uint32_t hi = smem_desc_hi(8 * CH, G::SWZ);
+          const uint32_t a_lo0 = smem_desc_lo(ring, 16), a_step = (uint32_t)p.tall_stride >> 4, a_tap = ((uint32_t)p.conv_W * CH) >> 4;
+          const uint32_t b_box = b_box_bytes >> 4;
+          const uint32_t b_tap = b_res ? 3u * (uint32_t)p.conv_cpt * b_box : b_box;
+          const uint32_t b_lo0 = b_res ? smem_desc_lo(bres_base, 16) : a_lo0 + ((TC_TALL_ROWS * CH) >> 4);
+          uint32_t acc = 0u, chunk = 0u;   // chunk = ts * cpt + cc
+          for (int n = 3 * p.conv_cpt; n > 0; --n, ++chunk) {
+            const uint32_t s = tall_s, ph = tall_ph;   // ring position, kept by counting (no division in this loop)
+            if (++tall_s == slots) tall_s = 0u, tall_ph ^= 1u;
+            if (!mbar_wait<PAIR>(bar_full + 8 * s, ph, abort_flag)) {
+              ok = false;
+              break;
             }
+            tc_fence_after();
+            const uint32_t a_lo = a_lo0 + s * a_step;
+            const uint32_t b_lo = b_lo0 + (b_res ? chunk * b_box : s * a_step);
+#pragma unroll
+            for (int tr = 0; tr < 3; ++tr) {
+#pragma unroll
+              for (int k = 0; k < G::MMAS; ++k) {
+                tc_mma_i8<NCTA>(d_tmem, smem_desc_join(a_lo + tr * a_tap + 2 * k, hi), smem_desc_join(b_lo + tr * b_tap + 2 * k, hi), idesc, acc);
+                acc = 1u;
+              }
+            }
+            tc_commit<NCTA>(bar_empty + 8 * s);
+          }
           if (ok) tc_commit<NCTA>(bar_tfull + 8 * as);
           continue;
         }
