@@ -316,6 +316,25 @@ ff_status ff_poll_status(ff_ctx* ctx, void* cuda_stream);
  * Nothing else is touched. */
 ff_status ff_selftest_bounded_wait(ff_ctx* ctx, uint64_t limit_ns, void* cuda_stream);
 
+/* How the library would cut a layer's weight gradient so that no INT32 sum can wrap (Sec. IV-B: INT8 operands,
+ * INT32 accumulation; a sum over more than 133144 = floor((2^31 - 1) / 127^2) products could).  Host arithmetic
+ * only - no context, no device: the planning functions the launches themselves call, for tests and for inspection.
+ * route: FF_PLAN_TENSOR_SLABS (tcgen05 split contraction of 3x3 / pointwise convolutions), FF_PLAN_FIRST_LAYER
+ * (3x3 layers with at most four input channels), FF_PLAN_DP4A_SLABS (the fallback kernels; workspace_bytes limits
+ * its slabs).  On FF_OK: `splits` work items along the contraction, `parts` INT32 arrays left for the 64-bit reduce +
+ * update kernel, `longest_register_sum` / `longest_part_sum` the most products any accumulator / any array element
+ * sums (contraction elements of one set).  FF_ERR_ARG: the route does not take this layer; FF_ERR_WORKSPACE: the
+ * workspace cannot hold as many slabs as safety needs. */
+enum { FF_PLAN_TENSOR_SLABS = 0, FF_PLAN_FIRST_LAYER = 1, FF_PLAN_DP4A_SLABS = 2 };
+typedef struct ff_wgrad_plan {
+  int32_t splits;
+  int32_t parts;
+  int64_t longest_register_sum;
+  int64_t longest_part_sum;
+} ff_wgrad_plan;
+ff_status ff_plan_wgrad(const ff_layer_desc* layer, int32_t B, int32_t sm_count, int32_t route, uint64_t workspace_bytes,
+                        ff_wgrad_plan* out);
+
 /* Text of the last error returned for this context (host string, valid until the next call). */
 const char* ff_last_error(const ff_ctx* ctx);
 

@@ -24,7 +24,9 @@ EXPORTS = ["ff_create", "ff_destroy", "ff_workspace_bytes", "ff_set_workspace", 
            "ff_embed_labels",
            "ff_layer_forward", "ff_layer_loss_grad", "ff_layer_update", "ff_train_step", "ff_train_step_from",
            "ff_poll_status", "ff_last_error", "ff_launch_count", "ff_int8_gemm",
-           "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict", "ff_selftest_bounded_wait"]
+           "ff_profile_start", "ff_profile_stop", "ff_loss_coef_static", "ff_predict", "ff_selftest_bounded_wait",
+           "ff_plan_wgrad"]
+FF_PLAN_TENSOR_SLABS, FF_PLAN_FIRST_LAYER, FF_PLAN_DP4A_SLABS = 0, 1, 2
 FF_STATIC_LOSS_MAX_SAMPLES = 65536
 FF_K_NAMES = ["absmax", "quantize", "fwd_gemm", "finalize", "normalize", "loss", "dh_quantize",
               "upd_gemm", "raw_gemm", "classify", "dw_fwd", "dw_upd"]
@@ -54,6 +56,11 @@ FF_DP_MAX, FF_DP_SUM = 0, 1
 class ff_dp_reduce(C.Structure):
     _fields_ = [("dev_ptr", C.c_void_p), ("count", C.c_uint64), ("dtype", C.c_int32), ("op", C.c_int32),
                 ("needed_by_phase", C.c_int32), ("reserved", C.c_int32)]
+
+
+class ff_wgrad_plan(C.Structure):
+    _fields_ = [("splits", C.c_int32), ("parts", C.c_int32), ("longest_register_sum", C.c_int64),
+                ("longest_part_sum", C.c_int64)]
 
 
 class FFError(RuntimeError):
@@ -107,6 +114,7 @@ def load(build_if_missing: bool = True):
     lib.ff_int8_gemm.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ff_profile_start.argtypes = [vp]
     lib.ff_selftest_bounded_wait.argtypes = [vp, u64, vp]
+    lib.ff_plan_wgrad.argtypes = [C.POINTER(ff_layer_desc), i32, i32, i32, u64, C.POINTER(ff_wgrad_plan)]
     lib.ff_predict.argtypes = [vp, C.POINTER(ff_layer_desc), C.POINTER(ff_layer_bufs), i32, i32, i32, i32, vp, vp, u64, vp]
     lib.ff_loss_coef_static.argtypes = [vp, f32, C.POINTER(vp), C.POINTER(f32), i32, f32, i32, vp, vp, vp, vp, vp,
                                         C.c_char_p, C.c_size_t]
@@ -219,6 +227,13 @@ def ff_predict(ctx, descs_arr, bufs_arr, n_layers: int, B: int, n_classes: int, 
 
 def ff_poll_status(ctx, stream: int = 0):
     _check(ctx, load().ff_poll_status(ctx, stream))
+
+
+def ff_plan_wgrad(desc, B: int, sm_count: int, route: int, workspace_bytes: int = 1 << 62):
+    """Host arithmetic only (no device): (status code, ff_wgrad_plan)."""
+    out = ff_wgrad_plan()
+    code = load().ff_plan_wgrad(C.byref(desc), B, sm_count, route, workspace_bytes, C.byref(out))
+    return code, out
 
 
 def ff_selftest_bounded_wait(ctx, limit_ns: int, stream: int = 0):

@@ -17,7 +17,7 @@ constexpr uint32_t ST_RANGE = 8u;      // a weight-gradient sum left the INT32 r
 // Longest contraction whose INT8 x INT8 products cannot leave INT32 whatever the codes: 127*127*n <= 2^31 - 1.
 // Longer weight-gradient contractions (convolutions sum over every position of a set) are cut into parts of at
 // most this length; the parts are added in 64 bits and a sum outside INT32 raises ST_RANGE.
-constexpr long long WG_SAFE_LEN = ((1LL << 31) - 1) / (127LL * 127LL);   // 133143
+constexpr long long WG_SAFE_LEN = ((1LL << 31) - 1) / (127LL * 127LL);   // 133144
 
 constexpr int ROUND_NEAREST = 0;
 constexpr int ROUND_STOCHASTIC = 1;

@@ -524,19 +524,27 @@ ff_status conv_small_forward(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer
 
 // Weight gradient of the same layers: direct dp4a kernel into (slab, set) planes of INT32 sums, then the common
 // reduce + update kernel (which also checks the INT32 range of the whole sums).
-ff_status conv_small_wgrad(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+// How the first-layer weight-gradient kernel cuts a set's positions: chunks of CW_CHUNK, slabs of at most
+// WG_SAFE_LEN positions (at least two when a shard's sums must pass through the range check), blocks per plane.
+ConvSmallWgradGeom conv_small_wgrad_plan(const ff_layer_desc& L, int B, int sm_count, bool two_slabs) {
   ConvSmallWgradGeom g;
   g.H = L.H, g.W = L.Wd, g.Ho = tc_out_h(L), g.Wo = tc_out_w(L), g.stride = tc_conv_stride(L), g.B = B;
   g.rows_per_pass = B * g.Ho * g.Wo;
   g.chunks = (g.rows_per_pass + CW_CHUNK - 1) / CW_CHUNK;
   const int safe_chunks = (int)(WG_SAFE_LEN / CW_CHUNK);
   g.n_slabs = (g.chunks + safe_chunks - 1) / safe_chunks;
-  if (dp_checks_needed(ctx, L) && g.n_slabs < 2) g.n_slabs = 2;   // a shard's sums pass through the range check
+  if (two_slabs && g.n_slabs < 2) g.n_slabs = 2;
   g.chunks_per_slab = (g.chunks + g.n_slabs - 1) / g.n_slabs;
   const int planes = 2 * g.n_slabs;
-  g.blocks_per_plane = ctx->sm_count * 2 / planes;
+  g.blocks_per_plane = sm_count * 2 / planes;
   if (g.blocks_per_plane > g.chunks_per_slab) g.blocks_per_plane = g.chunks_per_slab;
   if (g.blocks_per_plane < 1) g.blocks_per_plane = 1;
+  return g;
+}
+
+ff_status conv_small_wgrad(ff_ctx* ctx, const ff_layer_desc& L, const ff_layer_bufs& b, int B, cudaStream_t st) {
+  const ConvSmallWgradGeom g = conv_small_wgrad_plan(L, B, ctx->sm_count, dp_checks_needed(ctx, L));
+  const int planes = 2 * g.n_slabs;
   const size_t bytes = (size_t)planes * L.N * L.K * sizeof(int32_t);
   if (ctx->workspace_bytes < WS_BYTES + bytes) return fail(ctx, FF_ERR_WORKSPACE, "workspace has no room for the weight-gradient slabs");
   int32_t* slabs = reinterpret_cast<int32_t*>(static_cast<char*>(ctx->workspace) + WS_BYTES);
@@ -1593,6 +1601,50 @@ ff_status ff_profile_stop(ff_ctx* ctx, void* cuda_stream, float* ms_per_kernel, 
   }
   ctx->prof_recs.clear();
   return FF_OK;
+}
+
+ff_status ff_plan_wgrad(const ff_layer_desc* layer, int32_t B, int32_t sm_count, int32_t route, uint64_t workspace_bytes,
+                        ff_wgrad_plan* out) {
+  if (!layer || !out || B < 1 || sm_count < 1) return FF_ERR_ARG;
+  const ff_layer_desc& L = *layer;
+  if (L.kind != FF_CONV3X3 && L.kind != FF_CONV1X1 && L.kind != FF_LINEAR) return FF_ERR_ARG;
+  const long long clen = (long long)B * rows_per_sample(L);   // contraction length: positions (rows) of one set
+  memset(out, 0, sizeof(*out));
+  if (route == FF_PLAN_TENSOR_SLABS) {
+    // the split contraction of the tcgen05 kernels: work items per tile, consecutive splits sharing a slab
+    if (L.kind == FF_LINEAR || !tc_update_supported(L, B)) return FF_ERR_ARG;
+    const long long kblocks = L.kind == FF_CONV3X3 ? clen / 128 : (clen + 127) / 128;
+    int splits = L.kind == FF_CONV3X3 ? tc_conv_update_splits(L, B, sm_count, 0)
+                                      : tc_dense_slab_splits(L.N, L.K, clen, sm_count);
+    if (splits < tc_min_splits(kblocks)) splits = tc_min_splits(kblocks);
+    int per, kb_per_split;
+    out->parts = tc_shared_slab_plan((int)kblocks, splits, &per, &kb_per_split);
+    out->splits = (int)((kblocks + kb_per_split - 1) / kb_per_split);
+    out->longest_register_sum = (long long)kb_per_split * 128;
+    out->longest_part_sum = (long long)per * kb_per_split * 128;
+    return FF_OK;
+  }
+  if (route == FF_PLAN_FIRST_LAYER) {
+    if (!conv_small_ok(L.kind == FF_CONV3X3, L.Cin, L.N)) return FF_ERR_ARG;
+    const ConvSmallWgradGeom g = conv_small_wgrad_plan(L, B, sm_count, false);
+    out->parts = g.n_slabs;
+    out->splits = g.n_slabs * g.blocks_per_plane;
+    // a block strides through its plane's chunks; a plane holds chunks_per_slab chunks
+    out->longest_register_sum = (long long)((g.chunks_per_slab + g.blocks_per_plane - 1) / g.blocks_per_plane) * CW_CHUNK;
+    out->longest_part_sum = (long long)g.chunks_per_slab * CW_CHUNK;
+    return FF_OK;
+  }
+  if (route == FF_PLAN_DP4A_SLABS) {
+    int splits = simt_wgrad_splits(L, B, (size_t)workspace_bytes);
+    if (splits < simt_min_splits(L, B)) return FF_ERR_WORKSPACE;
+    const long long csplit = splits > 1 ? ((clen + splits - 1) / splits + SG_BK - 1) / SG_BK * SG_BK : clen;
+    out->splits = splits > 1 ? simt_split_count((int)clen, splits) : 1;
+    out->parts = out->splits;
+    out->longest_register_sum = csplit;
+    out->longest_part_sum = csplit;
+    return FF_OK;
+  }
+  return FF_ERR_ARG;
 }
 
 ff_status ff_selftest_bounded_wait(ff_ctx* ctx, uint64_t limit_ns, void* cuda_stream) {

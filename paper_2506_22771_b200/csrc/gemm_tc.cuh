@@ -1346,14 +1346,19 @@ inline int tc_conv_update_splits(const ff_layer_desc& L, int B, int sm_count, in
 // Splits that may share one slab: as many consecutive ones as keep the slab's whole contraction within
 // TC_SAFE_KBLOCKS blocks, so that a shared INT32 sum cannot wrap either.  Sets p.splits_per_slab, clears the
 // slabs a shared accumulation adds into, and returns the number of slabs the launch will leave.
+// The arithmetic alone: *per = splits that share a slab, *kb_per_split = contraction blocks of a split; returns the slabs.
+inline int tc_shared_slab_plan(int kblocks, int splits_asked, int* per, int* kb_per_split) {
+  *kb_per_split = cdiv(kblocks, splits_asked < 1 ? 1 : splits_asked);
+  const int splits = cdiv(kblocks, *kb_per_split);
+  *per = TC_SAFE_KBLOCKS / *kb_per_split;
+  if (*per < 1) *per = 1;
+  if (*per > splits) *per = splits;
+  return cdiv(splits, *per);
+}
 inline int tc_plan_shared_slabs(TcParams& p, size_t plane, cudaStream_t st, cudaError_t* err) {
-  const int kb_per_split = cdiv(p.kblocks, p.splits < 1 ? 1 : p.splits);
-  const int splits = cdiv(p.kblocks, kb_per_split);
-  int per = TC_SAFE_KBLOCKS / kb_per_split;
-  if (per < 1) per = 1;
-  if (per > splits) per = splits;
+  int per, kb_per_split;
+  const int slabs = tc_shared_slab_plan(p.kblocks, p.splits, &per, &kb_per_split);
   p.splits_per_slab = per;
-  const int slabs = cdiv(splits, per);
   *err = cudaSuccess;
   if (per > 1) *err = cudaMemsetAsync(p.slabs, 0, (size_t)slabs * 2 * plane * sizeof(int32_t), st);
   return slabs;

@@ -1,7 +1,7 @@
 """INT32 range of the weight-gradient sums (Sec. IV-B: INT8 operands, INT32 accumulation).
 
 A convolution's weight gradient sums over every output position of a set, so its worst case (all codes
-+-127) leaves INT32 once a set has more than 133143 positions.  The library cuts such contractions into
++-127) leaves INT32 once a set has more than 133144 positions.  The library cuts such contractions into
 parts that cannot wrap, adds the parts in 64 bits and reports a sum outside INT32 as FF_ERR_RANGE through
 ff_poll_status (the weight concerned keeps its value); the oracle raises OverflowError for the same
 codes.  The cases here call ff_layer_update on INT8 tensors the test writes itself:
@@ -18,7 +18,7 @@ from paper_2506_22771_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-SAFE = (2 ** 31 - 1) // (127 * 127)     # 133143 positions
+SAFE = (2 ** 31 - 1) // (127 * 127)     # 133144 positions
 HW = 32
 
 # (name, kind, Cin, N): routes - tensor-core implicit GEMM slabs, explicit im2col, dp4a, pointwise dense slabs, depthwise
