@@ -41,7 +41,7 @@ BURST_SECONDS = 2.0         # timed regions shorter than this are compared with 
 # was profiled (hash below) and the workload matches; otherwise the key is null.
 NCU_TRAFFIC = {
     "source": "paper_2506_22771_b200/csrc/gemm_tc.cuh",
-    "sha256": "13b5dce810e6cca29729e2d038e75368b958f1779e51183b6ca7a358dcd21cdb",
+    "sha256": "eaf84a93e525880e0bbfee3cd5fd52077da6694dcbb03a57deb5dee0f41fadba",
     "workload": "roofline", "B": 16384,
     "bytes_per_launch": {"fwd_gemm": 2058.7e6, "upd_gemm": 2868.2e6},
 }
